@@ -1,0 +1,370 @@
+"""CPU fp64 oracle for the per-module ADMM path of structured SparseLLM / STRUPRUNE.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain restatement of what the paper computes.  It
+shares no code with the CUDA library and must never be imported by the product path; only the tests,
+the smoke check and the benchmark's CPU-baseline leg may call it.
+
+Conventions follow the paper: a calibration tensor holds one token per COLUMN, so the module input
+is X = a_{l-1}^pre in R^{d x N}, the up-projection is W1 = W_l in R^{n x d}, the down-projection is
+W2 = W_{l+1} in R^{d x n}, the auxiliary variables are Z = z_l and A = a_l in R^{n x N}, and the
+pre-trained module output is Ypre = z_{l+1}^pre in R^{d x N}.  (The CUDA library stores the same
+tensors token-major, i.e. the transposes.)  Everything is float64 numpy.
+
+Readings of points where the paper is silent or inconsistent (each is a named switch here and is
+implemented identically by the CUDA path):
+  * ridge: the weight recovery W = z a^+ (Appendix A.1, "Reversely recovering the weight matrix") is
+    computed as the Tikhonov-regularised least squares W = R (G + rho_eff I)^-1 with G = a a^T and
+    R = z a^T.  rho_eff = rho * trace(G)/dim(G) when `rho_relative`, else rho.  rho -> 0 with a of
+    full row rank gives z a^+ back.
+  * a-update: the formula of Appendix A.1 ("Updating activation") and Algorithm 3 (GSPO), not the
+    dimensionally inconsistent copy printed in Algorithm 2.
+  * z-update: rule "paper" is the literal select of Algorithms 2 and 3 (test the OLD z, strict < 0);
+    rule "exact" is the true minimiser of the scalar problem in "Updating output".
+  * dual variables: absent from the paper.  dual_mode adds the textbook scaled dual U of the
+    constraint a = phi(z): phi(z) is replaced by phi(z) - U in the a-update, a by a + U in the
+    z-update, and U += a - phi(z) afterwards.  U = 0 reproduces the paper exactly.
+  * Lemma 1 over N calibration tokens: products of scalars become inner products over tokens.
+  * threshold: exactly k units are kept (the k largest scores, lower index wins ties, NaN lowest), so
+    that the mask budget of Eq. (1) holds with equality.
+  * allocation: r_l is the fraction PRUNED in layer l, as Algorithm 1 uses it (clip at 0.95, "mask with
+    sparsity r_l"); kept count = n_l - round_half_up(r_l n_l).
+
+Parity unpinned (no statement in the paper fixes them; only self-consistency tests exist): the
+SwiGLU extension `swiglu_zu_update`, and the default values of alpha, beta, rho, T.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------------------------------
+# Gram and cross products (what W = z a^+ needs; Appendix A.1 "Reversely recovering the weight matrix")
+# --------------------------------------------------------------------------------------------------
+def gram_accumulate(G, R, Xc, Yc=None, rowstats=None):
+    """G += Xc Xc^T, R += Yc Xc^T over one chunk of token columns; rowstats[:,0] += sum|x|, [:,1] += sum x^2."""
+    Xc = np.asarray(Xc, F64)
+    G += Xc @ Xc.T
+    if Yc is not None:
+        R += np.asarray(Yc, F64) @ Xc.T
+    if rowstats is not None:
+        rowstats[:, 0] += np.abs(Xc).sum(axis=1)
+        rowstats[:, 1] += (Xc * Xc).sum(axis=1)
+    return G, R
+
+
+def effective_ridge(G, rho, rho_relative=True):
+    """rho_eff of the Tikhonov term (see header)."""
+    G = np.asarray(G, F64)
+    return float(rho) * float(np.trace(G)) / G.shape[0] if rho_relative else float(rho)
+
+
+def ridge_solve(R, G, rho_eff):
+    """W = R (G + rho_eff I)^-1  — regularised form of W = z a^+ (Appendix A.1)."""
+    G = np.asarray(G, F64)
+    K = G + rho_eff * np.eye(G.shape[0])
+    return np.linalg.solve(K, np.asarray(R, F64).T).T  # K symmetric
+
+
+def restricted_refit(R, G, keep, rho_eff):
+    """Recovery solver on a kept support S (Algorithm 2, "prune by importance + recovery solver"):
+    W[:, S] = R[:, S] (G[S,S] + rho_eff I)^-1, W[:, S^c] = 0."""
+    R = np.asarray(R, F64)
+    G = np.asarray(G, F64)
+    S = np.flatnonzero(np.asarray(keep))
+    W = np.zeros_like(R)
+    if S.size:
+        W[:, S] = ridge_solve(R[:, S], G[np.ix_(S, S)], rho_eff)
+    return W
+
+
+# --------------------------------------------------------------------------------------------------
+# Activation, a-update, z-update (Appendix A.1; Algorithm 3 lines for a_l, z^(1), z^(2), select)
+# --------------------------------------------------------------------------------------------------
+def phi(Z, act="relu"):
+    Z = np.asarray(Z, F64)
+    if act == "relu":
+        return np.maximum(Z, 0.0)
+    raise ValueError(act)
+
+
+def a_update(W2, Ypre, Z, alpha, beta, U=None, act="relu"):
+    """a_l = (alpha W2^T W2 + beta I)^-1 (alpha W2^T Ypre + beta (phi(z_l) - U))."""
+    W2 = np.asarray(W2, F64)
+    n = W2.shape[1]
+    H = phi(Z, act) - (0.0 if U is None else np.asarray(U, F64))
+    lhs = alpha * (W2.T @ W2) + beta * np.eye(n)
+    rhs = alpha * (W2.T @ np.asarray(Ypre, F64)) + beta * H
+    return np.linalg.solve(lhs, rhs)
+
+
+def z_candidates(W1, X, A, alpha, beta, U=None):
+    """z^(1) = W1 X and z^(2) = (beta (a + U) + alpha z^(1)) / (alpha + beta)."""
+    z1 = np.asarray(W1, F64) @ np.asarray(X, F64)
+    Au = np.asarray(A, F64) + (0.0 if U is None else np.asarray(U, F64))
+    z2 = (beta * Au + alpha * z1) / (alpha + beta)
+    return z1, z2
+
+
+def z_select(Zold, z1, z2, A, alpha, beta, rule="paper", U=None):
+    """Elementwise select of the z-update."""
+    Zold = np.asarray(Zold, F64)
+    if rule == "paper":
+        # Algorithms 2/3: entry takes z^(1) if the current z entry is negative, z^(2) otherwise.
+        return np.where(Zold < 0.0, z1, z2)
+    if rule == "exact":
+        # argmin_z beta (a - relu(z))^2 + alpha (z - z1)^2: best point of each half line, then compare.
+        Au = np.asarray(A, F64) + (0.0 if U is None else np.asarray(U, F64))
+        zn = np.minimum(z1, 0.0)
+        zp = np.maximum(z2, 0.0)
+        fn = beta * Au ** 2 + alpha * (zn - z1) ** 2
+        fp = beta * (Au - zp) ** 2 + alpha * (zp - z1) ** 2
+        return np.where(fn < fp, zn, zp)
+    raise ValueError(rule)
+
+
+def dual_update(U, A, Znew, act="relu"):
+    """Scaled dual ascent on a = phi(z) (not in the paper; see header)."""
+    return np.asarray(U, F64) + np.asarray(A, F64) - phi(Znew, act)
+
+
+# --------------------------------------------------------------------------------------------------
+# Structured scores (Lemma 1 / Eq. (3); Section 3.4 Eq. (Wanda); Algorithm 1 Step 3)
+# --------------------------------------------------------------------------------------------------
+def _group_sum(v, group):
+    v = np.asarray(v, F64)
+    assert v.shape[0] % group == 0
+    return v.reshape(v.shape[0] // group, group).sum(axis=1)
+
+
+def lemma1_scores(b, c, dd, t, group=1):
+    """s_j = (<c_j,b_j> + <d_j,t_j>) / (|c_j|^2 + |d_j|^2) with inner products over tokens (columns);
+    t is the target paired with d (printed z^pre in Lemma 1).  With N = 1 this is Eq. (3) literally.
+    A unit made of `group` consecutive rows sums numerators and denominators over its rows.
+    Returns (scores, layer value r_l = mean_j s_j (Lemma 1, derivation form 1/n sum over units), e_j)."""
+    b, c, dd, t = (np.asarray(v, F64).reshape(np.shape(v)[0], -1) for v in (b, c, dd, t))
+    num = _group_sum((c * b).sum(axis=1) + (dd * t).sum(axis=1), group)
+    den = _group_sum((c * c).sum(axis=1) + (dd * dd).sum(axis=1), group)
+    s = num / den
+    return s, float(s.mean()), den
+
+
+def relaxed_mask(s, e, r_layer):
+    """Relaxed mask of Appendix B (Eq. Mlj): M_j = s_j - (1/e_j) (sum_k s_k - r_l n) / sum_k (1/e_k)."""
+    s = np.asarray(s, F64)
+    e = np.asarray(e, F64)
+    n = s.shape[0]
+    lam_half = (s.sum() - r_layer * n) / (1.0 / e).sum()
+    return s - lam_half / e
+
+
+def wanda_scores(W, colsq=None, colabs_mean=None, kind="l2", group=1):
+    """Structured Wanda score of the units feeding the columns of W (W in R^{out x n}).
+    l2 (Eq. Wanda): elementwise |W_ij| * |a_j|_2 reduced with the l2 norm over the unit's block,
+        i.e. sqrt(sum_{j in unit} |W[:,j]|_2^2 * colsq_j), colsq_j = sum_t a_jt^2.
+    l1 (Algorithm 1, Step 3): sum_{j in unit} |W[:,j]|_1 * mean_t |a_jt|.
+    Returns (scores, layer importance I = mean over units)."""
+    W = np.asarray(W, F64)
+    if kind == "l2":
+        per = (W * W).sum(axis=0) * np.asarray(colsq, F64)
+        s = np.sqrt(_group_sum(per, group))
+    elif kind == "l1":
+        per = np.abs(W).sum(axis=0) * np.asarray(colabs_mean, F64)
+        s = _group_sum(per, group)
+    else:
+        raise ValueError(kind)
+    return s, float(s.mean())
+
+
+# --------------------------------------------------------------------------------------------------
+# Softmax allocation (Lemma 2; Algorithm 1 Step 2; Algorithm 2' inverse weighting)
+# --------------------------------------------------------------------------------------------------
+def _round_half_up(x):
+    return int(math.floor(x + 0.5))
+
+
+def allocate_sparsity(I, n_units, rbar, T, mode="softmax", clip_hi=0.95):
+    """Per-layer pruned fractions r_l and kept counts.
+    softmax: w = softmax(-I/T); r = rbar L w; clip to [0, clip_hi]; if nothing hit clip_hi, rescale to mean
+             rbar and clip again (Algorithm 1, Step 2).
+    inverse: r = clip(rbar L (1 - w)/sum(1 - w), 0, clip_hi)      (Algorithm "-distribute", Step 2).
+    uniform: r = rbar."""
+    I = np.asarray(I, F64)
+    L = I.shape[0]
+    if mode == "uniform":
+        r = np.full(L, float(rbar))
+    else:
+        a = -I / T
+        a = a - a.max()
+        w = np.exp(a)
+        w = w / w.sum()
+        if mode == "softmax":
+            raw = rbar * L * w
+            r = np.minimum(np.maximum(raw, 0.0), clip_hi)
+            if not np.any(raw > clip_hi):
+                mu = r.mean()
+                if mu > 0:
+                    r = r * (rbar / mu)
+                r = np.minimum(np.maximum(r, 0.0), clip_hi)
+        elif mode == "inverse":
+            r = rbar * L * (1.0 - w) / (1.0 - w).sum() if L > 1 else np.full(L, float(rbar))
+            r = np.minimum(np.maximum(r, 0.0), clip_hi)
+        else:
+            raise ValueError(mode)
+    n_units = np.asarray(n_units, np.int64)
+    k_keep = np.array([int(n_units[l]) - _round_half_up(r[l] * int(n_units[l])) for l in range(L)], np.int64)
+    return r, k_keep
+
+
+# --------------------------------------------------------------------------------------------------
+# Top-k mask and mask application (Algorithm 1 Step 3; Algorithm 3 threshold + M (.) W)
+# --------------------------------------------------------------------------------------------------
+def topk_mask(scores, k_keep):
+    """Keep exactly the k largest scores (ties: lower index kept; NaN sorts lowest).  Returns (mask u8, tau)."""
+    s = np.asarray(scores, F64).copy()
+    n = s.shape[0]
+    s[np.isnan(s)] = -np.inf
+    order = np.lexsort((np.arange(n), -s))  # primary: descending score, secondary: ascending index
+    mask = np.zeros(n, np.uint8)
+    k = int(k_keep)
+    if k > 0:
+        mask[order[:k]] = 1
+    tau = float(s[order[k - 1]]) if 0 < k <= n else float("nan")
+    return mask, tau
+
+
+def apply_mask(mask, group=1, W_rows=None, W_cols=None):
+    """M (.) W: zero the row groups of W_rows and the column groups of W_cols of pruned units."""
+    m = np.repeat(np.asarray(mask).astype(bool), group)
+    out_r = None if W_rows is None else np.where(m[:, None], np.asarray(W_rows, F64), 0.0)
+    out_c = None if W_cols is None else np.where(m[None, :], np.asarray(W_cols, F64), 0.0)
+    return out_r, out_c
+
+
+# --------------------------------------------------------------------------------------------------
+# The FFN module loop (Algorithm 2, SparseLLM1, merged with Algorithm 3's per-step order)
+# --------------------------------------------------------------------------------------------------
+@dataclasses.dataclass
+class AdmmParams:
+    alpha: float = 1.0
+    beta: float = 1.0
+    rho: float = 0.1
+    rho_relative: bool = True
+    z_rule: str = "paper"
+    dual_mode: bool = False
+    score_kind: str = "wanda_l2"  # "wanda_l2" | "wanda_l1" | "lemma1"
+    k_keep: int = 0
+    reselect_mask: bool = True
+    refit: bool = True
+    act: str = "relu"
+
+
+@dataclasses.dataclass
+class FfnState:
+    Z: np.ndarray
+    U: np.ndarray | None
+    G_X: np.ndarray
+    G_A: np.ndarray
+    R1: np.ndarray
+    R2: np.ndarray
+    absA: np.ndarray  # sum_t |a_jt| of the A that produced G_A
+    W1: np.ndarray | None = None
+    W2: np.ndarray | None = None
+    mask: np.ndarray | None = None
+    it: int = 0
+
+
+def ffn_init(X, W1_0, W2_0, act="relu", dual_mode=False):
+    """Initialisation of SparseLLM1: z = z^pre = W1_0 X, a = a^pre = phi(z^pre), target Ypre = W2_0 a^pre,
+    and the Gram / cross products the first weight recovery needs."""
+    X = np.asarray(X, F64)
+    Zpre = np.asarray(W1_0, F64) @ X
+    Apre = phi(Zpre, act)
+    Ypre = np.asarray(W2_0, F64) @ Apre
+    st = FfnState(
+        Z=Zpre.copy(), U=np.zeros_like(Zpre) if dual_mode else None,
+        G_X=X @ X.T, G_A=Apre @ Apre.T, R1=Zpre @ X.T, R2=Ypre @ Apre.T, absA=np.abs(Apre).sum(axis=1))
+    return st, Ypre
+
+
+def admm_weight_phase(st, W1_0, p, N):
+    """Weight recovery, unit scores, top-k mask and recovery on the kept support for the current accumulators."""
+    rho1 = effective_ridge(st.G_X, p.rho, p.rho_relative)
+    rho2 = effective_ridge(st.G_A, p.rho, p.rho_relative)
+    W1t = ridge_solve(st.R1, st.G_X, rho1)          # W_l     = z_l a_{l-1}^+
+    W2t = ridge_solve(st.R2, st.G_A, rho2)          # W_{l+1} = z_{l+1}^pre a_l^+
+    if p.score_kind == "wanda_l2":
+        s, I = wanda_scores(W2t, colsq=np.diag(st.G_A), kind="l2")
+    elif p.score_kind == "wanda_l1":
+        s, I = wanda_scores(W2t, colabs_mean=st.absA / N, kind="l1")
+    elif p.score_kind == "lemma1":
+        # b = W1~ X, c = d = t = z^pre = W1_0 X, all expressed through G_X = X X^T
+        W10 = np.asarray(W1_0, F64)
+        cb = ((W10 @ st.G_X) * W1t).sum(axis=1)
+        cc = ((W10 @ st.G_X) * W10).sum(axis=1)
+        s = (cb + cc) / (2.0 * cc)
+        I = float(s.mean())
+    else:
+        raise ValueError(p.score_kind)
+    if p.reselect_mask or st.mask is None:
+        st.mask, tau = topk_mask(s, p.k_keep)
+    W1, _ = apply_mask(st.mask, 1, W_rows=W1t)       # row masking is already the restricted solution for W1
+    if p.refit:
+        W2 = restricted_refit(st.R2, st.G_A, st.mask, rho2)
+    else:
+        _, W2 = apply_mask(st.mask, 1, W_cols=W2t)
+    st.W1, st.W2 = W1, W2
+    return s, I
+
+
+def admm_step(st, X, Ypre, W1_0, p):
+    """One outer step: weights from the accumulators, then a-, z- (and dual) updates, then the accumulators
+    of the new auxiliary variables.  Returns (scores, layer importance, report dict, A)."""
+    X = np.asarray(X, F64)
+    Ypre = np.asarray(Ypre, F64)
+    N = X.shape[1]
+    s, I = admm_weight_phase(st, W1_0, p, N)
+    U = st.U if p.dual_mode else None
+    A = a_update(st.W2, Ypre, st.Z, p.alpha, p.beta, U, p.act)
+    z1, z2 = z_candidates(st.W1, X, A, p.alpha, p.beta, U)
+    Znew = z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule, U)
+    if p.dual_mode:
+        st.U = dual_update(st.U, A, Znew, p.act)
+    st.Z = Znew
+    st.G_A = A @ A.T
+    st.R1 = Znew @ X.T
+    st.R2 = Ypre @ A.T
+    st.absA = np.abs(A).sum(axis=1)
+    st.it += 1
+    rep = {
+        "res_act": float(((A - phi(Znew, p.act)) ** 2).sum()),
+        "res_out": float(p.alpha * ((Ypre - st.W2 @ A) ** 2).sum()),
+        "res_in": float(p.alpha * ((Znew - st.W1 @ X) ** 2).sum()),
+    }
+    return s, I, rep, A
+
+
+def ffn_objective(st_W1, st_W2, X, Ypre, Z, A, alpha, beta, act="relu"):
+    """alpha |Ypre - W2 A|^2 + beta |A - phi(Z)|^2 + alpha |Z - W1 X|^2 (Appendix A.1, FFN objective)."""
+    X = np.asarray(X, F64)
+    return (alpha * ((np.asarray(Ypre, F64) - st_W2 @ A) ** 2).sum()
+            + beta * ((A - phi(Z, act)) ** 2).sum()
+            + alpha * ((Z - st_W1 @ X) ** 2).sum())
+
+
+# --------------------------------------------------------------------------------------------------
+# SwiGLU extension (not in the paper; parity unpinned)
+# --------------------------------------------------------------------------------------------------
+def silu(x):
+    x = np.asarray(x, F64)
+    return x / (1.0 + np.exp(-x))
+
+
+def swiglu_zu_update(A, g, z1u, alpha, beta, U=None):
+    """argmin_zu beta (a + u - g zu)^2 + alpha (zu - z1u)^2 for a gated unit a = g * zu, g = SiLU(gate)."""
+    Au = np.asarray(A, F64) + (0.0 if U is None else np.asarray(U, F64))
+    return (beta * g * Au + alpha * z1u) / (beta * g * g + alpha)
