@@ -1,0 +1,244 @@
+/*
+ * sp.h — C ABI of libsp: the per-module ADMM solve of structured SparseLLM / STRUPRUNE on one B200.
+ *
+ * What the library computes (paper: "StructPrune", arXiv 2510.03246):
+ *   for one FFN module with input X = a_{l-1}^pre, up-projection W1 = W_l, down-projection W2 = W_{l+1},
+ *   auxiliary variables Z = z_l, A = a_l and target Ypre = z_{l+1}^pre, minimise
+ *       alpha |Ypre - W2 A|^2 + beta |A - phi(Z)|^2 + alpha |Z - W1 X|^2          (Appendix A.1, FFN objective)
+ *   by alternating weight recovery W = z a^+ (Appendix A.1 "Reversely recovering the weight matrix"), the structured
+ *   mask step (Lemma 1 / Section 3.4 scores, Lemma 2 / Algorithm 1 Step 2 allocation, Algorithm 1 Step 3 /
+ *   Algorithm 3 threshold and M (.) W), the closed-form a-update and the z^(1)/z^(2) select (Algorithms 2 and 3).
+ *
+ * Conventions common to every call
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns every buffer; the
+ *     library allocates no device memory.  Scratch comes from a caller workspace sized by sp_workspace_bytes().
+ *   - All calls are asynchronous on the given CUDA stream (passed as void*, a cudaStream_t) and never synchronise.
+ *   - Matrices are row-major with an explicit leading dimension `ld` (elements between consecutive rows).
+ *     Calibration tensors are TOKEN-MAJOR: [tokens, channels] (the transpose of the paper's channel x token
+ *     notation, i.e. the paper's matrix in column-major order).  Weights are [out, in].
+ *   - Storage types: SP_BF16 or SP_F32 for activations (the "bf16 mode" / "fp32 mode"); accumulators, weights,
+ *     Z and U are fp32; statistics and the allocation are fp64.
+ *       bf16 mode: contractions run on the tensor cores with bf16 operands and fp32 accumulation; linear systems
+ *                  are factorised in fp32.
+ *       fp32 mode: contractions run in fp32 storage with fp64 accumulation; linear systems are factorised in fp64.
+ *   - Return value: SP_OK or an error detected on the host before any launch (argument / shape / alignment /
+ *     workspace errors).  Numerical failures found on the device (non-positive Cholesky pivot, a bounded wait that
+ *     ran out) are written to the caller's `status_dev[4]` = {code, index, aux, 0}; nothing traps or spins forever.
+ *   - Symmetric accumulators (Gram matrices) are stored as full squares; calls that update them keep the LOWER
+ *     triangle (including the diagonal) authoritative.  sp_symmetrize() mirrors it to the upper triangle.
+ */
+#ifndef SP_H_
+#define SP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SP_OK = 0,
+  SP_ERR_INVALID_ARG = 1,
+  SP_ERR_SHAPE = 2,
+  SP_ERR_DTYPE = 3,
+  SP_ERR_ALIGNMENT = 4,
+  SP_ERR_WORKSPACE = 5,
+  SP_ERR_NOT_SPD = 6,
+  SP_ERR_TIMEOUT = 7,
+  SP_ERR_CUDA = 8,
+  SP_ERR_UNSUPPORTED = 9
+} sp_status;
+
+typedef enum { SP_F32 = 0, SP_BF16 = 1, SP_F64 = 2 } sp_dtype;
+typedef enum { SP_ACT_RELU = 0 } sp_act_kind;
+typedef enum { SP_Z_PAPER = 0, SP_Z_EXACT = 1 } sp_z_rule;
+typedef enum { SP_SCORE_WANDA_L2 = 0, SP_SCORE_WANDA_L1 = 1, SP_SCORE_LEMMA1 = 2 } sp_score_kind;
+typedef enum { SP_ALLOC_SOFTMAX = 0, SP_ALLOC_INVERSE = 1, SP_ALLOC_UNIFORM = 2 } sp_alloc_mode;
+typedef enum { SP_WS_GRAM = 0, SP_WS_ADMM_STEP = 1, SP_WS_SCORES = 2, SP_WS_APPLY_MASK = 3, SP_WS_FFN_INIT = 4,
+               SP_WS_LINEAR_REFIT = 5, SP_WS_GEMM = 6, SP_WS_RIDGE_SOLVE = 7 } sp_ws_op;
+
+/* A row-major device matrix view. */
+typedef struct {
+  void* ptr;
+  int32_t dtype; /* sp_dtype */
+  int32_t reserved;
+  int64_t rows, cols, ld;
+} sp_mat;
+
+/* Inputs of one FFN module (inputs of Algorithm 2, SparseLLM1). All read-only. */
+typedef struct {
+  sp_mat X;    /* [N, d]  module input a_{l-1}^pre, token-major, SP_BF16 or SP_F32 (selects the mode)          */
+  sp_mat Ypre; /* [N, d]  pre-trained module output z_{l+1}^pre, same dtype as X (sp_ffn_init writes it)        */
+  sp_mat W1_0; /* [n, d]  pre-trained up-projection, fp32 (used by sp_ffn_init and by the Lemma-1 score)         */
+  sp_mat W2_0; /* [d, n]  pre-trained down-projection, fp32 (used by sp_ffn_init only)                           */
+  int64_t d, n, N;
+  int32_t act; /* sp_act_kind */
+  int32_t reserved;
+} sp_ffn_module;
+
+/* ADMM state of one FFN module; every buffer is caller-owned device memory. */
+typedef struct {
+  float* Z;        /* [N, n] ld = n   auxiliary pre-activation z_l                                               */
+  float* U;        /* [N, n] ld = n   scaled dual of a = phi(z), or NULL when dual_mode == 0                      */
+  float* G_X;      /* [d, d]          X^T X (constant over the iterations)                                       */
+  float* G_A;      /* [n, n]          A^T A of the current auxiliary activation                                  */
+  float* R1;       /* [n, d]          Z^T X                                                                      */
+  float* R2;       /* [d, n]          Ypre^T A                                                                   */
+  double* absA;    /* [n]             sum over tokens of |A| per channel (Wanda l1 score)                         */
+  float* W1;       /* [n, d]          out: masked recovered up-projection                                        */
+  float* W2;       /* [d, n]          out: recovered down-projection on the kept support                          */
+  float* scores;   /* [n]             out: unit scores of this step                                              */
+  uint8_t* mask;   /* [n]             in/out: 1 = kept                                                           */
+  double* importance; /* [1]          out: layer importance I_l = mean_j s_j                                      */
+} sp_ffn_state;
+
+typedef struct {
+  double alpha, beta;      /* penalty weights of the FFN objective (Appendix A.1)                                  */
+  double rho;              /* Tikhonov term of the weight recovery: W = R (G + rho_eff I)^-1                       */
+  int32_t rho_relative;    /* 1: rho_eff = rho * trace(G)/dim(G);  0: rho_eff = rho                                */
+  int32_t z_rule;          /* sp_z_rule: literal select of Algorithms 2/3, or exact scalar minimiser               */
+  int32_t dual_mode;       /* 0: paper's penalty form; 1: scaled dual U on a = phi(z) (an extension of the paper)  */
+  int32_t score_kind;      /* sp_score_kind                                                                       */
+  int64_t k_keep;          /* units kept in this module (from sp_allocate_sparsity)                                */
+  int32_t reselect_mask;   /* 1: recompute the top-k mask from this step's scores; 0: keep st->mask                */
+  int32_t refit;           /* 1: recovery solver on the kept support (Algorithm 2); 0: plain M (.) W               */
+  int64_t token_chunk;     /* tokens per streamed chunk (0 = library default)                                      */
+  int32_t compute_objective; /* 1: also report alpha|Ypre-W2A|^2 and alpha|Z-W1X|^2                               */
+  int32_t reserved;
+} sp_admm_params;
+
+/* Device-side report of one step (all double). */
+typedef struct {
+  double res_act;   /* |A - phi(Z_new)|^2                                                                         */
+  double res_out;   /* alpha |Ypre - W2 A|^2   (NaN unless compute_objective)                                      */
+  double res_in;    /* alpha |Z_new - W1 X|^2  (NaN unless compute_objective)                                      */
+  double z_sq;      /* |Z_new|^2                                                                                  */
+  double a_sq;      /* |A|^2                                                                                      */
+  double rho1_eff, rho2_eff; /* ridge terms actually used                                                         */
+  double kept;      /* number of kept units                                                                       */
+} sp_step_report;
+
+/* Inputs of sp_struct_scores; only the fields of the chosen kind are read. */
+typedef struct {
+  sp_mat W;              /* WANDA kinds: fp32 weight [out, n_units*group] whose COLUMNS belong to the units         */
+  const float* colsq;    /* WANDA_L2: sum_t a_jt^2 per column, element j at colsq[j*colsq_stride] (e.g. diag of G)  */
+  int64_t colsq_stride;
+  const double* colabs;  /* WANDA_L1: sum_t |a_jt| per column                                                       */
+  double inv_tokens;     /* WANDA_L1: 1/N                                                                           */
+  sp_mat b, c, dd, t;    /* LEMMA1: token-major [N, n_units*group] streams (fp32 or bf16), see Lemma 1              */
+} sp_score_inputs;
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_gram_accumulate — Gram and cross-product accumulation over one chunk of calibration tokens.
+ * Paper: these are the two products the weight recovery W = z a^+ = (z a^T)(a a^T)^-1 needs (Appendix A.1,
+ * "Reversely recovering the weight matrix"; Algorithm 3 first line of the step).
+ *   G[C,C] += Xc^T Xc (lower triangle authoritative),  R[Rr,C] += Yc^T Xc (skipped when Yc == NULL),
+ *   rowstats[c,0] += sum_t |Xc[t,c]|, rowstats[c,1] += sum_t Xc[t,c]^2 (skipped when NULL; fp64).
+ * Xc: [T, C], Yc: [T, Rr], same dtype (SP_BF16 or SP_F32).  G, R: fp32, ldg >= C, ldr >= C.
+ * Workspace: sp_workspace_bytes(SP_WS_GRAM, C, Rr, T, 0, dtype).  status_dev may be NULL.
+ * Errors: SP_ERR_INVALID_ARG (null pointers), SP_ERR_SHAPE (row counts differ, ld too small), SP_ERR_DTYPE,
+ *         SP_ERR_WORKSPACE.
+ */
+sp_status sp_gram_accumulate(const sp_mat* Xc, const sp_mat* Yc, float* G, int64_t ldg, float* R, int64_t ldr,
+                             double* rowstats, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_ffn_init — initialisation of Algorithm 2 (SparseLLM1): z = z^pre = X W1_0^T, a = a^pre = phi(z^pre),
+ * Ypre = a^pre W2_0^T (written to m->Ypre), and the accumulators G_X, G_A, R1, R2, absA of that state.
+ * U (if not NULL) is cleared.  Workspace: sp_workspace_bytes(SP_WS_FFN_INIT, d, n, N, token_chunk, dtype).
+ */
+sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_chunk, int32_t* status_dev,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_admm_step — one outer step of Algorithm 2 (SparseLLM1) in the per-step order of Algorithm 3 (GSPO):
+ *   1. W1~ = R1 (G_X + rho1 I)^-1, W2~ = R2 (G_A + rho2 I)^-1        (weight recovery, Appendix A.1)
+ *   2. unit scores (p->score_kind) and layer importance              (Lemma 1 / Section 3.4 / Algorithm 1 Step 3)
+ *   3. top-k mask with k = p->k_keep if p->reselect_mask             (Algorithm 3 threshold; exactly k kept)
+ *   4. W1 = diag(M) W1~;  W2[:,S] = R2[:,S] (G_A[S,S] + rho2 I)^-1   (recovery on the kept support, or M (.) W2~)
+ *   5. per token chunk: A = h + (Ypre - h W2^T)(gamma I + W2 W2^T)^-1 W2 with h = phi(Z) - U, gamma = beta/alpha,
+ *      which equals a_l = (alpha W2^T W2 + beta I)^-1 (alpha W2^T Ypre + beta h) of Appendix A.1;
+ *      z^(1) = X W1^T, z^(2) = (beta (A+U) + alpha z^(1))/(alpha+beta); select; U += A - phi(Z_new);
+ *      G_A, R1, R2, absA are rebuilt from the new A and Z.
+ * In/out: st (Z, U, accumulators, mask); out: st->W1, st->W2, st->scores, st->importance, *rep_dev.
+ * rep_dev and status_dev are device pointers (status_dev: int32[4], must be zeroed by the caller beforehand).
+ * Workspace: sp_workspace_bytes(SP_WS_ADMM_STEP, d, n, N, token_chunk, dtype).
+ * Errors: SP_ERR_INVALID_ARG, SP_ERR_SHAPE (k_keep outside [1, n], N/d/n mismatch), SP_ERR_DTYPE, SP_ERR_WORKSPACE.
+ */
+sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* p, sp_step_report* rep_dev,
+                       int32_t* status_dev, void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_struct_scores — per-unit importance scores and the layer importance I = mean over units.
+ *   SP_SCORE_WANDA_L2 (Section 3.4, Eq. "wanda"): s_u = sqrt( sum_{j in unit u} |W[:,j]|_2^2 * colsq_j )
+ *   SP_SCORE_WANDA_L1 (Algorithm 1, Step 3):       s_u = sum_{j in unit u} |W[:,j]|_1 * colabs_j * inv_tokens
+ *   SP_SCORE_LEMMA1   (Lemma 1, Eq. 3; inner products over tokens):
+ *        s_u = sum_{j in u}(<c_j,b_j> + <d_j,t_j>) / sum_{j in u}(|c_j|^2 + |d_j|^2)
+ * group = rows/columns per unit (1 = channel, d_head = attention head).
+ * scores: fp32 [n_units]; layer_importance: fp64 [1]; relaxed_mask (optional, fp64 [n_units], LEMMA1 only):
+ *   M_u = s_u - (1/e_u)(sum_k s_k - r_layer n_units)/sum_k(1/e_k), e_u the denominator of s_u (Appendix B, Eq. Mlj).
+ * Workspace: sp_workspace_bytes(SP_WS_SCORES, n_units*group, 0, N, 0, dtype).
+ */
+sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* in, int64_t n_units, float* scores,
+                           double* layer_importance, double* relaxed_mask, double r_layer, void* ws, size_t ws_bytes,
+                           void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_allocate_sparsity — softmax-form sparsity allocation across L layers (Lemma 2; Algorithm 1, Step 2).
+ *   SOFTMAX: w = softmax(-I/T); r = rbar L w; clip to [0, clip_hi]; if no entry hit clip_hi: rescale to mean rbar,
+ *            clip again.  INVERSE: r = clip(rbar L (1-w)/sum(1-w)) (Algorithm "-distribute", Step 2).  UNIFORM: rbar.
+ *   r_l is the fraction PRUNED; k_keep_out[l] = n_units[l] - floor(r_l n_units[l] + 0.5).  All fp64 / int64, device.
+ * Errors: SP_ERR_INVALID_ARG (null, T <= 0, rbar outside [0,1]), SP_ERR_SHAPE (L < 1 or L > 65536).
+ */
+sp_status sp_allocate_sparsity(const double* I, const int64_t* n_units, int32_t L, double rbar, double T, int32_t mode,
+                               double clip_hi, double* r_out, int64_t* k_keep_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_apply_mask — top-k selection and M (.) W (Algorithm 1 Step 3; Algorithm 3 threshold and mask lines).
+ * Keeps exactly k_keep units: the k largest scores, equal scores resolved toward the lower index, NaN lowest.
+ * mask_out: u8 [n_units] (1 = kept); tau_out (optional): the k-th largest score; kept_idx_out (optional): int32
+ * [k_keep] ascending indices of kept units.  W_rows (optional, fp32 [n_units*group, cols]): rows of pruned units are
+ * zeroed.  W_cols (optional, fp32 [rows, n_units*group]): columns of pruned units are zeroed.
+ * Errors: SP_ERR_SHAPE (k_keep outside [0, n_units], matrix sizes do not match n_units*group).
+ */
+sp_status sp_apply_mask(const float* scores, int64_t n_units, int64_t k_keep, int32_t group, uint8_t* mask_out,
+                        float* tau_out, int32_t* kept_idx_out, const sp_mat* W_rows, const sp_mat* W_cols, void* ws,
+                        size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * Helpers.
+ * sp_ridge_solve   — W[m,n] = R[m,n] (G[n,n] + rho_eff I)^-1 by Cholesky and two triangular solves (weight
+ *                    recovery of Appendix A.1).  G, R, W fp32; factorisation in fp64 when precise != 0, else fp32.
+ *                    rho_eff as in sp_admm_params.  G is read from its lower triangle and left unchanged.
+ * sp_linear_refit  — recovery on a kept support of column groups: W[:, S] = R[:, S](G[S,S] + rho_eff I)^-1,
+ *                    other columns zero (Algorithm 2, "importance + recovery solver"; used for W2 and for W_O heads).
+ *                    mask: u8 [n_units] with exactly k_keep ones (k_keep is a host value).
+ * sp_gemm          — C[M,N] = alpha * opA(A) opB(B) + beta * C, opX(X) = X or X^T; test and utility entry.
+ *                    use_tensor_cores != 0 requests the tcgen05 path (bf16 operands only; falls back with
+ *                    SP_ERR_UNSUPPORTED when shapes or alignment do not allow it).
+ * sp_symmetrize    — mirror the lower triangle of a square fp32 matrix onto its upper triangle.
+ */
+sp_status sp_ridge_solve(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n, double rho,
+                         int32_t rho_relative, int32_t precise, float* W, int64_t ldw, int32_t* status_dev, void* ws,
+                         size_t ws_bytes, void* stream);
+sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_units,
+                          int32_t group, const uint8_t* mask, int64_t k_keep, double rho_eff, int32_t precise,
+                          float* W, int64_t ldw, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream);
+sp_status sp_gemm(int32_t transA, int32_t transB, int64_t M, int64_t N, int64_t K, double alpha, const sp_mat* A,
+                  const sp_mat* B, double beta, const sp_mat* C, int32_t lower_only, int32_t use_tensor_cores,
+                  int32_t* status_dev, void* stream);
+sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream);
+
+/* Bytes of workspace the named call needs.  Meaning of (d, n, N, token_chunk, dtype) per op:
+ *   SP_WS_GRAM: d = channels C, N = tokens T.   SP_WS_ADMM_STEP / SP_WS_FFN_INIT: module sizes, dtype of X.
+ *   SP_WS_SCORES: d = n_units*group, N = tokens (LEMMA1) or rows of W (WANDA).
+ *   SP_WS_RIDGE_SOLVE / SP_WS_LINEAR_REFIT: d = m (rows of R), n = system size, dtype SP_F64 when precise != 0. */
+size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t token_chunk, int32_t dtype);
+const char* sp_status_string(int32_t status);
+int32_t sp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SP_H_ */

@@ -1,0 +1,347 @@
+"""Thin ctypes binding over libsp.so (argument marshalling and buffer allocation only).
+
+Every function here has the name of the C entry point it forwards to (see include/sp.h); all arithmetic runs in the
+CUDA library.  PyTorch supplies device memory and the current stream.  There is no CPU fallback: if libsp.so is
+missing or a CUDA device is absent the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsp.so")
+
+SP_OK = 0
+SP_F32, SP_BF16, SP_F64 = 0, 1, 2
+SP_ACT_RELU = 0
+SP_Z_PAPER, SP_Z_EXACT = 0, 1
+SP_SCORE_WANDA_L2, SP_SCORE_WANDA_L1, SP_SCORE_LEMMA1 = 0, 1, 2
+SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
+(SP_WS_GRAM, SP_WS_ADMM_STEP, SP_WS_SCORES, SP_WS_APPLY_MASK, SP_WS_FFN_INIT, SP_WS_LINEAR_REFIT, SP_WS_GEMM,
+ SP_WS_RIDGE_SOLVE) = range(8)
+
+EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
+           "sp_apply_mask", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes",
+           "sp_status_string", "sp_version"]
+
+
+class SpError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (sp_status {code})")
+
+
+class SpMat(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("dtype", C.c_int32), ("reserved", C.c_int32), ("rows", C.c_int64),
+                ("cols", C.c_int64), ("ld", C.c_int64)]
+
+
+class SpFfnModule(C.Structure):
+    _fields_ = [("X", SpMat), ("Ypre", SpMat), ("W1_0", SpMat), ("W2_0", SpMat), ("d", C.c_int64), ("n", C.c_int64),
+                ("N", C.c_int64), ("act", C.c_int32), ("reserved", C.c_int32)]
+
+
+class SpFfnState(C.Structure):
+    _fields_ = [("Z", C.c_void_p), ("U", C.c_void_p), ("G_X", C.c_void_p), ("G_A", C.c_void_p), ("R1", C.c_void_p),
+                ("R2", C.c_void_p), ("absA", C.c_void_p), ("W1", C.c_void_p), ("W2", C.c_void_p),
+                ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p)]
+
+
+class SpAdmmParams(C.Structure):
+    _fields_ = [("alpha", C.c_double), ("beta", C.c_double), ("rho", C.c_double), ("rho_relative", C.c_int32),
+                ("z_rule", C.c_int32), ("dual_mode", C.c_int32), ("score_kind", C.c_int32), ("k_keep", C.c_int64),
+                ("reselect_mask", C.c_int32), ("refit", C.c_int32), ("token_chunk", C.c_int64),
+                ("compute_objective", C.c_int32), ("reserved", C.c_int32)]
+
+
+class SpScoreInputs(C.Structure):
+    _fields_ = [("W", SpMat), ("colsq", C.c_void_p), ("colsq_stride", C.c_int64), ("colabs", C.c_void_p),
+                ("inv_tokens", C.c_double), ("b", SpMat), ("c", SpMat), ("dd", SpMat), ("t", SpMat)]
+
+
+REPORT_FIELDS = ["res_act", "res_out", "res_in", "z_sq", "a_sq", "rho1_eff", "rho2_eff", "kept"]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libsp.so (built in-tree by paper_2510_03246_b200/build.py); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2510_03246_b200.build` first")
+        L = C.CDLL(LIB_PATH)
+        L.sp_workspace_bytes.restype = C.c_size_t
+        L.sp_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_int32]
+        L.sp_status_string.restype = C.c_char_p
+        L.sp_status_string.argtypes = [C.c_int32]
+        L.sp_version.restype = C.c_int32
+        vp, i32, i64, dbl, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_double, C.c_size_t
+        pm = C.POINTER(SpMat)
+        L.sp_gram_accumulate.argtypes = [pm, pm, vp, i64, vp, i64, vp, vp, vp, sz, vp]
+        L.sp_ffn_init.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), i64, vp, vp, sz, vp]
+        L.sp_admm_step.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), C.POINTER(SpAdmmParams), vp, vp, vp,
+                                   sz, vp]
+        L.sp_struct_scores.argtypes = [i32, i32, C.POINTER(SpScoreInputs), i64, vp, vp, vp, dbl, vp, sz, vp]
+        L.sp_allocate_sparsity.argtypes = [vp, vp, i32, dbl, dbl, i32, dbl, vp, vp, vp]
+        L.sp_apply_mask.argtypes = [vp, i64, i64, i32, vp, vp, vp, pm, pm, vp, sz, vp]
+        L.sp_ridge_solve.argtypes = [vp, i64, vp, i64, i64, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
+        L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, vp, i64, vp, vp, sz, vp]
+        L.sp_gemm.argtypes = [i32, i32, i64, i64, i64, dbl, pm, pm, dbl, pm, i32, i32, vp, vp]
+        L.sp_symmetrize.argtypes = [vp, i64, i64, vp]
+        for name in EXPORTS:
+            if name not in ("sp_workspace_bytes", "sp_status_string", "sp_version"):
+                getattr(L, name).restype = C.c_int32
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().sp_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str):
+    if code != SP_OK:
+        raise SpError(code, where)
+
+
+def _require_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise RuntimeError("libsp operates on CUDA tensors only (there is no CPU path)")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dt(t: torch.Tensor) -> int:
+    return {torch.float32: SP_F32, torch.bfloat16: SP_BF16, torch.float64: SP_F64}[t.dtype]
+
+
+def mat(t: torch.Tensor | None) -> SpMat:
+    """Row-major matrix view of a 2-D tensor whose last dimension is contiguous."""
+    if t is None:
+        return SpMat(None, 0, 0, 0, 0, 0)
+    assert t.dim() == 2 and (t.stride(1) == 1 or t.shape[1] <= 1), "need a row-major 2-D tensor"
+    return SpMat(t.data_ptr(), _dt(t), 0, t.shape[0], t.shape[1], t.stride(0) if t.shape[0] > 1 else max(t.shape[1], t.stride(0)))
+
+
+def _ptr(t: torch.Tensor | None):
+    return None if t is None else t.data_ptr()
+
+
+def workspace_bytes(op: int, d: int, n: int, N: int, token_chunk: int = 0, dtype: int = SP_F32) -> int:
+    return int(lib().sp_workspace_bytes(op, d, n, N, token_chunk, dtype))
+
+
+def _ws(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def new_status(device="cuda") -> torch.Tensor:
+    return torch.zeros(4, dtype=torch.int32, device=device)
+
+
+# ---------------------------------------------------------------------------------------------- direct calls
+def sp_gemm(A, B, C_, transA=False, transB=False, alpha=1.0, beta=0.0, lower_only=False, use_tensor_cores=False,
+            status=None, M=None, N=None, K=None):
+    """C = alpha * op(A) op(B) + beta * C."""
+    _require_cuda(A, B, C_)
+    M = C_.shape[0] if M is None else M
+    N = C_.shape[1] if N is None else N
+    K = (A.shape[0] if transA else A.shape[1]) if K is None else K
+    a, b, c = mat(A), mat(B), mat(C_)
+    _check(lib().sp_gemm(int(transA), int(transB), M, N, K, alpha, C.byref(a), C.byref(b), beta, C.byref(c),
+                         int(lower_only), int(use_tensor_cores), _ptr(status), _stream()), "sp_gemm")
+
+
+def sp_symmetrize(G):
+    _require_cuda(G)
+    _check(lib().sp_symmetrize(G.data_ptr(), G.shape[0], G.stride(0), _stream()), "sp_symmetrize")
+
+
+def sp_gram_accumulate(Xc, Yc, G, R=None, rowstats=None, status=None, ws=None):
+    _require_cuda(Xc, Yc, G, R, rowstats)
+    x = mat(Xc)
+    y = mat(Yc) if Yc is not None else None
+    if ws is None:
+        ws = _ws(workspace_bytes(SP_WS_GRAM, Xc.shape[1], 0, Xc.shape[0], 0, _dt(Xc)), Xc.device)
+    _check(lib().sp_gram_accumulate(C.byref(x), C.byref(y) if y is not None else None, G.data_ptr(), G.stride(0),
+                                    _ptr(R), R.stride(0) if R is not None else 0, _ptr(rowstats), _ptr(status),
+                                    ws.data_ptr(), ws.numel(), _stream()), "sp_gram_accumulate")
+
+
+def sp_ridge_solve(R, G, rho, rho_relative=True, precise=False, W=None, status=None, ws=None):
+    _require_cuda(R, G, W)
+    m, n = R.shape
+    if W is None:
+        W = torch.empty_like(R)
+    if ws is None:
+        ws = _ws(workspace_bytes(SP_WS_RIDGE_SOLVE, m, n, 0, 0, SP_F64 if precise else SP_F32), R.device)
+    _check(lib().sp_ridge_solve(R.data_ptr(), R.stride(0), G.data_ptr(), G.stride(0), m, n, float(rho),
+                                int(rho_relative), int(precise), W.data_ptr(), W.stride(0), _ptr(status),
+                                ws.data_ptr(), ws.numel(), _stream()), "sp_ridge_solve")
+    return W
+
+
+def sp_linear_refit(R, G, mask, k_keep, rho_eff, group=1, precise=False, W=None, status=None, ws=None):
+    _require_cuda(R, G, mask, W)
+    m, n = R.shape
+    if W is None:
+        W = torch.empty_like(R)
+    if ws is None:
+        ws = _ws(workspace_bytes(SP_WS_LINEAR_REFIT, m, n, 0, 0, SP_F64 if precise else SP_F32), R.device)
+    _check(lib().sp_linear_refit(R.data_ptr(), R.stride(0), G.data_ptr(), G.stride(0), m, n // group, group,
+                                 mask.data_ptr(), int(k_keep), float(rho_eff), int(precise), W.data_ptr(),
+                                 W.stride(0), _ptr(status), ws.data_ptr(), ws.numel(), _stream()), "sp_linear_refit")
+    return W
+
+
+def sp_struct_scores(kind, n_units, group=1, W=None, colsq=None, colsq_stride=1, colabs=None, inv_tokens=0.0,
+                     b=None, c=None, dd=None, t=None, r_layer=0.0, want_relaxed=False, ws=None):
+    """Returns (scores fp32 [n_units], importance fp64 [1], relaxed fp64 [n_units] or None)."""
+    dev = (W if W is not None else b).device
+    _require_cuda(W, colsq, colabs, b, c, dd, t)
+    inp = SpScoreInputs(mat(W), _ptr(colsq), colsq_stride, _ptr(colabs), float(inv_tokens), mat(b), mat(c), mat(dd),
+                        mat(t))
+    scores = torch.empty(n_units, dtype=torch.float32, device=dev)
+    imp = torch.empty(1, dtype=torch.float64, device=dev)
+    relaxed = torch.empty(n_units, dtype=torch.float64, device=dev) if want_relaxed else None
+    rows = W.shape[0] if W is not None else b.shape[0]
+    if ws is None:
+        ws = _ws(workspace_bytes(SP_WS_SCORES, n_units * group, 0, rows, 0, SP_F32), dev)
+    _check(lib().sp_struct_scores(kind, group, C.byref(inp), n_units, scores.data_ptr(), imp.data_ptr(),
+                                  _ptr(relaxed), float(r_layer), ws.data_ptr(), ws.numel(), _stream()),
+           "sp_struct_scores")
+    return scores, imp, relaxed
+
+
+def sp_allocate_sparsity(I, n_units, rbar, T, mode=SP_ALLOC_SOFTMAX, clip_hi=0.95):
+    """I: fp64 [L] device, n_units: int64 [L] device.  Returns (r fp64 [L], k_keep int64 [L])."""
+    _require_cuda(I, n_units)
+    L = I.numel()
+    r = torch.empty(L, dtype=torch.float64, device=I.device)
+    k = torch.empty(L, dtype=torch.int64, device=I.device)
+    _check(lib().sp_allocate_sparsity(I.data_ptr(), n_units.data_ptr(), L, float(rbar), float(T), mode,
+                                      float(clip_hi), r.data_ptr(), k.data_ptr(), _stream()), "sp_allocate_sparsity")
+    return r, k
+
+
+def sp_apply_mask(scores, k_keep, group=1, W_rows=None, W_cols=None, want_index=False):
+    """Returns (mask u8 [n_units], tau fp32 [1], kept_idx int32 [k_keep] or None); W_rows / W_cols are zeroed in place."""
+    _require_cuda(scores, W_rows, W_cols)
+    n = scores.numel()
+    mask = torch.empty(n, dtype=torch.uint8, device=scores.device)
+    tau = torch.empty(1, dtype=torch.float32, device=scores.device)
+    idx = torch.empty(max(int(k_keep), 1), dtype=torch.int32, device=scores.device) if want_index else None
+    wr = mat(W_rows) if W_rows is not None else None
+    wc = mat(W_cols) if W_cols is not None else None
+    _check(lib().sp_apply_mask(scores.data_ptr(), n, int(k_keep), group, mask.data_ptr(), tau.data_ptr(), _ptr(idx),
+                               C.byref(wr) if wr is not None else None, C.byref(wc) if wc is not None else None,
+                               None, 0, _stream()), "sp_apply_mask")
+    return mask, tau, (idx[:int(k_keep)] if idx is not None else None)
+
+
+# ---------------------------------------------------------------------------------------------- module driver
+@dataclass
+class AdmmParams:
+    alpha: float = 1.0
+    beta: float = 1.0
+    rho: float = 0.1
+    rho_relative: bool = True
+    z_rule: int = SP_Z_PAPER
+    dual_mode: bool = False
+    score_kind: int = SP_SCORE_WANDA_L2
+    k_keep: int = 0
+    reselect_mask: bool = True
+    refit: bool = True
+    token_chunk: int = 0
+    compute_objective: bool = False
+
+    def to_c(self) -> SpAdmmParams:
+        return SpAdmmParams(self.alpha, self.beta, self.rho, int(self.rho_relative), self.z_rule, int(self.dual_mode),
+                            self.score_kind, int(self.k_keep), int(self.reselect_mask), int(self.refit),
+                            int(self.token_chunk), int(self.compute_objective), 0)
+
+
+class FfnModule:
+    """Owns the device buffers of one FFN module and forwards to sp_ffn_init / sp_admm_step."""
+
+    def __init__(self, X: torch.Tensor, W1_0: torch.Tensor, W2_0: torch.Tensor, dual_mode: bool = False,
+                 token_chunk: int = 0):
+        _require_cuda(X, W1_0, W2_0)
+        assert X.dtype in (torch.float32, torch.bfloat16)
+        self.X = X.contiguous()
+        self.N, self.d = X.shape
+        self.n = W1_0.shape[0]
+        dev = X.device
+        self.dev = dev
+        self.W1_0 = W1_0.to(torch.float32).contiguous()
+        self.W2_0 = W2_0.to(torch.float32).contiguous()
+        N, d, n = self.N, self.d, self.n
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.Ypre = torch.empty(N, d, dtype=X.dtype, device=dev)
+        self.Z = torch.empty(N, n, **f32)
+        self.U = torch.zeros(N, n, **f32) if dual_mode else None
+        self.G_X = torch.empty(d, d, **f32)
+        self.G_A = torch.empty(n, n, **f32)
+        self.R1 = torch.empty(n, d, **f32)
+        self.R2 = torch.empty(d, n, **f32)
+        self.absA = torch.empty(n, dtype=torch.float64, device=dev)
+        self.W1 = torch.zeros(n, d, **f32)
+        self.W2 = torch.zeros(d, n, **f32)
+        self.scores = torch.zeros(n, **f32)
+        self.mask = torch.ones(n, dtype=torch.uint8, device=dev)
+        self.importance = torch.zeros(1, dtype=torch.float64, device=dev)
+        self.report = torch.zeros(len(REPORT_FIELDS), dtype=torch.float64, device=dev)
+        self.status = new_status(dev)
+        self.token_chunk = token_chunk
+        self._ws = None
+        self.iteration = 0
+
+    def _module(self) -> SpFfnModule:
+        return SpFfnModule(mat(self.X), mat(self.Ypre), mat(self.W1_0), mat(self.W2_0), self.d, self.n, self.N,
+                           SP_ACT_RELU, 0)
+
+    def _state(self) -> SpFfnState:
+        return SpFfnState(self.Z.data_ptr(), _ptr(self.U), self.G_X.data_ptr(), self.G_A.data_ptr(),
+                          self.R1.data_ptr(), self.R2.data_ptr(), self.absA.data_ptr(), self.W1.data_ptr(),
+                          self.W2.data_ptr(), self.scores.data_ptr(), self.mask.data_ptr(),
+                          self.importance.data_ptr())
+
+    def _workspace(self, chunk: int) -> torch.Tensor:
+        need = max(workspace_bytes(SP_WS_ADMM_STEP, self.d, self.n, self.N, chunk, _dt(self.X)),
+                   workspace_bytes(SP_WS_FFN_INIT, self.d, self.n, self.N, chunk, _dt(self.X)))
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = _ws(need, self.dev)
+        return self._ws
+
+    def sp_ffn_init(self):
+        ws = self._workspace(self.token_chunk)
+        m, st = self._module(), self._state()
+        _check(lib().sp_ffn_init(C.byref(m), C.byref(st), self.token_chunk, self.status.data_ptr(), ws.data_ptr(),
+                                 ws.numel(), _stream()), "sp_ffn_init")
+        self.iteration = 0
+
+    def sp_admm_step(self, p: AdmmParams):
+        chunk = p.token_chunk or self.token_chunk
+        ws = self._workspace(chunk)
+        m, st = self._module(), self._state()
+        cp = p.to_c()
+        cp.token_chunk = chunk
+        _check(lib().sp_admm_step(C.byref(m), C.byref(st), C.byref(cp), self.report.data_ptr(),
+                                  self.status.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "sp_admm_step")
+        self.iteration += 1
+
+    def read_report(self) -> dict:
+        return dict(zip(REPORT_FIELDS, self.report.cpu().tolist()))
+
+    def check_status(self):
+        s = self.status.cpu().tolist()
+        if s[0] != 0:
+            raise SpError(s[0], f"device status (index {s[1]}, aux {s[2]})")

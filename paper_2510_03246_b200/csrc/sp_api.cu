@@ -1,0 +1,616 @@
+// C-ABI entry points of libsp and the host-side orchestration of the per-module ADMM step.
+#include <math.h>
+#include <string.h>
+
+#include "sp_common.cuh"
+
+using namespace sp;
+
+#define CU(x)                                  \
+  do {                                         \
+    if ((x) != cudaSuccess) return SP_ERR_CUDA; \
+  } while (0)
+#define SPCHK(x)               \
+  do {                         \
+    sp_status _s = (x);        \
+    if (_s != SP_OK) return _s; \
+  } while (0)
+
+namespace {
+
+constexpr int64_t kDefaultChunk = 16384;
+
+struct MatRef {
+  const void* ptr;
+  int32_t dtype;
+  int64_t ld;
+};
+
+// C[M,N] = alpha * sum_k A(i,k) B(k,j) + beta * Cin.
+//   a_kmajor: A stored [M,K] (ld) else [K,M];  b_kmajor: B stored [N,K] (ld) else [K,N].
+// bf16 operands go to the tensor-core kernel when its alignment rules hold; everything else (and the fp32 mode,
+// which accumulates in fp64) runs on the CUDA-core kernel.
+sp_status contract(int64_t M, int64_t N, int64_t K, double alpha, MatRef A, bool a_kmajor, MatRef B, bool b_kmajor,
+                   double beta, MatRef Cin, MatRef C, bool lower_only, bool acc64, bool allow_tc, int32_t* status,
+                   cudaStream_t stream) {
+  if (M <= 0 || N <= 0) return SP_OK;
+  Operand cin{Cin.ptr, Cin.dtype, Cin.ld, 1};
+  OutOperand out{const_cast<void*>(C.ptr), C.dtype, C.ld};
+  if (allow_tc && A.dtype == SP_BF16 && B.dtype == SP_BF16 && K > 0 && C.dtype != SP_F64 &&
+      (beta == 0.0 || Cin.dtype != SP_F64)) {
+    TcOperand ta{A.ptr, A.ld, a_kmajor}, tb{B.ptr, B.ld, b_kmajor};
+    if (gemm_tc_supported(M, N, K, ta, tb)) return gemm_tc(M, N, K, (float)alpha, ta, tb, (float)beta, cin, out,
+                                                           lower_only, status, stream);
+  }
+  Operand a{A.ptr, A.dtype, a_kmajor ? A.ld : 1, a_kmajor ? 1 : A.ld};
+  Operand b{B.ptr, B.dtype, b_kmajor ? 1 : B.ld, b_kmajor ? B.ld : 1};
+  CU(gemm_simt(M, N, K, alpha, a, b, beta, cin, out, lower_only, acc64, stream));
+  return SP_OK;
+}
+
+struct Carver {
+  uint8_t* base;
+  size_t off = 0;
+  explicit Carver(void* p) : base(reinterpret_cast<uint8_t*>(p)) {}
+  template <typename T>
+  T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = reinterpret_cast<T*>(base + off);
+    off += count * sizeof(T);
+    return p;
+  }
+  void* take_bytes(size_t bytes) {
+    off = align_up(off, 256);
+    void* p = base + off;
+    off += bytes;
+    return p;
+  }
+};
+
+size_t dinv_elems(int64_t n) { return (size_t)ceil_div(n, (int64_t)kCholNB) * kCholNB * kCholNB; }
+
+// Buffers of the regularised solve for systems up to nmax with up to mmax right-hand sides.
+struct SolveBufs {
+  void* Gs;
+  void* dinv;
+  void* Rs;
+  int32_t* idx;
+  double* rho;  // [4] device scalars
+};
+
+SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
+  SolveBufs b;
+  b.rho = c.take<double>(4);
+  b.idx = c.take<int32_t>((size_t)nmax);
+  b.Gs = c.take_bytes((size_t)nmax * nmax * tsize);
+  b.dinv = c.take_bytes(dinv_elems(nmax) * tsize);
+  b.Rs = c.take_bytes((size_t)nmax * mmax * tsize);
+  return b;
+}
+
+// W[m, n_full] = R[:, idx] (G[idx, idx] + rho I)^-1 scattered back to the idx columns (idx == nullptr: identity).
+template <typename T>
+sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_full,
+                     const int32_t* idx, int64_t k, const double* rho_dev, float* W, int64_t ldw, SolveBufs& b,
+                     int32_t* status, cudaStream_t stream) {
+  const int64_t nn = idx ? k : n_full;
+  T* Gs = reinterpret_cast<T*>(b.Gs);
+  T* dinv = reinterpret_cast<T*>(b.dinv);
+  T* Rs = reinterpret_cast<T*>(b.Rs);
+  if (idx) CU(load_spd_gather<T>(G, ldg, idx, nn, rho_dev, Gs, nn, stream));
+  else CU(load_spd<T>(G, ldg, nn, rho_dev, Gs, nn, stream));
+  CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
+  CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
+  CU(potrs_right<T>(Rs, m, nn, nn, Gs, nn, dinv, stream));
+  CU(scatter_cols<T>(Rs, nn, idx, m, nn, n_full, W, ldw, stream));
+  return SP_OK;
+}
+
+__global__ void expand_group_index_kernel(const int32_t* unit_idx, int64_t k_units, int group, int32_t* col_idx) {
+  const int64_t total = k_units * group;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x)
+    col_idx[e] = unit_idx[e / group] * group + (int32_t)(e % group);
+}
+
+bool valid_act_dtype(int32_t dt) { return dt == SP_F32 || dt == SP_BF16; }
+
+// ------------------------------------------------------------------------------------------------ workspace plans
+struct AdmmPlan {
+  int64_t d, n, N, chunk;
+  int32_t cdt;
+  bool bf16;
+  size_t tsize;
+  // device buffers
+  SolveBufs sb;
+  float *W1t, *W2t, *Qt, *T0, *Cf;
+  void *W1b, *W2b, *Qtb;       // storage-dtype copies (bf16 mode only)
+  void *H, *E, *Ac, *Zb;
+  float *D, *z1;
+  double *partial, *absA_part, *score_scratch;
+  int row_blocks, nblocks;
+  size_t bytes;
+};
+
+AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int32_t cdt) {
+  AdmmPlan p;
+  p.d = d; p.n = n; p.N = N;
+  p.chunk = chunk > 0 ? chunk : kDefaultChunk;
+  if (p.chunk > N) p.chunk = N;
+  if (p.chunk < 1) p.chunk = 1;
+  p.cdt = cdt;
+  p.bf16 = cdt == SP_BF16;
+  p.tsize = p.bf16 ? 4 : 8;
+  const size_t csz = p.bf16 ? 2 : 4;
+  Carver c(ws);
+  const int64_t nmax = n > d ? n : d;
+  p.sb = carve_solve(c, nmax, nmax == n ? d : n, p.tsize);
+  p.W1t = c.take<float>((size_t)n * d);
+  p.W2t = c.take<float>((size_t)n * d);
+  p.Qt = c.take<float>((size_t)n * d);
+  p.T0 = c.take<float>((size_t)n * d);
+  p.Cf = c.take<float>((size_t)d * d);
+  p.W1b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.W2b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.Qtb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.H = c.take_bytes((size_t)p.chunk * n * csz);
+  p.E = c.take_bytes((size_t)p.chunk * d * csz);
+  p.Ac = c.take_bytes((size_t)p.chunk * n * csz);
+  p.Zb = p.bf16 ? c.take_bytes((size_t)p.chunk * n * csz) : nullptr;
+  p.D = c.take<float>((size_t)p.chunk * n);
+  p.z1 = c.take<float>((size_t)p.chunk * n);
+  p.nblocks = fused_update_grid(p.chunk, n, &p.row_blocks);
+  p.partial = c.take<double>((size_t)p.nblocks * 3);
+  p.absA_part = c.take<double>((size_t)p.row_blocks * n);
+  p.score_scratch = c.take<double>((size_t)score_row_blocks(d, n) * n * 2 + 16);
+  p.bytes = align_up(c.off, 256);
+  return p;
+}
+
+struct InitPlan {
+  int64_t chunk;
+  bool bf16;
+  void *W10b, *W20b, *Ac, *Zb;
+  double* absA_part;
+  int row_blocks;
+  size_t bytes;
+};
+
+InitPlan plan_init(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int32_t cdt) {
+  InitPlan p;
+  p.chunk = chunk > 0 ? chunk : kDefaultChunk;
+  if (p.chunk > N) p.chunk = N;
+  if (p.chunk < 1) p.chunk = 1;
+  p.bf16 = cdt == SP_BF16;
+  const size_t csz = p.bf16 ? 2 : 4;
+  Carver c(ws);
+  p.W10b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.W20b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.Ac = c.take_bytes((size_t)p.chunk * n * csz);
+  p.Zb = p.bf16 ? c.take_bytes((size_t)p.chunk * n * csz) : nullptr;
+  fused_update_grid(p.chunk, n, &p.row_blocks);
+  p.absA_part = c.take<double>((size_t)p.row_blocks * n);
+  p.bytes = align_up(c.off, 256);
+  return p;
+}
+
+size_t ridge_ws_bytes(int64_t m, int64_t n, bool precise) {
+  Carver c(nullptr);
+  carve_solve(c, n, m, precise ? 8 : 4);
+  return align_up(c.off, 256);
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t sp_version(void) { return 100; }
+
+const char* sp_status_string(int32_t s) {
+  switch (s) {
+    case SP_OK: return "ok";
+    case SP_ERR_INVALID_ARG: return "invalid argument";
+    case SP_ERR_SHAPE: return "shape mismatch";
+    case SP_ERR_DTYPE: return "unsupported dtype";
+    case SP_ERR_ALIGNMENT: return "misaligned pointer or leading dimension";
+    case SP_ERR_WORKSPACE: return "workspace too small";
+    case SP_ERR_NOT_SPD: return "matrix not positive definite";
+    case SP_ERR_TIMEOUT: return "bounded device wait ran out";
+    case SP_ERR_CUDA: return "CUDA runtime error";
+    case SP_ERR_UNSUPPORTED: return "unsupported configuration";
+    default: return "unknown status";
+  }
+}
+
+size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t token_chunk, int32_t dtype) {
+  switch (op) {
+    case SP_WS_GRAM: {
+      // d = channels C, N = tokens T
+      const int rb = column_stats_row_blocks(N > 0 ? N : 1, d > 0 ? d : 1);
+      return align_up((size_t)rb * (size_t)(d > 0 ? d : 1) * 2 * sizeof(double), 256) + 256;
+    }
+    case SP_WS_ADMM_STEP: return plan_admm(nullptr, d, n, N, token_chunk, dtype).bytes + 256;
+    case SP_WS_FFN_INIT: return plan_init(nullptr, d, n, N, token_chunk, dtype).bytes + 256;
+    case SP_WS_SCORES: {
+      // d = number of columns (n_units * group), N = tokens (LEMMA1) or weight rows (WANDA)
+      const int64_t cols = d > 0 ? d : 1;
+      const int rb = score_row_blocks(N > 0 ? N : 1, cols);
+      return align_up(((size_t)rb * cols * 2 + (size_t)cols * 2 + 16) * sizeof(double), 256) + 256;
+    }
+    case SP_WS_APPLY_MASK: return 256;
+    case SP_WS_LINEAR_REFIT: return ridge_ws_bytes(d, n, dtype == SP_F64) + align_up((size_t)(n > 0 ? n : 1) * 4, 256) + 512;
+    case SP_WS_RIDGE_SOLVE: return ridge_ws_bytes(d, n, dtype == SP_F64) + 256;
+    case SP_WS_GEMM: return 256;
+    default: return 0;
+  }
+}
+
+sp_status sp_gemm(int32_t transA, int32_t transB, int64_t M, int64_t N, int64_t K, double alpha, const sp_mat* A,
+                  const sp_mat* B, double beta, const sp_mat* C, int32_t lower_only, int32_t use_tensor_cores,
+                  int32_t* status_dev, void* stream) {
+  if (!A || !B || !C || !A->ptr || !B->ptr || !C->ptr) return SP_ERR_INVALID_ARG;
+  if (M < 0 || N < 0 || K < 0) return SP_ERR_SHAPE;
+  // op(A) is M x K: stored [M,K] when !transA (K-major), [K,M] when transA.
+  // op(B) is K x N: stored [K,N] when !transB (N contiguous), [N,K] when transB (K-major).
+  const bool a_kmajor = !transA, b_kmajor = transB != 0;
+  if (A->ld < (a_kmajor ? K : M) || B->ld < (b_kmajor ? K : N) || C->ld < N) return SP_ERR_SHAPE;
+  MatRef a{A->ptr, A->dtype, A->ld}, b{B->ptr, B->dtype, B->ld}, c{C->ptr, C->dtype, C->ld};
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (use_tensor_cores) {
+    if (A->dtype != SP_BF16 || B->dtype != SP_BF16 || C->dtype == SP_F64 || K <= 0) return SP_ERR_UNSUPPORTED;
+    TcOperand ta{A->ptr, A->ld, a_kmajor}, tb{B->ptr, B->ld, b_kmajor};
+    if (!gemm_tc_supported(M, N, K, ta, tb)) return SP_ERR_UNSUPPORTED;
+    if (M == 0 || N == 0) return SP_OK;
+    return gemm_tc(M, N, K, (float)alpha, ta, tb, (float)beta, Operand{c.ptr, c.dtype, c.ld, 1},
+                   OutOperand{const_cast<void*>(c.ptr), c.dtype, c.ld}, lower_only != 0, status_dev, s);
+  }
+  const bool acc64 = !(A->dtype == SP_BF16 && B->dtype == SP_BF16);
+  return contract(M, N, K, alpha, a, a_kmajor, b, b_kmajor, beta, c, c, lower_only != 0, acc64, false, status_dev, s);
+}
+
+sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream) {
+  if (!G) return SP_ERR_INVALID_ARG;
+  if (n < 0 || ldg < n) return SP_ERR_SHAPE;
+  CU(symmetrize_lower(G, n, ldg, reinterpret_cast<cudaStream_t>(stream)));
+  return SP_OK;
+}
+
+sp_status sp_gram_accumulate(const sp_mat* Xc, const sp_mat* Yc, float* G, int64_t ldg, float* R, int64_t ldr,
+                             double* rowstats, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+  if (!Xc || !Xc->ptr || !G) return SP_ERR_INVALID_ARG;
+  if (!valid_act_dtype(Xc->dtype)) return SP_ERR_DTYPE;
+  const int64_t T = Xc->rows, C = Xc->cols;
+  if (T < 0 || C < 0 || Xc->ld < C || ldg < C) return SP_ERR_SHAPE;
+  if (Yc) {
+    if (!Yc->ptr || !R) return SP_ERR_INVALID_ARG;
+    if (Yc->dtype != Xc->dtype) return SP_ERR_DTYPE;
+    if (Yc->rows != T || Yc->ld < Yc->cols || ldr < C) return SP_ERR_SHAPE;
+  }
+  if (rowstats && (!ws || ws_bytes < sp_workspace_bytes(SP_WS_GRAM, C, 0, T, 0, Xc->dtype))) return SP_ERR_WORKSPACE;
+  if (T == 0 || C == 0) return SP_OK;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const bool bf16 = Xc->dtype == SP_BF16;
+  MatRef x{Xc->ptr, Xc->dtype, Xc->ld};
+  MatRef g{G, SP_F32, ldg};
+  SPCHK(contract(C, C, T, 1.0, x, false, x, false, 1.0, g, g, true, !bf16, bf16, status_dev, s));
+  if (Yc && Yc->cols > 0) {
+    MatRef y{Yc->ptr, Yc->dtype, Yc->ld};
+    MatRef r{R, SP_F32, ldr};
+    SPCHK(contract(Yc->cols, C, T, 1.0, y, false, x, false, 1.0, r, r, false, !bf16, bf16, status_dev, s));
+  }
+  if (rowstats) CU(column_stats(Xc->ptr, Xc->dtype, Xc->ld, T, C, rowstats, reinterpret_cast<double*>(ws), s));
+  return SP_OK;
+}
+
+sp_status sp_ridge_solve(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n, double rho,
+                         int32_t rho_relative, int32_t precise, float* W, int64_t ldw, int32_t* status_dev, void* ws,
+                         size_t ws_bytes, void* stream) {
+  if (!R || !G || !W) return SP_ERR_INVALID_ARG;
+  if (m < 0 || n < 0 || ldr < n || ldg < n || ldw < n) return SP_ERR_SHAPE;
+  if (m == 0 || n == 0) return SP_OK;
+  if (!ws || ws_bytes < ridge_ws_bytes(m, n, precise != 0)) return SP_ERR_WORKSPACE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  Carver c(ws);
+  SolveBufs b = carve_solve(c, n, m, precise ? 8 : 4);
+  CU(effective_ridge(G, ldg, n, rho, rho_relative, b.rho, s));
+  if (precise) return ridge_core<double>(R, ldr, G, ldg, m, n, nullptr, n, b.rho, W, ldw, b, status_dev, s);
+  return ridge_core<float>(R, ldr, G, ldg, m, n, nullptr, n, b.rho, W, ldw, b, status_dev, s);
+}
+
+sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_units,
+                          int32_t group, const uint8_t* mask, int64_t k_keep, double rho_eff, int32_t precise,
+                          float* W, int64_t ldw, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+  if (!R || !G || !W || !mask) return SP_ERR_INVALID_ARG;
+  if (group < 1 || n_units < 0 || m < 0 || k_keep < 0 || k_keep > n_units) return SP_ERR_SHAPE;
+  const int64_t n = n_units * group;
+  if (ldr < n || ldg < n || ldw < n) return SP_ERR_SHAPE;
+  if (m == 0 || n == 0) return SP_OK;
+  // workspace: solve buffers for the full size + the unit index list
+  const size_t need = ridge_ws_bytes(m, n, precise != 0) + align_up((size_t)n_units * 4, 256);
+  if (!ws || ws_bytes < need) return SP_ERR_WORKSPACE;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  Carver c(ws);
+  SolveBufs b = carve_solve(c, n, m, precise ? 8 : 4);
+  int32_t* unit_idx = c.take<int32_t>((size_t)n_units);
+  CU(effective_ridge(nullptr, 0, 1, rho_eff, 0, b.rho, s));
+  CU(mask_to_index(mask, n_units, unit_idx, s));
+  const int64_t k = k_keep * group;
+  if (k > 0) {
+    expand_group_index_kernel<<<(unsigned)ceil_div(k, 256), 256, 0, s>>>(unit_idx, k_keep, group, b.idx);
+    CU(cudaGetLastError());
+  }
+  if (precise) return ridge_core<double>(R, ldr, G, ldg, m, n, b.idx, k, b.rho, W, ldw, b, status_dev, s);
+  return ridge_core<float>(R, ldr, G, ldg, m, n, b.idx, k, b.rho, W, ldw, b, status_dev, s);
+}
+
+sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* in, int64_t n_units, float* scores,
+                           double* layer_importance, double* relaxed_mask, double r_layer, void* ws, size_t ws_bytes,
+                           void* stream) {
+  if (!in || !scores) return SP_ERR_INVALID_ARG;
+  if (group < 1 || n_units < 1) return SP_ERR_SHAPE;
+  const int64_t cols = n_units * group;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (kind == SP_SCORE_WANDA_L2 || kind == SP_SCORE_WANDA_L1) {
+    if (!in->W.ptr) return SP_ERR_INVALID_ARG;
+    if (in->W.dtype != SP_F32) return SP_ERR_DTYPE;
+    if (in->W.cols != cols || in->W.ld < cols || in->W.rows < 1) return SP_ERR_SHAPE;
+    if (kind == SP_SCORE_WANDA_L2 && (!in->colsq || in->colsq_stride < 1)) return SP_ERR_INVALID_ARG;
+    if (kind == SP_SCORE_WANDA_L1 && !in->colabs) return SP_ERR_INVALID_ARG;
+    if (relaxed_mask) return SP_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < sp_workspace_bytes(SP_WS_SCORES, cols, 0, in->W.rows, 0, SP_F32)) return SP_ERR_WORKSPACE;
+    CU(wanda_scores(kind, group, reinterpret_cast<const float*>(in->W.ptr), in->W.rows, in->W.ld, in->colsq,
+                    in->colsq_stride, in->colabs, in->inv_tokens, n_units, scores, layer_importance,
+                    reinterpret_cast<double*>(ws), s));
+    return SP_OK;
+  }
+  if (kind == SP_SCORE_LEMMA1) {
+    const sp_mat* ms[4] = {&in->b, &in->c, &in->dd, &in->t};
+    const int64_t N = in->b.rows;
+    for (const sp_mat* m : ms) {
+      if (!m->ptr) return SP_ERR_INVALID_ARG;
+      if (!valid_act_dtype(m->dtype)) return SP_ERR_DTYPE;
+      if (m->rows != N || m->cols != cols || m->ld < cols) return SP_ERR_SHAPE;
+    }
+    if (N < 1) return SP_ERR_SHAPE;
+    if (!ws || ws_bytes < sp_workspace_bytes(SP_WS_SCORES, cols, 0, N, 0, SP_F32)) return SP_ERR_WORKSPACE;
+    CU(lemma1_scores_stream(in->b, in->c, in->dd, in->t, group, n_units, scores, layer_importance, relaxed_mask,
+                            r_layer, reinterpret_cast<double*>(ws), s));
+    return SP_OK;
+  }
+  return SP_ERR_UNSUPPORTED;
+}
+
+sp_status sp_allocate_sparsity(const double* I, const int64_t* n_units, int32_t L, double rbar, double T, int32_t mode,
+                               double clip_hi, double* r_out, int64_t* k_keep_out, void* stream) {
+  if (!I || !n_units || !r_out || !k_keep_out) return SP_ERR_INVALID_ARG;
+  if (L < 1 || L > 65536) return SP_ERR_SHAPE;
+  if (!(T > 0.0) || !(rbar >= 0.0 && rbar <= 1.0) || !(clip_hi > 0.0 && clip_hi <= 1.0)) return SP_ERR_INVALID_ARG;
+  if (mode != SP_ALLOC_SOFTMAX && mode != SP_ALLOC_INVERSE && mode != SP_ALLOC_UNIFORM) return SP_ERR_UNSUPPORTED;
+  CU(allocate_sparsity(I, n_units, L, rbar, T, mode, clip_hi, r_out, k_keep_out,
+                       reinterpret_cast<cudaStream_t>(stream)));
+  return SP_OK;
+}
+
+sp_status sp_apply_mask(const float* scores, int64_t n_units, int64_t k_keep, int32_t group, uint8_t* mask_out,
+                        float* tau_out, int32_t* kept_idx_out, const sp_mat* W_rows, const sp_mat* W_cols, void* ws,
+                        size_t ws_bytes, void* stream) {
+  (void)ws; (void)ws_bytes;
+  if (!scores || !mask_out) return SP_ERR_INVALID_ARG;
+  if (n_units < 0 || n_units > 0x7fffffff || group < 1 || k_keep < 0 || k_keep > n_units) return SP_ERR_SHAPE;
+  if (W_rows) {
+    if (!W_rows->ptr) return SP_ERR_INVALID_ARG;
+    if (W_rows->dtype != SP_F32) return SP_ERR_DTYPE;
+    if (W_rows->rows != n_units * group || W_rows->ld < W_rows->cols) return SP_ERR_SHAPE;
+  }
+  if (W_cols) {
+    if (!W_cols->ptr) return SP_ERR_INVALID_ARG;
+    if (W_cols->dtype != SP_F32) return SP_ERR_DTYPE;
+    if (W_cols->cols != n_units * group || W_cols->ld < W_cols->cols) return SP_ERR_SHAPE;
+  }
+  if (n_units == 0) return SP_OK;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  CU(topk_select(scores, n_units, k_keep, mask_out, tau_out, kept_idx_out, s));
+  CU(zero_pruned(mask_out, group, W_rows ? reinterpret_cast<float*>(W_rows->ptr) : nullptr,
+                 W_rows ? W_rows->rows : 0, W_rows ? W_rows->cols : 0, W_rows ? W_rows->ld : 0,
+                 W_cols ? reinterpret_cast<float*>(W_cols->ptr) : nullptr, W_cols ? W_cols->rows : 0,
+                 W_cols ? W_cols->cols : 0, W_cols ? W_cols->ld : 0, s));
+  return SP_OK;
+}
+
+static sp_status check_module(const sp_ffn_module* m, const sp_ffn_state* st, bool need_w0) {
+  if (!m || !st) return SP_ERR_INVALID_ARG;
+  if (m->d < 1 || m->n < 1 || m->N < 1) return SP_ERR_SHAPE;
+  if (m->act != SP_ACT_RELU) return SP_ERR_UNSUPPORTED;
+  if (!m->X.ptr || !m->Ypre.ptr) return SP_ERR_INVALID_ARG;
+  if (!valid_act_dtype(m->X.dtype) || m->Ypre.dtype != m->X.dtype) return SP_ERR_DTYPE;
+  if (m->X.rows != m->N || m->X.cols != m->d || m->X.ld < m->d) return SP_ERR_SHAPE;
+  if (m->Ypre.rows != m->N || m->Ypre.cols != m->d || m->Ypre.ld < m->d) return SP_ERR_SHAPE;
+  if (need_w0) {
+    if (!m->W1_0.ptr || !m->W2_0.ptr) return SP_ERR_INVALID_ARG;
+    if (m->W1_0.dtype != SP_F32 || m->W2_0.dtype != SP_F32) return SP_ERR_DTYPE;
+    if (m->W1_0.rows != m->n || m->W1_0.cols != m->d || m->W1_0.ld < m->d) return SP_ERR_SHAPE;
+    if (m->W2_0.rows != m->d || m->W2_0.cols != m->n || m->W2_0.ld < m->n) return SP_ERR_SHAPE;
+  }
+  if (!st->Z || !st->G_X || !st->G_A || !st->R1 || !st->R2 || !st->absA) return SP_ERR_INVALID_ARG;
+  return SP_OK;
+}
+
+sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_chunk, int32_t* status_dev, void* ws,
+                      size_t ws_bytes, void* stream) {
+  SPCHK(check_module(m, st, true));
+  if (token_chunk < 0) return SP_ERR_INVALID_ARG;
+  const int64_t d = m->d, n = m->n, N = m->N;
+  const int32_t cdt = m->X.dtype;
+  if (!ws || ws_bytes < plan_init(nullptr, d, n, N, token_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
+  InitPlan p = plan_init(ws, d, n, N, token_chunk, cdt);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const bool bf16 = p.bf16;
+  const bool acc64 = !bf16;
+  MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, w20{m->W2_0.ptr, SP_F32, m->W2_0.ld};
+  if (bf16) {
+    CU(convert_matrix(m->W1_0.ptr, SP_F32, m->W1_0.ld, p.W10b, SP_BF16, d, n, d, s));
+    CU(convert_matrix(m->W2_0.ptr, SP_F32, m->W2_0.ld, p.W20b, SP_BF16, n, d, n, s));
+    w10 = MatRef{p.W10b, SP_BF16, d};
+    w20 = MatRef{p.W20b, SP_BF16, n};
+  }
+  if (st->U) CU(cudaMemsetAsync(st->U, 0, (size_t)N * n * sizeof(float), s));
+  const size_t esz = bf16 ? 2 : 4;
+  MatRef gx{st->G_X, SP_F32, d}, ga{st->G_A, SP_F32, n}, r1{st->R1, SP_F32, d}, r2{st->R2, SP_F32, n};
+  for (int64_t t0 = 0, ci = 0; t0 < N; t0 += p.chunk, ++ci) {
+    const int64_t Tc = (N - t0 < p.chunk) ? N - t0 : p.chunk;
+    const double acc = ci > 0 ? 1.0 : 0.0;
+    MatRef xc{reinterpret_cast<const uint8_t*>(m->X.ptr) + (size_t)t0 * m->X.ld * esz, cdt, m->X.ld};
+    MatRef yc{reinterpret_cast<uint8_t*>(m->Ypre.ptr) + (size_t)t0 * m->Ypre.ld * esz, cdt, m->Ypre.ld};
+    float* Zc = st->Z + (size_t)t0 * n;
+    MatRef zc{Zc, SP_F32, n};
+    MatRef ac{p.Ac, cdt, n};
+    MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : zc;
+    // z^pre = X W1_0^T
+    SPCHK(contract(Tc, n, d, 1.0, xc, true, w10, true, 0.0, zc, zc, false, acc64, bf16, status_dev, s));
+    int rb;
+    fused_update_grid(Tc, n, &rb);
+    CU(launch_init_act(Zc, p.Ac, p.Zb, cdt, Tc, n, p.absA_part, rb, s));
+    CU(reduce_col_partials(p.absA_part, rb, n, st->absA, ci > 0, s));
+    // Ypre = a^pre W2_0^T
+    SPCHK(contract(Tc, d, n, 1.0, ac, true, w20, true, 0.0, yc, yc, false, acc64, bf16, status_dev, s));
+    // accumulators
+    SPCHK(contract(d, d, Tc, 1.0, xc, false, xc, false, acc, gx, gx, true, acc64, bf16, status_dev, s));
+    SPCHK(contract(n, n, Tc, 1.0, ac, false, ac, false, acc, ga, ga, true, acc64, bf16, status_dev, s));
+    SPCHK(contract(n, d, Tc, 1.0, zb, false, xc, false, acc, r1, r1, false, acc64, bf16, status_dev, s));
+    SPCHK(contract(d, n, Tc, 1.0, yc, false, ac, false, acc, r2, r2, false, acc64, bf16, status_dev, s));
+  }
+  CU(symmetrize_lower(st->G_X, d, d, s));
+  CU(symmetrize_lower(st->G_A, n, n, s));
+  return SP_OK;
+}
+
+sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* prm, sp_step_report* rep_dev,
+                       int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+  if (!prm) return SP_ERR_INVALID_ARG;
+  SPCHK(check_module(m, st, prm->score_kind == SP_SCORE_LEMMA1));
+  if (!st->W1 || !st->W2 || !st->scores || !st->mask || !st->importance) return SP_ERR_INVALID_ARG;
+  if (prm->dual_mode && !st->U) return SP_ERR_INVALID_ARG;
+  const int64_t d = m->d, n = m->n, N = m->N;
+  if (prm->k_keep < 1 || prm->k_keep > n) return SP_ERR_SHAPE;
+  if (!(prm->alpha > 0.0) || !(prm->beta > 0.0) || !(prm->rho >= 0.0) || prm->token_chunk < 0) return SP_ERR_INVALID_ARG;
+  if (prm->z_rule != SP_Z_PAPER && prm->z_rule != SP_Z_EXACT) return SP_ERR_UNSUPPORTED;
+  if (prm->score_kind < SP_SCORE_WANDA_L2 || prm->score_kind > SP_SCORE_LEMMA1) return SP_ERR_UNSUPPORTED;
+  const int32_t cdt = m->X.dtype;
+  if (!ws || ws_bytes < plan_admm(nullptr, d, n, N, prm->token_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
+  AdmmPlan p = plan_admm(ws, d, n, N, prm->token_chunk, cdt);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const bool bf16 = p.bf16;
+  const bool acc64 = !bf16;
+  const int64_t k = prm->k_keep;
+  double* rho1 = p.sb.rho;
+  double* rho2 = p.sb.rho + 1;
+  double* gam = p.sb.rho + 2;
+
+  // ---- 1. weight recovery W1~ = R1 (G_X + rho1 I)^-1, W2~ = R2 (G_A + rho2 I)^-1
+  CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, s));
+  CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
+  if (bf16) {
+    SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sb, status_dev, s));
+    SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
+  } else {
+    SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sb, status_dev, s));
+    SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
+  }
+
+  // ---- 2. unit scores and layer importance
+  if (prm->score_kind == SP_SCORE_LEMMA1) {
+    // b = W1~ X, c = d = t = z^pre = W1_0 X, written through G_X:  T0 = W1_0 G_X
+    MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, gx{st->G_X, SP_F32, d}, t0{p.T0, SP_F32, d};
+    SPCHK(contract(n, d, d, 1.0, w10, true, gx, false, 0.0, t0, t0, false, true, false, status_dev, s));
+    if (m->W1_0.ld != d) return SP_ERR_SHAPE;
+    CU(lemma1_scores_gram(p.T0, p.W1t, reinterpret_cast<const float*>(m->W1_0.ptr), n, d, st->scores, st->importance,
+                          p.score_scratch, s));
+  } else {
+    CU(wanda_scores(prm->score_kind, 1, p.W2t, d, n, st->G_A, n + 1, st->absA, 1.0 / (double)N, n, st->scores,
+                    st->importance, p.score_scratch, s));
+  }
+
+  // ---- 3. top-k mask
+  if (prm->reselect_mask) CU(topk_select(st->scores, n, k, st->mask, nullptr, p.sb.idx, s));
+  else CU(mask_to_index(st->mask, n, p.sb.idx, s));
+
+  // ---- 4. masked weights: W1 = diag(M) W1~ ; W2 = recovery on the kept support (or M (.) W2~)
+  CU(mask_rows_copy(st->mask, p.W1t, d, st->W1, d, n, d, s));
+  if (prm->refit) {
+    if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s));
+    else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s));
+  } else {
+    CU(cudaMemcpyAsync(st->W2, p.W2t, (size_t)d * n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    CU(zero_pruned(st->mask, 1, nullptr, 0, 0, 0, st->W2, d, n, n, s));
+  }
+
+  // ---- 5a. operands of the a-update: C = gamma I + W2 W2^T (d x d), Qt = W2^T C^-1 (n x d)
+  MatRef w1{st->W1, SP_F32, d}, w2{st->W2, SP_F32, n}, qt{p.Qt, SP_F32, d};
+  if (bf16) {
+    CU(convert_matrix(st->W1, SP_F32, d, p.W1b, SP_BF16, d, n, d, s));
+    CU(convert_matrix(st->W2, SP_F32, n, p.W2b, SP_BF16, n, d, n, s));
+    w1 = MatRef{p.W1b, SP_BF16, d};
+    w2 = MatRef{p.W2b, SP_BF16, n};
+  }
+  {
+    MatRef cf{p.Cf, SP_F32, d};
+    SPCHK(contract(d, d, n, 1.0, w2, true, w2, true, 0.0, cf, cf, true, acc64, bf16, status_dev, s));
+    CU(effective_ridge(nullptr, 0, 1, prm->beta / prm->alpha, 0, gam, s));
+    if (bf16) {
+      float* Gs = reinterpret_cast<float*>(p.sb.Gs);
+      float* Rs = reinterpret_cast<float*>(p.sb.Rs);
+      CU(load_spd<float>(p.Cf, d, d, gam, Gs, d, s));
+      CU(potrf_lower<float>(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), status_dev, s));
+      // right-hand sides: the rows of W2^T as the tensor-core path sees them (bf16-rounded W2)
+      CU(convert_matrix(p.W2b, SP_BF16, n, p.W2t, SP_F32, n, d, n, s));
+      CU(transpose_convert<float>(p.W2t, n, d, n, Rs, d, s));
+      CU(potrs_right<float>(Rs, n, d, d, Gs, d, reinterpret_cast<float*>(p.sb.dinv), s));
+      CU(convert_matrix(Rs, SP_F32, d, p.Qt, SP_F32, d, n, d, s));
+      CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, n, d, s));
+      qt = MatRef{p.Qtb, SP_BF16, d};
+    } else {
+      double* Gs = reinterpret_cast<double*>(p.sb.Gs);
+      double* Rs = reinterpret_cast<double*>(p.sb.Rs);
+      CU(load_spd<double>(p.Cf, d, d, gam, Gs, d, s));
+      CU(potrf_lower<double>(Gs, d, d, reinterpret_cast<double*>(p.sb.dinv), status_dev, s));
+      CU(transpose_convert<double>(st->W2, n, d, n, Rs, d, s));
+      CU(potrs_right<double>(Rs, n, d, d, Gs, d, reinterpret_cast<double*>(p.sb.dinv), s));
+      CU(convert_matrix(Rs, SP_F64, d, p.Qt, SP_F32, d, n, d, s));
+    }
+  }
+
+  // ---- 5b. token pass
+  if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, s));
+  const size_t esz = bf16 ? 2 : 4;
+  MatRef ga{st->G_A, SP_F32, n}, r1{st->R1, SP_F32, d}, r2{st->R2, SP_F32, n};
+  for (int64_t t0 = 0, ci = 0; t0 < N; t0 += p.chunk, ++ci) {
+    const int64_t Tc = (N - t0 < p.chunk) ? N - t0 : p.chunk;
+    const double acc = ci > 0 ? 1.0 : 0.0;
+    MatRef xc{reinterpret_cast<const uint8_t*>(m->X.ptr) + (size_t)t0 * m->X.ld * esz, cdt, m->X.ld};
+    MatRef yc{reinterpret_cast<const uint8_t*>(m->Ypre.ptr) + (size_t)t0 * m->Ypre.ld * esz, cdt, m->Ypre.ld};
+    float* Zc = st->Z + (size_t)t0 * n;
+    float* Uc = (prm->dual_mode && st->U) ? st->U + (size_t)t0 * n : nullptr;
+    MatRef h{p.H, cdt, n}, e{p.E, cdt, d}, dd{p.D, SP_F32, n}, z1{p.z1, SP_F32, n}, ac{p.Ac, cdt, n};
+    MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : MatRef{Zc, SP_F32, n};
+    CU(launch_prep_h(Zc, Uc, p.H, cdt, Tc, n, s));
+    // E = Ypre - h W2^T ; D = E Qt^T ; z1 = X W1^T
+    SPCHK(contract(Tc, d, n, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
+    SPCHK(contract(Tc, n, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
+    SPCHK(contract(Tc, n, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, bf16, status_dev, s));
+    UpdateArgs ua;
+    ua.Z = Zc; ua.U = Uc; ua.z1 = p.z1; ua.D = p.D; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
+    ua.out_dtype = cdt; ua.T = Tc; ua.n = n; ua.alpha = (float)prm->alpha; ua.beta = (float)prm->beta;
+    ua.z_rule = prm->z_rule; ua.partial = p.partial; ua.absA_part = p.absA_part;
+    const int nblk = fused_update_grid(Tc, n, &ua.row_blocks);
+    CU(launch_fused_update(ua, s));
+    if (rep_dev) CU(reduce_report(p.partial, nblk, rep_dev, ci > 0, s));
+    CU(reduce_col_partials(p.absA_part, ua.row_blocks, n, st->absA, ci > 0, s));
+    // accumulators of the new auxiliary variables
+    SPCHK(contract(n, n, Tc, 1.0, ac, false, ac, false, acc, ga, ga, true, acc64, bf16, status_dev, s));
+    SPCHK(contract(d, n, Tc, 1.0, yc, false, ac, false, acc, r2, r2, false, acc64, bf16, status_dev, s));
+    SPCHK(contract(n, d, Tc, 1.0, zb, false, xc, false, acc, r1, r1, false, acc64, bf16, status_dev, s));
+  }
+  CU(symmetrize_lower(st->G_A, n, n, s));
+  return SP_OK;
+}
+
+}  // extern "C"

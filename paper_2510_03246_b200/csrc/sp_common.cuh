@@ -1,0 +1,157 @@
+// Shared declarations of the libsp translation units (host-side launchers and small device helpers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sp.h"
+
+namespace sp {
+
+// Device status word layout: status_dev[0] = code, [1] = failing index, [2] = aux, [3] = reserved.
+__device__ __forceinline__ void report_status(int32_t* status, int32_t code, int32_t index, int32_t aux) {
+  if (status == nullptr) return;
+  if (atomicCAS(status, 0, code) == 0) {
+    status[1] = index;
+    status[2] = aux;
+  }
+}
+
+__host__ __device__ __forceinline__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+__host__ __device__ __forceinline__ size_t align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
+
+inline size_t dtype_size(int32_t dt) { return dt == SP_BF16 ? 2 : (dt == SP_F64 ? 8 : 4); }
+
+// A strided operand of the SIMT GEMM: element (i, k) lives at ptr[i * s0 + k * s1].
+struct Operand {
+  const void* ptr;
+  int32_t dtype;
+  int64_t s0, s1;
+};
+
+struct OutOperand {
+  void* ptr;
+  int32_t dtype;
+  int64_t ld;
+};
+
+// C[M,N] (row-major) = alpha * sum_k A(i,k) B(k,j) + beta * Cin[i,j].  Cin may alias C or be another matrix of
+// another dtype; beta == 0 never reads Cin.  lower_only skips tiles that lie strictly above the diagonal.
+// acc64: accumulate in fp64 (else fp32).
+cudaError_t gemm_simt(int64_t M, int64_t N, int64_t K, double alpha, Operand A, Operand B, double beta,
+                      Operand Cin, OutOperand C, bool lower_only, bool acc64, cudaStream_t stream);
+
+// tcgen05 path: bf16 operands, fp32 accumulation in tensor memory.
+//   a_kmajor: A is stored [M, K] row-major (K contiguous) ; else [K, M] row-major (M contiguous).
+//   b_kmajor: B is stored [N, K] row-major (K contiguous) ; else [K, N] row-major (N contiguous).
+// Returns SP_ERR_UNSUPPORTED when alignment rules of the tensor maps are not met (the caller may then use gemm_simt).
+struct TcOperand {
+  const void* ptr;  // bf16
+  int64_t ld;       // elements between consecutive rows of the stored matrix
+  bool kmajor;
+};
+sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
+                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream);
+bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B);
+
+// Dense symmetric positive definite solve in precision T (float or double), all on `stream`.
+//   potrf: in-place lower Cholesky of the n x n matrix A (ld lda); the strict upper triangle is not referenced.
+//   inv diag blocks are kept in `dinv` (n x NB row-major slabs) for the triangular solves.
+struct CholWork {
+  void* dinv;  // [ceil(n/NB) * NB * NB] elements of T
+};
+template <typename T>
+cudaError_t potrf_lower(T* A, int64_t n, int64_t lda, T* dinv, int32_t* status_dev, cudaStream_t stream);
+// X[m,n] <- X L^-T L^-1 (right solves with the factor of potrf_lower), i.e. X (L L^T)^-1.
+template <typename T>
+cudaError_t potrs_right(T* X, int64_t m, int64_t n, int64_t ldx, const T* L, int64_t ldl, const T* dinv,
+                        cudaStream_t stream);
+constexpr int kCholNB = 64;
+
+// ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
+cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
+                           int64_t rows, int64_t cols, cudaStream_t stream);
+cudaError_t symmetrize_lower(float* G, int64_t n, int64_t ld, cudaStream_t stream);
+// dst[j, i] = (TD) src[i, j]
+template <typename TD>
+cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64_t cols, TD* dst, int64_t ldd,
+                              cudaStream_t stream);
+int column_stats_row_blocks(int64_t T, int64_t C);
+int score_row_blocks(int64_t rows, int64_t cols);
+// dst[i,j] = (T) G[i*ld + j] (+ rho on the diagonal) for the lower triangle; rho read from device (rho_dev[0]).
+template <typename T>
+cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_dev, T* dst, int64_t ldd,
+                     cudaStream_t stream);
+// gathered version: dst[a,b] = G[idx[a], idx[b]] (+rho on diagonal), count read from host k.
+template <typename T>
+cudaError_t load_spd_gather(const float* G, int64_t ldg, const int32_t* idx, int64_t k, const double* rho_dev, T* dst,
+                            int64_t ldd, cudaStream_t stream);
+// dst[i, a] = (T) src[i, idx[a]]  (idx == nullptr: identity)
+template <typename T>
+cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
+                        int64_t ldd, cudaStream_t stream);
+// dst (fp32, [rows, n]) = 0 ; dst[i, idx[a]] = src[i, a]
+template <typename T>
+cudaError_t scatter_cols(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, int64_t n,
+                         float* dst, int64_t ldd, cudaStream_t stream);
+// rho_out[0] = rho * trace(G)/n (relative) or rho
+cudaError_t effective_ridge(const float* G, int64_t ldg, int64_t n, double rho, int rel, double* rho_out,
+                            cudaStream_t stream);
+
+struct UpdateArgs {
+  float* Z;          // [T, n] in/out
+  float* U;          // [T, n] in/out or null
+  const float* z1;   // [T, n]
+  const float* D;    // [T, n] correction term of the a-update
+  void* A_out;       // [T, n] storage dtype
+  void* Zb_out;      // [T, n] storage dtype copy of Z_new
+  int32_t out_dtype;
+  int64_t T, n;
+  float alpha, beta;
+  int32_t z_rule;
+  double* partial;   // [gridDim.x * 3] block partial sums: res_act, z_sq, a_sq
+  double* absA_part; // [row_blocks, n] partial column sums of |A|
+  int32_t row_blocks;
+};
+cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n,
+                          cudaStream_t stream);
+cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
+int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
+// out[j] (+)= sum_r part[r, j]
+cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
+                                cudaStream_t stream);
+// rep[field] (+)= sum of partial triples
+cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate,
+                          cudaStream_t stream);
+cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
+                        cudaStream_t stream);
+// relu + storage conversion for the init pass: A = phi(Z) -> storage dtype, and |A| column partials
+cudaError_t launch_init_act(const float* Z, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T, int64_t n,
+                            double* absA_part, int32_t row_blocks, cudaStream_t stream);
+cudaError_t column_stats(const void* X, int32_t dt, int64_t ld, int64_t T, int64_t C, double* rowstats,
+                         double* scratch, cudaStream_t stream);
+
+// ---- scores / allocation / selection (sp_mask.cu) -----------------------------------------------------------------
+cudaError_t wanda_scores(int kind, int group, const float* W, int64_t rows, int64_t ldw, const float* colsq,
+                         int64_t colsq_stride, const double* colabs, double inv_tokens, int64_t n_units,
+                         float* scores, double* importance, double* scratch, cudaStream_t stream);
+cudaError_t lemma1_scores_stream(const sp_mat& b, const sp_mat& c, const sp_mat& dd, const sp_mat& t, int group,
+                                 int64_t n_units, float* scores, double* importance, double* relaxed, double r_layer,
+                                 double* scratch, cudaStream_t stream);
+// s_j = (cb_j + cc_j) / (2 cc_j) with cb_j = <T0[j,:], W1t[j,:]>, cc_j = <T0[j,:], W10[j,:]>, T0 = W10 G_X
+cudaError_t lemma1_scores_gram(const float* T0, const float* W1t, const float* W10, int64_t n, int64_t d,
+                               float* scores, double* importance, double* scratch, cudaStream_t stream);
+cudaError_t allocate_sparsity(const double* I, const int64_t* n_units, int L, double rbar, double T, int mode,
+                              double clip_hi, double* r_out, int64_t* k_out, cudaStream_t stream);
+cudaError_t topk_select(const float* scores, int64_t n, int64_t k, uint8_t* mask, float* tau, int32_t* kept_idx,
+                        cudaStream_t stream);
+// kept_idx from an existing mask (ascending), count must equal k
+cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream);
+cudaError_t zero_pruned(const uint8_t* mask, int group, float* W_rows, int64_t r_rows, int64_t r_cols, int64_t r_ld,
+                        float* W_cols, int64_t c_rows, int64_t c_cols, int64_t c_ld, cudaStream_t stream);
+// dst[i,:] = mask[i] ? src[i,:] : 0
+cudaError_t mask_rows_copy(const uint8_t* mask, const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows,
+                           int64_t cols, cudaStream_t stream);
+
+}  // namespace sp

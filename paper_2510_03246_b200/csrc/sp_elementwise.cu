@@ -1,0 +1,535 @@
+// Elementwise and reduction kernels of the ADMM step: the fused auxiliary-variable update (a-update epilogue,
+// z^(2), select, dual update, residual and |A| statistics in one pass over the chunk), operand preparation,
+// conversions, gathers and small reductions.  All reductions use a fixed order (no floating-point atomics).
+#include "sp_common.cuh"
+
+namespace sp {
+namespace {
+
+__device__ __forceinline__ float ld_any(const void* p, int32_t dt, int64_t i) {
+  return dt == SP_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
+                       : (dt == SP_F64 ? (float)reinterpret_cast<const double*>(p)[i]
+                                       : reinterpret_cast<const float*>(p)[i]);
+}
+
+template <typename T>
+__device__ __forceinline__ T block_sum(T v, T* smem) {
+  // fixed-order tree: warp shuffles, then warp 0 adds the warp results in order
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) smem[w] = v;
+  __syncthreads();
+  T r = (T)0;
+  if (threadIdx.x == 0) {
+    const int nw = (blockDim.x + 31) >> 5;
+    for (int i = 0; i < nw; ++i) r += smem[i];
+  }
+  return r;  // valid in thread 0
+}
+
+// ------------------------------------------------------------------------------------------------ conversions
+__global__ void convert_kernel(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
+                               int64_t rows, int64_t cols) {
+  const int64_t total = rows * cols;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / cols, j = e % cols;
+    const int64_t si = i * lds + j, di = i * ldd + j;
+    if (sdt == SP_F64) {
+      const double v = reinterpret_cast<const double*>(src)[si];
+      if (ddt == SP_F64) reinterpret_cast<double*>(dst)[di] = v;
+      else if (ddt == SP_BF16) reinterpret_cast<__nv_bfloat16*>(dst)[di] = __float2bfloat16_rn((float)v);
+      else reinterpret_cast<float*>(dst)[di] = (float)v;
+    } else {
+      const float v = ld_any(src, sdt, si);
+      if (ddt == SP_F64) reinterpret_cast<double*>(dst)[di] = (double)v;
+      else if (ddt == SP_BF16) reinterpret_cast<__nv_bfloat16*>(dst)[di] = __float2bfloat16_rn(v);
+      else reinterpret_cast<float*>(dst)[di] = v;
+    }
+  }
+}
+
+// dst[j, i] = src[i, j] through a 32 x 32 shared tile
+template <typename TD>
+__global__ void transpose_convert_kernel(const float* src, int64_t lds, int64_t rows, int64_t cols, TD* dst,
+                                         int64_t ldd) {
+  __shared__ float tile[32][33];
+  const int64_t c0 = (int64_t)blockIdx.x * 32, r0 = (int64_t)blockIdx.y * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int64_t i = r0 + r, j = c0 + threadIdx.x;
+    tile[r][threadIdx.x] = (i < rows && j < cols) ? src[i * lds + j] : 0.f;
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int64_t j = c0 + r, i = r0 + threadIdx.x;
+    if (i < rows && j < cols) {
+      if constexpr (sizeof(TD) == 2) dst[j * ldd + i] = __float2bfloat16_rn(tile[threadIdx.x][r]);
+      else dst[j * ldd + i] = (TD)tile[threadIdx.x][r];
+    }
+  }
+}
+
+__global__ void symmetrize_kernel(float* G, int64_t n, int64_t ld) {
+  __shared__ float tile[32][33];
+  // block (bx, by) with bx > by mirrors lower tile (row block bx, col block by) to (by, bx); diagonal blocks in place
+  const int64_t bx = blockIdx.x, by = blockIdx.y;
+  if (bx < by) return;
+  const int64_t r0 = bx * 32, c0 = by * 32;
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int64_t i = r0 + r, j = c0 + threadIdx.x;
+    tile[r][threadIdx.x] = (i < n && j < n) ? G[i * ld + j] : 0.f;
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+    const int64_t i = c0 + r, j = r0 + threadIdx.x;  // element (i, j) of the upper part = lower (j, i)
+    if (i < n && j < n && j > i) G[i * ld + j] = tile[threadIdx.x][r];
+  }
+}
+
+template <typename T>
+__global__ void load_spd_kernel(const float* G, int64_t ldg, const int32_t* idx, int64_t n, const double* rho, T* dst,
+                                int64_t ldd) {
+  const double r = rho ? rho[0] : 0.0;
+  const int64_t total = n * n;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / n, j = e % n;
+    if (j > i) continue;
+    const int64_t gi = idx ? idx[i] : i, gj = idx ? idx[j] : j;
+    // the lower triangle of G is authoritative: read (max, min)
+    const int64_t a = gi > gj ? gi : gj, b = gi > gj ? gj : gi;
+    double v = (double)G[a * ldg + b];
+    if (i == j) v += r;
+    dst[i * ldd + j] = (T)v;
+  }
+}
+
+template <typename T>
+__global__ void gather_cols_kernel(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
+                                   int64_t ldd) {
+  const int64_t total = rows * k;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / k, a = e % k;
+    dst[i * ldd + a] = (T)src[i * lds + (idx ? idx[a] : a)];
+  }
+}
+
+template <typename T>
+__global__ void scatter_cols_kernel(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k,
+                                    float* dst, int64_t ldd) {
+  const int64_t total = rows * k;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / k, a = e % k;
+    dst[i * ldd + (idx ? idx[a] : a)] = (float)src[i * lds + a];
+  }
+}
+
+__global__ void fill_zero_kernel(float* dst, int64_t ld, int64_t rows, int64_t cols) {
+  const int64_t total = rows * cols;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x)
+    dst[(e / cols) * ld + (e % cols)] = 0.f;
+}
+
+__global__ void effective_ridge_kernel(const float* G, int64_t ldg, int64_t n, double rho, int rel, double* out) {
+  __shared__ double sm[32];
+  double s = 0.0;
+  if (rel)
+    for (int64_t i = threadIdx.x; i < n; i += blockDim.x) s += (double)G[i * ldg + i];
+  s = block_sum<double>(s, sm);
+  if (threadIdx.x == 0) out[0] = rel ? rho * s / (double)n : rho;
+}
+
+// ------------------------------------------------------------------------------------------------ chunk kernels
+// H = storage(phi(Z) - U)
+__global__ void prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U, void* H, int32_t hdt,
+                              int64_t total) {
+  for (int64_t e = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; e < total;
+       e += (int64_t)gridDim.x * blockDim.x * 4) {
+    if (e + 3 < total) {
+      const float4 z = *reinterpret_cast<const float4*>(Z + e);
+      float4 h = make_float4(fmaxf(z.x, 0.f), fmaxf(z.y, 0.f), fmaxf(z.z, 0.f), fmaxf(z.w, 0.f));
+      if (U) {
+        const float4 u = *reinterpret_cast<const float4*>(U + e);
+        h.x -= u.x; h.y -= u.y; h.z -= u.z; h.w -= u.w;
+      }
+      if (hdt == SP_BF16) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(h.x, h.y), hi = __floats2bfloat162_rn(h.z, h.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(H) + e) = pk;
+      } else {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(H) + e) = h;
+      }
+    } else {
+      for (int64_t q = e; q < total; ++q) {
+        float h = fmaxf(Z[q], 0.f) - (U ? U[q] : 0.f);
+        if (hdt == SP_BF16) reinterpret_cast<__nv_bfloat16*>(H)[q] = __float2bfloat16_rn(h);
+        else reinterpret_cast<float*>(H)[q] = h;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void store4(void* base, int32_t dt, int64_t e, float a, float b, float c, float d) {
+  if (dt == SP_BF16) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(base) + e) = pk;
+  } else {
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e) = make_float4(a, b, c, d);
+  }
+}
+
+// One element of the fused update.  Returns A; writes the new z (and u).
+__device__ __forceinline__ float update_one(float zold, float z1, float dcorr, float& u, bool has_u, float alpha,
+                                            float beta, float inv_ab, int z_rule, float& znew) {
+  const float h = fmaxf(zold, 0.f) - (has_u ? u : 0.f);
+  const float a = h + dcorr;
+  const float au = a + (has_u ? u : 0.f);
+  const float z2 = (beta * au + alpha * z1) * inv_ab;
+  if (z_rule == SP_Z_PAPER) {
+    znew = (zold < 0.f) ? z1 : z2;
+  } else {
+    const float zn = fminf(z1, 0.f), zp = fmaxf(z2, 0.f);
+    const float fn = beta * au * au + alpha * (zn - z1) * (zn - z1);
+    const float fp = beta * (au - zp) * (au - zp) + alpha * (zp - z1) * (zp - z1);
+    znew = (fn < fp) ? zn : zp;
+  }
+  if (has_u) u = u + a - fmaxf(znew, 0.f);
+  return a;
+}
+
+// grid: (col blocks of 1024, row blocks).  Thread owns 4 consecutive columns and walks its block's rows.
+__global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
+  __shared__ double sm[32];
+  const int64_t c0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+  const int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
+  const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
+  const int64_t r_end = (r_begin + rows_per < g.T) ? r_begin + rows_per : g.T;
+  const bool has_u = g.U != nullptr;
+  const float inv_ab = 1.f / (g.alpha + g.beta);
+  double s_res = 0.0, s_z = 0.0, s_a = 0.0;
+  double cs[4] = {0.0, 0.0, 0.0, 0.0};
+  const bool vec = (g.n % 4 == 0);
+  if (c0 < g.n) {
+    for (int64_t r = r_begin; r < r_end; ++r) {
+      const int64_t e = r * g.n + c0;
+      float zo[4], z1[4], dc[4], u[4] = {0.f, 0.f, 0.f, 0.f}, a[4], zn[4];
+      const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
+      if (vec) {
+        const float4 v0 = *reinterpret_cast<const float4*>(g.Z + e);
+        const float4 v1 = *reinterpret_cast<const float4*>(g.z1 + e);
+        const float4 v2 = *reinterpret_cast<const float4*>(g.D + e);
+        zo[0] = v0.x; zo[1] = v0.y; zo[2] = v0.z; zo[3] = v0.w;
+        z1[0] = v1.x; z1[1] = v1.y; z1[2] = v1.z; z1[3] = v1.w;
+        dc[0] = v2.x; dc[1] = v2.y; dc[2] = v2.z; dc[3] = v2.w;
+        if (has_u) {
+          const float4 v3 = *reinterpret_cast<const float4*>(g.U + e);
+          u[0] = v3.x; u[1] = v3.y; u[2] = v3.z; u[3] = v3.w;
+        }
+      } else {
+        for (int q = 0; q < cnt; ++q) {
+          zo[q] = g.Z[e + q]; z1[q] = g.z1[e + q]; dc[q] = g.D[e + q];
+          if (has_u) u[q] = g.U[e + q];
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q < cnt) {
+          a[q] = update_one(zo[q], z1[q], dc[q], u[q], has_u, g.alpha, g.beta, inv_ab, g.z_rule, zn[q]);
+          const double diff = (double)a[q] - (double)fmaxf(zn[q], 0.f);
+          s_res += diff * diff;
+          s_z += (double)zn[q] * (double)zn[q];
+          s_a += (double)a[q] * (double)a[q];
+          cs[q] += fabs((double)a[q]);
+        } else {
+          a[q] = 0.f; zn[q] = 0.f;
+        }
+      }
+      if (vec) {
+        *reinterpret_cast<float4*>(g.Z + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        if (has_u) *reinterpret_cast<float4*>(g.U + e) = make_float4(u[0], u[1], u[2], u[3]);
+        store4(g.A_out, g.out_dtype, e, a[0], a[1], a[2], a[3]);
+        if (g.Zb_out) store4(g.Zb_out, g.out_dtype, e, zn[0], zn[1], zn[2], zn[3]);
+      } else {
+        for (int q = 0; q < cnt; ++q) {
+          g.Z[e + q] = zn[q];
+          if (has_u) g.U[e + q] = u[q];
+          if (g.out_dtype == SP_BF16) {
+            reinterpret_cast<__nv_bfloat16*>(g.A_out)[e + q] = __float2bfloat16_rn(a[q]);
+            if (g.Zb_out) reinterpret_cast<__nv_bfloat16*>(g.Zb_out)[e + q] = __float2bfloat16_rn(zn[q]);
+          } else {
+            reinterpret_cast<float*>(g.A_out)[e + q] = a[q];
+            if (g.Zb_out) reinterpret_cast<float*>(g.Zb_out)[e + q] = zn[q];
+          }
+        }
+      }
+    }
+    if (g.absA_part) {
+      const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
+      for (int q = 0; q < cnt; ++q) g.absA_part[(int64_t)blockIdx.y * g.n + c0 + q] = cs[q];
+    }
+  }
+  const int64_t bid = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+  const double r0 = block_sum<double>(s_res, sm);
+  const double r1 = block_sum<double>(s_z, sm);
+  const double r2 = block_sum<double>(s_a, sm);
+  if (threadIdx.x == 0) {
+    g.partial[bid * 3 + 0] = r0;
+    g.partial[bid * 3 + 1] = r1;
+    g.partial[bid * 3 + 2] = r2;
+  }
+}
+
+// init pass: A = phi(Z) in storage dtype, optional storage copy of Z, |A| column partials
+__global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__ Z, void* A_out, void* Zb_out,
+                                                       int32_t out_dtype, int64_t T, int64_t n, double* absA_part,
+                                                       int32_t row_blocks) {
+  const int64_t c0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+  if (c0 >= n) return;
+  const int64_t rows_per = ceil_div(T, (int64_t)row_blocks);
+  const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
+  const int64_t r_end = (r_begin + rows_per < T) ? r_begin + rows_per : T;
+  const int cnt = (n - c0 >= 4) ? 4 : (int)(n - c0);
+  double cs[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int64_t r = r_begin; r < r_end; ++r) {
+    const int64_t e = r * n + c0;
+    for (int q = 0; q < cnt; ++q) {
+      const float z = Z[e + q];
+      const float a = fmaxf(z, 0.f);
+      cs[q] += (double)a;
+      if (out_dtype == SP_BF16) {
+        reinterpret_cast<__nv_bfloat16*>(A_out)[e + q] = __float2bfloat16_rn(a);
+        if (Zb_out) reinterpret_cast<__nv_bfloat16*>(Zb_out)[e + q] = __float2bfloat16_rn(z);
+      } else {
+        reinterpret_cast<float*>(A_out)[e + q] = a;
+        if (Zb_out) reinterpret_cast<float*>(Zb_out)[e + q] = z;
+      }
+    }
+  }
+  if (absA_part)
+    for (int q = 0; q < cnt; ++q) absA_part[(int64_t)blockIdx.y * n + c0 + q] = cs[q];
+}
+
+__global__ void reduce_col_partials_kernel(const double* part, int32_t row_blocks, int64_t n, double* out, int acc) {
+  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x) {
+    double s = acc ? out[j] : 0.0;
+    for (int r = 0; r < row_blocks; ++r) s += part[(int64_t)r * n + j];
+    out[j] = s;
+  }
+}
+
+__global__ void reduce_report_kernel(const double* partial, int nblocks, sp_step_report* rep, int acc) {
+  __shared__ double sm[32];
+  double s[3] = {0.0, 0.0, 0.0};
+  for (int i = threadIdx.x; i < nblocks; i += blockDim.x)
+    for (int f = 0; f < 3; ++f) s[f] += partial[(int64_t)i * 3 + f];
+  for (int f = 0; f < 3; ++f) {
+    const double r = block_sum<double>(s[f], sm);
+    if (threadIdx.x == 0) {
+      double* dst = f == 0 ? &rep->res_act : (f == 1 ? &rep->z_sq : &rep->a_sq);
+      *dst = (acc ? *dst : 0.0) + r;
+    }
+  }
+}
+
+__global__ void init_report_kernel(sp_step_report* rep, const double* rho1, const double* rho2, double kept) {
+  rep->res_act = 0.0;
+  rep->res_out = nan("");
+  rep->res_in = nan("");
+  rep->z_sq = 0.0;
+  rep->a_sq = 0.0;
+  rep->rho1_eff = rho1 ? rho1[0] : 0.0;
+  rep->rho2_eff = rho2 ? rho2[0] : 0.0;
+  rep->kept = kept;
+}
+
+// per-column sum |x| and sum x^2 of a [T, C] chunk: grid (col blocks of 256, row blocks) -> scratch, then reduced
+__global__ void column_stats_kernel(const void* X, int32_t dt, int64_t ld, int64_t T, int64_t C, double* scratch,
+                                    int32_t row_blocks) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  const int64_t rows_per = ceil_div(T, (int64_t)row_blocks);
+  const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
+  const int64_t r_end = (r_begin + rows_per < T) ? r_begin + rows_per : T;
+  double s1 = 0.0, s2 = 0.0;
+  for (int64_t r = r_begin; r < r_end; ++r) {
+    const double v = (double)ld_any(X, dt, r * ld + c);
+    s1 += fabs(v);
+    s2 += v * v;
+  }
+  scratch[((int64_t)blockIdx.y * C + c) * 2 + 0] = s1;
+  scratch[((int64_t)blockIdx.y * C + c) * 2 + 1] = s2;
+}
+
+__global__ void column_stats_reduce_kernel(const double* scratch, int32_t row_blocks, int64_t C, double* rowstats) {
+  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= C) return;
+  double s1 = rowstats[c * 2 + 0], s2 = rowstats[c * 2 + 1];
+  for (int r = 0; r < row_blocks; ++r) {
+    s1 += scratch[((int64_t)r * C + c) * 2 + 0];
+    s2 += scratch[((int64_t)r * C + c) * 2 + 1];
+  }
+  rowstats[c * 2 + 0] = s1;
+  rowstats[c * 2 + 1] = s2;
+}
+
+inline int grid_for(int64_t total, int threads, int per_thread = 1) {
+  int64_t b = ceil_div(total, (int64_t)threads * per_thread);
+  const int64_t cap = 148 * 16;
+  if (b > cap) b = cap;
+  if (b < 1) b = 1;
+  return (int)b;
+}
+
+}  // namespace
+
+cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
+                           int64_t rows, int64_t cols, cudaStream_t stream) {
+  if (rows * cols == 0) return cudaSuccess;
+  convert_kernel<<<grid_for(rows * cols, 256), 256, 0, stream>>>(src, sdt, lds, dst, ddt, ldd, rows, cols);
+  return cudaGetLastError();
+}
+
+template <typename TD>
+cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64_t cols, TD* dst, int64_t ldd,
+                              cudaStream_t stream) {
+  if (rows * cols == 0) return cudaSuccess;
+  dim3 grid((unsigned)ceil_div(cols, 32), (unsigned)ceil_div(rows, 32));
+  transpose_convert_kernel<TD><<<grid, dim3(32, 8), 0, stream>>>(src, lds, rows, cols, dst, ldd);
+  return cudaGetLastError();
+}
+template cudaError_t transpose_convert<float>(const float*, int64_t, int64_t, int64_t, float*, int64_t, cudaStream_t);
+template cudaError_t transpose_convert<double>(const float*, int64_t, int64_t, int64_t, double*, int64_t,
+                                               cudaStream_t);
+template cudaError_t transpose_convert<__nv_bfloat16>(const float*, int64_t, int64_t, int64_t, __nv_bfloat16*,
+                                                      int64_t, cudaStream_t);
+
+cudaError_t symmetrize_lower(float* G, int64_t n, int64_t ld, cudaStream_t stream) {
+  if (n == 0) return cudaSuccess;
+  const unsigned nb = (unsigned)ceil_div(n, 32);
+  symmetrize_kernel<<<dim3(nb, nb), dim3(32, 8), 0, stream>>>(G, n, ld);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_dev, T* dst, int64_t ldd,
+                     cudaStream_t stream) {
+  if (n == 0) return cudaSuccess;
+  load_spd_kernel<T><<<grid_for(n * n, 256), 256, 0, stream>>>(G, ldg, nullptr, n, rho_dev, dst, ldd);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t load_spd_gather(const float* G, int64_t ldg, const int32_t* idx, int64_t k, const double* rho_dev, T* dst,
+                            int64_t ldd, cudaStream_t stream) {
+  if (k == 0) return cudaSuccess;
+  load_spd_kernel<T><<<grid_for(k * k, 256), 256, 0, stream>>>(G, ldg, idx, k, rho_dev, dst, ldd);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
+                        int64_t ldd, cudaStream_t stream) {
+  if (rows * k == 0) return cudaSuccess;
+  gather_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
+  return cudaGetLastError();
+}
+template <typename T>
+cudaError_t scatter_cols(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, int64_t n,
+                         float* dst, int64_t ldd, cudaStream_t stream) {
+  if (rows * n == 0) return cudaSuccess;
+  if (idx) fill_zero_kernel<<<grid_for(rows * n, 256), 256, 0, stream>>>(dst, ldd, rows, n);
+  if (rows * k == 0) return cudaGetLastError();
+  scatter_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
+  return cudaGetLastError();
+}
+#define SP_INST(T)                                                                                                  \
+  template cudaError_t load_spd<T>(const float*, int64_t, int64_t, const double*, T*, int64_t, cudaStream_t);      \
+  template cudaError_t load_spd_gather<T>(const float*, int64_t, const int32_t*, int64_t, const double*, T*,       \
+                                          int64_t, cudaStream_t);                                                   \
+  template cudaError_t gather_cols<T>(const float*, int64_t, const int32_t*, int64_t, int64_t, T*, int64_t,        \
+                                      cudaStream_t);                                                                \
+  template cudaError_t scatter_cols<T>(const T*, int64_t, const int32_t*, int64_t, int64_t, int64_t, float*,       \
+                                       int64_t, cudaStream_t);
+SP_INST(float)
+SP_INST(double)
+#undef SP_INST
+
+cudaError_t effective_ridge(const float* G, int64_t ldg, int64_t n, double rho, int rel, double* rho_out,
+                            cudaStream_t stream) {
+  effective_ridge_kernel<<<1, 1024, 0, stream>>>(G, ldg, n, rho, rel, rho_out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n,
+                          cudaStream_t stream) {
+  const int64_t total = T * n;
+  if (total == 0) return cudaSuccess;
+  prep_h_kernel<<<grid_for(total, 256, 4), 256, 0, stream>>>(Z, U, H, hdt, total);
+  return cudaGetLastError();
+}
+
+int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
+  const int col_blocks = (int)ceil_div(n, 1024);
+  int rb = (148 * 4 + col_blocks - 1) / col_blocks;
+  if (rb > T) rb = (int)T;
+  if (rb < 1) rb = 1;
+  if (rb > 65535) rb = 65535;
+  *row_blocks = rb;
+  return col_blocks * rb;
+}
+
+cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
+  if (a.T * a.n == 0) return cudaSuccess;
+  dim3 grid((unsigned)ceil_div(a.n, 1024), (unsigned)a.row_blocks);
+  fused_update_kernel<<<grid, 256, 0, stream>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_init_act(const float* Z, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T, int64_t n,
+                            double* absA_part, int32_t row_blocks, cudaStream_t stream) {
+  if (T * n == 0) return cudaSuccess;
+  dim3 grid((unsigned)ceil_div(n, 1024), (unsigned)row_blocks);
+  init_act_kernel<<<grid, 256, 0, stream>>>(Z, A_out, Zb_out, out_dtype, T, n, absA_part, row_blocks);
+  return cudaGetLastError();
+}
+
+cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
+                                cudaStream_t stream) {
+  if (n == 0) return cudaSuccess;
+  reduce_col_partials_kernel<<<grid_for(n, 256), 256, 0, stream>>>(part, row_blocks, n, out, accumulate ? 1 : 0);
+  return cudaGetLastError();
+}
+
+cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate,
+                          cudaStream_t stream) {
+  reduce_report_kernel<<<1, 256, 0, stream>>>(partial, nblocks, rep, accumulate ? 1 : 0);
+  return cudaGetLastError();
+}
+
+cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
+                        cudaStream_t stream) {
+  init_report_kernel<<<1, 1, 0, stream>>>(rep, rho1, rho2, kept);
+  return cudaGetLastError();
+}
+
+cudaError_t column_stats(const void* X, int32_t dt, int64_t ld, int64_t T, int64_t C, double* rowstats,
+                         double* scratch, cudaStream_t stream) {
+  if (T * C == 0) return cudaSuccess;
+  const int rb = column_stats_row_blocks(T, C);
+  dim3 grid((unsigned)ceil_div(C, 256), (unsigned)rb);
+  column_stats_kernel<<<grid, 256, 0, stream>>>(X, dt, ld, T, C, scratch, rb);
+  column_stats_reduce_kernel<<<(unsigned)ceil_div(C, 256), 256, 0, stream>>>(scratch, rb, C, rowstats);
+  return cudaGetLastError();
+}
+
+int column_stats_row_blocks(int64_t T, int64_t C) {
+  const int64_t cb = ceil_div(C, 256);
+  int64_t rb = ceil_div(148 * 4, cb);
+  if (rb > T) rb = T;
+  if (rb < 1) rb = 1;
+  return (int)rb;
+}
+
+}  // namespace sp

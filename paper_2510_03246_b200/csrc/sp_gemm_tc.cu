@@ -1,0 +1,492 @@
+// bf16 tensor-core GEMM for sm_100a: TMA-fed shared-memory pipeline, tcgen05.mma with fp32 accumulators in tensor
+// memory, warp-specialised persistent CTAs (one per SM).
+//
+//   C[M,N] = alpha * A B^T-like contraction over K + beta * Cin
+//
+// Both operands may be K-major (stored [rows, K], K contiguous: the weight/activation products z^(1) = X W1^T, ...)
+// or MN-major (stored [K, rows], rows contiguous: the token-axis contractions A^T A, Z^T X, Ypre^T A).  Each
+// major-ness has its own TMA box shape and shared-memory matrix descriptor; the MMA instruction descriptor carries
+// the two major bits.  No cluster launch and no multicast loads are used.
+//
+// Roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = tensor-memory allocator + MMA issuer (one lane),
+// warps 2..5 = epilogue (each owns the 32 accumulator lanes its warp id maps to).  Two 256-column accumulators are
+// ping-ponged so that the epilogue of tile i overlaps the main loop of tile i+1.
+// Every wait is bounded by a clock budget; on expiry the CTA records SP_ERR_TIMEOUT, drains its copies and MMAs,
+// frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "sp_common.cuh"
+
+namespace sp {
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long WAIT_BUDGET_CYCLES = 6000000000LL;   // ~3 s at 2 GHz
+constexpr long long DRAIN_BUDGET_CYCLES = 200000000LL;   // ~0.1 s
+
+struct TcParams {
+  int64_t M, N, K;
+  float alpha, beta;
+  const void* cin;
+  int32_t cin_dtype;
+  int64_t cin_ld;
+  void* c;
+  int32_t c_dtype;
+  int64_t c_ld;
+  int32_t a_kmajor, b_kmajor, lower_only;
+  int32_t tiles_m, tiles_n, num_tiles;
+  int32_t* status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the budget ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t it = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++it & 0x3ffu) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > budget) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a 128-byte-swizzled operand tile.
+//   K-major : rows of 64 bf16 (128 B); 8-row groups 1024 B apart (stride byte offset); leading offset unused (1).
+//   MN-major: 64-element (128 B) runs along MN, one per K index; 8-K-index groups 1024 B apart (stride offset);
+//             consecutive 64-element MN blocks `mn_block_bytes` apart (leading offset).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, bool kmajor, uint32_t mn_block_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+  const uint32_t lbo = kmajor ? 1u : (mn_block_bytes >> 4);
+  d |= (uint64_t)(lbo & 0x3fffu) << 16;
+  d |= (uint64_t)((1024u >> 4) & 0x3fffu) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;  // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ uint32_t make_instr_desc(bool a_kmajor, bool b_kmajor) {
+  uint32_t d = 0;
+  d |= 1u << 4;                       // accumulator format: fp32
+  d |= 1u << 7;                       // A format: bf16
+  d |= 1u << 10;                      // B format: bf16
+  d |= (a_kmajor ? 0u : 1u) << 15;    // A major-ness
+  d |= (b_kmajor ? 0u : 1u) << 16;    // B major-ness
+  d |= (uint32_t)(BN >> 3) << 17;     // N
+  d |= (uint32_t)(BM >> 4) << 24;     // M
+  return d;
+}
+
+__device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, int& tn) {
+  if (!p.lower_only) {
+    tm = t % p.tiles_m;
+    tn = t / p.tiles_m;
+  } else {
+    // column block tn owns row blocks first(tn)..tiles_m-1 with first = tn * BN / BM
+    tn = 0;
+    for (;;) {
+      const int first = tn * (BN / BM);
+      const int cnt = p.tiles_m - first;
+      if (t < cnt) { tm = first + t; break; }
+      t -= cnt;
+      ++tn;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort;
+
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;            // 1024-byte aligned operand stages
+  const uint32_t bars = tiles + STAGES * STAGE_BYTES;       // 8-byte aligned barrier block
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+  const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  volatile int* abort_flag = &s_abort;
+
+  if (threadIdx.x == 0) {
+    s_abort = 0;
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    mbar_init(drain_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"((uint32_t)TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem_base;
+
+  const int num_kb = (int)((p.K + BK - 1) / BK);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      uint32_t armed = 0;          // bit s: stage s has been armed at least once
+      uint32_t armed_parity = 0;   // bit s: parity of the phase the last arming of stage s completes
+      bool ok = true;
+      for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+        int tm, tn;
+        tile_coords(p, t, tm, tn);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          armed |= 1u << s;
+          armed_parity = (armed_parity & ~(1u << s)) | (ph << s);
+          const uint32_t a_dst = tiles + s * STAGE_BYTES;
+          const uint32_t b_dst = a_dst + A_BYTES;
+          const int k0 = kb * BK;
+          if (p.a_kmajor) {
+            tma_load_2d(a_dst, &tmA, k0, tm * BM, full_bar(s));
+          } else {
+#pragma unroll
+            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, tm * BM + mb * 64, k0, full_bar(s));
+          }
+          if (p.b_kmajor) {
+            tma_load_2d(b_dst, &tmB, k0, tn * BN, full_bar(s));
+          } else {
+#pragma unroll
+            for (int nb = 0; nb < BN / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, tn * BN + nb * 64, k0, full_bar(s));
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 1);
+        // let copies already in flight land before the shared memory is released
+        for (int q = 0; q < STAGES; ++q)
+          if (armed & (1u << q)) {
+            const long long t0 = clock64();
+            while (!mbar_try(full_bar(q), (armed_parity >> q) & 1u) && clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
+          }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_instr_desc(p.a_kmajor != 0, p.b_kmajor != 0);
+      int s = 0;
+      uint32_t ph = 0;
+      int acc = 0;
+      uint32_t aph = 0;
+      bool ok = true;
+      bool issued = false;
+      for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(s), ph, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = tiles + s * STAGE_BYTES;
+          const uint32_t b_src = a_src + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // K-major: 16 bf16 = 32 B further along the swizzled row; MN-major: 16 K indices = 16 * 128 B further
+            const uint32_t a_off = p.a_kmajor ? (uint32_t)(k * UMMA_K * 2) : (uint32_t)(k * UMMA_K * 128);
+            const uint32_t b_off = p.b_kmajor ? (uint32_t)(k * UMMA_K * 2) : (uint32_t)(k * UMMA_K * 128);
+            const uint64_t adesc = make_smem_desc(a_src + a_off, p.a_kmajor != 0, 64 * BK * 2);
+            const uint64_t bdesc = make_smem_desc(b_src + b_off, p.b_kmajor != 0, 64 * BK * 2);
+            tc_mma_bf16(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          issued = true;
+          tc_commit(empty_bar(s));   // frees the stage once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));   // accumulator complete
+        if (++acc == 2) { acc = 0; aph ^= 1u; }
+      }
+      if (!ok) {
+        report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 2);
+        if (issued) {   // wait for MMAs in flight before shared and tensor memory are released
+          tc_commit(drain_bar);
+          const long long t0 = clock64();
+          while (!mbar_try(drain_bar, 0u) && clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps 2..5
+    const int q = warp & 3;                 // accumulator lane quarter this warp may read
+    const int row_in_tile = q * 32 + lane;
+    int acc = 0;
+    uint32_t aph = 0;
+    bool ok = true;
+    const bool c_vec = (p.c_ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.c) & 15u) == 0);
+    const bool cin_vec = (p.cin_ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.cin) & 15u) == 0);
+    for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+      int tm, tn;
+      tile_coords(p, t, tm, tn);
+      // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
+      const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
+      if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t gi = (int64_t)tm * BM + row_in_tile;
+      const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(taddr + (uint32_t)c0, r);
+        tc_wait_ld();
+        const int64_t gj = (int64_t)tn * BN + c0;
+        if (gi < p.M && gj < p.N) {
+          float v[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = p.alpha * __uint_as_float(r[i]);
+          const bool full = gj + 32 <= p.N;
+          if (p.beta != 0.f) {
+            if (p.cin_dtype == SP_F32) {
+              const float* src = reinterpret_cast<const float*>(p.cin) + gi * p.cin_ld + gj;
+              if (full && cin_vec) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                  const float4 x = *reinterpret_cast<const float4*>(src + i);
+                  v[i] += p.beta * x.x; v[i + 1] += p.beta * x.y; v[i + 2] += p.beta * x.z; v[i + 3] += p.beta * x.w;
+                }
+              } else {
+                for (int i = 0; i < 32; ++i) if (gj + i < p.N) v[i] += p.beta * src[i];
+              }
+            } else {
+              const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(p.cin) + gi * p.cin_ld + gj;
+              for (int i = 0; i < 32; ++i) if (gj + i < p.N) v[i] += p.beta * __bfloat162float(src[i]);
+            }
+          }
+          if (p.c_dtype == SP_F32) {
+            float* dst = reinterpret_cast<float*>(p.c) + gi * p.c_ld + gj;
+            if (full && c_vec) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            } else {
+              for (int i = 0; i < 32; ++i) if (gj + i < p.N) dst[i] = v[i];
+            }
+          } else {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.c) + gi * p.c_ld + gj;
+            if (full && (p.c_ld % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.c) & 15u) == 0)) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 8) {
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[i], v[i + 1]), h1 = __floats2bfloat162_rn(v[i + 2], v[i + 3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[i + 4], v[i + 5]), h3 = __floats2bfloat162_rn(v[i + 6], v[i + 7]);
+                uint4 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                *reinterpret_cast<uint4*>(dst + i) = pk;
+              }
+            } else {
+              for (int i = 0; i < 32; ++i) if (gj + i < p.N) dst[i] = __float2bfloat16_rn(v[i]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; aph ^= 1u; }
+    }
+    if (!ok && lane == 0) report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 3);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Tensor map of a bf16 operand.  stored matrix: [outer, inner] row-major with leading dimension ld.
+//   K-major : inner = K, outer = rows, box = {64, box_rows}
+//   MN-major: inner = rows, outer = K, box = {64, 64}
+bool make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+              int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+}  // namespace
+
+bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B) {
+  if (M <= 0 || N <= 0 || K <= 0) return false;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return false;
+  if ((reinterpret_cast<uintptr_t>(A.ptr) & 15u) || (reinterpret_cast<uintptr_t>(B.ptr) & 15u)) return false;
+  if (A.ld % 8 != 0 || B.ld % 8 != 0) return false;
+  if (A.ld < (A.kmajor ? K : M) || B.ld < (B.kmajor ? K : N)) return false;
+  return true;
+}
+
+sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
+                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream) {
+  if (!gemm_tc_supported(M, N, K, A, B)) return SP_ERR_UNSUPPORTED;
+  if (lower_only && M != N) return SP_ERR_SHAPE;
+  if (beta != 0.f && (Cin.ptr == nullptr || Cin.s1 != 1)) return SP_ERR_INVALID_ARG;
+  if (C.dtype != SP_F32 && C.dtype != SP_BF16) return SP_ERR_DTYPE;
+  if (beta != 0.f && Cin.dtype != SP_F32 && Cin.dtype != SP_BF16) return SP_ERR_DTYPE;
+
+  CUtensorMap tmA, tmB;
+  bool ok = A.kmajor ? make_map(&tmA, A.ptr, K, M, A.ld, BK, BM) : make_map(&tmA, A.ptr, M, K, A.ld, 64, BK);
+  ok = ok && (B.kmajor ? make_map(&tmB, B.ptr, K, N, B.ld, BK, BN) : make_map(&tmB, B.ptr, N, K, B.ld, 64, BK));
+  if (!ok) return SP_ERR_CUDA;
+
+  TcParams p;
+  p.M = M; p.N = N; p.K = K;
+  p.alpha = alpha; p.beta = beta;
+  p.cin = Cin.ptr; p.cin_dtype = Cin.dtype; p.cin_ld = Cin.s0;
+  p.c = C.ptr; p.c_dtype = C.dtype; p.c_ld = C.ld;
+  p.a_kmajor = A.kmajor ? 1 : 0;
+  p.b_kmajor = B.kmajor ? 1 : 0;
+  p.lower_only = lower_only ? 1 : 0;
+  p.tiles_m = (int32_t)ceil_div(M, BM);
+  p.tiles_n = (int32_t)ceil_div(N, BN);
+  if (lower_only) {
+    int64_t cnt = 0;
+    for (int tn = 0; tn < p.tiles_n; ++tn) {
+      const int first = tn * (BN / BM);
+      if (first < p.tiles_m) cnt += p.tiles_m - first;
+    }
+    p.num_tiles = (int32_t)cnt;
+  } else {
+    p.num_tiles = p.tiles_m * p.tiles_n;
+  }
+  p.status = status_dev;
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) !=
+        cudaSuccess)
+      return SP_ERR_CUDA;
+    attr_set = true;
+  }
+  int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
+  gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
+  return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
+}
+
+}  // namespace sp

@@ -1,0 +1,427 @@
+"""Parity of the CUDA library (called through its C ABI) against the CPU oracle, element by element.
+
+Every test feeds ONE seeded input to both sides.  Sizes are small enough for the oracle to finish in seconds but
+span several tiles of the kernels (128 x 256 tensor-core tiles, 64 / 128 CUDA-core tiles, 64-wide Cholesky panels)
+and ragged tails.  Integer / byte results (masks, kept counts, indices) are compared bit-exactly.
+"""
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import struprune_oracle as O
+from paper_2510_03246_b200 import api, synth
+from tests._util import TOL, bf16_half_ulp, np64, oracle_state_from_gpu, relerr
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _gauss(shape, seed, dtype=torch.float32, scale=1.0):
+    n = int(np.prod(shape))
+    x = synth.standard_variates(seed, 77, n, "gauss").view(*shape) * scale
+    return x.to(dtype)
+
+
+def _assert_status_clean(status):
+    assert status.cpu().tolist()[0] == 0, f"device status {status.cpu().tolist()}"
+
+
+# ------------------------------------------------------------------------------------------------ GEMM kernels
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("transA,transB", [(False, False), (False, True), (True, False), (True, True)])
+def test_gemm_cuda_core(dtype, transA, transB):
+    M, N, K = 197, 141, 83
+    A = _gauss((K, M) if transA else (M, K), 1, dtype).to(DEV)
+    B = _gauss((N, K) if transB else (K, N), 2, dtype).to(DEV)
+    Cm = _gauss((M, N), 3).to(DEV)
+    C0 = np64(Cm)
+    api.sp_gemm(A, B, Cm, transA, transB, alpha=0.7, beta=-1.3)
+    a = np64(A).T if transA else np64(A)
+    b = np64(B).T if transB else np64(B)
+    ref = 0.7 * a @ b - 1.3 * C0
+    assert relerr(np64(Cm), ref) < (1e-6 if dtype == torch.float32 else 2e-5)
+
+
+@pytest.mark.parametrize("a_kmajor,b_kmajor", [(True, True), (False, False), (True, False), (False, True)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (300, 520, 200), (1000, 264, 1100), (64, 72, 40)])
+def test_gemm_tensor_core(a_kmajor, b_kmajor, M, N, K):
+    # op(A) is M x K: stored [M,K] (K-major) or [K,M]; op(B) is K x N: stored [N,K] (K-major) or [K,N]
+    A = _gauss((M, K) if a_kmajor else (K, M), 4, torch.bfloat16).to(DEV)
+    B = _gauss((N, K) if b_kmajor else (K, N), 5, torch.bfloat16).to(DEV)
+    status = api.new_status()
+    for out_dtype, beta in ((torch.float32, 0.0), (torch.float32, 1.0), (torch.bfloat16, 1.0)):
+        Cm = _gauss((M, N), 6, out_dtype).to(DEV)
+        C0 = np64(Cm)
+        api.sp_gemm(A, B, Cm, transA=not a_kmajor, transB=b_kmajor, alpha=-1.0, beta=beta, use_tensor_cores=True,
+                    status=status)
+        torch.cuda.synchronize()
+        _assert_status_clean(status)
+        a = np64(A) if a_kmajor else np64(A).T
+        b = np64(B).T if b_kmajor else np64(B)
+        ref = -1.0 * a @ b + beta * C0
+        got = np64(Cm)
+        if out_dtype == torch.float32:
+            assert relerr(got, ref) < 2e-6
+        else:
+            assert np.all(np.abs(got - ref) <= 2e-6 * np.abs(ref).max() + bf16_half_ulp(ref) * 1.001)
+
+
+def test_gemm_tensor_core_lower_only_and_persistence():
+    # square Gram-type product with more tiles than SMs, lower triangle only
+    n, K = 2304, 520
+    A = _gauss((K, n), 7, torch.bfloat16).to(DEV)
+    G = torch.zeros(n, n, device=DEV)
+    G.fill_(-7.0)
+    status = api.new_status()
+    api.sp_gemm(A, A, G, transA=True, transB=False, lower_only=True, use_tensor_cores=True, status=status)
+    torch.cuda.synchronize()
+    _assert_status_clean(status)
+    ref = np64(A).T @ np64(A)
+    got = np64(G)
+    il = np.tril_indices(n)
+    assert np.abs(got[il] - ref[il]).max() / np.abs(ref).max() < 2e-6
+    # tiles strictly above the diagonal are not touched (here: last row-block vs first column-block is lower; the
+    # first row-block against the last column-block is upper)
+    assert np.all(got[:128, 512:] == -7.0)
+    api.sp_symmetrize(G)
+    assert relerr(np64(G), ref) < 2e-6
+
+
+def test_gemm_tensor_core_rejects_unaligned():
+    A = _gauss((64, 36), 8, torch.bfloat16).to(DEV)   # ld = 36 is not a multiple of 8
+    B = _gauss((72, 36), 9, torch.bfloat16).to(DEV)
+    Cm = torch.zeros(64, 72, device=DEV)
+    with pytest.raises(api.SpError) as e:
+        api.sp_gemm(A, B, Cm, transB=True, use_tensor_cores=True)
+    assert e.value.code == 9  # SP_ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------------------------------------ Gram accumulation
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T,Cc,Rr", [(333, 200, 72), (1500, 520, 264), (64, 8, 8)])
+def test_gram_accumulate(dtype, T, Cc, Rr):
+    X = _gauss((T, Cc), 10, dtype).to(DEV)
+    Y = _gauss((T, Rr), 11, dtype).to(DEV)
+    G = torch.zeros(Cc, Cc, device=DEV)
+    R = torch.zeros(Rr, Cc, device=DEV)
+    st = torch.zeros(Cc, 2, dtype=torch.float64, device=DEV)
+    status = api.new_status()
+    # two chunks with a ragged split
+    cut = (T * 5) // 8
+    api.sp_gram_accumulate(X[:cut], Y[:cut], G, R, st, status)
+    api.sp_gram_accumulate(X[cut:], Y[cut:], G, R, st, status)
+    api.sp_symmetrize(G)
+    torch.cuda.synchronize()
+    _assert_status_clean(status)
+    Go = np.zeros((Cc, Cc)); Ro = np.zeros((Rr, Cc)); so = np.zeros((Cc, 2))
+    O.gram_accumulate(Go, Ro, np64(X).T, np64(Y).T, so)
+    tol = 1e-6
+    assert relerr(np64(G), Go) < tol and relerr(np64(R), Ro) < tol
+    assert relerr(np64(st), so) < 1e-12
+
+
+def test_gram_accumulate_empty_and_errors():
+    X = torch.zeros(0, 16, device=DEV)
+    G = torch.ones(16, 16, device=DEV)
+    api.sp_gram_accumulate(X, None, G)
+    assert torch.all(G == 1.0)
+    X = torch.zeros(8, 16, device=DEV)
+    Y = torch.zeros(9, 4, device=DEV)
+    with pytest.raises(api.SpError) as e:
+        api.sp_gram_accumulate(X, Y, G, torch.zeros(4, 16, device=DEV))
+    assert e.value.code == 2
+
+
+# ------------------------------------------------------------------------------------------------ ridge solve
+@pytest.mark.parametrize("precise", [True, False])
+@pytest.mark.parametrize("m,n", [(50, 64), (130, 200), (9, 333)])
+def test_ridge_solve(precise, m, n):
+    A = _gauss((n, 2 * n + 5), 12).numpy().astype(np.float64)
+    A = np.maximum(A, 0)                                 # ReLU-like, strongly correlated columns
+    G = torch.tensor(A @ A.T, dtype=torch.float32)
+    R = _gauss((m, n), 13)
+    status = api.new_status()
+    W = api.sp_ridge_solve(R.to(DEV), G.to(DEV), 0.1, True, precise, status=status)
+    torch.cuda.synchronize()
+    _assert_status_clean(status)
+    Gd = np64(G)
+    ref = O.ridge_solve(np64(R), Gd, O.effective_ridge(Gd, 0.1, True))
+    assert relerr(np64(W), ref) < (1e-6 if precise else 5e-4)
+
+
+def test_ridge_solve_reports_indefinite():
+    n = 96
+    G = -torch.eye(n)
+    status = api.new_status()
+    api.sp_ridge_solve(torch.ones(4, n, device=DEV), G.to(DEV), 0.0, False, True, status=status)
+    torch.cuda.synchronize()
+    s = status.cpu().tolist()
+    assert s[0] == 6 and s[1] == 0      # SP_ERR_NOT_SPD at pivot 0
+
+
+@pytest.mark.parametrize("group", [1, 4])
+def test_linear_refit(group):
+    nu, m = 60, 37
+    n = nu * group
+    A = _gauss((n, 3 * n), 14).numpy().astype(np.float64)
+    G = torch.tensor(A @ A.T, dtype=torch.float32)
+    R = _gauss((m, n), 15)
+    mask_u = (synth.uniform_bits(5, 1, 0, nu) % 3 != 0).to(torch.uint8)
+    k = int(mask_u.sum())
+    W = api.sp_linear_refit(R.to(DEV), G.to(DEV), mask_u.to(DEV), k, 0.37, group=group, precise=True)
+    keep_cols = np.repeat(mask_u.numpy(), group)
+    ref = O.restricted_refit(np64(R), np64(G), keep_cols, 0.37)
+    assert relerr(np64(W), ref) < 1e-6
+    assert np.all(np64(W)[:, keep_cols == 0] == 0.0)
+
+
+# ------------------------------------------------------------------------------------------------ scores
+@pytest.mark.parametrize("group", [1, 8])
+def test_wanda_scores(group):
+    d, nu, N = 70, 96, 500
+    n = nu * group
+    W = _gauss((d, n), 16).to(DEV)
+    A = _gauss((N, n), 17)
+    colsq = (A.double() ** 2).sum(0).float().to(DEV)
+    colabs = A.double().abs().sum(0).to(DEV)
+    s2, i2, _ = api.sp_struct_scores(api.SP_SCORE_WANDA_L2, nu, group, W=W, colsq=colsq)
+    s1, i1, _ = api.sp_struct_scores(api.SP_SCORE_WANDA_L1, nu, group, W=W, colabs=colabs, inv_tokens=1.0 / N)
+    o2, oi2 = O.wanda_scores(np64(W), colsq=np64(colsq), kind="l2", group=group)
+    o1, oi1 = O.wanda_scores(np64(W), colabs_mean=np64(colabs) / N, kind="l1", group=group)
+    assert relerr(np64(s2), o2) < 1e-6 and relerr(np64(s1), o1) < 1e-6
+    assert abs(i2.item() - oi2) < 1e-6 * abs(oi2) and abs(i1.item() - oi1) < 1e-6 * abs(oi1)
+    # diagonal of a Gram matrix as the column energy (stride n + 1)
+    Gm = (A.double().T @ A.double()).float().to(DEV)
+    s2b, _, _ = api.sp_struct_scores(api.SP_SCORE_WANDA_L2, nu, group, W=W, colsq=Gm, colsq_stride=n + 1)
+    assert relerr(np64(s2b), o2) < 1e-6
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("group", [1, 4])
+def test_lemma1_scores_stream(dtype, group):
+    N, nu = 777, 50
+    n = nu * group
+    b, c, dd, t = (_gauss((N, n), 20 + i, dtype).to(DEV) for i in range(4))
+    s, imp, relaxed = api.sp_struct_scores(api.SP_SCORE_LEMMA1, nu, group, b=b, c=c, dd=dd, t=t, r_layer=0.4,
+                                           want_relaxed=True)
+    so, rl, e = O.lemma1_scores(np64(b).T, np64(c).T, np64(dd).T, np64(t).T, group)
+    assert relerr(np64(s), so) < 1e-6
+    assert abs(imp.item() - rl) < 1e-9 + 1e-6 * abs(rl)
+    Mo = O.relaxed_mask(so, e, 0.4)
+    assert relerr(np64(relaxed), Mo) < 1e-9
+    assert abs(np64(relaxed).sum() - 0.4 * nu) < 1e-9 * nu
+
+
+# ------------------------------------------------------------------------------------------------ allocation
+@pytest.mark.parametrize("mode,name", [(api.SP_ALLOC_SOFTMAX, "softmax"), (api.SP_ALLOC_INVERSE, "inverse"),
+                                       (api.SP_ALLOC_UNIFORM, "uniform")])
+@pytest.mark.parametrize("L", [1, 24, 64, 1000])
+def test_allocate_sparsity(mode, name, L):
+    u = synth.uniform_bits(9, 3, 0, L).double() / 2 ** 32
+    for spread, T in ((0.6, 1.0), (3.0, 0.2)):          # second case clips some layers at 0.95
+        I = (0.8 + spread * u)
+        nu = (1000 + (synth.uniform_bits(9, 4, 0, L) % 7000)).to(torch.int64)
+        r, k = api.sp_allocate_sparsity(I.to(DEV), nu.to(DEV), 0.5, T, mode)
+        ro, ko = O.allocate_sparsity(I.numpy(), nu.numpy(), 0.5, T, name)
+        assert np.abs(np64(r) - ro).max() < 1e-12
+        kg = k.cpu().numpy()
+        # kept counts are integers decided by floor(r n + 0.5): bit-exact unless r n sits within 1e-9 of a half
+        frac = ro * nu.numpy() + 0.5
+        safe = np.abs(frac - np.round(frac)) > 1e-9
+        assert np.array_equal(kg[safe], ko[safe])
+        assert np.all(np.abs(kg - ko) <= 1)
+
+
+# ------------------------------------------------------------------------------------------------ top-k + mask
+@pytest.mark.parametrize("n,k", [(1, 1), (17, 0), (17, 17), (1000, 1), (1000, 999), (3072, 1536), (28672, 5734),
+                                 (200000, 77777)])
+def test_apply_mask_topk(n, k):
+    s = _gauss((n,), 30 + n % 7)
+    s = torch.round(s * 50) / 50          # many exact ties
+    if n >= 1000:
+        s[5] = float("nan"); s[n - 3] = float("nan"); s[7] = float("-inf"); s[11] = float("inf"); s[13] = -0.0
+    mask, tau, idx = api.sp_apply_mask(s.to(DEV), k, want_index=True)
+    mo, tauo = O.topk_mask(s.numpy(), k)
+    assert np.array_equal(mask.cpu().numpy(), mo)
+    if 0 < k:
+        assert np.array_equal(idx.cpu().numpy(), np.flatnonzero(mo).astype(np.int32))
+        assert tau.item() == tauo or (np.isnan(tau.item()) and np.isnan(tauo))
+
+
+@pytest.mark.parametrize("group", [1, 64])
+def test_apply_mask_zeroes_pruned_units(group):
+    nu, k, other = 48, 20, 70
+    s = _gauss((nu,), 41)
+    W1 = _gauss((nu * group, other), 42).to(DEV)
+    W2 = _gauss((other, nu * group), 43).to(DEV)
+    W1o, W2o = np64(W1), np64(W2)
+    mask, _, _ = api.sp_apply_mask(s.to(DEV), k, group, W_rows=W1, W_cols=W2)
+    mo, _ = O.topk_mask(s.numpy(), k)
+    assert np.array_equal(mask.cpu().numpy(), mo)
+    r_, c_ = O.apply_mask(mo, group, W1o, W2o)
+    assert np.array_equal(np64(W1), r_) and np.array_equal(np64(W2), c_)
+
+
+def test_apply_mask_argument_errors():
+    s = torch.zeros(10, device=DEV)
+    with pytest.raises(api.SpError) as e:
+        api.sp_apply_mask(s, 11)
+    assert e.value.code == 2
+
+
+# ------------------------------------------------------------------------------------------------ module: init + step
+def _make_module(cfg, dual=False, chunk=0, seed_layer=0):
+    X = synth.make_activations(cfg, seed_layer)
+    W1, W2 = synth.make_weights(cfg, seed_layer)
+    mod = api.FfnModule(X.to(DEV), W1.to(DEV), W2.to(DEV), dual_mode=dual, token_chunk=chunk)
+    return mod, X, W1, W2
+
+
+SMALL_F32 = synth.scaled(synth.CONFIGS["C1"], d=96, n=328, tokens=600, sparsity=0.5)
+SMALL_BF16 = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=1300, sparsity=0.5, outlier_frac=0.02)
+
+
+@pytest.mark.parametrize("cfg,chunk", [(SMALL_F32, 0), (SMALL_F32, 256), (SMALL_BF16, 0), (SMALL_BF16, 512)])
+def test_ffn_init(cfg, chunk):
+    mod, X, W1, W2 = _make_module(cfg, chunk=chunk)
+    mod.sp_ffn_init()
+    torch.cuda.synchronize()
+    mod.check_status()
+    st, Y = O.ffn_init(np64(X).T, np64(W1), np64(W2))
+    tol = TOL[X.dtype]
+    assert relerr(np64(mod.Z).T, st.Z) < tol
+    if X.dtype == torch.bfloat16:   # Ypre is stored in bf16: arithmetic tolerance plus one rounding of the stored value
+        assert np.all(np.abs(np64(mod.Ypre).T - Y) <= tol * np.abs(Y).max() + bf16_half_ulp(Y) * 1.001)
+    else:
+        assert relerr(np64(mod.Ypre).T, Y) < tol
+    assert relerr(np64(mod.G_X), st.G_X) < tol and relerr(np64(mod.G_A), st.G_A) < tol
+    assert relerr(np64(mod.R1), st.R1) < tol and relerr(np64(mod.R2), st.R2) < tol
+    assert relerr(np64(mod.absA), st.absA) < tol
+
+
+def _step_and_compare(mod, X, W1_0, p_gpu, p_or, tol, audit):
+    """One teacher-forced step: the oracle restarts from the GPU's state before the call."""
+    st = oracle_state_from_gpu(mod)
+    Xo, Yo = np64(X).T, np64(mod.Ypre).T
+    N = Xo.shape[1]
+    mod.sp_admm_step(p_gpu)
+    torch.cuda.synchronize()
+    mod.check_status()
+    # scores: the oracle's own
+    st_s = copy.deepcopy(st)
+    p_s = copy.deepcopy(p_or)
+    s_or, I_or = O.admm_weight_phase(st_s, np64(W1_0), p_s, N)
+    s_gpu = np64(mod.scores)
+    assert relerr(s_gpu, s_or) < tol
+    assert abs(mod.importance.item() - I_or) < tol * abs(I_or)
+    # the integer decision is taken in the GPU's precision: mask == exact top-k of the GPU's scores
+    mask_gpu = mod.mask.cpu().numpy()
+    if p_gpu.reselect_mask:
+        m_ref, _ = O.topk_mask(mod.scores.cpu().numpy(), p_gpu.k_keep)
+        assert np.array_equal(mask_gpu, m_ref)
+        # audit against the oracle's own mask: disagreements only at units whose score is within tol of the threshold
+        diff = np.flatnonzero(mask_gpu != st_s.mask)
+        if diff.size:
+            tau = np.sort(s_or)[::-1][p_gpu.k_keep - 1]
+            assert np.all(np.abs(s_or[diff] - tau) <= tol * np.abs(s_or).max())
+        audit.append(diff.size)
+    assert mask_gpu.sum() == p_gpu.k_keep
+    # continue the oracle with the GPU's mask
+    st.mask = mask_gpu.copy()
+    p_t = copy.deepcopy(p_or)
+    p_t.reselect_mask = False
+    _, _, rep, A = O.admm_step(st, Xo, Yo, np64(W1_0), p_t)
+    assert relerr(np64(mod.W1), st.W1) < tol, "W1"
+    assert relerr(np64(mod.W2), st.W2) < tol, "W2"
+    assert np.all(np64(mod.W1)[mask_gpu == 0] == 0) and np.all(np64(mod.W2)[:, mask_gpu == 0] == 0)
+    assert relerr(np64(mod.Z).T, st.Z) < tol, "Z"
+    if p_gpu.dual_mode:
+        assert relerr(np64(mod.U).T, st.U) < tol, "U"
+    assert relerr(np64(mod.G_A), st.G_A) < tol, "G_A"
+    assert relerr(np64(mod.R1), st.R1) < tol, "R1"
+    assert relerr(np64(mod.R2), st.R2) < tol, "R2"
+    assert relerr(np64(mod.absA), st.absA) < tol, "absA"
+    rep_gpu = mod.read_report()
+    assert abs(rep_gpu["res_act"] - rep["res_act"]) <= 5 * tol * max(rep_gpu["a_sq"], 1e-30)
+    assert abs(rep_gpu["a_sq"] - (A * A).sum()) <= 5 * tol * (A * A).sum()
+    assert rep_gpu["kept"] == p_gpu.k_keep
+
+
+STEP_CASES = [
+    # cfg, chunk, score kind, z rule, dual, refit
+    (SMALL_F32, 0, "wanda_l2", "paper", False, True),
+    (SMALL_F32, 256, "wanda_l1", "exact", True, True),
+    (SMALL_F32, 0, "lemma1", "paper", False, False),
+    (SMALL_BF16, 0, "wanda_l2", "paper", False, True),
+    (SMALL_BF16, 512, "wanda_l1", "exact", True, True),
+    (SMALL_BF16, 512, "lemma1", "paper", False, False),
+]
+_KIND = {"wanda_l2": api.SP_SCORE_WANDA_L2, "wanda_l1": api.SP_SCORE_WANDA_L1, "lemma1": api.SP_SCORE_LEMMA1}
+_RULE = {"paper": api.SP_Z_PAPER, "exact": api.SP_Z_EXACT}
+
+
+@pytest.mark.parametrize("cfg,chunk,kind,rule,dual,refit", STEP_CASES)
+def test_admm_step_teacher_forced(cfg, chunk, kind, rule, dual, refit):
+    mod, X, W1, W2 = _make_module(cfg, dual=dual, chunk=chunk)
+    mod.sp_ffn_init()
+    k = cfg.k_keep
+    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=_RULE[rule], dual_mode=dual,
+                           score_kind=_KIND[kind], refit=refit, token_chunk=chunk)
+    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=rule, dual_mode=dual, score_kind=kind,
+                        refit=refit)
+    audit = []
+    for it in range(3):
+        _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
+
+
+def test_admm_step_fixed_mask():
+    cfg = SMALL_F32
+    mod, X, W1, W2 = _make_module(cfg)
+    mod.sp_ffn_init()
+    k = cfg.k_keep
+    p_gpu = api.AdmmParams(k_keep=k, rho=cfg.rho)
+    p_or = O.AdmmParams(k_keep=k, rho=cfg.rho)
+    audit = []
+    _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
+    mask1 = mod.mask.clone()
+    p_gpu.reselect_mask = False
+    p_or.reselect_mask = False
+    _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
+    assert torch.equal(mask1, mod.mask)
+
+
+def test_admm_step_argument_errors():
+    mod, X, W1, W2 = _make_module(SMALL_F32)
+    mod.sp_ffn_init()
+    with pytest.raises(api.SpError) as e:
+        mod.sp_admm_step(api.AdmmParams(k_keep=0))
+    assert e.value.code == 2
+    with pytest.raises(api.SpError) as e:
+        mod.sp_admm_step(api.AdmmParams(k_keep=10, alpha=-1.0))
+    assert e.value.code == 1
+    with pytest.raises(api.SpError) as e:
+        mod.sp_admm_step(api.AdmmParams(k_keep=10, dual_mode=True))      # no U buffer was allocated
+    assert e.value.code == 1
+
+
+def test_free_running_iterations_fp32():
+    """K iterations without teacher forcing on a reduced copy of the smallest config: the two trajectories stay
+    together (same masks up to near-ties, values within a loose bound that allows for chaotic amplification)."""
+    cfg = synth.scaled(synth.CONFIGS["C1"], d=128, n=512, tokens=1024)
+    mod, X, W1, W2 = _make_module(cfg)
+    mod.sp_ffn_init()
+    torch.cuda.synchronize()
+    st, Y = O.ffn_init(np64(X).T, np64(W1), np64(W2))
+    p_gpu = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho)
+    p_or = O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho)
+    for it in range(cfg.iters):
+        mod.sp_admm_step(p_gpu)
+        O.admm_step(st, np64(X).T, Y, np64(W1), p_or)
+    torch.cuda.synchronize()
+    mod.check_status()
+    agree = (mod.mask.cpu().numpy() == st.mask).mean()
+    assert agree > 0.99
+    if agree == 1.0:
+        assert relerr(np64(mod.W2), st.W2) < 1e-3 and relerr(np64(mod.Z).T, st.Z) < 1e-3
