@@ -110,6 +110,17 @@ def z_candidates(W1, X, A, alpha, beta, U=None):
     return z1, z2
 
 
+def z_exact_candidates(z1, z2, A, alpha, beta, U=None):
+    """Best point of each half line of the scalar problem beta (a - relu(z))^2 + alpha (z - z1)^2 and its value:
+    returns (zn, zp, fn, fp) with zn = min(z1, 0) on z <= 0 and zp = max(z2, 0) on z >= 0."""
+    Au = np.asarray(A, F64) + (0.0 if U is None else np.asarray(U, F64))
+    zn = np.minimum(z1, 0.0)
+    zp = np.maximum(z2, 0.0)
+    fn = beta * Au ** 2 + alpha * (zn - z1) ** 2
+    fp = beta * (Au - zp) ** 2 + alpha * (zp - z1) ** 2
+    return zn, zp, fn, fp
+
+
 def z_select(Zold, z1, z2, A, alpha, beta, rule="paper", U=None):
     """Elementwise select of the z-update."""
     Zold = np.asarray(Zold, F64)
@@ -118,11 +129,7 @@ def z_select(Zold, z1, z2, A, alpha, beta, rule="paper", U=None):
         return np.where(Zold < 0.0, z1, z2)
     if rule == "exact":
         # argmin_z beta (a - relu(z))^2 + alpha (z - z1)^2: best point of each half line, then compare.
-        Au = np.asarray(A, F64) + (0.0 if U is None else np.asarray(U, F64))
-        zn = np.minimum(z1, 0.0)
-        zp = np.maximum(z2, 0.0)
-        fn = beta * Au ** 2 + alpha * (zn - z1) ** 2
-        fp = beta * (Au - zp) ** 2 + alpha * (zp - z1) ** 2
+        zn, zp, fn, fp = z_exact_candidates(z1, z2, A, alpha, beta, U)
         return np.where(fn < fp, zn, zp)
     raise ValueError(rule)
 
@@ -321,9 +328,11 @@ def admm_weight_phase(st, W1_0, p, N):
     return s, I
 
 
-def admm_step(st, X, Ypre, W1_0, p):
+def admm_step(st, X, Ypre, W1_0, p, z_hook=None):
     """One outer step: weights from the accumulators, then a-, z- (and dual) updates, then the accumulators
-    of the new auxiliary variables.  Returns (scores, layer importance, report dict, A)."""
+    of the new auxiliary variables.  Returns (scores, layer importance, report dict, A).
+    z_hook(Znew, z1, z2, A, U) may replace Znew before it is used further; parity tests use it to adopt the other
+    side's choice where the two candidates of the exact rule tie within rounding."""
     X = np.asarray(X, F64)
     Ypre = np.asarray(Ypre, F64)
     N = X.shape[1]
@@ -332,6 +341,8 @@ def admm_step(st, X, Ypre, W1_0, p):
     A = a_update(st.W2, Ypre, st.Z, p.alpha, p.beta, U, p.act)
     z1, z2 = z_candidates(st.W1, X, A, p.alpha, p.beta, U)
     Znew = z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule, U)
+    if z_hook is not None:
+        Znew = z_hook(Znew, z1, z2, A, U)
     if p.dual_mode:
         st.U = dual_update(st.U, A, Znew, p.act)
     st.Z = Znew

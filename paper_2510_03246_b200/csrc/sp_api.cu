@@ -48,6 +48,24 @@ sp_status contract(int64_t M, int64_t N, int64_t K, double alpha, MatRef A, bool
   return SP_OK;
 }
 
+// C[M,N] = A W^T with fp32 weights W[N,K]: on the tensor cores W is split into bf16 hi + lo parts stored side by side
+// ([N, 2*kpad]) so that no weight bit beyond ~16 is lost; A (bf16, [M,K], ld) is read once per part.
+// Falls back to the CUDA-core kernel (fp32 W as is) when the tensor-core path's alignment rules do not hold.
+int64_t split_kpad(int64_t K) { return (K + 63) / 64 * 64; }
+
+sp_status contract_split_weights(int64_t M, int64_t N, int64_t K, MatRef A, const void* Wsplit, MatRef Wf32, MatRef C,
+                                 int32_t* status, cudaStream_t stream) {
+  if (M <= 0 || N <= 0) return SP_OK;
+  const int64_t kp = split_kpad(K);
+  TcOperand ta{A.ptr, A.ld, true}, tb{Wsplit, 2 * kp, true};
+  OutOperand out{const_cast<void*>(C.ptr), C.dtype, C.ld};
+  Operand cin{C.ptr, C.dtype, C.ld, 1};
+  if (Wsplit && A.dtype == SP_BF16 && gemm_tc_supported(M, N, K, ta, TcOperand{Wsplit, 2 * kp, true})) {
+    return gemm_tc(M, N, K + kp, 1.f, ta, tb, 0.f, cin, out, false, status, stream, kp, K);
+  }
+  return contract(M, N, K, 1.0, A, true, Wf32, true, 0.0, C, C, false, false, false, status, stream);
+}
+
 struct Carver {
   uint8_t* base;
   size_t off = 0;
@@ -149,7 +167,7 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.Qt = c.take<float>((size_t)n * d);
   p.T0 = c.take<float>((size_t)n * d);
   p.Cf = c.take<float>((size_t)d * d);
-  p.W1b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.W1b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // hi | lo split of W1
   p.W2b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
   p.Qtb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
   p.H = c.take_bytes((size_t)p.chunk * n * csz);
@@ -183,7 +201,7 @@ InitPlan plan_init(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.bf16 = cdt == SP_BF16;
   const size_t csz = p.bf16 ? 2 : 4;
   Carver c(ws);
-  p.W10b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.W10b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;  // hi | lo split of W1_0
   p.W20b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
   p.Ac = c.take_bytes((size_t)p.chunk * n * csz);
   p.Zb = p.bf16 ? c.take_bytes((size_t)p.chunk * n * csz) : nullptr;
@@ -276,12 +294,13 @@ sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream) {
 
 sp_status sp_gram_accumulate(const sp_mat* Xc, const sp_mat* Yc, float* G, int64_t ldg, float* R, int64_t ldr,
                              double* rowstats, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
-  if (!Xc || !Xc->ptr || !G) return SP_ERR_INVALID_ARG;
+  if (!Xc || !G) return SP_ERR_INVALID_ARG;
   if (!valid_act_dtype(Xc->dtype)) return SP_ERR_DTYPE;
   const int64_t T = Xc->rows, C = Xc->cols;
   if (T < 0 || C < 0 || Xc->ld < C || ldg < C) return SP_ERR_SHAPE;
+  if (!Xc->ptr && T * C > 0) return SP_ERR_INVALID_ARG;   // an empty chunk may carry a null pointer
   if (Yc) {
-    if (!Yc->ptr || !R) return SP_ERR_INVALID_ARG;
+    if ((!Yc->ptr && T * Yc->cols > 0) || !R) return SP_ERR_INVALID_ARG;
     if (Yc->dtype != Xc->dtype) return SP_ERR_DTYPE;
     if (Yc->rows != T || Yc->ld < Yc->cols || ldr < C) return SP_ERR_SHAPE;
   }
@@ -447,9 +466,8 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   const bool acc64 = !bf16;
   MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, w20{m->W2_0.ptr, SP_F32, m->W2_0.ld};
   if (bf16) {
-    CU(convert_matrix(m->W1_0.ptr, SP_F32, m->W1_0.ld, p.W10b, SP_BF16, d, n, d, s));
+    CU(split_bf16(reinterpret_cast<const float*>(m->W1_0.ptr), m->W1_0.ld, n, d, split_kpad(d), p.W10b, s));
     CU(convert_matrix(m->W2_0.ptr, SP_F32, m->W2_0.ld, p.W20b, SP_BF16, n, d, n, s));
-    w10 = MatRef{p.W10b, SP_BF16, d};
     w20 = MatRef{p.W20b, SP_BF16, n};
   }
   if (st->U) CU(cudaMemsetAsync(st->U, 0, (size_t)N * n * sizeof(float), s));
@@ -465,7 +483,8 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
     MatRef ac{p.Ac, cdt, n};
     MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : zc;
     // z^pre = X W1_0^T
-    SPCHK(contract(Tc, n, d, 1.0, xc, true, w10, true, 0.0, zc, zc, false, acc64, bf16, status_dev, s));
+    if (bf16) SPCHK(contract_split_weights(Tc, n, d, xc, p.W10b, w10, zc, status_dev, s));
+    else SPCHK(contract(Tc, n, d, 1.0, xc, true, w10, true, 0.0, zc, zc, false, acc64, false, status_dev, s));
     int rb;
     fused_update_grid(Tc, n, &rb);
     CU(launch_init_act(Zc, p.Ac, p.Zb, cdt, Tc, n, p.absA_part, rb, s));
@@ -491,6 +510,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   if (prm->dual_mode && !st->U) return SP_ERR_INVALID_ARG;
   const int64_t d = m->d, n = m->n, N = m->N;
   if (prm->k_keep < 1 || prm->k_keep > n) return SP_ERR_SHAPE;
+  if (prm->score_kind == SP_SCORE_LEMMA1 && m->W1_0.ld != d) return SP_ERR_SHAPE;
   if (!(prm->alpha > 0.0) || !(prm->beta > 0.0) || !(prm->rho >= 0.0) || prm->token_chunk < 0) return SP_ERR_INVALID_ARG;
   if (prm->z_rule != SP_Z_PAPER && prm->z_rule != SP_Z_EXACT) return SP_ERR_UNSUPPORTED;
   if (prm->score_kind < SP_SCORE_WANDA_L2 || prm->score_kind > SP_SCORE_LEMMA1) return SP_ERR_UNSUPPORTED;
@@ -521,7 +541,6 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     // b = W1~ X, c = d = t = z^pre = W1_0 X, written through G_X:  T0 = W1_0 G_X
     MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, gx{st->G_X, SP_F32, d}, t0{p.T0, SP_F32, d};
     SPCHK(contract(n, d, d, 1.0, w10, true, gx, false, 0.0, t0, t0, false, true, false, status_dev, s));
-    if (m->W1_0.ld != d) return SP_ERR_SHAPE;
     CU(lemma1_scores_gram(p.T0, p.W1t, reinterpret_cast<const float*>(m->W1_0.ptr), n, d, st->scores, st->importance,
                           p.score_scratch, s));
   } else {
@@ -546,9 +565,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   // ---- 5a. operands of the a-update: C = gamma I + W2 W2^T (d x d), Qt = W2^T C^-1 (n x d)
   MatRef w1{st->W1, SP_F32, d}, w2{st->W2, SP_F32, n}, qt{p.Qt, SP_F32, d};
   if (bf16) {
-    CU(convert_matrix(st->W1, SP_F32, d, p.W1b, SP_BF16, d, n, d, s));
+    CU(split_bf16(st->W1, d, n, d, split_kpad(d), p.W1b, s));
     CU(convert_matrix(st->W2, SP_F32, n, p.W2b, SP_BF16, n, d, n, s));
-    w1 = MatRef{p.W1b, SP_BF16, d};
     w2 = MatRef{p.W2b, SP_BF16, n};
   }
   {
@@ -595,7 +613,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     // E = Ypre - h W2^T ; D = E Qt^T ; z1 = X W1^T
     SPCHK(contract(Tc, d, n, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
     SPCHK(contract(Tc, n, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
-    SPCHK(contract(Tc, n, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, bf16, status_dev, s));
+    if (bf16) SPCHK(contract_split_weights(Tc, n, d, xc, p.W1b, w1, z1, status_dev, s));
+    else SPCHK(contract(Tc, n, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, false, status_dev, s));
     UpdateArgs ua;
     ua.Z = Zc; ua.U = Uc; ua.z1 = p.z1; ua.D = p.D; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
     ua.out_dtype = cdt; ua.T = Tc; ua.n = n; ua.alpha = (float)prm->alpha; ua.beta = (float)prm->beta;

@@ -51,8 +51,11 @@ struct TcOperand {
   int64_t ld;       // elements between consecutive rows of the stored matrix
   bool kmajor;
 };
+// a_kwrap > 0 (a multiple of 64): A holds only a_kext <= a_kwrap K indices (zero beyond) and is read again for the
+// K range [a_kwrap, K), so that B may hold two K segments (hi and lo parts of split weights) against the same A.
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
-                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream);
+                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, int64_t a_kwrap = 0,
+                  int64_t a_kext = 0);
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B);
 
 // Dense symmetric positive definite solve in precision T (float or double), all on `stream`.
@@ -73,6 +76,10 @@ constexpr int kCholNB = 64;
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
                            int64_t rows, int64_t cols, cudaStream_t stream);
 cudaError_t symmetrize_lower(float* G, int64_t n, int64_t ld, cudaStream_t stream);
+// dst[i, 0:cols] = bf16(src[i,:]) and dst[i, kpad:kpad+cols] = bf16(src - hi); padding columns are zero.
+// dst is [rows, 2*kpad] bf16.
+cudaError_t split_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad, void* dst,
+                       cudaStream_t stream);
 // dst[j, i] = (TD) src[i, j]
 template <typename TD>
 cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64_t cols, TD* dst, int64_t ldd,

@@ -44,6 +44,8 @@ struct TcParams {
   int32_t c_dtype;
   int64_t c_ld;
   int32_t a_kmajor, b_kmajor, lower_only;
+  int32_t a_kwrap;   // > 0: the A operand's K coordinate wraps at this multiple of BK (A is read again for a
+                     // second K segment of B, used for hi/lo-split bf16 weights)
   int32_t tiles_m, tiles_n, num_tiles;
   int32_t* status;
 };
@@ -225,11 +227,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t a_dst = tiles + s * STAGE_BYTES;
           const uint32_t b_dst = a_dst + A_BYTES;
           const int k0 = kb * BK;
+          const int ka = (p.a_kwrap > 0 && k0 >= p.a_kwrap) ? k0 - p.a_kwrap : k0;
           if (p.a_kmajor) {
-            tma_load_2d(a_dst, &tmA, k0, tm * BM, full_bar(s));
+            tma_load_2d(a_dst, &tmA, ka, tm * BM, full_bar(s));
           } else {
 #pragma unroll
-            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, tm * BM + mb * 64, k0, full_bar(s));
+            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, tm * BM + mb * 64, ka, full_bar(s));
           }
           if (p.b_kmajor) {
             tma_load_2d(b_dst, &tmB, k0, tn * BN, full_bar(s));
@@ -443,15 +446,19 @@ bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B
 }
 
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
-                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream) {
-  if (!gemm_tc_supported(M, N, K, A, B)) return SP_ERR_UNSUPPORTED;
+                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, int64_t a_kwrap,
+                  int64_t a_kext) {
+  if (a_kwrap < 0 || a_kwrap % BK != 0 || (a_kwrap > 0 && (K > 2 * a_kwrap || a_kext < 1 || a_kext > a_kwrap)))
+    return SP_ERR_INVALID_ARG;
+  const int64_t Ka = a_kwrap > 0 ? a_kext : K;   // extent of A along K
+  if (!gemm_tc_supported(M, N, Ka, A, B) || (B.kmajor && B.ld < K)) return SP_ERR_UNSUPPORTED;
   if (lower_only && M != N) return SP_ERR_SHAPE;
   if (beta != 0.f && (Cin.ptr == nullptr || Cin.s1 != 1)) return SP_ERR_INVALID_ARG;
   if (C.dtype != SP_F32 && C.dtype != SP_BF16) return SP_ERR_DTYPE;
   if (beta != 0.f && Cin.dtype != SP_F32 && Cin.dtype != SP_BF16) return SP_ERR_DTYPE;
 
   CUtensorMap tmA, tmB;
-  bool ok = A.kmajor ? make_map(&tmA, A.ptr, K, M, A.ld, BK, BM) : make_map(&tmA, A.ptr, M, K, A.ld, 64, BK);
+  bool ok = A.kmajor ? make_map(&tmA, A.ptr, Ka, M, A.ld, BK, BM) : make_map(&tmA, A.ptr, M, Ka, A.ld, 64, BK);
   ok = ok && (B.kmajor ? make_map(&tmB, B.ptr, K, N, B.ld, BK, BN) : make_map(&tmB, B.ptr, N, K, B.ld, 64, BK));
   if (!ok) return SP_ERR_CUDA;
 
@@ -463,6 +470,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   p.a_kmajor = A.kmajor ? 1 : 0;
   p.b_kmajor = B.kmajor ? 1 : 0;
   p.lower_only = lower_only ? 1 : 0;
+  p.a_kwrap = (int32_t)a_kwrap;
   p.tiles_m = (int32_t)ceil_div(M, BM);
   p.tiles_n = (int32_t)ceil_div(N, BN);
   if (lower_only) {

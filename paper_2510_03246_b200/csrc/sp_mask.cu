@@ -226,10 +226,11 @@ __global__ void __launch_bounds__(1024) allocate_kernel(const double* I, const i
 }
 
 // ------------------------------------------------------------------------------------------------ top-k
-// Order-preserving key: larger float -> larger key; NaN is treated as -infinity.
+// Order-preserving key: larger float -> larger key; NaN is treated as -infinity, -0 as +0.
 __device__ __forceinline__ uint32_t score_key(float v) {
   if (v != v) v = -INFINITY;
-  const uint32_t b = __float_as_uint(v);
+  uint32_t b = __float_as_uint(v);
+  if ((b & 0x7fffffffu) == 0u) b = 0u;   // -0 and +0 are the same score
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
