@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the per-module ADMM path (STRUPRUNE hot path) on B200.
+
+A step = one pass of the whole hot path over one FFN module: sp_admm_step (weight recovery by Cholesky solves, unit
+scores, top-k mask, recovery on the kept support, a-/z-(dual-)updates and Gram / cross-product accumulation over all
+calibration tokens) followed by sp_allocate_sparsity over the model's layer importances.
+
+Workload at N = 1 GPU: config C2 of the task (OPT-1.3B-shaped FFN module: d = 2048, n = 8192, 128 x 2048 = 262144
+calibration tokens in bf16, 50 % channel sparsity), synthetic seeded inputs generated on the device.
+With N > 1 GPUs every rank owns its own module (modules are independent once the kept counts are fixed), so the
+scaling is weak and the data path has no collective.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (a deliberately plain fp64
+restatement of the paper; context only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "ADMM iterations/sec per module"
+UNIT = "iterations/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C2")
+    ap.add_argument("--tokens", type=int, default=0, help="override the token count (profiling on a small case)")
+    ap.add_argument("--chunk", type=int, default=16384)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------ reference arm
+def oracle_iteration_seconds(cfg, sample_tokens: int, repeats: int = 1):
+    """Times one oracle ADMM iteration at the config's d and n on `sample_tokens` tokens.  Returns the seconds of the
+    token-independent weight phase and of the token-dependent phase (a-, z-update, accumulators)."""
+    import numpy as np
+    from oracle import struprune_oracle as O
+    from paper_2510_03246_b200 import synth
+
+    X = synth.make_activations(cfg, tokens=sample_tokens).double().numpy().T.copy()
+    W1, W2 = synth.make_weights(cfg)
+    W1 = W1.double().numpy(); W2 = W2.double().numpy()
+    st, Y = O.ffn_init(X, W1, W2)
+    p = O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho)
+    tw = tt = 0.0
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.admm_weight_phase(st, W1, p, X.shape[1])
+        t1 = time.perf_counter()
+        A = O.a_update(st.W2, Y, st.Z, p.alpha, p.beta)
+        z1, z2 = O.z_candidates(st.W1, X, A, p.alpha, p.beta)
+        st.Z = O.z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule)
+        st.G_A = A @ A.T; st.R1 = st.Z @ X.T; st.R2 = Y @ A.T; st.absA = np.abs(A).sum(axis=1)
+        O.allocate_sparsity(np.linspace(1.0, 1.5, cfg.layers), [cfg.n] * cfg.layers, cfg.sparsity, 1.25)
+        t2 = time.perf_counter()
+        tw += t1 - t0
+        tt += t2 - t1
+    return tw / repeats, tt / repeats
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [d.get("num_threads", 0) for d in threadpool_info()]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def cpu_baseline(cfg, sample_tokens: int) -> dict:
+    tw, tt = oracle_iteration_seconds(cfg, sample_tokens)
+    full = tw + tt * (cfg.tokens / sample_tokens)
+    return {"value": 1.0 / full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "sample": (f"one oracle iteration at d={cfg.d}, n={cfg.n} on {sample_tokens} of {cfg.tokens} tokens "
+                       f"({tw + tt:.1f} s measured: weight phase {tw:.1f} s + token phase {tt:.1f} s); the token "
+                       f"phase is scaled x{cfg.tokens // sample_tokens} to the full token count (extrapolated)")}
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    for _ in range(min(args.warmup, 1)):
+        oracle_iteration_seconds(cfg, args.cpu_sample_tokens)
+    t0 = time.perf_counter()
+    tws = tts = 0.0
+    steps = max(1, args.steps)
+    for _ in range(steps):
+        tw, tt = oracle_iteration_seconds(cfg, args.cpu_sample_tokens)
+        tws += tw; tts += tt
+    tw, tt = tws / steps, tts / steps
+    full = tw + tt * (cfg.tokens / args.cpu_sample_tokens)
+    value = 1.0 / full
+    sample = (f"each step: one oracle iteration at d={cfg.d}, n={cfg.n} on {args.cpu_sample_tokens} of {cfg.tokens} "
+              f"tokens; token phase scaled x{cfg.tokens // args.cpu_sample_tokens} (extrapolated)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": 1e3 * full, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(cfg)},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "wall_s": time.perf_counter() - t0}
+    print(json.dumps(line))
+
+
+def workload_name(cfg) -> str:
+    return (f"{cfg.name}: OPT-1.3B-shaped FFN module, d={cfg.d}, n={cfg.n}, N={cfg.tokens} tokens, "
+            f"{cfg.storage} activations, {int(cfg.sparsity * 100)}% channel sparsity (k_keep={cfg.k_keep})")
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+def main():
+    args = parse()
+    from paper_2510_03246_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    if args.tokens:
+        cfg = synth.scaled(cfg, tokens=args.tokens)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_03246_b200 import api, parallel
+
+    rank, local_rank, world = parallel.env_world()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    api.lib()
+
+    # ---- inputs resident in HBM: this rank's module (layer index = rank)
+    layer = rank
+    X = synth.make_activations(cfg, layer, device=dev)
+    W1_0, W2_0 = synth.make_weights(cfg, layer, device=dev)
+    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=args.chunk)
+    I_all = synth.make_importances(cfg, device=dev)
+    n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
+    T_soft = float(I_all.abs().mean())
+    mod.sp_ffn_init()
+    torch.cuda.synchronize()
+    mod.check_status()
+    prm = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk)
+
+    def step():
+        mod.sp_admm_step(prm)
+        # layer importances -> per-layer kept counts (this module's own importance replaces its slot)
+        I_all[layer:layer + 1].copy_(mod.importance)
+        api.sp_allocate_sparsity(I_all, n_units, cfg.sparsity, T_soft)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    mod.check_status()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    api.sp_profile_begin(True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    ms_local = ev0.elapsed_time(ev1)
+    launches = api.sp_launch_count()
+    prof = api.sp_profile_read()
+    api.sp_profile_begin(False)
+    mod.check_status()
+    ms = parallel.max_over_ranks(ms_local, dev)
+    value = world * args.steps / (ms * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the tcgen05 GEMM), from CUDA events recorded around each launch
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    tc = prof["gemm_tc"]
+    peak_tf = peaks.get("bf16_tflops_sustained", 1400.0)
+    peak_src = "measured (sustained, MEASURED_PEAKS.json)" if peaks else "fallback (1.4 PFLOP/s sustained)"
+    achieved = tc["flops"] / (tc["ms"] * 1e-3) / 1e12 if tc["ms"] > 0 else 0.0
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None, "peak_source": peak_src,
+                "launches": tc["records"], "avg_launch_ms": tc["ms"] / max(tc["records"], 1),
+                "algorithmic_flops_per_launch": tc["flops"] / max(tc["records"], 1)}
+    hbm = peaks.get("hbm_gbs", 6650.0)
+    fu = prof["fused_update"]
+    breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / args.steps,
+                     **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),
+                     **({"gbs": v["bytes"] / (v["ms"] * 1e-3) / 1e9, "hbm_frac": v["bytes"] / (v["ms"] * 1e-3) / 1e9 / hbm}
+                        if v["bytes"] and v["ms"] else {})}
+                 for k, v in prof.items() if v["records"]}
+
+    # ---- end to end: host buffers in, host results out, one whole module job of cfg.iters iterations
+    e2e = None
+    if not args.no_e2e:
+        del mod
+        torch.cuda.empty_cache()
+        hX = X.cpu().pin_memory(); hW1 = W1_0.cpu().pin_memory(); hW2 = W2_0.cpu().pin_memory()
+        del X, W1_0, W2_0
+        torch.cuda.empty_cache()
+        iters = cfg.iters
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
+        m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk)
+        m2.sp_ffn_init()
+        for _ in range(iters):
+            m2.sp_admm_step(prm)
+        oW1 = m2.W1.cpu(); oW2 = m2.W2.cpu(); omask = m2.mask.cpu()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        m2.check_status()
+        h2d = hX.numel() * hX.element_size() + hW1.numel() * hW1.element_size() + hW2.numel() * hW2.element_size()
+        d2h = oW1.numel() * 4 + oW2.numel() * 4 + omask.numel()
+        e2e = {"value": iters / (t1 - t0), "unit": UNIT, "h2d_bytes_per_step": h2d / iters,
+               "d2h_bytes_per_step": d2h / iters, "iterations": iters,
+               "note": "one module job: pinned-host X, W1_0, W2_0 in; init + iterations; W1, W2, mask back to host"}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        cpu = cpu_baseline(cfg, args.cpu_sample_tokens)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "token_chunk": args.chunk,
+                       "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
+                       "parallelism": f"modules x{world} (independent, no collective)"},
+            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "breakdown": breakdown}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

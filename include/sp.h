@@ -230,6 +230,20 @@ sp_status sp_gemm(int32_t transA, int32_t transB, int64_t M, int64_t N, int64_t 
                   int32_t* status_dev, void* stream);
 sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------------
+ * Launch accounting and profiling (the paper has no counterpart; used by the benchmark).
+ * sp_profile_begin(enable): resets the launch counter and the event records; enable != 0 brackets every kernel (or
+ *   phase) the library launches afterwards with a CUDA event pair on the launching stream.
+ * sp_profile_read(out_host): after the caller synchronised the stream(s): out_host[kind*4 + {0,1,2,3}] =
+ *   {records, total milliseconds, algorithmic flops, algorithmic bytes} for kind in [0, sp_profile_kinds()).
+ * sp_launch_count(): kernels launched by the library since the last sp_profile_begin.
+ */
+sp_status sp_profile_begin(int32_t enable);
+sp_status sp_profile_read(double* out_host);
+int32_t sp_profile_kinds(void);
+const char* sp_profile_kind_name(int32_t kind);
+int64_t sp_launch_count(void);
+
 /* Bytes of workspace the named call needs.  Meaning of (d, n, N, token_chunk, dtype) per op:
  *   SP_WS_GRAM: d = channels C, N = tokens T.   SP_WS_ADMM_STEP / SP_WS_FFN_INIT: module sizes, dtype of X.
  *   SP_WS_SCORES: d = n_units*group, N = tokens (LEMMA1) or rows of W (WANDA).

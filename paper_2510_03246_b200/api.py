@@ -26,7 +26,8 @@ SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
 
 EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
            "sp_apply_mask", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes",
-           "sp_status_string", "sp_version"]
+           "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
+           "sp_profile_kind_name", "sp_launch_count"]
 
 
 class SpError(RuntimeError):
@@ -93,8 +94,15 @@ def lib() -> C.CDLL:
         L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, vp, i64, vp, vp, sz, vp]
         L.sp_gemm.argtypes = [i32, i32, i64, i64, i64, dbl, pm, pm, dbl, pm, i32, i32, vp, vp]
         L.sp_symmetrize.argtypes = [vp, i64, i64, vp]
+        L.sp_profile_begin.argtypes = [i32]
+        L.sp_profile_read.argtypes = [vp]
+        L.sp_profile_kinds.restype = i32
+        L.sp_profile_kind_name.restype = C.c_char_p
+        L.sp_profile_kind_name.argtypes = [i32]
+        L.sp_launch_count.restype = i64
         for name in EXPORTS:
-            if name not in ("sp_workspace_bytes", "sp_status_string", "sp_version"):
+            if name not in ("sp_workspace_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
+                            "sp_profile_kind_name", "sp_launch_count"):
                 getattr(L, name).restype = C.c_int32
         _lib = L
     return _lib
@@ -145,6 +153,27 @@ def _ws(nbytes: int, device) -> torch.Tensor:
 
 def new_status(device="cuda") -> torch.Tensor:
     return torch.zeros(4, dtype=torch.int32, device=device)
+
+
+def sp_profile_begin(enable: bool = True):
+    _check(lib().sp_profile_begin(int(enable)), "sp_profile_begin")
+
+
+def sp_profile_read() -> dict:
+    """Per kernel kind: records, total ms, algorithmic flops and bytes (call after synchronising the stream)."""
+    L = lib()
+    nk = L.sp_profile_kinds()
+    buf = (C.c_double * (nk * 4))()
+    _check(L.sp_profile_read(buf), "sp_profile_read")
+    out = {}
+    for k in range(nk):
+        name = L.sp_profile_kind_name(k).decode()
+        out[name] = dict(records=int(buf[k * 4]), ms=buf[k * 4 + 1], flops=buf[k * 4 + 2], bytes=buf[k * 4 + 3])
+    return out
+
+
+def sp_launch_count() -> int:
+    return int(lib().sp_launch_count())
 
 
 # ---------------------------------------------------------------------------------------------- direct calls

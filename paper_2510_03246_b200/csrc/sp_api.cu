@@ -112,6 +112,7 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
                      const int32_t* idx, int64_t k, const double* rho_dev, float* W, int64_t ldw, SolveBufs& b,
                      int32_t* status, cudaStream_t stream) {
   const int64_t nn = idx ? k : n_full;
+  ProfScope prof(PK_SOLVE, (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
   T* Gs = reinterpret_cast<T*>(b.Gs);
   T* dinv = reinterpret_cast<T*>(b.dinv);
   T* Rs = reinterpret_cast<T*>(b.Rs);
@@ -354,6 +355,7 @@ sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t l
   CU(mask_to_index(mask, n_units, unit_idx, s));
   const int64_t k = k_keep * group;
   if (k > 0) {
+    count_launch();
     expand_group_index_kernel<<<(unsigned)ceil_div(k, 256), 256, 0, s>>>(unit_idx, k_keep, group, b.idx);
     CU(cudaGetLastError());
   }
@@ -573,6 +575,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     MatRef cf{p.Cf, SP_F32, d};
     SPCHK(contract(d, d, n, 1.0, w2, true, w2, true, 0.0, cf, cf, true, acc64, bf16, status_dev, s));
     CU(effective_ridge(nullptr, 0, 1, prm->beta / prm->alpha, 0, gam, s));
+    ProfScope prof(PK_SOLVE, (double)d * d * d / 3.0 + 2.0 * (double)n * d * d, 0.0, s);
     if (bf16) {
       float* Gs = reinterpret_cast<float*>(p.sb.Gs);
       float* Rs = reinterpret_cast<float*>(p.sb.Rs);

@@ -18,6 +18,21 @@ __device__ __forceinline__ void report_status(int32_t* status, int32_t code, int
   }
 }
 
+// ---- launch accounting and CUDA-event profiling (sp_profile.cu) ---------------------------------------------------
+enum ProfKind : int {
+  PK_GEMM_TC = 0, PK_GEMM_SIMT = 1, PK_SOLVE = 2, PK_FUSED_UPDATE = 3, PK_PREP_H = 4, PK_SCORES = 5, PK_TOPK = 6,
+  PK_ELEMENTWISE = 7, PK_ALLOCATE = 8, PK_COUNT = 9
+};
+void count_launch(int n = 1);
+// Brackets the kernels launched during its lifetime with a CUDA event pair on `stream` when profiling is enabled.
+// Scopes nest: only the outermost one records, so a phase scope absorbs the kernels launched inside it.
+struct ProfScope {
+  ProfScope(int kind, double flops, double bytes, cudaStream_t stream);
+  ~ProfScope();
+  int slot;
+  cudaStream_t stream;
+};
+
 __host__ __device__ __forceinline__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 __host__ __device__ __forceinline__ size_t align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
 

@@ -405,6 +405,8 @@ inline int grid_for(int64_t total, int threads, int per_thread = 1) {
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
                            int64_t rows, int64_t cols, cudaStream_t stream) {
   if (rows * cols == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   convert_kernel<<<grid_for(rows * cols, 256), 256, 0, stream>>>(src, sdt, lds, dst, ddt, ldd, rows, cols);
   return cudaGetLastError();
 }
@@ -414,6 +416,8 @@ cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64
                               cudaStream_t stream) {
   if (rows * cols == 0) return cudaSuccess;
   dim3 grid((unsigned)ceil_div(cols, 32), (unsigned)ceil_div(rows, 32));
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   transpose_convert_kernel<TD><<<grid, dim3(32, 8), 0, stream>>>(src, lds, rows, cols, dst, ldd);
   return cudaGetLastError();
 }
@@ -426,6 +430,8 @@ template cudaError_t transpose_convert<__nv_bfloat16>(const float*, int64_t, int
 cudaError_t split_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad, void* dst,
                        cudaStream_t stream) {
   if (rows * kpad == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   split_bf16_kernel<<<grid_for(rows * kpad, 256), 256, 0, stream>>>(src, lds, rows, cols, kpad,
                                                                      reinterpret_cast<__nv_bfloat16*>(dst));
   return cudaGetLastError();
@@ -434,6 +440,8 @@ cudaError_t split_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols
 cudaError_t symmetrize_lower(float* G, int64_t n, int64_t ld, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
   const unsigned nb = (unsigned)ceil_div(n, 32);
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   symmetrize_kernel<<<dim3(nb, nb), dim3(32, 8), 0, stream>>>(G, n, ld);
   return cudaGetLastError();
 }
@@ -442,6 +450,8 @@ template <typename T>
 cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_dev, T* dst, int64_t ldd,
                      cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   load_spd_kernel<T><<<grid_for(n * n, 256), 256, 0, stream>>>(G, ldg, nullptr, n, rho_dev, dst, ldd);
   return cudaGetLastError();
 }
@@ -449,6 +459,8 @@ template <typename T>
 cudaError_t load_spd_gather(const float* G, int64_t ldg, const int32_t* idx, int64_t k, const double* rho_dev, T* dst,
                             int64_t ldd, cudaStream_t stream) {
   if (k == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   load_spd_kernel<T><<<grid_for(k * k, 256), 256, 0, stream>>>(G, ldg, idx, k, rho_dev, dst, ldd);
   return cudaGetLastError();
 }
@@ -456,6 +468,8 @@ template <typename T>
 cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
                         int64_t ldd, cudaStream_t stream) {
   if (rows * k == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   gather_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
   return cudaGetLastError();
 }
@@ -463,8 +477,13 @@ template <typename T>
 cudaError_t scatter_cols(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, int64_t n,
                          float* dst, int64_t ldd, cudaStream_t stream) {
   if (rows * n == 0) return cudaSuccess;
-  if (idx) fill_zero_kernel<<<grid_for(rows * n, 256), 256, 0, stream>>>(dst, ldd, rows, n);
+  if (idx) {
+    ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+    count_launch();
+    fill_zero_kernel<<<grid_for(rows * n, 256), 256, 0, stream>>>(dst, ldd, rows, n);
+  }
   if (rows * k == 0) return cudaGetLastError();
+  count_launch();
   scatter_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
   return cudaGetLastError();
 }
@@ -482,6 +501,8 @@ SP_INST(double)
 
 cudaError_t effective_ridge(const float* G, int64_t ldg, int64_t n, double rho, int rel, double* rho_out,
                             cudaStream_t stream) {
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   effective_ridge_kernel<<<1, 1024, 0, stream>>>(G, ldg, n, rho, rel, rho_out);
   return cudaGetLastError();
 }
@@ -490,6 +511,8 @@ cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, 
                           cudaStream_t stream) {
   const int64_t total = T * n;
   if (total == 0) return cudaSuccess;
+  ProfScope prof(PK_PREP_H, 0.0, (double)total * ((U ? 8.0 : 4.0) + (hdt == SP_BF16 ? 2.0 : 4.0)), stream);
+  count_launch();
   prep_h_kernel<<<grid_for(total, 256, 4), 256, 0, stream>>>(Z, U, H, hdt, total);
   return cudaGetLastError();
 }
@@ -507,6 +530,11 @@ int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   if (a.T * a.n == 0) return cudaSuccess;
   dim3 grid((unsigned)ceil_div(a.n, 1024), (unsigned)a.row_blocks);
+  // algorithmic bytes per element: read Z, z1, D (+U); write Z (+U), A and the storage copy of Z
+  const double esz = a.out_dtype == SP_BF16 ? 2.0 : 4.0;
+  const double per = 12.0 + 4.0 + (a.U ? 8.0 : 0.0) + esz + (a.Zb_out ? esz : 0.0);
+  ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * (double)a.n * per, stream);
+  count_launch();
   fused_update_kernel<<<grid, 256, 0, stream>>>(a);
   return cudaGetLastError();
 }
@@ -515,6 +543,8 @@ cudaError_t launch_init_act(const float* Z, void* A_out, void* Zb_out, int32_t o
                             double* absA_part, int32_t row_blocks, cudaStream_t stream) {
   if (T * n == 0) return cudaSuccess;
   dim3 grid((unsigned)ceil_div(n, 1024), (unsigned)row_blocks);
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   init_act_kernel<<<grid, 256, 0, stream>>>(Z, A_out, Zb_out, out_dtype, T, n, absA_part, row_blocks);
   return cudaGetLastError();
 }
@@ -522,18 +552,23 @@ cudaError_t launch_init_act(const float* Z, void* A_out, void* Zb_out, int32_t o
 cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
                                 cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   reduce_col_partials_kernel<<<grid_for(n, 256), 256, 0, stream>>>(part, row_blocks, n, out, accumulate ? 1 : 0);
   return cudaGetLastError();
 }
 
 cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate,
                           cudaStream_t stream) {
+  count_launch();
   reduce_report_kernel<<<1, 256, 0, stream>>>(partial, nblocks, rep, accumulate ? 1 : 0);
   return cudaGetLastError();
 }
 
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
                         cudaStream_t stream) {
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   init_report_kernel<<<1, 1, 0, stream>>>(rep, rho1, rho2, kept);
   return cudaGetLastError();
 }
@@ -543,7 +578,10 @@ cudaError_t column_stats(const void* X, int32_t dt, int64_t ld, int64_t T, int64
   if (T * C == 0) return cudaSuccess;
   const int rb = column_stats_row_blocks(T, C);
   dim3 grid((unsigned)ceil_div(C, 256), (unsigned)rb);
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   column_stats_kernel<<<grid, 256, 0, stream>>>(X, dt, ld, T, C, scratch, rb);
+  count_launch();
   column_stats_reduce_kernel<<<(unsigned)ceil_div(C, 256), 256, 0, stream>>>(scratch, rb, C, rowstats);
   return cudaGetLastError();
 }

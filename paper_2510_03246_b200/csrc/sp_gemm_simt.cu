@@ -128,6 +128,8 @@ gemm_simt_kernel(int64_t M, int64_t N, int64_t K, Acc alpha, Operand A, Operand 
 cudaError_t gemm_simt(int64_t M, int64_t N, int64_t K, double alpha, Operand A, Operand B, double beta, Operand Cin,
                       OutOperand C, bool lower_only, bool acc64, cudaStream_t stream) {
   if (M <= 0 || N <= 0) return cudaSuccess;
+  count_launch();
+  ProfScope prof(PK_GEMM_SIMT, (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K, 0.0, stream);
   if (acc64) {
     constexpr int BM = 64, BN = 64;
     dim3 grid((unsigned)ceil_div(N, BN), (unsigned)ceil_div(M, BM));

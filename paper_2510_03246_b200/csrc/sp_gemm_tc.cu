@@ -492,6 +492,9 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
       return SP_ERR_CUDA;
     attr_set = true;
   }
+  count_launch();
+  const double k_alg = (double)(a_kwrap > 0 ? a_kext : K);   // the lo pass of split weights is not algorithmic work
+  ProfScope prof(PK_GEMM_TC, (lower_only ? 1.0 : 2.0) * (double)M * (double)N * k_alg, 0.0, stream);
   int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
   gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;

@@ -96,6 +96,7 @@ cudaError_t potrf_lower(T* A, int64_t n, int64_t lda, T* dinv, int32_t* status_d
     const int nb = (int)((n - k0 < NB) ? (n - k0) : NB);
     T* Akk = A + k0 * lda + k0;
     T* dk = dinv + (k0 / NB) * NB * NB;
+    count_launch();
     chol_diag_kernel<T><<<1, 256, diag_smem_bytes<T>(), stream>>>(Akk, lda, nb, dk, k0, status_dev);
     const int64_t rem = n - k0 - nb;
     if (rem <= 0) break;

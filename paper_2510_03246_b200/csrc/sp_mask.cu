@@ -392,8 +392,11 @@ cudaError_t wanda_scores(int kind, int group, const float* W, int64_t rows, int6
   if (cols == 0) return cudaSuccess;
   const int rb = row_blocks_for(rows, cols);
   const int k = kind == SP_SCORE_WANDA_L2 ? 0 : 1;
+  ProfScope prof(PK_SCORES, 0.0, (double)rows * (double)cols * 4.0, stream);
+  count_launch();
   weight_col_partials_kernel<<<dim3((unsigned)ceil_div(cols, 256), (unsigned)rb), 256, 0, stream>>>(W, rows, cols, ldw,
                                                                                                    k, rb, scratch);
+  count_launch();
   wanda_finish_kernel<<<1, 1024, 0, stream>>>(scratch, rb, cols, k, group, colsq, colsq_stride, colabs, inv_tokens,
                                               n_units, scores, importance);
   return cudaGetLastError();
@@ -408,8 +411,13 @@ cudaError_t lemma1_scores_stream(const sp_mat& b, const sp_mat& c, const sp_mat&
   const int rb = row_blocks_for(N, cols);
   double* part = scratch;
   double* unit_e = scratch + (size_t)rb * cols * 2;
+  ProfScope prof(PK_SCORES, 0.0, (double)N * (double)cols * (double)(dtype_size(b.dtype) + dtype_size(c.dtype) +
+                                                                    dtype_size(dd.dtype) + dtype_size(t.dtype)),
+                 stream);
+  count_launch();
   lemma1_partials_kernel<<<dim3((unsigned)ceil_div(cols, 256), (unsigned)rb), 256, 0, stream>>>(b, c, dd, t, N, cols,
                                                                                                rb, part);
+  count_launch();
   lemma1_finish_kernel<<<1, 1024, 0, stream>>>(part, rb, cols, group, n_units, scores, importance, relaxed, r_layer,
                                                unit_e);
   return cudaGetLastError();
@@ -419,13 +427,18 @@ cudaError_t lemma1_scores_gram(const float* T0, const float* W1t, const float* W
                                float* scores, double* importance, double* scratch, cudaStream_t stream) {
   (void)scratch;
   if (n == 0) return cudaSuccess;
+  ProfScope prof(PK_SCORES, 0.0, (double)n * (double)d * 12.0, stream);
+  count_launch();
   lemma1_gram_rows_kernel<<<(unsigned)ceil_div(n * 32, 256), 256, 0, stream>>>(T0, W1t, W10, n, d, scores);
+  count_launch();
   mean_scores_kernel<<<1, 1024, 0, stream>>>(scores, n, importance);
   return cudaGetLastError();
 }
 
 cudaError_t allocate_sparsity(const double* I, const int64_t* n_units, int L, double rbar, double T, int mode,
                               double clip_hi, double* r_out, int64_t* k_out, cudaStream_t stream) {
+  ProfScope prof(PK_ALLOCATE, 0.0, (double)L * 32.0, stream);
+  count_launch();
   allocate_kernel<<<1, 1024, 0, stream>>>(I, n_units, L, rbar, T, mode, clip_hi, r_out, k_out);
   return cudaGetLastError();
 }
@@ -433,28 +446,38 @@ cudaError_t allocate_sparsity(const double* I, const int64_t* n_units, int L, do
 cudaError_t topk_select(const float* scores, int64_t n, int64_t k, uint8_t* mask, float* tau, int32_t* kept_idx,
                         cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
+  ProfScope prof(PK_TOPK, 0.0, (double)n * 5.0, stream);
+  count_launch();
   topk_select_kernel<<<1, 1024, 0, stream>>>(scores, n, k, mask, tau, kept_idx);
   return cudaGetLastError();
 }
 
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
+  count_launch();
   mask_to_index_kernel<<<1, 1024, 0, stream>>>(mask, n, kept_idx);
   return cudaGetLastError();
 }
 
 cudaError_t zero_pruned(const uint8_t* mask, int group, float* W_rows, int64_t r_rows, int64_t r_cols, int64_t r_ld,
                         float* W_cols, int64_t c_rows, int64_t c_cols, int64_t c_ld, cudaStream_t stream) {
-  if (W_rows && r_rows * r_cols > 0)
+  if (W_rows && r_rows * r_cols > 0) {
+    ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+    count_launch();
     zero_rows_kernel<<<grid_for(r_rows * r_cols, 256), 256, 0, stream>>>(mask, group, W_rows, r_rows, r_cols, r_ld);
-  if (W_cols && c_rows * c_cols > 0)
+  }
+  if (W_cols && c_rows * c_cols > 0) {
+    count_launch();
     zero_cols_kernel<<<grid_for(c_rows * c_cols, 256), 256, 0, stream>>>(mask, group, W_cols, c_rows, c_cols, c_ld);
+  }
   return cudaGetLastError();
 }
 
 cudaError_t mask_rows_copy(const uint8_t* mask, const float* src, int64_t lds, float* dst, int64_t ldd, int64_t rows,
                            int64_t cols, cudaStream_t stream) {
   if (rows * cols == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
   mask_rows_copy_kernel<<<grid_for(rows * cols, 256), 256, 0, stream>>>(mask, src, lds, dst, ldd, rows, cols);
   return cudaGetLastError();
 }

@@ -1,0 +1,82 @@
+// Launch counter and optional CUDA-event timing of the library's kernels, per kernel kind.
+#include <atomic>
+#include <vector>
+
+#include "sp_common.cuh"
+
+namespace sp {
+namespace {
+
+constexpr int kMaxSlots = 16384;
+struct Slot {
+  cudaEvent_t start, stop;
+  int kind;
+  double flops, bytes;
+};
+std::atomic<long long> g_launches{0};
+bool g_enabled = false;
+std::vector<Slot> g_slots;
+int g_used = 0;
+thread_local int g_depth = 0;
+
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+ProfScope::ProfScope(int kind, double flops, double bytes, cudaStream_t s) : slot(-1), stream(s) {
+  if (g_depth++ > 0 || !g_enabled || g_used >= kMaxSlots) return;
+  if ((int)g_slots.size() <= g_used) {
+    Slot sl;
+    if (cudaEventCreate(&sl.start) != cudaSuccess || cudaEventCreate(&sl.stop) != cudaSuccess) return;
+    g_slots.push_back(sl);
+  }
+  slot = g_used++;
+  g_slots[slot].kind = kind;
+  g_slots[slot].flops = flops;
+  g_slots[slot].bytes = bytes;
+  cudaEventRecord(g_slots[slot].start, stream);
+}
+
+ProfScope::~ProfScope() {
+  --g_depth;
+  if (slot >= 0) cudaEventRecord(g_slots[slot].stop, stream);
+}
+
+}  // namespace sp
+
+extern "C" {
+
+int64_t sp_launch_count(void) { return (int64_t)sp::g_launches.load(); }
+
+sp_status sp_profile_begin(int32_t enable) {
+  sp::g_enabled = enable != 0;
+  sp::g_used = 0;
+  sp::g_launches.store(0);
+  return SP_OK;
+}
+
+int32_t sp_profile_kinds(void) { return sp::PK_COUNT; }
+
+const char* sp_profile_kind_name(int32_t kind) {
+  static const char* names[sp::PK_COUNT] = {"gemm_tc", "gemm_simt", "solve_phase", "fused_update", "prep_h",
+                                            "scores", "topk_select", "elementwise", "allocate"};
+  return (kind >= 0 && kind < sp::PK_COUNT) ? names[kind] : "unknown";
+}
+
+sp_status sp_profile_read(double* out_host) {
+  if (!out_host) return SP_ERR_INVALID_ARG;
+  for (int i = 0; i < sp::PK_COUNT * 4; ++i) out_host[i] = 0.0;
+  for (int i = 0; i < sp::g_used; ++i) {
+    const sp::Slot& s = sp::g_slots[i];
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, s.start, s.stop) != cudaSuccess) return SP_ERR_CUDA;
+    double* o = out_host + s.kind * 4;
+    o[0] += 1.0;
+    o[1] += (double)ms;
+    o[2] += s.flops;
+    o[3] += s.bytes;
+  }
+  return SP_OK;
+}
+
+}  // extern "C"
