@@ -47,7 +47,8 @@ typedef enum {
   SP_ERR_NOT_SPD = 6,
   SP_ERR_TIMEOUT = 7,
   SP_ERR_CUDA = 8,
-  SP_ERR_UNSUPPORTED = 9
+  SP_ERR_UNSUPPORTED = 9,
+  SP_ERR_STATIC_LIMIT = 10
 } sp_status;
 
 typedef enum { SP_F32 = 0, SP_BF16 = 1, SP_F64 = 2 } sp_dtype;
@@ -183,6 +184,29 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
 sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* in, int64_t n_units, float* scores,
                            double* layer_importance, double* relaxed_mask, double r_layer, void* ws, size_t ws_bytes,
                            void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_struct_scores_static — the two Wanda kinds of sp_struct_scores with NO workspace argument and no allocation.
+ * The paper has no counterpart; this is a packaging variant of the call above.
+ * Who needs it: a caller that owns no spare device memory and cannot obtain any — for example a service whose device
+ * memory was carved up once at start-up, or code that runs between other asynchronous work and must not stall the
+ * whole device the way an allocation call does.  Such a caller passes only the inputs and the outputs; the partial
+ * column sums go to a fixed array of 2 MiB that is part of the library image (every GPU that loads libsp.so holds
+ * it until the process ends).
+ * Limits: n_units*group <= SP_STATIC_SCORES_MAX_COLS, and the partial sums must fit the array; anything larger
+ * returns SP_ERR_STATIC_LIMIT before any launch (use sp_struct_scores with a workspace instead).  kind must be
+ * SP_SCORE_WANDA_L2 or SP_SCORE_WANDA_L1 (else SP_ERR_UNSUPPORTED).  Other argument errors as sp_struct_scores.
+ * Results are the same as sp_struct_scores gives for the same inputs (same kernels, same reduction order).
+ * Set-up: the first call on each device looks up the device address of the array (one runtime query, with that device
+ * current); make that first call outside any stream capture.
+ * Sharing: all calls on one device use the same array.  Calls on the same stream are ordered and safe; two calls that
+ * may overlap on the GPU (different streams without an ordering between them) race on it.  The array keeps the last
+ * call's partial sums; no call reads a value it did not write itself, so nothing has to be cleared.
+ * The call itself performs no device or host allocation and calls no allocating library routine.
+ */
+#define SP_STATIC_SCORES_MAX_COLS 32768
+sp_status sp_struct_scores_static(int32_t kind, int32_t group, const sp_score_inputs* in, int64_t n_units,
+                                  float* scores, double* layer_importance, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
  * sp_allocate_sparsity — softmax-form sparsity allocation across L layers (Lemma 2; Algorithm 1, Step 2).

@@ -25,7 +25,7 @@ SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
  SP_WS_RIDGE_SOLVE) = range(8)
 
 EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
-           "sp_apply_mask", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes",
+           "sp_apply_mask", "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
            "sp_profile_kind_name", "sp_launch_count"]
 
@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
         L.sp_admm_step.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), C.POINTER(SpAdmmParams), vp, vp, vp,
                                    sz, vp]
         L.sp_struct_scores.argtypes = [i32, i32, C.POINTER(SpScoreInputs), i64, vp, vp, vp, dbl, vp, sz, vp]
+        L.sp_struct_scores_static.argtypes = [i32, i32, C.POINTER(SpScoreInputs), i64, vp, vp, vp]
         L.sp_allocate_sparsity.argtypes = [vp, vp, i32, dbl, dbl, i32, dbl, vp, vp, vp]
         L.sp_apply_mask.argtypes = [vp, i64, i64, i32, vp, vp, vp, pm, pm, vp, sz, vp]
         L.sp_ridge_solve.argtypes = [vp, i64, vp, i64, i64, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
@@ -248,6 +249,22 @@ def sp_struct_scores(kind, n_units, group=1, W=None, colsq=None, colsq_stride=1,
                                   _ptr(relaxed), float(r_layer), ws.data_ptr(), ws.numel(), _stream()),
            "sp_struct_scores")
     return scores, imp, relaxed
+
+
+STATIC_SCORES_MAX_COLS = 32768
+
+
+def sp_struct_scores_static(kind, n_units, scores, importance, group=1, W=None, colsq=None, colsq_stride=1,
+                            colabs=None, inv_tokens=0.0):
+    """Wanda scores without a workspace: for callers that cannot allocate device memory at the time of the call.
+
+    `scores` (fp32 [n_units]) and `importance` (fp64 [1]) are caller-provided outputs; nothing is allocated here or in
+    the library.  Sizes beyond the built-in scratch raise SpError (SP_ERR_STATIC_LIMIT)."""
+    _require_cuda(W, colsq, colabs, scores, importance)
+    inp = SpScoreInputs(mat(W), _ptr(colsq), colsq_stride, _ptr(colabs), float(inv_tokens), mat(None), mat(None),
+                        mat(None), mat(None))
+    _check(lib().sp_struct_scores_static(kind, group, C.byref(inp), n_units, scores.data_ptr(), _ptr(importance),
+                                         _stream()), "sp_struct_scores_static")
 
 
 def sp_allocate_sparsity(I, n_units, rbar, T, mode=SP_ALLOC_SOFTMAX, clip_hi=0.95):

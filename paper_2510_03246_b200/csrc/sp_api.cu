@@ -236,6 +236,7 @@ const char* sp_status_string(int32_t s) {
     case SP_ERR_TIMEOUT: return "bounded device wait ran out";
     case SP_ERR_CUDA: return "CUDA runtime error";
     case SP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SP_ERR_STATIC_LIMIT: return "size exceeds the limit of the built-in static scratch";
     default: return "unknown status";
   }
 }

@@ -2,6 +2,8 @@
 // Lemma 2 / Algorithm 1 Step 2, the exact top-k selection by radix select, and M (.) W.
 #include <math.h>
 
+#include <mutex>
+
 #include "sp_common.cuh"
 
 namespace sp {
@@ -483,3 +485,59 @@ cudaError_t mask_rows_copy(const uint8_t* mask, const float* src, int64_t lds, f
 }
 
 }  // namespace sp
+
+// ------------------------------------------------------------------------------------ static-scratch score entry
+// Wanda scores for callers that hold no workspace and must not allocate one.  The partial column sums live in a
+// file-scope device array that every GPU loading the library carries until the process exits.
+namespace {
+
+constexpr size_t kStaticScratchDoubles = (size_t)1 << 18;   // 2 MiB
+static __device__ __align__(256) double g_static_scratch[kStaticScratchDoubles];
+
+constexpr int kMaxDevices = 64;
+double* g_static_scratch_addr[kMaxDevices] = {};
+std::mutex g_static_scratch_mutex;
+
+// Device address of g_static_scratch on the current device.  In host code the array's name is only a handle, so the
+// address is looked up once per device (with that device current) and cached.
+sp_status static_scratch_address(double** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SP_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SP_ERR_CUDA;
+    g_static_scratch_addr[dev] = reinterpret_cast<double*>(p);
+  }
+  *out = g_static_scratch_addr[dev];
+  return SP_OK;
+}
+
+}  // namespace
+
+extern "C" sp_status sp_struct_scores_static(int32_t kind, int32_t group, const sp_score_inputs* in, int64_t n_units,
+                                             float* scores, double* layer_importance, void* stream) {
+  if (!in || !scores) return SP_ERR_INVALID_ARG;
+  if (kind != SP_SCORE_WANDA_L2 && kind != SP_SCORE_WANDA_L1) return SP_ERR_UNSUPPORTED;
+  if (group < 1 || n_units < 1) return SP_ERR_SHAPE;
+  if (n_units > SP_STATIC_SCORES_MAX_COLS / group) return SP_ERR_STATIC_LIMIT;
+  const int64_t cols = n_units * group;
+  if (!in->W.ptr) return SP_ERR_INVALID_ARG;
+  if (in->W.dtype != SP_F32) return SP_ERR_DTYPE;
+  if (in->W.cols != cols || in->W.ld < cols || in->W.rows < 1) return SP_ERR_SHAPE;
+  if (kind == SP_SCORE_WANDA_L2 && (!in->colsq || in->colsq_stride < 1)) return SP_ERR_INVALID_ARG;
+  if (kind == SP_SCORE_WANDA_L1 && !in->colabs) return SP_ERR_INVALID_ARG;
+  // the partial sums take row_blocks x cols doubles; row_blocks shrinks as cols grows, so the product stays bounded
+  if ((size_t)sp::score_row_blocks(in->W.rows, cols) * (size_t)cols > kStaticScratchDoubles)
+    return SP_ERR_STATIC_LIMIT;
+  double* scratch = nullptr;
+  const sp_status st = static_scratch_address(&scratch);
+  if (st != SP_OK) return st;
+  // every partial sum that the finishing kernel reads is written by the first kernel of this same call, so nothing
+  // left behind by an earlier call is ever read and no clearing is needed
+  if (sp::wanda_scores(kind, group, reinterpret_cast<const float*>(in->W.ptr), in->W.rows, in->W.ld, in->colsq,
+                       in->colsq_stride, in->colabs, in->inv_tokens, n_units, scores, layer_importance, scratch,
+                       reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return SP_ERR_CUDA;
+  return SP_OK;
+}
