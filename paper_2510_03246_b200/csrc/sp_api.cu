@@ -58,10 +58,14 @@ sp_status contract_split_weights(int64_t M, int64_t N, int64_t K, MatRef A, cons
   if (M <= 0 || N <= 0) return SP_OK;
   const int64_t kp = split_kpad(K);
   TcOperand ta{A.ptr, A.ld, true}, tb{Wsplit, 2 * kp, true};
+  tb.kext = 2 * kp;
   OutOperand out{const_cast<void*>(C.ptr), C.dtype, C.ld};
   Operand cin{C.ptr, C.dtype, C.ld, 1};
-  if (Wsplit && A.dtype == SP_BF16 && gemm_tc_supported(M, N, K, ta, TcOperand{Wsplit, 2 * kp, true})) {
-    return gemm_tc(M, N, K + kp, 1.f, ta, tb, 0.f, cin, out, false, status, stream, kp, K);
+  if (Wsplit && A.dtype == SP_BF16 && gemm_tc_supported(M, N, K, ta, tb)) {
+    TcSegments sg;
+    sg.nseg = 2;            // hi part, then lo part, against the same A tile
+    sg.b_k[1] = (int32_t)kp;
+    return gemm_tc(M, N, K, 1.f, ta, tb, 0.f, cin, out, false, status, stream, &sg, 2.0 * (double)M * N * K);
   }
   return contract(M, N, K, 1.0, A, true, Wf32, true, 0.0, C, C, false, false, false, status, stream);
 }
@@ -85,7 +89,11 @@ struct Carver {
   }
 };
 
-size_t dinv_elems(int64_t n) { return (size_t)ceil_div(n, (int64_t)kCholNB) * kCholNB * kCholNB; }
+size_t dinv_elems(int64_t n) {
+  const size_t simt = (size_t)ceil_div(n, (int64_t)kCholNB) * kCholNB * kCholNB;
+  const size_t tc = (size_t)ceil_div(n, (int64_t)kCholTcNB) * kCholTcNB * kCholTcNB;
+  return simt > tc ? simt : tc;
+}
 
 // Buffers of the regularised solve for systems up to nmax with up to mmax right-hand sides.
 struct SolveBufs {
@@ -94,6 +102,8 @@ struct SolveBufs {
   void* Rs;
   int32_t* idx;
   double* rho;  // [4] device scalars
+  void* P;      // fp32 path: bf16 parts of the Cholesky factor
+  void* Xs;     // fp32 path: bf16 parts of one block column of right-hand sides
 };
 
 SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
@@ -103,6 +113,14 @@ SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
   b.Gs = c.take_bytes((size_t)nmax * nmax * tsize);
   b.dinv = c.take_bytes(dinv_elems(nmax) * tsize);
   b.Rs = c.take_bytes((size_t)nmax * mmax * tsize);
+  b.P = nullptr;
+  b.Xs = nullptr;
+  if (tsize == 4) {
+    const size_t np = (size_t)chol_tc_pad(nmax);
+    b.P = c.take_bytes(np * 3 * np * 2);
+    const size_t rows = (size_t)(nmax > mmax ? nmax : mmax);   // either dimension may be the right-hand-side count
+    b.Xs = c.take_bytes(rows * 3 * kCholTcNB * 2);
+  }
   return b;
 }
 
@@ -118,9 +136,15 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
   T* Rs = reinterpret_cast<T*>(b.Rs);
   if (idx) CU(load_spd_gather<T>(G, ldg, idx, nn, rho_dev, Gs, nn, stream));
   else CU(load_spd<T>(G, ldg, nn, rho_dev, Gs, nn, stream));
-  CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
-  CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
-  CU(potrs_right<T>(Rs, m, nn, nn, Gs, nn, dinv, stream));
+  if constexpr (sizeof(T) == 4) {
+    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream));
+    CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
+    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream));
+  } else {
+    CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
+    CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
+    CU(potrs_right<T>(Rs, m, nn, nn, Gs, nn, dinv, stream));
+  }
   CU(scatter_cols<T>(Rs, nn, idx, m, nn, n_full, W, ldw, stream));
   return SP_OK;
 }
@@ -581,11 +605,11 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
       float* Gs = reinterpret_cast<float*>(p.sb.Gs);
       float* Rs = reinterpret_cast<float*>(p.sb.Rs);
       CU(load_spd<float>(p.Cf, d, d, gam, Gs, d, s));
-      CU(potrf_lower<float>(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), status_dev, s));
+      SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s));
       // right-hand sides: the rows of W2^T as the tensor-core path sees them (bf16-rounded W2)
       CU(convert_matrix(p.W2b, SP_BF16, n, p.W2t, SP_F32, n, d, n, s));
       CU(transpose_convert<float>(p.W2t, n, d, n, Rs, d, s));
-      CU(potrs_right<float>(Rs, n, d, d, Gs, d, reinterpret_cast<float*>(p.sb.dinv), s));
+      SPCHK(potrs_right_tc(Rs, n, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s));
       CU(convert_matrix(Rs, SP_F32, d, p.Qt, SP_F32, d, n, d, s));
       CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, n, d, s));
       qt = MatRef{p.Qtb, SP_BF16, d};

@@ -65,12 +65,22 @@ struct TcOperand {
   const void* ptr;  // bf16
   int64_t ld;       // elements between consecutive rows of the stored matrix
   bool kmajor;
+  int64_t kext = 0;   // extent of the stored matrix along K (0: the K of the call); reads beyond it return zero
+  int64_t mnext = 0;  // extent along M (for A) or N (for B) (0: the M / N of the call)
 };
-// a_kwrap > 0 (a multiple of 64): A holds only a_kext <= a_kwrap K indices (zero beyond) and is read again for the
-// K range [a_kwrap, K), so that B may hold two K segments (hi and lo parts of split weights) against the same A.
+// K segments: the contraction runs over nseg segments of K indices each; segment s reads A at K offset a_k[s] and
+// M offset a_mn[s], B at K offset b_k[s] and N offset b_mn[s] (elements).  This is how split operands (an fp32 value
+// held as a sum of bf16 parts stored side by side) are multiplied: one segment per kept product of parts.
+constexpr int kTcMaxSegments = 6;
+struct TcSegments {
+  int32_t nseg = 1;
+  int32_t a_k[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, a_mn[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
+  int32_t b_k[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, b_mn[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
+};
+// K is the extent of ONE segment.  alg_flops >= 0 overrides the flop count recorded for profiling.
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
-                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, int64_t a_kwrap = 0,
-                  int64_t a_kext = 0);
+                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream,
+                  const TcSegments* segs = nullptr, double alg_flops = -1.0);
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B);
 
 // Dense symmetric positive definite solve in precision T (float or double), all on `stream`.
@@ -86,6 +96,17 @@ template <typename T>
 cudaError_t potrs_right(T* X, int64_t m, int64_t n, int64_t ldx, const T* L, int64_t ldl, const T* dinv,
                         cudaStream_t stream);
 constexpr int kCholNB = 64;
+
+// fp32 factorisation / solves with tensor-core trailing updates (sp_linalg_tc.cu).  Panels are kCholTcNB wide.
+//   dinv: ceil(n / kCholTcNB) blocks of kCholTcNB^2 floats (inverse diagonal blocks)
+//   P   : bf16 [chol_tc_pad(n), 3 * chol_tc_pad(n)] — the factor below its diagonal blocks as three bf16 parts
+//   Xs  : bf16 [m, 3 * kCholTcNB] — the current block column of the right-hand sides as three bf16 parts
+constexpr int kCholTcNB = 128;
+int64_t chol_tc_pad(int64_t n);
+sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P, int32_t* status_dev,
+                         cudaStream_t stream);
+sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* P, const float* dinv, void* Xs,
+                         int32_t* status_dev, cudaStream_t stream);
 
 // ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,

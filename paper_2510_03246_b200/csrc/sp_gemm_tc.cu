@@ -44,8 +44,9 @@ struct TcParams {
   int32_t c_dtype;
   int64_t c_ld;
   int32_t a_kmajor, b_kmajor, lower_only;
-  int32_t a_kwrap;   // > 0: the A operand's K coordinate wraps at this multiple of BK (A is read again for a
-                     // second K segment of B, used for hi/lo-split bf16 weights)
+  int32_t n_fast;    // tile order: 1 = consecutive tiles walk N first (they share the A row block)
+  TcSegments seg;    // K segments: segment s reads A at (k + a_k[s], m + a_mn[s]) and B at (k + b_k[s], n + b_mn[s])
+  int32_t seg_kb;    // k-blocks per segment
   int32_t tiles_m, tiles_n, num_tiles;
   int32_t* status;
 };
@@ -153,8 +154,13 @@ __device__ __forceinline__ uint32_t make_instr_desc(bool a_kmajor, bool b_kmajor
 
 __device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, int& tn) {
   if (!p.lower_only) {
-    tm = t % p.tiles_m;
-    tn = t / p.tiles_m;
+    if (p.n_fast) {
+      tn = t % p.tiles_n;
+      tm = t / p.tiles_n;
+    } else {
+      tm = t % p.tiles_m;
+      tn = t / p.tiles_m;
+    }
   } else {
     // column block tn owns row blocks first(tn)..tiles_m-1 with first = tn * BN / BM
     tn = 0;
@@ -173,6 +179,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
+  __shared__ float s_stage[4][32][33];   // per epilogue warp: one 32 x 32 accumulator block, padded
 
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;            // 1024-byte aligned operand stages
@@ -206,7 +213,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
 
-  const int num_kb = (int)((p.K + BK - 1) / BK);
+  const int num_kb = p.seg_kb * p.seg.nseg;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -226,19 +233,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           armed_parity = (armed_parity & ~(1u << s)) | (ph << s);
           const uint32_t a_dst = tiles + s * STAGE_BYTES;
           const uint32_t b_dst = a_dst + A_BYTES;
-          const int k0 = kb * BK;
-          const int ka = (p.a_kwrap > 0 && k0 >= p.a_kwrap) ? k0 - p.a_kwrap : k0;
+          const int sg = kb / p.seg_kb;
+          const int kk = (kb - sg * p.seg_kb) * BK;
+          const int ka = kk + p.seg.a_k[sg], kbb = kk + p.seg.b_k[sg];
+          const int am = tm * BM + p.seg.a_mn[sg], bn = tn * BN + p.seg.b_mn[sg];
           if (p.a_kmajor) {
-            tma_load_2d(a_dst, &tmA, ka, tm * BM, full_bar(s));
+            tma_load_2d(a_dst, &tmA, ka, am, full_bar(s));
           } else {
 #pragma unroll
-            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, tm * BM + mb * 64, ka, full_bar(s));
+            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, am + mb * 64, ka, full_bar(s));
           }
           if (p.b_kmajor) {
-            tma_load_2d(b_dst, &tmB, k0, tn * BN, full_bar(s));
+            tma_load_2d(b_dst, &tmB, kbb, bn, full_bar(s));
           } else {
 #pragma unroll
-            for (int nb = 0; nb < BN / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, tn * BN + nb * 64, k0, full_bar(s));
+            for (int nb = 0; nb < BN / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, bn + nb * 64, kbb, full_bar(s));
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -300,13 +309,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps 2..5
+    // tcgen05.ld hands every lane one accumulator row (32 consecutive columns per load).  The 32 x 32 block is turned
+    // through a padded shared-memory tile so that global loads and stores see a warp on 32 consecutive columns of one
+    // row (128-byte lines) instead of 32 different rows.
     const int q = warp & 3;                 // accumulator lane quarter this warp may read
-    const int row_in_tile = q * 32 + lane;
+    float (*stg)[33] = s_stage[q];
     int acc = 0;
     uint32_t aph = 0;
     bool ok = true;
-    const bool c_vec = (p.c_ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.c) & 15u) == 0);
-    const bool cin_vec = (p.cin_ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.cin) & 15u) == 0);
     for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
       int tm, tn;
       tile_coords(p, t, tm, tn);
@@ -314,61 +324,53 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
       tc_fence_after();
-      const int64_t gi = (int64_t)tm * BM + row_in_tile;
+      const int64_t row0 = (int64_t)tm * BM + q * 32;      // first global row of this warp's 32 rows
       const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
+      const int rows_here = (p.M - row0 < 32) ? (int)(p.M - row0) : 32;   // may be <= 0 on a ragged last tile
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
+        const int64_t gj0 = (int64_t)tn * BN + c0;
+        if (gj0 >= p.N) break;                  // uniform over the warp
         uint32_t r[32];
         tc_ld32(taddr + (uint32_t)c0, r);
         tc_wait_ld();
-        const int64_t gj = (int64_t)tn * BN + c0;
-        if (gi < p.M && gj < p.N) {
-          float v[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = p.alpha * __uint_as_float(r[i]);
-          const bool full = gj + 32 <= p.N;
-          if (p.beta != 0.f) {
-            if (p.cin_dtype == SP_F32) {
-              const float* src = reinterpret_cast<const float*>(p.cin) + gi * p.cin_ld + gj;
-              if (full && cin_vec) {
+        for (int i = 0; i < 32; ++i) stg[lane][i] = p.alpha * __uint_as_float(r[i]);
+        __syncwarp();
+        const int64_t gj = gj0 + lane;
+        if (gj < p.N) {
+          const bool has_cin = p.beta != 0.f;
+          const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
+          const int64_t cin_off = row0 * p.cin_ld + gj, c_off = row0 * p.c_ld + gj;
+#pragma unroll 1
+          for (int r8 = 0; r8 < 32; r8 += 8) {
+            float cv[8];
+            if (has_cin) {   // issue the eight row loads together
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  const float4 x = *reinterpret_cast<const float4*>(src + i);
-                  v[i] += p.beta * x.x; v[i + 1] += p.beta * x.y; v[i + 2] += p.beta * x.z; v[i + 3] += p.beta * x.w;
+              for (int u = 0; u < 8; ++u) {
+                const int rr = r8 + u;
+                cv[u] = 0.f;
+                if (rr < rows_here) {
+                  const int64_t o = cin_off + (int64_t)rr * p.cin_ld;
+                  cv[u] = cin_f32 ? reinterpret_cast<const float*>(p.cin)[o]
+                                  : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.cin)[o]);
                 }
-              } else {
-                for (int i = 0; i < 32; ++i) if (gj + i < p.N) v[i] += p.beta * src[i];
               }
-            } else {
-              const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(p.cin) + gi * p.cin_ld + gj;
-              for (int i = 0; i < 32; ++i) if (gj + i < p.N) v[i] += p.beta * __bfloat162float(src[i]);
             }
-          }
-          if (p.c_dtype == SP_F32) {
-            float* dst = reinterpret_cast<float*>(p.c) + gi * p.c_ld + gj;
-            if (full && c_vec) {
 #pragma unroll
-              for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
-            } else {
-              for (int i = 0; i < 32; ++i) if (gj + i < p.N) dst[i] = v[i];
-            }
-          } else {
-            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.c) + gi * p.c_ld + gj;
-            if (full && (p.c_ld % 8 == 0) && ((reinterpret_cast<uintptr_t>(p.c) & 15u) == 0)) {
-#pragma unroll
-              for (int i = 0; i < 32; i += 8) {
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[i], v[i + 1]), h1 = __floats2bfloat162_rn(v[i + 2], v[i + 3]);
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[i + 4], v[i + 5]), h3 = __floats2bfloat162_rn(v[i + 6], v[i + 7]);
-                uint4 pk;
-                pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                *reinterpret_cast<uint4*>(dst + i) = pk;
+            for (int u = 0; u < 8; ++u) {
+              const int rr = r8 + u;
+              if (rr < rows_here) {
+                float v = stg[rr][lane];
+                if (has_cin) v += p.beta * cv[u];
+                const int64_t o = c_off + (int64_t)rr * p.c_ld;
+                if (c_f32) reinterpret_cast<float*>(p.c)[o] = v;
+                else reinterpret_cast<__nv_bfloat16*>(p.c)[o] = __float2bfloat16_rn(v);
               }
-            } else {
-              for (int i = 0; i < 32; ++i) if (gj + i < p.N) dst[i] = __float2bfloat16_rn(v[i]);
             }
           }
         }
+        __syncwarp();
       }
       tc_fence_before();
       __syncwarp();
@@ -441,25 +443,35 @@ bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B
   if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return false;
   if ((reinterpret_cast<uintptr_t>(A.ptr) & 15u) || (reinterpret_cast<uintptr_t>(B.ptr) & 15u)) return false;
   if (A.ld % 8 != 0 || B.ld % 8 != 0) return false;
-  if (A.ld < (A.kmajor ? K : M) || B.ld < (B.kmajor ? K : N)) return false;
   return true;
 }
 
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
-                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, int64_t a_kwrap,
-                  int64_t a_kext) {
-  if (a_kwrap < 0 || a_kwrap % BK != 0 || (a_kwrap > 0 && (K > 2 * a_kwrap || a_kext < 1 || a_kext > a_kwrap)))
-    return SP_ERR_INVALID_ARG;
-  const int64_t Ka = a_kwrap > 0 ? a_kext : K;   // extent of A along K
-  if (!gemm_tc_supported(M, N, Ka, A, B) || (B.kmajor && B.ld < K)) return SP_ERR_UNSUPPORTED;
+                  OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, const TcSegments* segs,
+                  double alg_flops) {
+  TcSegments sg;
+  if (segs) sg = *segs;
+  else { sg = TcSegments{}; sg.nseg = 1; }
+  if (sg.nseg < 1 || sg.nseg > kTcMaxSegments) return SP_ERR_INVALID_ARG;
+  // extents of the stored operands along K and along M / N (the tensor maps zero-fill beyond them)
+  const int64_t a_kext = A.kext > 0 ? A.kext : K, b_kext = B.kext > 0 ? B.kext : K;
+  const int64_t a_mext = A.mnext > 0 ? A.mnext : M, b_next = B.mnext > 0 ? B.mnext : N;
+  if (M <= 0 || N <= 0 || K <= 0) return SP_ERR_SHAPE;
+  if (!gemm_tc_supported(M, N, K, A, B)) return SP_ERR_UNSUPPORTED;
+  for (int i = 0; i < sg.nseg; ++i) {
+    // TMA: the innermost coordinate times the element size must be a multiple of 16 bytes
+    const int a_inner = A.kmajor ? sg.a_k[i] : sg.a_mn[i], b_inner = B.kmajor ? sg.b_k[i] : sg.b_mn[i];
+    if (a_inner % 8 != 0 || b_inner % 8 != 0) return SP_ERR_ALIGNMENT;
+    if (sg.a_k[i] < 0 || sg.a_mn[i] < 0 || sg.b_k[i] < 0 || sg.b_mn[i] < 0) return SP_ERR_INVALID_ARG;
+  }
   if (lower_only && M != N) return SP_ERR_SHAPE;
   if (beta != 0.f && (Cin.ptr == nullptr || Cin.s1 != 1)) return SP_ERR_INVALID_ARG;
   if (C.dtype != SP_F32 && C.dtype != SP_BF16) return SP_ERR_DTYPE;
   if (beta != 0.f && Cin.dtype != SP_F32 && Cin.dtype != SP_BF16) return SP_ERR_DTYPE;
 
   CUtensorMap tmA, tmB;
-  bool ok = A.kmajor ? make_map(&tmA, A.ptr, Ka, M, A.ld, BK, BM) : make_map(&tmA, A.ptr, M, Ka, A.ld, 64, BK);
-  ok = ok && (B.kmajor ? make_map(&tmB, B.ptr, K, N, B.ld, BK, BN) : make_map(&tmB, B.ptr, N, K, B.ld, 64, BK));
+  bool ok = A.kmajor ? make_map(&tmA, A.ptr, a_kext, a_mext, A.ld, BK, BM) : make_map(&tmA, A.ptr, a_mext, a_kext, A.ld, 64, BK);
+  ok = ok && (B.kmajor ? make_map(&tmB, B.ptr, b_kext, b_next, B.ld, BK, BN) : make_map(&tmB, B.ptr, b_next, b_kext, B.ld, 64, BK));
   if (!ok) return SP_ERR_CUDA;
 
   TcParams p;
@@ -470,9 +482,12 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   p.a_kmajor = A.kmajor ? 1 : 0;
   p.b_kmajor = B.kmajor ? 1 : 0;
   p.lower_only = lower_only ? 1 : 0;
-  p.a_kwrap = (int32_t)a_kwrap;
+  p.seg = sg;
+  p.seg_kb = (int32_t)ceil_div(K, BK);
   p.tiles_m = (int32_t)ceil_div(M, BM);
   p.tiles_n = (int32_t)ceil_div(N, BN);
+  // consecutive tiles (which run at the same time on neighbouring SMs) should share the larger operand panel
+  p.n_fast = p.tiles_n < p.tiles_m ? 1 : 0;
   if (lower_only) {
     int64_t cnt = 0;
     for (int tn = 0; tn < p.tiles_n; ++tn) {
@@ -493,8 +508,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
     attr_set = true;
   }
   count_launch();
-  const double k_alg = (double)(a_kwrap > 0 ? a_kext : K);   // the lo pass of split weights is not algorithmic work
-  ProfScope prof(PK_GEMM_TC, (lower_only ? 1.0 : 2.0) * (double)M * (double)N * k_alg, 0.0, stream);
+  const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
+  ProfScope prof(PK_GEMM_TC, flops, 0.0, stream);
   int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
   gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
