@@ -256,8 +256,9 @@ sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
  * Launch accounting and profiling (the paper has no counterpart; used by the benchmark).
- * sp_profile_begin(enable): resets the launch counter and the event records; enable != 0 brackets every kernel (or
- *   phase) the library launches afterwards with a CUDA event pair on the launching stream.
+ * sp_profile_begin(enable): resets the launch counter and the event records; enable = 1 brackets every kernel (or
+ *   phase: a phase absorbs the kernels launched inside it) the library launches afterwards with a CUDA event pair on
+ *   the launching stream; enable = 2 also records the kernels inside a phase (they are then counted twice).
  * sp_profile_read(out_host): after the caller synchronised the stream(s): out_host[kind*4 + {0,1,2,3}] =
  *   {records, total milliseconds, algorithmic flops, algorithmic bytes} for kind in [0, sp_profile_kinds()).
  * sp_launch_count(): kernels launched by the library since the last sp_profile_begin.

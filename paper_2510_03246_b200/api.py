@@ -156,7 +156,8 @@ def new_status(device="cuda") -> torch.Tensor:
     return torch.zeros(4, dtype=torch.int32, device=device)
 
 
-def sp_profile_begin(enable: bool = True):
+def sp_profile_begin(enable=True):
+    """0 / False: off; 1 / True: outermost kernels and phases; 2: every kernel, also inside a phase."""
     _check(lib().sp_profile_begin(int(enable)), "sp_profile_begin")
 
 

@@ -91,7 +91,7 @@ struct Carver {
 
 size_t dinv_elems(int64_t n) {
   const size_t simt = (size_t)ceil_div(n, (int64_t)kCholNB) * kCholNB * kCholNB;
-  const size_t tc = (size_t)ceil_div(n, (int64_t)kCholTcNB) * kCholTcNB * kCholTcNB;
+  const size_t tc = (size_t)ceil_div(n, (int64_t)kCholTcNB) * 2 * kCholTcNB * kCholTcNB;
   return simt > tc ? simt : tc;
 }
 

@@ -21,7 +21,7 @@ __device__ __forceinline__ void report_status(int32_t* status, int32_t code, int
 // ---- launch accounting and CUDA-event profiling (sp_profile.cu) ---------------------------------------------------
 enum ProfKind : int {
   PK_GEMM_TC = 0, PK_GEMM_SIMT = 1, PK_SOLVE = 2, PK_FUSED_UPDATE = 3, PK_PREP_H = 4, PK_SCORES = 5, PK_TOPK = 6,
-  PK_ELEMENTWISE = 7, PK_ALLOCATE = 8, PK_COUNT = 9
+  PK_ELEMENTWISE = 7, PK_ALLOCATE = 8, PK_CHOL_DIAG = 9, PK_PANEL_APPLY = 10, PK_COUNT = 11
 };
 void count_launch(int n = 1);
 // Brackets the kernels launched during its lifetime with a CUDA event pair on `stream` when profiling is enabled.
@@ -98,7 +98,7 @@ cudaError_t potrs_right(T* X, int64_t m, int64_t n, int64_t ldx, const T* L, int
 constexpr int kCholNB = 64;
 
 // fp32 factorisation / solves with tensor-core trailing updates (sp_linalg_tc.cu).  Panels are kCholTcNB wide.
-//   dinv: ceil(n / kCholTcNB) blocks of kCholTcNB^2 floats (inverse diagonal blocks)
+//   dinv: ceil(n / kCholTcNB) blocks of 2 * kCholTcNB^2 floats (inverse diagonal blocks and their transposes)
 //   P   : bf16 [chol_tc_pad(n), 3 * chol_tc_pad(n)] — the factor below its diagonal blocks as three bf16 parts
 //   Xs  : bf16 [m, 3 * kCholTcNB] — the current block column of the right-hand sides as three bf16 parts
 constexpr int kCholTcNB = 128;

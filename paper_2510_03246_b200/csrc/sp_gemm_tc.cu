@@ -44,6 +44,7 @@ struct TcParams {
   int32_t c_dtype;
   int64_t c_ld;
   int32_t a_kmajor, b_kmajor, lower_only;
+  int32_t red_add;   // 1: C += alpha * acc by global reductions (beta == 1, Cin == C, fp32)
   int32_t n_fast;    // tile order: 1 = consecutive tiles walk N first (they share the A row block)
   TcSegments seg;    // K segments: segment s reads A at (k + a_k[s], m + a_mn[s]) and B at (k + b_k[s], n + b_mn[s])
   int32_t seg_kb;    // k-blocks per segment
@@ -327,42 +328,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int64_t row0 = (int64_t)tm * BM + q * 32;      // first global row of this warp's 32 rows
       const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
       const int rows_here = (p.M - row0 < 32) ? (int)(p.M - row0) : 32;   // may be <= 0 on a ragged last tile
+      const bool has_cin = p.beta != 0.f && !p.red_add;
+      const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         const int64_t gj0 = (int64_t)tn * BN + c0;
         if (gj0 >= p.N) break;                  // uniform over the warp
+        const int64_t gj = gj0 + lane;
+        // the 32 rows of Cin for this column are fetched first (independent loads in flight while the accumulator
+        // block is read from tensor memory and turned)
+        float cv[32];
+        if (has_cin) {
+          const int64_t cin_off = row0 * p.cin_ld + gj;
+#pragma unroll
+          for (int rr = 0; rr < 32; ++rr) {
+            cv[rr] = 0.f;
+            if (gj < p.N && rr < rows_here) {
+              const int64_t o = cin_off + (int64_t)rr * p.cin_ld;
+              cv[rr] = cin_f32 ? reinterpret_cast<const float*>(p.cin)[o]
+                               : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.cin)[o]);
+            }
+          }
+        }
         uint32_t r[32];
         tc_ld32(taddr + (uint32_t)c0, r);
         tc_wait_ld();
 #pragma unroll
         for (int i = 0; i < 32; ++i) stg[lane][i] = p.alpha * __uint_as_float(r[i]);
         __syncwarp();
-        const int64_t gj = gj0 + lane;
         if (gj < p.N) {
-          const bool has_cin = p.beta != 0.f;
-          const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
-          const int64_t cin_off = row0 * p.cin_ld + gj, c_off = row0 * p.c_ld + gj;
-#pragma unroll 1
-          for (int r8 = 0; r8 < 32; r8 += 8) {
-            float cv[8];
-            if (has_cin) {   // issue the eight row loads together
+          const int64_t c_off = row0 * p.c_ld + gj;
+          if (p.red_add) {
+            // C += alpha * acc: one reduction per element, no read round trip (each address is touched once per launch)
+            float* dst = reinterpret_cast<float*>(p.c) + c_off;
 #pragma unroll
-              for (int u = 0; u < 8; ++u) {
-                const int rr = r8 + u;
-                cv[u] = 0.f;
-                if (rr < rows_here) {
-                  const int64_t o = cin_off + (int64_t)rr * p.cin_ld;
-                  cv[u] = cin_f32 ? reinterpret_cast<const float*>(p.cin)[o]
-                                  : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.cin)[o]);
-                }
-              }
-            }
+            for (int rr = 0; rr < 32; ++rr)
+              if (rr < rows_here)
+                asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst + (int64_t)rr * p.c_ld), "f"(stg[rr][lane]) : "memory");
+          } else {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const int rr = r8 + u;
+            for (int rr = 0; rr < 32; ++rr) {
               if (rr < rows_here) {
                 float v = stg[rr][lane];
-                if (has_cin) v += p.beta * cv[u];
+                if (has_cin) v = fmaf(p.beta, cv[rr], v);
                 const int64_t o = c_off + (int64_t)rr * p.c_ld;
                 if (c_f32) reinterpret_cast<float*>(p.c)[o] = v;
                 else reinterpret_cast<__nv_bfloat16*>(p.c)[o] = __float2bfloat16_rn(v);
@@ -482,6 +490,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   p.a_kmajor = A.kmajor ? 1 : 0;
   p.b_kmajor = B.kmajor ? 1 : 0;
   p.lower_only = lower_only ? 1 : 0;
+  p.red_add = (beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && C.dtype == SP_F32 && Cin.s0 == C.ld) ? 1 : 0;
   p.seg = sg;
   p.seg_kb = (int32_t)ceil_div(K, BK);
   p.tiles_m = (int32_t)ceil_div(M, BM);

@@ -21,17 +21,22 @@ constexpr int TB = kCholTcNB;          // 128
 constexpr int DIAG_BLOCKS = (TB / 4) * (TB / 4 + 1) / 2;   // 528 lower-triangular 4 x 4 blocks
 constexpr int DIAG_THREADS = 544;      // 17 warps
 
-// Factorise the nb x nb diagonal block at A (lower triangle) and write L back; dinv (TB x TB, row-major) receives
-// inv(L), zero above the diagonal, identity on the padding rows nb..TB-1.  A non-positive pivot is reported once
-// through `status` and replaced by 1.
+// Factorise the nb x nb diagonal block at A (lower triangle), write L back, and write inv(L) and its transpose to
+// dinv[0 : TB*TB] and dinv[TB*TB : 2*TB*TB] (row-major TB x TB, zero above / below the diagonal respectively,
+// identity on the padding rows nb..TB-1).  A non-positive pivot is reported once through `status` and replaced by 1.
 //
-// Elimination without square roots in the loop: step j subtracts a_ij a_cj / p_j from the trailing part (p_j the
-// pivot), and applies the same row operations to an identity block B.  At the end L_ic = a_ic / sqrt(p_c) and
-// inv(L)_ic = B_ic / sqrt(p_i).
+// One thread owns one 4 x 4 block of the lower triangle in registers.  Elimination without square roots in the
+// loop: step j subtracts a_ij a_cj / p_j from the trailing columns c > j (p_j the pivot) and applies the same row
+// operations to an identity block B on the columns c <= j.  A column of the trailing matrix is final when its step
+// comes: it is scaled by 1/sqrt(p_j) and stored as column j of L, and its registers then carry column j of B.  So a
+// single register block m holds "a" on the columns still to be eliminated and "B" on the others, and one shared
+// vector w per step feeds both updates: w[i] = a_ij for i > j, w[c] = B_jc for c < j, w[j] = 1 / p_j.
+// A thread owns part of the eliminated column only while j runs through its own block column, so it keeps those
+// four unscaled columns in a second register block and scales them after the loop: L_ic = a_ic / sqrt(p_c),
+// inv(L)_ic = B_ic / sqrt(p_i).  The loop's critical path per step is barrier, one shared load, one multiply-add.
 __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, int64_t lda, int nb, float* dinv,
                                                                     int64_t row0, int32_t* status) {
-  __shared__ float colbuf[2][TB];   // column j of the trailing matrix (unscaled), double buffered
-  __shared__ float rowbuf[2][TB];   // row j of B
+  __shared__ __align__(16) float wbuf[2][TB];   // double buffered: one barrier per step
   __shared__ float piv[TB];
   const int t = threadIdx.x;
   const bool active = t < DIAG_BLOCKS;
@@ -41,7 +46,7 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
   while (bi * (bi + 1) / 2 > t) --bi;
   const int bj = t - bi * (bi + 1) / 2;
 
-  float a[4][4], b[4][4];
+  float m[4][4], lcol[4][4];
 #pragma unroll
   for (int r = 0; r < 4; ++r)
 #pragma unroll
@@ -50,14 +55,17 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
       float v = 0.f;
       if (active && i < nb && c <= i) v = A[(int64_t)i * lda + c];
       if (i >= nb && i == c) v = 1.f;
-      a[r][s] = v;
-      b[r][s] = (i == c) ? 1.f : 0.f;
+      m[r][s] = v;
+      lcol[r][s] = v;
     }
   if (t < TB) piv[t] = 1.f;
-  // zero the part of dinv that no thread owns (blocks strictly above the diagonal)
+  // zero the parts of the two inverse blocks that no thread owns (blocks strictly above the diagonal of inv(L))
   for (int e = t; e < TB * TB; e += DIAG_THREADS) {
     const int i = e / TB, c = e % TB;
-    if ((c >> 2) > (i >> 2)) dinv[e] = 0.f;
+    if ((c >> 2) > (i >> 2)) {
+      dinv[e] = 0.f;
+      dinv[TB * TB + c * TB + i] = 0.f;
+    }
   }
   __syncthreads();
 
@@ -67,46 +75,56 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
     for (int jj = 0; jj < 4; ++jj) {
       const int j = jb * 4 + jj;
       if (j < nb) {                     // uniform over the block
-        const int buf = j & 1;
-        if (active && bj == jb) {       // owners of column j
+        float* wb = wbuf[j & 1];
+        if (active && bj == jb) {       // owners of column j: live values below the diagonal, and the pivot
 #pragma unroll
-          for (int r = 0; r < 4; ++r) colbuf[buf][4 * bi + r] = a[r][jj];
+          for (int r = 0; r < 4; ++r)
+            if (4 * bi + r > j) wb[4 * bi + r] = m[r][jj];
           if (bi == jb) {
-            float p = a[jj][jj];
+            float p = m[jj][jj];
             if (!(p > 0.f)) {
               report_status(status, SP_ERR_NOT_SPD, (int32_t)(row0 + j), 0);
               p = 1.f;
-              a[jj][jj] = 1.f;
-              colbuf[buf][j] = 1.f;
+              m[jj][jj] = 1.f;
             }
+            // reciprocal of the pivot: hardware approximation refined by one Newton step (error below 1 ulp)
+            float ip;
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ip) : "f"(p));
+            ip = fmaf(ip, fmaf(-p, ip, 1.f), ip);
+            wb[j] = ip;
             piv[j] = p;
           }
         }
-        if (active && bi == jb) {       // owners of row j of B
+        if (active && bi == jb) {       // owners of row j of B (columns left of j)
 #pragma unroll
-          for (int s = 0; s < 4; ++s) rowbuf[buf][4 * bj + s] = b[jj][s];
+          for (int s = 0; s < 4; ++s)
+            if (4 * bj + s < j) wb[4 * bj + s] = m[jj][s];
         }
         __syncthreads();
-        if (active && 4 * bi + 3 > j) {
-          const float inv = 1.f / colbuf[buf][j];
-          float cr[4], cc[4], rb[4];
+        if (active && 4 * bi + 3 >= j) {
+          const float inv = wb[j];
+          if (bj == jb) {               // column j is final: keep it for L, its registers now carry column j of B
 #pragma unroll
-          for (int r = 0; r < 4; ++r) cr[r] = colbuf[buf][4 * bi + r] * inv;
-#pragma unroll
-          for (int s = 0; s < 4; ++s) {
-            cc[s] = colbuf[buf][4 * bj + s];
-            rb[s] = rowbuf[buf][4 * bj + s];
+            for (int r = 0; r < 4; ++r) {
+              const int i = 4 * bi + r;
+              if (i >= j) {
+                lcol[r][jj] = m[r][jj];
+                m[r][jj] = (i == j) ? 1.f : 0.f;
+              }
+            }
           }
+          const float4 wr = *reinterpret_cast<const float4*>(&wb[4 * bi]);
+          const float4 wc = *reinterpret_cast<const float4*>(&wb[4 * bj]);
+          const float wrv[4] = {wr.x, wr.y, wr.z, wr.w}, wcv[4] = {wc.x, wc.y, wc.z, wc.w};
+          float cr[4], w[4];
+#pragma unroll
+          for (int r = 0; r < 4; ++r) cr[r] = (4 * bi + r > j) ? wrv[r] * inv : 0.f;
+#pragma unroll
+          for (int s = 0; s < 4; ++s) w[s] = (4 * bj + s == j) ? 1.f : wcv[s];
 #pragma unroll
           for (int r = 0; r < 4; ++r)
 #pragma unroll
-            for (int s = 0; s < 4; ++s) {
-              const int i = 4 * bi + r, c = 4 * bj + s;
-              if (i > j) {
-                if (c > j) a[r][s] -= cr[r] * cc[s];
-                else b[r][s] -= cr[r] * rb[s];
-              }
-            }
+            for (int s = 0; s < 4; ++s) m[r][s] = fmaf(-cr[r], w[s], m[r][s]);
         }
       }
     }
@@ -116,16 +134,14 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const int i = 4 * bi + r;
-      const float inv_sqrt_i = rsqrtf(piv[i]);
+      const float inv_sqrt_i = 1.f / sqrtf(piv[i]);
 #pragma unroll
       for (int s = 0; s < 4; ++s) {
         const int c = 4 * bj + s;
-        if (c <= i) {
-          if (i < nb) A[(int64_t)i * lda + c] = a[r][s] / sqrtf(piv[c]);
-          dinv[i * TB + c] = b[r][s] * inv_sqrt_i;
-        } else {
-          dinv[i * TB + c] = 0.f;
-        }
+        const float v = (c <= i) ? m[r][s] * inv_sqrt_i : 0.f;
+        dinv[i * TB + c] = v;
+        dinv[TB * TB + c * TB + i] = v;
+        if (c <= i && i < nb) A[(int64_t)i * lda + c] = lcol[r][s] / sqrtf(piv[c]);
       }
     }
   }
@@ -139,34 +155,61 @@ __device__ __forceinline__ void split3(float v, __nv_bfloat16& hi, __nv_bfloat16
   lo = __float2bfloat16_rn(r2);
 }
 
-constexpr int PA_ROWS = 64;
-constexpr int PA_THREADS = 256;
-constexpr size_t PA_SMEM = (size_t)(TB + PA_ROWS) * (TB + 1) * sizeof(float);
+constexpr int PA_ROWS = 32;
+constexpr int PA_THREADS = 128;
+constexpr int PA_APAD = PA_ROWS + 4;
+constexpr size_t PA_SMEM = ((size_t)TB * TB + (size_t)TB * PA_APAD) * sizeof(float);
 
 // X[i, 0:nb] <- X[i, 0:nb] inv(L)^T (TRANS == false) or X[i, 0:nb] inv(L) (TRANS == true), for `rows` rows.
-// dinv is the TB x TB block written by chol_diag128_kernel.  The result is written back in fp32 (write_f32) and as
-// three bf16 parts to S[i * lds + part * s_seg + c] for all TB columns (zero beyond nb).
+// dinv is the pair of TB x TB blocks written by chol_diag128_kernel.  The result is written back in fp32 (write_f32)
+// and as three bf16 parts to S[i * lds + part * s_seg + c] for all TB columns (zero beyond nb).
+// One CTA takes 32 rows; a thread computes 4 rows x 8 columns.
 template <bool TRANS>
 __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64_t ldx, int64_t rows, int nb,
                                                                  const float* __restrict__ dinv, __nv_bfloat16* S,
                                                                  int64_t lds, int64_t s_seg, int write_f32) {
-  extern __shared__ float pa_smem[];
-  float (*Lt)[TB + 1] = reinterpret_cast<float (*)[TB + 1]>(pa_smem);               // Lt[k][c]
-  float (*As)[TB + 1] = reinterpret_cast<float (*)[TB + 1]>(pa_smem + TB * (TB + 1));  // As[row][k]
+  extern __shared__ __align__(16) float pa_smem[];
+  float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(pa_smem);                       // Lt[k][c]
+  float (*At)[PA_APAD] = reinterpret_cast<float (*)[PA_APAD]>(pa_smem + TB * TB);   // At[k][row]
   const int t = threadIdx.x;
   const int64_t r0 = (int64_t)blockIdx.x * PA_ROWS;
-  for (int e = t; e < TB * TB; e += PA_THREADS) {
-    const int u = e / TB, v = e % TB;          // dinv[u][v], v contiguous
-    if (TRANS) Lt[u][v] = dinv[e];             // Lt[k][c] = inv(L)[k][c]
-    else Lt[v][u] = dinv[e];                   // Lt[k][c] = inv(L)[c][k]
-  }
-  for (int e = t; e < PA_ROWS * TB; e += PA_THREADS) {
-    const int i = e / TB, k = e % TB;
-    const int64_t gi = r0 + i;
-    As[i][k] = (gi < rows && k < nb) ? X[gi * ldx + k] : 0.f;
+  const bool x_al = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0);
+  {
+    // the rows of X first (the loads of all 8 float4 of a thread are in flight together) ...
+    float4 xv[PA_ROWS * TB / 4 / PA_THREADS];
+#pragma unroll
+    for (int q = 0; q < PA_ROWS * TB / 4 / PA_THREADS; ++q) {
+      const int e = t + q * PA_THREADS;
+      const int i = e / (TB / 4), k = (e % (TB / 4)) * 4;
+      const int64_t gi = r0 + i;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (gi < rows) {
+        const float* src = X + gi * ldx + k;
+        if (x_al && k + 4 <= nb) {
+          v = *reinterpret_cast<const float4*>(src);
+        } else {
+          if (k < nb) v.x = src[0];
+          if (k + 1 < nb) v.y = src[1];
+          if (k + 2 < nb) v.z = src[2];
+          if (k + 3 < nb) v.w = src[3];
+        }
+      }
+      xv[q] = v;
+    }
+    // ... then Lt[k][c] = inv(L)[c][k] (the transposed copy) or inv(L)[k][c]: a straight copy either way
+    const float4* src = reinterpret_cast<const float4*>(dinv + (TRANS ? 0 : TB * TB));
+    float4* dst = reinterpret_cast<float4*>(pa_smem);
+#pragma unroll 16
+    for (int e = t; e < TB * TB / 4; e += PA_THREADS) dst[e] = src[e];
+#pragma unroll
+    for (int q = 0; q < PA_ROWS * TB / 4 / PA_THREADS; ++q) {
+      const int e = t + q * PA_THREADS;
+      const int i = e / (TB / 4), k = (e % (TB / 4)) * 4;
+      At[k][i] = xv[q].x; At[k + 1][i] = xv[q].y; At[k + 2][i] = xv[q].z; At[k + 3][i] = xv[q].w;
+    }
   }
   __syncthreads();
-  const int tx = t & 15, ty = t >> 4;          // 16 column groups (columns tx + 16 j), 16 row groups of 4 rows
+  const int tx = t & 15, ty = t >> 4;          // columns 8 tx .. 8 tx + 7, rows 4 ty .. 4 ty + 3
   float acc[4][8];
 #pragma unroll
   for (int r = 0; r < 4; ++r)
@@ -174,33 +217,43 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
     for (int j = 0; j < 8; ++j) acc[r][j] = 0.f;
 #pragma unroll 4
   for (int k = 0; k < TB; ++k) {
-    float av[4], lv[8];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) av[r] = As[ty * 4 + r][k];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) lv[j] = Lt[k][tx + 16 * j];
+    const float4 a0 = *reinterpret_cast<const float4*>(&At[k][4 * ty]);
+    const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][8 * tx]);
+    const float4 l1 = *reinterpret_cast<const float4*>(&Lt[k][8 * tx + 4]);
+    const float av[4] = {a0.x, a0.y, a0.z, a0.w};
+    const float lv[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
   }
+  const int c0 = 8 * tx;
+  const bool x_vec = write_f32 && c0 + 8 <= nb && x_al;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
-    const int64_t gi = r0 + ty * 4 + r;
+    const int64_t gi = r0 + 4 * ty + r;
     if (gi >= rows) continue;
+    float v[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int c = tx + 16 * j;
-      const float v = (c < nb) ? acc[r][j] : 0.f;
-      if (write_f32 && c < nb) X[gi * ldx + c] = v;
-      if (S) {
-        __nv_bfloat16 hi, mid, lo;
-        split3(v, hi, mid, lo);
-        __nv_bfloat16* dst = S + gi * lds + c;
-        dst[0] = hi;
-        dst[s_seg] = mid;
-        dst[2 * s_seg] = lo;
+    for (int j = 0; j < 8; ++j) v[j] = (c0 + j < nb) ? acc[r][j] : 0.f;
+    if (write_f32) {
+      float* dst = X + gi * ldx + c0;
+      if (x_vec) {
+        *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (c0 + j < nb) dst[j] = v[j];
       }
+    }
+    if (S) {   // S + gi * lds + part * s_seg + c0 is 16-byte aligned by construction (lds, s_seg multiples of 8)
+      __align__(16) __nv_bfloat16 part[3][8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) split3(v[j], part[0][j], part[1][j], part[2][j]);
+#pragma unroll
+      for (int q = 0; q < 3; ++q)
+        *reinterpret_cast<uint4*>(S + gi * lds + q * s_seg + c0) = *reinterpret_cast<const uint4*>(part[q]);
     }
   }
 }
@@ -217,6 +270,7 @@ cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, cons
   }
   if (rows <= 0) return cudaSuccess;
   count_launch();
+  ProfScope prof(PK_PANEL_APPLY, 2.0 * (double)rows * TB * TB, 0.0, stream);
   panel_apply_kernel<TRANS><<<(unsigned)ceil_div(rows, PA_ROWS), PA_THREADS, PA_SMEM, stream>>>(
       X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0);
   return cudaGetLastError();
@@ -237,10 +291,13 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
   for (int64_t k0 = 0; k0 < n; k0 += TB) {
     const int nb = (int)((n - k0 < TB) ? (n - k0) : TB);
-    float* dk = dinv + (k0 / TB) * TB * TB;
-    count_launch();
-    chol_diag128_kernel<<<1, DIAG_THREADS, 0, stream>>>(A + k0 * lda + k0, lda, nb, dk, k0, status_dev);
-    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    float* dk = dinv + (k0 / TB) * 2 * TB * TB;
+    {
+      count_launch();
+      ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
+      chol_diag128_kernel<<<1, DIAG_THREADS, 0, stream>>>(A + k0 * lda + k0, lda, nb, dk, k0, status_dev);
+      if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    }
     const int64_t rem = n - k0 - nb;
     if (rem <= 0) break;
     // L21 = A21 inv(L11)^T, fp32 in place and as bf16 parts in P[k0+nb.., part * np + k0 ..]
@@ -277,7 +334,7 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
   // Y L^T = X, block columns left to right
   for (int64_t j0 = 0; j0 < n; j0 += TB) {
     const int nb = (int)((n - j0 < TB) ? (n - j0) : TB);
-    const float* dj = dinv + (j0 / TB) * TB * TB;
+    const float* dj = dinv + (j0 / TB) * 2 * TB * TB;
     if (launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xs, lds, TB, true, stream) != cudaSuccess) return SP_ERR_CUDA;
     const int64_t rem = n - j0 - nb;
     if (rem <= 0) break;
@@ -301,7 +358,7 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
   for (int64_t jb = nblk - 1; jb >= 0; --jb) {
     const int64_t j0 = jb * TB;
     const int nb = (int)((n - j0 < TB) ? (n - j0) : TB);
-    const float* dj = dinv + jb * TB * TB;
+    const float* dj = dinv + jb * 2 * TB * TB;
     if (launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xs, lds, TB, true, stream) != cudaSuccess) return SP_ERR_CUDA;
     if (j0 == 0) break;
     // X[:, :j0] -= W_j L[j0:j0+nb, :j0] : B(k, c) = L[j0 + k, c], rows of P with the columns (N) contiguous

@@ -7,14 +7,14 @@
 namespace sp {
 namespace {
 
-constexpr int kMaxSlots = 16384;
+constexpr int kMaxSlots = 65536;
 struct Slot {
   cudaEvent_t start, stop;
   int kind;
   double flops, bytes;
 };
 std::atomic<long long> g_launches{0};
-bool g_enabled = false;
+int g_enabled = 0;   // 0 off, 1 outermost scopes only, 2 every scope (nested ones are then counted twice)
 std::vector<Slot> g_slots;
 int g_used = 0;
 thread_local int g_depth = 0;
@@ -24,7 +24,8 @@ thread_local int g_depth = 0;
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 ProfScope::ProfScope(int kind, double flops, double bytes, cudaStream_t s) : slot(-1), stream(s) {
-  if (g_depth++ > 0 || !g_enabled || g_used >= kMaxSlots) return;
+  const bool nested = g_depth++ > 0;
+  if (!g_enabled || (nested && g_enabled < 2) || g_used >= kMaxSlots) return;
   if ((int)g_slots.size() <= g_used) {
     Slot sl;
     if (cudaEventCreate(&sl.start) != cudaSuccess || cudaEventCreate(&sl.stop) != cudaSuccess) return;
@@ -49,7 +50,7 @@ extern "C" {
 int64_t sp_launch_count(void) { return (int64_t)sp::g_launches.load(); }
 
 sp_status sp_profile_begin(int32_t enable) {
-  sp::g_enabled = enable != 0;
+  sp::g_enabled = enable;
   sp::g_used = 0;
   sp::g_launches.store(0);
   return SP_OK;
@@ -59,7 +60,8 @@ int32_t sp_profile_kinds(void) { return sp::PK_COUNT; }
 
 const char* sp_profile_kind_name(int32_t kind) {
   static const char* names[sp::PK_COUNT] = {"gemm_tc", "gemm_simt", "solve_phase", "fused_update", "prep_h",
-                                            "scores", "topk_select", "elementwise", "allocate"};
+                                            "scores", "topk_select", "elementwise", "allocate", "chol_diag",
+                                            "panel_apply"};
   return (kind >= 0 && kind < sp::PK_COUNT) ? names[kind] : "unknown";
 }
 
