@@ -67,7 +67,11 @@ sp_status contract_split_weights(int64_t M, int64_t N, int64_t K, MatRef A, cons
     sg.b_k[1] = (int32_t)kp;
     return gemm_tc(M, N, K, 1.f, ta, tb, 0.f, cin, out, false, status, stream, &sg, 2.0 * (double)M * N * K);
   }
-  return contract(M, N, K, 1.0, A, true, Wf32, true, 0.0, C, C, false, false, false, status, stream);
+  if (Wf32.ptr) return contract(M, N, K, 1.0, A, true, Wf32, true, 0.0, C, C, false, false, false, status, stream);
+  // no fp32 copy at hand: hi and lo parts one after the other on the CUDA cores
+  MatRef hi{Wsplit, SP_BF16, 2 * kp}, lo{reinterpret_cast<const __nv_bfloat16*>(Wsplit) + kp, SP_BF16, 2 * kp};
+  SPCHK(contract(M, N, K, 1.0, A, true, hi, true, 0.0, C, C, false, false, false, status, stream));
+  return contract(M, N, K, 1.0, A, true, lo, true, 1.0, C, C, false, false, false, status, stream);
 }
 
 struct Carver {
@@ -166,7 +170,10 @@ struct AdmmPlan {
   // device buffers
   SolveBufs sb;
   float *W1t, *W2t, *Qt, *T0, *Cf;
-  void *W1b, *W2b, *Qtb;       // storage-dtype copies (bf16 mode only)
+  float *W2cf, *W1c;           // compact fp32 copies on the kept support: W2[:, S] ([d, kp]) and W1[S, :] ([k, d])
+  int32_t* grp_base;           // kept-channel map of the elementwise kernels
+  uint8_t* grp_mask;
+  void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
   void *H, *E, *Ac, *Zb;
   float *D, *z1;
   double *partial, *absA_part, *score_scratch;
@@ -192,15 +199,20 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.Qt = c.take<float>((size_t)n * d);
   p.T0 = c.take<float>((size_t)n * d);
   p.Cf = c.take<float>((size_t)d * d);
+  p.W2cf = c.take<float>((size_t)n * d + 8 * (size_t)d);
+  p.W1c = p.bf16 ? nullptr : c.take<float>((size_t)n * d);
+  p.grp_base = c.take<int32_t>((size_t)ceil_div(n, (int64_t)8));
+  p.grp_mask = c.take<uint8_t>((size_t)ceil_div(n, (int64_t)8));
   p.W1b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // hi | lo split of W1
-  p.W2b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.W2b = p.bf16 ? c.take_bytes(((size_t)n + 8) * d * csz) : nullptr;
   p.Qtb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
-  p.H = c.take_bytes((size_t)p.chunk * n * csz);
+  const size_t npad = (size_t)(n + 7) / 8 * 8;   // leading dimension bound of the compact tensors
+  p.H = c.take_bytes((size_t)p.chunk * npad * csz);
   p.E = c.take_bytes((size_t)p.chunk * d * csz);
   p.Ac = c.take_bytes((size_t)p.chunk * n * csz);
   p.Zb = p.bf16 ? c.take_bytes((size_t)p.chunk * n * csz) : nullptr;
-  p.D = c.take<float>((size_t)p.chunk * n);
-  p.z1 = c.take<float>((size_t)p.chunk * n);
+  p.D = c.take<float>((size_t)p.chunk * npad);
+  p.z1 = c.take<float>((size_t)p.chunk * npad);
   p.nblocks = fused_update_grid(p.chunk, n, &p.row_blocks);
   p.partial = c.take<double>((size_t)p.nblocks * 3);
   p.absA_part = c.take<double>((size_t)p.row_blocks * n);
@@ -493,7 +505,7 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   const bool acc64 = !bf16;
   MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, w20{m->W2_0.ptr, SP_F32, m->W2_0.ld};
   if (bf16) {
-    CU(split_bf16(reinterpret_cast<const float*>(m->W1_0.ptr), m->W1_0.ld, n, d, split_kpad(d), p.W10b, s));
+    CU(split_bf16(reinterpret_cast<const float*>(m->W1_0.ptr), m->W1_0.ld, nullptr, n, d, split_kpad(d), p.W10b, s));
     CU(convert_matrix(m->W2_0.ptr, SP_F32, m->W2_0.ld, p.W20b, SP_BF16, n, d, n, s));
     w20 = MatRef{p.W20b, SP_BF16, n};
   }
@@ -589,38 +601,45 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     CU(zero_pruned(st->mask, 1, nullptr, 0, 0, 0, st->W2, d, n, n, s));
   }
 
-  // ---- 5a. operands of the a-update: C = gamma I + W2 W2^T (d x d), Qt = W2^T C^-1 (n x d)
-  MatRef w1{st->W1, SP_F32, d}, w2{st->W2, SP_F32, n}, qt{p.Qt, SP_F32, d};
+  // ---- 5a. operands of the token pass, all on the kept support S (k channels, compact, ascending channel order):
+  //      W1[S, :], W2[:, S], C = gamma I + W2 W2^T (d x d), Qt = W2[:, S]^T C^-1 (k x d)
+  const int64_t kp = (k + 7) / 8 * 8;            // leading dimension of the compact [., k] tensors
+  const int32_t* idx = p.sb.idx;
+  CU(build_group_map(st->mask, n, p.grp_base, p.grp_mask, s));
+  CU(gather_cols<float>(st->W2, n, idx, d, k, p.W2cf, kp, s));
+  MatRef w1{nullptr, SP_F32, d}, w2{p.W2cf, SP_F32, kp}, qt{p.Qt, SP_F32, d};
   if (bf16) {
-    CU(split_bf16(st->W1, d, n, d, split_kpad(d), p.W1b, s));
-    CU(convert_matrix(st->W2, SP_F32, n, p.W2b, SP_BF16, n, d, n, s));
-    w2 = MatRef{p.W2b, SP_BF16, n};
+    CU(split_bf16(st->W1, d, idx, k, d, split_kpad(d), p.W1b, s));
+    CU(convert_matrix(p.W2cf, SP_F32, kp, p.W2b, SP_BF16, kp, d, k, s));
+    w2 = MatRef{p.W2b, SP_BF16, kp};
+  } else {
+    CU(gather_rows(st->W1, d, idx, k, d, p.W1c, d, s));
+    w1 = MatRef{p.W1c, SP_F32, d};
   }
   {
     MatRef cf{p.Cf, SP_F32, d};
-    SPCHK(contract(d, d, n, 1.0, w2, true, w2, true, 0.0, cf, cf, true, acc64, bf16, status_dev, s));
+    SPCHK(contract(d, d, k, 1.0, w2, true, w2, true, 0.0, cf, cf, true, acc64, bf16, status_dev, s));
     CU(effective_ridge(nullptr, 0, 1, prm->beta / prm->alpha, 0, gam, s));
-    ProfScope prof(PK_SOLVE, (double)d * d * d / 3.0 + 2.0 * (double)n * d * d, 0.0, s);
+    ProfScope prof(PK_SOLVE, (double)d * d * d / 3.0 + 2.0 * (double)k * d * d, 0.0, s);
     if (bf16) {
       float* Gs = reinterpret_cast<float*>(p.sb.Gs);
       float* Rs = reinterpret_cast<float*>(p.sb.Rs);
       CU(load_spd<float>(p.Cf, d, d, gam, Gs, d, s));
       SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s));
-      // right-hand sides: the rows of W2^T as the tensor-core path sees them (bf16-rounded W2)
-      CU(convert_matrix(p.W2b, SP_BF16, n, p.W2t, SP_F32, n, d, n, s));
-      CU(transpose_convert<float>(p.W2t, n, d, n, Rs, d, s));
-      SPCHK(potrs_right_tc(Rs, n, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s));
-      CU(convert_matrix(Rs, SP_F32, d, p.Qt, SP_F32, d, n, d, s));
-      CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, n, d, s));
+      // right-hand sides: the rows of W2[:, S]^T as the tensor-core path sees them (bf16-rounded)
+      CU(convert_matrix(p.W2b, SP_BF16, kp, p.W2cf, SP_F32, kp, d, k, s));
+      CU(transpose_convert<float>(p.W2cf, kp, d, k, Rs, d, s));
+      SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s));
+      CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));
       qt = MatRef{p.Qtb, SP_BF16, d};
     } else {
       double* Gs = reinterpret_cast<double*>(p.sb.Gs);
       double* Rs = reinterpret_cast<double*>(p.sb.Rs);
       CU(load_spd<double>(p.Cf, d, d, gam, Gs, d, s));
       CU(potrf_lower<double>(Gs, d, d, reinterpret_cast<double*>(p.sb.dinv), status_dev, s));
-      CU(transpose_convert<double>(st->W2, n, d, n, Rs, d, s));
-      CU(potrs_right<double>(Rs, n, d, d, Gs, d, reinterpret_cast<double*>(p.sb.dinv), s));
-      CU(convert_matrix(Rs, SP_F64, d, p.Qt, SP_F32, d, n, d, s));
+      CU(transpose_convert<double>(p.W2cf, kp, d, k, Rs, d, s));
+      CU(potrs_right<double>(Rs, k, d, d, Gs, d, reinterpret_cast<double*>(p.sb.dinv), s));
+      CU(convert_matrix(Rs, SP_F64, d, p.Qt, SP_F32, d, k, d, s));
     }
   }
 
@@ -635,16 +654,17 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     MatRef yc{reinterpret_cast<const uint8_t*>(m->Ypre.ptr) + (size_t)t0 * m->Ypre.ld * esz, cdt, m->Ypre.ld};
     float* Zc = st->Z + (size_t)t0 * n;
     float* Uc = (prm->dual_mode && st->U) ? st->U + (size_t)t0 * n : nullptr;
-    MatRef h{p.H, cdt, n}, e{p.E, cdt, d}, dd{p.D, SP_F32, n}, z1{p.z1, SP_F32, n}, ac{p.Ac, cdt, n};
+    MatRef h{p.H, cdt, kp}, e{p.E, cdt, d}, dd{p.D, SP_F32, kp}, z1{p.z1, SP_F32, kp}, ac{p.Ac, cdt, n};
     MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : MatRef{Zc, SP_F32, n};
-    CU(launch_prep_h(Zc, Uc, p.H, cdt, Tc, n, s));
-    // E = Ypre - h W2^T ; D = E Qt^T ; z1 = X W1^T
-    SPCHK(contract(Tc, d, n, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
-    SPCHK(contract(Tc, n, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
-    if (bf16) SPCHK(contract_split_weights(Tc, n, d, xc, p.W1b, w1, z1, status_dev, s));
-    else SPCHK(contract(Tc, n, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, false, status_dev, s));
+    CU(launch_prep_h(Zc, Uc, p.H, cdt, Tc, n, kp, k, p.grp_base, p.grp_mask, s));
+    // E = Ypre - h_S W2[:, S]^T ; D_S = E Qt^T ; z1_S = X W1[S, :]^T
+    SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
+    SPCHK(contract(Tc, k, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
+    if (bf16) SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, w1, z1, status_dev, s));
+    else SPCHK(contract(Tc, k, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, false, status_dev, s));
     UpdateArgs ua;
-    ua.Z = Zc; ua.U = Uc; ua.z1 = p.z1; ua.D = p.D; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
+    ua.Z = Zc; ua.U = Uc; ua.z1 = p.z1; ua.D = p.D; ua.ldk = kp; ua.k = k; ua.grp_base = p.grp_base;
+    ua.grp_mask = p.grp_mask; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
     ua.out_dtype = cdt; ua.T = Tc; ua.n = n; ua.alpha = (float)prm->alpha; ua.beta = (float)prm->beta;
     ua.z_rule = prm->z_rule; ua.partial = p.partial; ua.absA_part = p.absA_part;
     const int nblk = fused_update_grid(Tc, n, &ua.row_blocks);

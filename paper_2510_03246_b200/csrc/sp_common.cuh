@@ -114,8 +114,9 @@ cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst,
 cudaError_t symmetrize_lower(float* G, int64_t n, int64_t ld, cudaStream_t stream);
 // dst[i, 0:cols] = bf16(src[i,:]) and dst[i, kpad:kpad+cols] = bf16(src - hi); padding columns are zero.
 // dst is [rows, 2*kpad] bf16.
-cudaError_t split_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad, void* dst,
-                       cudaStream_t stream);
+// row_idx != nullptr: row i of dst comes from row row_idx[i] of src.
+cudaError_t split_bf16(const float* src, int64_t lds, const int32_t* row_idx, int64_t rows, int64_t cols, int64_t kpad,
+                       void* dst, cudaStream_t stream);
 // dst[j, i] = (TD) src[i, j]
 template <typename TD>
 cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64_t cols, TD* dst, int64_t ldd,
@@ -134,6 +135,9 @@ cudaError_t load_spd_gather(const float* G, int64_t ldg, const int32_t* idx, int
 template <typename T>
 cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
                         int64_t ldd, cudaStream_t stream);
+// dst[i, :] = src[idx[i], :]
+cudaError_t gather_rows(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t cols, float* dst,
+                        int64_t ldd, cudaStream_t stream);
 // dst (fp32, [rows, n]) = 0 ; dst[i, idx[a]] = src[i, a]
 template <typename T>
 cudaError_t scatter_cols(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, int64_t n,
@@ -145,8 +149,11 @@ cudaError_t effective_ridge(const float* G, int64_t ldg, int64_t n, double rho, 
 struct UpdateArgs {
   float* Z;          // [T, n] in/out
   float* U;          // [T, n] in/out or null
-  const float* z1;   // [T, n]
-  const float* D;    // [T, n] correction term of the a-update
+  const float* z1;   // [T, ldk] compact on the kept channels
+  const float* D;    // [T, ldk] compact: correction term of the a-update
+  int64_t ldk, k;    // leading dimension of the compact tensors, number of kept channels
+  const int32_t* grp_base;   // per group of 8 channels: kept channels before the group
+  const uint8_t* grp_mask;   // per group of 8 channels: bit q = channel 8 g + q is kept
   void* A_out;       // [T, n] storage dtype
   void* Zb_out;      // [T, n] storage dtype copy of Z_new
   int32_t out_dtype;
@@ -157,8 +164,11 @@ struct UpdateArgs {
   double* absA_part; // [row_blocks, n] partial column sums of |A|
   int32_t row_blocks;
 };
-cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n,
-                          cudaStream_t stream);
+// grp_base / grp_mask of a u8 mask over n channels (see sp_elementwise.cu)
+cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream);
+// H[T, ldh] (compact on the k kept channels) = storage(phi(Z) - U)
+cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n, int64_t ldh,
+                          int64_t k, const int32_t* grp_base, const uint8_t* grp_mask, cudaStream_t stream);
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]

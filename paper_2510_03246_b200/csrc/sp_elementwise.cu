@@ -69,14 +69,14 @@ __global__ void transpose_convert_kernel(const float* src, int64_t lds, int64_t 
   }
 }
 
-__global__ void split_bf16_kernel(const float* __restrict__ src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad,
-                                  __nv_bfloat16* __restrict__ dst) {
+__global__ void split_bf16_kernel(const float* __restrict__ src, int64_t lds, const int32_t* __restrict__ row_idx,
+                                  int64_t rows, int64_t cols, int64_t kpad, __nv_bfloat16* __restrict__ dst) {
   const int64_t total = rows * kpad;
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t i = e / kpad, j = e % kpad;
     __nv_bfloat16 hi = __float2bfloat16_rn(0.f), lo = hi;
     if (j < cols) {
-      const float v = src[i * lds + j];
+      const float v = src[(row_idx ? (int64_t)row_idx[i] : i) * lds + j];
       hi = __float2bfloat16_rn(v);
       lo = __float2bfloat16_rn(v - __bfloat162float(hi));
     }
@@ -129,6 +129,15 @@ __global__ void gather_cols_kernel(const float* src, int64_t lds, const int32_t*
   }
 }
 
+__global__ void gather_rows_kernel(const float* __restrict__ src, int64_t lds, const int32_t* __restrict__ idx,
+                                   int64_t rows, int64_t cols, float* __restrict__ dst, int64_t ldd) {
+  const int64_t total = rows * cols;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / cols, j = e % cols;
+    dst[i * ldd + j] = src[(int64_t)idx[i] * lds + j];
+  }
+}
+
 template <typename T>
 __global__ void scatter_cols_kernel(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k,
                                     float* dst, int64_t ldd) {
@@ -155,46 +164,90 @@ __global__ void effective_ridge_kernel(const float* G, int64_t ldg, int64_t n, d
 }
 
 // ------------------------------------------------------------------------------------------------ chunk kernels
-// H = storage(phi(Z) - U)
-__global__ void prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U, void* H, int32_t hdt,
-                              int64_t total) {
-  for (int64_t e = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; e < total;
-       e += (int64_t)gridDim.x * blockDim.x * 4) {
-    if (e + 3 < total) {
-      const float4 z = *reinterpret_cast<const float4*>(Z + e);
-      float4 h = make_float4(fmaxf(z.x, 0.f), fmaxf(z.y, 0.f), fmaxf(z.z, 0.f), fmaxf(z.w, 0.f));
-      if (U) {
-        const float4 u = *reinterpret_cast<const float4*>(U + e);
-        h.x -= u.x; h.y -= u.y; h.z -= u.z; h.w -= u.w;
-      }
-      if (hdt == SP_BF16) {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(h.x, h.y), hi = __floats2bfloat162_rn(h.z, h.w);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(H) + e) = pk;
-      } else {
-        *reinterpret_cast<float4*>(reinterpret_cast<float*>(H) + e) = h;
-      }
-    } else {
-      for (int64_t q = e; q < total; ++q) {
-        float h = fmaxf(Z[q], 0.f) - (U ? U[q] : 0.f);
-        if (hdt == SP_BF16) reinterpret_cast<__nv_bfloat16*>(H)[q] = __float2bfloat16_rn(h);
-        else reinterpret_cast<float*>(H)[q] = h;
-      }
+// The kept units of a module are a subset S of its n channels.  Tensors that exist only on S are stored COMPACT:
+// column p of a compact [T, k] tensor belongs to channel idx[p] (idx ascending).  For the elementwise kernels the
+// channels are cut into groups of 8 consecutive ones: grp_base[g] = number of kept channels before channel 8 g,
+// grp_mask[g] = bit q set when channel 8 g + q is kept.  The kept channels of a group then sit at compact positions
+// grp_base[g], grp_base[g] + 1, ... in channel order.
+__global__ void __launch_bounds__(1024) group_map_kernel(const uint8_t* __restrict__ mask, int64_t n,
+                                                         int32_t* grp_base, uint8_t* grp_mask) {
+  __shared__ int warp_tot[32];
+  __shared__ int s_before;
+  const int64_t groups = ceil_div(n, (int64_t)8);
+  if (threadIdx.x == 0) s_before = 0;
+  __syncthreads();
+  for (int64_t g0 = 0; g0 < groups; g0 += blockDim.x) {
+    const int64_t g = g0 + threadIdx.x;
+    unsigned bits = 0;
+    if (g < groups)
+      for (int q = 0; q < 8; ++q)
+        if (8 * g + q < n && mask[8 * g + q]) bits |= 1u << q;
+    const int cnt = __popc(bits);
+    // inclusive scan of cnt over the block
+    int v = cnt;
+    const int l = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, v, o);
+      if (l >= o) v += u;
     }
+    if (l == 31) warp_tot[w] = v;
+    __syncthreads();
+    int before = s_before;
+    for (int i = 0; i < w; ++i) before += warp_tot[i];
+    if (g < groups) {
+      grp_base[g] = before + v - cnt;
+      grp_mask[g] = (uint8_t)bits;
+    }
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) s_before = before + v;
+    __syncthreads();
   }
 }
 
-__device__ __forceinline__ void store4(void* base, int32_t dt, int64_t e, float a, float b, float c, float d) {
-  if (dt == SP_BF16) {
-    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-    uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(base) + e) = pk;
-  } else {
-    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e) = make_float4(a, b, c, d);
+// H_S = storage(phi(Z) - U) on the kept channels, compact [T, ldh].  One thread per group of 8 channels and row.
+__global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U, void* H,
+                                                     int32_t hdt, int64_t T, int64_t n, int64_t ldh,
+                                                     const int32_t* __restrict__ grp_base,
+                                                     const uint8_t* __restrict__ grp_mask, int32_t rows_per_block) {
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t c0 = g * 8;
+  if (c0 >= n) return;
+  const unsigned bits = grp_mask[g];
+  if (bits == 0) return;
+  const int base = grp_base[g];
+  const bool vec = (n % 4 == 0) && c0 + 8 <= n;
+  const int64_t r_begin = (int64_t)blockIdx.y * rows_per_block;
+  const int64_t r_end = (r_begin + rows_per_block < T) ? r_begin + rows_per_block : T;
+#pragma unroll 2
+  for (int64_t r = r_begin; r < r_end; ++r) {
+    const int64_t e = r * n + c0;
+    float h[8];
+    if (vec) {
+      const float4 z0 = *reinterpret_cast<const float4*>(Z + e), z1 = *reinterpret_cast<const float4*>(Z + e + 4);
+      h[0] = fmaxf(z0.x, 0.f); h[1] = fmaxf(z0.y, 0.f); h[2] = fmaxf(z0.z, 0.f); h[3] = fmaxf(z0.w, 0.f);
+      h[4] = fmaxf(z1.x, 0.f); h[5] = fmaxf(z1.y, 0.f); h[6] = fmaxf(z1.z, 0.f); h[7] = fmaxf(z1.w, 0.f);
+      if (U) {
+        const float4 u0 = *reinterpret_cast<const float4*>(U + e), u1 = *reinterpret_cast<const float4*>(U + e + 4);
+        h[0] -= u0.x; h[1] -= u0.y; h[2] -= u0.z; h[3] -= u0.w;
+        h[4] -= u1.x; h[5] -= u1.y; h[6] -= u1.z; h[7] -= u1.w;
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        h[q] = 0.f;
+        if (c0 + q < n) h[q] = fmaxf(Z[e + q], 0.f) - (U ? U[e + q] : 0.f);
+      }
+    }
+    int pos = base;
+    const int64_t ho = r * ldh;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (bits & (1u << q)) {
+        if (hdt == SP_BF16) reinterpret_cast<__nv_bfloat16*>(H)[ho + pos] = __float2bfloat16_rn(h[q]);
+        else reinterpret_cast<float*>(H)[ho + pos] = h[q];
+        ++pos;
+      }
+    }
   }
 }
 
@@ -217,58 +270,99 @@ __device__ __forceinline__ float update_one(float zold, float z1, float dcorr, f
   return a;
 }
 
-// grid: (col blocks of 1024, row blocks).  Thread owns 4 consecutive columns and walks its block's rows.
+__device__ __forceinline__ void store8(void* base, int32_t dt, int64_t e, const float* v) {
+  if (dt == SP_BF16) {
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(v[4], v[5]), h3 = __floats2bfloat162_rn(v[6], v[7]);
+    uint4 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
+    pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
+    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(base) + e) = pk;
+  } else {
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+// The fused auxiliary-variable update of one chunk: per element a = h + D (h = phi(z) - u), z2, the select, the dual
+// update, the residual / norm partial sums and the column sums of |a|, reading Z (and U) once and writing Z (and U),
+// A and the storage copy of Z once.  D and z1 exist on the kept channels only (compact, see above); on a pruned
+// channel both are zero (its row of W1 and its row of Q are zero).
+// grid: (column blocks of 2048 channels, row blocks).  A thread owns 8 consecutive channels and walks its rows.
 __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   __shared__ double sm[32];
-  const int64_t c0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+  const int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int64_t c0 = grp * 8;
   const int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
   const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
   const int64_t r_end = (r_begin + rows_per < g.T) ? r_begin + rows_per : g.T;
   const bool has_u = g.U != nullptr;
   const float inv_ab = 1.f / (g.alpha + g.beta);
   double s_res = 0.0, s_z = 0.0, s_a = 0.0;
-  double cs[4] = {0.0, 0.0, 0.0, 0.0};
-  const bool vec = (g.n % 4 == 0);
+  double cs[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
   if (c0 < g.n) {
+    const int cnt = (g.n - c0 >= 8) ? 8 : (int)(g.n - c0);
+    const bool vec = (g.n % 8 == 0);
+    const unsigned bits = g.grp_mask[grp];
+    const int base = g.grp_base[grp];
     for (int64_t r = r_begin; r < r_end; ++r) {
       const int64_t e = r * g.n + c0;
-      float zo[4], z1[4], dc[4], u[4] = {0.f, 0.f, 0.f, 0.f}, a[4], zn[4];
-      const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
+      float zo[8], u[8], z1[8], dc[8], a[8], zn[8];
       if (vec) {
-        const float4 v0 = *reinterpret_cast<const float4*>(g.Z + e);
-        const float4 v1 = *reinterpret_cast<const float4*>(g.z1 + e);
-        const float4 v2 = *reinterpret_cast<const float4*>(g.D + e);
-        zo[0] = v0.x; zo[1] = v0.y; zo[2] = v0.z; zo[3] = v0.w;
-        z1[0] = v1.x; z1[1] = v1.y; z1[2] = v1.z; z1[3] = v1.w;
-        dc[0] = v2.x; dc[1] = v2.y; dc[2] = v2.z; dc[3] = v2.w;
+        const float4 v0 = *reinterpret_cast<const float4*>(g.Z + e), v1 = *reinterpret_cast<const float4*>(g.Z + e + 4);
+        zo[0] = v0.x; zo[1] = v0.y; zo[2] = v0.z; zo[3] = v0.w; zo[4] = v1.x; zo[5] = v1.y; zo[6] = v1.z; zo[7] = v1.w;
         if (has_u) {
-          const float4 v3 = *reinterpret_cast<const float4*>(g.U + e);
-          u[0] = v3.x; u[1] = v3.y; u[2] = v3.z; u[3] = v3.w;
+          const float4 w0 = *reinterpret_cast<const float4*>(g.U + e), w1 = *reinterpret_cast<const float4*>(g.U + e + 4);
+          u[0] = w0.x; u[1] = w0.y; u[2] = w0.z; u[3] = w0.w; u[4] = w1.x; u[5] = w1.y; u[6] = w1.z; u[7] = w1.w;
         }
       } else {
-        for (int q = 0; q < cnt; ++q) {
-          zo[q] = g.Z[e + q]; z1[q] = g.z1[e + q]; dc[q] = g.D[e + q];
-          if (has_u) u[q] = g.U[e + q];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          zo[q] = (q < cnt) ? g.Z[e + q] : 0.f;
+          if (has_u) u[q] = (q < cnt) ? g.U[e + q] : 0.f;
+        }
+      }
+      if (!has_u) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) u[q] = 0.f;
+      }
+      {
+        const float* zp = g.z1 + r * g.ldk + base;
+        const float* dp = g.D + r * g.ldk + base;
+        int pos = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          z1[q] = 0.f;
+          dc[q] = 0.f;
+          if (bits & (1u << q)) {
+            z1[q] = zp[pos];
+            dc[q] = dp[pos];
+            ++pos;
+          }
         }
       }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < 8; ++q) {
         if (q < cnt) {
           a[q] = update_one(zo[q], z1[q], dc[q], u[q], has_u, g.alpha, g.beta, inv_ab, g.z_rule, zn[q]);
-          const double diff = (double)a[q] - (double)fmaxf(zn[q], 0.f);
-          s_res += diff * diff;
+          const float diff = a[q] - fmaxf(zn[q], 0.f);
+          s_res += (double)diff * (double)diff;
           s_z += (double)zn[q] * (double)zn[q];
           s_a += (double)a[q] * (double)a[q];
-          cs[q] += fabs((double)a[q]);
+          cs[q] += (double)fabsf(a[q]);
         } else {
           a[q] = 0.f; zn[q] = 0.f;
         }
       }
       if (vec) {
         *reinterpret_cast<float4*>(g.Z + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
-        if (has_u) *reinterpret_cast<float4*>(g.U + e) = make_float4(u[0], u[1], u[2], u[3]);
-        store4(g.A_out, g.out_dtype, e, a[0], a[1], a[2], a[3]);
-        if (g.Zb_out) store4(g.Zb_out, g.out_dtype, e, zn[0], zn[1], zn[2], zn[3]);
+        *reinterpret_cast<float4*>(g.Z + e + 4) = make_float4(zn[4], zn[5], zn[6], zn[7]);
+        if (has_u) {
+          *reinterpret_cast<float4*>(g.U + e) = make_float4(u[0], u[1], u[2], u[3]);
+          *reinterpret_cast<float4*>(g.U + e + 4) = make_float4(u[4], u[5], u[6], u[7]);
+        }
+        store8(g.A_out, g.out_dtype, e, a);
+        if (g.Zb_out) store8(g.Zb_out, g.out_dtype, e, zn);
       } else {
         for (int q = 0; q < cnt; ++q) {
           g.Z[e + q] = zn[q];
@@ -283,10 +377,8 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
         }
       }
     }
-    if (g.absA_part) {
-      const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
+    if (g.absA_part)
       for (int q = 0; q < cnt; ++q) g.absA_part[(int64_t)blockIdx.y * g.n + c0 + q] = cs[q];
-    }
   }
   const int64_t bid = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
   const double r0 = block_sum<double>(s_res, sm);
@@ -427,12 +519,12 @@ template cudaError_t transpose_convert<double>(const float*, int64_t, int64_t, i
 template cudaError_t transpose_convert<__nv_bfloat16>(const float*, int64_t, int64_t, int64_t, __nv_bfloat16*,
                                                       int64_t, cudaStream_t);
 
-cudaError_t split_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad, void* dst,
-                       cudaStream_t stream) {
+cudaError_t split_bf16(const float* src, int64_t lds, const int32_t* row_idx, int64_t rows, int64_t cols, int64_t kpad,
+                       void* dst, cudaStream_t stream) {
   if (rows * kpad == 0) return cudaSuccess;
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  split_bf16_kernel<<<grid_for(rows * kpad, 256), 256, 0, stream>>>(src, lds, rows, cols, kpad,
+  split_bf16_kernel<<<grid_for(rows * kpad, 256), 256, 0, stream>>>(src, lds, row_idx, rows, cols, kpad,
                                                                      reinterpret_cast<__nv_bfloat16*>(dst));
   return cudaGetLastError();
 }
@@ -473,6 +565,15 @@ cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64
   gather_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
   return cudaGetLastError();
 }
+cudaError_t gather_rows(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t cols, float* dst,
+                        int64_t ldd, cudaStream_t stream) {
+  if (rows * cols == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
+  gather_rows_kernel<<<grid_for(rows * cols, 256), 256, 0, stream>>>(src, lds, idx, rows, cols, dst, ldd);
+  return cudaGetLastError();
+}
+
 template <typename T>
 cudaError_t scatter_cols(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, int64_t n,
                          float* dst, int64_t ldd, cudaStream_t stream) {
@@ -507,19 +608,35 @@ cudaError_t effective_ridge(const float* G, int64_t ldg, int64_t n, double rho, 
   return cudaGetLastError();
 }
 
-cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n,
-                          cudaStream_t stream) {
-  const int64_t total = T * n;
-  if (total == 0) return cudaSuccess;
-  ProfScope prof(PK_PREP_H, 0.0, (double)total * ((U ? 8.0 : 4.0) + (hdt == SP_BF16 ? 2.0 : 4.0)), stream);
+cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream) {
+  if (n == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  prep_h_kernel<<<grid_for(total, 256, 4), 256, 0, stream>>>(Z, U, H, hdt, total);
+  group_map_kernel<<<1, 1024, 0, stream>>>(mask, n, grp_base, grp_mask);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n, int64_t ldh,
+                          int64_t k, const int32_t* grp_base, const uint8_t* grp_mask, cudaStream_t stream) {
+  if (T * n == 0) return cudaSuccess;
+  // algorithmic bytes: Z (and U) read once, the kept part written once
+  ProfScope prof(PK_PREP_H, 0.0, (double)T * ((double)n * (U ? 8.0 : 4.0) + (double)k * (hdt == SP_BF16 ? 2.0 : 4.0)),
+                 stream);
+  const int64_t groups = ceil_div(n, (int64_t)8);
+  const unsigned gx = (unsigned)ceil_div(groups, (int64_t)256);
+  int64_t rb = ceil_div((int64_t)148 * 8, (int64_t)gx);
+  if (rb > T) rb = T;
+  if (rb > 65535) rb = 65535;
+  const int32_t rows_per = (int32_t)ceil_div(T, rb);
+  count_launch();
+  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, H, hdt, T, n, ldh, grp_base,
+                                                                                        grp_mask, rows_per);
   return cudaGetLastError();
 }
 
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
-  const int col_blocks = (int)ceil_div(n, 1024);
-  int rb = (148 * 4 + col_blocks - 1) / col_blocks;
+  const int col_blocks = (int)ceil_div(n, 2048);
+  int rb = (148 * 8 + col_blocks - 1) / col_blocks;
   if (rb > T) rb = (int)T;
   if (rb < 1) rb = 1;
   if (rb > 65535) rb = 65535;
@@ -529,11 +646,12 @@ int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
 
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   if (a.T * a.n == 0) return cudaSuccess;
-  dim3 grid((unsigned)ceil_div(a.n, 1024), (unsigned)a.row_blocks);
-  // algorithmic bytes per element: read Z, z1, D (+U); write Z (+U), A and the storage copy of Z
+  dim3 grid((unsigned)ceil_div(a.n, 2048), (unsigned)a.row_blocks);
+  // algorithmic bytes per row: Z (and U) read and written, A and the storage copy of Z written, z1 and D read on the
+  // kept channels
   const double esz = a.out_dtype == SP_BF16 ? 2.0 : 4.0;
-  const double per = 12.0 + 4.0 + (a.U ? 8.0 : 0.0) + esz + (a.Zb_out ? esz : 0.0);
-  ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * (double)a.n * per, stream);
+  const double per_n = 8.0 + (a.U ? 8.0 : 0.0) + esz + (a.Zb_out ? esz : 0.0);
+  ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * ((double)a.n * per_n + (double)a.k * 8.0), stream);
   count_launch();
   fused_update_kernel<<<grid, 256, 0, stream>>>(a);
   return cudaGetLastError();
