@@ -656,7 +656,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     float* Uc = (prm->dual_mode && st->U) ? st->U + (size_t)t0 * n : nullptr;
     MatRef h{p.H, cdt, kp}, e{p.E, cdt, d}, dd{p.D, SP_F32, kp}, z1{p.z1, SP_F32, kp}, ac{p.Ac, cdt, n};
     MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : MatRef{Zc, SP_F32, n};
-    CU(launch_prep_h(Zc, Uc, p.H, cdt, Tc, n, kp, k, p.grp_base, p.grp_mask, s));
+    CU(launch_prep_h(Zc, Uc, p.H, cdt, Tc, n, kp, k, idx, s));
     // E = Ypre - h_S W2[:, S]^T ; D_S = E Qt^T ; z1_S = X W1[S, :]^T
     SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
     SPCHK(contract(Tc, k, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));

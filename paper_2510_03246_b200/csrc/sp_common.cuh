@@ -166,9 +166,9 @@ struct UpdateArgs {
 };
 // grp_base / grp_mask of a u8 mask over n channels (see sp_elementwise.cu)
 cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream);
-// H[T, ldh] (compact on the k kept channels) = storage(phi(Z) - U)
+// H[T, ldh] (compact on the k kept channels idx[0..k), ldh a multiple of 8) = storage(phi(Z) - U)
 cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n, int64_t ldh,
-                          int64_t k, const int32_t* grp_base, const uint8_t* grp_mask, cudaStream_t stream);
+                          int64_t k, const int32_t* idx, cudaStream_t stream);
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]

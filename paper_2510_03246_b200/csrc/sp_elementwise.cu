@@ -204,50 +204,47 @@ __global__ void __launch_bounds__(1024) group_map_kernel(const uint8_t* __restri
   }
 }
 
-// H_S = storage(phi(Z) - U) on the kept channels, compact [T, ldh].  One thread per group of 8 channels and row.
-__global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U, void* H,
-                                                     int32_t hdt, int64_t T, int64_t n, int64_t ldh,
-                                                     const int32_t* __restrict__ grp_base,
-                                                     const uint8_t* __restrict__ grp_mask, int32_t rows_per_block) {
-  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t c0 = g * 8;
-  if (c0 >= n) return;
-  const unsigned bits = grp_mask[g];
-  if (bits == 0) return;
-  const int base = grp_base[g];
-  const bool vec = (n % 4 == 0) && c0 + 8 <= n;
+__device__ __forceinline__ void store8(void* base, int32_t dt, int64_t e, const float* v) {
+  if (dt == SP_BF16) {
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(v[4], v[5]), h3 = __floats2bfloat162_rn(v[6], v[7]);
+    uint4 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
+    pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
+    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(base) + e) = pk;
+  } else {
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  }
+}
+
+// H_S = storage(phi(Z) - U) on the kept channels, compact [T, ldh].  A thread owns 8 consecutive COMPACT columns: it
+// gathers their channels (ascending, so close together in a row of Z) and writes one 16-byte (bf16) or two 16-byte
+// (fp32) vectors per row.  Columns k..ldh-1 of H are written as zero.
+__global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U,
+                                                     void* __restrict__ H, int32_t hdt, int64_t T, int64_t n,
+                                                     int64_t ldh, int64_t k, const int32_t* __restrict__ idx,
+                                                     int32_t rows_per_block) {
+  const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (p0 >= ldh) return;
+  int ch[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) ch[q] = (p0 + q < k) ? idx[p0 + q] : -1;
   const int64_t r_begin = (int64_t)blockIdx.y * rows_per_block;
   const int64_t r_end = (r_begin + rows_per_block < T) ? r_begin + rows_per_block : T;
 #pragma unroll 2
   for (int64_t r = r_begin; r < r_end; ++r) {
-    const int64_t e = r * n + c0;
+    const float* zr = Z + r * n;
     float h[8];
-    if (vec) {
-      const float4 z0 = *reinterpret_cast<const float4*>(Z + e), z1 = *reinterpret_cast<const float4*>(Z + e + 4);
-      h[0] = fmaxf(z0.x, 0.f); h[1] = fmaxf(z0.y, 0.f); h[2] = fmaxf(z0.z, 0.f); h[3] = fmaxf(z0.w, 0.f);
-      h[4] = fmaxf(z1.x, 0.f); h[5] = fmaxf(z1.y, 0.f); h[6] = fmaxf(z1.z, 0.f); h[7] = fmaxf(z1.w, 0.f);
-      if (U) {
-        const float4 u0 = *reinterpret_cast<const float4*>(U + e), u1 = *reinterpret_cast<const float4*>(U + e + 4);
-        h[0] -= u0.x; h[1] -= u0.y; h[2] -= u0.z; h[3] -= u0.w;
-        h[4] -= u1.x; h[5] -= u1.y; h[6] -= u1.z; h[7] -= u1.w;
-      }
-    } else {
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        h[q] = 0.f;
-        if (c0 + q < n) h[q] = fmaxf(Z[e + q], 0.f) - (U ? U[e + q] : 0.f);
-      }
-    }
-    int pos = base;
-    const int64_t ho = r * ldh;
+    for (int q = 0; q < 8; ++q) h[q] = (ch[q] >= 0) ? fmaxf(zr[ch[q]], 0.f) : 0.f;
+    if (U) {
+      const float* ur = U + r * n;
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      if (bits & (1u << q)) {
-        if (hdt == SP_BF16) reinterpret_cast<__nv_bfloat16*>(H)[ho + pos] = __float2bfloat16_rn(h[q]);
-        else reinterpret_cast<float*>(H)[ho + pos] = h[q];
-        ++pos;
-      }
+      for (int q = 0; q < 8; ++q)
+        if (ch[q] >= 0) h[q] -= ur[ch[q]];
     }
+    store8(H, hdt, r * ldh + p0, h);
   }
 }
 
@@ -270,25 +267,14 @@ __device__ __forceinline__ float update_one(float zold, float z1, float dcorr, f
   return a;
 }
 
-__device__ __forceinline__ void store8(void* base, int32_t dt, int64_t e, const float* v) {
-  if (dt == SP_BF16) {
-    __nv_bfloat162 h0 = __floats2bfloat162_rn(v[0], v[1]), h1 = __floats2bfloat162_rn(v[2], v[3]);
-    __nv_bfloat162 h2 = __floats2bfloat162_rn(v[4], v[5]), h3 = __floats2bfloat162_rn(v[6], v[7]);
-    uint4 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
-    pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
-    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(base) + e) = pk;
-  } else {
-    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e + 4) = make_float4(v[4], v[5], v[6], v[7]);
-  }
-}
-
 // The fused auxiliary-variable update of one chunk: per element a = h + D (h = phi(z) - u), z2, the select, the dual
 // update, the residual / norm partial sums and the column sums of |a|, reading Z (and U) once and writing Z (and U),
 // A and the storage copy of Z once.  D and z1 exist on the kept channels only (compact, see above); on a pruned
 // channel both are zero (its row of W1 and its row of Q are zero).
 // grid: (column blocks of 2048 channels, row blocks).  A thread owns 8 consecutive channels and walks its rows.
+// Sums: fp32 within one row of 8 elements and per column over the thread's rows (at most a few hundred terms), fp64
+// across rows and blocks.
+template <bool HAS_U, int Z_RULE>
 __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   __shared__ double sm[32];
   const int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x;
@@ -296,89 +282,105 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   const int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
   const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
   const int64_t r_end = (r_begin + rows_per < g.T) ? r_begin + rows_per : g.T;
-  const bool has_u = g.U != nullptr;
   const float inv_ab = 1.f / (g.alpha + g.beta);
+  float* __restrict__ Zp = g.Z;
+  float* __restrict__ Up = g.U;
+  const float* __restrict__ z1p = g.z1;
+  const float* __restrict__ Dp = g.D;
   double s_res = 0.0, s_z = 0.0, s_a = 0.0;
-  double cs[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+  float cs[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (c0 < g.n) {
     const int cnt = (g.n - c0 >= 8) ? 8 : (int)(g.n - c0);
     const bool vec = (g.n % 8 == 0);
     const unsigned bits = g.grp_mask[grp];
     const int base = g.grp_base[grp];
+    // compact offset of each of the 8 channels (valid where its bit is set)
+    int off[8];
+    {
+      int pos = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        off[q] = pos;
+        pos += (bits >> q) & 1u;
+      }
+    }
+#pragma unroll 2
     for (int64_t r = r_begin; r < r_end; ++r) {
       const int64_t e = r * g.n + c0;
       float zo[8], u[8], z1[8], dc[8], a[8], zn[8];
       if (vec) {
-        const float4 v0 = *reinterpret_cast<const float4*>(g.Z + e), v1 = *reinterpret_cast<const float4*>(g.Z + e + 4);
+        const float4 v0 = *reinterpret_cast<const float4*>(Zp + e), v1 = *reinterpret_cast<const float4*>(Zp + e + 4);
         zo[0] = v0.x; zo[1] = v0.y; zo[2] = v0.z; zo[3] = v0.w; zo[4] = v1.x; zo[5] = v1.y; zo[6] = v1.z; zo[7] = v1.w;
-        if (has_u) {
-          const float4 w0 = *reinterpret_cast<const float4*>(g.U + e), w1 = *reinterpret_cast<const float4*>(g.U + e + 4);
+        if (HAS_U) {
+          const float4 w0 = *reinterpret_cast<const float4*>(Up + e), w1 = *reinterpret_cast<const float4*>(Up + e + 4);
           u[0] = w0.x; u[1] = w0.y; u[2] = w0.z; u[3] = w0.w; u[4] = w1.x; u[5] = w1.y; u[6] = w1.z; u[7] = w1.w;
         }
       } else {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          zo[q] = (q < cnt) ? g.Z[e + q] : 0.f;
-          if (has_u) u[q] = (q < cnt) ? g.U[e + q] : 0.f;
+          zo[q] = (q < cnt) ? Zp[e + q] : 0.f;
+          if (HAS_U) u[q] = (q < cnt) ? Up[e + q] : 0.f;
         }
       }
-      if (!has_u) {
+      if (!HAS_U) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) u[q] = 0.f;
       }
       {
-        const float* zp = g.z1 + r * g.ldk + base;
-        const float* dp = g.D + r * g.ldk + base;
-        int pos = 0;
+        const float* zp = z1p + r * g.ldk + base;
+        const float* dp = Dp + r * g.ldk + base;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          z1[q] = 0.f;
-          dc[q] = 0.f;
-          if (bits & (1u << q)) {
-            z1[q] = zp[pos];
-            dc[q] = dp[pos];
-            ++pos;
-          }
+          const bool kept = (bits >> q) & 1u;
+          z1[q] = kept ? zp[off[q]] : 0.f;
+          dc[q] = kept ? dp[off[q]] : 0.f;
         }
       }
+      float p_res = 0.f, p_z = 0.f, p_a = 0.f;
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
-        if (q < cnt) {
-          a[q] = update_one(zo[q], z1[q], dc[q], u[q], has_u, g.alpha, g.beta, inv_ab, g.z_rule, zn[q]);
-          const float diff = a[q] - fmaxf(zn[q], 0.f);
-          s_res += (double)diff * (double)diff;
-          s_z += (double)zn[q] * (double)zn[q];
-          s_a += (double)a[q] * (double)a[q];
-          cs[q] += (double)fabsf(a[q]);
-        } else {
-          a[q] = 0.f; zn[q] = 0.f;
-        }
+        a[q] = update_one(zo[q], z1[q], dc[q], u[q], HAS_U, g.alpha, g.beta, inv_ab, Z_RULE, zn[q]);
+        if (!vec && q >= cnt) { a[q] = 0.f; zn[q] = 0.f; }
+        const float diff = a[q] - fmaxf(zn[q], 0.f);
+        p_res = fmaf(diff, diff, p_res);
+        p_z = fmaf(zn[q], zn[q], p_z);
+        p_a = fmaf(a[q], a[q], p_a);
+        cs[q] += fabsf(a[q]);
       }
+      s_res += (double)p_res;
+      s_z += (double)p_z;
+      s_a += (double)p_a;
       if (vec) {
-        *reinterpret_cast<float4*>(g.Z + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
-        *reinterpret_cast<float4*>(g.Z + e + 4) = make_float4(zn[4], zn[5], zn[6], zn[7]);
-        if (has_u) {
-          *reinterpret_cast<float4*>(g.U + e) = make_float4(u[0], u[1], u[2], u[3]);
-          *reinterpret_cast<float4*>(g.U + e + 4) = make_float4(u[4], u[5], u[6], u[7]);
+        *reinterpret_cast<float4*>(Zp + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        *reinterpret_cast<float4*>(Zp + e + 4) = make_float4(zn[4], zn[5], zn[6], zn[7]);
+        if (HAS_U) {
+          *reinterpret_cast<float4*>(Up + e) = make_float4(u[0], u[1], u[2], u[3]);
+          *reinterpret_cast<float4*>(Up + e + 4) = make_float4(u[4], u[5], u[6], u[7]);
         }
         store8(g.A_out, g.out_dtype, e, a);
         if (g.Zb_out) store8(g.Zb_out, g.out_dtype, e, zn);
       } else {
-        for (int q = 0; q < cnt; ++q) {
-          g.Z[e + q] = zn[q];
-          if (has_u) g.U[e + q] = u[q];
-          if (g.out_dtype == SP_BF16) {
-            reinterpret_cast<__nv_bfloat16*>(g.A_out)[e + q] = __float2bfloat16_rn(a[q]);
-            if (g.Zb_out) reinterpret_cast<__nv_bfloat16*>(g.Zb_out)[e + q] = __float2bfloat16_rn(zn[q]);
-          } else {
-            reinterpret_cast<float*>(g.A_out)[e + q] = a[q];
-            if (g.Zb_out) reinterpret_cast<float*>(g.Zb_out)[e + q] = zn[q];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (q < cnt) {
+            Zp[e + q] = zn[q];
+            if (HAS_U) Up[e + q] = u[q];
+            if (g.out_dtype == SP_BF16) {
+              reinterpret_cast<__nv_bfloat16*>(g.A_out)[e + q] = __float2bfloat16_rn(a[q]);
+              if (g.Zb_out) reinterpret_cast<__nv_bfloat16*>(g.Zb_out)[e + q] = __float2bfloat16_rn(zn[q]);
+            } else {
+              reinterpret_cast<float*>(g.A_out)[e + q] = a[q];
+              if (g.Zb_out) reinterpret_cast<float*>(g.Zb_out)[e + q] = zn[q];
+            }
           }
         }
       }
     }
-    if (g.absA_part)
-      for (int q = 0; q < cnt; ++q) g.absA_part[(int64_t)blockIdx.y * g.n + c0 + q] = cs[q];
+    if (g.absA_part) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (q < cnt) g.absA_part[(int64_t)blockIdx.y * g.n + c0 + q] = (double)cs[q];
+    }
   }
   const int64_t bid = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
   const double r0 = block_sum<double>(s_res, sm);
@@ -617,20 +619,19 @@ cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, u
 }
 
 cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n, int64_t ldh,
-                          int64_t k, const int32_t* grp_base, const uint8_t* grp_mask, cudaStream_t stream) {
-  if (T * n == 0) return cudaSuccess;
+                          int64_t k, const int32_t* idx, cudaStream_t stream) {
+  if (T * ldh == 0) return cudaSuccess;
   // algorithmic bytes: Z (and U) read once, the kept part written once
   ProfScope prof(PK_PREP_H, 0.0, (double)T * ((double)n * (U ? 8.0 : 4.0) + (double)k * (hdt == SP_BF16 ? 2.0 : 4.0)),
                  stream);
-  const int64_t groups = ceil_div(n, (int64_t)8);
-  const unsigned gx = (unsigned)ceil_div(groups, (int64_t)256);
-  int64_t rb = ceil_div((int64_t)148 * 8, (int64_t)gx);
+  const unsigned gx = (unsigned)ceil_div(ldh, (int64_t)(8 * 256));
+  int64_t rb = ceil_div((int64_t)148 * 16, (int64_t)gx);
   if (rb > T) rb = T;
   if (rb > 65535) rb = 65535;
   const int32_t rows_per = (int32_t)ceil_div(T, rb);
   count_launch();
-  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, H, hdt, T, n, ldh, grp_base,
-                                                                                        grp_mask, rows_per);
+  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, H, hdt, T, n, ldh, k, idx,
+                                                                                        rows_per);
   return cudaGetLastError();
 }
 
@@ -653,7 +654,14 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   const double per_n = 8.0 + (a.U ? 8.0 : 0.0) + esz + (a.Zb_out ? esz : 0.0);
   ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * ((double)a.n * per_n + (double)a.k * 8.0), stream);
   count_launch();
-  fused_update_kernel<<<grid, 256, 0, stream>>>(a);
+  const bool pz = a.z_rule == SP_Z_PAPER;
+  if (a.U) {
+    if (pz) fused_update_kernel<true, SP_Z_PAPER><<<grid, 256, 0, stream>>>(a);
+    else fused_update_kernel<true, SP_Z_EXACT><<<grid, 256, 0, stream>>>(a);
+  } else {
+    if (pz) fused_update_kernel<false, SP_Z_PAPER><<<grid, 256, 0, stream>>>(a);
+    else fused_update_kernel<false, SP_Z_EXACT><<<grid, 256, 0, stream>>>(a);
+  }
   return cudaGetLastError();
 }
 
