@@ -7,8 +7,8 @@
 // mid.mid), each a K segment of one tcgen05 GEMM with fp32 accumulation.  The dropped terms are below 2^-23.
 //
 // Blocked right-looking algorithm with 128-wide panels:
-//   diagonal block : one CTA factorises it in registers (4 x 4 elements per thread) and forms inv(L11) in the same
-//                    sweep (the row operations of the elimination applied to an identity block);
+//   diagonal block : one CTA factorises it in registers (4 x 4 elements per thread, four columns per step) and forms
+//                    inv(L11) in the same sweep (the row operations of the elimination applied to an identity block);
 //   panel          : L21 = A21 inv(L11)^T on the CUDA cores (K = 128), written as fp32 and as the three bf16 parts;
 //   trailing update: A22 -= L21 L21^T (lower triangle) as one six-segment tensor-core GEMM.
 // The triangular solves X L^T = R, W L = X use the same two kernels block column by block column.
@@ -21,24 +21,41 @@ constexpr int TB = kCholTcNB;          // 128
 constexpr int DIAG_BLOCKS = (TB / 4) * (TB / 4 + 1) / 2;   // 528 lower-triangular 4 x 4 blocks
 constexpr int DIAG_THREADS = 544;      // 17 warps
 
+// 1 / sqrt(x) to about 1 ulp: hardware approximation plus one Newton step.
+__device__ __forceinline__ float rsqrt_refined(float x) {
+  float r;
+  asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r * fmaf(-0.5f * x, r * r, 1.5f);
+}
+
+constexpr int DIAG_TPAD = TB + 1;
+constexpr size_t DIAG_SMEM = (size_t)TB * DIAG_TPAD * sizeof(float);
+
 // Factorise the nb x nb diagonal block at A (lower triangle), write L back, and write inv(L) and its transpose to
 // dinv[0 : TB*TB] and dinv[TB*TB : 2*TB*TB] (row-major TB x TB, zero above / below the diagonal respectively,
 // identity on the padding rows nb..TB-1).  A non-positive pivot is reported once through `status` and replaced by 1.
 //
-// One thread owns one 4 x 4 block of the lower triangle in registers.  Elimination without square roots in the
-// loop: step j subtracts a_ij a_cj / p_j from the trailing columns c > j (p_j the pivot) and applies the same row
-// operations to an identity block B on the columns c <= j.  A column of the trailing matrix is final when its step
-// comes: it is scaled by 1/sqrt(p_j) and stored as column j of L, and its registers then carry column j of B.  So a
-// single register block m holds "a" on the columns still to be eliminated and "B" on the others, and one shared
-// vector w per step feeds both updates: w[i] = a_ij for i > j, w[c] = B_jc for c < j, w[j] = 1 / p_j.
-// A thread owns part of the eliminated column only while j runs through its own block column, so it keeps those
-// four unscaled columns in a second register block and scales them after the loop: L_ic = a_ic / sqrt(p_c),
-// inv(L)_ic = B_ic / sqrt(p_i).  The loop's critical path per step is barrier, one shared load, one multiply-add.
+// One thread owns one 4 x 4 block (bi, bj), bj <= bi, of the lower triangle in registers.  Blocked right-looking
+// elimination, four columns per step jb, that carries inv(L) along (the row operations of the elimination applied to
+// an identity block B).  Register block m holds the trailing matrix on block columns > jb and B on block columns
+// <= jb; a block column of the trailing matrix is final when its step comes and moves to lcol.  Per step:
+//   1. the owner of the diagonal block factorises it, D = C C^T, and inverts C (sequential, one thread; it runs while
+//      the other threads still finish step jb - 1);
+//   2. owners of block column jb:  L_i = A_i C^-T (final);  owners of block row jb:  B_jb <- C^-1 B_jb (final rows of
+//      inv(L)).  Both go to the shared array W (4 values per index): W[:, i] = L[i, j0:j0+4] for rows below the
+//      block, W[:, c] = inv(L)[j0:j0+4, c] for columns up to the block;
+//   3. every block below block row jb:  m -= W[:, rows]^T W[:, cols]  — the trailing update where the block still
+//      holds the matrix, the update of B where it holds B (a block of block column jb starts its life as B from 0).
+// Global input and output go through a padded shared tile so that every global access is a full coalesced row.
 __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, int64_t lda, int nb, float* dinv,
                                                                     int64_t row0, int32_t* status) {
-  __shared__ __align__(16) float wbuf[2][TB];   // double buffered: one barrier per step
-  __shared__ float piv[TB];
+  extern __shared__ __align__(16) float diag_tile[];          // T[TB][TB + 1]
+  float (*T)[DIAG_TPAD] = reinterpret_cast<float (*)[DIAG_TPAD]>(diag_tile);
+  __shared__ __align__(16) float W[2][4][TB];   // W[k][index]: conflict-free 16-byte accesses along the index
+  __shared__ __align__(16) float Ci_s[2][16];   // inverse of the diagonal factor, row-major 4 x 4 (lower)
   const int t = threadIdx.x;
+  const int lane = t & 31, warp = t >> 5;
+  constexpr int NWARP = DIAG_THREADS / 32;
   const bool active = t < DIAG_BLOCKS;
   // t = bi (bi + 1) / 2 + bj with bj <= bi
   int bi = (int)((sqrtf(8.f * (float)t + 1.f) - 1.f) * 0.5f);
@@ -46,105 +63,184 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
   while (bi * (bi + 1) / 2 > t) --bi;
   const int bj = t - bi * (bi + 1) / 2;
 
+  // ---- load: one warp per row, lanes along the columns; identity on the padding
+  for (int i = warp; i < TB; i += NWARP)
+    for (int c = lane; c < TB; c += 32) {
+      float v = 0.f;
+      if (i < nb && c <= i) v = A[(int64_t)i * lda + c];
+      if (i >= nb && i == c) v = 1.f;
+      T[i][c] = v;
+    }
+  __syncthreads();
   float m[4][4], lcol[4][4];
 #pragma unroll
   for (int r = 0; r < 4; ++r)
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-      const int i = 4 * bi + r, c = 4 * bj + s;
-      float v = 0.f;
-      if (active && i < nb && c <= i) v = A[(int64_t)i * lda + c];
-      if (i >= nb && i == c) v = 1.f;
-      m[r][s] = v;
-      lcol[r][s] = v;
+      m[r][s] = active ? T[4 * bi + r][4 * bj + s] : 0.f;
+      lcol[r][s] = 0.f;
     }
-  if (t < TB) piv[t] = 1.f;
-  // zero the parts of the two inverse blocks that no thread owns (blocks strictly above the diagonal of inv(L))
-  for (int e = t; e < TB * TB; e += DIAG_THREADS) {
-    const int i = e / TB, c = e % TB;
-    if ((c >> 2) > (i >> 2)) {
-      dinv[e] = 0.f;
-      dinv[TB * TB + c * TB + i] = 0.f;
-    }
-  }
-  __syncthreads();
 
-  for (int jb = 0; jb < TB / 4; ++jb) {
-    if (jb * 4 >= nb) break;
+  // step 1 for block jb by its diagonal owner: C -> lcol, C^-1 -> m, shared copies of C^-1
+  auto factor_diag = [&](int jb) {
+    float c[4][4], ci[4][4];
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-      const int j = jb * 4 + jj;
-      if (j < nb) {                     // uniform over the block
-        float* wb = wbuf[j & 1];
-        if (active && bj == jb) {       // owners of column j: live values below the diagonal, and the pivot
+    for (int r = 0; r < 4; ++r)
 #pragma unroll
-          for (int r = 0; r < 4; ++r)
-            if (4 * bi + r > j) wb[4 * bi + r] = m[r][jj];
-          if (bi == jb) {
-            float p = m[jj][jj];
-            if (!(p > 0.f)) {
-              report_status(status, SP_ERR_NOT_SPD, (int32_t)(row0 + j), 0);
-              p = 1.f;
-              m[jj][jj] = 1.f;
-            }
-            // reciprocal of the pivot: hardware approximation refined by one Newton step (error below 1 ulp)
-            float ip;
-            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ip) : "f"(p));
-            ip = fmaf(ip, fmaf(-p, ip, 1.f), ip);
-            wb[j] = ip;
-            piv[j] = p;
-          }
-        }
-        if (active && bi == jb) {       // owners of row j of B (columns left of j)
+      for (int s = 0; s < 4; ++s) { c[r][s] = 0.f; ci[r][s] = 0.f; }
+    float rd[4];   // reciprocals of the diagonal of C
 #pragma unroll
-          for (int s = 0; s < 4; ++s)
-            if (4 * bj + s < j) wb[4 * bj + s] = m[jj][s];
-        }
-        __syncthreads();
-        if (active && 4 * bi + 3 >= j) {
-          const float inv = wb[j];
-          if (bj == jb) {               // column j is final: keep it for L, its registers now carry column j of B
+    for (int k = 0; k < 4; ++k) {
+      float p = m[k][k];
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-              const int i = 4 * bi + r;
-              if (i >= j) {
-                lcol[r][jj] = m[r][jj];
-                m[r][jj] = (i == j) ? 1.f : 0.f;
-              }
-            }
-          }
-          const float4 wr = *reinterpret_cast<const float4*>(&wb[4 * bi]);
-          const float4 wc = *reinterpret_cast<const float4*>(&wb[4 * bj]);
-          const float wrv[4] = {wr.x, wr.y, wr.z, wr.w}, wcv[4] = {wc.x, wc.y, wc.z, wc.w};
-          float cr[4], w[4];
+      for (int q = 0; q < 4; ++q)
+        if (q < k) p = fmaf(-c[k][q], c[k][q], p);
+      if (!(p > 0.f)) {
+        report_status(status, SP_ERR_NOT_SPD, (int32_t)(row0 + 4 * jb + k), 0);
+        p = 1.f;
+      }
+      rd[k] = rsqrt_refined(p);
+      c[k][k] = p * rd[k];
 #pragma unroll
-          for (int r = 0; r < 4; ++r) cr[r] = (4 * bi + r > j) ? wrv[r] * inv : 0.f;
+      for (int r = 0; r < 4; ++r) {
+        if (r > k) {
+          float v = m[r][k];
 #pragma unroll
-          for (int s = 0; s < 4; ++s) w[s] = (4 * bj + s == j) ? 1.f : wcv[s];
-#pragma unroll
-          for (int r = 0; r < 4; ++r)
-#pragma unroll
-            for (int s = 0; s < 4; ++s) m[r][s] = fmaf(-cr[r], w[s], m[r][s]);
+          for (int q = 0; q < 4; ++q)
+            if (q < k) v = fmaf(-c[r][q], c[k][q], v);
+          c[r][k] = v * rd[k];
         }
       }
     }
+    // inverse of the lower-triangular C by forward substitution, column by column
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      ci[s][s] = rd[s];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        if (r > s) {
+          float v = 0.f;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (q >= s && q < r) v = fmaf(c[r][q], ci[q][s], v);
+          ci[r][s] = -v * rd[r];
+        }
+      }
+    }
+    float* cs = Ci_s[jb & 1];
+    float (*w)[TB] = W[jb & 1];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        lcol[r][s] = c[r][s];
+        m[r][s] = ci[r][s];
+        cs[r * 4 + s] = ci[r][s];
+        w[r][4 * jb + s] = ci[r][s];          // W[k][c] = inv(L)[j0 + k][c]
+      }
+  };
+
+  if (active && bi == 0) factor_diag(0);
+  const int nsteps = (nb + 3) / 4;
+  for (int jb = 0; jb < nsteps; ++jb) {
+    float (*w)[TB] = W[jb & 1];
+    __syncthreads();
+    if (active && bj == jb && bi > jb) {
+      // L_i = A_i C^-T : L_i[r][k] = sum_{s <= k} A_i[r][s] Ci[k][s]
+      const float* cs = Ci_s[jb & 1];
+      float l[4][4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          float v = 0.f;
+#pragma unroll
+          for (int s2 = 0; s2 < 4; ++s2)
+            if (s2 <= k) v = fmaf(m[r][s2], cs[k * 4 + s2], v);
+          l[r][k] = v;
+        }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        *reinterpret_cast<float4*>(&w[k][4 * bi]) = make_float4(l[0][k], l[1][k], l[2][k], l[3][k]);
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { lcol[r][k] = l[r][k]; m[r][k] = 0.f; }
+    }
+    if (active && bi == jb && bj < jb) {
+      // B_jb <- C^-1 B_jb : Bn[k][s] = sum_{r <= k} Ci[k][r] B[r][s]
+      const float* cs = Ci_s[jb & 1];
+      float bn[4][4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int s2 = 0; s2 < 4; ++s2) {
+          float v = 0.f;
+#pragma unroll
+          for (int r = 0; r < 4; ++r)
+            if (r <= k) v = fmaf(cs[k * 4 + r], m[r][s2], v);
+          bn[k][s2] = v;
+        }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        *reinterpret_cast<float4*>(&w[k][4 * bj]) = make_float4(bn[k][0], bn[k][1], bn[k][2], bn[k][3]);
+#pragma unroll
+        for (int s2 = 0; s2 < 4; ++s2) m[k][s2] = bn[k][s2];
+      }
+    }
+    __syncthreads();
+    if (active && bi > jb) {
+      float wr[4][4], wc[4][4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float4 v = *reinterpret_cast<const float4*>(&w[k][4 * bi]);
+        wr[0][k] = v.x; wr[1][k] = v.y; wr[2][k] = v.z; wr[3][k] = v.w;
+        const float4 u = *reinterpret_cast<const float4*>(&w[k][4 * bj]);
+        wc[0][k] = u.x; wc[1][k] = u.y; wc[2][k] = u.z; wc[3][k] = u.w;
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int s2 = 0; s2 < 4; ++s2) {
+          float v = m[r][s2];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) v = fmaf(-wr[r][k], wc[s2][k], v);
+          m[r][s2] = v;
+        }
+      // the owner of the next diagonal block goes straight on to factorise it
+      if (bi == jb + 1 && bj == jb + 1 && jb + 1 < nsteps) factor_diag(jb + 1);
+    }
   }
+
+  // ---- store inv(L) and its transpose through the tile
+  __syncthreads();
+  for (int e = t; e < TB * TB; e += DIAG_THREADS) T[e / TB][e % TB] = 0.f;
   __syncthreads();
   if (active) {
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int i = 4 * bi + r;
-      const float inv_sqrt_i = 1.f / sqrtf(piv[i]);
+    for (int r = 0; r < 4; ++r)
 #pragma unroll
-      for (int s = 0; s < 4; ++s) {
-        const int c = 4 * bj + s;
-        const float v = (c <= i) ? m[r][s] * inv_sqrt_i : 0.f;
-        dinv[i * TB + c] = v;
-        dinv[TB * TB + c * TB + i] = v;
-        if (c <= i && i < nb) A[(int64_t)i * lda + c] = lcol[r][s] / sqrtf(piv[c]);
-      }
-    }
+      for (int s = 0; s < 4; ++s)
+        if (4 * bj + s <= 4 * bi + r) T[4 * bi + r][4 * bj + s] = m[r][s];
   }
+  __syncthreads();
+  for (int i = warp; i < TB; i += NWARP)
+    for (int c = lane; c < TB; c += 32) {
+      dinv[i * TB + c] = T[i][c];
+      dinv[TB * TB + i * TB + c] = T[c][i];      // row i of the transpose = column i of inv(L)
+    }
+  // ---- store L (lower triangle of the nb x nb block)
+  __syncthreads();
+  if (active) {
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int s = 0; s < 4; ++s)
+        if (4 * bj + s <= 4 * bi + r) T[4 * bi + r][4 * bj + s] = lcol[r][s];
+  }
+  __syncthreads();
+  for (int i = warp; i < nb; i += NWARP)
+    for (int c = lane; c <= i; c += 32) A[(int64_t)i * lda + c] = T[i][c];
 }
 
 __device__ __forceinline__ void split3(float v, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
@@ -163,7 +259,8 @@ constexpr size_t PA_SMEM = ((size_t)TB * TB + (size_t)TB * PA_APAD) * sizeof(flo
 // X[i, 0:nb] <- X[i, 0:nb] inv(L)^T (TRANS == false) or X[i, 0:nb] inv(L) (TRANS == true), for `rows` rows.
 // dinv is the pair of TB x TB blocks written by chol_diag128_kernel.  The result is written back in fp32 (write_f32)
 // and as three bf16 parts to S[i * lds + part * s_seg + c] for all TB columns (zero beyond nb).
-// One CTA takes 32 rows; a thread computes 4 rows x 8 columns.
+// One CTA takes 32 rows; a thread computes 4 rows x 8 columns (two groups of 4, half a block apart, so that the
+// 16-byte shared loads of a warp fall on distinct banks).
 template <bool TRANS>
 __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64_t ldx, int64_t rows, int nb,
                                                                  const float* __restrict__ dinv, __nv_bfloat16* S,
@@ -209,7 +306,7 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
     }
   }
   __syncthreads();
-  const int tx = t & 15, ty = t >> 4;          // columns 8 tx .. 8 tx + 7, rows 4 ty .. 4 ty + 3
+  const int tx = t & 15, ty = t >> 4;   // columns 4 tx .. 4 tx + 3 and 64 + 4 tx .. 64 + 4 tx + 3, rows 4 ty .. 4 ty + 3
   float acc[4][8];
 #pragma unroll
   for (int r = 0; r < 4; ++r)
@@ -218,8 +315,8 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
 #pragma unroll 4
   for (int k = 0; k < TB; ++k) {
     const float4 a0 = *reinterpret_cast<const float4*>(&At[k][4 * ty]);
-    const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][8 * tx]);
-    const float4 l1 = *reinterpret_cast<const float4*>(&Lt[k][8 * tx + 4]);
+    const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][4 * tx]);
+    const float4 l1 = *reinterpret_cast<const float4*>(&Lt[k][TB / 2 + 4 * tx]);
     const float av[4] = {a0.x, a0.y, a0.z, a0.w};
     const float lv[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
 #pragma unroll
@@ -227,33 +324,35 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
   }
-  const int c0 = 8 * tx;
-  const bool x_vec = write_f32 && c0 + 8 <= nb && x_al;
+  const bool x_vec = write_f32 && x_al;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int64_t gi = r0 + 4 * ty + r;
     if (gi >= rows) continue;
-    float v[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = (c0 + j < nb) ? acc[r][j] : 0.f;
-    if (write_f32) {
-      float* dst = X + gi * ldx + c0;
-      if (x_vec) {
-        *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-        *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
-      } else {
+    for (int half = 0; half < 2; ++half) {
+      const int c0 = half * (TB / 2) + 4 * tx;
+      float v[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          if (c0 + j < nb) dst[j] = v[j];
+      for (int j = 0; j < 4; ++j) v[j] = (c0 + j < nb) ? acc[r][half * 4 + j] : 0.f;
+      if (write_f32) {
+        float* dst = X + gi * ldx + c0;
+        if (x_vec && c0 + 4 <= nb) {
+          *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (c0 + j < nb) dst[j] = v[j];
+        }
       }
-    }
-    if (S) {   // S + gi * lds + part * s_seg + c0 is 16-byte aligned by construction (lds, s_seg multiples of 8)
-      __align__(16) __nv_bfloat16 part[3][8];
+      if (S) {   // S + gi * lds + part * s_seg + c0 is 8-byte aligned by construction (lds, s_seg multiples of 8)
+        __align__(8) __nv_bfloat16 part[3][4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) split3(v[j], part[0][j], part[1][j], part[2][j]);
+        for (int j = 0; j < 4; ++j) split3(v[j], part[0][j], part[1][j], part[2][j]);
 #pragma unroll
-      for (int q = 0; q < 3; ++q)
-        *reinterpret_cast<uint4*>(S + gi * lds + q * s_seg + c0) = *reinterpret_cast<const uint4*>(part[q]);
+        for (int q = 0; q < 3; ++q)
+          *reinterpret_cast<uint2*>(S + gi * lds + q * s_seg + c0) = *reinterpret_cast<const uint2*>(part[q]);
+      }
     }
   }
 }
@@ -289,13 +388,20 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
                          cudaStream_t stream) {
   __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
+  static bool diag_attr = false;
+  if (!diag_attr) {
+    if (cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM) !=
+        cudaSuccess)
+      return SP_ERR_CUDA;
+    diag_attr = true;
+  }
   for (int64_t k0 = 0; k0 < n; k0 += TB) {
     const int nb = (int)((n - k0 < TB) ? (n - k0) : TB);
     float* dk = dinv + (k0 / TB) * 2 * TB * TB;
     {
       count_launch();
       ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
-      chol_diag128_kernel<<<1, DIAG_THREADS, 0, stream>>>(A + k0 * lda + k0, lda, nb, dk, k0, status_dev);
+      chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(A + k0 * lda + k0, lda, nb, dk, k0, status_dev);
       if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     }
     const int64_t rem = n - k0 - nb;
