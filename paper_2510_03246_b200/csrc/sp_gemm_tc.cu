@@ -1,38 +1,54 @@
 // bf16 tensor-core GEMM for sm_100a: TMA-fed shared-memory pipeline, tcgen05.mma with fp32 accumulators in tensor
-// memory, warp-specialised persistent CTAs (one per SM).
+// memory, warp-specialised persistent CTAs working in pairs.
 //
 //   C[M,N] = alpha * A B^T-like contraction over K + beta * Cin
 //
 // Both operands may be K-major (stored [rows, K], K contiguous: the weight/activation products z^(1) = X W1^T, ...)
 // or MN-major (stored [K, rows], rows contiguous: the token-axis contractions A^T A, Z^T X, Ypre^T A).  Each
 // major-ness has its own TMA box shape and shared-memory matrix descriptor; the MMA instruction descriptor carries
-// the two major bits.  No cluster launch and no multicast loads are used.
+// the two major bits.
 //
-// Roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = tensor-memory allocator + MMA issuer (one lane),
-// warps 2..5 = epilogue (each owns the 32 accumulator lanes its warp id maps to).  Two 256-column accumulators are
-// ping-ponged so that the epilogue of tile i overlaps the main loop of tile i+1.
-// Every wait is bounded by a clock budget; on expiry the CTA records SP_ERR_TIMEOUT, drains its copies and MMAs,
-// frees its tensor memory and returns.
+// Two CTAs on neighbouring SMs (a cluster of 2) share one 256 x 256 output tile: every CTA loads its own 128 rows of
+// A and ONE HALF (128 columns) of B per k-block, and the pair's leader issues one cta_group::2 MMA of shape
+// 256 x 256 x 16 that reads both halves.  A CTA therefore moves 32 KB per k-block through the L2 -> SM path instead
+// of the 48 KB a lone 128 x 256 tile needs, which is what bounded the single-CTA form of this kernel.  Every load is
+// an ordinary one-destination TMA load: it lands in the issuing CTA's own shared memory and completes on the
+// leader's barrier.
+//
+// Roles (192 threads per CTA): warp 0 = TMA producer (one lane), warp 1 = tensor-memory allocator and, in the
+// leader, MMA issuer (one lane), warps 2..5 = epilogue (each owns the 32 accumulator lanes its warp id maps to).  Two
+// 256-column accumulators are ping-ponged so that the epilogue of tile i overlaps the main loop of tile i+1.
+// Epilogue: the accumulator block of a warp (32 rows x 32 columns) goes through a 128-byte-swizzled shared tile and
+// leaves by a TMA store, or a TMA add-reduction when the call accumulates into C; other cases (bf16 output, a
+// separate Cin, unaligned C) use plain coalesced loads and stores through a padded tile.
+// Every wait is bounded by a clock budget; on expiry the CTA records SP_ERR_TIMEOUT and leaves its loops, and both
+// CTAs still meet at the final cluster barrier before tensor memory is freed.
 #include <cuda.h>
+#include <string.h>
 
 #include "sp_common.cuh"
 
 namespace sp {
 namespace {
 
-constexpr int BM = 128;
-constexpr int BN = 256;
+constexpr int BM = 128;            // rows of A (and of the accumulator) per CTA
+constexpr int BNH = 128;           // columns of B loaded per CTA (half of the pair's tile)
+constexpr int TILE_M = 2 * BM;     // tile of the CTA pair
+constexpr int TILE_N = 2 * BNH;
 constexpr int BK = 64;
-constexpr int STAGES = 4;
+constexpr int STAGES = 6;
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int B_BYTES = BNH * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 32 KB
+constexpr int STG_BYTES = 8192;                          // per epilogue warp: two 32 x 32 fp32 blocks
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr long long WAIT_BUDGET_CYCLES = 6000000000LL;   // ~3 s at 2 GHz
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * STG_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long WAIT_BUDGET_CYCLES = 4000000000LL;   // ~2 s
 constexpr long long DRAIN_BUDGET_CYCLES = 200000000LL;   // ~0.1 s
+
+enum EpiMode : int { EPI_DIRECT = 0, EPI_TMA_STORE = 1, EPI_TMA_ADD = 2 };
 
 struct TcParams {
   int64_t M, N, K;
@@ -44,7 +60,7 @@ struct TcParams {
   int32_t c_dtype;
   int64_t c_ld;
   int32_t a_kmajor, b_kmajor, lower_only;
-  int32_t red_add;   // 1: C += alpha * acc by global reductions (beta == 1, Cin == C, fp32)
+  int32_t epi_mode;  // EpiMode
   int32_t n_fast;    // tile order: 1 = consecutive tiles walk N first (they share the A row block)
   TcSegments seg;    // K segments: segment s reads A at (k + a_k[s], m + a_mn[s]) and B at (k + b_k[s], n + b_mn[s])
   int32_t seg_kb;    // k-blocks per segment
@@ -54,11 +70,27 @@ struct TcParams {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// arrive on a barrier given by its shared::cluster address (own CTA or the peer)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -74,7 +106,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false when the budget ran out or another role already gave up.
+// Bounded wait.  Returns false when the budget ran out or another role of this CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
@@ -91,24 +123,46 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t bar) {
+// Load of one box into this CTA's shared memory; the bytes complete on the barrier `bar_cluster_addr`, which is the
+// pair leader's (cta_group::2 form: the barrier may live in the peer CTA).
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
+                                            uint32_t bar_cluster_addr) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// The MMAs issued so far by this thread arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"(mask)
+      : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -141,15 +195,16 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, bool kmajor, u
   return d;
 }
 
+// Instruction descriptor of the pair's MMA: 256 x 256 x 16, bf16 operands, fp32 accumulator.
 __device__ __forceinline__ uint32_t make_instr_desc(bool a_kmajor, bool b_kmajor) {
   uint32_t d = 0;
-  d |= 1u << 4;                       // accumulator format: fp32
-  d |= 1u << 7;                       // A format: bf16
-  d |= 1u << 10;                      // B format: bf16
-  d |= (a_kmajor ? 0u : 1u) << 15;    // A major-ness
-  d |= (b_kmajor ? 0u : 1u) << 16;    // B major-ness
-  d |= (uint32_t)(BN >> 3) << 17;     // N
-  d |= (uint32_t)(BM >> 4) << 24;     // M
+  d |= 1u << 4;                          // accumulator format: fp32
+  d |= 1u << 7;                          // A format: bf16
+  d |= 1u << 10;                         // B format: bf16
+  d |= (a_kmajor ? 0u : 1u) << 15;       // A major-ness
+  d |= (b_kmajor ? 0u : 1u) << 16;       // B major-ness
+  d |= (uint32_t)(TILE_N >> 3) << 17;    // N
+  d |= (uint32_t)(TILE_M >> 4) << 24;    // M
   return d;
 }
 
@@ -163,28 +218,34 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, i
       tn = t / p.tiles_m;
     }
   } else {
-    // column block tn owns row blocks first(tn)..tiles_m-1 with first = tn * BN / BM
+    // column block tn owns row blocks tn..tiles_m-1 (square tiles)
     tn = 0;
     for (;;) {
-      const int first = tn * (BN / BM);
-      const int cnt = p.tiles_m - first;
-      if (t < cnt) { tm = first + t; break; }
+      const int cnt = p.tiles_m - tn;
+      if (t < cnt) { tm = tn + t; break; }
       t -= cnt;
       ++tn;
     }
   }
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p) {
+__device__ __forceinline__ void tc_commit_local(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
-  __shared__ float s_stage[4][32][33];   // per epilogue warp: one 32 x 32 accumulator block, padded
 
+  // identical offsets in both CTAs of the pair: the leader's MMA reads the peer's operand tiles at the offsets of
+  // its own, and barrier addresses are exchanged by offset
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;            // 1024-byte aligned operand stages
-  const uint32_t bars = tiles + STAGES * STAGE_BYTES;       // 8-byte aligned barrier block
+  const uint32_t stg_base = tiles + STAGES * STAGE_BYTES;   // 1024-byte aligned epilogue tiles
+  const uint32_t bars = stg_base + 4 * STG_BYTES;           // 8-byte aligned barrier block
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
@@ -193,79 +254,79 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
+  const int cid = (int)(blockIdx.x >> 1);        // pair index
+  const int ncl = (int)(gridDim.x >> 1);
   volatile int* abort_flag = &s_abort;
 
   if (threadIdx.x == 0) {
     s_abort = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }   // 4 warps x 2 CTAs
     mbar_init(drain_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+  if (warp == 1) {   // the same warp in both CTAs allocates the pair's tensor memory
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
                  "r"((uint32_t)TMEM_COLS)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();      // the peer's barriers exist before anything is sent to them
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
 
   const int num_kb = p.seg_kb * p.seg.nseg;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
-      uint32_t armed = 0;          // bit s: stage s has been armed at least once
-      uint32_t armed_parity = 0;   // bit s: parity of the phase the last arming of stage s completes
       bool ok = true;
-      for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+      for (int t = cid; t < p.num_tiles && ok; t += ncl) {
         int tm, tn;
         tile_coords(p, t, tm, tn);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), STAGE_BYTES);
-          armed |= 1u << s;
-          armed_parity = (armed_parity & ~(1u << s)) | (ph << s);
+          // the leader's barrier collects the bytes of both CTAs' loads of this stage
+          if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+          const uint32_t fbar = map_to_cta(full_bar(s), 0);
           const uint32_t a_dst = tiles + s * STAGE_BYTES;
           const uint32_t b_dst = a_dst + A_BYTES;
           const int sg = kb / p.seg_kb;
           const int kk = (kb - sg * p.seg_kb) * BK;
           const int ka = kk + p.seg.a_k[sg], kbb = kk + p.seg.b_k[sg];
-          const int am = tm * BM + p.seg.a_mn[sg], bn = tn * BN + p.seg.b_mn[sg];
+          const int am = tm * TILE_M + (int)rank * BM + p.seg.a_mn[sg];
+          const int bn = tn * TILE_N + (int)rank * BNH + p.seg.b_mn[sg];
           if (p.a_kmajor) {
-            tma_load_2d(a_dst, &tmA, ka, am, full_bar(s));
+            tma_load_2d(a_dst, &tmA, ka, am, fbar);
           } else {
 #pragma unroll
-            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, am + mb * 64, ka, full_bar(s));
+            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, am + mb * 64, ka, fbar);
           }
           if (p.b_kmajor) {
-            tma_load_2d(b_dst, &tmB, kbb, bn, full_bar(s));
+            tma_load_2d(b_dst, &tmB, kbb, bn, fbar);
           } else {
 #pragma unroll
-            for (int nb = 0; nb < BN / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, bn + nb * 64, kbb, full_bar(s));
+            for (int nb = 0; nb < BNH / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, bn + nb * 64, kbb, fbar);
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
       }
       if (!ok) {
         report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 1);
-        // let copies already in flight land before the shared memory is released
-        for (int q = 0; q < STAGES; ++q)
-          if (armed & (1u << q)) {
-            const long long t0 = clock64();
-            while (!mbar_try(full_bar(q), (armed_parity >> q) & 1u) && clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
-          }
+        // give copies already in flight time to land before shared memory is released
+        const long long t0 = clock64();
+        while (clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
       const uint32_t idesc = make_instr_desc(p.a_kmajor != 0, p.b_kmajor != 0);
       int s = 0;
       uint32_t ph = 0;
@@ -273,10 +334,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t aph = 0;
       bool ok = true;
       bool issued = false;
-      for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+      for (int t = cid; t < p.num_tiles && ok; t += ncl) {
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(s), ph, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           tc_fence_after();
@@ -289,83 +350,110 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t b_off = p.b_kmajor ? (uint32_t)(k * UMMA_K * 2) : (uint32_t)(k * UMMA_K * 128);
             const uint64_t adesc = make_smem_desc(a_src + a_off, p.a_kmajor != 0, 64 * BK * 2);
             const uint64_t bdesc = make_smem_desc(b_src + b_off, p.b_kmajor != 0, 64 * BK * 2);
-            tc_mma_bf16(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            tc_mma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
           }
           issued = true;
-          tc_commit(empty_bar(s));   // frees the stage once these MMAs have read it
+          tc_commit_pair(empty_bar(s));   // frees the stage in both CTAs once these MMAs have read it
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        tc_commit(tfull_bar(acc));   // accumulator complete
+        tc_commit_pair(tfull_bar(acc));   // accumulator complete: wakes the epilogue warps of both CTAs
         if (++acc == 2) { acc = 0; aph ^= 1u; }
       }
       if (!ok) {
         report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 2);
         if (issued) {   // wait for MMAs in flight before shared and tensor memory are released
-          tc_commit(drain_bar);
+          tc_commit_local(drain_bar);
           const long long t0 = clock64();
           while (!mbar_try(drain_bar, 0u) && clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue warps 2..5
-    // tcgen05.ld hands every lane one accumulator row (32 consecutive columns per load).  The 32 x 32 block is turned
-    // through a padded shared-memory tile so that global loads and stores see a warp on 32 consecutive columns of one
-    // row (128-byte lines) instead of 32 different rows.
+    // ------------------------------------------------------------------ epilogue warps 2..5 (both CTAs)
+    // tcgen05.ld hands every lane one accumulator row (32 consecutive columns per load).
     const int q = warp & 3;                 // accumulator lane quarter this warp may read
-    float (*stg)[33] = s_stage[q];
+    const uint32_t wstg = stg_base + (uint32_t)q * STG_BYTES;
+    uint8_t* wstg_ptr = smem_raw + (wstg - raw);
+    float (*stg)[33] = reinterpret_cast<float (*)[33]>(wstg_ptr);   // padded tile of the plain path
+    const uint32_t tempty_leader[2] = {map_to_cta(tempty_bar(0), 0), map_to_cta(tempty_bar(1), 0)};
     int acc = 0;
     uint32_t aph = 0;
+    int buf = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+    const bool has_cin = p.beta != 0.f;
+    const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
+    for (int t = cid; t < p.num_tiles && ok; t += ncl) {
       int tm, tn;
       tile_coords(p, t, tm, tn);
       // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
       const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
       tc_fence_after();
-      const int64_t row0 = (int64_t)tm * BM + q * 32;      // first global row of this warp's 32 rows
-      const uint32_t taddr = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
+      const int64_t row0 = (int64_t)tm * TILE_M + (int64_t)rank * BM + q * 32;   // first global row of this warp
+      const uint32_t taddr = tmem_base + (uint32_t)(acc * TILE_N) + ((uint32_t)(q * 32) << 16);
       const int rows_here = (p.M - row0 < 32) ? (int)(p.M - row0) : 32;   // may be <= 0 on a ragged last tile
-      const bool has_cin = p.beta != 0.f && !p.red_add;
-      const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
+      if (p.epi_mode != EPI_DIRECT) {
+        // 32 x 32 fp32 block -> 128-byte-swizzled shared tile (16-byte chunk j of row r sits at chunk j ^ (r & 7))
+        // -> one TMA store / add-reduction, which clips at the edges of C.  Two tiles per warp alternate.
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        const int64_t gj0 = (int64_t)tn * BN + c0;
-        if (gj0 >= p.N) break;                  // uniform over the warp
-        const int64_t gj = gj0 + lane;
-        // the 32 rows of Cin for this column are fetched first (independent loads in flight while the accumulator
-        // block is read from tensor memory and turned)
-        float cv[32];
-        if (has_cin) {
-          const int64_t cin_off = row0 * p.cin_ld + gj;
+        for (int c0 = 0; c0 < TILE_N; c0 += 32) {
+          const int64_t gj0 = (int64_t)tn * TILE_N + c0;
+          if (gj0 >= p.N) break;                  // uniform over the warp
+          uint32_t r[32];
+          tc_ld32(taddr + (uint32_t)c0, r);
+          tc_wait_ld();
+          if (lane == 0) bulk_wait_read_1();      // the copy that last read this tile (two blocks ago) is done
+          __syncwarp();
+          uint8_t* tile = wstg_ptr + buf * 4096 + lane * 128;
 #pragma unroll
-          for (int rr = 0; rr < 32; ++rr) {
-            cv[rr] = 0.f;
-            if (gj < p.N && rr < rows_here) {
-              const int64_t o = cin_off + (int64_t)rr * p.cin_ld;
-              cv[rr] = cin_f32 ? reinterpret_cast<const float*>(p.cin)[o]
-                               : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.cin)[o]);
+          for (int j = 0; j < 8; ++j) {
+            const float4 v = make_float4(p.alpha * __uint_as_float(r[4 * j]), p.alpha * __uint_as_float(r[4 * j + 1]),
+                                         p.alpha * __uint_as_float(r[4 * j + 2]), p.alpha * __uint_as_float(r[4 * j + 3]));
+            *reinterpret_cast<float4*>(tile + ((j ^ (lane & 7)) << 4)) = v;
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (rows_here > 0) {
+              if (p.epi_mode == EPI_TMA_STORE) tma_store_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+              else tma_reduce_add_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+            }
+            bulk_commit();
+          }
+          buf ^= 1;
+        }
+      } else {
+        // plain path: the block is turned through a padded tile so that global loads and stores see a warp on 32
+        // consecutive columns of one row (128-byte lines) instead of 32 different rows
+#pragma unroll 1
+        for (int c0 = 0; c0 < TILE_N; c0 += 32) {
+          const int64_t gj0 = (int64_t)tn * TILE_N + c0;
+          if (gj0 >= p.N) break;                  // uniform over the warp
+          const int64_t gj = gj0 + lane;
+          // the 32 rows of Cin for this column are fetched first (independent loads in flight while the accumulator
+          // block is read from tensor memory and turned)
+          float cv[32];
+          if (has_cin) {
+            const int64_t cin_off = row0 * p.cin_ld + gj;
+#pragma unroll
+            for (int rr = 0; rr < 32; ++rr) {
+              cv[rr] = 0.f;
+              if (gj < p.N && rr < rows_here) {
+                const int64_t o = cin_off + (int64_t)rr * p.cin_ld;
+                cv[rr] = cin_f32 ? reinterpret_cast<const float*>(p.cin)[o]
+                                 : __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.cin)[o]);
+              }
             }
           }
-        }
-        uint32_t r[32];
-        tc_ld32(taddr + (uint32_t)c0, r);
-        tc_wait_ld();
+          uint32_t r[32];
+          tc_ld32(taddr + (uint32_t)c0, r);
+          tc_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) stg[lane][i] = p.alpha * __uint_as_float(r[i]);
-        __syncwarp();
-        if (gj < p.N) {
-          const int64_t c_off = row0 * p.c_ld + gj;
-          if (p.red_add) {
-            // C += alpha * acc: one reduction per element, no read round trip (each address is touched once per launch)
-            float* dst = reinterpret_cast<float*>(p.c) + c_off;
-#pragma unroll
-            for (int rr = 0; rr < 32; ++rr)
-              if (rr < rows_here)
-                asm volatile("red.global.add.f32 [%0], %1;" ::"l"(dst + (int64_t)rr * p.c_ld), "f"(stg[rr][lane]) : "memory");
-          } else {
+          for (int i = 0; i < 32; ++i) stg[lane][i] = p.alpha * __uint_as_float(r[i]);
+          __syncwarp();
+          if (gj < p.N) {
+            const int64_t c_off = row0 * p.c_ld + gj;
 #pragma unroll
             for (int rr = 0; rr < 32; ++rr) {
               if (rr < rows_here) {
@@ -377,22 +465,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               }
             }
           }
+          __syncwarp();
         }
-        __syncwarp();
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (lane == 0) mbar_arrive_cluster(tempty_leader[acc]);   // the leader's MMA thread counts both CTAs' warps
       if (++acc == 2) { acc = 0; aph ^= 1u; }
     }
+    if (lane == 0) bulk_wait_all();         // shared tiles and C are settled before the CTA leaves
     if (!ok && lane == 0) report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 3);
   }
 
+  // both CTAs are done with each other's shared memory and barriers before either leaves
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
                  : "memory");
   }
 }
@@ -416,20 +507,21 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map of a bf16 operand.  stored matrix: [outer, inner] row-major with leading dimension ld.
-//   K-major : inner = K, outer = rows, box = {64, box_rows}
-//   MN-major: inner = rows, outer = K, box = {64, 64}
-bool make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+// Tensor map of a row-major matrix [outer, inner] with leading dimension ld (elements), 128-byte swizzle.
+//   bf16 operand, K-major : inner = K, outer = rows, box = {64, 128}
+//   bf16 operand, MN-major: inner = rows, outer = K, box = {64, 64}
+//   fp32 output C         : inner = N, outer = M, box = {32, 32}
+bool make_map(CUtensorMap* map, bool f32, const void* ptr, int64_t inner, int64_t outer, int64_t ld, int box_inner,
               int box_outer) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * (f32 ? 4 : 2)};
   cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -477,9 +569,12 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   if (C.dtype != SP_F32 && C.dtype != SP_BF16) return SP_ERR_DTYPE;
   if (beta != 0.f && Cin.dtype != SP_F32 && Cin.dtype != SP_BF16) return SP_ERR_DTYPE;
 
-  CUtensorMap tmA, tmB;
-  bool ok = A.kmajor ? make_map(&tmA, A.ptr, a_kext, a_mext, A.ld, BK, BM) : make_map(&tmA, A.ptr, a_mext, a_kext, A.ld, 64, BK);
-  ok = ok && (B.kmajor ? make_map(&tmB, B.ptr, b_kext, b_next, B.ld, BK, BN) : make_map(&tmB, B.ptr, b_next, b_kext, B.ld, 64, BK));
+  CUtensorMap tmA, tmB, tmC;
+  memset(&tmC, 0, sizeof(tmC));
+  bool ok = A.kmajor ? make_map(&tmA, false, A.ptr, a_kext, a_mext, A.ld, BK, BM)
+                     : make_map(&tmA, false, A.ptr, a_mext, a_kext, A.ld, 64, BK);
+  ok = ok && (B.kmajor ? make_map(&tmB, false, B.ptr, b_kext, b_next, B.ld, BK, BNH)
+                       : make_map(&tmB, false, B.ptr, b_next, b_kext, B.ld, 64, BK));
   if (!ok) return SP_ERR_CUDA;
 
   TcParams p;
@@ -490,19 +585,22 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   p.a_kmajor = A.kmajor ? 1 : 0;
   p.b_kmajor = B.kmajor ? 1 : 0;
   p.lower_only = lower_only ? 1 : 0;
-  p.red_add = (beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && C.dtype == SP_F32 && Cin.s0 == C.ld) ? 1 : 0;
+  // fp32 C that a tensor map can describe leaves through TMA: a store when nothing is added, an add-reduction when
+  // the call accumulates into C itself (each element of C is touched once per launch, so the result is the same sum)
+  p.epi_mode = EPI_DIRECT;
+  const bool c_tma = C.dtype == SP_F32 && C.ld % 4 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0;
+  if (c_tma && beta == 0.f) p.epi_mode = EPI_TMA_STORE;
+  if (c_tma && beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && Cin.s0 == C.ld) p.epi_mode = EPI_TMA_ADD;
+  if (p.epi_mode != EPI_DIRECT && !make_map(&tmC, true, C.ptr, N, M, C.ld, 32, 32)) return SP_ERR_CUDA;
   p.seg = sg;
   p.seg_kb = (int32_t)ceil_div(K, BK);
-  p.tiles_m = (int32_t)ceil_div(M, BM);
-  p.tiles_n = (int32_t)ceil_div(N, BN);
+  p.tiles_m = (int32_t)ceil_div(M, TILE_M);
+  p.tiles_n = (int32_t)ceil_div(N, TILE_N);
   // consecutive tiles (which run at the same time on neighbouring SMs) should share the larger operand panel
   p.n_fast = p.tiles_n < p.tiles_m ? 1 : 0;
   if (lower_only) {
     int64_t cnt = 0;
-    for (int tn = 0; tn < p.tiles_n; ++tn) {
-      const int first = tn * (BN / BM);
-      if (first < p.tiles_m) cnt += p.tiles_m - first;
-    }
+    for (int tn = 0; tn < p.tiles_n && tn < p.tiles_m; ++tn) cnt += p.tiles_m - tn;
     p.num_tiles = (int32_t)cnt;
   } else {
     p.num_tiles = p.tiles_m * p.tiles_n;
@@ -519,8 +617,9 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   count_launch();
   const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
   ProfScope prof(PK_GEMM_TC, flops, 0.0, stream);
-  int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, p);
+  const int pairs_max = sm_count() / 2;
+  const int pairs = p.num_tiles < pairs_max ? p.num_tiles : pairs_max;
+  gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
 }
 
