@@ -18,7 +18,7 @@ using namespace sp;
 
 namespace {
 
-constexpr int64_t kDefaultChunk = 16384;
+constexpr int64_t kDefaultChunk = 32768;
 
 struct MatRef {
   const void* ptr;

@@ -24,6 +24,7 @@
 // Every wait is bounded by a clock budget; on expiry the CTA records SP_ERR_TIMEOUT and leaves its loops, and both
 // CTAs still meet at the final cluster barrier before tensor memory is freed.
 #include <cuda.h>
+#include <math.h>
 #include <string.h>
 
 #include "sp_common.cuh"
@@ -65,6 +66,9 @@ struct TcParams {
   TcSegments seg;    // K segments: segment s reads A at (k + a_k[s], m + a_mn[s]) and B at (k + b_k[s], n + b_mn[s])
   int32_t seg_kb;    // k-blocks per segment
   int32_t tiles_m, tiles_n, num_tiles;
+  // Work units: unit u is tile u % num_tiles restricted to k-blocks [ks * kb_per_split, (ks + 1) * kb_per_split) with
+  // ks = u / num_tiles.  ksplit > 1 only with the add-reduction epilogue (partial products add up in C).
+  int32_t ksplit, kb_per_split, num_units;
   int32_t* status;
 };
 
@@ -287,10 +291,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int t = cid; t < p.num_tiles && ok; t += ncl) {
+      for (int u = cid; u < p.num_units && ok; u += ncl) {
         int tm, tn;
-        tile_coords(p, t, tm, tn);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        tile_coords(p, u % p.num_tiles, tm, tn);
+        const int kb0 = (u / p.num_tiles) * p.kb_per_split;
+        const int kb1 = (kb0 + p.kb_per_split < num_kb) ? kb0 + p.kb_per_split : num_kb;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           // the leader's barrier collects the bytes of both CTAs' loads of this stage
           if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
@@ -334,11 +340,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t aph = 0;
       bool ok = true;
       bool issued = false;
-      for (int t = cid; t < p.num_tiles && ok; t += ncl) {
+      for (int u = cid; u < p.num_units && ok; u += ncl) {
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        const int kb0 = (u / p.num_tiles) * p.kb_per_split;
+        const int kb1 = (kb0 + p.kb_per_split < num_kb) ? kb0 + p.kb_per_split : num_kb;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(s), ph, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles + s * STAGE_BYTES;
@@ -350,7 +358,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t b_off = p.b_kmajor ? (uint32_t)(k * UMMA_K * 2) : (uint32_t)(k * UMMA_K * 128);
             const uint64_t adesc = make_smem_desc(a_src + a_off, p.a_kmajor != 0, 64 * BK * 2);
             const uint64_t bdesc = make_smem_desc(b_src + b_off, p.b_kmajor != 0, 64 * BK * 2);
-            tc_mma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            tc_mma_bf16_pair(d_tmem, adesc, bdesc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
           }
           issued = true;
           tc_commit_pair(empty_bar(s));   // frees the stage in both CTAs once these MMAs have read it
@@ -383,9 +391,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     bool ok = true;
     const bool has_cin = p.beta != 0.f;
     const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
-    for (int t = cid; t < p.num_tiles && ok; t += ncl) {
+    for (int u = cid; u < p.num_units && ok; u += ncl) {
       int tm, tn;
-      tile_coords(p, t, tm, tn);
+      tile_coords(p, u % p.num_tiles, tm, tn);
       // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
       const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
@@ -607,6 +615,34 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   }
   p.status = status_dev;
 
+  // Tile counts that do not fill the last wave of CTA pairs leave SMs idle.  A call that accumulates into C through
+  // the add-reduction epilogue may cut K into a few ranges per tile instead: the partial products add up in C (in an
+  // order that is not fixed, so the last bits of such sums can differ between runs).  A plain store into an fp32 C
+  // is turned into "clear C, then accumulate" when that pays.
+  const int pairs_max = sm_count() / 2;
+  const int num_kb = p.seg_kb * sg.nseg;
+  p.ksplit = 1;
+  if (p.epi_mode != EPI_DIRECT && p.num_tiles > 0) {
+    auto eff = [&](int ks) {
+      const double u = (double)p.num_tiles * ks;
+      return u / (ceil(u / pairs_max) * pairs_max);
+    };
+    int best = 1;
+    for (int ks = 2; ks <= 4; ++ks)
+      if (num_kb / ks >= 32 && eff(ks) > eff(best) + 0.03) best = ks;
+    if (best > 1) {
+      if (p.epi_mode == EPI_TMA_STORE) {
+        if (cudaMemset2DAsync(C.ptr, (size_t)C.ld * 4, 0, (size_t)N * 4, (size_t)M, stream) != cudaSuccess)
+          return SP_ERR_CUDA;
+        p.epi_mode = EPI_TMA_ADD;
+      }
+      p.ksplit = best;
+    }
+  }
+  p.kb_per_split = (int32_t)ceil_div(num_kb, p.ksplit);
+  p.ksplit = (int32_t)ceil_div(num_kb, p.kb_per_split);
+  p.num_units = p.num_tiles * p.ksplit;
+
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) !=
@@ -617,8 +653,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   count_launch();
   const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
   ProfScope prof(PK_GEMM_TC, flops, 0.0, stream);
-  const int pairs_max = sm_count() / 2;
-  const int pairs = p.num_tiles < pairs_max ? p.num_tiles : pairs_max;
+  const int pairs = p.num_units < pairs_max ? p.num_units : pairs_max;
   gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
 }
