@@ -49,7 +49,7 @@ constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 4 * STG_BYTES + 102
 constexpr long long WAIT_BUDGET_CYCLES = 4000000000LL;   // ~2 s
 constexpr long long DRAIN_BUDGET_CYCLES = 200000000LL;   // ~0.1 s
 
-enum EpiMode : int { EPI_DIRECT = 0, EPI_TMA_STORE = 1, EPI_TMA_ADD = 2 };
+enum EpiMode : int { EPI_DIRECT = 0, EPI_TMA_STORE = 1, EPI_TMA_ADD = 2, EPI_TMA_BF16_CIN = 3 };
 
 struct TcParams {
   int64_t M, N, K;
@@ -134,6 +134,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
+      : "memory");
+}
+// plain one-CTA load (epilogue: a block of Cin into this warp's shared tile, completing on this CTA's barrier)
+__device__ __forceinline__ void tma_load_2d_local(uint32_t dst, const CUtensorMap* map, int32_t c0, int32_t c1,
+                                                  uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int32_t c0, int32_t c1, uint32_t src) {
@@ -239,7 +247,7 @@ __device__ __forceinline__ void tc_commit_local(uint32_t bar) {
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmC, const TcParams p) {
+               const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmCin, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
@@ -255,6 +263,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
   const uint32_t drain_bar = bars + 8u * (2 * STAGES + 4);
+  auto cin_bar = [&](int q, int b) { return bars + 8u * (2 * STAGES + 5 + 2 * q + b); };   // per epilogue warp
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -268,6 +277,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }   // 4 warps x 2 CTAs
     mbar_init(drain_bar, 1);
+    for (int q = 0; q < 4; ++q) { mbar_init(cin_bar(q, 0), 1); mbar_init(cin_bar(q, 1), 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -387,7 +397,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t tempty_leader[2] = {map_to_cta(tempty_bar(0), 0), map_to_cta(tempty_bar(1), 0)};
     int acc = 0;
     uint32_t aph = 0;
-    int buf = 0;
+    int buf = 0, cbuf = 0;
+    uint32_t cph = 0;           // phase bit of each of the two Cin barriers
     bool ok = true;
     const bool has_cin = p.beta != 0.f;
     const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
@@ -401,7 +412,65 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int64_t row0 = (int64_t)tm * TILE_M + (int64_t)rank * BM + q * 32;   // first global row of this warp
       const uint32_t taddr = tmem_base + (uint32_t)(acc * TILE_N) + ((uint32_t)(q * 32) << 16);
       const int rows_here = (p.M - row0 < 32) ? (int)(p.M - row0) : 32;   // may be <= 0 on a ragged last tile
-      if (p.epi_mode != EPI_DIRECT) {
+      if (p.epi_mode == EPI_TMA_BF16_CIN) {
+        // bf16 C = beta * Cin + alpha * acc with both matrices moved by TMA: the warp's tile holds two 32 x 32 bf16
+        // blocks of Cin (loaded one block ahead) and two blocks of C.  64-byte rows, 64-byte swizzle: 16-byte chunk j
+        // of row r sits at chunk j ^ ((r >> 1) & 3).
+        const bool rows_ok = rows_here > 0;
+        const int nsl = (int)(((p.N - (int64_t)tn * TILE_N < TILE_N) ? (p.N - (int64_t)tn * TILE_N) : TILE_N) + 31) / 32;
+        if (rows_ok && lane == 0 && nsl > 0) {
+          fence_async_smem();
+          mbar_expect_tx(cin_bar(q, cbuf), 2048);
+          tma_load_2d_local(wstg + cbuf * 2048, &tmCin, (int32_t)((int64_t)tn * TILE_N), (int32_t)row0, cin_bar(q, cbuf));
+        }
+#pragma unroll 1
+        for (int sl = 0; sl < nsl; ++sl) {
+          const int64_t gj0 = (int64_t)tn * TILE_N + sl * 32;
+          uint32_t r[32];
+          tc_ld32(taddr + (uint32_t)(sl * 32), r);
+          tc_wait_ld();
+          if (rows_ok) {
+            if (lane == 0 && sl + 1 < nsl) {     // next block of Cin into the other half (its last reader is done)
+              fence_async_smem();
+              mbar_expect_tx(cin_bar(q, cbuf ^ 1), 2048);
+              tma_load_2d_local(wstg + (cbuf ^ 1) * 2048, &tmCin, (int32_t)(gj0 + 32), (int32_t)row0,
+                                cin_bar(q, cbuf ^ 1));
+            }
+            const bool got_c = mbar_wait(cin_bar(q, cbuf), (cph >> cbuf) & 1u, abort_flag, WAIT_BUDGET_CYCLES);
+            if (!__all_sync(0xffffffffu, got_c)) { ok = false; break; }
+            if (lane == 0) bulk_wait_read_1();
+            __syncwarp();
+            const uint8_t* in_row = wstg_ptr + cbuf * 2048 + lane * 64;
+            uint8_t* out_row = wstg_ptr + 4096 + buf * 2048 + lane * 64;
+            const int sw = (lane >> 1) & 3;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 cw = *reinterpret_cast<const uint4*>(in_row + ((j ^ sw) << 4));
+              const uint32_t cwv[4] = {cw.x, cw.y, cw.z, cw.w};
+              uint32_t ow[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 c2 = *reinterpret_cast<const __nv_bfloat162*>(&cwv[e]);
+                const float v0 = fmaf(p.beta, __low2float(c2), p.alpha * __uint_as_float(r[8 * j + 2 * e]));
+                const float v1 = fmaf(p.beta, __high2float(c2), p.alpha * __uint_as_float(r[8 * j + 2 * e + 1]));
+                const __nv_bfloat162 o2 = __floats2bfloat162_rn(v0, v1);
+                ow[e] = *reinterpret_cast<const uint32_t*>(&o2);
+              }
+              *reinterpret_cast<uint4*>(out_row + ((j ^ sw) << 4)) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + 4096 + buf * 2048);
+              bulk_commit();
+            }
+            cph ^= 1u << cbuf;
+            cbuf ^= 1;
+            buf ^= 1;
+          }
+        }
+        if (!ok) break;
+      } else if (p.epi_mode != EPI_DIRECT) {
         // 32 x 32 fp32 block -> 128-byte-swizzled shared tile (16-byte chunk j of row r sits at chunk j ^ (r & 7))
         // -> one TMA store / add-reduction, which clips at the edges of C.  Two tiles per warp alternate.
 #pragma unroll 1
@@ -519,8 +588,9 @@ EncodeTiledFn encode_fn() {
 //   bf16 operand, K-major : inner = K, outer = rows, box = {64, 128}
 //   bf16 operand, MN-major: inner = rows, outer = K, box = {64, 64}
 //   fp32 output C         : inner = N, outer = M, box = {32, 32}
+//   bf16 C / Cin          : inner = N, outer = M, box = {32, 32}, 64-byte swizzle
 bool make_map(CUtensorMap* map, bool f32, const void* ptr, int64_t inner, int64_t outer, int64_t ld, int box_inner,
-              int box_outer) {
+              int box_outer, bool swizzle64 = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
@@ -529,7 +599,8 @@ bool make_map(CUtensorMap* map, bool f32, const void* ptr, int64_t inner, int64_
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                   const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -577,8 +648,9 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   if (C.dtype != SP_F32 && C.dtype != SP_BF16) return SP_ERR_DTYPE;
   if (beta != 0.f && Cin.dtype != SP_F32 && Cin.dtype != SP_BF16) return SP_ERR_DTYPE;
 
-  CUtensorMap tmA, tmB, tmC;
+  CUtensorMap tmA, tmB, tmC, tmCin;
   memset(&tmC, 0, sizeof(tmC));
+  memset(&tmCin, 0, sizeof(tmCin));
   bool ok = A.kmajor ? make_map(&tmA, false, A.ptr, a_kext, a_mext, A.ld, BK, BM)
                      : make_map(&tmA, false, A.ptr, a_mext, a_kext, A.ld, 64, BK);
   ok = ok && (B.kmajor ? make_map(&tmB, false, B.ptr, b_kext, b_next, B.ld, BK, BNH)
@@ -600,6 +672,15 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   if (c_tma && beta == 0.f) p.epi_mode = EPI_TMA_STORE;
   if (c_tma && beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && Cin.s0 == C.ld) p.epi_mode = EPI_TMA_ADD;
   if (p.epi_mode != EPI_DIRECT && !make_map(&tmC, true, C.ptr, N, M, C.ld, 32, 32)) return SP_ERR_CUDA;
+  // bf16 C = beta * Cin + alpha * acc with a bf16 Cin: both through TMA
+  if (p.epi_mode == EPI_DIRECT && beta != 0.f && C.dtype == SP_BF16 && Cin.dtype == SP_BF16 && C.ld % 8 == 0 &&
+      Cin.s0 % 8 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0 &&
+      (reinterpret_cast<uintptr_t>(Cin.ptr) & 15u) == 0) {
+    if (!make_map(&tmC, false, C.ptr, N, M, C.ld, 32, 32, true) ||
+        !make_map(&tmCin, false, Cin.ptr, N, M, Cin.s0, 32, 32, true))
+      return SP_ERR_CUDA;
+    p.epi_mode = EPI_TMA_BF16_CIN;
+  }
   p.seg = sg;
   p.seg_kb = (int32_t)ceil_div(K, BK);
   p.tiles_m = (int32_t)ceil_div(M, TILE_M);
@@ -622,7 +703,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   const int pairs_max = sm_count() / 2;
   const int num_kb = p.seg_kb * sg.nseg;
   p.ksplit = 1;
-  if (p.epi_mode != EPI_DIRECT && p.num_tiles > 0) {
+  if ((p.epi_mode == EPI_TMA_STORE || p.epi_mode == EPI_TMA_ADD) && p.num_tiles > 0) {
     auto eff = [&](int ks) {
       const double u = (double)p.num_tiles * ks;
       return u / (ceil(u / pairs_max) * pairs_max);
@@ -654,7 +735,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
   ProfScope prof(PK_GEMM_TC, flops, 0.0, stream);
   const int pairs = p.num_units < pairs_max ? p.num_units : pairs_max;
-  gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, p);
+  gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
 }
 
