@@ -267,12 +267,22 @@ def main():
     peak_tf = peaks.get("bf16_tflops_sustained", 1400.0)
     peak_src = "measured (sustained, MEASURED_PEAKS.json)" if peaks else "fallback (1.4 PFLOP/s sustained)"
     achieved = tc["flops"] / (tc["ms"] * 1e-3) / 1e12 if tc["ms"] > 0 else 0.0
+    # DRAM traffic of the token-pass GEMMs from the ncu capture in profiles/gemm_tc_kernel_C2_one_chunk.md: the six
+    # products of one 16384-token chunk of C2 moved 4.84 GB; traffic grows in proportion to the tokens a launch covers.
+    traffic = None
+    if cfg.name == "C2" and cfg.d == 2048 and cfg.n == 8192 and cfg.k_keep == 4096 and tc["records"]:
+        traffic = 4.84e9 * (cfg.tokens / 16384.0) * args.steps / tc["records"]
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak_tf,
-                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None, "peak_source": peak_src,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": traffic,
+                "traffic_unit": "DRAM bytes per launch (ncu, one chunk, scaled by tokens)", "peak_source": peak_src,
                 "launches": tc["records"], "avg_launch_ms": tc["ms"] / max(tc["records"], 1),
                 "algorithmic_flops_per_launch": tc["flops"] / max(tc["records"], 1)}
     hbm = peaks.get("hbm_gbs", 6650.0)
     fu = prof["fused_update"]
+    roofline_hbm = {"bound": "hbm", "kernel": "fused_update_kernel",
+                    "achieved": fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 if fu["ms"] else 0.0, "peak": hbm, "unit": "GB/s",
+                    "frac": (fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 / hbm) if fu["ms"] else 0.0, "traffic": None,
+                    "launches": fu["records"]}
     breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / args.steps,
                      **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),
                      **({"gbs": v["bytes"] / (v["ms"] * 1e-3) / 1e9, "hbm_frac": v["bytes"] / (v["ms"] * 1e-3) / 1e9 / hbm}
@@ -315,7 +325,7 @@ def main():
             "config": {"workload": workload_name(cfg), "token_chunk": args.chunk,
                        "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
                        "parallelism": f"modules x{world} (independent, no collective)"},
-            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e, "cpu_baseline": cpu,
             "breakdown": breakdown}
     print(json.dumps(line))
     if world > 1:
