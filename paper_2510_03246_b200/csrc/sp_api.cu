@@ -159,6 +159,31 @@ __global__ void expand_group_index_kernel(const int32_t* unit_idx, int64_t k_uni
     col_idx[e] = unit_idx[e / group] * group + (int32_t)(e % group);
 }
 
+// A library-owned side stream per device: independent parts of one call (the W1 recovery next to the W2 recovery)
+// are forked onto it from the caller's stream and joined back with events, so the call stays asynchronous and
+// ordered on the caller's stream.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+SideStream* side_stream() {
+  static SideStream table[64];
+  static bool failed[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || failed[dev]) return nullptr;
+  SideStream& ss = table[dev];
+  if (!ss.stream) {
+    if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) != cudaSuccess) {
+      failed[dev] = true;
+      ss.stream = nullptr;
+      return nullptr;
+    }
+  }
+  return &ss;
+}
+
 bool valid_act_dtype(int32_t dt) { return dt == SP_F32 || dt == SP_BF16; }
 
 // ------------------------------------------------------------------------------------------------ workspace plans
@@ -169,6 +194,7 @@ struct AdmmPlan {
   size_t tsize;
   // device buffers
   SolveBufs sb;
+  SolveBufs sbA;               // buffers of the W1 recovery (system d, n right-hand sides), which runs concurrently
   float *W1t, *W2t, *Qt, *T0, *Cf;
   float *W2cf, *W1c;           // compact fp32 copies on the kept support: W2[:, S] ([d, kp]) and W1[S, :] ([k, d])
   int32_t* grp_base;           // kept-channel map of the elementwise kernels
@@ -194,6 +220,7 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   Carver c(ws);
   const int64_t nmax = n > d ? n : d;
   p.sb = carve_solve(c, nmax, nmax == n ? d : n, p.tsize);
+  p.sbA = carve_solve(c, d, n, p.tsize);
   p.W1t = c.take<float>((size_t)n * d);
   p.W2t = c.take<float>((size_t)n * d);
   p.Qt = c.take<float>((size_t)n * d);
@@ -565,18 +592,26 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   double* gam = p.sb.rho + 2;
 
   // ---- 1. weight recovery W1~ = R1 (G_X + rho1 I)^-1, W2~ = R2 (G_A + rho2 I)^-1
-  CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, s));
-  CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
-  if (bf16) {
-    SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sb, status_dev, s));
-    SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
-  } else {
-    SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sb, status_dev, s));
-    SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
+  // The two recoveries are independent; both are chains of short kernels that leave most SMs idle, so the W1 chain
+  // runs on the side stream while the caller's stream carries the W2 chain.
+  SideStream* side = side_stream();
+  cudaStream_t sa = side ? side->stream : s;
+  if (side) {
+    CU(cudaEventRecord(side->fork, s));
+    CU(cudaStreamWaitEvent(sa, side->fork, 0));
   }
+  CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
+  if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa));
+  else SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa));
+  if (side) CU(cudaEventRecord(side->join, sa));
+  bool joined = side == nullptr;
+  CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
+  if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
+  else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
 
   // ---- 2. unit scores and layer importance
   if (prm->score_kind == SP_SCORE_LEMMA1) {
+    if (!joined) { CU(cudaStreamWaitEvent(s, side->join, 0)); joined = true; }   // this score reads W1~
     // b = W1~ X, c = d = t = z^pre = W1_0 X, written through G_X:  T0 = W1_0 G_X
     MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, gx{st->G_X, SP_F32, d}, t0{p.T0, SP_F32, d};
     SPCHK(contract(n, d, d, 1.0, w10, true, gx, false, 0.0, t0, t0, false, true, false, status_dev, s));
@@ -592,6 +627,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   else CU(mask_to_index(st->mask, n, p.sb.idx, s));
 
   // ---- 4. masked weights: W1 = diag(M) W1~ ; W2 = recovery on the kept support (or M (.) W2~)
+  if (!joined) { CU(cudaStreamWaitEvent(s, side->join, 0)); joined = true; }
   CU(mask_rows_copy(st->mask, p.W1t, d, st->W1, d, n, d, s));
   if (prm->refit) {
     if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s));
