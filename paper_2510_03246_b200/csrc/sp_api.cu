@@ -123,7 +123,7 @@ SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
     const size_t np = (size_t)chol_tc_pad(nmax);
     b.P = c.take_bytes(np * 3 * np * 2);
     const size_t rows = (size_t)(nmax > mmax ? nmax : mmax);   // either dimension may be the right-hand-side count
-    b.Xs = c.take_bytes(rows * 3 * kCholTcNB * 2);
+    b.Xs = c.take_bytes(2 * rows * 3 * kCholTcNB * 2);
   }
   return b;
 }
@@ -132,7 +132,7 @@ SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
 template <typename T>
 sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_full,
                      const int32_t* idx, int64_t k, const double* rho_dev, float* W, int64_t ldw, SolveBufs& b,
-                     int32_t* status, cudaStream_t stream) {
+                     int32_t* status, cudaStream_t stream, const SolveAssist* assist = nullptr) {
   const int64_t nn = idx ? k : n_full;
   ProfScope prof(PK_SOLVE, (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
   T* Gs = reinterpret_cast<T*>(b.Gs);
@@ -143,7 +143,7 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
   if constexpr (sizeof(T) == 4) {
     SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream));
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
-    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream));
+    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist));
   } else {
     CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
@@ -165,7 +165,14 @@ __global__ void expand_group_index_kernel(const int32_t* unit_idx, int64_t k_uni
 struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, join = nullptr;
+  SolveAssist assist_main{}, assist_side{};   // helpers of the solves on the caller's stream / on `stream`
 };
+bool make_assist(SolveAssist& a) {
+  return cudaStreamCreateWithFlags(&a.stream, cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.panel_done, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.rest_done[0], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.rest_done[1], cudaEventDisableTiming) == cudaSuccess;
+}
 SideStream* side_stream() {
   static SideStream table[64];
   static bool failed[64] = {};
@@ -175,7 +182,8 @@ SideStream* side_stream() {
   if (!ss.stream) {
     if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) != cudaSuccess ||
+        !make_assist(ss.assist_main) || !make_assist(ss.assist_side)) {
       failed[dev] = true;
       ss.stream = nullptr;
       return nullptr;
@@ -397,7 +405,9 @@ sp_status sp_ridge_solve(const float* R, int64_t ldr, const float* G, int64_t ld
   SolveBufs b = carve_solve(c, n, m, precise ? 8 : 4);
   CU(effective_ridge(G, ldg, n, rho, rho_relative, b.rho, s));
   if (precise) return ridge_core<double>(R, ldr, G, ldg, m, n, nullptr, n, b.rho, W, ldw, b, status_dev, s);
-  return ridge_core<float>(R, ldr, G, ldg, m, n, nullptr, n, b.rho, W, ldw, b, status_dev, s);
+  SideStream* side = side_stream();
+  return ridge_core<float>(R, ldr, G, ldg, m, n, nullptr, n, b.rho, W, ldw, b, status_dev, s,
+                           side ? &side->assist_main : nullptr);
 }
 
 sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_units,
@@ -424,7 +434,9 @@ sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t l
     CU(cudaGetLastError());
   }
   if (precise) return ridge_core<double>(R, ldr, G, ldg, m, n, b.idx, k, b.rho, W, ldw, b, status_dev, s);
-  return ridge_core<float>(R, ldr, G, ldg, m, n, b.idx, k, b.rho, W, ldw, b, status_dev, s);
+  SideStream* side = side_stream();
+  return ridge_core<float>(R, ldr, G, ldg, m, n, b.idx, k, b.rho, W, ldw, b, status_dev, s,
+                           side ? &side->assist_main : nullptr);
 }
 
 sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* in, int64_t n_units, float* scores,
@@ -601,13 +613,17 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     CU(cudaStreamWaitEvent(sa, side->fork, 0));
   }
   CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
-  if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa));
-  else SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa));
+  if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
+                                    side ? &side->assist_side : nullptr));
+  else SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
+                                    side ? &side->assist_side : nullptr));
   if (side) CU(cudaEventRecord(side->join, sa));
   bool joined = side == nullptr;
   CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
-  if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
-  else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s));
+  if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
+                                    side ? &side->assist_main : nullptr));
+  else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
+                                    side ? &side->assist_main : nullptr));
 
   // ---- 2. unit scores and layer importance
   if (prm->score_kind == SP_SCORE_LEMMA1) {
@@ -630,8 +646,10 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   if (!joined) { CU(cudaStreamWaitEvent(s, side->join, 0)); joined = true; }
   CU(mask_rows_copy(st->mask, p.W1t, d, st->W1, d, n, d, s));
   if (prm->refit) {
-    if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s));
-    else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s));
+    if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
+                                      side ? &side->assist_main : nullptr));
+    else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
+                                      side ? &side->assist_main : nullptr));
   } else {
     CU(cudaMemcpyAsync(st->W2, p.W2t, (size_t)d * n * sizeof(float), cudaMemcpyDeviceToDevice, s));
     CU(zero_pruned(st->mask, 1, nullptr, 0, 0, 0, st->W2, d, n, n, s));
@@ -665,7 +683,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
       // right-hand sides: the rows of W2[:, S]^T as the tensor-core path sees them (bf16-rounded)
       CU(convert_matrix(p.W2b, SP_BF16, kp, p.W2cf, SP_F32, kp, d, k, s));
       CU(transpose_convert<float>(p.W2cf, kp, d, k, Rs, d, s));
-      SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s));
+      SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s,
+                           side ? &side->assist_main : nullptr));
       CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));
       qt = MatRef{p.Qtb, SP_BF16, d};
     } else {

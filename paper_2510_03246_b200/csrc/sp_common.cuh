@@ -100,13 +100,19 @@ constexpr int kCholNB = 64;
 // fp32 factorisation / solves with tensor-core trailing updates (sp_linalg_tc.cu).  Panels are kCholTcNB wide.
 //   dinv: ceil(n / kCholTcNB) blocks of 2 * kCholTcNB^2 floats (inverse diagonal blocks and their transposes)
 //   P   : bf16 [chol_tc_pad(n), 3 * chol_tc_pad(n)] — the factor below its diagonal blocks as three bf16 parts
-//   Xs  : bf16 [m, 3 * kCholTcNB] — the current block column of the right-hand sides as three bf16 parts
+//   Xs  : 2 x bf16 [m, 3 * kCholTcNB] — the current block column of the right-hand sides as three bf16 parts
 constexpr int kCholTcNB = 128;
 int64_t chol_tc_pad(int64_t n);
 sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P, int32_t* status_dev,
                          cudaStream_t stream);
+// Optional second stream (with three events) that carries the far part of each solve step's update.
+struct SolveAssist {
+  cudaStream_t stream;
+  cudaEvent_t panel_done, rest_done[2];
+};
+// Xs holds TWO buffers of [m, 3 * kCholTcNB] bf16.
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* P, const float* dinv, void* Xs,
-                         int32_t* status_dev, cudaStream_t stream);
+                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist = nullptr);
 
 // ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,

@@ -39,6 +39,7 @@ constexpr int TILE_N = 2 * BNH;
 constexpr int BK = 64;
 constexpr int STAGES = 6;
 constexpr int UMMA_K = 16;
+constexpr int kBandRows = 8;        // tile rows per band of a lower-triangle product
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BNH * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;          // 32 KB
@@ -230,13 +231,22 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, i
       tn = t / p.tiles_m;
     }
   } else {
-    // column block tn owns row blocks tn..tiles_m-1 (square tiles)
-    tn = 0;
+    // Lower triangle of a square grid of tiles, walked in bands of kBandRows tile rows, column by column inside a
+    // band: the tiles that run at the same time then share the band's few row panels (which stay in L2) and stream
+    // each column panel once per band.
+    int r0 = 0, r1 = 0;
     for (;;) {
-      const int cnt = p.tiles_m - tn;
-      if (t < cnt) { tm = tn + t; break; }
+      r1 = (r0 + kBandRows < p.tiles_m) ? r0 + kBandRows : p.tiles_m;
+      const int cnt = (r1 * (r1 + 1) - r0 * (r0 + 1)) / 2;     // sum over rows r0..r1-1 of (row + 1)
+      if (t < cnt || r1 >= p.tiles_m) break;     // the second test only bounds the loop
       t -= cnt;
-      ++tn;
+      r0 = r1;
+    }
+    for (tn = 0;; ++tn) {
+      const int first = tn > r0 ? tn : r0;
+      const int c = r1 - first;
+      if (t < c || tn >= p.tiles_m - 1) { tm = first + (t < c ? t : 0); break; }
+      t -= c;
     }
   }
 }

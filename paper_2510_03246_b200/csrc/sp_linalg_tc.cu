@@ -429,59 +429,89 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
 }
 
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* Pv, const float* dinv, void* Xsv,
-                         int32_t* status_dev, cudaStream_t stream) {
+                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist) {
   const __nv_bfloat16* P = reinterpret_cast<const __nv_bfloat16*>(Pv);
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(Xsv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
   const int64_t lds = 3 * TB;
-  TcOperand ta{Xs, lds, true};
-  ta.kext = lds;
-  ta.mnext = m;
-  // Y L^T = X, block columns left to right
-  for (int64_t j0 = 0; j0 < n; j0 += TB) {
-    const int nb = (int)((n - j0 < TB) ? (n - j0) : TB);
-    const float* dj = dinv + (j0 / TB) * 2 * TB * TB;
-    if (launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xs, lds, TB, true, stream) != cudaSuccess) return SP_ERR_CUDA;
-    const int64_t rem = n - j0 - nb;
-    if (rem <= 0) break;
-    // X[:, j1:] -= Y_j L[j1:, j0:j0+nb]^T : B(k, c) = L[j1 + c, j0 + k], K-major rows of P
-    TcOperand tb{P + (j0 + nb) * ldp, ldp, true};
-    tb.kext = ldp;
-    tb.mnext = rem;
-    TcSegments sg;
-    sg.nseg = 6;
-    for (int s = 0; s < 6; ++s) {
-      sg.a_k[s] = kPartA[s] * TB;
-      sg.b_k[s] = (int32_t)(kPartB[s] * np + j0);
-    }
-    float* Xr = X + j0 + nb;
-    sp_status st = gemm_tc(m, rem, TB, -1.f, ta, tb, 1.f, Operand{Xr, SP_F32, ldx, 1}, OutOperand{Xr, SP_F32, ldx},
-                           false, status_dev, stream, &sg, 2.0 * (double)m * (double)rem * (double)nb);
-    if (st != SP_OK) return st;
-  }
-  // W L = Y, block columns right to left
   const int64_t nblk = ceil_div(n, (int64_t)TB);
-  for (int64_t jb = nblk - 1; jb >= 0; --jb) {
-    const int64_t j0 = jb * TB;
-    const int nb = (int)((n - j0 < TB) ? (n - j0) : TB);
-    const float* dj = dinv + jb * 2 * TB * TB;
-    if (launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xs, lds, TB, true, stream) != cudaSuccess) return SP_ERR_CUDA;
-    if (j0 == 0) break;
-    // X[:, :j0] -= W_j L[j0:j0+nb, :j0] : B(k, c) = L[j0 + k, c], rows of P with the columns (N) contiguous
-    TcOperand tb{P + j0 * ldp, ldp, false};
-    tb.kext = n - j0;      // rows of L that exist; beyond them the tensor map returns zero
-    tb.mnext = ldp;
-    TcSegments sg;
-    sg.nseg = 6;
-    for (int s = 0; s < 6; ++s) {
-      sg.a_k[s] = kPartA[s] * TB;
-      sg.b_mn[s] = (int32_t)(kPartB[s] * np);
+  // Every step applies the inverse diagonal block to one block column (panel) and then updates the columns still to
+  // come.  With an assisting stream the update is cut in two: the next block column, which the next panel needs, stays
+  // on `stream`; the rest runs on the assisting stream and overlaps the next panel.  Panel jj then needs the "rest"
+  // update of step jj - 2 (and reuses its buffer of bf16 parts), which is what the two alternating events order.
+#define SP_CUDA_OK(x) do { if ((x) != cudaSuccess) return SP_ERR_CUDA; } while (0)
+  bool rec[2] = {false, false};
+  auto run_sweep = [&](bool forward) -> sp_status {
+    for (int64_t step = 0; step < nblk; ++step) {
+      const int64_t jb = forward ? step : nblk - 1 - step;
+      const int64_t j0 = jb * TB;
+      const int nb = (int)((n - j0 < TB) ? (n - j0) : TB);
+      const float* dj = dinv + jb * 2 * TB * TB;
+      __nv_bfloat16* Xcur = Xs + (step & 1) * m * lds;
+      if (assist && rec[step & 1]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[step & 1], 0));
+      cudaError_t e = forward ? launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, stream)
+                              : launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, stream);
+      if (e != cudaSuccess) return SP_ERR_CUDA;
+      // columns still to be updated: [lo, hi)
+      const int64_t lo = forward ? j0 + nb : 0, hi = forward ? n : j0;
+      if (hi <= lo) break;
+      if (assist) SP_CUDA_OK(cudaEventRecord(assist->panel_done, stream));
+      TcOperand ta{Xcur, lds, true};
+      ta.kext = lds;
+      ta.mnext = m;
+      // near part (next block column) and far part of the update
+      const int64_t wn = (hi - lo < TB) ? hi - lo : TB;
+      const int64_t near_lo = forward ? lo : hi - wn, far_lo = forward ? lo + wn : lo, far_w = hi - lo - wn;
+      for (int part = 0; part < 2; ++part) {
+        const int64_t c0 = part == 0 ? near_lo : far_lo, w = part == 0 ? wn : far_w;
+        if (w <= 0) continue;
+        const bool on_assist = assist && part == 1;
+        cudaStream_t st_run = on_assist ? assist->stream : stream;
+        if (on_assist) SP_CUDA_OK(cudaStreamWaitEvent(st_run, assist->panel_done, 0));
+        TcSegments sg;
+        sg.nseg = 6;
+        TcOperand tb{nullptr, ldp, forward};
+        if (forward) {
+          // X[:, c0:c0+w] -= Y_j L[c0:c0+w, j0:j0+nb]^T : B(k, c) = L[c0 + c, j0 + k], K-major rows of P
+          tb.ptr = P + c0 * ldp;
+          tb.kext = ldp;
+          tb.mnext = w;
+          for (int q = 0; q < 6; ++q) {
+            sg.a_k[q] = kPartA[q] * TB;
+            sg.b_k[q] = (int32_t)(kPartB[q] * np + j0);
+          }
+        } else {
+          // X[:, c0:c0+w] -= W_j L[j0:j0+nb, c0:c0+w] : B(k, c) = L[j0 + k, c0 + c], rows of P, columns (N) contiguous
+          tb.ptr = P + j0 * ldp;
+          tb.kext = n - j0;      // rows of L that exist; beyond them the tensor map returns zero
+          tb.mnext = ldp;
+          for (int q = 0; q < 6; ++q) {
+            sg.a_k[q] = kPartA[q] * TB;
+            sg.b_mn[q] = (int32_t)(kPartB[q] * np + c0);
+          }
+        }
+        float* Xc = X + c0;
+        sp_status stt = gemm_tc(m, w, TB, -1.f, ta, tb, 1.f, Operand{Xc, SP_F32, ldx, 1}, OutOperand{Xc, SP_F32, ldx},
+                                false, status_dev, st_run, &sg, 2.0 * (double)m * (double)w * (double)nb);
+        if (stt != SP_OK) return stt;
+        if (on_assist) {
+          SP_CUDA_OK(cudaEventRecord(assist->rest_done[step & 1], st_run));
+          rec[step & 1] = true;
+        }
+      }
     }
-    sp_status st = gemm_tc(m, j0, TB, -1.f, ta, tb, 1.f, Operand{X, SP_F32, ldx, 1}, OutOperand{X, SP_F32, ldx}, false,
-                           status_dev, stream, &sg, 2.0 * (double)m * (double)j0 * (double)nb);
-    if (st != SP_OK) return st;
-  }
-  return SP_OK;
+    // the sweep is complete on `stream` once the far updates still in flight have landed
+    for (int q = 0; q < 2; ++q)
+      if (assist && rec[q]) {
+        SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[q], 0));
+        rec[q] = false;
+      }
+    return SP_OK;
+  };
+  sp_status r = run_sweep(true);    // Y L^T = X, block columns left to right
+  if (r != SP_OK) return r;
+  return run_sweep(false);          // W L = Y, block columns right to left
+#undef SP_CUDA_OK
 }
 
 }  // namespace sp
