@@ -267,18 +267,37 @@ __device__ __forceinline__ float update_one(float zold, float z1, float dcorr, f
   return a;
 }
 
+__device__ __forceinline__ void store4(void* base, int32_t dt, int64_t e, const float* v) {
+  if (dt == SP_BF16) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]), hi = __floats2bfloat162_rn(v[2], v[3]);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(base) + e) = pk;
+  } else {
+    *reinterpret_cast<float4*>(reinterpret_cast<float*>(base) + e) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+}
+
 // The fused auxiliary-variable update of one chunk: per element a = h + D (h = phi(z) - u), z2, the select, the dual
 // update, the residual / norm partial sums and the column sums of |a|, reading Z (and U) once and writing Z (and U),
 // A and the storage copy of Z once.  D and z1 exist on the kept channels only (compact, see above); on a pruned
 // channel both are zero (its row of W1 and its row of Q are zero).
-// grid: (column blocks of 2048 channels, row blocks).  A thread owns 8 consecutive channels and walks its rows.
-// Sums: fp32 within one row of 8 elements and per column over the thread's rows (at most a few hundred terms), fp64
-// across rows and blocks.
+// grid: (column blocks of 1024 channels, row blocks).  A thread owns 4 consecutive channels and walks its rows two at
+// a time: all loads of both rows are issued before the first store, so that enough bytes are in flight per SM to
+// cover the DRAM latency (the kernel moves 12 n + 8 k bytes per token and does almost no arithmetic).
+// Sums: fp32 within one row and per column over the thread's rows (at most a few hundred terms), fp64 across rows
+// and blocks.
+template <bool HAS_U>
+struct UpdRow {
+  float zo[4], u[4], z1[4], dc[4];
+};
+
 template <bool HAS_U, int Z_RULE>
 __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   __shared__ double sm[32];
-  const int64_t grp = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  const int64_t c0 = grp * 8;
+  const int64_t grp4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int64_t c0 = grp4 * 4;
   const int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
   const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
   const int64_t r_end = (r_begin + rows_per < g.T) ? r_begin + rows_per : g.T;
@@ -288,58 +307,60 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   const float* __restrict__ z1p = g.z1;
   const float* __restrict__ Dp = g.D;
   double s_res = 0.0, s_z = 0.0, s_a = 0.0;
-  float cs[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float cs[4] = {0.f, 0.f, 0.f, 0.f};
   if (c0 < g.n) {
-    const int cnt = (g.n - c0 >= 8) ? 8 : (int)(g.n - c0);
-    const bool vec = (g.n % 8 == 0);
-    const unsigned bits = g.grp_mask[grp];
-    const int base = g.grp_base[grp];
-    // compact offset of each of the 8 channels (valid where its bit is set)
-    int off[8];
+    const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
+    const bool vec = (g.n % 4 == 0);
+    // kept channels of this half group and their compact offsets
+    const unsigned bits8 = g.grp_mask[grp4 >> 1];
+    const bool upper = (grp4 & 1) != 0;
+    const unsigned bits = upper ? (bits8 >> 4) : (bits8 & 0xFu);
+    const int base = g.grp_base[grp4 >> 1] + (upper ? __popc(bits8 & 0xFu) : 0);
+    int off[4];
     {
       int pos = 0;
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
+      for (int q = 0; q < 4; ++q) {
         off[q] = pos;
         pos += (bits >> q) & 1u;
       }
     }
-#pragma unroll 2
-    for (int64_t r = r_begin; r < r_end; ++r) {
+    auto load_row = [&](int64_t r, UpdRow<HAS_U>& w) {
       const int64_t e = r * g.n + c0;
-      float zo[8], u[8], z1[8], dc[8], a[8], zn[8];
       if (vec) {
-        const float4 v0 = *reinterpret_cast<const float4*>(Zp + e), v1 = *reinterpret_cast<const float4*>(Zp + e + 4);
-        zo[0] = v0.x; zo[1] = v0.y; zo[2] = v0.z; zo[3] = v0.w; zo[4] = v1.x; zo[5] = v1.y; zo[6] = v1.z; zo[7] = v1.w;
+        const float4 v = *reinterpret_cast<const float4*>(Zp + e);
+        w.zo[0] = v.x; w.zo[1] = v.y; w.zo[2] = v.z; w.zo[3] = v.w;
         if (HAS_U) {
-          const float4 w0 = *reinterpret_cast<const float4*>(Up + e), w1 = *reinterpret_cast<const float4*>(Up + e + 4);
-          u[0] = w0.x; u[1] = w0.y; u[2] = w0.z; u[3] = w0.w; u[4] = w1.x; u[5] = w1.y; u[6] = w1.z; u[7] = w1.w;
+          const float4 x = *reinterpret_cast<const float4*>(Up + e);
+          w.u[0] = x.x; w.u[1] = x.y; w.u[2] = x.z; w.u[3] = x.w;
         }
       } else {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          zo[q] = (q < cnt) ? Zp[e + q] : 0.f;
-          if (HAS_U) u[q] = (q < cnt) ? Up[e + q] : 0.f;
+        for (int q = 0; q < 4; ++q) {
+          w.zo[q] = (q < cnt) ? Zp[e + q] : 0.f;
+          if (HAS_U) w.u[q] = (q < cnt) ? Up[e + q] : 0.f;
         }
       }
       if (!HAS_U) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) u[q] = 0.f;
+        for (int q = 0; q < 4; ++q) w.u[q] = 0.f;
       }
-      {
-        const float* zp = z1p + r * g.ldk + base;
-        const float* dp = Dp + r * g.ldk + base;
+      const float* zp = z1p + r * g.ldk + base;
+      const float* dp = Dp + r * g.ldk + base;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const bool kept = (bits >> q) & 1u;
-          z1[q] = kept ? zp[off[q]] : 0.f;
-          dc[q] = kept ? dp[off[q]] : 0.f;
-        }
+      for (int q = 0; q < 4; ++q) {
+        const bool kept = (bits >> q) & 1u;
+        w.z1[q] = kept ? zp[off[q]] : 0.f;
+        w.dc[q] = kept ? dp[off[q]] : 0.f;
       }
+    };
+    auto finish_row = [&](int64_t r, UpdRow<HAS_U>& w) {
+      const int64_t e = r * g.n + c0;
+      float a[4], zn[4];
       float p_res = 0.f, p_z = 0.f, p_a = 0.f;
 #pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        a[q] = update_one(zo[q], z1[q], dc[q], u[q], HAS_U, g.alpha, g.beta, inv_ab, Z_RULE, zn[q]);
+      for (int q = 0; q < 4; ++q) {
+        a[q] = update_one(w.zo[q], w.z1[q], w.dc[q], w.u[q], HAS_U, g.alpha, g.beta, inv_ab, Z_RULE, zn[q]);
         if (!vec && q >= cnt) { a[q] = 0.f; zn[q] = 0.f; }
         const float diff = a[q] - fmaxf(zn[q], 0.f);
         p_res = fmaf(diff, diff, p_res);
@@ -352,19 +373,15 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
       s_a += (double)p_a;
       if (vec) {
         *reinterpret_cast<float4*>(Zp + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
-        *reinterpret_cast<float4*>(Zp + e + 4) = make_float4(zn[4], zn[5], zn[6], zn[7]);
-        if (HAS_U) {
-          *reinterpret_cast<float4*>(Up + e) = make_float4(u[0], u[1], u[2], u[3]);
-          *reinterpret_cast<float4*>(Up + e + 4) = make_float4(u[4], u[5], u[6], u[7]);
-        }
-        store8(g.A_out, g.out_dtype, e, a);
-        if (g.Zb_out) store8(g.Zb_out, g.out_dtype, e, zn);
+        if (HAS_U) *reinterpret_cast<float4*>(Up + e) = make_float4(w.u[0], w.u[1], w.u[2], w.u[3]);
+        store4(g.A_out, g.out_dtype, e, a);
+        if (g.Zb_out) store4(g.Zb_out, g.out_dtype, e, zn);
       } else {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < 4; ++q) {
           if (q < cnt) {
             Zp[e + q] = zn[q];
-            if (HAS_U) Up[e + q] = u[q];
+            if (HAS_U) Up[e + q] = w.u[q];
             if (g.out_dtype == SP_BF16) {
               reinterpret_cast<__nv_bfloat16*>(g.A_out)[e + q] = __float2bfloat16_rn(a[q]);
               if (g.Zb_out) reinterpret_cast<__nv_bfloat16*>(g.Zb_out)[e + q] = __float2bfloat16_rn(zn[q]);
@@ -375,10 +392,27 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
           }
         }
       }
+    };
+    int64_t r = r_begin;
+    for (; r + 3 < r_end; r += 4) {
+      UpdRow<HAS_U> w0, w1, w2, w3;
+      load_row(r, w0);
+      load_row(r + 1, w1);
+      load_row(r + 2, w2);
+      load_row(r + 3, w3);
+      finish_row(r, w0);
+      finish_row(r + 1, w1);
+      finish_row(r + 2, w2);
+      finish_row(r + 3, w3);
+    }
+    for (; r < r_end; ++r) {
+      UpdRow<HAS_U> w0;
+      load_row(r, w0);
+      finish_row(r, w0);
     }
     if (g.absA_part) {
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
+      for (int q = 0; q < 4; ++q)
         if (q < cnt) g.absA_part[(int64_t)blockIdx.y * g.n + c0 + q] = (double)cs[q];
     }
   }
@@ -636,8 +670,8 @@ cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, 
 }
 
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
-  const int col_blocks = (int)ceil_div(n, 2048);
-  int rb = (148 * 8 + col_blocks - 1) / col_blocks;
+  const int col_blocks = (int)ceil_div(n, 1024);
+  int rb = (148 * 16 + col_blocks - 1) / col_blocks;
   if (rb > T) rb = (int)T;
   if (rb < 1) rb = 1;
   if (rb > 65535) rb = 65535;
@@ -647,7 +681,7 @@ int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
 
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   if (a.T * a.n == 0) return cudaSuccess;
-  dim3 grid((unsigned)ceil_div(a.n, 2048), (unsigned)a.row_blocks);
+  dim3 grid((unsigned)ceil_div(a.n, 1024), (unsigned)a.row_blocks);
   // algorithmic bytes per row: Z (and U) read and written, A and the storage copy of Z written, z1 and D read on the
   // kept channels
   const double esz = a.out_dtype == SP_BF16 ? 2.0 : 4.0;
