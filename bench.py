@@ -208,7 +208,7 @@ def main():
     layer = rank
     X = synth.make_activations(cfg, layer, device=dev)
     W1_0, W2_0 = synth.make_weights(cfg, layer, device=dev)
-    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=args.chunk)
+    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=args.chunk, overlap_k=cfg.k_keep)
     I_all = synth.make_importances(cfg, device=dev)
     n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
     T_soft = float(I_all.abs().mean())
@@ -301,7 +301,7 @@ def main():
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
-        m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk)
+        m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk, overlap_k=cfg.k_keep)
         m2.sp_ffn_init()
         for _ in range(iters):
             m2.sp_admm_step(prm)

@@ -274,6 +274,11 @@ int64_t sp_launch_count(void);
  *   SP_WS_SCORES: d = n_units*group, N = tokens (LEMMA1) or rows of W (WANDA).
  *   SP_WS_RIDGE_SOLVE / SP_WS_LINEAR_REFIT: d = m (rows of R), n = system size, dtype SP_F64 when precise != 0. */
 size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t token_chunk, int32_t dtype);
+/* Optional extra workspace of sp_admm_step (bf16 mode): when ws_bytes >= sp_workspace_bytes(SP_WS_ADMM_STEP, ...) +
+ * sp_admm_overlap_bytes(N, k_keep), the step keeps z^(1) = W1 X of all N tokens on the kept channels (fp32) in the
+ * tail of the workspace and computes it concurrently with the recovery of W2 on the kept support; results are the
+ * same, the step is faster. */
+size_t sp_admm_overlap_bytes(int64_t N, int64_t k_keep);
 const char* sp_status_string(int32_t status);
 int32_t sp_version(void);
 

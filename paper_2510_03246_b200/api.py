@@ -25,7 +25,7 @@ SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
  SP_WS_RIDGE_SOLVE) = range(8)
 
 EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
-           "sp_apply_mask", "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes",
+           "sp_apply_mask", "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
            "sp_profile_kind_name", "sp_launch_count"]
 
@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
         L = C.CDLL(LIB_PATH)
         L.sp_workspace_bytes.restype = C.c_size_t
         L.sp_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_int32]
+        L.sp_admm_overlap_bytes.restype = C.c_size_t
+        L.sp_admm_overlap_bytes.argtypes = [C.c_int64, C.c_int64]
         L.sp_status_string.restype = C.c_char_p
         L.sp_status_string.argtypes = [C.c_int32]
         L.sp_version.restype = C.c_int32
@@ -102,7 +104,7 @@ def lib() -> C.CDLL:
         L.sp_profile_kind_name.argtypes = [i32]
         L.sp_launch_count.restype = i64
         for name in EXPORTS:
-            if name not in ("sp_workspace_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
+            if name not in ("sp_workspace_bytes", "sp_admm_overlap_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
                             "sp_profile_kind_name", "sp_launch_count"):
                 getattr(L, name).restype = C.c_int32
         _lib = L
@@ -320,7 +322,9 @@ class FfnModule:
     """Owns the device buffers of one FFN module and forwards to sp_ffn_init / sp_admm_step."""
 
     def __init__(self, X: torch.Tensor, W1_0: torch.Tensor, W2_0: torch.Tensor, dual_mode: bool = False,
-                 token_chunk: int = 0):
+                 token_chunk: int = 0, overlap_k: int = 0):
+        """overlap_k > 0: also reserve the optional workspace tail that lets sp_admm_step compute z1 of all tokens
+        beside the kept-support recovery, sized for overlap_k kept units (see sp_admm_overlap_bytes)."""
         _require_cuda(X, W1_0, W2_0)
         assert X.dtype in (torch.float32, torch.bfloat16)
         self.X = X.contiguous()
@@ -348,6 +352,7 @@ class FfnModule:
         self.report = torch.zeros(len(REPORT_FIELDS), dtype=torch.float64, device=dev)
         self.status = new_status(dev)
         self.token_chunk = token_chunk
+        self.overlap_k = int(overlap_k)
         self._ws = None
         self.iteration = 0
 
@@ -364,6 +369,8 @@ class FfnModule:
     def _workspace(self, chunk: int) -> torch.Tensor:
         need = max(workspace_bytes(SP_WS_ADMM_STEP, self.d, self.n, self.N, chunk, _dt(self.X)),
                    workspace_bytes(SP_WS_FFN_INIT, self.d, self.n, self.N, chunk, _dt(self.X)))
+        if self.overlap_k > 0:
+            need += int(lib().sp_admm_overlap_bytes(self.N, self.overlap_k))
         if self._ws is None or self._ws.numel() < need:
             self._ws = _ws(need, self.dev)
         return self._ws

@@ -1,5 +1,6 @@
 // C-ABI entry points of libsp and the host-side orchestration of the per-module ADMM step.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "sp_common.cuh"
@@ -19,6 +20,17 @@ using namespace sp;
 namespace {
 
 constexpr int64_t kDefaultChunk = 32768;
+// SM pairs given to the z1 products that run beside the kept-support recovery (of 74 on a B200); the environment
+// variable SP_Z1_AHEAD_PAIRS overrides it (a tuning knob, read once).
+int z1_ahead_pairs() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SP_Z1_AHEAD_PAIRS");
+    v = e ? atoi(e) : 58;
+    if (v < 1) v = 58;
+  }
+  return v;
+}
 
 struct MatRef {
   const void* ptr;
@@ -54,7 +66,7 @@ sp_status contract(int64_t M, int64_t N, int64_t K, double alpha, MatRef A, bool
 int64_t split_kpad(int64_t K) { return (K + 63) / 64 * 64; }
 
 sp_status contract_split_weights(int64_t M, int64_t N, int64_t K, MatRef A, const void* Wsplit, MatRef Wf32, MatRef C,
-                                 int32_t* status, cudaStream_t stream) {
+                                 int32_t* status, cudaStream_t stream, int max_pairs = 0) {
   if (M <= 0 || N <= 0) return SP_OK;
   const int64_t kp = split_kpad(K);
   TcOperand ta{A.ptr, A.ld, true}, tb{Wsplit, 2 * kp, true};
@@ -65,7 +77,8 @@ sp_status contract_split_weights(int64_t M, int64_t N, int64_t K, MatRef A, cons
     TcSegments sg;
     sg.nseg = 2;            // hi part, then lo part, against the same A tile
     sg.b_k[1] = (int32_t)kp;
-    return gemm_tc(M, N, K, 1.f, ta, tb, 0.f, cin, out, false, status, stream, &sg, 2.0 * (double)M * N * K);
+    return gemm_tc(M, N, K, 1.f, ta, tb, 0.f, cin, out, false, status, stream, &sg, 2.0 * (double)M * N * K,
+                   max_pairs);
   }
   if (Wf32.ptr) return contract(M, N, K, 1.0, A, true, Wf32, true, 0.0, C, C, false, false, false, status, stream);
   // no fp32 copy at hand: hi and lo parts one after the other on the CUDA cores
@@ -164,7 +177,7 @@ __global__ void expand_group_index_kernel(const int32_t* unit_idx, int64_t k_uni
 // ordered on the caller's stream.
 struct SideStream {
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, z1_done = nullptr;
   SolveAssist assist_main{}, assist_side{};   // helpers of the solves on the caller's stream / on `stream`
 };
 bool make_assist(SolveAssist& a) {
@@ -183,6 +196,7 @@ SideStream* side_stream() {
     if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ss.z1_done, cudaEventDisableTiming) != cudaSuccess ||
         !make_assist(ss.assist_main) || !make_assist(ss.assist_side)) {
       failed[dev] = true;
       ss.stream = nullptr;
@@ -210,6 +224,7 @@ struct AdmmPlan {
   void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
   void *H, *E, *Ac, *Zb;
   float *D, *z1;
+  float* z1_all;               // [N, kp] behind the planned bytes when the caller's workspace has room for it
   double *partial, *absA_part, *score_scratch;
   int row_blocks, nblocks;
   size_t bytes;
@@ -253,8 +268,11 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.absA_part = c.take<double>((size_t)p.row_blocks * n);
   p.score_scratch = c.take<double>((size_t)score_row_blocks(d, n) * n * 2 + 16);
   p.bytes = align_up(c.off, 256);
+  p.z1_all = ws ? reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(ws) + p.bytes) : nullptr;   // optional tail
   return p;
 }
+
+size_t overlap_bytes(int64_t N, int64_t k) { return (size_t)N * (size_t)((k + 7) / 8 * 8) * sizeof(float); }
 
 struct InitPlan {
   int64_t chunk;
@@ -294,6 +312,8 @@ size_t ridge_ws_bytes(int64_t m, int64_t n, bool precise) {
 extern "C" {
 
 int32_t sp_version(void) { return 100; }
+
+size_t sp_admm_overlap_bytes(int64_t N, int64_t k_keep) { return (N > 0 && k_keep > 0) ? overlap_bytes(N, k_keep) : 0; }
 
 const char* sp_status_string(int32_t s) {
   switch (s) {
@@ -645,6 +665,25 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   // ---- 4. masked weights: W1 = diag(M) W1~ ; W2 = recovery on the kept support (or M (.) W2~)
   if (!joined) { CU(cudaStreamWaitEvent(s, side->join, 0)); joined = true; }
   CU(mask_rows_copy(st->mask, p.W1t, d, st->W1, d, n, d, s));
+  // z1 = X W1[S, :]^T needs only the mask and W1: when the workspace has room for z1 of all tokens, these products
+  // run on the side stream, on a subset of the SMs, while the caller's stream carries the recovery of W2 on the kept
+  // support and the operands of the a-update (chains of short kernels that cannot fill the GPU).
+  const int64_t kp_ahead = (k + 7) / 8 * 8;
+  const bool z1_ahead = bf16 && side != nullptr && ws_bytes >= p.bytes + overlap_bytes(N, k);
+  if (z1_ahead) {
+    CU(cudaEventRecord(side->fork, s));
+    CU(cudaStreamWaitEvent(side->stream, side->fork, 0));
+    CU(split_bf16(st->W1, d, p.sb.idx, k, d, split_kpad(d), p.W1b, side->stream));
+    const size_t esz_x = 2;
+    for (int64_t t0 = 0; t0 < N; t0 += p.chunk) {
+      const int64_t Tc = (N - t0 < p.chunk) ? N - t0 : p.chunk;
+      MatRef xc{reinterpret_cast<const uint8_t*>(m->X.ptr) + (size_t)t0 * m->X.ld * esz_x, cdt, m->X.ld};
+      MatRef z1c{p.z1_all + (size_t)t0 * kp_ahead, SP_F32, kp_ahead};
+      SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, MatRef{nullptr, SP_F32, d}, z1c, status_dev, side->stream,
+                                   z1_ahead_pairs()));
+    }
+    CU(cudaEventRecord(side->z1_done, side->stream));
+  }
   if (prm->refit) {
     if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
                                       side ? &side->assist_main : nullptr));
@@ -663,7 +702,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   CU(gather_cols<float>(st->W2, n, idx, d, k, p.W2cf, kp, s));
   MatRef w1{nullptr, SP_F32, d}, w2{p.W2cf, SP_F32, kp}, qt{p.Qt, SP_F32, d};
   if (bf16) {
-    CU(split_bf16(st->W1, d, idx, k, d, split_kpad(d), p.W1b, s));
+    if (!z1_ahead) CU(split_bf16(st->W1, d, idx, k, d, split_kpad(d), p.W1b, s));
     CU(convert_matrix(p.W2cf, SP_F32, kp, p.W2b, SP_BF16, kp, d, k, s));
     w2 = MatRef{p.W2b, SP_BF16, kp};
   } else {
@@ -699,6 +738,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   }
 
   // ---- 5b. token pass
+  if (z1_ahead) CU(cudaStreamWaitEvent(s, side->z1_done, 0));
   if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, s));
   const size_t esz = bf16 ? 2 : 4;
   MatRef ga{st->G_A, SP_F32, n}, r1{st->R1, SP_F32, d}, r2{st->R2, SP_F32, n};
@@ -715,10 +755,11 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     // E = Ypre - h_S W2[:, S]^T ; D_S = E Qt^T ; z1_S = X W1[S, :]^T
     SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
     SPCHK(contract(Tc, k, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
-    if (bf16) SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, w1, z1, status_dev, s));
+    if (z1_ahead) {}   // already there for all tokens
+    else if (bf16) SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, w1, z1, status_dev, s));
     else SPCHK(contract(Tc, k, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, false, status_dev, s));
     UpdateArgs ua;
-    ua.Z = Zc; ua.U = Uc; ua.z1 = p.z1; ua.D = p.D; ua.ldk = kp; ua.k = k; ua.grp_base = p.grp_base;
+    ua.Z = Zc; ua.U = Uc; ua.z1 = z1_ahead ? p.z1_all + (size_t)t0 * kp : p.z1; ua.D = p.D; ua.ldk = kp; ua.k = k; ua.grp_base = p.grp_base;
     ua.grp_mask = p.grp_mask; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
     ua.out_dtype = cdt; ua.T = Tc; ua.n = n; ua.alpha = (float)prm->alpha; ua.beta = (float)prm->beta;
     ua.z_rule = prm->z_rule; ua.partial = p.partial; ua.absA_part = p.absA_part;

@@ -77,10 +77,11 @@ struct TcSegments {
   int32_t a_k[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, a_mn[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
   int32_t b_k[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, b_mn[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
 };
-// K is the extent of ONE segment.  alg_flops >= 0 overrides the flop count recorded for profiling.
+// K is the extent of ONE segment.  alg_flops >= 0 overrides the flop count recorded for profiling.  max_pairs > 0
+// limits the launch to that many CTA pairs (SM pairs), leaving the other SMs to kernels of another stream.
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
                   OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream,
-                  const TcSegments* segs = nullptr, double alg_flops = -1.0);
+                  const TcSegments* segs = nullptr, double alg_flops = -1.0, int max_pairs = 0);
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B);
 
 // Dense symmetric positive definite solve in precision T (float or double), all on `stream`.

@@ -637,7 +637,7 @@ bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B
 
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
                   OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, const TcSegments* segs,
-                  double alg_flops) {
+                  double alg_flops, int max_pairs) {
   TcSegments sg;
   if (segs) sg = *segs;
   else { sg = TcSegments{}; sg.nseg = 1; }
@@ -710,7 +710,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   // the add-reduction epilogue may cut K into a few ranges per tile instead: the partial products add up in C (in an
   // order that is not fixed, so the last bits of such sums can differ between runs).  A plain store into an fp32 C
   // is turned into "clear C, then accumulate" when that pays.
-  const int pairs_max = sm_count() / 2;
+  int pairs_max = sm_count() / 2;
+  if (max_pairs > 0 && max_pairs < pairs_max) pairs_max = max_pairs;
   const int num_kb = p.seg_kb * sg.nseg;
   p.ksplit = 1;
   if ((p.epi_mode == EPI_TMA_STORE || p.epi_mode == EPI_TMA_ADD) && p.num_tiles > 0) {

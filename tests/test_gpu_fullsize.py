@@ -43,7 +43,7 @@ def run():
     cfg = CFG
     X = synth.make_activations(cfg, 0, device=DEV)
     W1_0, W2_0 = synth.make_weights(cfg, 0, device=DEV)
-    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=CHUNK)
+    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=CHUNK, overlap_k=cfg.k_keep)
     mod.sp_ffn_init()
     torch.cuda.synchronize()
     mod.check_status()

@@ -272,10 +272,10 @@ def test_apply_mask_argument_errors():
 
 
 # ------------------------------------------------------------------------------------------------ module: init + step
-def _make_module(cfg, dual=False, chunk=0, seed_layer=0):
+def _make_module(cfg, dual=False, chunk=0, seed_layer=0, overlap_k=0):
     X = synth.make_activations(cfg, seed_layer)
     W1, W2 = synth.make_weights(cfg, seed_layer)
-    mod = api.FfnModule(X.to(DEV), W1.to(DEV), W2.to(DEV), dual_mode=dual, token_chunk=chunk)
+    mod = api.FfnModule(X.to(DEV), W1.to(DEV), W2.to(DEV), dual_mode=dual, token_chunk=chunk, overlap_k=overlap_k)
     return mod, X, W1, W2
 
 
@@ -390,6 +390,19 @@ def test_admm_step_teacher_forced(cfg, chunk, kind, rule, dual, refit):
                            score_kind=_KIND[kind], refit=refit, token_chunk=chunk)
     p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=rule, dual_mode=dual, score_kind=kind,
                         refit=refit)
+    audit = []
+    for it in range(3):
+        _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
+
+
+def test_admm_step_with_z1_computed_ahead():
+    """Same step with the optional workspace tail: z1 of all tokens is computed on the side stream beside the
+    kept-support recovery (the configuration bench.py runs)."""
+    cfg = SMALL_BF16
+    mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=cfg.k_keep)
+    mod.sp_ffn_init()
+    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, token_chunk=512)
+    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep)
     audit = []
     for it in range(3):
         _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
