@@ -176,7 +176,8 @@ def run_reference(args, cfg):
 
 
 def workload_name(cfg) -> str:
-    return (f"{cfg.name}: OPT-1.3B-shaped FFN module, d={cfg.d}, n={cfg.n}, N={cfg.tokens} tokens, "
+    shape = {"C1": "OPT-125M", "C2": "OPT-1.3B", "C3": "OPT-6.7B", "C4": "LLaMA-2-7B", "C5": "OPT-30B"}.get(cfg.name, "OPT")
+    return (f"{cfg.name}: {shape}-shaped FFN module, d={cfg.d}, n={cfg.n}, N={cfg.tokens} tokens, "
             f"{cfg.storage} activations, {int(cfg.sparsity * 100)}% channel sparsity (k_keep={cfg.k_keep})")
 
 
