@@ -105,7 +105,7 @@ typedef struct {
   int32_t reselect_mask;   /* 1: recompute the top-k mask from this step's scores; 0: keep st->mask                */
   int32_t refit;           /* 1: recovery solver on the kept support (Algorithm 2); 0: plain M (.) W               */
   int64_t token_chunk;     /* tokens per streamed chunk (0 = library default)                                      */
-  int32_t compute_objective; /* 1: also report alpha|Ypre-W2A|^2 and alpha|Z-W1X|^2                               */
+  int32_t compute_objective; /* 1: also report alpha|Ypre-W2A|^2 (one more product per token chunk)                 */
   int32_t reserved;
 } sp_admm_params;
 
@@ -113,7 +113,7 @@ typedef struct {
 typedef struct {
   double res_act;   /* |A - phi(Z_new)|^2                                                                         */
   double res_out;   /* alpha |Ypre - W2 A|^2   (NaN unless compute_objective)                                      */
-  double res_in;    /* alpha |Z_new - W1 X|^2  (NaN unless compute_objective)                                      */
+  double res_in;    /* alpha |Z_new - W1 X|^2                                                                      */
   double z_sq;      /* |Z_new|^2                                                                                  */
   double a_sq;      /* |A|^2                                                                                      */
   double rho1_eff, rho2_eff; /* ridge terms actually used                                                         */

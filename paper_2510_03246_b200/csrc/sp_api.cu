@@ -223,7 +223,8 @@ struct AdmmPlan {
   uint8_t* grp_mask;
   void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
   void *H, *E, *Ac, *Zb;
-  float *D, *z1;
+  float *D, *z1, *Eo;          // Eo: Ypre - A W2^T of a chunk (objective reporting)
+  void* W2fb;                  // bf16 copy of the full W2 (objective reporting)
   float* z1_all;               // [N, kp] behind the planned bytes when the caller's workspace has room for it
   double *partial, *absA_part, *score_scratch;
   int row_blocks, nblocks;
@@ -264,7 +265,9 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.D = c.take<float>((size_t)p.chunk * npad);
   p.z1 = c.take<float>((size_t)p.chunk * npad);
   p.nblocks = fused_update_grid(p.chunk, n, &p.row_blocks);
-  p.partial = c.take<double>((size_t)p.nblocks * 3);
+  p.partial = c.take<double>((size_t)p.nblocks * 4 + kSumsqBlocks);
+  p.Eo = c.take<float>((size_t)p.chunk * d);
+  p.W2fb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
   p.absA_part = c.take<double>((size_t)p.row_blocks * n);
   p.score_scratch = c.take<double>((size_t)score_row_blocks(d, n) * n * 2 + 16);
   p.bytes = align_up(c.off, 256);
@@ -737,6 +740,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     }
   }
 
+  if (rep_dev && prm->compute_objective && bf16) CU(convert_matrix(st->W2, SP_F32, n, p.W2fb, SP_BF16, n, d, n, s));
+
   // ---- 5b. token pass
   if (z1_ahead) CU(cudaStreamWaitEvent(s, side->z1_done, 0));
   if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, s));
@@ -765,7 +770,14 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     ua.z_rule = prm->z_rule; ua.partial = p.partial; ua.absA_part = p.absA_part;
     const int nblk = fused_update_grid(Tc, n, &ua.row_blocks);
     CU(launch_fused_update(ua, s));
-    if (rep_dev) CU(reduce_report(p.partial, nblk, rep_dev, ci > 0, s));
+    if (rep_dev) CU(reduce_report(p.partial, nblk, rep_dev, ci > 0, prm->alpha, s));
+    if (rep_dev && prm->compute_objective) {
+      // alpha |Ypre - W2 A|^2 of the new A: one more product per chunk, only on request
+      MatRef w2f = bf16 ? MatRef{p.W2fb, SP_BF16, n} : MatRef{st->W2, SP_F32, n};
+      MatRef eo{p.Eo, SP_F32, d};
+      SPCHK(contract(Tc, d, n, -1.0, ac, true, w2f, true, 1.0, yc, eo, false, acc64, bf16, status_dev, s));
+      CU(sumsq_accumulate(p.Eo, d, Tc, d, prm->alpha, &rep_dev->res_out, ci > 0, p.partial + (size_t)p.nblocks * 4, s));
+    }
     CU(reduce_col_partials(p.absA_part, ua.row_blocks, n, st->absA, ci > 0, s));
     // accumulators of the new auxiliary variables
     SPCHK(contract(n, n, Tc, 1.0, ac, false, ac, false, acc, ga, ga, true, acc64, bf16, status_dev, s));

@@ -167,7 +167,7 @@ struct UpdateArgs {
   int64_t T, n;
   float alpha, beta;
   int32_t z_rule;
-  double* partial;   // [gridDim.x * 3] block partial sums: res_act, z_sq, a_sq
+  double* partial;   // [blocks * 4] block partial sums: res_act, z_sq, a_sq, |z_new - z1|^2
   double* absA_part; // [row_blocks, n] partial column sums of |A|
   int32_t row_blocks;
 };
@@ -182,8 +182,12 @@ int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
                                 cudaStream_t stream);
 // rep[field] (+)= sum of partial triples
-cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate,
+cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate, double alpha,
                           cudaStream_t stream);
+// out[0] (+)= scale * sum of squares of a fp32 matrix; scratch: kSumsqBlocks doubles
+constexpr int kSumsqBlocks = 592;
+cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t cols, double scale, double* out,
+                             bool accumulate, double* scratch, cudaStream_t stream);
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
                         cudaStream_t stream);
 // relu + storage conversion for the init pass: A = phi(Z) -> storage dtype, and |A| column partials

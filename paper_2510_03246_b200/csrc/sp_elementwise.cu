@@ -306,7 +306,7 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   float* __restrict__ Up = g.U;
   const float* __restrict__ z1p = g.z1;
   const float* __restrict__ Dp = g.D;
-  double s_res = 0.0, s_z = 0.0, s_a = 0.0;
+  double s_res = 0.0, s_z = 0.0, s_a = 0.0, s_in = 0.0;
   float cs[4] = {0.f, 0.f, 0.f, 0.f};
   if (c0 < g.n) {
     const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
@@ -357,11 +357,13 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
     auto finish_row = [&](int64_t r, UpdRow<HAS_U>& w) {
       const int64_t e = r * g.n + c0;
       float a[4], zn[4];
-      float p_res = 0.f, p_z = 0.f, p_a = 0.f;
+      float p_res = 0.f, p_z = 0.f, p_a = 0.f, p_in = 0.f;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         a[q] = update_one(w.zo[q], w.z1[q], w.dc[q], w.u[q], HAS_U, g.alpha, g.beta, inv_ab, Z_RULE, zn[q]);
-        if (!vec && q >= cnt) { a[q] = 0.f; zn[q] = 0.f; }
+        if (!vec && q >= cnt) { a[q] = 0.f; zn[q] = 0.f; w.z1[q] = 0.f; }
+        const float din = zn[q] - w.z1[q];
+        p_in = fmaf(din, din, p_in);
         const float diff = a[q] - fmaxf(zn[q], 0.f);
         p_res = fmaf(diff, diff, p_res);
         p_z = fmaf(zn[q], zn[q], p_z);
@@ -371,6 +373,7 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
       s_res += (double)p_res;
       s_z += (double)p_z;
       s_a += (double)p_a;
+      s_in += (double)p_in;
       if (vec) {
         *reinterpret_cast<float4*>(Zp + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
         if (HAS_U) *reinterpret_cast<float4*>(Up + e) = make_float4(w.u[0], w.u[1], w.u[2], w.u[3]);
@@ -420,10 +423,12 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
   const double r0 = block_sum<double>(s_res, sm);
   const double r1 = block_sum<double>(s_z, sm);
   const double r2 = block_sum<double>(s_a, sm);
+  const double r3 = block_sum<double>(s_in, sm);
   if (threadIdx.x == 0) {
-    g.partial[bid * 3 + 0] = r0;
-    g.partial[bid * 3 + 1] = r1;
-    g.partial[bid * 3 + 2] = r2;
+    g.partial[bid * 4 + 0] = r0;
+    g.partial[bid * 4 + 1] = r1;
+    g.partial[bid * 4 + 2] = r2;
+    g.partial[bid * 4 + 3] = r3;
   }
 }
 
@@ -465,24 +470,45 @@ __global__ void reduce_col_partials_kernel(const double* part, int32_t row_block
   }
 }
 
-__global__ void reduce_report_kernel(const double* partial, int nblocks, sp_step_report* rep, int acc) {
+__global__ void reduce_report_kernel(const double* partial, int nblocks, sp_step_report* rep, int acc, double alpha) {
   __shared__ double sm[32];
-  double s[3] = {0.0, 0.0, 0.0};
+  double s[4] = {0.0, 0.0, 0.0, 0.0};
   for (int i = threadIdx.x; i < nblocks; i += blockDim.x)
-    for (int f = 0; f < 3; ++f) s[f] += partial[(int64_t)i * 3 + f];
-  for (int f = 0; f < 3; ++f) {
+    for (int f = 0; f < 4; ++f) s[f] += partial[(int64_t)i * 4 + f];
+  for (int f = 0; f < 4; ++f) {
     const double r = block_sum<double>(s[f], sm);
     if (threadIdx.x == 0) {
-      double* dst = f == 0 ? &rep->res_act : (f == 1 ? &rep->z_sq : &rep->a_sq);
-      *dst = (acc ? *dst : 0.0) + r;
+      double* dst = f == 0 ? &rep->res_act : (f == 1 ? &rep->z_sq : (f == 2 ? &rep->a_sq : &rep->res_in));
+      *dst = (acc ? *dst : 0.0) + (f == 3 ? alpha * r : r);
     }
   }
+}
+
+// out[0] (+)= scale * sum x^2 over a [rows, cols] fp32 matrix: block partials, then one block adds them in order
+__global__ void __launch_bounds__(256) sumsq_partial_kernel(const float* __restrict__ x, int64_t ld, int64_t rows,
+                                                            int64_t cols, double* part) {
+  __shared__ double sm[32];
+  double s = 0.0;
+  const int64_t total = rows * cols;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const float v = x[(e / cols) * ld + (e % cols)];
+    s += (double)v * (double)v;
+  }
+  const double r = block_sum<double>(s, sm);
+  if (threadIdx.x == 0) part[blockIdx.x] = r;
+}
+__global__ void sumsq_finish_kernel(const double* part, int nblocks, double scale, double* out, int acc) {
+  __shared__ double sm[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < nblocks; i += blockDim.x) s += part[i];
+  const double r = block_sum<double>(s, sm);
+  if (threadIdx.x == 0) out[0] = (acc ? out[0] : 0.0) + scale * r;
 }
 
 __global__ void init_report_kernel(sp_step_report* rep, const double* rho1, const double* rho2, double kept) {
   rep->res_act = 0.0;
   rep->res_out = nan("");
-  rep->res_in = nan("");
+  rep->res_in = 0.0;
   rep->z_sq = 0.0;
   rep->a_sq = 0.0;
   rep->rho1_eff = rho1 ? rho1[0] : 0.0;
@@ -718,10 +744,21 @@ cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t 
   return cudaGetLastError();
 }
 
-cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate,
+cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* rep, bool accumulate, double alpha,
                           cudaStream_t stream) {
   count_launch();
-  reduce_report_kernel<<<1, 256, 0, stream>>>(partial, nblocks, rep, accumulate ? 1 : 0);
+  reduce_report_kernel<<<1, 256, 0, stream>>>(partial, nblocks, rep, accumulate ? 1 : 0, alpha);
+  return cudaGetLastError();
+}
+
+cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t cols, double scale, double* out,
+                             bool accumulate, double* scratch, cudaStream_t stream) {
+  if (rows * cols == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, (double)rows * cols * 4.0, stream);
+  const int nb = kSumsqBlocks;
+  count_launch(2);
+  sumsq_partial_kernel<<<nb, 256, 0, stream>>>(x, ld, rows, cols, scratch);
+  sumsq_finish_kernel<<<1, 256, 0, stream>>>(scratch, nb, scale, out, accumulate ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -366,6 +366,12 @@ def _step_and_compare(mod, X, W1_0, p_gpu, p_or, tol, audit):
     assert abs(rep_gpu["res_act"] - rep["res_act"]) <= 5 * tol * max(rep_gpu["a_sq"], 1e-30)
     assert abs(rep_gpu["a_sq"] - (A * A).sum()) <= 5 * tol * (A * A).sum()
     assert rep_gpu["kept"] == p_gpu.k_keep
+    # objective terms of Appendix A.1: alpha |Z - W1 X|^2 always, alpha |Ypre - W2 A|^2 on request
+    assert abs(rep_gpu["res_in"] - rep["res_in"]) <= 5 * tol * p_or.alpha * max(rep_gpu["z_sq"], 1e-30)
+    if p_gpu.compute_objective:
+        assert abs(rep_gpu["res_out"] - rep["res_out"]) <= 5 * tol * p_or.alpha * (Yo * Yo).sum()
+    else:
+        assert np.isnan(rep_gpu["res_out"])
 
 
 STEP_CASES = [
@@ -387,7 +393,7 @@ def test_admm_step_teacher_forced(cfg, chunk, kind, rule, dual, refit):
     mod.sp_ffn_init()
     k = cfg.k_keep
     p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=_RULE[rule], dual_mode=dual,
-                           score_kind=_KIND[kind], refit=refit, token_chunk=chunk)
+                           score_kind=_KIND[kind], refit=refit, token_chunk=chunk, compute_objective=True)
     p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=rule, dual_mode=dual, score_kind=kind,
                         refit=refit)
     audit = []
