@@ -312,9 +312,10 @@ def main():
         m2.check_status()
         h2d = hX.numel() * hX.element_size() + hW1.numel() * hW1.element_size() + hW2.numel() * hW2.element_size()
         d2h = oW1.numel() * 4 + oW2.numel() * 4 + omask.numel()
-        e2e = {"value": iters / (t1 - t0), "unit": UNIT, "h2d_bytes_per_step": h2d / iters,
+        e2e = {"value": iters / (t1 - t0), "unit": UNIT, "layers_per_s": 1.0 / (t1 - t0), "h2d_bytes_per_step": h2d / iters,
                "d2h_bytes_per_step": d2h / iters, "iterations": iters,
-               "note": "one module job: pinned-host X, W1_0, W2_0 in; init + iterations; W1, W2, mask back to host"}
+               "note": "one module job (= one pruned FFN layer): pinned-host X, W1_0, W2_0 in; init + iterations; W1, W2, "
+                       "mask back to host; layers_per_s is that whole job per second"}
 
     cpu = None
     if not args.no_cpu_baseline:
