@@ -5,7 +5,7 @@ A step = one pass of the whole hot path over one FFN module: sp_admm_step (weigh
 scores, top-k mask, recovery on the kept support, a-/z-(dual-)updates and Gram / cross-product accumulation over all
 calibration tokens) followed by sp_allocate_sparsity over the model's layer importances.
 
-Workload at N = 1 GPU: config C2 of the task (OPT-1.3B-shaped FFN module: d = 2048, n = 8192, 128 x 2048 = 262144
+Workload at N = 1 GPU: workload C2 (OPT-1.3B-shaped FFN module: d = 2048, n = 8192, 128 x 2048 = 262144
 calibration tokens in bf16, 50 % channel sparsity), synthetic seeded inputs generated on the device.
 With N > 1 GPUs every rank owns its own module (modules are independent once the kept counts are fixed), so the
 scaling is weak and the data path has no collective.

@@ -6,7 +6,7 @@ import torch
 
 from oracle import struprune_oracle as O
 
-# Tolerances stated by the task for values (weights, auxiliary variables, accumulators):
+# Tolerances for values (weights, auxiliary variables, accumulators):
 #   bf16 GEMM inputs with fp32 accumulation: 2e-3;  fp32 mode: 1e-5   (max |x - y| / max |y| per tensor).
 TOL = {torch.bfloat16: 2e-3, torch.float32: 1e-5}
 
