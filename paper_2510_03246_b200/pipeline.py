@@ -1,0 +1,89 @@
+"""Model-level flow of Algorithm 1 ("Importance-Guided Global Structured Pruning") over the FFN modules of a model,
+built from the library calls only (argument marshalling and loop control; all arithmetic runs in libsp).
+
+    Step 1  layer importances I_l        sp_ffn_init + sp_struct_scores on the pre-trained module
+    Step 2  softmax-form allocation      sp_allocate_sparsity  (r_l -> kept units per layer)
+    Step 3/4 per-module ADMM             sp_admm_step x K with the layer's kept count
+
+One module is resident at a time (the paper's memory argument), so a layer is initialised twice: once for its
+importance, once for its ADMM loop.  With several ranks each rank owns the layers `parallel.layers_of_rank` gives it;
+the only exchange is the vector of importances before Step 2.
+"""
+from __future__ import annotations
+
+import time
+from dataclasses import dataclass, field
+from typing import Callable
+
+import torch
+
+from . import api, parallel
+
+
+@dataclass
+class LayerResult:
+    layer: int
+    importance: float
+    k_keep: int
+    mask: torch.Tensor            # u8 [n]
+    W1: torch.Tensor              # fp32 [n, d]
+    W2: torch.Tensor              # fp32 [d, n]
+    reports: list = field(default_factory=list)
+
+
+def layer_importance(X, W1_0, W2_0, score_kind=api.SP_SCORE_WANDA_L2, token_chunk=0) -> float:
+    """I_l of one pre-trained FFN module: mean unit score of W2_0 against the pre-trained activation statistics."""
+    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=token_chunk)
+    mod.sp_ffn_init()
+    n = mod.n
+    if score_kind == api.SP_SCORE_WANDA_L2:
+        _, imp, _ = api.sp_struct_scores(score_kind, n, W=mod.W2_0, colsq=mod.G_A, colsq_stride=n + 1)
+    elif score_kind == api.SP_SCORE_WANDA_L1:
+        _, imp, _ = api.sp_struct_scores(score_kind, n, W=mod.W2_0, colabs=mod.absA, inv_tokens=1.0 / mod.N)
+    else:
+        raise ValueError("layer importance uses one of the Wanda score kinds")
+    mod.check_status()
+    return float(imp.item())
+
+
+def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_units: int, rbar: float, iters: int,
+                     params: api.AdmmParams | None = None, T_rel: float = 1.0, alloc_mode=api.SP_ALLOC_SOFTMAX,
+                     token_chunk: int = 0, device="cuda"):
+    """Runs Algorithm 1 over `n_layers` FFN modules.  layer_inputs(l) returns (X [N, d], W1_0 [n, d], W2_0 [d, n]) on the
+    device for layer l.  Returns (results of the layers this rank owns, r per layer, kept counts per layer, timings)."""
+    rank, _, world = parallel.env_world()
+    mine = parallel.layers_of_rank(n_layers, rank, world)
+    p = params or api.AdmmParams()
+    t0 = time.perf_counter()
+    # Step 1
+    local = {}
+    for l in mine:
+        X, W1_0, W2_0 = layer_inputs(l)
+        local[l] = layer_importance(X, W1_0, W2_0, p.score_kind, token_chunk)
+    I_all = parallel.gather_importances(local, n_layers, device=device)
+    # Step 2 (the temperature is given relative to the magnitude of the importances)
+    T = T_rel * float(I_all.abs().mean())
+    nu = torch.full((n_layers,), n_units, dtype=torch.int64, device=device)
+    r, k_keep = api.sp_allocate_sparsity(I_all.to(device), nu, rbar, T, alloc_mode)
+    k_host = k_keep.cpu().tolist()
+    t1 = time.perf_counter()
+    # Steps 3 and 4
+    results = []
+    for l in mine:
+        X, W1_0, W2_0 = layer_inputs(l)
+        k = max(1, int(k_host[l]))
+        mod = api.FfnModule(X, W1_0, W2_0, dual_mode=p.dual_mode, token_chunk=token_chunk, overlap_k=k)
+        mod.sp_ffn_init()
+        pl = api.AdmmParams(**{**p.__dict__, "k_keep": k, "token_chunk": token_chunk})
+        res = LayerResult(l, float(I_all[l].item()), k, None, None, None)
+        for _ in range(iters):
+            mod.sp_admm_step(pl)
+            res.reports.append(mod.report.clone())
+        mod.check_status()
+        res.mask, res.W1, res.W2 = mod.mask.clone(), mod.W1.clone(), mod.W2.clone()
+        res.reports = [dict(zip(api.REPORT_FIELDS, t.cpu().tolist())) for t in res.reports]
+        results.append(res)
+        del mod
+    torch.cuda.synchronize()
+    t2 = time.perf_counter()
+    return results, r, k_keep, {"importance_s": t1 - t0, "admm_s": t2 - t1, "layers_per_s": len(mine) / max(t2 - t0, 1e-9)}

@@ -1,0 +1,49 @@
+"""Algorithm 1 end to end on a tiny three-layer model: importances, softmax-form allocation, per-layer ADMM loops, all
+through the C ABI, checked against the oracle step by step (the oracle is fed the GPU's importances for the
+allocation, and each layer's first iteration is compared like the single-module tests)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import struprune_oracle as O
+from paper_2510_03246_b200 import api, pipeline, synth
+from tests._util import TOL, np64, relerr
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+CFG = synth.scaled(synth.CONFIGS["C1"], layers=3, d=96, n=328, tokens=600)
+
+
+def _inputs(layer):
+    X = synth.make_activations(CFG, layer)
+    W1, W2 = synth.make_weights(CFG, layer)
+    # make the layers differ in scale so that the allocation is not uniform
+    return X.to(DEV), (W1 * (1.0 + 0.5 * layer)).to(DEV), (W2 * (1.0 + 0.25 * layer)).to(DEV)
+
+
+def test_algorithm1_three_layers():
+    rbar, iters = 0.5, 2
+    p = api.AdmmParams(rho=CFG.rho)
+    results, r, k_keep, timing = pipeline.prune_ffn_layers(_inputs, CFG.layers, CFG.n, rbar, iters, params=p)
+    assert len(results) == CFG.layers and timing["layers_per_s"] > 0
+    # Step 1: layer importances against the oracle on the same inputs
+    I_gpu = np.array([res.importance for res in results])
+    for l, res in enumerate(results):
+        X, W1, W2 = _inputs(l)
+        st, _ = O.ffn_init(np64(X).T, np64(W1), np64(W2))
+        _, I_or = O.wanda_scores(np64(W2), colsq=np.diag(st.G_A), kind="l2")
+        assert abs(res.importance - I_or) < TOL[torch.float32] * abs(I_or) * 10
+    # Step 2: allocation from the GPU's importances, fp64 on both sides
+    T = float(np.abs(I_gpu).mean())
+    r_or, k_or = O.allocate_sparsity(I_gpu, [CFG.n] * CFG.layers, rbar, T)
+    assert np.abs(np64(r) - r_or).max() < 1e-12
+    assert np.array_equal(k_keep.cpu().numpy(), k_or)
+    assert abs(r_or.sum() - rbar * CFG.layers) < 1e-9          # nothing clipped: the budget holds with equality
+    assert len(set(k_or.tolist())) > 1                           # and the allocation is not uniform here
+    # Steps 3/4: every layer ends with exactly its kept count, pruned rows / columns zero, residuals reported
+    for l, res in enumerate(results):
+        m = res.mask.cpu().numpy()
+        assert int(m.sum()) == int(k_or[l]) == res.k_keep
+        assert np.all(np64(res.W1)[m == 0] == 0) and np.all(np64(res.W2)[:, m == 0] == 0)
+        assert len(res.reports) == iters and all(rep["kept"] == res.k_keep for rep in res.reports)
+        assert all(np.isfinite(rep["res_act"]) and rep["res_act"] >= 0 for rep in res.reports)
