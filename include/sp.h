@@ -231,6 +231,20 @@ sp_status sp_apply_mask(const float* scores, int64_t n_units, int64_t k_keep, in
                         size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
+ * sp_apply_mask_batched — the top-k selection of Algorithm 1 Step 3 for all L layers of a model in one launch.
+ * Layer l has its own score vector scores + l * ld_scores (n_units each) and its own kept count k_keep[l], read on the
+ * DEVICE (the integer counts sp_allocate_sparsity wrote can be passed on without a host round trip); counts outside
+ * [0, n_units] are clamped.  Same selection rule as sp_apply_mask.  Outputs per layer: mask_out + l * ld_mask (u8
+ * [n_units]); tau_out[l] (optional); kept_idx_out + l * ld_idx (optional, int32, the first k_keep[l] entries are
+ * written).  No weights are touched.  All pointers are device pointers.
+ * Errors: SP_ERR_INVALID_ARG (null scores / k_keep / mask_out), SP_ERR_SHAPE (negative sizes, a leading dimension
+ * smaller than n_units).
+ */
+sp_status sp_apply_mask_batched(const float* scores, int64_t ld_scores, int64_t n_units, int32_t L,
+                                const int64_t* k_keep, uint8_t* mask_out, int64_t ld_mask, float* tau_out,
+                                int32_t* kept_idx_out, int64_t ld_idx, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
  * Helpers.
  * sp_ridge_solve   — W[m,n] = R[m,n] (G[n,n] + rho_eff I)^-1 by Cholesky and two triangular solves (weight
  *                    recovery of Appendix A.1).  G, R, W fp32; factorisation in fp64 when precise != 0, else fp32.

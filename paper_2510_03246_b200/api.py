@@ -25,7 +25,7 @@ SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
  SP_WS_RIDGE_SOLVE) = range(8)
 
 EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
-           "sp_apply_mask", "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
+           "sp_apply_mask", "sp_apply_mask_batched", "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
            "sp_profile_kind_name", "sp_launch_count"]
 
@@ -93,6 +93,7 @@ def lib() -> C.CDLL:
         L.sp_struct_scores_static.argtypes = [i32, i32, C.POINTER(SpScoreInputs), i64, vp, vp, vp]
         L.sp_allocate_sparsity.argtypes = [vp, vp, i32, dbl, dbl, i32, dbl, vp, vp, vp]
         L.sp_apply_mask.argtypes = [vp, i64, i64, i32, vp, vp, vp, pm, pm, vp, sz, vp]
+        L.sp_apply_mask_batched.argtypes = [vp, i64, i64, i32, vp, vp, i64, vp, vp, i64, vp]
         L.sp_ridge_solve.argtypes = [vp, i64, vp, i64, i64, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
         L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, vp, i64, vp, vp, sz, vp]
         L.sp_gemm.argtypes = [i32, i32, i64, i64, i64, dbl, pm, pm, dbl, pm, i32, i32, vp, vp]
@@ -294,6 +295,23 @@ def sp_apply_mask(scores, k_keep, group=1, W_rows=None, W_cols=None, want_index=
                                C.byref(wr) if wr is not None else None, C.byref(wc) if wc is not None else None,
                                None, 0, _stream()), "sp_apply_mask")
     return mask, tau, (idx[:int(k_keep)] if idx is not None else None)
+
+
+def sp_apply_mask_batched(scores, k_keep, want_index=False):
+    """Top-k selection of all layers in one launch.  scores fp32 [L, n_units]; k_keep int64 [L] on the device.
+    Returns (mask u8 [L, n_units], tau fp32 [L], kept_idx int32 [L, n_units] or None; row l holds k_keep[l] entries)."""
+    _require_cuda(scores, k_keep)
+    if scores.dim() != 2 or scores.dtype != torch.float32 or scores.stride(1) != 1:
+        raise ValueError("scores must be fp32 [L, n_units] with unit inner stride")
+    if k_keep.dtype != torch.int64 or k_keep.numel() != scores.shape[0] or not k_keep.is_contiguous():
+        raise ValueError("k_keep must be contiguous int64 [L]")
+    L, n = scores.shape
+    mask = torch.empty(L, n, dtype=torch.uint8, device=scores.device)
+    tau = torch.empty(L, dtype=torch.float32, device=scores.device)
+    idx = torch.full((L, n), -1, dtype=torch.int32, device=scores.device) if want_index else None
+    _check(lib().sp_apply_mask_batched(scores.data_ptr(), scores.stride(0), n, L, k_keep.data_ptr(), mask.data_ptr(), n,
+                                       tau.data_ptr(), _ptr(idx), n, _stream()), "sp_apply_mask_batched")
+    return mask, tau, idx
 
 
 # ---------------------------------------------------------------------------------------------- module driver

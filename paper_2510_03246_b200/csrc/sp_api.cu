@@ -269,7 +269,7 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.Eo = c.take<float>((size_t)p.chunk * d);
   p.W2fb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
   p.absA_part = c.take<double>((size_t)p.row_blocks * n);
-  p.score_scratch = c.take<double>((size_t)score_row_blocks(d, n) * n * 2 + 16);
+  p.score_scratch = c.take<double>(std::max((size_t)score_row_blocks(d, n) * n * 2 + 16, wanda_scratch_doubles(d, n)));
   p.bytes = align_up(c.off, 256);
   p.z1_all = ws ? reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(ws) + p.bytes) : nullptr;   // optional tail
   return p;
@@ -348,7 +348,8 @@ size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t t
       // d = number of columns (n_units * group), N = tokens (LEMMA1) or weight rows (WANDA)
       const int64_t cols = d > 0 ? d : 1;
       const int rb = score_row_blocks(N > 0 ? N : 1, cols);
-      return align_up(((size_t)rb * cols * 2 + (size_t)cols * 2 + 16) * sizeof(double), 256) + 256;
+      const size_t lemma = (size_t)rb * cols * 2 + (size_t)cols * 4 + 16;
+      return align_up(std::max(lemma, wanda_scratch_doubles(N > 0 ? N : 1, cols)) * sizeof(double), 256) + 256;
     }
     case SP_WS_APPLY_MASK: return 256;
     case SP_WS_LINEAR_REFIT: return ridge_ws_bytes(d, n, dtype == SP_F64) + align_up((size_t)(n > 0 ? n : 1) * 4, 256) + 512;
@@ -533,6 +534,18 @@ sp_status sp_apply_mask(const float* scores, int64_t n_units, int64_t k_keep, in
                  W_rows ? W_rows->rows : 0, W_rows ? W_rows->cols : 0, W_rows ? W_rows->ld : 0,
                  W_cols ? reinterpret_cast<float*>(W_cols->ptr) : nullptr, W_cols ? W_cols->rows : 0,
                  W_cols ? W_cols->cols : 0, W_cols ? W_cols->ld : 0, s));
+  return SP_OK;
+}
+
+sp_status sp_apply_mask_batched(const float* scores, int64_t ld_scores, int64_t n_units, int32_t L,
+                                const int64_t* k_keep, uint8_t* mask_out, int64_t ld_mask, float* tau_out,
+                                int32_t* kept_idx_out, int64_t ld_idx, void* stream) {
+  if (!scores || !k_keep || !mask_out) return SP_ERR_INVALID_ARG;
+  if (n_units < 0 || n_units > 0x7fffffff || L < 0) return SP_ERR_SHAPE;
+  if (ld_scores < n_units || ld_mask < n_units || (kept_idx_out && ld_idx < n_units)) return SP_ERR_SHAPE;
+  if (n_units == 0 || L == 0) return SP_OK;
+  CU(topk_select_batched(scores, ld_scores, n_units, L, 0, k_keep, mask_out, ld_mask, tau_out, kept_idx_out, ld_idx,
+                         reinterpret_cast<cudaStream_t>(stream)));
   return SP_OK;
 }
 

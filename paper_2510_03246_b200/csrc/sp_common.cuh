@@ -130,6 +130,7 @@ cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64
                               cudaStream_t stream);
 int column_stats_row_blocks(int64_t T, int64_t C);
 int score_row_blocks(int64_t rows, int64_t cols);
+size_t wanda_scratch_doubles(int64_t rows, int64_t cols);
 // dst[i,j] = (T) G[i*ld + j] (+ rho on the diagonal) for the lower triangle; rho read from device (rho_dev[0]).
 template <typename T>
 cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_dev, T* dst, int64_t ldd,
@@ -211,6 +212,10 @@ cudaError_t allocate_sparsity(const double* I, const int64_t* n_units, int L, do
 cudaError_t topk_select(const float* scores, int64_t n, int64_t k, uint8_t* mask, float* tau, int32_t* kept_idx,
                         cudaStream_t stream);
 // kept_idx from an existing mask (ascending), count must equal k
+// `batch` independent problems in one launch (one block each); k_list (device, may be nullptr) overrides k_all.
+cudaError_t topk_select_batched(const float* scores, int64_t ld_scores, int64_t n, int64_t batch, int64_t k_all,
+                                const int64_t* k_list, uint8_t* mask, int64_t ld_mask, float* tau, int32_t* kept_idx,
+                                int64_t ld_idx, cudaStream_t stream);
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream);
 cudaError_t zero_pruned(const uint8_t* mask, int group, float* W_rows, int64_t r_rows, int64_t r_cols, int64_t r_ld,
                         float* W_cols, int64_t c_rows, int64_t c_cols, int64_t c_ld, cudaStream_t stream);

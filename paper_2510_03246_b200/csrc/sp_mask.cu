@@ -53,43 +53,160 @@ __device__ double block_max_bcast(double v, double* smem) {
 }
 
 // ------------------------------------------------------------------------------------------------ Wanda scores
-// partial column sums of W^2 (kind 0) or |W| (kind 1): grid (col blocks, row blocks) -> part[rb, cols]
-__global__ void weight_col_partials_kernel(const float* __restrict__ W, int64_t rows, int64_t cols, int64_t ldw,
-                                           int kind, int row_blocks, double* part) {
-  const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
+// s_u = sqrt(sum_{j in unit u} |W[:, j]|_2^2 * colsq[j])  (L2 form)  or  sum_j |W[:, j]|_1 * colabs[j] / tokens  (L1 form),
+// and the layer importance mean_u s_u, in ONE launch that reads W once.
+//   grid (column groups of 128, row blocks); a lane owns 4 adjacent columns (one 16-byte load per row), the 8 warps of a
+//   block take every 8th row of the block's row range, 8 rows of loads in flight per thread.
+//   stage 1: every block writes its 128 partial column sums (fp64, fixed order) to part[row block][col];
+//   stage 2: the block that arrives last at its column group's ticket adds the row blocks' partials in order; when
+//            units do not straddle column groups (128 % group == 0) it writes their scores and the sum of them,
+//            else the finished per-column values;
+//   stage 3: the block that arrives last at the final ticket adds the groups' sums (or first turns column values
+//            into unit scores) and writes the mean.
+// Which block is last varies; what it adds, and in which order, does not: the result is deterministic.
+// tickets[0 .. gridDim.x] must be zero at launch; each is set back to zero by the block that consumed it.
+constexpr int kWsCols = 128, kWsWarps = 8, kWsUnroll = 8;
+
+__global__ void __launch_bounds__(kWsWarps * 32) wanda_scores_kernel(
+    const float* __restrict__ W, int64_t rows, int64_t cols, int64_t ldw, int vec_ok, int kind, int group,
+    const float* __restrict__ colsq, int64_t colsq_stride, const double* __restrict__ colabs, double inv_tokens,
+    int64_t n_units, float* scores, double* importance, double* part, double* colval, unsigned int* tickets) {
+  __shared__ double red[kWsWarps][kWsCols];
+  __shared__ double sm[33];
+  __shared__ int s_last;
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int row_blocks = (int)gridDim.y;
+  const int64_t c0 = (int64_t)blockIdx.x * kWsCols + 4 * lane;
   const int64_t rows_per = ceil_div(rows, (int64_t)row_blocks);
   const int64_t r0 = (int64_t)blockIdx.y * rows_per;
   const int64_t r1 = (r0 + rows_per < rows) ? r0 + rows_per : rows;
-  double s = 0.0;
-  for (int64_t r = r0; r < r1; ++r) {
-    const double v = (double)W[r * ldw + c];
-    s += kind == 0 ? v * v : fabs(v);
-  }
-  part[(int64_t)blockIdx.y * cols + c] = s;
-}
-
-__global__ void __launch_bounds__(1024) wanda_finish_kernel(const double* part, int row_blocks, int64_t cols,
-                                                            int kind, int group, const float* colsq,
-                                                            int64_t colsq_stride, const double* colabs,
-                                                            double inv_tokens, int64_t n_units, float* scores,
-                                                            double* importance) {
-  __shared__ double sm[33];
-  double acc = 0.0;
-  for (int64_t u = threadIdx.x; u < n_units; u += blockDim.x) {
-    double s = 0.0;
-    for (int g = 0; g < group; ++g) {
-      const int64_t j = u * group + g;
-      double w = 0.0;
-      for (int r = 0; r < row_blocks; ++r) w += part[(int64_t)r * cols + j];
-      s += kind == 0 ? w * (double)colsq[j * colsq_stride] : w * colabs[j] * inv_tokens;
+  const bool full = vec_ok && c0 + 3 < cols;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int64_t rb = r0 + warp; rb < r1; rb += (int64_t)kWsWarps * kWsUnroll) {
+    float4 v[kWsUnroll];
+#pragma unroll
+    for (int q = 0; q < kWsUnroll; ++q) {
+      const int64_t r = rb + (int64_t)q * kWsWarps;
+      v[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < r1) {
+        const float* src = W + r * ldw + c0;
+        if (full) {
+          v[q] = *reinterpret_cast<const float4*>(src);
+        } else {
+          if (c0 < cols) v[q].x = src[0];
+          if (c0 + 1 < cols) v[q].y = src[1];
+          if (c0 + 2 < cols) v[q].z = src[2];
+          if (c0 + 3 < cols) v[q].w = src[3];
+        }
+      }
     }
-    const float sc = (float)(kind == 0 ? sqrt(s) : s);
-    scores[u] = sc;
-    acc += (double)sc;
+#pragma unroll
+    for (int q = 0; q < kWsUnroll; ++q) {
+      const double x = v[q].x, y = v[q].y, z = v[q].z, w = v[q].w;
+      if (kind == 0) {
+        acc[0] = fma(x, x, acc[0]); acc[1] = fma(y, y, acc[1]); acc[2] = fma(z, z, acc[2]); acc[3] = fma(w, w, acc[3]);
+      } else {
+        acc[0] += fabs(x); acc[1] += fabs(y); acc[2] += fabs(z); acc[3] += fabs(w);
+      }
+    }
   }
-  const double tot = block_sum_bcast(acc, sm);
-  if (threadIdx.x == 0 && importance) importance[0] = tot / (double)n_units;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) red[warp][4 * lane + j] = acc[j];
+  __syncthreads();
+  if (t < kWsCols) {
+    const int64_t c = (int64_t)blockIdx.x * kWsCols + t;
+    if (c < cols) {
+      double sum = 0.0;
+#pragma unroll
+      for (int w = 0; w < kWsWarps; ++w) sum += red[w][t];
+      part[(int64_t)blockIdx.y * cols + c] = sum;
+    }
+  }
+  // ---- stage 2: last block of this column group
+  __threadfence();
+  __syncthreads();
+  if (t == 0) s_last = atomicAdd(&tickets[blockIdx.x], 1u) == (unsigned)(row_blocks - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // units that lie inside one column group are finished here; otherwise stage 3 adds column values across groups
+  const bool direct = (kWsCols % group) == 0;
+  double* cv = &red[0][0];
+  if (t < kWsCols) {
+    const int64_t c = (int64_t)blockIdx.x * kWsCols + t;
+    double val = 0.0;
+    if (c < cols) {
+      double w = 0.0;
+      int r = 0;
+      for (; r + 8 <= row_blocks; r += 8) {          // independent loads, added in order
+        double pv[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) pv[q] = __ldcg(&part[(int64_t)(r + q) * cols + c]);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) w += pv[q];
+      }
+      for (; r < row_blocks; ++r) w += __ldcg(&part[(int64_t)r * cols + c]);
+      val = kind == 0 ? w * (double)colsq[c * colsq_stride] : w * colabs[c] * inv_tokens;
+      if (!direct) colval[c] = val;
+    }
+    cv[t] = val;
+  }
+  __syncthreads();
+  if (direct) {
+    const int upg = kWsCols / group;                  // units per column group
+    double mine = 0.0;
+    if (t < upg) {
+      const int64_t u = (int64_t)blockIdx.x * upg + t;
+      if (u < n_units) {
+        double sc = 0.0;
+        for (int g = 0; g < group; ++g) sc += cv[t * group + g];
+        const float f = (float)(kind == 0 ? sqrt(sc) : sc);
+        scores[u] = f;
+        mine = (double)f;
+      }
+    }
+    mine = block_sum_bcast(mine, sm);
+    if (t == 0) colval[blockIdx.x] = mine;            // sum of this group's scores
+  }
+  // ---- stage 3: last column group
+  __threadfence();
+  __syncthreads();
+  if (t == 0) {
+    tickets[blockIdx.x] = 0u;
+    s_last = atomicAdd(&tickets[gridDim.x], 1u) == gridDim.x - 1u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  double tot = 0.0;
+  if (direct) {
+    for (int64_t gq = t; gq < (int64_t)gridDim.x; gq += blockDim.x) tot += __ldcg(&colval[gq]);
+  } else {
+    for (int64_t u0 = 0; u0 < n_units; u0 += (int64_t)blockDim.x * 4) {
+      double sc[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int g = 0; g < group; ++g) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int64_t u = u0 + (int64_t)q * blockDim.x + t;
+          if (u < n_units) sc[q] += __ldcg(&colval[u * group + g]);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int64_t u = u0 + (int64_t)q * blockDim.x + t;
+        if (u < n_units) {
+          const float f = (float)(kind == 0 ? sqrt(sc[q]) : sc[q]);
+          scores[u] = f;
+          tot += (double)f;
+        }
+      }
+    }
+  }
+  tot = block_sum_bcast(tot, sm);
+  if (t == 0) {
+    if (importance) importance[0] = tot / (double)n_units;
+    tickets[gridDim.x] = 0u;
+  }
 }
 
 // ------------------------------------------------------------------------------------------------ Lemma 1
@@ -111,6 +228,114 @@ __global__ void lemma1_partials_kernel(sp_mat b, sp_mat c, sp_mat dd, sp_mat t, 
   }
   part[((int64_t)blockIdx.y * cols + j) * 2 + 0] = num;
   part[((int64_t)blockIdx.y * cols + j) * 2 + 1] = den;
+}
+
+// Vector form of the kernel above for four tensors of one dtype with 16-byte aligned rows: a lane owns V = 16 / sizeof(T)
+// adjacent columns (one 16-byte load per tensor and row), the 8 warps of a block take every 8th row of the block's
+// range, two rows (8 loads) in flight per thread.  grid (column groups of 32 V, row blocks).
+template <typename T>
+struct L1Vec;
+template <>
+struct L1Vec<float> {
+  static constexpr int V = 4;
+  typedef float4 Raw;
+  __device__ static Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+  __device__ static float get(const Raw& v, int j) { return j == 0 ? v.x : j == 1 ? v.y : j == 2 ? v.z : v.w; }
+};
+template <>
+struct L1Vec<__nv_bfloat16> {
+  static constexpr int V = 8;
+  typedef uint4 Raw;
+  __device__ static Raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
+  __device__ static float get(const Raw& v, int j) {
+    const uint32_t w = (j >> 1) == 0 ? v.x : (j >> 1) == 1 ? v.y : (j >> 1) == 2 ? v.z : v.w;
+    return __uint_as_float((j & 1) ? (w & 0xffff0000u) : (w << 16));
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256, 2) lemma1_partials_vec_kernel(const T* __restrict__ b, const T* __restrict__ c,
+                                                                     const T* __restrict__ dd,
+                                                                     const T* __restrict__ tt, int64_t ldb,
+                                                                     int64_t ldc, int64_t ldd, int64_t ldt, int64_t N,
+                                                                     int64_t cols, double* part) {
+  typedef typename L1Vec<T>::Raw Raw;
+  constexpr int V = L1Vec<T>::V, CB = 32 * V;
+  __shared__ double red[8][CB + 1];
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int row_blocks = (int)gridDim.y;
+  const int64_t c0 = (int64_t)blockIdx.x * CB + (int64_t)V * lane;    // cols % V == 0: a lane is all in or all out
+  const int64_t rows_per = ceil_div(N, (int64_t)row_blocks);
+  const int64_t r0 = (int64_t)blockIdx.y * rows_per;
+  const int64_t r1 = (r0 + rows_per < N) ? r0 + rows_per : N;
+  double num[V], den[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) num[j] = den[j] = 0.0;
+  if (c0 < cols) {
+    for (int64_t rb = r0 + warp; rb < r1; rb += 16) {
+      Raw raw[2][4];    // the packed loads of two rows stay in flight; values are unpacked one column at a time
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int64_t r = rb + 8 * q;
+        if (r < r1) {
+          raw[q][0] = *reinterpret_cast<const Raw*>(b + r * ldb + c0);
+          raw[q][1] = *reinterpret_cast<const Raw*>(c + r * ldc + c0);
+          raw[q][2] = *reinterpret_cast<const Raw*>(dd + r * ldd + c0);
+          raw[q][3] = *reinterpret_cast<const Raw*>(tt + r * ldt + c0);
+        } else {
+          raw[q][0] = raw[q][1] = raw[q][2] = raw[q][3] = L1Vec<T>::zero();
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 2; ++q)
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+          const double xb = L1Vec<T>::get(raw[q][0], j), xc = L1Vec<T>::get(raw[q][1], j);
+          const double xd = L1Vec<T>::get(raw[q][2], j), xt = L1Vec<T>::get(raw[q][3], j);
+          num[j] += xc * xb + xd * xt;
+          den[j] += xc * xc + xd * xd;
+        }
+    }
+  }
+  // cross-warp sums in a fixed order, numerators then denominators
+  for (int pass = 0; pass < 2; ++pass) {
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < V; ++j) red[warp][V * lane + j] = pass == 0 ? num[j] : den[j];
+    __syncthreads();
+    for (int cc = t; cc < CB; cc += 256) {
+      const int64_t col = (int64_t)blockIdx.x * CB + cc;
+      if (col < cols) {
+        double sum = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) sum += red[w][cc];
+        part[((int64_t)blockIdx.y * cols + col) * 2 + pass] = sum;
+      }
+    }
+  }
+}
+
+// colred[j] = (sum over row blocks of the numerators, of the denominators) of column j
+__global__ void __launch_bounds__(256) lemma1_colred_kernel(const double* __restrict__ part, int row_blocks,
+                                                            int64_t cols, double* colred) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= cols) return;
+  const double2* p2 = reinterpret_cast<const double2*>(part);
+  double num = 0.0, den = 0.0;
+  int r = 0;
+  for (; r + 8 <= row_blocks; r += 8) {
+    double2 v[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = p2[(int64_t)(r + q) * cols + j];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) { num += v[q].x; den += v[q].y; }
+  }
+  for (; r < row_blocks; ++r) {
+    const double2 v = p2[(int64_t)r * cols + j];
+    num += v.x;
+    den += v.y;
+  }
+  reinterpret_cast<double2*>(colred)[j] = make_double2(num, den);
 }
 
 __global__ void __launch_bounds__(1024) lemma1_finish_kernel(const double* part, int row_blocks, int64_t cols,
@@ -255,13 +480,59 @@ __device__ int block_excl_scan(int flag, int* warp_tot, int* total) {
   return before + within;
 }
 
-__global__ void __launch_bounds__(1024) topk_select_kernel(const float* __restrict__ scores, int64_t n, int64_t k,
-                                                           uint8_t* mask, float* tau, int32_t* kept_idx) {
+// exclusive scan of a pair of counts over the block (1024 threads max, every thread calls it);
+// returns the exclusive prefixes, the block totals through *total
+__device__ int2 block_excl_scan2(int a, int b, int2* warp_tot, int2* total) {
+  const int l = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int ia = a, ib = b;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int va = __shfl_up_sync(0xffffffffu, ia, o), vb = __shfl_up_sync(0xffffffffu, ib, o);
+    if (l >= o) { ia += va; ib += vb; }
+  }
+  __syncthreads();
+  if (l == 31) warp_tot[w] = make_int2(ia, ib);
+  __syncthreads();
+  if (w == 0) {
+    const int nw = (blockDim.x + 31) >> 5;
+    int2 v = l < nw ? warp_tot[l] : make_int2(0, 0);
+    int sa = v.x, sb = v.y;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int va = __shfl_up_sync(0xffffffffu, sa, o), vb = __shfl_up_sync(0xffffffffu, sb, o);
+      if (l >= o) { sa += va; sb += vb; }
+    }
+    warp_tot[l] = make_int2(sa - v.x, sb - v.y);          // exclusive over warps
+    if (l == 31) warp_tot[32] = make_int2(sa, sb);        // totals
+  }
+  __syncthreads();
+  const int2 base = warp_tot[w];
+  *total = warp_tot[32];
+  return make_int2(base.x + ia - a, base.y + ib - b);
+}
+
+// Exact top-k of one score vector per block (blockIdx.x = problem of a batch): the k largest scores are kept, among
+// equal scores the lower index first (radix select on order-preserving keys, 8 bits per pass from the top).
+//   scores + b * ld_scores, mask + b * ld_mask, kept_idx + b * ld_idx, tau + b;  k = k_list ? k_list[b] : k_all.
+// The keys are staged once in shared memory when they fit (smem_keys != 0), else re-read from global memory.
+__global__ void __launch_bounds__(1024) topk_select_kernel(const float* __restrict__ scores_all, int64_t ld_scores,
+                                                           int64_t n, int64_t k_all, const int64_t* k_list,
+                                                           uint8_t* mask_all, int64_t ld_mask, float* tau_all,
+                                                           int32_t* kept_all, int64_t ld_idx, int smem_keys) {
+  extern __shared__ uint32_t s_keys[];
+  __shared__ int hist_w[32][256];     // one histogram per warp: adds collide only inside a warp
   __shared__ int hist[256];
-  __shared__ int warp_tot[32];
+  __shared__ int2 warp_tot[33];
   __shared__ uint32_t s_prefix;
   __shared__ int64_t s_krem;
-  const int t = threadIdx.x;
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int64_t prob = blockIdx.x;
+  const float* scores = scores_all + prob * ld_scores;
+  uint8_t* mask = mask_all + prob * ld_mask;
+  float* tau = tau_all ? tau_all + prob : nullptr;
+  int32_t* kept_idx = kept_all ? kept_all + prob * ld_idx : nullptr;
+  int64_t k = k_list ? k_list[prob] : k_all;
+  if (k < 0) k = 0;
   if (k <= 0 || k >= n) {
     for (int64_t i = t; i < n; i += blockDim.x) {
       mask[i] = k >= n ? 1 : 0;
@@ -273,60 +544,103 @@ __global__ void __launch_bounds__(1024) topk_select_kernel(const float* __restri
         uint32_t best = 0xffffffffu;
         for (int64_t i = 0; i < n; ++i) best = min(best, score_key(scores[i]));
         for (int64_t i = 0; i < n; ++i)
-          if (score_key(scores[i]) == best) { m = scores[i]; break; }
+          if (score_key(scores[i]) == best) { m = scores[i] != scores[i] ? -INFINITY : scores[i]; break; }
       }
       tau[0] = m;
     }
     return;
   }
+  if (smem_keys) {
+    for (int64_t base = 0; base < n; base += (int64_t)blockDim.x * 4) {   // four loads in flight per thread
+      float v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int64_t i = base + (int64_t)q * blockDim.x + t;
+        v[q] = i < n ? scores[i] : 0.f;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int64_t i = base + (int64_t)q * blockDim.x + t;
+        if (i < n) s_keys[i] = score_key(v[q]);
+      }
+    }
+  }
   if (t == 0) { s_prefix = 0u; s_krem = k; }
   __syncthreads();
-  // find the key of the k-th largest score, 8 bits per pass from the top
+  auto key_at = [&](int64_t i) -> uint32_t { return smem_keys ? s_keys[i] : score_key(scores[i]); };
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-    for (int i = t; i < 256; i += blockDim.x) hist[i] = 0;
+    for (int i = t; i < 32 * 256; i += blockDim.x) (&hist_w[0][0])[i] = 0;
     __syncthreads();
     const uint32_t prefix = s_prefix;
     for (int64_t i = t; i < n; i += blockDim.x) {
-      const uint32_t key = score_key(scores[i]);
-      if ((key & hi_mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xffu], 1);
+      const uint32_t key = key_at(i);
+      if ((key & hi_mask) == prefix) atomicAdd(&hist_w[warp][(key >> shift) & 0xffu], 1);
     }
     __syncthreads();
-    if (t == 0) {
-      int64_t rem = s_krem;
-      int bin = 255;
-      for (; bin > 0; --bin) {
-        if (hist[bin] >= rem) break;
-        rem -= hist[bin];
+    if (t < 256) {
+      int sum = 0;
+#pragma unroll 8
+      for (int w = 0; w < 32; ++w) sum += hist_w[w][t];
+      hist[t] = sum;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane l owns bins 255 - 8 l down to 248 - 8 l: walk from the largest digit down
+      int c[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c[j] = hist[255 - (8 * lane + j)]; tot += c[j]; }
+      int incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
       }
-      s_krem = rem;  // how many to take from this bin
-      s_prefix = prefix | ((uint32_t)bin << shift);
+      const int64_t rem = s_krem, excl = incl - tot;
+      __syncwarp();
+      if (excl < rem && rem <= (int64_t)incl) {
+        int64_t r = rem - excl;
+        int bin = 255 - 8 * lane;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if ((int64_t)c[j] >= r) { bin = 255 - (8 * lane + j); break; }
+          r -= c[j];
+        }
+        s_krem = r;   // how many to take from this bin
+        s_prefix = prefix | ((uint32_t)bin << shift);
+      }
     }
     __syncthreads();
   }
   const uint32_t tkey = s_prefix;
   const int64_t take_eq = s_krem;  // ties at the threshold that are kept (lowest indices first)
-  int64_t eq_before = 0, kept_before = 0;
-  bool tau_written = false;
-  for (int64_t base = 0; base < n; base += blockDim.x) {
-    const int64_t i = base + t;
-    uint32_t key = 0;
-    const bool valid = i < n;
-    if (valid) key = score_key(scores[i]);
-    const int is_eq = valid && key == tkey;
-    int tot_eq, tot_keep;
-    const int eq_rank = block_excl_scan(is_eq, warp_tot, &tot_eq);
-    const int keep = valid && (key > tkey || (is_eq && eq_before + eq_rank < take_eq));
-    const int keep_rank = block_excl_scan(keep, warp_tot, &tot_keep);
-    if (valid) {
-      mask[i] = (uint8_t)keep;
-      if (keep && kept_idx) kept_idx[kept_before + keep_rank] = (int32_t)i;
-      if (is_eq && !tau_written && tau && eq_before + eq_rank == 0) tau[0] = scores[i] != scores[i] ? -INFINITY : scores[i];
+  // thread t owns the contiguous indices [t * per, (t + 1) * per): one scan orders the whole vector
+  const int64_t per = ceil_div(n, (int64_t)blockDim.x);
+  const int64_t i0 = (int64_t)t * per, i1 = (i0 + per < n) ? i0 + per : n;
+  int n_eq = 0, n_gt = 0;
+  for (int64_t i = i0; i < i1; ++i) {
+    const uint32_t key = key_at(i);
+    n_eq += key == tkey;
+    n_gt += key > tkey;
+  }
+  int2 total;
+  const int2 before = block_excl_scan2(n_eq, n_gt, warp_tot, &total);
+  int64_t eq_seen = before.x, gt_seen = before.y;
+  for (int64_t i = i0; i < i1; ++i) {
+    const uint32_t key = key_at(i);
+    const bool is_eq = key == tkey;
+    const bool keep = key > tkey || (is_eq && eq_seen < take_eq);
+    mask[i] = (uint8_t)keep;
+    if (keep && kept_idx) kept_idx[gt_seen + (eq_seen < take_eq ? eq_seen : take_eq)] = (int32_t)i;
+    if (is_eq) {
+      if (eq_seen == 0 && tau) {
+        const float v = scores[i];
+        tau[0] = v != v ? -INFINITY : v;
+      }
+      ++eq_seen;
     }
-    eq_before += tot_eq;
-    kept_before += tot_keep;
-    if (eq_before > 0) tau_written = true;
+    gt_seen += key > tkey;
   }
 }
 
@@ -377,7 +691,7 @@ inline int grid_for(int64_t total, int threads) {
 
 inline int row_blocks_for(int64_t rows, int64_t cols) {
   const int64_t cb = ceil_div(cols, 256);
-  int64_t rb = ceil_div(148 * 4, cb);
+  int64_t rb = ceil_div(148 * 8, cb);
   if (rb > rows) rb = rows;
   if (rb < 1) rb = 1;
   return (int)rb;
@@ -387,20 +701,43 @@ inline int row_blocks_for(int64_t rows, int64_t cols) {
 
 int score_row_blocks(int64_t rows, int64_t cols) { return row_blocks_for(rows, cols); }
 
+// Launch shape of wanda_scores_kernel: column groups and row blocks (about 8 resident blocks on each of 148 SMs).
+static void wanda_grid(int64_t rows, int64_t cols, int64_t* col_groups, int64_t* row_blocks) {
+  const int64_t cg = ceil_div(cols, (int64_t)kWsCols);
+  int64_t rb = (148 * 8) / cg;
+  const int64_t rb_max = ceil_div(rows, (int64_t)kWsWarps);
+  if (rb > rb_max) rb = rb_max;
+  if (rb < 1) rb = 1;
+  *col_groups = cg;
+  *row_blocks = rb;
+}
+
+// doubles of scratch: part[row_blocks][cols], colval[cols], then the tickets (32-bit, col_groups + 1 of them)
+size_t wanda_scratch_doubles(int64_t rows, int64_t cols) {
+  int64_t cg, rb;
+  wanda_grid(rows, cols, &cg, &rb);
+  return (size_t)(rb + 1) * (size_t)cols + (size_t)(cg + 2) / 2 + 1;
+}
+
 cudaError_t wanda_scores(int kind, int group, const float* W, int64_t rows, int64_t ldw, const float* colsq,
                          int64_t colsq_stride, const double* colabs, double inv_tokens, int64_t n_units,
                          float* scores, double* importance, double* scratch, cudaStream_t stream) {
   const int64_t cols = n_units * group;
   if (cols == 0) return cudaSuccess;
-  const int rb = row_blocks_for(rows, cols);
+  int64_t cg, rb;
+  wanda_grid(rows, cols, &cg, &rb);
   const int k = kind == SP_SCORE_WANDA_L2 ? 0 : 1;
+  double* part = scratch;
+  double* colval = scratch + (size_t)rb * cols;
+  unsigned int* tickets = reinterpret_cast<unsigned int*>(colval + cols);
+  const int vec_ok = (ldw % 4 == 0) && ((reinterpret_cast<uintptr_t>(W) & 15u) == 0);
   ProfScope prof(PK_SCORES, 0.0, (double)rows * (double)cols * 4.0, stream);
+  cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)(cg + 1) * sizeof(unsigned int), stream);
+  if (e != cudaSuccess) return e;
   count_launch();
-  weight_col_partials_kernel<<<dim3((unsigned)ceil_div(cols, 256), (unsigned)rb), 256, 0, stream>>>(W, rows, cols, ldw,
-                                                                                                   k, rb, scratch);
-  count_launch();
-  wanda_finish_kernel<<<1, 1024, 0, stream>>>(scratch, rb, cols, k, group, colsq, colsq_stride, colabs, inv_tokens,
-                                              n_units, scores, importance);
+  wanda_scores_kernel<<<dim3((unsigned)cg, (unsigned)rb), kWsWarps * 32, 0, stream>>>(
+      W, rows, cols, ldw, vec_ok, k, group, colsq, colsq_stride, colabs, inv_tokens, n_units, scores, importance, part,
+      colval, tickets);
   return cudaGetLastError();
 }
 
@@ -411,12 +748,44 @@ cudaError_t lemma1_scores_stream(const sp_mat& b, const sp_mat& c, const sp_mat&
   const int64_t N = b.rows;
   if (cols == 0) return cudaSuccess;
   const int rb = row_blocks_for(N, cols);
+  // scratch: part[rb][cols][2], colred[cols][2] (column sums over the row blocks), unit_e[cols][2] (finish kernel)
   double* part = scratch;
-  double* unit_e = scratch + (size_t)rb * cols * 2;
+  double* colred = scratch + (size_t)rb * cols * 2;
+  double* unit_e = colred + (size_t)cols * 2;
   ProfScope prof(PK_SCORES, 0.0, (double)N * (double)cols * (double)(dtype_size(b.dtype) + dtype_size(c.dtype) +
                                                                     dtype_size(dd.dtype) + dtype_size(t.dtype)),
                  stream);
+  const int32_t dt = b.dtype;
+  const int V = dt == SP_BF16 ? 8 : 4;
+  auto ok = [&](const sp_mat& m) {
+    return m.dtype == dt && m.ld % V == 0 && (reinterpret_cast<uintptr_t>(m.ptr) & 15u) == 0;
+  };
+  const bool vec = (dt == SP_BF16 || dt == SP_F32) && cols % V == 0 && ok(b) && ok(c) && ok(dd) && ok(t);
   count_launch();
+  if (vec) {
+    // about 148 * 8 blocks, never more row blocks than the scratch was sized for
+    const int64_t cg = ceil_div(cols, (int64_t)(32 * V));
+    int64_t rbv = (148 * 8) / cg;
+    if (rbv > rb) rbv = rb;
+    if (rbv < 1) rbv = 1;
+    const dim3 grid((unsigned)cg, (unsigned)rbv);
+    if (dt == SP_BF16)
+      lemma1_partials_vec_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
+          reinterpret_cast<const __nv_bfloat16*>(b.ptr), reinterpret_cast<const __nv_bfloat16*>(c.ptr),
+          reinterpret_cast<const __nv_bfloat16*>(dd.ptr), reinterpret_cast<const __nv_bfloat16*>(t.ptr), b.ld, c.ld,
+          dd.ld, t.ld, N, cols, part);
+    else
+      lemma1_partials_vec_kernel<float><<<grid, 256, 0, stream>>>(
+          reinterpret_cast<const float*>(b.ptr), reinterpret_cast<const float*>(c.ptr),
+          reinterpret_cast<const float*>(dd.ptr), reinterpret_cast<const float*>(t.ptr), b.ld, c.ld, dd.ld, t.ld, N,
+          cols, part);
+    count_launch();
+    lemma1_colred_kernel<<<(unsigned)ceil_div(cols, (int64_t)256), 256, 0, stream>>>(part, (int)rbv, cols, colred);
+    count_launch();
+    lemma1_finish_kernel<<<1, 1024, 0, stream>>>(colred, 1, cols, group, n_units, scores, importance, relaxed, r_layer,
+                                                 unit_e);
+    return cudaGetLastError();
+  }
   lemma1_partials_kernel<<<dim3((unsigned)ceil_div(cols, 256), (unsigned)rb), 256, 0, stream>>>(b, c, dd, t, N, cols,
                                                                                                rb, part);
   count_launch();
@@ -448,9 +817,26 @@ cudaError_t allocate_sparsity(const double* I, const int64_t* n_units, int L, do
 cudaError_t topk_select(const float* scores, int64_t n, int64_t k, uint8_t* mask, float* tau, int32_t* kept_idx,
                         cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
-  ProfScope prof(PK_TOPK, 0.0, (double)n * 5.0, stream);
+  return topk_select_batched(scores, n, n, 1, k, nullptr, mask, n, tau, kept_idx, n, stream);
+}
+
+cudaError_t topk_select_batched(const float* scores, int64_t ld_scores, int64_t n, int64_t batch, int64_t k_all,
+                                const int64_t* k_list, uint8_t* mask, int64_t ld_mask, float* tau, int32_t* kept_idx,
+                                int64_t ld_idx, cudaStream_t stream) {
+  if (n == 0 || batch == 0) return cudaSuccess;
+  constexpr int64_t kMaxSmemKeys = 47104;      // 184 KiB of keys beside the 33 KiB of histograms
+  static bool attr_set = false;
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)(kMaxSmemKeys * sizeof(uint32_t)));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int smem_keys = n <= kMaxSmemKeys ? 1 : 0;
+  ProfScope prof(PK_TOPK, 0.0, (double)batch * (double)n * 5.0, stream);
   count_launch();
-  topk_select_kernel<<<1, 1024, 0, stream>>>(scores, n, k, mask, tau, kept_idx);
+  topk_select_kernel<<<(unsigned)batch, 1024, smem_keys ? (size_t)n * sizeof(uint32_t) : 0, stream>>>(
+      scores, ld_scores, n, k_all, k_list, mask, ld_mask, tau, kept_idx, ld_idx, smem_keys);
   return cudaGetLastError();
 }
 
@@ -527,14 +913,14 @@ extern "C" sp_status sp_struct_scores_static(int32_t kind, int32_t group, const 
   if (in->W.cols != cols || in->W.ld < cols || in->W.rows < 1) return SP_ERR_SHAPE;
   if (kind == SP_SCORE_WANDA_L2 && (!in->colsq || in->colsq_stride < 1)) return SP_ERR_INVALID_ARG;
   if (kind == SP_SCORE_WANDA_L1 && !in->colabs) return SP_ERR_INVALID_ARG;
-  // the partial sums take row_blocks x cols doubles; row_blocks shrinks as cols grows, so the product stays bounded
-  if ((size_t)sp::score_row_blocks(in->W.rows, cols) * (size_t)cols > kStaticScratchDoubles)
-    return SP_ERR_STATIC_LIMIT;
+  // the partial sums take (row_blocks + 1) x cols doubles; row_blocks shrinks as cols grows, so the product stays
+  // bounded
+  if (sp::wanda_scratch_doubles(in->W.rows, cols) > kStaticScratchDoubles) return SP_ERR_STATIC_LIMIT;
   double* scratch = nullptr;
   const sp_status st = static_scratch_address(&scratch);
   if (st != SP_OK) return st;
-  // every partial sum that the finishing kernel reads is written by the first kernel of this same call, so nothing
-  // left behind by an earlier call is ever read and no clearing is needed
+  // every partial sum that is read was written earlier in this same call, so nothing an earlier call left behind
+  // is read; only the few arrival tickets are cleared (a memset on the stream, no allocation)
   if (sp::wanda_scores(kind, group, reinterpret_cast<const float*>(in->W.ptr), in->W.rows, in->W.ld, in->colsq,
                        in->colsq_stride, in->colabs, in->inv_tokens, n_units, scores, layer_importance, scratch,
                        reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)

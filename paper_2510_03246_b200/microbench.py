@@ -2,6 +2,8 @@
 
     python -m paper_2510_03246_b200.microbench gemm  [--reps 5 --warm 2]   GEMM shapes of one C2 token chunk
     python -m paper_2510_03246_b200.microbench solve [--reps 3 --warm 1]   regularised solves of a C2 step
+    python -m paper_2510_03246_b200.microbench mask  [--reps 5 --warm 2]   scores, allocation and top-k as standalone
+                                                                           kernels (L2 flushed before every call)
 
 Inputs are random (torch.randn on the device): these runs time kernels, they check nothing.
 """
@@ -79,16 +81,94 @@ def solve_cases(reps, warm):
     print("status", st.cpu().tolist())
 
 
+def _timeit_cold(fn, reps, warm, flush):
+    """Mean device time of fn() in ms with the L2 overwritten before every call.  The flush (a 1 GiB fill) also keeps
+    the stream busy long enough for the host to have queued fn() and the closing event before the GPU gets there."""
+    tot = 0.0
+    for it in range(warm + reps):
+        flush.fill_(it)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= warm:
+            tot += e0.elapsed_time(e1)
+    return tot / reps
+
+
+def mask_cases(reps, warm, hbm_gbs):
+    flush = torch.empty(1 << 30, dtype=torch.uint8, device=DEV)
+
+    def line(name, ms, nbytes):
+        gbs = nbytes / ms / 1e6
+        print(f"{name:58s} {1e3 * ms:9.1f} us  {nbytes / 1e6:9.2f} MB  {gbs:8.1f} GB/s  {gbs / hbm_gbs:5.2f} of HBM peak",
+              flush=True)
+
+    # Wanda scores: one pass over the fp32 weight matrix [d, n] (C2, C3 and C5 shapes), channel and head units
+    for d, n, group in ((2048, 8192, 1), (4096, 16384, 1), (7168, 28672, 1), (4096, 4096, 128)):
+        W = torch.randn(d, n, device=DEV)
+        colsq = torch.rand(n, device=DEV)
+        colabs = torch.rand(n, device=DEV, dtype=torch.float64)
+        nu = n // group
+        ws = torch.empty(api.workspace_bytes(api.SP_WS_SCORES, n, 0, d, 0, api.SP_F32), dtype=torch.uint8, device=DEV)
+        for kind, nm in ((api.SP_SCORE_WANDA_L2, "L2"), (api.SP_SCORE_WANDA_L1, "L1")):
+            ms = _timeit_cold(lambda: api.sp_struct_scores(kind, nu, group, W=W, colsq=colsq, colabs=colabs,
+                                                           inv_tokens=1e-5, ws=ws), reps, warm, flush)
+            line(f"scores Wanda-{nm}  W [{d}, {n}] fp32, units of {group}", ms, 4.0 * d * n)
+        del W
+    # Lemma-1 scores streamed from four [N, n] tensors
+    for N, n, dt, sz in ((32768, 8192, torch.bfloat16, 2), (16384, 8192, torch.float32, 4)):
+        b, c, dd, t = (_rnd((N, n), dt) for _ in range(4))
+        ws = torch.empty(api.workspace_bytes(api.SP_WS_SCORES, n, 0, N, 0, api.SP_F32), dtype=torch.uint8, device=DEV)
+        ms = _timeit_cold(lambda: api.sp_struct_scores(api.SP_SCORE_LEMMA1, n, 1, b=b, c=c, dd=dd, t=t, ws=ws), reps,
+                          warm, flush)
+        line(f"scores Lemma-1 streamed  4 x [{N}, {n}] {str(dt)[6:]}", ms, 4.0 * N * n * sz)
+        del b, c, dd, t
+    # allocation over the layers of a model
+    for L in (24, 32, 64):
+        I = torch.rand(L, dtype=torch.float64, device=DEV) + 0.5
+        nu = torch.full((L,), 8192, dtype=torch.int64, device=DEV)
+        ms = _timeit_cold(lambda: api.sp_allocate_sparsity(I, nu, 0.5, 1.0), reps, warm, flush)
+        line(f"allocate  L = {L}", ms, 32.0 * L)
+    # top-k: one layer, and all layers of a model in one launch (4 B score read + 1 B mask written per unit)
+    for n, k in ((8192, 4096), (28672, 5734)):
+        sc = torch.randn(n, device=DEV)
+        ms = _timeit_cold(lambda: api.sp_apply_mask(sc, k, want_index=True), reps, warm, flush)
+        line(f"top-k  n = {n}, k = {k}", ms, 9.0 * n)
+    for L, n in ((24, 8192), (32, 16384), (32, 28672), (148, 28672)):
+        sc = torch.randn(L, n, device=DEV)
+        kk = torch.full((L,), n // 2, dtype=torch.int64, device=DEV)
+        ms = _timeit_cold(lambda: api.sp_apply_mask_batched(sc, kk), reps, warm, flush)
+        line(f"top-k batched  L = {L}, n = {n}", ms, 5.0 * L * n)
+
+
+def _hbm_peak():
+    import json
+    import os
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except (OSError, KeyError, ValueError):
+        return 6650.0, "fallback"
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "solve"])
+    ap.add_argument("what", choices=["gemm", "solve", "mask"])
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warm", type=int, default=2)
     a = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("microbench needs a CUDA device")
     api.lib()
-    (gemm_cases if a.what == "gemm" else solve_cases)(a.reps, a.warm)
+    if a.what == "mask":
+        peak, src = _hbm_peak()
+        print(f"HBM peak {peak:.0f} GB/s ({src})")
+        mask_cases(a.reps, a.warm, peak)
+    else:
+        (gemm_cases if a.what == "gemm" else solve_cases)(a.reps, a.warm)
 
 
 if __name__ == "__main__":

@@ -235,8 +235,8 @@ def test_allocate_sparsity(mode, name, L):
 
 
 # ------------------------------------------------------------------------------------------------ top-k + mask
-@pytest.mark.parametrize("n,k", [(1, 1), (17, 0), (17, 17), (1000, 1), (1000, 999), (3072, 1536), (28672, 5734),
-                                 (200000, 77777)])
+@pytest.mark.parametrize("n,k", [(1, 1), (17, 0), (17, 17), (1000, 1), (1000, 999), (1025, 513), (3072, 1536),
+                                 (28672, 5734), (47104, 20000), (47105, 123), (200000, 77777)])
 def test_apply_mask_topk(n, k):
     s = _gauss((n,), 30 + n % 7)
     s = torch.round(s * 50) / 50          # many exact ties
@@ -248,6 +248,28 @@ def test_apply_mask_topk(n, k):
     if 0 < k:
         assert np.array_equal(idx.cpu().numpy(), np.flatnonzero(mo).astype(np.int32))
         assert tau.item() == tauo or (np.isnan(tau.item()) and np.isnan(tauo))
+
+
+def test_apply_mask_batched_all_layers_in_one_launch():
+    """Algorithm 1 Step 3 for every layer at once: per-layer kept counts read on the device, rows with a leading
+    dimension larger than n_units, counts 0 and n_units among them, many exact ties."""
+    L, n, ld = 7, 3001, 3008
+    buf = torch.full((L, ld), float("nan"))
+    for l in range(L):
+        buf[l, :n] = torch.round(_gauss((n,), 60 + l) * 20) / 20
+    buf[2, 5] = float("nan"); buf[3, 9] = float("inf"); buf[3, 10] = -0.0
+    ks = [1500, 0, n, 1, n - 1, 777, 2999]
+    sg = buf.to(DEV)
+    mask, tau, idx = api.sp_apply_mask_batched(sg[:, :n], torch.tensor(ks, dtype=torch.int64, device=DEV),
+                                               want_index=True)
+    mask, tau, idx = mask.cpu().numpy(), tau.cpu().numpy(), idx.cpu().numpy()
+    for l in range(L):
+        mo, tauo = O.topk_mask(buf[l, :n].numpy(), ks[l])
+        assert np.array_equal(mask[l], mo), l
+        assert np.array_equal(idx[l, :ks[l]], np.flatnonzero(mo).astype(np.int32)), l
+        assert np.all(idx[l, ks[l]:] == -1)
+        if ks[l] > 0:
+            assert tau[l] == tauo or (np.isnan(tau[l]) and np.isnan(tauo))
 
 
 @pytest.mark.parametrize("group", [1, 64])
