@@ -108,7 +108,7 @@ struct Carver {
 
 size_t dinv_elems(int64_t n) {
   const size_t simt = (size_t)ceil_div(n, (int64_t)kCholNB) * kCholNB * kCholNB;
-  const size_t tc = (size_t)ceil_div(n, (int64_t)kCholTcNB) * 2 * kCholTcNB * kCholTcNB;
+  const size_t tc = ((size_t)ceil_div(n, (int64_t)kCholTcNB) + 1) * 2 * kCholTcNB * kCholTcNB;   // + scratch pair
   return simt > tc ? simt : tc;
 }
 
@@ -145,7 +145,8 @@ SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
 template <typename T>
 sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_full,
                      const int32_t* idx, int64_t k, const double* rho_dev, float* W, int64_t ldw, SolveBufs& b,
-                     int32_t* status, cudaStream_t stream, const SolveAssist* assist = nullptr) {
+                     int32_t* status, cudaStream_t stream, const SolveAssist* assist = nullptr,
+                     bool factor_lookahead = true) {
   const int64_t nn = idx ? k : n_full;
   ProfScope prof(PK_SOLVE, (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
   T* Gs = reinterpret_cast<T*>(b.Gs);
@@ -154,7 +155,7 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
   if (idx) CU(load_spd_gather<T>(G, ldg, idx, nn, rho_dev, Gs, nn, stream));
   else CU(load_spd<T>(G, ldg, nn, rho_dev, Gs, nn, stream));
   if constexpr (sizeof(T) == 4) {
-    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream));
+    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, factor_lookahead ? assist : nullptr));
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
     SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist));
   } else {
@@ -701,8 +702,10 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     CU(cudaEventRecord(side->z1_done, side->stream));
   }
   if (prm->refit) {
+    // beside the z1 products the factorisation keeps to one stream: its lookahead kernel is a cluster of 8 CTAs,
+    // which finds no free group of SMs while the persistent GEMM CTAs hold most of them
     if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
-                                      side ? &side->assist_main : nullptr));
+                                      side ? &side->assist_main : nullptr, !z1_ahead));
     else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
                                       side ? &side->assist_main : nullptr));
   } else {
@@ -734,7 +737,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
       float* Gs = reinterpret_cast<float*>(p.sb.Gs);
       float* Rs = reinterpret_cast<float*>(p.sb.Rs);
       CU(load_spd<float>(p.Cf, d, d, gam, Gs, d, s));
-      SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s));
+      SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s,
+                           (side && !z1_ahead) ? &side->assist_main : nullptr));
       // right-hand sides: the rows of W2[:, S]^T as the tensor-core path sees them (bf16-rounded)
       CU(convert_matrix(p.W2b, SP_BF16, kp, p.W2cf, SP_F32, kp, d, k, s));
       CU(transpose_convert<float>(p.W2cf, kp, d, k, Rs, d, s));

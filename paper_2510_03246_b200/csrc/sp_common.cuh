@@ -104,13 +104,15 @@ constexpr int kCholNB = 64;
 //   Xs  : 2 x bf16 [m, 3 * kCholTcNB] — the current block column of the right-hand sides as three bf16 parts
 constexpr int kCholTcNB = 128;
 int64_t chol_tc_pad(int64_t n);
-sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P, int32_t* status_dev,
-                         cudaStream_t stream);
-// Optional second stream (with three events) that carries the far part of each solve step's update.
+// Optional second stream (with three events) that carries the part of each step that the next step's first kernel
+// does not wait for: the far part of a solve step's update; the panel and trailing update of a factorisation step.
 struct SolveAssist {
   cudaStream_t stream;
   cudaEvent_t panel_done, rest_done[2];
 };
+// dinv must have room for ceil(n / 128) + 1 pairs of 128 x 128 blocks (the last pair is scratch).
+sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P, int32_t* status_dev,
+                         cudaStream_t stream, const SolveAssist* assist = nullptr);
 // Xs holds TWO buffers of [m, 3 * kCholTcNB] bf16.
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* P, const float* dinv, void* Xs,
                          int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist = nullptr);

@@ -251,28 +251,71 @@ __device__ __forceinline__ void split3(float v, __nv_bfloat16& hi, __nv_bfloat16
   lo = __float2bfloat16_rn(r2);
 }
 
+// ---- staging of one 128 x 128 fp32 block (64 KiB) into shared memory by bulk asynchronous copies
+__device__ __forceinline__ uint32_t lin_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// One thread: arm the barrier with the byte count and issue the copies (four of 16 KiB).
+__device__ __forceinline__ void stage_block_issue(float* dst_smem, const float* src, uint64_t* bar) {
+  const uint32_t b = lin_smem_u32(bar);
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"((uint32_t)(TB * TB * 4))
+               : "memory");
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(lin_smem_u32(dst_smem + q * (TB * TB / 4))), "l"(src + q * (TB * TB / 4)),
+                   "r"((uint32_t)(TB * TB)), "r"(b)
+                 : "memory");
+}
+__device__ __forceinline__ void stage_bar_init(uint64_t* bar) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(lin_smem_u32(bar)) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+// Every thread: wait for the block (phase `parity`), at most about a second.  Returns false when the wait ran out.
+__device__ __forceinline__ bool stage_block_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t b = lin_smem_u32(bar);
+  const long long t0 = clock64();
+  for (uint32_t it = 0;; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(b), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((it & 0xffu) == 0xffu && clock64() - t0 > 2000000000ll) return false;
+  }
+}
+
 constexpr int PA_ROWS = 32;
-constexpr int PA_THREADS = 128;
+constexpr int PA_THREADS = 256;
 constexpr int PA_APAD = PA_ROWS + 4;
-constexpr size_t PA_SMEM = ((size_t)TB * TB + (size_t)TB * PA_APAD) * sizeof(float);
+constexpr size_t PA_SMEM = ((size_t)TB * TB + (size_t)TB * PA_APAD) * sizeof(float) + 16;
 
 // X[i, 0:nb] <- X[i, 0:nb] inv(L)^T (TRANS == false) or X[i, 0:nb] inv(L) (TRANS == true), for `rows` rows.
 // dinv is the pair of TB x TB blocks written by chol_diag128_kernel.  The result is written back in fp32 (write_f32)
 // and as three bf16 parts to S[i * lds + part * s_seg + c] for all TB columns (zero beyond nb).
-// One CTA takes 32 rows; a thread computes 4 rows x 8 columns (two groups of 4, half a block apart, so that the
-// 16-byte shared loads of a warp fall on distinct banks).
+// One CTA takes 32 rows.  The 64 KiB block of inv(L) comes in by bulk copies while the threads fetch and transpose
+// the rows of X; a thread then computes 4 rows x 4 columns (a warp: 4 rows x 128 columns).
 template <bool TRANS>
 __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64_t ldx, int64_t rows, int nb,
                                                                  const float* __restrict__ dinv, __nv_bfloat16* S,
-                                                                 int64_t lds, int64_t s_seg, int write_f32) {
-  extern __shared__ __align__(16) float pa_smem[];
+                                                                 int64_t lds, int64_t s_seg, int write_f32,
+                                                                 int32_t* status) {
+  extern __shared__ __align__(128) float pa_smem[];
   float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(pa_smem);                       // Lt[k][c]
   float (*At)[PA_APAD] = reinterpret_cast<float (*)[PA_APAD]>(pa_smem + TB * TB);   // At[k][row]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(pa_smem + TB * TB + TB * PA_APAD);
   const int t = threadIdx.x;
   const int64_t r0 = (int64_t)blockIdx.x * PA_ROWS;
   const bool x_al = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0);
+  if (t == 0) stage_bar_init(bar);
+  __syncthreads();
+  // Lt[k][c] = inv(L)[c][k] (the transposed copy) or inv(L)[k][c]: a straight copy either way
+  if (t == 0) stage_block_issue(pa_smem, dinv + (TRANS ? 0 : TB * TB), bar);
   {
-    // the rows of X first (the loads of all 8 float4 of a thread are in flight together) ...
     float4 xv[PA_ROWS * TB / 4 / PA_THREADS];
 #pragma unroll
     for (int q = 0; q < PA_ROWS * TB / 4 / PA_THREADS; ++q) {
@@ -293,11 +336,6 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
       }
       xv[q] = v;
     }
-    // ... then Lt[k][c] = inv(L)[c][k] (the transposed copy) or inv(L)[k][c]: a straight copy either way
-    const float4* src = reinterpret_cast<const float4*>(dinv + (TRANS ? 0 : TB * TB));
-    float4* dst = reinterpret_cast<float4*>(pa_smem);
-#pragma unroll 16
-    for (int e = t; e < TB * TB / 4; e += PA_THREADS) dst[e] = src[e];
 #pragma unroll
     for (int q = 0; q < PA_ROWS * TB / 4 / PA_THREADS; ++q) {
       const int e = t + q * PA_THREADS;
@@ -305,61 +343,62 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
       At[k][i] = xv[q].x; At[k + 1][i] = xv[q].y; At[k + 2][i] = xv[q].z; At[k + 3][i] = xv[q].w;
     }
   }
+  const bool staged = stage_block_wait(bar, 0);
   __syncthreads();
-  const int tx = t & 15, ty = t >> 4;   // columns 4 tx .. 4 tx + 3 and 64 + 4 tx .. 64 + 4 tx + 3, rows 4 ty .. 4 ty + 3
-  float acc[4][8];
+  if (!staged) {   // the copies did not land in time: report and leave X untouched
+    if (t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 10);
+    return;
+  }
+  const int tx = t & 31, ty = t >> 5;   // columns 4 tx .. 4 tx + 3, rows 4 ty .. 4 ty + 3
+  float acc[4][4];
 #pragma unroll
   for (int r = 0; r < 4; ++r)
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[r][j] = 0.f;
-#pragma unroll 4
+    for (int j = 0; j < 4; ++j) acc[r][j] = 0.f;
+#pragma unroll 8
   for (int k = 0; k < TB; ++k) {
     const float4 a0 = *reinterpret_cast<const float4*>(&At[k][4 * ty]);
     const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][4 * tx]);
-    const float4 l1 = *reinterpret_cast<const float4*>(&Lt[k][TB / 2 + 4 * tx]);
     const float av[4] = {a0.x, a0.y, a0.z, a0.w};
-    const float lv[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+    const float lv[4] = {l0.x, l0.y, l0.z, l0.w};
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
+      for (int j = 0; j < 4; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
   }
   const bool x_vec = write_f32 && x_al;
+  const int c0 = 4 * tx;
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
     const int64_t gi = r0 + 4 * ty + r;
     if (gi >= rows) continue;
+    float v[4];
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int c0 = half * (TB / 2) + 4 * tx;
-      float v[4];
+    for (int j = 0; j < 4; ++j) v[j] = (c0 + j < nb) ? acc[r][j] : 0.f;
+    if (write_f32) {
+      float* dst = X + gi * ldx + c0;
+      if (x_vec && c0 + 4 <= nb) {
+        *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) v[j] = (c0 + j < nb) ? acc[r][half * 4 + j] : 0.f;
-      if (write_f32) {
-        float* dst = X + gi * ldx + c0;
-        if (x_vec && c0 + 4 <= nb) {
-          *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if (c0 + j < nb) dst[j] = v[j];
-        }
+        for (int j = 0; j < 4; ++j)
+          if (c0 + j < nb) dst[j] = v[j];
       }
-      if (S) {   // S + gi * lds + part * s_seg + c0 is 8-byte aligned by construction (lds, s_seg multiples of 8)
-        __align__(8) __nv_bfloat16 part[3][4];
+    }
+    if (S) {   // S + gi * lds + part * s_seg + c0 is 8-byte aligned by construction (lds, s_seg multiples of 8)
+      __align__(8) __nv_bfloat16 part[3][4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) split3(v[j], part[0][j], part[1][j], part[2][j]);
+      for (int j = 0; j < 4; ++j) split3(v[j], part[0][j], part[1][j], part[2][j]);
 #pragma unroll
-        for (int q = 0; q < 3; ++q)
-          *reinterpret_cast<uint2*>(S + gi * lds + q * s_seg + c0) = *reinterpret_cast<const uint2*>(part[q]);
-      }
+      for (int q = 0; q < 3; ++q)
+        *reinterpret_cast<uint2*>(S + gi * lds + q * s_seg + c0) = *reinterpret_cast<const uint2*>(part[q]);
     }
   }
 }
 
 template <bool TRANS>
 cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, const float* dinv, __nv_bfloat16* S,
-                               int64_t lds, int64_t s_seg, bool write_f32, cudaStream_t stream) {
+                               int64_t lds, int64_t s_seg, bool write_f32, int32_t* status, cudaStream_t stream) {
   static bool attr = false;
   if (!attr) {
     cudaError_t e = cudaFuncSetAttribute(panel_apply_kernel<TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -371,12 +410,111 @@ cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, cons
   count_launch();
   ProfScope prof(PK_PANEL_APPLY, 2.0 * (double)rows * TB * TB, 0.0, stream);
   panel_apply_kernel<TRANS><<<(unsigned)ceil_div(rows, PA_ROWS), PA_THREADS, PA_SMEM, stream>>>(
-      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0);
+      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status);
   return cudaGetLastError();
 }
 
 // The six kept part products of two three-part operands: A parts (hi, hi, mid, hi, lo, mid) against B parts
 // (hi, mid, hi, lo, hi, mid).
+// ---------------------------------------------------------------------------------------------------------------
+// Lookahead of the factorisation: the NEXT diagonal block, updated with the block column just factored, in one small
+// launch, so that its factorisation does not wait for the full panel and the trailing update:
+//   Lm = A21 inv(L_kk)^T  (nb2 x 128),   S = A22 - Lm Lm^T  (nb2 x nb2, fp32, into a scratch block with ld 128)
+// with A21 = A[next block rows, block k columns] and A22 = A[next block, next block] as the trailing updates up to
+// step k - 1 left them.  One cluster of 8 CTAs, 16 rows each: every CTA forms its rows of Lm, publishes them
+// (transposed, in global scratch LmT[c][row]), the cluster meets, and every CTA forms its rows of S from all of Lm.
+constexpr int NM_ROWS = 16, NM_THREADS = 256, NM_APAD = NM_ROWS + 4, NM_CTAS = TB / NM_ROWS;
+constexpr size_t NM_SMEM = ((size_t)TB * TB + (size_t)TB * NM_APAD) * sizeof(float) + 16;
+static_assert(NM_CTAS == 8, "one portable cluster covers the block");
+
+__device__ __forceinline__ void cluster_meet() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
+    chol_next_diag_kernel(const float* __restrict__ A21, const float* __restrict__ A22, int64_t lda, int nb2,
+                          const float* __restrict__ dinv, float* LmT, float* S, int32_t* status) {
+  extern __shared__ __align__(128) float nm_smem[];
+  float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(nm_smem);                       // Lt[k][c]
+  float (*At)[NM_APAD] = reinterpret_cast<float (*)[NM_APAD]>(nm_smem + TB * TB);   // At[k][row]
+  uint64_t* bar = reinterpret_cast<uint64_t*>(nm_smem + TB * TB + TB * NM_APAD);
+  const int t = threadIdx.x;
+  const int i0 = (int)blockIdx.x * NM_ROWS;
+  const int tx = t & 31, ty = t >> 5;   // columns 4 tx .. 4 tx + 3; rows 2 ty, 2 ty + 1
+  // ---- stage 1: rows i0 .. i0 + 15 of Lm; Lt[k][c] = inv(L)[c][k] comes in by bulk copies
+  if (t == 0) stage_bar_init(bar);
+  __syncthreads();
+  if (t == 0) stage_block_issue(nm_smem, dinv + TB * TB, bar);
+  for (int e = t; e < NM_ROWS * TB; e += NM_THREADS) {
+    const int i = e / TB, k = e % TB;
+    At[k][i] = (i0 + i < nb2) ? A21[(int64_t)(i0 + i) * lda + k] : 0.f;
+  }
+  const bool staged = stage_block_wait(bar, 0);
+  __syncthreads();
+  if (!staged && t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 11);
+  // (a CTA whose copies did not land still takes part in the cluster barrier below; its rows are then wrong and the
+  //  status says so)
+  float acc[2][4];
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[r][j] = 0.f;
+#pragma unroll 8
+  for (int k = 0; k < TB; ++k) {
+    const float2 a = *reinterpret_cast<const float2*>(&At[k][2 * ty]);
+    const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][4 * tx]);
+    const float av[2] = {a.x, a.y};
+    const float lv[4] = {l0.x, l0.y, l0.z, l0.w};
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
+  }
+  __syncthreads();   // everyone is done with At and Lt
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = 4 * tx + j;
+    const float2 v = make_float2(acc[0][j], acc[1][j]);
+    *reinterpret_cast<float2*>(&At[c][2 * ty]) = v;                              // own rows, left operand of stage 2
+    *reinterpret_cast<float2*>(&LmT[(int64_t)c * TB + i0 + 2 * ty]) = v;         // for the other CTAs
+  }
+  cluster_meet();
+  // ---- stage 2: rows i0 .. i0 + 15 of S; Lt[c][j] = Lm[j][c]
+  {
+    const float4* src = reinterpret_cast<const float4*>(LmT);
+    float4* dst = reinterpret_cast<float4*>(nm_smem);
+#pragma unroll
+    for (int q = 0; q < TB * TB / 4 / NM_THREADS; ++q) dst[t + q * NM_THREADS] = __ldcg(src + t + q * NM_THREADS);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[r][j] = 0.f;
+#pragma unroll 8
+  for (int k = 0; k < TB; ++k) {
+    const float2 a = *reinterpret_cast<const float2*>(&At[k][2 * ty]);
+    const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][4 * tx]);
+    const float av[2] = {a.x, a.y};
+    const float lv[4] = {l0.x, l0.y, l0.z, l0.w};
+#pragma unroll
+    for (int r = 0; r < 2; ++r)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int i = i0 + 2 * ty + r;
+    float v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = 4 * tx + j;
+      v[j] = (i < nb2 && c <= i) ? A22[(int64_t)i * lda + c] - acc[r][j] : 0.f;
+    }
+    *reinterpret_cast<float4*>(&S[i * TB + 4 * tx]) = make_float4(v[0], v[1], v[2], v[3]);
+  }
+}
+
 constexpr int kPartA[6] = {0, 0, 1, 0, 2, 1};
 constexpr int kPartB[6] = {0, 1, 0, 2, 0, 1};
 
@@ -385,30 +523,62 @@ constexpr int kPartB[6] = {0, 1, 0, 2, 0, 1};
 int64_t chol_tc_pad(int64_t n) { return (n + TB - 1) / TB * TB; }
 
 sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv, int32_t* status_dev,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, const SolveAssist* assist) {
   __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
-  static bool diag_attr = false;
-  if (!diag_attr) {
+  const int64_t nblk = ceil_div(n, (int64_t)TB);
+  static bool attr_set = false;
+  if (!attr_set) {
     if (cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM) !=
-        cudaSuccess)
+            cudaSuccess ||
+        cudaFuncSetAttribute(chol_next_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NM_SMEM) !=
+            cudaSuccess)
       return SP_ERR_CUDA;
-    diag_attr = true;
+    attr_set = true;
   }
-  for (int64_t k0 = 0; k0 < n; k0 += TB) {
+#define SP_CUDA_OK(x) do { if ((x) != cudaSuccess) return SP_ERR_CUDA; } while (0)
+  // With an assisting stream the chain of diagonal blocks runs ahead: after block k is factored, a small kernel
+  // forms the next diagonal block (into scratch behind the inverses), and the next factorisation starts from it while
+  // the full panel and the trailing update of step k run on the assisting stream.
+  float* S = dinv + nblk * 2 * TB * TB;      // [128, 128] next diagonal block
+  float* LmT = S + TB * TB;                  // [128, 128] scratch of the lookahead kernel
+  bool rec[2] = {false, false};
+  for (int64_t kb = 0; kb < nblk; ++kb) {
+    const int64_t k0 = kb * TB;
     const int nb = (int)((n - k0 < TB) ? (n - k0) : TB);
-    float* dk = dinv + (k0 / TB) * 2 * TB * TB;
+    float* dk = dinv + kb * 2 * TB * TB;
     {
+      const bool from_scratch = assist && kb > 0;
       count_launch();
       ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
-      chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(A + k0 * lda + k0, lda, nb, dk, k0, status_dev);
+      chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
+                                                                  from_scratch ? (int64_t)TB : lda, nb, dk, k0,
+                                                                  status_dev);
       if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     }
     const int64_t rem = n - k0 - nb;
     if (rem <= 0) break;
+    cudaStream_t sb = stream;
+    if (assist) {
+      // next diagonal block: needs the trailing update of step kb - 1 (assisting stream)
+      if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
+      const int nb2 = (int)(rem < TB ? rem : TB);
+      {
+        count_launch();
+        ProfScope prof(PK_PANEL_APPLY, 4.0 * TB * TB * TB, 0.0, stream);
+        chol_next_diag_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + k0,
+                                                                        A + (k0 + nb) * lda + (k0 + nb), lda, nb2, dk,
+                                                                        LmT, S, status_dev);
+        if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+      }
+      // the panel overwrites A21 in place: it starts behind the lookahead kernel
+      SP_CUDA_OK(cudaEventRecord(assist->panel_done, stream));
+      sb = assist->stream;
+      SP_CUDA_OK(cudaStreamWaitEvent(sb, assist->panel_done, 0));
+    }
     // L21 = A21 inv(L11)^T, fp32 in place and as bf16 parts in P[k0+nb.., part * np + k0 ..]
     if (launch_panel_apply<false>(A + (k0 + nb) * lda + k0, lda, rem, nb, dk, P + (k0 + nb) * ldp + k0, ldp, np, true,
-                                  stream) != cudaSuccess)
+                                  status_dev, sb) != cudaSuccess)
       return SP_ERR_CUDA;
     // A22 -= L21 L21^T on the lower triangle
     TcOperand ta{P + (k0 + nb) * ldp, ldp, true};
@@ -416,15 +586,23 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     ta.mnext = rem;
     TcSegments sg;
     sg.nseg = 6;
-    for (int s = 0; s < 6; ++s) {
-      sg.a_k[s] = (int32_t)(kPartA[s] * np + k0);
-      sg.b_k[s] = (int32_t)(kPartB[s] * np + k0);
+    for (int q = 0; q < 6; ++q) {
+      sg.a_k[q] = (int32_t)(kPartA[q] * np + k0);
+      sg.b_k[q] = (int32_t)(kPartB[q] * np + k0);
     }
     float* A22 = A + (k0 + nb) * lda + (k0 + nb);
     sp_status st = gemm_tc(rem, rem, TB, -1.f, ta, ta, 1.f, Operand{A22, SP_F32, lda, 1}, OutOperand{A22, SP_F32, lda},
-                           true, status_dev, stream, &sg, (double)rem * (double)rem * (double)nb);
+                           true, status_dev, sb, &sg, (double)rem * (double)rem * (double)nb);
     if (st != SP_OK) return st;
+    if (assist) {
+      SP_CUDA_OK(cudaEventRecord(assist->rest_done[kb & 1], sb));
+      rec[kb & 1] = true;
+    }
   }
+  // the factor is complete on `stream` once the assisting stream has drained
+  for (int q = 0; q < 2; ++q)
+    if (assist && rec[q]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[q], 0));
+#undef SP_CUDA_OK
   return SP_OK;
 }
 
@@ -449,8 +627,8 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
       const float* dj = dinv + jb * 2 * TB * TB;
       __nv_bfloat16* Xcur = Xs + (step & 1) * m * lds;
       if (assist && rec[step & 1]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[step & 1], 0));
-      cudaError_t e = forward ? launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, stream)
-                              : launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, stream);
+      cudaError_t e = forward ? launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, status_dev, stream)
+                              : launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, status_dev, stream);
       if (e != cudaSuccess) return SP_ERR_CUDA;
       // columns still to be updated: [lo, hi)
       const int64_t lo = forward ? j0 + nb : 0, hi = forward ? n : j0;
