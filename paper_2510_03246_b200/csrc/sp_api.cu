@@ -116,7 +116,6 @@ size_t dinv_elems(int64_t n) {
 struct SolveBufs {
   void* Gs;
   void* dinv;
-  void* Rs;
   int32_t* idx;
   double* rho;  // [4] device scalars
   void* P;      // fp32 path: bf16 parts of the Cholesky factor
@@ -127,14 +126,14 @@ SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
   SolveBufs b;
   b.rho = c.take<double>(4);
   b.idx = c.take<int32_t>((size_t)nmax);
-  b.Gs = c.take_bytes((size_t)nmax * nmax * tsize);
+  // the system matrix and, right behind its nn x nn elements, the right-hand sides (one [nn + m, nn] array)
+  b.Gs = c.take_bytes((size_t)(nmax + mmax) * nmax * tsize);
   b.dinv = c.take_bytes(dinv_elems(nmax) * tsize);
-  b.Rs = c.take_bytes((size_t)nmax * mmax * tsize);
   b.P = nullptr;
   b.Xs = nullptr;
   if (tsize == 4) {
     const size_t np = (size_t)chol_tc_pad(nmax);
-    b.P = c.take_bytes(np * 3 * np * 2);
+    b.P = c.take_bytes((np + (size_t)mmax) * 3 * np * 2);
     const size_t rows = (size_t)(nmax > mmax ? nmax : mmax);   // either dimension may be the right-hand-side count
     b.Xs = c.take_bytes(2 * rows * 3 * kCholTcNB * 2);
   }
@@ -151,13 +150,15 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
   ProfScope prof(PK_SOLVE, (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
   T* Gs = reinterpret_cast<T*>(b.Gs);
   T* dinv = reinterpret_cast<T*>(b.dinv);
-  T* Rs = reinterpret_cast<T*>(b.Rs);
+  T* Rs = Gs + (size_t)nn * nn;     // the right-hand sides sit right below the system matrix, same leading dimension
   if (idx) CU(load_spd_gather<T>(G, ldg, idx, nn, rho_dev, Gs, nn, stream));
   else CU(load_spd<T>(G, ldg, nn, rho_dev, Gs, nn, stream));
   if constexpr (sizeof(T) == 4) {
-    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, factor_lookahead ? assist : nullptr));
+    // the right-hand sides ride through the factorisation as m more rows (their forward substitution); the solve
+    // proper is then only the backward sweep
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
-    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist));
+    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, factor_lookahead ? assist : nullptr, m));
+    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist, true));
   } else {
     CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
@@ -735,20 +736,20 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     ProfScope prof(PK_SOLVE, (double)d * d * d / 3.0 + 2.0 * (double)k * d * d, 0.0, s);
     if (bf16) {
       float* Gs = reinterpret_cast<float*>(p.sb.Gs);
-      float* Rs = reinterpret_cast<float*>(p.sb.Rs);
+      float* Rs = Gs + (size_t)d * d;     // right-hand sides below the system matrix: they ride through the factorisation
       CU(load_spd<float>(p.Cf, d, d, gam, Gs, d, s));
-      SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s,
-                           (side && !z1_ahead) ? &side->assist_main : nullptr));
       // right-hand sides: the rows of W2[:, S]^T as the tensor-core path sees them (bf16-rounded)
       CU(convert_matrix(p.W2b, SP_BF16, kp, p.W2cf, SP_F32, kp, d, k, s));
       CU(transpose_convert<float>(p.W2cf, kp, d, k, Rs, d, s));
+      SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s,
+                           (side && !z1_ahead) ? &side->assist_main : nullptr, k));
       SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s,
-                           side ? &side->assist_main : nullptr));
+                           side ? &side->assist_main : nullptr, true));
       CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));
       qt = MatRef{p.Qtb, SP_BF16, d};
     } else {
       double* Gs = reinterpret_cast<double*>(p.sb.Gs);
-      double* Rs = reinterpret_cast<double*>(p.sb.Rs);
+      double* Rs = Gs + (size_t)d * d;
       CU(load_spd<double>(p.Cf, d, d, gam, Gs, d, s));
       CU(potrf_lower<double>(Gs, d, d, reinterpret_cast<double*>(p.sb.dinv), status_dev, s));
       CU(transpose_convert<double>(p.W2cf, kp, d, k, Rs, d, s));

@@ -111,11 +111,15 @@ struct SolveAssist {
   cudaEvent_t panel_done, rest_done[2];
 };
 // dinv must have room for ceil(n / 128) + 1 pairs of 128 x 128 blocks (the last pair is scratch).
+// m_extra > 0: A has m_extra more rows below row n (same lda), the right-hand sides B of a system X L^T = B; they
+// are carried through the panels and trailing updates and hold X on return (P then needs n + m_extra rows).
 sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P, int32_t* status_dev,
-                         cudaStream_t stream, const SolveAssist* assist = nullptr);
+                         cudaStream_t stream, const SolveAssist* assist = nullptr, int64_t m_extra = 0);
 // Xs holds TWO buffers of [m, 3 * kCholTcNB] bf16.
+// forward_done: X already holds the solution of the forward system (it rode along with the factorisation).
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* P, const float* dinv, void* Xs,
-                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist = nullptr);
+                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist = nullptr,
+                         bool forward_done = false);
 
 // ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,

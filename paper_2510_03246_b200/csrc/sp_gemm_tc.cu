@@ -231,21 +231,23 @@ __device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, i
       tn = t / p.tiles_m;
     }
   } else {
-    // Lower triangle of a square grid of tiles, walked in bands of kBandRows tile rows, column by column inside a
-    // band: the tiles that run at the same time then share the band's few row panels (which stay in L2) and stream
-    // each column panel once per band.
+    // Tiles (tm, tn) with tn <= tm of a tiles_m x tiles_n grid (tiles_m >= tiles_n: the lower triangle of a square
+    // product, with any rows below the square taking part in full), walked in bands of kBandRows tile rows, column by
+    // column inside a band: the tiles that run at the same time then share the band's few row panels (which stay in
+    // L2) and stream each column panel once per band.
     int r0 = 0, r1 = 0;
     for (;;) {
       r1 = (r0 + kBandRows < p.tiles_m) ? r0 + kBandRows : p.tiles_m;
-      const int cnt = (r1 * (r1 + 1) - r0 * (r0 + 1)) / 2;     // sum over rows r0..r1-1 of (row + 1)
+      int cnt = 0;
+      for (int r = r0; r < r1; ++r) cnt += (r + 1 < p.tiles_n) ? r + 1 : p.tiles_n;
       if (t < cnt || r1 >= p.tiles_m) break;     // the second test only bounds the loop
       t -= cnt;
       r0 = r1;
     }
     for (tn = 0;; ++tn) {
       const int first = tn > r0 ? tn : r0;
-      const int c = r1 - first;
-      if (t < c || tn >= p.tiles_m - 1) { tm = first + (t < c ? t : 0); break; }
+      const int c = r1 > first ? r1 - first : 0;
+      if (t < c || tn >= p.tiles_n - 1) { tm = first + (t < c ? t : 0); break; }
       t -= c;
     }
   }
@@ -653,7 +655,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
     if (a_inner % 8 != 0 || b_inner % 8 != 0) return SP_ERR_ALIGNMENT;
     if (sg.a_k[i] < 0 || sg.a_mn[i] < 0 || sg.b_k[i] < 0 || sg.b_mn[i] < 0) return SP_ERR_INVALID_ARG;
   }
-  if (lower_only && M != N) return SP_ERR_SHAPE;
+  if (lower_only && M < N) return SP_ERR_SHAPE;
   if (beta != 0.f && (Cin.ptr == nullptr || Cin.s1 != 1)) return SP_ERR_INVALID_ARG;
   if (C.dtype != SP_F32 && C.dtype != SP_BF16) return SP_ERR_DTYPE;
   if (beta != 0.f && Cin.dtype != SP_F32 && Cin.dtype != SP_BF16) return SP_ERR_DTYPE;

@@ -523,7 +523,7 @@ constexpr int kPartB[6] = {0, 1, 0, 2, 0, 1};
 int64_t chol_tc_pad(int64_t n) { return (n + TB - 1) / TB * TB; }
 
 sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv, int32_t* status_dev,
-                         cudaStream_t stream, const SolveAssist* assist) {
+                         cudaStream_t stream, const SolveAssist* assist, int64_t m_extra) {
   __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
   const int64_t nblk = ceil_div(n, (int64_t)TB);
@@ -557,9 +557,15 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     }
     const int64_t rem = n - k0 - nb;
-    if (rem <= 0) break;
+    // rows below the block that the panel covers: the rest of the matrix and the m_extra appended rows (right-hand
+    // sides of a system X L^T = B stored below A: the panel and the trailing update are exactly their forward
+    // substitution, so it costs no steps of its own)
+    const int64_t prow = rem + m_extra;
+    if (prow <= 0) break;
     cudaStream_t sb = stream;
-    if (assist) {
+    // last block with appended rows: their panel runs on `stream`, behind the assisting stream's last update
+    if (assist && rem <= 0 && kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
+    if (assist && rem > 0) {
       // next diagonal block: needs the trailing update of step kb - 1 (assisting stream)
       if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
       const int nb2 = (int)(rem < TB ? rem : TB);
@@ -577,13 +583,15 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       SP_CUDA_OK(cudaStreamWaitEvent(sb, assist->panel_done, 0));
     }
     // L21 = A21 inv(L11)^T, fp32 in place and as bf16 parts in P[k0+nb.., part * np + k0 ..]
-    if (launch_panel_apply<false>(A + (k0 + nb) * lda + k0, lda, rem, nb, dk, P + (k0 + nb) * ldp + k0, ldp, np, true,
+    if (launch_panel_apply<false>(A + (k0 + nb) * lda + k0, lda, prow, nb, dk, P + (k0 + nb) * ldp + k0, ldp, np, true,
                                   status_dev, sb) != cudaSuccess)
       return SP_ERR_CUDA;
+    if (rem <= 0) break;     // last block: the appended rows are done, nothing is left to update
     // A22 -= L21 L21^T on the lower triangle
-    TcOperand ta{P + (k0 + nb) * ldp, ldp, true};
-    ta.kext = ldp;
-    ta.mnext = rem;
+    TcOperand ta{P + (k0 + nb) * ldp, ldp, true}, tb{P + (k0 + nb) * ldp, ldp, true};
+    ta.kext = tb.kext = ldp;
+    ta.mnext = prow;
+    tb.mnext = rem;
     TcSegments sg;
     sg.nseg = 6;
     for (int q = 0; q < 6; ++q) {
@@ -591,8 +599,9 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       sg.b_k[q] = (int32_t)(kPartB[q] * np + k0);
     }
     float* A22 = A + (k0 + nb) * lda + (k0 + nb);
-    sp_status st = gemm_tc(rem, rem, TB, -1.f, ta, ta, 1.f, Operand{A22, SP_F32, lda, 1}, OutOperand{A22, SP_F32, lda},
-                           true, status_dev, sb, &sg, (double)rem * (double)rem * (double)nb);
+    sp_status st = gemm_tc(prow, rem, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1}, OutOperand{A22, SP_F32, lda},
+                           true, status_dev, sb, &sg,
+                           ((double)rem * (double)rem + 2.0 * (double)m_extra * (double)rem) * (double)nb);
     if (st != SP_OK) return st;
     if (assist) {
       SP_CUDA_OK(cudaEventRecord(assist->rest_done[kb & 1], sb));
@@ -607,7 +616,7 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
 }
 
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* Pv, const float* dinv, void* Xsv,
-                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist) {
+                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist, bool forward_done) {
   const __nv_bfloat16* P = reinterpret_cast<const __nv_bfloat16*>(Pv);
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(Xsv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
@@ -686,8 +695,10 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
       }
     return SP_OK;
   };
-  sp_status r = run_sweep(true);    // Y L^T = X, block columns left to right
-  if (r != SP_OK) return r;
+  if (!forward_done) {               // (done already when X rode along with the factorisation as appended rows)
+    sp_status r = run_sweep(true);    // Y L^T = X, block columns left to right
+    if (r != SP_OK) return r;
+  }
   return run_sweep(false);          // W L = Y, block columns right to left
 #undef SP_CUDA_OK
 }
