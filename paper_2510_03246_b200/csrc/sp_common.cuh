@@ -21,7 +21,9 @@ __device__ __forceinline__ void report_status(int32_t* status, int32_t code, int
 // ---- launch accounting and CUDA-event profiling (sp_profile.cu) ---------------------------------------------------
 enum ProfKind : int {
   PK_GEMM_TC = 0, PK_GEMM_SIMT = 1, PK_SOLVE = 2, PK_FUSED_UPDATE = 3, PK_PREP_H = 4, PK_SCORES = 5, PK_TOPK = 6,
-  PK_ELEMENTWISE = 7, PK_ALLOCATE = 8, PK_CHOL_DIAG = 9, PK_PANEL_APPLY = 10, PK_COUNT = 11
+  PK_ELEMENTWISE = 7, PK_ALLOCATE = 8, PK_CHOL_DIAG = 9, PK_PANEL_APPLY = 10,
+  PK_GEMM_TC_SHARED = 11,   // tensor-core GEMMs launched on a subset of the SM pairs, beside other work
+  PK_COUNT = 12
 };
 void count_launch(int n = 1);
 // Brackets the kernels launched during its lifetime with a CUDA event pair on `stream` when profiling is enabled.

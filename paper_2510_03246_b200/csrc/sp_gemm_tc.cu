@@ -746,7 +746,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   }
   count_launch();
   const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
-  ProfScope prof(PK_GEMM_TC, flops, 0.0, stream);
+  ProfScope prof(max_pairs > 0 ? PK_GEMM_TC_SHARED : PK_GEMM_TC, flops, 0.0, stream);
   const int pairs = p.num_units < pairs_max ? p.num_units : pairs_max;
   gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
