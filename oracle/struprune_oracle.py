@@ -26,6 +26,8 @@ implemented identically by the CUDA path):
   * Lemma 1 over N calibration tokens: products of scalars become inner products over tokens.
   * threshold: exactly k units are kept (the k largest scores, lower index wins ties, NaN lowest), so
     that the mask budget of Eq. (1) holds with equality.
+  * "-distribute" importances: a head's weight matrix W_h is read as its rows of W_Q, W_K, W_V and its
+    columns of W_O taken together; Var is the population variance over those entries; layers count from 1.
   * allocation: r_l is the fraction PRUNED in layer l, as Algorithm 1 uses it (clip at 0.95, "mask with
     sparsity r_l"); kept count = n_l - round_half_up(r_l n_l).
 
@@ -225,6 +227,47 @@ def allocate_sparsity(I, n_units, rbar, T, mode="softmax", clip_hi=0.95):
     n_units = np.asarray(n_units, np.int64)
     k_keep = np.array([int(n_units[l]) - _round_half_up(r[l] * int(n_units[l])) for l in range(L)], np.int64)
     return r, k_keep
+
+
+# --------------------------------------------------------------------------------------------------
+# Weight-statistic importances (Algorithm "-distribute", Step 1)
+# --------------------------------------------------------------------------------------------------
+def weight_stats(parts):
+    """(l1 norm, variance, l2 norm) of the entries of one or several weight slices taken together
+    (Algorithm "-distribute", Step 1: the three statistics of a head's or a layer's weight matrix).
+    The variance is the population variance over all entries; the l2 norm is the root of the sum of squares."""
+    v = np.concatenate([np.asarray(p, F64).ravel() for p in parts])
+    m = v.shape[0]
+    mean = v.sum() / m
+    return float(np.abs(v).sum()), float(((v - mean) ** 2).sum() / m), float(math.sqrt((v * v).sum()))
+
+
+def head_slices(Wq, Wk, Wv, Wo, h, d_head):
+    """The weights of attention head h: its d_head rows of W_Q, W_K, W_V and its d_head columns of W_O."""
+    r = slice(h * d_head, (h + 1) * d_head)
+    return [np.asarray(Wq)[r, :], np.asarray(Wk)[r, :], np.asarray(Wv)[r, :], np.asarray(Wo)[:, r]]
+
+
+def distribute_importance(layers, n_heads, d_head, rho, gamma):
+    """Algorithm "-distribute", Step 1.  layers[l] = dict(Wq, Wk, Wv, Wo, fc1, fc2); layer l (counted from 1 as
+    the algorithm does) has depth weight d_l = gamma^l.
+      I_attn[l] = d_l rho sum_h (|W_h|_1 + 0.1 Var(W_h) + 0.01 |W_h|_2)
+      I_mlp[l]  = d_l sum_{m in fc1, fc2} (|W_m|_1 + 0.05 Var(W_m))"""
+    L = len(layers)
+    I_attn, I_mlp = np.zeros(L, F64), np.zeros(L, F64)
+    for l, w in enumerate(layers):
+        dl = gamma ** (l + 1)
+        acc = 0.0
+        for h in range(n_heads):
+            l1, var, l2 = weight_stats(head_slices(w["Wq"], w["Wk"], w["Wv"], w["Wo"], h, d_head))
+            acc += l1 + 0.1 * var + 0.01 * l2
+        I_attn[l] = dl * rho * acc
+        acc = 0.0
+        for name in ("fc1", "fc2"):
+            l1, var, _ = weight_stats([w[name]])
+            acc += l1 + 0.05 * var
+        I_mlp[l] = dl * acc
+    return I_attn, I_mlp
 
 
 # --------------------------------------------------------------------------------------------------

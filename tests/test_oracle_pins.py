@@ -457,3 +457,59 @@ def test_swiglu_zu_is_stationary_point():
     grad = -2 * beta * g * (a - g * zu) + 2 * alpha * (zu - z1)
     assert np.abs(grad).max() < 1e-12
     assert np.allclose(O.silu(np.array([0.0, 1.0])), [0.0, 1.0 / (1.0 + np.exp(-1.0))])
+
+
+def test_weight_stats_closed_forms():
+    """Algorithm "-distribute" Step 1 statistics against textbook closed forms: the entries 0, 1, ..., m-1 have
+    l1 = m(m-1)/2, variance (m^2-1)/12 and sum of squares (m-1)m(2m-1)/6, however they are cut into slices."""
+    m = 60
+    v = np.arange(m, dtype=np.float64)
+    rng = np.random.default_rng(5)
+    perm = rng.permutation(m)
+    parts = [v[perm[:7]].reshape(7, 1), v[perm[7:31]].reshape(4, 6), v[perm[31:]].reshape(1, 29)]
+    l1, var, l2 = O.weight_stats(parts)
+    assert l1 == m * (m - 1) / 2
+    assert abs(var - (m * m - 1) / 12.0) < 1e-12
+    assert abs(l2 - np.sqrt((m - 1) * m * (2 * m - 1) / 6.0)) < 1e-12
+    # signs: the l1 norm ignores them, the variance does not (a +-1 checkerboard has mean 0, variance 1)
+    cb = np.where((np.add.outer(np.arange(6), np.arange(8)) % 2) == 0, 1.0, -1.0)
+    assert O.weight_stats([cb]) == (48.0, 1.0, np.sqrt(48.0))
+    assert O.weight_stats([np.full((3, 5), -2.0)]) == (30.0, 0.0, np.sqrt(60.0))
+    # scaling by c: l1 and l2 scale with |c|, the variance with c^2
+    a = rng.standard_normal((5, 9))
+    s1, s3 = O.weight_stats([a]), O.weight_stats([-3.0 * a])
+    assert abs(s3[0] - 3 * s1[0]) < 1e-12 and abs(s3[1] - 9 * s1[1]) < 1e-12 and abs(s3[2] - 3 * s1[2]) < 1e-12
+
+
+def test_distribute_importance_structure():
+    """Depth decay, the attention/MLP ratio and the head slicing of Algorithm "-distribute" Step 1."""
+    d, n, H = 8, 12, 4
+    dh = d // H
+    rng = np.random.default_rng(9)
+    base = dict(Wq=rng.standard_normal((d, d)), Wk=rng.standard_normal((d, d)), Wv=rng.standard_normal((d, d)),
+                Wo=rng.standard_normal((d, d)), fc1=rng.standard_normal((n, d)), fc2=rng.standard_normal((d, n)))
+    layers = [base, base, base]
+    Ia, Im = O.distribute_importance(layers, H, dh, rho=2.5, gamma=0.9)
+    # identical layers: consecutive importances differ by the factor gamma; layer 1 carries gamma^1
+    assert np.allclose(Ia[1:] / Ia[:-1], 0.9) and np.allclose(Im[1:] / Im[:-1], 0.9)
+    Ia1, Im1 = O.distribute_importance(layers, H, dh, rho=1.0, gamma=1.0)
+    assert np.allclose(Ia, 2.5 * Ia1 * 0.9 ** np.arange(1, 4)) and np.allclose(Im, Im1 * 0.9 ** np.arange(1, 4))
+    # the MLP term by hand: l1 and population variance of fc1 and fc2
+    want = sum(np.abs(base[k]).sum() + 0.05 * base[k].var() for k in ("fc1", "fc2"))
+    assert abs(Im1[0] - want) < 1e-9 * want
+    # head slicing: the l1 parts of all heads together are the l1 norms of the four attention matrices
+    l1_heads = sum(O.weight_stats(O.head_slices(base["Wq"], base["Wk"], base["Wv"], base["Wo"], h, dh))[0]
+                   for h in range(H))
+    assert abs(l1_heads - sum(np.abs(base[k]).sum() for k in ("Wq", "Wk", "Wv", "Wo"))) < 1e-9
+    # a head whose weights are zero contributes nothing; only W_O's COLUMNS of that head count
+    z = {k: v.copy() for k, v in base.items()}
+    z["Wq"][:dh] = 0; z["Wk"][:dh] = 0; z["Wv"][:dh] = 0; z["Wo"][:, :dh] = 0
+    parts0 = O.head_slices(z["Wq"], z["Wk"], z["Wv"], z["Wo"], 0, dh)
+    assert O.weight_stats(parts0) == (0.0, 0.0, 0.0)
+    z["Wo"][:dh, dh:] = 7.0      # rows of W_O are not part of head 0
+    assert O.weight_stats(O.head_slices(z["Wq"], z["Wk"], z["Wv"], z["Wo"], 0, dh)) == (0.0, 0.0, 0.0)
+    # inverse allocation on these importances, as printed (Step 2): w falls with the importance, r = rbar L (1 - w) /
+    # sum(1 - w) rises with it, so the first (most important, least decayed) layer gets the largest pruned fraction;
+    # the mean stays rbar
+    r, _ = O.allocate_sparsity(Im, np.full(3, n), 0.5, T=float(np.abs(Im).mean()), mode="inverse")
+    assert np.all(np.diff(Im) < 0) and np.all(np.diff(r) < 0) and abs(r.mean() - 0.5) < 1e-12
