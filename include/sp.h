@@ -57,7 +57,7 @@ typedef enum { SP_Z_PAPER = 0, SP_Z_EXACT = 1 } sp_z_rule;
 typedef enum { SP_SCORE_WANDA_L2 = 0, SP_SCORE_WANDA_L1 = 1, SP_SCORE_LEMMA1 = 2 } sp_score_kind;
 typedef enum { SP_ALLOC_SOFTMAX = 0, SP_ALLOC_INVERSE = 1, SP_ALLOC_UNIFORM = 2 } sp_alloc_mode;
 typedef enum { SP_WS_GRAM = 0, SP_WS_ADMM_STEP = 1, SP_WS_SCORES = 2, SP_WS_APPLY_MASK = 3, SP_WS_FFN_INIT = 4,
-               SP_WS_LINEAR_REFIT = 5, SP_WS_GEMM = 6, SP_WS_RIDGE_SOLVE = 7 } sp_ws_op;
+               SP_WS_LINEAR_REFIT = 5, SP_WS_GEMM = 6, SP_WS_RIDGE_SOLVE = 7, SP_WS_WEIGHT_STATS = 8 } sp_ws_op;
 
 /* A row-major device matrix view. */
 typedef struct {
@@ -245,6 +245,29 @@ sp_status sp_apply_mask_batched(const float* scores, int64_t ld_scores, int64_t 
                                 int32_t* kept_idx_out, int64_t ld_idx, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
+ * sp_weight_stats, sp_distribute_importance — the weight-statistic importances of the "-distribute" variant of
+ * Algorithm 1 (its Step 1): per attention head |W_h|_1 + 0.1 Var(W_h) + 0.01 |W_h|_2, per MLP matrix
+ * |W_m|_1 + 0.05 Var(W_m), times the depth weight gamma^l (layers counted from 1) and, for attention, the
+ * attention/MLP ratio rho.  Step 2 of that algorithm is sp_allocate_sparsity with SP_ALLOC_INVERSE.
+ *
+ * sp_weight_stats: sums over slices of one weight matrix W (fp32 or bf16, [rows, cols], device).
+ *   axis = 0: block b is rows [b*group, (b+1)*group) (all columns);  axis = 1: block b is columns [b*group, ...)
+ *   (all rows);  group = 0: the whole matrix is one block.  rows (axis 0) / cols (axis 1) must be a multiple of group.
+ *   stats: fp64 [n_blocks, 4] on the device = {sum |w|, sum w, sum w^2, number of entries}; accumulate != 0 adds to
+ *   what it holds, so the slices of one head in W_Q, W_K, W_V (axis 0) and W_O (axis 1) add up to that head's sums.
+ *   Workspace: sp_workspace_bytes(SP_WS_WEIGHT_STATS, n_blocks, 0, 0, 0, 0).  Deterministic (fixed summation order).
+ *   Errors: SP_ERR_INVALID_ARG (null pointers, axis not 0/1), SP_ERR_DTYPE, SP_ERR_SHAPE (group does not divide the
+ *   extent, ld < cols), SP_ERR_WORKSPACE.
+ * sp_distribute_importance: head_stats fp64 [L, n_heads, 4] and fc_stats fp64 [L, n_fc, 4] as written above (either
+ *   may be NULL, then its output is not written); I_attn, I_mlp fp64 [L] on the device.  The variance is the
+ *   population variance sum w^2 / c - (sum w / c)^2 over the c entries, the l2 norm sqrt(sum w^2).
+ */
+sp_status sp_weight_stats(const sp_mat* W, int32_t axis, int64_t group, int32_t accumulate, double* stats, void* ws,
+                          size_t ws_bytes, void* stream);
+sp_status sp_distribute_importance(const double* head_stats, int32_t n_heads, const double* fc_stats, int32_t n_fc,
+                                   int32_t L, double rho, double gamma, double* I_attn, double* I_mlp, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
  * Helpers.
  * sp_ridge_solve   — W[m,n] = R[m,n] (G[n,n] + rho_eff I)^-1 by Cholesky and two triangular solves (weight
  *                    recovery of Appendix A.1).  G, R, W fp32; factorisation in fp64 when precise != 0, else fp32.
@@ -286,7 +309,8 @@ int64_t sp_launch_count(void);
 /* Bytes of workspace the named call needs.  Meaning of (d, n, N, token_chunk, dtype) per op:
  *   SP_WS_GRAM: d = channels C, N = tokens T.   SP_WS_ADMM_STEP / SP_WS_FFN_INIT: module sizes, dtype of X.
  *   SP_WS_SCORES: d = n_units*group, N = tokens (LEMMA1) or rows of W (WANDA).
- *   SP_WS_RIDGE_SOLVE / SP_WS_LINEAR_REFIT: d = m (rows of R), n = system size, dtype SP_F64 when precise != 0. */
+ *   SP_WS_RIDGE_SOLVE / SP_WS_LINEAR_REFIT: d = m (rows of R), n = system size, dtype SP_F64 when precise != 0.
+ *   SP_WS_WEIGHT_STATS: d = number of blocks. */
 size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t token_chunk, int32_t dtype);
 /* Optional extra workspace of sp_admm_step (bf16 mode): when ws_bytes >= sp_workspace_bytes(SP_WS_ADMM_STEP, ...) +
  * sp_admm_overlap_bytes(N, k_keep), the step keeps z^(1) = W1 X of all N tokens on the kept channels (fp32) in the

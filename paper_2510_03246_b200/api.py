@@ -25,7 +25,8 @@ SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
  SP_WS_RIDGE_SOLVE) = range(8)
 
 EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
-           "sp_apply_mask", "sp_apply_mask_batched", "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
+           "sp_apply_mask", "sp_apply_mask_batched", "sp_weight_stats", "sp_distribute_importance",
+           "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
            "sp_profile_kind_name", "sp_launch_count"]
 
@@ -94,6 +95,8 @@ def lib() -> C.CDLL:
         L.sp_allocate_sparsity.argtypes = [vp, vp, i32, dbl, dbl, i32, dbl, vp, vp, vp]
         L.sp_apply_mask.argtypes = [vp, i64, i64, i32, vp, vp, vp, pm, pm, vp, sz, vp]
         L.sp_apply_mask_batched.argtypes = [vp, i64, i64, i32, vp, vp, i64, vp, vp, i64, vp]
+        L.sp_weight_stats.argtypes = [pm, i32, i64, i32, vp, vp, sz, vp]
+        L.sp_distribute_importance.argtypes = [vp, i32, vp, i32, i32, dbl, dbl, vp, vp, vp]
         L.sp_ridge_solve.argtypes = [vp, i64, vp, i64, i64, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
         L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, vp, i64, vp, vp, sz, vp]
         L.sp_gemm.argtypes = [i32, i32, i64, i64, i64, dbl, pm, pm, dbl, pm, i32, i32, vp, vp]
@@ -312,6 +315,39 @@ def sp_apply_mask_batched(scores, k_keep, want_index=False):
     _check(lib().sp_apply_mask_batched(scores.data_ptr(), scores.stride(0), n, L, k_keep.data_ptr(), mask.data_ptr(), n,
                                        tau.data_ptr(), _ptr(idx), n, _stream()), "sp_apply_mask_batched")
     return mask, tau, idx
+
+
+SP_WS_WEIGHT_STATS = 8
+
+
+def sp_weight_stats(W, axis=0, group=0, stats=None, accumulate=False):
+    """Sums {|w|, w, w^2, count} over row blocks (axis 0) or column blocks (axis 1) of `group` rows / columns of W
+    (group 0: the whole matrix).  Returns stats fp64 [n_blocks, 4]; with accumulate the sums are added to `stats`."""
+    _require_cuda(W, stats)
+    rows, cols = W.shape
+    nb = 1 if group == 0 else (rows // group if axis == 0 else cols // group)
+    if stats is None:
+        stats = torch.zeros(nb, 4, dtype=torch.float64, device=W.device)
+        accumulate = False
+    ws = _ws(workspace_bytes(SP_WS_WEIGHT_STATS, nb, 0, 0), W.device)
+    m = mat(W)
+    _check(lib().sp_weight_stats(C.byref(m), axis, group, int(accumulate), stats.data_ptr(), ws.data_ptr(), ws.numel(),
+                                 _stream()), "sp_weight_stats")
+    return stats
+
+
+def sp_distribute_importance(head_stats, fc_stats, rho, gamma):
+    """head_stats fp64 [L, H, 4] or None, fc_stats fp64 [L, n_fc, 4] or None.  Returns (I_attn [L] or None, I_mlp)."""
+    ref = head_stats if head_stats is not None else fc_stats
+    _require_cuda(head_stats, fc_stats)
+    L = ref.shape[0]
+    Ia = torch.empty(L, dtype=torch.float64, device=ref.device) if head_stats is not None else None
+    Im = torch.empty(L, dtype=torch.float64, device=ref.device) if fc_stats is not None else None
+    _check(lib().sp_distribute_importance(_ptr(head_stats), head_stats.shape[1] if head_stats is not None else 0,
+                                          _ptr(fc_stats), fc_stats.shape[1] if fc_stats is not None else 0, L,
+                                          float(rho), float(gamma), _ptr(Ia), _ptr(Im), _stream()),
+           "sp_distribute_importance")
+    return Ia, Im
 
 
 # ---------------------------------------------------------------------------------------------- module driver

@@ -357,6 +357,7 @@ size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t t
     case SP_WS_LINEAR_REFIT: return ridge_ws_bytes(d, n, dtype == SP_F64) + align_up((size_t)(n > 0 ? n : 1) * 4, 256) + 512;
     case SP_WS_RIDGE_SOLVE: return ridge_ws_bytes(d, n, dtype == SP_F64) + 256;
     case SP_WS_GEMM: return 256;
+    case SP_WS_WEIGHT_STATS: return align_up((size_t)(148 * 8 + (d > 0 ? d : 1)) * 3 * sizeof(double), 256) + 256;
     default: return 0;
   }
 }
@@ -548,6 +549,30 @@ sp_status sp_apply_mask_batched(const float* scores, int64_t ld_scores, int64_t 
   if (n_units == 0 || L == 0) return SP_OK;
   CU(topk_select_batched(scores, ld_scores, n_units, L, 0, k_keep, mask_out, ld_mask, tau_out, kept_idx_out, ld_idx,
                          reinterpret_cast<cudaStream_t>(stream)));
+  return SP_OK;
+}
+
+sp_status sp_weight_stats(const sp_mat* W, int32_t axis, int64_t group, int32_t accumulate, double* stats, void* ws,
+                          size_t ws_bytes, void* stream) {
+  if (!W || !W->ptr || !stats || (axis != 0 && axis != 1)) return SP_ERR_INVALID_ARG;
+  if (W->dtype != SP_F32 && W->dtype != SP_BF16) return SP_ERR_DTYPE;
+  if (W->rows < 0 || W->cols < 0 || W->ld < W->cols || group < 0) return SP_ERR_SHAPE;
+  if (group > 0 && (axis == 0 ? W->rows % group : W->cols % group) != 0) return SP_ERR_SHAPE;
+  if (W->rows == 0 || W->cols == 0) return SP_OK;
+  const int64_t n_blocks = group > 0 ? (axis == 0 ? W->rows / group : W->cols / group) : 1;
+  if (!ws || ws_bytes < sp_workspace_bytes(SP_WS_WEIGHT_STATS, n_blocks, 0, 0, 0, 0)) return SP_ERR_WORKSPACE;
+  CU(weight_stats(W->ptr, W->dtype, W->ld, W->rows, W->cols, axis, group, accumulate != 0, stats,
+                  reinterpret_cast<double*>(align_up(reinterpret_cast<uintptr_t>(ws), 256)),
+                  reinterpret_cast<cudaStream_t>(stream)));
+  return SP_OK;
+}
+
+sp_status sp_distribute_importance(const double* head_stats, int32_t n_heads, const double* fc_stats, int32_t n_fc,
+                                   int32_t L, double rho, double gamma, double* I_attn, double* I_mlp, void* stream) {
+  if (L < 0 || n_heads < 0 || n_fc < 0) return SP_ERR_SHAPE;
+  if ((head_stats && !I_attn) || (fc_stats && !I_mlp) || (!head_stats && !fc_stats)) return SP_ERR_INVALID_ARG;
+  CU(distribute_importance(head_stats, n_heads, fc_stats, n_fc, L, rho, gamma, I_attn, I_mlp,
+                           reinterpret_cast<cudaStream_t>(stream)));
   return SP_OK;
 }
 

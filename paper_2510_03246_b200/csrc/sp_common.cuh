@@ -139,6 +139,12 @@ cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64
 int column_stats_row_blocks(int64_t T, int64_t C);
 int score_row_blocks(int64_t rows, int64_t cols);
 size_t wanda_scratch_doubles(int64_t rows, int64_t cols);
+// weight statistics of the "-distribute" importances (sp_mask.cu); scratch: (148 * 8 + n_blocks) * 3 doubles
+int weight_stats_parts(int64_t n_blocks, int64_t block_rows);
+cudaError_t weight_stats(const void* W, int32_t dt, int64_t ld, int64_t rows, int64_t cols, int axis, int64_t group,
+                         bool accumulate, double* stats, double* scratch, cudaStream_t stream);
+cudaError_t distribute_importance(const double* head_stats, int n_heads, const double* fc_stats, int n_fc, int L,
+                                  double rho, double gamma, double* I_attn, double* I_mlp, cudaStream_t stream);
 // dst[i,j] = (T) G[i*ld + j] (+ rho on the diagonal) for the lower triangle; rho read from device (rho_dev[0]).
 template <typename T>
 cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_dev, T* dst, int64_t ldd,

@@ -209,6 +209,146 @@ __global__ void __launch_bounds__(kWsWarps * 32) wanda_scores_kernel(
   }
 }
 
+// ------------------------------------------------------------------------------------------------ weight statistics
+// Sums {|w|, w, w^2} over rectangular slices of a weight matrix (Algorithm "-distribute", Step 1).
+//   grid (blocks, parts): block b is the rectangle rows [r0, r1) x columns [c0, c1); its rows are cut into `parts`
+//   ranges, one CTA each.  Threads walk the CTA's range row-major in 16-byte pieces (scalars when the slice is not
+//   16-byte aligned), eight loads in flight each; fp32 sums over the 32 or 64 values of a round, fp64 running sums,
+//   fixed-order block reduction -> part[b][p][3].
+template <typename T>
+struct StatVec;
+template <>
+struct StatVec<float> {
+  static constexpr int V = 4;
+  typedef float4 Raw;
+  __device__ static Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+  __device__ static float get(const Raw& v, int j) { return j == 0 ? v.x : j == 1 ? v.y : j == 2 ? v.z : v.w; }
+};
+template <>
+struct StatVec<__nv_bfloat16> {
+  static constexpr int V = 8;
+  typedef uint4 Raw;
+  __device__ static Raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
+  __device__ static float get(const Raw& v, int j) {
+    const uint32_t w = (j >> 1) == 0 ? v.x : (j >> 1) == 1 ? v.y : (j >> 1) == 2 ? v.z : v.w;
+    return __uint_as_float((j & 1) ? (w & 0xffff0000u) : (w << 16));
+  }
+};
+__device__ __forceinline__ float stat_scalar(const float* p) { return *p; }
+__device__ __forceinline__ float stat_scalar(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+constexpr int kStatInFlight = 8;     // 16-byte loads a thread keeps in flight
+
+template <typename T>
+__global__ void __launch_bounds__(256, 4) weight_stats_partial_kernel(const T* __restrict__ W, int64_t ld,
+                                                                      int64_t rows, int64_t cols, int axis,
+                                                                      int64_t group, int vec_ok, double* part) {
+  typedef typename StatVec<T>::Raw Raw;
+  constexpr int V = StatVec<T>::V;
+  __shared__ double sm[33];
+  const int64_t b = blockIdx.x;
+  const int parts = (int)gridDim.y;
+  int64_t r0 = 0, r1 = rows, c0 = 0, c1 = cols;
+  if (group > 0) {
+    if (axis == 0) { r0 = b * group; r1 = r0 + group; }
+    else { c0 = b * group; c1 = c0 + group; }
+  }
+  const int64_t rows_per = ceil_div(r1 - r0, (int64_t)parts);
+  const int64_t pr0 = r0 + (int64_t)blockIdx.y * rows_per;
+  const int64_t pr1 = (pr0 + rows_per < r1) ? pr0 + rows_per : r1;
+  const int64_t width = c1 - c0;
+  double s_abs = 0.0, s_sum = 0.0, s_sq = 0.0;
+  if (pr0 < pr1) {
+    if (vec_ok && width % V == 0) {
+      const int64_t nq = width / V, total = (pr1 - pr0) * nq;
+      for (int64_t e0 = threadIdx.x; e0 < total; e0 += (int64_t)blockDim.x * kStatInFlight) {
+        Raw raw[kStatInFlight];
+#pragma unroll
+        for (int q = 0; q < kStatInFlight; ++q) {
+          const int64_t e = e0 + (int64_t)q * blockDim.x;
+          raw[q] = e < total ? *reinterpret_cast<const Raw*>(W + (pr0 + e / nq) * ld + c0 + (e % nq) * V)
+                             : StatVec<T>::zero();
+        }
+        // the values of this round are summed in fp32 (32 or 64 terms), the running sums are fp64: the fp64 pipe is
+        // narrow, and one conversion per value would make this kernel compute-bound
+        float fa = 0.f, fs = 0.f, fq = 0.f;
+#pragma unroll
+        for (int q = 0; q < kStatInFlight; ++q)
+#pragma unroll
+          for (int j = 0; j < V; ++j) {
+            const float x = StatVec<T>::get(raw[q], j);
+            fa += fabsf(x);
+            fs += x;
+            fq = fmaf(x, x, fq);
+          }
+        s_abs += (double)fa;
+        s_sum += (double)fs;
+        s_sq += (double)fq;
+      }
+    } else {
+      const int64_t total = (pr1 - pr0) * width;
+      for (int64_t e = threadIdx.x; e < total; e += blockDim.x) {
+        const double x = (double)stat_scalar(W + (pr0 + e / width) * ld + c0 + e % width);
+        s_abs += fabs(x);
+        s_sum += x;
+        s_sq = fma(x, x, s_sq);
+      }
+    }
+  }
+  s_abs = block_sum_bcast(s_abs, sm);
+  s_sum = block_sum_bcast(s_sum, sm);
+  s_sq = block_sum_bcast(s_sq, sm);
+  if (threadIdx.x == 0) {
+    double* o = part + (b * parts + blockIdx.y) * 3;
+    o[0] = s_abs; o[1] = s_sum; o[2] = s_sq;
+  }
+}
+
+// one CTA per block: the parts are added in a fixed order (strided over the threads, then the block tree)
+__global__ void __launch_bounds__(128) weight_stats_finish_kernel(const double* part, int parts, double count,
+                                                                  int accumulate, double* stats) {
+  __shared__ double sm[33];
+  const int64_t b = blockIdx.x;
+  double s[3] = {0.0, 0.0, 0.0};
+  for (int p = threadIdx.x; p < parts; p += blockDim.x)
+#pragma unroll
+    for (int j = 0; j < 3; ++j) s[j] += part[(b * parts + p) * 3 + j];
+#pragma unroll
+  for (int j = 0; j < 3; ++j) s[j] = block_sum_bcast(s[j], sm);
+  if (threadIdx.x == 0) {
+    double* o = stats + b * 4;
+    if (accumulate) { o[0] += s[0]; o[1] += s[1]; o[2] += s[2]; o[3] += count; }
+    else { o[0] = s[0]; o[1] = s[1]; o[2] = s[2]; o[3] = count; }
+  }
+}
+
+// One thread per layer: I_attn[l] = gamma^(l+1) rho sum_h (l1 + 0.1 var + 0.01 l2), I_mlp[l] = gamma^(l+1) sum_m
+// (l1 + 0.05 var), from {sum |w|, sum w, sum w^2, count} per head / per matrix.
+__global__ void distribute_importance_kernel(const double* head_stats, int n_heads, const double* fc_stats, int n_fc,
+                                             int L, double rho, double gamma, double* I_attn, double* I_mlp) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= L) return;
+  const double dl = pow(gamma, (double)(l + 1));
+  if (head_stats && I_attn) {
+    double acc = 0.0;
+    for (int h = 0; h < n_heads; ++h) {
+      const double* s = head_stats + ((int64_t)l * n_heads + h) * 4;
+      const double c = s[3] > 0.0 ? s[3] : 1.0, mean = s[1] / c;
+      acc += s[0] + 0.1 * (s[2] / c - mean * mean) + 0.01 * sqrt(s[2]);
+    }
+    I_attn[l] = dl * rho * acc;
+  }
+  if (fc_stats && I_mlp) {
+    double acc = 0.0;
+    for (int q = 0; q < n_fc; ++q) {
+      const double* s = fc_stats + ((int64_t)l * n_fc + q) * 4;
+      const double c = s[3] > 0.0 ? s[3] : 1.0, mean = s[1] / c;
+      acc += s[0] + 0.05 * (s[2] / c - mean * mean);
+    }
+    I_mlp[l] = dl * acc;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ Lemma 1
 __global__ void lemma1_partials_kernel(sp_mat b, sp_mat c, sp_mat dd, sp_mat t, int64_t N, int64_t cols,
                                        int row_blocks, double* part) {
@@ -738,6 +878,52 @@ cudaError_t wanda_scores(int kind, int group, const float* W, int64_t rows, int6
   wanda_scores_kernel<<<dim3((unsigned)cg, (unsigned)rb), kWsWarps * 32, 0, stream>>>(
       W, rows, cols, ldw, vec_ok, k, group, colsq, colsq_stride, colabs, inv_tokens, n_units, scores, importance, part,
       colval, tickets);
+  return cudaGetLastError();
+}
+
+// parts of a block's row range so that the launch has about 148 * 8 CTAs
+int weight_stats_parts(int64_t n_blocks, int64_t block_rows) {
+  int64_t parts = (148 * 8) / (n_blocks > 0 ? n_blocks : 1);
+  if (parts > block_rows) parts = block_rows;
+  if (parts < 1) parts = 1;
+  if (parts > 1024) parts = 1024;
+  return (int)parts;
+}
+
+cudaError_t weight_stats(const void* W, int32_t dt, int64_t ld, int64_t rows, int64_t cols, int axis, int64_t group,
+                         bool accumulate, double* stats, double* scratch, cudaStream_t stream) {
+  const int64_t n_blocks = group > 0 ? (axis == 0 ? rows / group : cols / group) : 1;
+  if (n_blocks <= 0 || rows <= 0 || cols <= 0) return cudaSuccess;
+  const int64_t block_rows = (group > 0 && axis == 0) ? group : rows;
+  const int64_t block_cols = (group > 0 && axis == 1) ? group : cols;
+  const int parts = weight_stats_parts(n_blocks, block_rows);
+  const size_t esz = dt == SP_BF16 ? 2 : 4;
+  // 16-byte pieces need aligned rows and an aligned first column of every block
+  const int64_t V = 16 / (int64_t)esz;
+  const bool vec_ok = (ld % V == 0) && ((reinterpret_cast<uintptr_t>(W) & 15u) == 0) && (block_cols % V == 0) &&
+                      (group == 0 || axis == 0 || group % V == 0);
+  ProfScope prof(PK_SCORES, 0.0, (double)rows * (double)cols * (double)esz, stream);
+  count_launch();
+  const dim3 grid((unsigned)n_blocks, (unsigned)parts);
+  if (dt == SP_BF16)
+    weight_stats_partial_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(W), ld,
+                                                                         rows, cols, axis, group, vec_ok ? 1 : 0,
+                                                                         scratch);
+  else
+    weight_stats_partial_kernel<float><<<grid, 256, 0, stream>>>(reinterpret_cast<const float*>(W), ld, rows, cols, axis,
+                                                                 group, vec_ok ? 1 : 0, scratch);
+  count_launch();
+  weight_stats_finish_kernel<<<(unsigned)n_blocks, 128, 0, stream>>>(
+      scratch, parts, (double)block_rows * (double)block_cols, accumulate ? 1 : 0, stats);
+  return cudaGetLastError();
+}
+
+cudaError_t distribute_importance(const double* head_stats, int n_heads, const double* fc_stats, int n_fc, int L,
+                                  double rho, double gamma, double* I_attn, double* I_mlp, cudaStream_t stream) {
+  if (L <= 0) return cudaSuccess;
+  count_launch();
+  distribute_importance_kernel<<<(unsigned)ceil_div((int64_t)L, (int64_t)128), 128, 0, stream>>>(
+      head_stats, n_heads, fc_stats, n_fc, L, rho, gamma, I_attn, I_mlp);
   return cudaGetLastError();
 }
 

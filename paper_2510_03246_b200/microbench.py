@@ -125,6 +125,16 @@ def mask_cases(reps, warm, hbm_gbs):
                           warm, flush)
         line(f"scores Lemma-1 streamed  4 x [{N}, {n}] {str(dt)[6:]}", ms, 4.0 * N * n * sz)
         del b, c, dd, t
+    # weight statistics of the "-distribute" importances: head slices (rows of W_Q, columns of W_O) and whole MLP matrices
+    for rows, cols, axis, group, dt, sz in ((4096, 4096, 0, 128, torch.bfloat16, 2), (4096, 4096, 1, 128, torch.bfloat16, 2),
+                                            (16384, 4096, 0, 0, torch.bfloat16, 2), (28672, 7168, 0, 0, torch.bfloat16, 2),
+                                            (16384, 4096, 0, 0, torch.float32, 4)):
+        W = _rnd((rows, cols), dt)
+        nb = 1 if group == 0 else (rows // group if axis == 0 else cols // group)
+        st = torch.zeros(nb, 4, dtype=torch.float64, device=DEV)
+        ms = _timeit_cold(lambda: api.sp_weight_stats(W, axis, group, st, accumulate=True), reps, warm, flush)
+        line(f"weight stats  W [{rows}, {cols}] {str(dt)[6:]}, axis {axis}, blocks of {group}", ms, float(sz) * rows * cols)
+        del W
     # allocation over the layers of a model
     for L in (24, 32, 64):
         I = torch.rand(L, dtype=torch.float64, device=DEV) + 0.5

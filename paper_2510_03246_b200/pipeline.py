@@ -6,6 +6,9 @@ built from the library calls only (argument marshalling and loop control; all ar
     Step 3/4 per-module ADMM             sp_admm_step x K with the layer's kept count
     Step 5  loss L(T) = sum_l L_l        the module objectives reported by the last step (temperature_search)
 
+plan_distribute covers Steps 1 and 2 of the "-distribute" variant (importances from weight statistics, attention and
+MLP modules allocated separately by inverse weighting).
+
 One module is resident at a time (the paper's memory argument), so a layer is initialised twice: once for its
 importance, once for its ADMM loop.  With several ranks each rank owns the layers `parallel.layers_of_rank` gives it;
 the only exchange is the vector of importances before Step 2.
@@ -88,6 +91,33 @@ def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_unit
     torch.cuda.synchronize()
     t2 = time.perf_counter()
     return results, r, k_keep, {"importance_s": t1 - t0, "admm_s": t2 - t1, "layers_per_s": len(mine) / max(t2 - t0, 1e-9)}
+
+
+def plan_distribute(layer_weights: Callable[[int], dict], n_layers: int, n_heads: int, n_ffn: int, rbar: float,
+                    T_rel: float = 1.0, rho: float = 1.0, gamma: float = 1.0, device="cuda"):
+    """Steps 1 and 2 of the "-distribute" variant of Algorithm 1: importances of the attention and MLP modules from
+    weight statistics (with depth decay gamma^l and the attention/MLP ratio rho), normalised separately, turned into
+    pruned fractions by the inverse weighting.  layer_weights(l) returns dict(Wq, Wk, Wv, Wo, fc1, fc2) on the device
+    for layer l (one layer resident at a time).  Returns dict(I_attn, I_mlp, r_attn, r_mlp, k_heads, k_channels)."""
+    head_stats = torch.zeros(n_layers, n_heads, 4, dtype=torch.float64, device=device)
+    fc_stats = torch.zeros(n_layers, 2, 4, dtype=torch.float64, device=device)
+    for l in range(n_layers):
+        w = layer_weights(l)
+        d_head = w["Wq"].shape[0] // n_heads
+        for name in ("Wq", "Wk", "Wv"):            # head h = rows [h d_head, (h + 1) d_head)
+            api.sp_weight_stats(w[name], 0, d_head, head_stats[l], accumulate=True)
+        api.sp_weight_stats(w["Wo"], 1, d_head, head_stats[l], accumulate=True)   # and the same columns of W_O
+        api.sp_weight_stats(w["fc1"], 0, 0, fc_stats[l, 0:1])
+        api.sp_weight_stats(w["fc2"], 0, 0, fc_stats[l, 1:2])
+    I_attn, I_mlp = api.sp_distribute_importance(head_stats, fc_stats, rho, gamma)
+    out = {"I_attn": I_attn, "I_mlp": I_mlp}
+    for key, I, units in (("attn", I_attn, n_heads), ("mlp", I_mlp, n_ffn)):
+        T = T_rel * float(I.abs().mean())
+        nu = torch.full((n_layers,), units, dtype=torch.int64, device=device)
+        r, k = api.sp_allocate_sparsity(I, nu, rbar, T, api.SP_ALLOC_INVERSE)
+        out["r_" + key] = r
+        out["k_heads" if key == "attn" else "k_channels"] = k
+    return out
 
 
 def module_loss(res: LayerResult, beta: float) -> float:
