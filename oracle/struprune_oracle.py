@@ -87,18 +87,22 @@ def restricted_refit(R, G, keep, rho_eff):
 # --------------------------------------------------------------------------------------------------
 # Activation, a-update, z-update (Appendix A.1; Algorithm 3 lines for a_l, z^(1), z^(2), select)
 # --------------------------------------------------------------------------------------------------
-def phi(Z, act="relu"):
+def phi(Z, act="relu", gate=None):
+    """Activation of the module: ReLU (the paper's case), or the gated form g * z of the SwiGLU extension, where
+    g = SiLU(gate pre-activation) is a fixed factor per entry (see the SwiGLU section below)."""
     Z = np.asarray(Z, F64)
     if act == "relu":
         return np.maximum(Z, 0.0)
+    if act == "swiglu":
+        return np.asarray(gate, F64) * Z
     raise ValueError(act)
 
 
-def a_update(W2, Ypre, Z, alpha, beta, U=None, act="relu"):
+def a_update(W2, Ypre, Z, alpha, beta, U=None, act="relu", gate=None):
     """a_l = (alpha W2^T W2 + beta I)^-1 (alpha W2^T Ypre + beta (phi(z_l) - U))."""
     W2 = np.asarray(W2, F64)
     n = W2.shape[1]
-    H = phi(Z, act) - (0.0 if U is None else np.asarray(U, F64))
+    H = phi(Z, act, gate) - (0.0 if U is None else np.asarray(U, F64))
     lhs = alpha * (W2.T @ W2) + beta * np.eye(n)
     rhs = alpha * (W2.T @ np.asarray(Ypre, F64)) + beta * H
     return np.linalg.solve(lhs, rhs)
@@ -136,9 +140,9 @@ def z_select(Zold, z1, z2, A, alpha, beta, rule="paper", U=None):
     raise ValueError(rule)
 
 
-def dual_update(U, A, Znew, act="relu"):
+def dual_update(U, A, Znew, act="relu", gate=None):
     """Scaled dual ascent on a = phi(z) (not in the paper; see header)."""
-    return np.asarray(U, F64) + np.asarray(A, F64) - phi(Znew, act)
+    return np.asarray(U, F64) + np.asarray(A, F64) - phi(Znew, act, gate)
 
 
 # --------------------------------------------------------------------------------------------------
@@ -326,6 +330,7 @@ class FfnState:
     W2: np.ndarray | None = None
     mask: np.ndarray | None = None
     it: int = 0
+    gate: np.ndarray | None = None   # SwiGLU extension: g = SiLU(Wg X), fixed over the iterations
 
 
 def ffn_init(X, W1_0, W2_0, act="relu", dual_mode=False):
@@ -381,13 +386,16 @@ def admm_step(st, X, Ypre, W1_0, p, z_hook=None):
     N = X.shape[1]
     s, I = admm_weight_phase(st, W1_0, p, N)
     U = st.U if p.dual_mode else None
-    A = a_update(st.W2, Ypre, st.Z, p.alpha, p.beta, U, p.act)
+    A = a_update(st.W2, Ypre, st.Z, p.alpha, p.beta, U, p.act, st.gate)
     z1, z2 = z_candidates(st.W1, X, A, p.alpha, p.beta, U)
-    Znew = z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule, U)
+    if p.act == "swiglu":
+        Znew = swiglu_zu_update(A, st.gate, z1, p.alpha, p.beta, U)    # one closed form, no select
+    else:
+        Znew = z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule, U)
     if z_hook is not None:
         Znew = z_hook(Znew, z1, z2, A, U)
     if p.dual_mode:
-        st.U = dual_update(st.U, A, Znew, p.act)
+        st.U = dual_update(st.U, A, Znew, p.act, st.gate)
     st.Z = Znew
     st.G_A = A @ A.T
     st.R1 = Znew @ X.T
@@ -395,27 +403,46 @@ def admm_step(st, X, Ypre, W1_0, p, z_hook=None):
     st.absA = np.abs(A).sum(axis=1)
     st.it += 1
     rep = {
-        "res_act": float(((A - phi(Znew, p.act)) ** 2).sum()),
+        "res_act": float(((A - phi(Znew, p.act, st.gate)) ** 2).sum()),
         "res_out": float(p.alpha * ((Ypre - st.W2 @ A) ** 2).sum()),
         "res_in": float(p.alpha * ((Znew - st.W1 @ X) ** 2).sum()),
     }
     return s, I, rep, A
 
 
-def ffn_objective(st_W1, st_W2, X, Ypre, Z, A, alpha, beta, act="relu"):
+def ffn_objective(st_W1, st_W2, X, Ypre, Z, A, alpha, beta, act="relu", gate=None):
     """alpha |Ypre - W2 A|^2 + beta |A - phi(Z)|^2 + alpha |Z - W1 X|^2 (Appendix A.1, FFN objective)."""
     X = np.asarray(X, F64)
     return (alpha * ((np.asarray(Ypre, F64) - st_W2 @ A) ** 2).sum()
-            + beta * ((A - phi(Z, act)) ** 2).sum()
+            + beta * ((A - phi(Z, act, gate)) ** 2).sum()
             + alpha * ((Z - st_W1 @ X) ** 2).sum())
 
 
 # --------------------------------------------------------------------------------------------------
-# SwiGLU extension (not in the paper; parity unpinned)
+# SwiGLU extension (not in the paper: its modules are ReLU FFNs).  Parity unpinned against the paper; what pins
+# it is the mathematics of the subproblems it solves (stationarity, monotone descent, the g = 1 special case).
+#   module: y = W2 (SiLU(Wg x) * (Wu x)).  Only the "up" branch is split: Z = z_u with Z ~ Wu X, A ~ g * Z, where
+#   g = SiLU(Wg_0 X) is computed once from the pre-trained gate and kept fixed; the gate weights are only row-masked.
+#   With g fixed, phi(z) = g z is linear, so every subproblem of the FFN objective of Appendix A.1 keeps its closed
+#   form: the weight recoveries and the a-update are unchanged (phi(Z) = g Z), the z-update is one quadratic.
 # --------------------------------------------------------------------------------------------------
 def silu(x):
     x = np.asarray(x, F64)
     return x / (1.0 + np.exp(-x))
+
+
+def swiglu_init(X, Wg_0, Wu_0, W2_0, dual_mode=False):
+    """Initialisation of a SwiGLU module: g = SiLU(Wg_0 X) (fixed), Z = Wu_0 X, A = g Z, Ypre = W2_0 A, and the
+    accumulators of the first weight recovery.  Returns (state with .gate = g, Ypre)."""
+    X = np.asarray(X, F64)
+    g = silu(np.asarray(Wg_0, F64) @ X)
+    Zpre = np.asarray(Wu_0, F64) @ X
+    Apre = g * Zpre
+    Ypre = np.asarray(W2_0, F64) @ Apre
+    st = FfnState(
+        Z=Zpre.copy(), U=np.zeros_like(Zpre) if dual_mode else None,
+        G_X=X @ X.T, G_A=Apre @ Apre.T, R1=Zpre @ X.T, R2=Ypre @ Apre.T, absA=np.abs(Apre).sum(axis=1), gate=g)
+    return st, Ypre
 
 
 def swiglu_zu_update(A, g, z1u, alpha, beta, U=None):

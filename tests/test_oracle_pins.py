@@ -459,6 +459,50 @@ def test_swiglu_zu_is_stationary_point():
     assert np.allclose(O.silu(np.array([0.0, 1.0])), [0.0, 1.0 / (1.0 + np.exp(-1.0))])
 
 
+def test_swiglu_module_special_cases_and_descent():
+    """The SwiGLU extension against what the mathematics fixes: with a gate factor of one it is the paper's linear
+    branch (z-update = z^(2)), its initial state reproduces the pre-trained module, and with a fixed mask every
+    sub-step solves its subproblem exactly, so the FFN objective of Appendix A.1 cannot rise."""
+    r = _rng(31)
+    d, n, N = 5, 9, 60
+    X = r.normal(size=(d, N)); Wg = 0.7 * r.normal(size=(n, d)); Wu = 0.7 * r.normal(size=(n, d))
+    W2 = 0.7 * r.normal(size=(d, n))
+    # gate factor one: the closed form is z^(2) of "Updating output", duals included
+    A = r.normal(size=(n, N)); U = r.normal(size=(n, N)); W1 = r.normal(size=(n, d))
+    z1, z2 = O.z_candidates(W1, X, A, 0.8, 1.3, U)
+    assert np.allclose(O.swiglu_zu_update(A, np.ones_like(A), z1, 0.8, 1.3, U), z2, atol=1e-13)
+    # initial state: the split variables reproduce the module output exactly, token by token
+    st, Ypre = O.swiglu_init(X, Wg, Wu, W2)
+    for t in (0, 17, N - 1):
+        x = X[:, t]
+        zg = Wg @ x
+        want = W2 @ ((zg / (1.0 + np.exp(-zg))) * (Wu @ x))
+        assert np.allclose(Ypre[:, t], want, atol=1e-12)
+    assert np.allclose(st.gate * st.Z, O.phi(st.Z, "swiglu", st.gate)) and np.allclose(st.R1, st.Z @ X.T)
+    # first step without pruning and a vanishing ridge: the recovered weights are the pre-trained ones, nothing moves
+    p = O.AdmmParams(k_keep=n, rho=1e-12, rho_relative=False, act="swiglu")
+    st0, _ = O.swiglu_init(X, Wg, Wu, W2)
+    _, _, rep, A0 = O.admm_step(st0, X, Ypre, Wu, p)
+    assert np.allclose(st0.W1, Wu, atol=1e-6) and np.allclose(st0.W2, W2, atol=1e-6)
+    assert rep["res_act"] < 1e-12 and rep["res_in"] < 1e-12 and rep["res_out"] < 1e-12
+    # block descent with a fixed mask (the ridge is part of what the recoveries minimise, so keep it negligible)
+    p = O.AdmmParams(k_keep=6, rho=1e-10, rho_relative=False, act="swiglu", reselect_mask=True)
+    st, _ = O.swiglu_init(X, Wg, Wu, W2)
+    prev = None
+    for it in range(8):
+        _, _, _, A = O.admm_step(st, X, Ypre, Wu, p)
+        p.reselect_mask = False
+        obj = O.ffn_objective(st.W1, st.W2, X, Ypre, st.Z, A, p.alpha, p.beta, "swiglu", st.gate)
+        if prev is not None:
+            assert obj <= prev * (1 + 1e-9), (it, obj, prev)
+        prev = obj
+    assert int(st.mask.sum()) == 6 and np.all(st.W1[st.mask == 0] == 0) and np.all(st.W2[:, st.mask == 0] == 0)
+    # stationarity of the a-update with the gated activation
+    Ares = O.a_update(st.W2, Ypre, st.Z, 0.9, 1.2, None, "swiglu", st.gate)
+    grad = -2 * 0.9 * st.W2.T @ (Ypre - st.W2 @ Ares) + 2 * 1.2 * (Ares - st.gate * st.Z)
+    assert np.abs(grad).max() < 1e-9
+
+
 def test_weight_stats_closed_forms():
     """Algorithm "-distribute" Step 1 statistics against textbook closed forms: the entries 0, 1, ..., m-1 have
     l1 = m(m-1)/2, variance (m^2-1)/12 and sum of squares (m-1)m(2m-1)/6, however they are cut into slices."""
