@@ -52,7 +52,7 @@ typedef enum {
 } sp_status;
 
 typedef enum { SP_F32 = 0, SP_BF16 = 1, SP_F64 = 2 } sp_dtype;
-typedef enum { SP_ACT_RELU = 0 } sp_act_kind;
+typedef enum { SP_ACT_RELU = 0, SP_ACT_SWIGLU = 1 } sp_act_kind;
 typedef enum { SP_Z_PAPER = 0, SP_Z_EXACT = 1 } sp_z_rule;
 typedef enum { SP_SCORE_WANDA_L2 = 0, SP_SCORE_WANDA_L1 = 1, SP_SCORE_LEMMA1 = 2 } sp_score_kind;
 typedef enum { SP_ALLOC_SOFTMAX = 0, SP_ALLOC_INVERSE = 1, SP_ALLOC_UNIFORM = 2 } sp_alloc_mode;
@@ -76,7 +76,15 @@ typedef struct {
   int64_t d, n, N;
   int32_t act; /* sp_act_kind */
   int32_t reserved;
+  sp_mat Wg_0; /* [n, d]  SP_ACT_SWIGLU only: pre-trained gate projection, fp32 (used by sp_ffn_init only)        */
 } sp_ffn_module;
+
+/* SP_ACT_SWIGLU is an extension: the paper's modules are ReLU FFNs.  The module is y = W2 (SiLU(Wg x) * (W1 x)); only
+ * the "up" branch is split (Z ~ W1 X, A ~ g * Z) and the gate factor g = SiLU(Wg_0 X) is computed once by sp_ffn_init
+ * into st->Gate and kept fixed, so phi(z) = g z is linear and every subproblem of the FFN objective keeps a closed
+ * form: the recoveries and the a-update are those of the paper with phi(Z) = g Z, and the z-update is the single
+ * quadratic minimiser Z = (beta g (A + U) + alpha z1) / (beta g^2 + alpha) (z_rule is not used).  The gate weights
+ * are not recovered; the caller masks their rows with st->mask.  SP_SCORE_LEMMA1 is not available for this kind. */
 
 /* ADMM state of one FFN module; every buffer is caller-owned device memory. */
 typedef struct {
@@ -92,6 +100,7 @@ typedef struct {
   float* scores;   /* [n]             out: unit scores of this step                                              */
   uint8_t* mask;   /* [n]             in/out: 1 = kept                                                           */
   double* importance; /* [1]          out: layer importance I_l = mean_j s_j                                      */
+  float* Gate;     /* [N, n] ld = n   SP_ACT_SWIGLU only: g = SiLU(Wg_0 X), written by sp_ffn_init, then read-only   */
 } sp_ffn_state;
 
 typedef struct {

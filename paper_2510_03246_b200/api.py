@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsp.so")
 
 SP_OK = 0
 SP_F32, SP_BF16, SP_F64 = 0, 1, 2
-SP_ACT_RELU = 0
+SP_ACT_RELU, SP_ACT_SWIGLU = 0, 1
 SP_Z_PAPER, SP_Z_EXACT = 0, 1
 SP_SCORE_WANDA_L2, SP_SCORE_WANDA_L1, SP_SCORE_LEMMA1 = 0, 1, 2
 SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
@@ -44,13 +44,13 @@ class SpMat(C.Structure):
 
 class SpFfnModule(C.Structure):
     _fields_ = [("X", SpMat), ("Ypre", SpMat), ("W1_0", SpMat), ("W2_0", SpMat), ("d", C.c_int64), ("n", C.c_int64),
-                ("N", C.c_int64), ("act", C.c_int32), ("reserved", C.c_int32)]
+                ("N", C.c_int64), ("act", C.c_int32), ("reserved", C.c_int32), ("Wg_0", SpMat)]
 
 
 class SpFfnState(C.Structure):
     _fields_ = [("Z", C.c_void_p), ("U", C.c_void_p), ("G_X", C.c_void_p), ("G_A", C.c_void_p), ("R1", C.c_void_p),
                 ("R2", C.c_void_p), ("absA", C.c_void_p), ("W1", C.c_void_p), ("W2", C.c_void_p),
-                ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p)]
+                ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p), ("Gate", C.c_void_p)]
 
 
 class SpAdmmParams(C.Structure):
@@ -376,10 +376,11 @@ class FfnModule:
     """Owns the device buffers of one FFN module and forwards to sp_ffn_init / sp_admm_step."""
 
     def __init__(self, X: torch.Tensor, W1_0: torch.Tensor, W2_0: torch.Tensor, dual_mode: bool = False,
-                 token_chunk: int = 0, overlap_k: int = 0):
+                 token_chunk: int = 0, overlap_k: int = 0, Wg_0: torch.Tensor | None = None):
         """overlap_k > 0: also reserve the optional workspace tail that lets sp_admm_step compute z1 of all tokens
-        beside the kept-support recovery, sized for overlap_k kept units (see sp_admm_overlap_bytes)."""
-        _require_cuda(X, W1_0, W2_0)
+        beside the kept-support recovery, sized for overlap_k kept units (see sp_admm_overlap_bytes).
+        Wg_0 (gate projection [n, d]) makes the module a SwiGLU one: W1_0 is then its up projection."""
+        _require_cuda(X, W1_0, W2_0, Wg_0)
         assert X.dtype in (torch.float32, torch.bfloat16)
         self.X = X.contiguous()
         self.N, self.d = X.shape
@@ -388,8 +389,11 @@ class FfnModule:
         self.dev = dev
         self.W1_0 = W1_0.to(torch.float32).contiguous()
         self.W2_0 = W2_0.to(torch.float32).contiguous()
+        self.Wg_0 = Wg_0.to(torch.float32).contiguous() if Wg_0 is not None else None
+        self.act = SP_ACT_SWIGLU if Wg_0 is not None else SP_ACT_RELU
         N, d, n = self.N, self.d, self.n
         f32 = dict(dtype=torch.float32, device=dev)
+        self.Gate = torch.empty(N, n, **f32) if Wg_0 is not None else None
         self.Ypre = torch.empty(N, d, dtype=X.dtype, device=dev)
         self.Z = torch.empty(N, n, **f32)
         self.U = torch.zeros(N, n, **f32) if dual_mode else None
@@ -412,13 +416,13 @@ class FfnModule:
 
     def _module(self) -> SpFfnModule:
         return SpFfnModule(mat(self.X), mat(self.Ypre), mat(self.W1_0), mat(self.W2_0), self.d, self.n, self.N,
-                           SP_ACT_RELU, 0)
+                           self.act, 0, mat(self.Wg_0))
 
     def _state(self) -> SpFfnState:
         return SpFfnState(self.Z.data_ptr(), _ptr(self.U), self.G_X.data_ptr(), self.G_A.data_ptr(),
                           self.R1.data_ptr(), self.R2.data_ptr(), self.absA.data_ptr(), self.W1.data_ptr(),
                           self.W2.data_ptr(), self.scores.data_ptr(), self.mask.data_ptr(),
-                          self.importance.data_ptr())
+                          self.importance.data_ptr(), _ptr(self.Gate))
 
     def _workspace(self, chunk: int) -> torch.Tensor:
         need = max(workspace_bytes(SP_WS_ADMM_STEP, self.d, self.n, self.N, chunk, _dt(self.X)),

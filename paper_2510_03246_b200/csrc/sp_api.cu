@@ -282,7 +282,7 @@ size_t overlap_bytes(int64_t N, int64_t k) { return (size_t)N * (size_t)((k + 7)
 struct InitPlan {
   int64_t chunk;
   bool bf16;
-  void *W10b, *W20b, *Ac, *Zb;
+  void *W10b, *W20b, *Wg0b, *Ac, *Zb;   // Wg0b: hi | lo split of the gate weights (gated modules)
   double* absA_part;
   int row_blocks;
   size_t bytes;
@@ -298,6 +298,7 @@ InitPlan plan_init(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   Carver c(ws);
   p.W10b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;  // hi | lo split of W1_0
   p.W20b = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.Wg0b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;
   p.Ac = c.take_bytes((size_t)p.chunk * n * csz);
   p.Zb = p.bf16 ? c.take_bytes((size_t)p.chunk * n * csz) : nullptr;
   fused_update_grid(p.chunk, n, &p.row_blocks);
@@ -579,7 +580,15 @@ sp_status sp_distribute_importance(const double* head_stats, int32_t n_heads, co
 static sp_status check_module(const sp_ffn_module* m, const sp_ffn_state* st, bool need_w0) {
   if (!m || !st) return SP_ERR_INVALID_ARG;
   if (m->d < 1 || m->n < 1 || m->N < 1) return SP_ERR_SHAPE;
-  if (m->act != SP_ACT_RELU) return SP_ERR_UNSUPPORTED;
+  if (m->act != SP_ACT_RELU && m->act != SP_ACT_SWIGLU) return SP_ERR_UNSUPPORTED;
+  if (m->act == SP_ACT_SWIGLU) {
+    if (!st->Gate) return SP_ERR_INVALID_ARG;
+    if (need_w0) {
+      if (!m->Wg_0.ptr) return SP_ERR_INVALID_ARG;
+      if (m->Wg_0.dtype != SP_F32) return SP_ERR_DTYPE;
+      if (m->Wg_0.rows != m->n || m->Wg_0.cols != m->d || m->Wg_0.ld < m->d) return SP_ERR_SHAPE;
+    }
+  }
   if (!m->X.ptr || !m->Ypre.ptr) return SP_ERR_INVALID_ARG;
   if (!valid_act_dtype(m->X.dtype) || m->Ypre.dtype != m->X.dtype) return SP_ERR_DTYPE;
   if (m->X.rows != m->N || m->X.cols != m->d || m->X.ld < m->d) return SP_ERR_SHAPE;
@@ -605,8 +614,12 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const bool bf16 = p.bf16;
   const bool acc64 = !bf16;
+  const bool gated = m->act == SP_ACT_SWIGLU;
   MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, w20{m->W2_0.ptr, SP_F32, m->W2_0.ld};
+  MatRef wg0{gated ? m->Wg_0.ptr : nullptr, SP_F32, gated ? m->Wg_0.ld : 0};
   if (bf16) {
+    if (gated)
+      CU(split_bf16(reinterpret_cast<const float*>(m->Wg_0.ptr), m->Wg_0.ld, nullptr, n, d, split_kpad(d), p.Wg0b, s));
     CU(split_bf16(reinterpret_cast<const float*>(m->W1_0.ptr), m->W1_0.ld, nullptr, n, d, split_kpad(d), p.W10b, s));
     CU(convert_matrix(m->W2_0.ptr, SP_F32, m->W2_0.ld, p.W20b, SP_BF16, n, d, n, s));
     w20 = MatRef{p.W20b, SP_BF16, n};
@@ -626,9 +639,15 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
     // z^pre = X W1_0^T
     if (bf16) SPCHK(contract_split_weights(Tc, n, d, xc, p.W10b, w10, zc, status_dev, s));
     else SPCHK(contract(Tc, n, d, 1.0, xc, true, w10, true, 0.0, zc, zc, false, acc64, false, status_dev, s));
+    float* Gc = gated ? st->Gate + (size_t)t0 * n : nullptr;
+    if (gated) {   // gate pre-activation X Wg_0^T into the gate buffer; the activation kernel turns it into SiLU
+      MatRef gc{Gc, SP_F32, n};
+      if (bf16) SPCHK(contract_split_weights(Tc, n, d, xc, p.Wg0b, wg0, gc, status_dev, s));
+      else SPCHK(contract(Tc, n, d, 1.0, xc, true, wg0, true, 0.0, gc, gc, false, acc64, false, status_dev, s));
+    }
     int rb;
     fused_update_grid(Tc, n, &rb);
-    CU(launch_init_act(Zc, p.Ac, p.Zb, cdt, Tc, n, p.absA_part, rb, s));
+    CU(launch_init_act(Zc, Gc, p.Ac, p.Zb, cdt, Tc, n, p.absA_part, rb, s));
     CU(reduce_col_partials(p.absA_part, rb, n, st->absA, ci > 0, s));
     // Ypre = a^pre W2_0^T
     SPCHK(contract(Tc, d, n, 1.0, ac, true, w20, true, 0.0, yc, yc, false, acc64, bf16, status_dev, s));
@@ -655,6 +674,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   if (!(prm->alpha > 0.0) || !(prm->beta > 0.0) || !(prm->rho >= 0.0) || prm->token_chunk < 0) return SP_ERR_INVALID_ARG;
   if (prm->z_rule != SP_Z_PAPER && prm->z_rule != SP_Z_EXACT) return SP_ERR_UNSUPPORTED;
   if (prm->score_kind < SP_SCORE_WANDA_L2 || prm->score_kind > SP_SCORE_LEMMA1) return SP_ERR_UNSUPPORTED;
+  if (m->act == SP_ACT_SWIGLU && prm->score_kind == SP_SCORE_LEMMA1) return SP_ERR_UNSUPPORTED;
   const int32_t cdt = m->X.dtype;
   if (!ws || ws_bytes < plan_admm(nullptr, d, n, N, prm->token_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
   AdmmPlan p = plan_admm(ws, d, n, N, prm->token_chunk, cdt);
@@ -799,7 +819,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     float* Uc = (prm->dual_mode && st->U) ? st->U + (size_t)t0 * n : nullptr;
     MatRef h{p.H, cdt, kp}, e{p.E, cdt, d}, dd{p.D, SP_F32, kp}, z1{p.z1, SP_F32, kp}, ac{p.Ac, cdt, n};
     MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : MatRef{Zc, SP_F32, n};
-    CU(launch_prep_h(Zc, Uc, p.H, cdt, Tc, n, kp, k, idx, s));
+    const float* Gc = (m->act == SP_ACT_SWIGLU) ? st->Gate + (size_t)t0 * n : nullptr;
+    CU(launch_prep_h(Zc, Uc, Gc, p.H, cdt, Tc, n, kp, k, idx, s));
     // E = Ypre - h_S W2[:, S]^T ; D_S = E Qt^T ; z1_S = X W1[S, :]^T
     SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
     SPCHK(contract(Tc, k, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
@@ -807,7 +828,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     else if (bf16) SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, w1, z1, status_dev, s));
     else SPCHK(contract(Tc, k, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, false, status_dev, s));
     UpdateArgs ua;
-    ua.Z = Zc; ua.U = Uc; ua.z1 = z1_ahead ? p.z1_all + (size_t)t0 * kp : p.z1; ua.D = p.D; ua.ldk = kp; ua.k = k; ua.grp_base = p.grp_base;
+    ua.Z = Zc; ua.U = Uc; ua.gate = Gc; ua.z1 = z1_ahead ? p.z1_all + (size_t)t0 * kp : p.z1; ua.D = p.D; ua.ldk = kp; ua.k = k; ua.grp_base = p.grp_base;
     ua.grp_mask = p.grp_mask; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
     ua.out_dtype = cdt; ua.T = Tc; ua.n = n; ua.alpha = (float)prm->alpha; ua.beta = (float)prm->beta;
     ua.z_rule = prm->z_rule; ua.partial = p.partial; ua.absA_part = p.absA_part;

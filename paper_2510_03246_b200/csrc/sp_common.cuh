@@ -173,6 +173,7 @@ struct UpdateArgs {
   float* U;          // [T, n] in/out or null
   const float* z1;   // [T, ldk] compact on the kept channels
   const float* D;    // [T, ldk] compact: correction term of the a-update
+  const float* gate; // [T, n] gate factor of a gated module (phi(z) = gate * z), or null: phi = ReLU
   int64_t ldk, k;    // leading dimension of the compact tensors, number of kept channels
   const int32_t* grp_base;   // per group of 8 channels: kept channels before the group
   const uint8_t* grp_mask;   // per group of 8 channels: bit q = channel 8 g + q is kept
@@ -188,9 +189,10 @@ struct UpdateArgs {
 };
 // grp_base / grp_mask of a u8 mask over n channels (see sp_elementwise.cu)
 cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream);
-// H[T, ldh] (compact on the k kept channels idx[0..k), ldh a multiple of 8) = storage(phi(Z) - U)
-cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n, int64_t ldh,
-                          int64_t k, const int32_t* idx, cudaStream_t stream);
+// H[T, ldh] (compact on the k kept channels idx[0..k), ldh a multiple of 8) = storage(phi(Z) - U);
+// phi(z) = gate * z when gate != nullptr, else ReLU
+cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, void* H, int32_t hdt, int64_t T,
+                          int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream);
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]
@@ -206,8 +208,9 @@ cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t c
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
                         cudaStream_t stream);
 // relu + storage conversion for the init pass: A = phi(Z) -> storage dtype, and |A| column partials
-cudaError_t launch_init_act(const float* Z, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T, int64_t n,
-                            double* absA_part, int32_t row_blocks, cudaStream_t stream);
+// gate_io (gated modules): holds the gate pre-activation on entry and SiLU of it on return; A = gate * Z then
+cudaError_t launch_init_act(const float* Z, float* gate_io, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T,
+                            int64_t n, double* absA_part, int32_t row_blocks, cudaStream_t stream);
 cudaError_t column_stats(const void* X, int32_t dt, int64_t ld, int64_t T, int64_t C, double* rowstats,
                          double* scratch, cudaStream_t stream);
 

@@ -222,7 +222,8 @@ __device__ __forceinline__ void store8(void* base, int32_t dt, int64_t e, const 
 // gathers their channels (ascending, so close together in a row of Z) and writes one 16-byte (bf16) or two 16-byte
 // (fp32) vectors per row.  Columns k..ldh-1 of H are written as zero.
 __global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U,
-                                                     void* __restrict__ H, int32_t hdt, int64_t T, int64_t n,
+                                                     const float* __restrict__ G, void* __restrict__ H, int32_t hdt,
+                                                     int64_t T, int64_t n,
                                                      int64_t ldh, int64_t k, const int32_t* __restrict__ idx,
                                                      int32_t rows_per_block) {
   const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
@@ -237,7 +238,13 @@ __global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z
     const float* zr = Z + r * n;
     float h[8];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) h[q] = (ch[q] >= 0) ? fmaxf(zr[ch[q]], 0.f) : 0.f;
+    for (int q = 0; q < 8; ++q) h[q] = (ch[q] >= 0) ? (G ? zr[ch[q]] : fmaxf(zr[ch[q]], 0.f)) : 0.f;
+    if (G) {           // gated module: phi(z) = g z
+      const float* gr = G + r * n;
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (ch[q] >= 0) h[q] *= gr[ch[q]];
+    }
     if (U) {
       const float* ur = U + r * n;
 #pragma unroll
@@ -249,8 +256,18 @@ __global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z
 }
 
 // One element of the fused update.  Returns A; writes the new z (and u).
+constexpr int kZGated = 2;   // internal rule of gated modules: phi(z) = gate * z, one closed-form minimiser
+
 __device__ __forceinline__ float update_one(float zold, float z1, float dcorr, float& u, bool has_u, float alpha,
-                                            float beta, float inv_ab, int z_rule, float& znew) {
+                                            float beta, float inv_ab, int z_rule, float gate, float& znew) {
+  if (z_rule == kZGated) {
+    const float h = gate * zold - (has_u ? u : 0.f);
+    const float a = h + dcorr;
+    const float au = a + (has_u ? u : 0.f);
+    znew = (beta * gate * au + alpha * z1) / fmaf(beta * gate, gate, alpha);
+    if (has_u) u = u + a - gate * znew;
+    return a;
+  }
   const float h = fmaxf(zold, 0.f) - (has_u ? u : 0.f);
   const float a = h + dcorr;
   const float au = a + (has_u ? u : 0.f);
@@ -290,7 +307,7 @@ __device__ __forceinline__ void store4(void* base, int32_t dt, int64_t e, const 
 // and blocks.
 template <bool HAS_U>
 struct UpdRow {
-  float zo[4], u[4], z1[4], dc[4];
+  float zo[4], u[4], z1[4], dc[4], gt[4];
 };
 
 template <bool HAS_U, int Z_RULE>
@@ -345,6 +362,18 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) w.u[q] = 0.f;
       }
+      if (Z_RULE == kZGated) {
+        if (vec) {
+          const float4 x = *reinterpret_cast<const float4*>(g.gate + e);
+          w.gt[0] = x.x; w.gt[1] = x.y; w.gt[2] = x.z; w.gt[3] = x.w;
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) w.gt[q] = (q < cnt) ? g.gate[e + q] : 0.f;
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) w.gt[q] = 0.f;
+      }
       const float* zp = z1p + r * g.ldk + base;
       const float* dp = Dp + r * g.ldk + base;
 #pragma unroll
@@ -360,11 +389,11 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
       float p_res = 0.f, p_z = 0.f, p_a = 0.f, p_in = 0.f;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        a[q] = update_one(w.zo[q], w.z1[q], w.dc[q], w.u[q], HAS_U, g.alpha, g.beta, inv_ab, Z_RULE, zn[q]);
+        a[q] = update_one(w.zo[q], w.z1[q], w.dc[q], w.u[q], HAS_U, g.alpha, g.beta, inv_ab, Z_RULE, w.gt[q], zn[q]);
         if (!vec && q >= cnt) { a[q] = 0.f; zn[q] = 0.f; w.z1[q] = 0.f; }
         const float din = zn[q] - w.z1[q];
         p_in = fmaf(din, din, p_in);
-        const float diff = a[q] - fmaxf(zn[q], 0.f);
+        const float diff = a[q] - (Z_RULE == kZGated ? w.gt[q] * zn[q] : fmaxf(zn[q], 0.f));
         p_res = fmaf(diff, diff, p_res);
         p_z = fmaf(zn[q], zn[q], p_z);
         p_a = fmaf(a[q], a[q], p_a);
@@ -433,9 +462,9 @@ __global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
 }
 
 // init pass: A = phi(Z) in storage dtype, optional storage copy of Z, |A| column partials
-__global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__ Z, void* A_out, void* Zb_out,
-                                                       int32_t out_dtype, int64_t T, int64_t n, double* absA_part,
-                                                       int32_t row_blocks) {
+__global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__ Z, float* gate_io, void* A_out,
+                                                       void* Zb_out, int32_t out_dtype, int64_t T, int64_t n,
+                                                       double* absA_part, int32_t row_blocks) {
   const int64_t c0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
   if (c0 >= n) return;
   const int64_t rows_per = ceil_div(T, (int64_t)row_blocks);
@@ -447,8 +476,16 @@ __global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__
     const int64_t e = r * n + c0;
     for (int q = 0; q < cnt; ++q) {
       const float z = Z[e + q];
-      const float a = fmaxf(z, 0.f);
-      cs[q] += (double)a;
+      float a;
+      if (gate_io) {       // gated module: the buffer holds the gate pre-activation, SiLU of it replaces it
+        const float zg = gate_io[e + q];
+        const float gt = zg / (1.f + expf(-zg));
+        gate_io[e + q] = gt;
+        a = gt * z;
+      } else {
+        a = fmaxf(z, 0.f);
+      }
+      cs[q] += (double)fabsf(a);
       if (out_dtype == SP_BF16) {
         reinterpret_cast<__nv_bfloat16*>(A_out)[e + q] = __float2bfloat16_rn(a);
         if (Zb_out) reinterpret_cast<__nv_bfloat16*>(Zb_out)[e + q] = __float2bfloat16_rn(z);
@@ -678,11 +715,12 @@ cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, u
   return cudaGetLastError();
 }
 
-cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, int64_t T, int64_t n, int64_t ldh,
-                          int64_t k, const int32_t* idx, cudaStream_t stream) {
+cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, void* H, int32_t hdt, int64_t T,
+                          int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream) {
   if (T * ldh == 0) return cudaSuccess;
   // algorithmic bytes: Z (and U) read once, the kept part written once
-  ProfScope prof(PK_PREP_H, 0.0, (double)T * ((double)n * (U ? 8.0 : 4.0) + (double)k * (hdt == SP_BF16 ? 2.0 : 4.0)),
+  ProfScope prof(PK_PREP_H, 0.0,
+                 (double)T * ((double)n * (U ? 8.0 : 4.0) + (double)k * ((hdt == SP_BF16 ? 2.0 : 4.0) + (gate ? 4.0 : 0.0))),
                  stream);
   const unsigned gx = (unsigned)ceil_div(ldh, (int64_t)(8 * 256));
   int64_t rb = ceil_div((int64_t)148 * 16, (int64_t)gx);
@@ -690,7 +728,7 @@ cudaError_t launch_prep_h(const float* Z, const float* U, void* H, int32_t hdt, 
   if (rb > 65535) rb = 65535;
   const int32_t rows_per = (int32_t)ceil_div(T, rb);
   count_launch();
-  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, H, hdt, T, n, ldh, k, idx,
+  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, gate, H, hdt, T, n, ldh, k, idx,
                                                                                         rows_per);
   return cudaGetLastError();
 }
@@ -711,11 +749,14 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   // algorithmic bytes per row: Z (and U) read and written, A and the storage copy of Z written, z1 and D read on the
   // kept channels
   const double esz = a.out_dtype == SP_BF16 ? 2.0 : 4.0;
-  const double per_n = 8.0 + (a.U ? 8.0 : 0.0) + esz + (a.Zb_out ? esz : 0.0);
+  const double per_n = 8.0 + (a.U ? 8.0 : 0.0) + esz + (a.Zb_out ? esz : 0.0) + (a.gate ? 4.0 : 0.0);
   ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * ((double)a.n * per_n + (double)a.k * 8.0), stream);
   count_launch();
   const bool pz = a.z_rule == SP_Z_PAPER;
-  if (a.U) {
+  if (a.gate) {
+    if (a.U) fused_update_kernel<true, kZGated><<<grid, 256, 0, stream>>>(a);
+    else fused_update_kernel<false, kZGated><<<grid, 256, 0, stream>>>(a);
+  } else if (a.U) {
     if (pz) fused_update_kernel<true, SP_Z_PAPER><<<grid, 256, 0, stream>>>(a);
     else fused_update_kernel<true, SP_Z_EXACT><<<grid, 256, 0, stream>>>(a);
   } else {
@@ -725,13 +766,13 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_init_act(const float* Z, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T, int64_t n,
-                            double* absA_part, int32_t row_blocks, cudaStream_t stream) {
+cudaError_t launch_init_act(const float* Z, float* gate_io, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T,
+                            int64_t n, double* absA_part, int32_t row_blocks, cudaStream_t stream) {
   if (T * n == 0) return cudaSuccess;
   dim3 grid((unsigned)ceil_div(n, 1024), (unsigned)row_blocks);
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  init_act_kernel<<<grid, 256, 0, stream>>>(Z, A_out, Zb_out, out_dtype, T, n, absA_part, row_blocks);
+  init_act_kernel<<<grid, 256, 0, stream>>>(Z, gate_io, A_out, Zb_out, out_dtype, T, n, absA_part, row_blocks);
   return cudaGetLastError();
 }
 

@@ -147,6 +147,13 @@ def make_weights(cfg: ModuleConfig, layer: int = 0, device="cpu"):
     return w1.to(dt), w2.to(dt)
 
 
+def make_gate_weights(cfg: ModuleConfig, layer: int = 0, device="cpu"):
+    """Pre-trained stand-in of the gate projection Wg_0 [n, d] of a SwiGLU module (tensor id 4), storage dtype."""
+    seed = module_seed(cfg, layer)
+    wg = standard_variates(seed, 4, cfg.n * cfg.d, "gauss", device).view(cfg.n, cfg.d) * cfg.weight_std
+    return wg.to(storage_dtype(cfg))
+
+
 def make_importances(cfg: ModuleConfig, device="cpu") -> torch.Tensor:
     """A seeded stand-in for the per-layer importances I_l (float64, positive, mildly depth dependent)."""
     u = _unit_open(uniform_bits(module_seed(cfg, 0), 9, 0, cfg.layers, device))
