@@ -110,16 +110,21 @@ def oracle_iteration_seconds(cfg, sample_tokens: int, repeats: int = 1):
     X = synth.make_activations(cfg, tokens=sample_tokens).double().numpy().T.copy()
     W1, W2 = synth.make_weights(cfg)
     W1 = W1.double().numpy(); W2 = W2.double().numpy()
-    st, Y = O.ffn_init(X, W1, W2)
-    p = O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho)
+    gated = cfg.act == "swiglu"
+    if gated:
+        st, Y = O.swiglu_init(X, synth.make_gate_weights(cfg).double().numpy(), W1, W2)
+    else:
+        st, Y = O.ffn_init(X, W1, W2)
+    p = O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, act=cfg.act)
     tw = tt = 0.0
     for _ in range(repeats):
         t0 = time.perf_counter()
         O.admm_weight_phase(st, W1, p, X.shape[1])
         t1 = time.perf_counter()
-        A = O.a_update(st.W2, Y, st.Z, p.alpha, p.beta)
+        A = O.a_update(st.W2, Y, st.Z, p.alpha, p.beta, None, cfg.act, st.gate)
         z1, z2 = O.z_candidates(st.W1, X, A, p.alpha, p.beta)
-        st.Z = O.z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule)
+        st.Z = (O.swiglu_zu_update(A, st.gate, z1, p.alpha, p.beta) if gated
+                else O.z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule))
         st.G_A = A @ A.T; st.R1 = st.Z @ X.T; st.R2 = Y @ A.T; st.absA = np.abs(A).sum(axis=1)
         O.allocate_sparsity(np.linspace(1.0, 1.5, cfg.layers), [cfg.n] * cfg.layers, cfg.sparsity, 1.25)
         t2 = time.perf_counter()
@@ -177,7 +182,8 @@ def run_reference(args, cfg):
 
 def workload_name(cfg) -> str:
     shape = {"C1": "OPT-125M", "C2": "OPT-1.3B", "C3": "OPT-6.7B", "C4": "LLaMA-2-7B", "C5": "OPT-30B"}.get(cfg.name, "OPT")
-    return (f"{cfg.name}: {shape}-shaped FFN module, d={cfg.d}, n={cfg.n}, N={cfg.tokens} tokens, "
+    kind = "SwiGLU FFN module (gate/up/down)" if cfg.act == "swiglu" else "FFN module"
+    return (f"{cfg.name}: {shape}-shaped {kind}, d={cfg.d}, n={cfg.n}, N={cfg.tokens} tokens, "
             f"{cfg.storage} activations, {int(cfg.sparsity * 100)}% channel sparsity (k_keep={cfg.k_keep})")
 
 
@@ -209,7 +215,8 @@ def main():
     layer = rank
     X = synth.make_activations(cfg, layer, device=dev)
     W1_0, W2_0 = synth.make_weights(cfg, layer, device=dev)
-    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=args.chunk, overlap_k=cfg.k_keep)
+    Wg_0 = synth.make_gate_weights(cfg, layer, device=dev) if cfg.act == "swiglu" else None
+    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
     I_all = synth.make_importances(cfg, device=dev)
     n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
     T_soft = float(I_all.abs().mean())
@@ -301,13 +308,15 @@ def main():
         del mod
         torch.cuda.empty_cache()
         hX = X.cpu().pin_memory(); hW1 = W1_0.cpu().pin_memory(); hW2 = W2_0.cpu().pin_memory()
-        del X, W1_0, W2_0
+        hWg = Wg_0.cpu().pin_memory() if Wg_0 is not None else None
+        del X, W1_0, W2_0, Wg_0
         torch.cuda.empty_cache()
         iters = cfg.iters
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
-        m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk, overlap_k=cfg.k_keep)
+        dWg = hWg.to(dev, non_blocking=True) if hWg is not None else None
+        m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=dWg)
         m2.sp_ffn_init()
         for _ in range(iters):
             m2.sp_admm_step(prm)
@@ -316,6 +325,8 @@ def main():
         t1 = time.perf_counter()
         m2.check_status()
         h2d = hX.numel() * hX.element_size() + hW1.numel() * hW1.element_size() + hW2.numel() * hW2.element_size()
+        if hWg is not None:
+            h2d += hWg.numel() * hWg.element_size()
         d2h = oW1.numel() * 4 + oW2.numel() * 4 + omask.numel()
         e2e = {"value": iters / (t1 - t0), "unit": UNIT, "layers_per_s": 1.0 / (t1 - t0), "h2d_bytes_per_step": h2d / iters,
                "d2h_bytes_per_step": d2h / iters, "iterations": iters,
