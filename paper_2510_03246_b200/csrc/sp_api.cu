@@ -158,7 +158,7 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
     // proper is then only the backward sweep
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
     SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, factor_lookahead ? assist : nullptr, m));
-    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist, true));
+    SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist, true, Gs, nn));
   } else {
     CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
@@ -789,7 +789,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
       SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s,
                            (side && !z1_ahead) ? &side->assist_main : nullptr, k));
       SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s,
-                           side ? &side->assist_main : nullptr, true));
+                           side ? &side->assist_main : nullptr, true, Gs, d));
       CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));
       qt = MatRef{p.Qtb, SP_BF16, d};
     } else {

@@ -119,9 +119,11 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P,
                          cudaStream_t stream, const SolveAssist* assist = nullptr, int64_t m_extra = 0);
 // Xs holds TWO buffers of [m, 3 * kCholTcNB] bf16.
 // forward_done: X already holds the solution of the forward system (it rode along with the factorisation).
+// Lf / ldl (optional): the fp32 factor potrf_lower_tc left in A; with it the backward sweep updates the next block
+// column inside the panel kernel instead of by a GEMM of its own.
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* P, const float* dinv, void* Xs,
                          int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist = nullptr,
-                         bool forward_done = false);
+                         bool forward_done = false, const float* Lf = nullptr, int64_t ldl = 0);
 
 // ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,

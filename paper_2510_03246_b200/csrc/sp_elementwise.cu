@@ -311,7 +311,7 @@ struct UpdRow {
 };
 
 template <bool HAS_U, int Z_RULE>
-__global__ void __launch_bounds__(256) fused_update_kernel(UpdateArgs g) {
+__global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
   __shared__ double sm[32];
   const int64_t grp4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t c0 = grp4 * 4;

@@ -292,7 +292,20 @@ __device__ __forceinline__ bool stage_block_wait(uint64_t* bar, uint32_t parity)
 constexpr int PA_ROWS = 32;
 constexpr int PA_THREADS = 256;
 constexpr int PA_APAD = PA_ROWS + 4;
-constexpr size_t PA_SMEM = ((size_t)TB * TB + (size_t)TB * PA_APAD) * sizeof(float) + 16;
+constexpr size_t PA_SMEM = ((size_t)TB * TB + (size_t)TB * PA_APAD) * sizeof(float) + 128;
+constexpr size_t PA_SMEM_NEAR = PA_SMEM + (size_t)TB * TB * sizeof(float);   // + the block of L of the second product
+
+// Optional second product of the same launch (backward triangular solve, TRANS form only): with W_j the block column
+// just computed, X[:, near columns] -= W_j L[j rows, near columns], the update of the block column the NEXT step
+// needs, so that the chain of a solve is one kernel per block column.  L: fp32 factor, pointer to its element
+// (first row of block j, first near column), leading dimension ldl (a multiple of 4, 16-byte aligned rows); Xn: first
+// near column of X.  The far columns are updated by a tensor-core GEMM on another stream, which may still be adding
+// into the near columns when this kernel runs: both add atomically.
+struct PanelNear {
+  const float* L;    // nullptr: no second product
+  int64_t ldl;
+  float* Xn;
+};
 
 // X[i, 0:nb] <- X[i, 0:nb] inv(L)^T (TRANS == false) or X[i, 0:nb] inv(L) (TRANS == true), for `rows` rows.
 // dinv is the pair of TB x TB blocks written by chol_diag128_kernel.  The result is written back in fp32 (write_f32)
@@ -303,18 +316,36 @@ template <bool TRANS>
 __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64_t ldx, int64_t rows, int nb,
                                                                  const float* __restrict__ dinv, __nv_bfloat16* S,
                                                                  int64_t lds, int64_t s_seg, int write_f32,
-                                                                 int32_t* status) {
+                                                                 int32_t* status, PanelNear near) {
   extern __shared__ __align__(128) float pa_smem[];
   float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(pa_smem);                       // Lt[k][c]
   float (*At)[PA_APAD] = reinterpret_cast<float (*)[PA_APAD]>(pa_smem + TB * TB);   // At[k][row]
-  uint64_t* bar = reinterpret_cast<uint64_t*>(pa_smem + TB * TB + TB * PA_APAD);
+  uint64_t* bar = reinterpret_cast<uint64_t*>(pa_smem + TB * TB + TB * PA_APAD);    // [0]: Lt landed, [1]: Bn landed
+  float (*Bn)[TB] = reinterpret_cast<float (*)[TB]>(pa_smem + TB * TB + TB * PA_APAD + 32);   // Bn[k][c] (near only)
   const int t = threadIdx.x;
   const int64_t r0 = (int64_t)blockIdx.x * PA_ROWS;
   const bool x_al = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0);
-  if (t == 0) stage_bar_init(bar);
+  const bool do_near = TRANS && near.L != nullptr;
+  if (t == 0) {
+    stage_bar_init(bar);
+    if (do_near) stage_bar_init(bar + 1);
+  }
   __syncthreads();
   // Lt[k][c] = inv(L)[c][k] (the transposed copy) or inv(L)[k][c]: a straight copy either way
   if (t == 0) stage_block_issue(pa_smem, dinv + (TRANS ? 0 : TB * TB), bar);
+  if (do_near && t < 32) {
+    // rows j0 .. j0 + nb - 1 of L, TB columns each (512 bytes per row), one bulk copy per row, four per lane
+    const uint32_t b1 = lin_smem_u32(bar + 1);
+    if (t == 0)
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b1), "r"((uint32_t)(nb * TB * 4))
+                   : "memory");
+    __syncwarp();
+    for (int k = t; k < nb; k += 32)
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(lin_smem_u32(&Bn[k][0])), "l"(near.L + (int64_t)k * near.ldl), "r"((uint32_t)(TB * 4)),
+                     "r"(b1)
+                   : "memory");
+  }
   {
     float4 xv[PA_ROWS * TB / 4 / PA_THREADS];
 #pragma unroll
@@ -394,23 +425,66 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
         *reinterpret_cast<uint2*>(S + gi * lds + q * s_seg + c0) = *reinterpret_cast<const uint2*>(part[q]);
     }
   }
+
+  if (do_near) {
+    // ---- second product: X[rows, near columns] -= W_j Bn.  W_j goes back to shared memory as the left operand
+    // (At[k][row], k = column of W_j); rows of Bn beyond nb are cleared by hand (no copy wrote them).
+    __syncthreads();     // everyone is done reading At
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) At[c0 + j][4 * ty + r] = (c0 + j < nb) ? acc[r][j] : 0.f;
+    for (int e = t; e < (TB - nb) * TB; e += PA_THREADS) Bn[nb + e / TB][e % TB] = 0.f;
+    const bool staged2 = stage_block_wait(bar + 1, 0);
+    __syncthreads();
+    if (!staged2) {
+      if (t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 12);
+      return;
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[r][j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < TB; ++k) {
+      const float4 a0 = *reinterpret_cast<const float4*>(&At[k][4 * ty]);
+      const float4 l0 = *reinterpret_cast<const float4*>(&Bn[k][4 * tx]);
+      const float av[4] = {a0.x, a0.y, a0.z, a0.w};
+      const float lv[4] = {l0.x, l0.y, l0.z, l0.w};
+#pragma unroll
+      for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int64_t gi = r0 + 4 * ty + r;
+      if (gi >= rows) continue;
+      float* dst = near.Xn + gi * ldx + c0;      // 16-byte aligned: the launcher checks ldx and the base
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(-acc[r][0]), "f"(-acc[r][1]),
+                   "f"(-acc[r][2]), "f"(-acc[r][3])
+                   : "memory");
+    }
+  }
 }
 
 template <bool TRANS>
 cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, const float* dinv, __nv_bfloat16* S,
-                               int64_t lds, int64_t s_seg, bool write_f32, int32_t* status, cudaStream_t stream) {
+                               int64_t lds, int64_t s_seg, bool write_f32, int32_t* status, cudaStream_t stream,
+                               PanelNear near = PanelNear{nullptr, 0, nullptr}) {
   static bool attr = false;
   if (!attr) {
     cudaError_t e = cudaFuncSetAttribute(panel_apply_kernel<TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)PA_SMEM);
+                                         (int)PA_SMEM_NEAR);
     if (e != cudaSuccess) return e;
     attr = true;
   }
   if (rows <= 0) return cudaSuccess;
   count_launch();
-  ProfScope prof(PK_PANEL_APPLY, 2.0 * (double)rows * TB * TB, 0.0, stream);
-  panel_apply_kernel<TRANS><<<(unsigned)ceil_div(rows, PA_ROWS), PA_THREADS, PA_SMEM, stream>>>(
-      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status);
+  const bool with_near = TRANS && near.L != nullptr;
+  ProfScope prof(PK_PANEL_APPLY, (with_near ? 4.0 : 2.0) * (double)rows * TB * TB, 0.0, stream);
+  panel_apply_kernel<TRANS><<<(unsigned)ceil_div(rows, PA_ROWS), PA_THREADS, with_near ? PA_SMEM_NEAR : PA_SMEM, stream>>>(
+      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status, near);
   return cudaGetLastError();
 }
 
@@ -616,7 +690,8 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
 }
 
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* Pv, const float* dinv, void* Xsv,
-                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist, bool forward_done) {
+                         int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist, bool forward_done,
+                         const float* Lf, int64_t ldl) {
   const __nv_bfloat16* P = reinterpret_cast<const __nv_bfloat16*>(Pv);
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(Xsv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
@@ -627,6 +702,15 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
   // on `stream`; the rest runs on the assisting stream and overlaps the next panel.  Panel jj then needs the "rest"
   // update of step jj - 2 (and reuses its buffer of bf16 parts), which is what the two alternating events order.
 #define SP_CUDA_OK(x) do { if ((x) != cudaSuccess) return SP_ERR_CUDA; } while (0)
+  // The tensor-core update adds atomically only through its TMA reduction, which needs 16-byte aligned rows of X;
+  // without it everything stays on one stream.
+  const bool x_al16 = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0);
+  if (!x_al16) assist = nullptr;
+  // Backward sweep: the update of the next block column can ride in the panel kernel (fp32, from the fp32 factor)
+  // when the factor's rows are 16-byte aligned too.
+  // (its 144 KB of shared memory allow one CTA per SM: only while all row blocks fit in one wave)
+  const bool fuse_near = Lf != nullptr && x_al16 && (ldl % 4 == 0) && ((reinterpret_cast<uintptr_t>(Lf) & 15u) == 0) &&
+                         ceil_div(m, (int64_t)PA_ROWS) <= 148;
   bool rec[2] = {false, false};
   auto run_sweep = [&](bool forward) -> sp_status {
     for (int64_t step = 0; step < nblk; ++step) {
@@ -636,11 +720,16 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
       const float* dj = dinv + jb * 2 * TB * TB;
       __nv_bfloat16* Xcur = Xs + (step & 1) * m * lds;
       if (assist && rec[step & 1]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[step & 1], 0));
-      cudaError_t e = forward ? launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, status_dev, stream)
-                              : launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, status_dev, stream);
-      if (e != cudaSuccess) return SP_ERR_CUDA;
       // columns still to be updated: [lo, hi)
       const int64_t lo = forward ? j0 + nb : 0, hi = forward ? n : j0;
+      // backward: the near columns are the whole block before j (TB wide)
+      const bool near_in_panel = !forward && fuse_near && hi > lo;
+      PanelNear pn{nullptr, 0, nullptr};
+      if (near_in_panel) pn = PanelNear{Lf + j0 * ldl + (hi - TB), ldl, X + (hi - TB)};
+      cudaError_t e = forward ? launch_panel_apply<false>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, status_dev, stream)
+                              : launch_panel_apply<true>(X + j0, ldx, m, nb, dj, Xcur, lds, TB, true, status_dev, stream,
+                                                         pn);
+      if (e != cudaSuccess) return SP_ERR_CUDA;
       if (hi <= lo) break;
       if (assist) SP_CUDA_OK(cudaEventRecord(assist->panel_done, stream));
       TcOperand ta{Xcur, lds, true};
@@ -651,7 +740,7 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
       const int64_t near_lo = forward ? lo : hi - wn, far_lo = forward ? lo + wn : lo, far_w = hi - lo - wn;
       for (int part = 0; part < 2; ++part) {
         const int64_t c0 = part == 0 ? near_lo : far_lo, w = part == 0 ? wn : far_w;
-        if (w <= 0) continue;
+        if (w <= 0 || (part == 0 && near_in_panel)) continue;
         const bool on_assist = assist && part == 1;
         cudaStream_t st_run = on_assist ? assist->stream : stream;
         if (on_assist) SP_CUDA_OK(cudaStreamWaitEvent(st_run, assist->panel_done, 0));
