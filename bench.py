@@ -312,26 +312,45 @@ def main():
         del X, W1_0, W2_0, Wg_0
         torch.cuda.empty_cache()
         iters = cfg.iters
+        # the attention half of the layer: fixed head outputs H and the output projection W_O (host, pinned)
+        from paper_2510_03246_b200 import pipeline
+        hH, hWo = synth.make_attention_inputs(cfg, layer)
+        hH = hH.pin_memory(); hWo = hWo.pin_memory()
+        k_heads = max(1, cfg.heads - int(cfg.heads * cfg.sparsity + 0.5))
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
         dWg = hWg.to(dev, non_blocking=True) if hWg is not None else None
         m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=dWg)
         m2.sp_ffn_init()
+        # this layer's share of pass 0: the importance of the pre-trained module
+        api.sp_struct_scores(api.SP_SCORE_WANDA_L2, cfg.n, W=m2.W2_0, colsq=m2.G_A, colsq_stride=cfg.n + 1)
         for _ in range(iters):
             m2.sp_admm_step(prm)
         oW1 = m2.W1.cpu(); oW2 = m2.W2.cpu(); omask = m2.mask.cpu()
+        t_ffn = time.perf_counter()
+        # attention module: pre-trained output of the projection, head scores, head mask, W_O recovery on the kept heads
+        dH = hH.to(dev, non_blocking=True); dWo = hWo.to(dev, non_blocking=True)
+        Ya = torch.empty(dH.shape[0], cfg.d, dtype=dH.dtype, device=dev)
+        api.sp_gemm(dH, dWo, Ya, transB=True, use_tensor_cores=(dH.dtype == torch.bfloat16))
+        hmask, Wo_new, _ = pipeline.prune_attention_heads(dH, Ya, dWo.float(), cfg.heads, k_heads, rho=cfg.rho,
+                                                          token_chunk=args.chunk)
+        oWo = Wo_new.cpu(); ohm = hmask.cpu()
         torch.cuda.synchronize()
         t1 = time.perf_counter()
         m2.check_status()
         h2d = hX.numel() * hX.element_size() + hW1.numel() * hW1.element_size() + hW2.numel() * hW2.element_size()
         if hWg is not None:
             h2d += hWg.numel() * hWg.element_size()
-        d2h = oW1.numel() * 4 + oW2.numel() * 4 + omask.numel()
+        h2d += hH.numel() * hH.element_size() + hWo.numel() * hWo.element_size()
+        d2h = oW1.numel() * 4 + oW2.numel() * 4 + omask.numel() + oWo.numel() * 4 + ohm.numel()
         e2e = {"value": iters / (t1 - t0), "unit": UNIT, "layers_per_s": 1.0 / (t1 - t0), "h2d_bytes_per_step": h2d / iters,
-               "d2h_bytes_per_step": d2h / iters, "iterations": iters,
-               "note": "one module job (= one pruned FFN layer): pinned-host X, W1_0, W2_0 in; init + iterations; W1, W2, "
-                       "mask back to host; layers_per_s is that whole job per second"}
+               "d2h_bytes_per_step": d2h / iters, "iterations": iters, "ffn_seconds": t_ffn - t0,
+               "attention_seconds": t1 - t_ffn,
+               "note": "one pruned layer: pinned-host X, W1_0, W2_0 in; init + importance of the pre-trained module + "
+                       "iterations; W1, W2, mask back to host; then the attention half with fixed head outputs (H, "
+                       "W_O in; head scores, head mask, W_O recovery on the kept heads; W_O, mask out); "
+                       "layers_per_s is that whole job per second, value = iterations / that time"}
 
     cpu = None
     if not args.no_cpu_baseline:

@@ -283,7 +283,9 @@ sp_status sp_distribute_importance(const double* head_stats, int32_t n_heads, co
  *                    rho_eff as in sp_admm_params.  G is read from its lower triangle and left unchanged.
  * sp_linear_refit  — recovery on a kept support of column groups: W[:, S] = R[:, S](G[S,S] + rho_eff I)^-1,
  *                    other columns zero (Algorithm 2, "importance + recovery solver"; used for W2 and for W_O heads).
- *                    mask: u8 [n_units] with exactly k_keep ones (k_keep is a host value).
+ *                    mask: u8 [n_units] with exactly k_keep ones (k_keep is a host value).  The ridge is that of the
+ *                    FULL system: rho_eff = rho * trace(G)/dim(G) when rho_relative != 0 (computed on the device),
+ *                    else rho.
  * sp_gemm          — C[M,N] = alpha * opA(A) opB(B) + beta * C, opX(X) = X or X^T; test and utility entry.
  *                    use_tensor_cores != 0 requests the tcgen05 path (bf16 operands only; falls back with
  *                    SP_ERR_UNSUPPORTED when shapes or alignment do not allow it).
@@ -293,8 +295,9 @@ sp_status sp_ridge_solve(const float* R, int64_t ldr, const float* G, int64_t ld
                          int32_t rho_relative, int32_t precise, float* W, int64_t ldw, int32_t* status_dev, void* ws,
                          size_t ws_bytes, void* stream);
 sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_units,
-                          int32_t group, const uint8_t* mask, int64_t k_keep, double rho_eff, int32_t precise,
-                          float* W, int64_t ldw, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream);
+                          int32_t group, const uint8_t* mask, int64_t k_keep, double rho, int32_t rho_relative,
+                          int32_t precise, float* W, int64_t ldw, int32_t* status_dev, void* ws, size_t ws_bytes,
+                          void* stream);
 sp_status sp_gemm(int32_t transA, int32_t transB, int64_t M, int64_t N, int64_t K, double alpha, const sp_mat* A,
                   const sp_mat* B, double beta, const sp_mat* C, int32_t lower_only, int32_t use_tensor_cores,
                   int32_t* status_dev, void* stream);

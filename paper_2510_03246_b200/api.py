@@ -98,7 +98,7 @@ def lib() -> C.CDLL:
         L.sp_weight_stats.argtypes = [pm, i32, i64, i32, vp, vp, sz, vp]
         L.sp_distribute_importance.argtypes = [vp, i32, vp, i32, i32, dbl, dbl, vp, vp, vp]
         L.sp_ridge_solve.argtypes = [vp, i64, vp, i64, i64, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
-        L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, vp, i64, vp, vp, sz, vp]
+        L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
         L.sp_gemm.argtypes = [i32, i32, i64, i64, i64, dbl, pm, pm, dbl, pm, i32, i32, vp, vp]
         L.sp_symmetrize.argtypes = [vp, i64, i64, vp]
         L.sp_profile_begin.argtypes = [i32]
@@ -226,7 +226,8 @@ def sp_ridge_solve(R, G, rho, rho_relative=True, precise=False, W=None, status=N
     return W
 
 
-def sp_linear_refit(R, G, mask, k_keep, rho_eff, group=1, precise=False, W=None, status=None, ws=None):
+def sp_linear_refit(R, G, mask, k_keep, rho, group=1, precise=False, W=None, status=None, ws=None,
+                    rho_relative=False):
     _require_cuda(R, G, mask, W)
     m, n = R.shape
     if W is None:
@@ -234,7 +235,7 @@ def sp_linear_refit(R, G, mask, k_keep, rho_eff, group=1, precise=False, W=None,
     if ws is None:
         ws = _ws(workspace_bytes(SP_WS_LINEAR_REFIT, m, n, 0, 0, SP_F64 if precise else SP_F32), R.device)
     _check(lib().sp_linear_refit(R.data_ptr(), R.stride(0), G.data_ptr(), G.stride(0), m, n // group, group,
-                                 mask.data_ptr(), int(k_keep), float(rho_eff), int(precise), W.data_ptr(),
+                                 mask.data_ptr(), int(k_keep), float(rho), int(rho_relative), int(precise), W.data_ptr(),
                                  W.stride(0), _ptr(status), ws.data_ptr(), ws.numel(), _stream()), "sp_linear_refit")
     return W
 

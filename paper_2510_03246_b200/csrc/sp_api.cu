@@ -439,8 +439,9 @@ sp_status sp_ridge_solve(const float* R, int64_t ldr, const float* G, int64_t ld
 }
 
 sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_units,
-                          int32_t group, const uint8_t* mask, int64_t k_keep, double rho_eff, int32_t precise,
-                          float* W, int64_t ldw, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+                          int32_t group, const uint8_t* mask, int64_t k_keep, double rho, int32_t rho_relative,
+                          int32_t precise, float* W, int64_t ldw, int32_t* status_dev, void* ws, size_t ws_bytes,
+                          void* stream) {
   if (!R || !G || !W || !mask) return SP_ERR_INVALID_ARG;
   if (group < 1 || n_units < 0 || m < 0 || k_keep < 0 || k_keep > n_units) return SP_ERR_SHAPE;
   const int64_t n = n_units * group;
@@ -453,7 +454,7 @@ sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t l
   Carver c(ws);
   SolveBufs b = carve_solve(c, n, m, precise ? 8 : 4);
   int32_t* unit_idx = c.take<int32_t>((size_t)n_units);
-  CU(effective_ridge(nullptr, 0, 1, rho_eff, 0, b.rho, s));
+  CU(effective_ridge(G, ldg, n, rho, rho_relative, b.rho, s));     // the ridge of the full system
   CU(mask_to_index(mask, n_units, unit_idx, s));
   const int64_t k = k_keep * group;
   if (k > 0) {

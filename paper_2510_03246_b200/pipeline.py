@@ -93,6 +93,30 @@ def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_unit
     return results, r, k_keep, {"importance_s": t1 - t0, "admm_s": t2 - t1, "layers_per_s": len(mine) / max(t2 - t0, 1e-9)}
 
 
+def prune_attention_heads(H: torch.Tensor, Ypre: torch.Tensor, W_O: torch.Tensor, n_heads: int, k_heads: int,
+                          rho: float = 0.1, token_chunk: int = 32768):
+    """Head pruning of one attention module with its head outputs held fixed (Algorithm 2, attention branch, W_O part;
+    Algorithm 1 Step 3 with heads as units).  H [N, d]: concatenated head outputs (the input of the output
+    projection), Ypre [N, d]: the pre-trained module output, W_O [d, d] fp32.  Head h owns columns
+    [h d_head, (h + 1) d_head) of W_O.  Steps, all library calls:
+      G_H = H^T H, R = Ypre^T H          sp_gram_accumulate over token chunks
+      head scores                       sp_struct_scores, Wanda-l2 over the head's column block of W_O
+      keep the k_heads best             sp_apply_mask
+      W_O[:, S] = R[:, S](G_H[S,S] + rho_eff I)^-1, other heads zero     sp_linear_refit (ridge of the full system)
+    Returns (mask u8 [n_heads], W_O_new fp32 [d, d], scores fp32 [n_heads])."""
+    N, d = H.shape
+    d_head = d // n_heads
+    G = torch.zeros(d, d, dtype=torch.float32, device=H.device)
+    R = torch.zeros(d, d, dtype=torch.float32, device=H.device)
+    for t0 in range(0, N, token_chunk):
+        api.sp_gram_accumulate(H[t0:t0 + token_chunk], Ypre[t0:t0 + token_chunk], G, R)
+    api.sp_symmetrize(G)
+    scores, _, _ = api.sp_struct_scores(api.SP_SCORE_WANDA_L2, n_heads, d_head, W=W_O, colsq=G, colsq_stride=d + 1)
+    mask, _, _ = api.sp_apply_mask(scores, k_heads)
+    W_new = api.sp_linear_refit(R, G, mask, k_heads, rho, group=d_head, rho_relative=True)
+    return mask, W_new, scores
+
+
 def plan_distribute(layer_weights: Callable[[int], dict], n_layers: int, n_heads: int, n_ffn: int, rbar: float,
                     T_rel: float = 1.0, rho: float = 1.0, gamma: float = 1.0, device="cuda"):
     """Steps 1 and 2 of the "-distribute" variant of Algorithm 1: importances of the attention and MLP modules from

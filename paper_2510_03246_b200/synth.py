@@ -154,6 +154,14 @@ def make_gate_weights(cfg: ModuleConfig, layer: int = 0, device="cpu"):
     return wg.to(storage_dtype(cfg))
 
 
+def make_attention_inputs(cfg: ModuleConfig, layer: int = 0, device="cpu", tokens: int | None = None):
+    """Stand-ins for one attention module with its head outputs held fixed: the concatenated head outputs H [N, d]
+    (drawn like the module input, tensor id 5) and the output projection W_O [d, d] (tensor id 6, storage dtype)."""
+    H = make_activations(cfg, layer, device, tokens, tensor_id=5)
+    wo = standard_variates(module_seed(cfg, layer), 6, cfg.d * cfg.d, "gauss", device).view(cfg.d, cfg.d) * cfg.weight_std
+    return H, wo.to(storage_dtype(cfg))
+
+
 def make_importances(cfg: ModuleConfig, device="cpu") -> torch.Tensor:
     """A seeded stand-in for the per-layer importances I_l (float64, positive, mildly depth dependent)."""
     u = _unit_open(uniform_bits(module_seed(cfg, 0), 9, 0, cfg.layers, device))

@@ -175,6 +175,10 @@ def test_linear_refit(group):
     ref = O.restricted_refit(np64(R), np64(G), keep_cols, 0.37)
     assert relerr(np64(W), ref) < 1e-6
     assert np.all(np64(W)[:, keep_cols == 0] == 0.0)
+    # relative ridge: rho * trace(G) / dim(G) of the FULL system, computed on the device
+    W = api.sp_linear_refit(R.to(DEV), G.to(DEV), mask_u.to(DEV), k, 0.05, group=group, precise=True, rho_relative=True)
+    ref = O.restricted_refit(np64(R), np64(G), keep_cols, O.effective_ridge(np64(G), 0.05, True))
+    assert relerr(np64(W), ref) < 1e-6
 
 
 # ------------------------------------------------------------------------------------------------ scores

@@ -60,3 +60,30 @@ def test_temperature_search_picks_the_smaller_loss():
     X, W1, W2 = _inputs(0)
     rep = res.reports[-1]
     assert rep["res_out"] >= 0 and rep["res_in"] >= 0 and np.isfinite(pipeline.module_loss(res, 1.0))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_attention_head_pruning_matches_oracle(dtype):
+    """Head scores, top-k heads and the W_O recovery on the kept heads, composed from the library calls, against the
+    same composition of oracle functions."""
+    N, d, H = 900, 96, 8
+    dh = d // H
+    Hout = (synth.standard_variates(71, 1, N * d, "gauss").view(N, d)).to(dtype)
+    scale = 0.2 + synth.standard_variates(71, 5, H, "gauss").abs().repeat_interleave(dh)      # heads of unequal weight
+    Wo = (synth.standard_variates(71, 2, d * d, "gauss").view(d, d) * 0.1 * scale[None, :]).float()
+    Ypre = (Hout.float() @ Wo.T).to(dtype)
+    k = 5
+    mask, W_new, scores = pipeline.prune_attention_heads(Hout.to(DEV), Ypre.to(DEV), Wo.to(DEV), H, k, rho=0.1,
+                                                         token_chunk=400)
+    tol = 1e-5 if dtype == torch.float32 else 2e-3
+    Hd, Yd, Wd = np64(Hout.float()).T, np64(Ypre.float()).T, np64(Wo)
+    G = Hd @ Hd.T
+    R = Yd @ Hd.T
+    s_or, _ = O.wanda_scores(Wd, colsq=np.diag(G), kind="l2", group=dh)
+    assert relerr(np64(scores), s_or) < tol
+    m_ref, _ = O.topk_mask(scores.cpu().numpy(), k)          # the integer decision in the GPU's precision
+    assert np.array_equal(mask.cpu().numpy(), m_ref) and int(mask.sum()) == k
+    keep_cols = np.repeat(mask.cpu().numpy(), dh)
+    ref = O.restricted_refit(R, G, keep_cols, O.effective_ridge(G, 0.1, True))
+    assert relerr(np64(W_new), ref) < tol
+    assert np.all(np64(W_new)[:, keep_cols == 0] == 0.0)
