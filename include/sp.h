@@ -210,7 +210,8 @@ sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* i
  * current); make that first call outside any stream capture.
  * Sharing: all calls on one device use the same array.  Calls on the same stream are ordered and safe; two calls that
  * may overlap on the GPU (different streams without an ordering between them) race on it.  The array keeps the last
- * call's partial sums; no call reads a value it did not write itself, so nothing has to be cleared.
+ * call's partial sums; no call reads a partial sum it did not write itself, and the few arrival counters at its end,
+ * which must start at zero, are cleared on the stream at the start of every call.
  * The call itself performs no device or host allocation and calls no allocating library routine.
  */
 #define SP_STATIC_SCORES_MAX_COLS 32768
