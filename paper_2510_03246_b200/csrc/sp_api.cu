@@ -186,7 +186,8 @@ bool make_assist(SolveAssist& a) {
   return cudaStreamCreateWithFlags(&a.stream, cudaStreamNonBlocking) == cudaSuccess &&
          cudaEventCreateWithFlags(&a.panel_done, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&a.rest_done[0], cudaEventDisableTiming) == cudaSuccess &&
-         cudaEventCreateWithFlags(&a.rest_done[1], cudaEventDisableTiming) == cudaSuccess;
+         cudaEventCreateWithFlags(&a.rest_done[1], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.near_done, cudaEventDisableTiming) == cudaSuccess;
 }
 SideStream* side_stream() {
   static SideStream table[64];
@@ -696,6 +697,14 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     CU(cudaEventRecord(side->fork, s));
     CU(cudaStreamWaitEvent(sa, side->fork, 0));
   }
+  // The long chain (W2, on the caller's stream) is queued first: queuing the W1 chain takes the host more than half a
+  // millisecond, during which the caller's stream would otherwise sit empty.  (Without a side stream both run on
+  // the caller's stream and the order does not matter.)
+  CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
+  if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
+                                    side ? &side->assist_main : nullptr));
+  else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
+                                    side ? &side->assist_main : nullptr));
   CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
   if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
                                     side ? &side->assist_side : nullptr));
@@ -703,11 +712,6 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
                                     side ? &side->assist_side : nullptr));
   if (side) CU(cudaEventRecord(side->join, sa));
   bool joined = side == nullptr;
-  CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
-  if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
-                                    side ? &side->assist_main : nullptr));
-  else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
-                                    side ? &side->assist_main : nullptr));
 
   // ---- 2. unit scores and layer importance
   if (prm->score_kind == SP_SCORE_LEMMA1) {

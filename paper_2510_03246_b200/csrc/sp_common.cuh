@@ -111,6 +111,7 @@ int64_t chol_tc_pad(int64_t n);
 struct SolveAssist {
   cudaStream_t stream;
   cudaEvent_t panel_done, rest_done[2];
+  cudaEvent_t near_done;   // factorisation: the first two block columns of a step's trailing update have landed
 };
 // dinv must have room for ceil(n / 128) + 1 pairs of 128 x 128 blocks (the last pair is scratch).
 // m_extra > 0: A has m_extra more rows below row n (same lda), the right-hand sides B of a system X L^T = B; they

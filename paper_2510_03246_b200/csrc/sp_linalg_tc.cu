@@ -640,8 +640,9 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     // last block with appended rows: their panel runs on `stream`, behind the assisting stream's last update
     if (assist && rem <= 0 && kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
     if (assist && rem > 0) {
-      // next diagonal block: needs the trailing update of step kb - 1 (assisting stream)
-      if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
+      // next diagonal block: it reads blocks (kb+1, kb) and (kb+1, kb+1), i.e. the first two block columns of the
+      // trailing update of step kb - 1, which that step issues first and signals on their own
+      if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->near_done, 0));
       const int nb2 = (int)(rem < TB ? rem : TB);
       {
         count_launch();
@@ -673,10 +674,32 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       sg.b_k[q] = (int32_t)(kPartB[q] * np + k0);
     }
     float* A22 = A + (k0 + nb) * lda + (k0 + nb);
-    sp_status st = gemm_tc(prow, rem, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1}, OutOperand{A22, SP_F32, lda},
-                           true, status_dev, sb, &sg,
-                           ((double)rem * (double)rem + 2.0 * (double)m_extra * (double)rem) * (double)nb);
-    if (st != SP_OK) return st;
+    constexpr int64_t kNear = 2 * TB;     // block columns of the update that the next step's chain kernels read
+    if (assist && rem > kNear) {
+      // two launches: the first two block columns (all rows below), signalled at once, then the rest
+      tb.mnext = kNear;
+      sp_status st = gemm_tc(prow, kNear, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1},
+                             OutOperand{A22, SP_F32, lda}, true, status_dev, sb, &sg,
+                             (2.0 * (double)prow * (double)kNear - (double)kNear * (double)kNear) * (double)nb);
+      if (st != SP_OK) return st;
+      SP_CUDA_OK(cudaEventRecord(assist->near_done, sb));
+      TcOperand fa{P + (k0 + nb + kNear) * ldp, ldp, true}, fb{P + (k0 + nb + kNear) * ldp, ldp, true};
+      fa.kext = fb.kext = ldp;
+      fa.mnext = prow - kNear;
+      fb.mnext = rem - kNear;
+      float* Afar = A22 + kNear * lda + kNear;
+      const double fr = (double)(rem - kNear);
+      st = gemm_tc(prow - kNear, rem - kNear, TB, -1.f, fa, fb, 1.f, Operand{Afar, SP_F32, lda, 1},
+                   OutOperand{Afar, SP_F32, lda}, true, status_dev, sb, &sg,
+                   (fr * fr + 2.0 * (double)m_extra * fr) * (double)nb);
+      if (st != SP_OK) return st;
+    } else {
+      sp_status st = gemm_tc(prow, rem, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1},
+                             OutOperand{A22, SP_F32, lda}, true, status_dev, sb, &sg,
+                             ((double)rem * (double)rem + 2.0 * (double)m_extra * (double)rem) * (double)nb);
+      if (st != SP_OK) return st;
+      if (assist) SP_CUDA_OK(cudaEventRecord(assist->near_done, sb));
+    }
     if (assist) {
       SP_CUDA_OK(cudaEventRecord(assist->rest_done[kb & 1], sb));
       rec[kb & 1] = true;
