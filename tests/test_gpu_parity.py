@@ -412,6 +412,8 @@ STEP_CASES = [
     (SMALL_BF16, 0, "wanda_l2", "paper", False, True),
     (SMALL_BF16, 512, "wanda_l1", "exact", True, True),
     (SMALL_BF16, 512, "lemma1", "paper", False, False),
+    # the smallest workload at its full size (d = 768, n = 3072, 2048 tokens, fp32), default chunking
+    (synth.CONFIGS["C1"], 0, "wanda_l2", "paper", False, True),
 ]
 _KIND = {"wanda_l2": api.SP_SCORE_WANDA_L2, "wanda_l1": api.SP_SCORE_WANDA_L1, "lemma1": api.SP_SCORE_LEMMA1}
 _RULE = {"paper": api.SP_Z_PAPER, "exact": api.SP_Z_EXACT}
