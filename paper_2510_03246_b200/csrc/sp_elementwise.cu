@@ -461,7 +461,10 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
   }
 }
 
-// init pass: A = phi(Z) in storage dtype, optional storage copy of Z, |A| column partials
+// init pass: A = phi(Z) in storage dtype, optional storage copy of Z, |A| column partials.
+// A thread owns 4 consecutive channels and walks its rows four at a time (16-byte loads of all four rows in flight
+// before the first store, as in the fused update); |A| is summed in fp32 over the four rows of a round and in fp64
+// across rounds.
 __global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__ Z, float* gate_io, void* A_out,
                                                        void* Zb_out, int32_t out_dtype, int64_t T, int64_t n,
                                                        double* absA_part, int32_t row_blocks) {
@@ -471,29 +474,72 @@ __global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__
   const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
   const int64_t r_end = (r_begin + rows_per < T) ? r_begin + rows_per : T;
   const int cnt = (n - c0 >= 4) ? 4 : (int)(n - c0);
+  const bool vec = (n % 4 == 0);
   double cs[4] = {0.0, 0.0, 0.0, 0.0};
-  for (int64_t r = r_begin; r < r_end; ++r) {
-    const int64_t e = r * n + c0;
-    for (int q = 0; q < cnt; ++q) {
-      const float z = Z[e + q];
-      float a;
-      if (gate_io) {       // gated module: the buffer holds the gate pre-activation, SiLU of it replaces it
-        const float zg = gate_io[e + q];
-        const float gt = zg / (1.f + expf(-zg));
-        gate_io[e + q] = gt;
-        a = gt * z;
-      } else {
-        a = fmaxf(z, 0.f);
-      }
-      cs[q] += (double)fabsf(a);
-      if (out_dtype == SP_BF16) {
-        reinterpret_cast<__nv_bfloat16*>(A_out)[e + q] = __float2bfloat16_rn(a);
-        if (Zb_out) reinterpret_cast<__nv_bfloat16*>(Zb_out)[e + q] = __float2bfloat16_rn(z);
-      } else {
-        reinterpret_cast<float*>(A_out)[e + q] = a;
-        if (Zb_out) reinterpret_cast<float*>(Zb_out)[e + q] = z;
+  auto load4 = [&](const float* base, int64_t e, float* v) {
+    if (vec) {
+      const float4 x = *reinterpret_cast<const float4*>(base + e);
+      v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+    } else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) v[q] = (q < cnt) ? base[e + q] : 0.f;
+    }
+  };
+  auto store_out = [&](void* base, int64_t e, const float* v) {
+    if (vec) {
+      store4(base, out_dtype, e, v);
+    } else {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q < cnt) {
+          if (out_dtype == SP_BF16) reinterpret_cast<__nv_bfloat16*>(base)[e + q] = __float2bfloat16_rn(v[q]);
+          else reinterpret_cast<float*>(base)[e + q] = v[q];
+        }
       }
     }
+  };
+  for (int64_t r0 = r_begin; r0 < r_end; r0 += 4) {
+    float z[4][4], zg[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int64_t r = r0 + i;
+      if (r < r_end) {
+        load4(Z, r * n + c0, z[i]);
+        if (gate_io) load4(gate_io, r * n + c0, zg[i]);
+      }
+    }
+    float ps[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int64_t r = r0 + i;
+      if (r >= r_end) continue;
+      const int64_t e = r * n + c0;
+      float a[4];
+      if (gate_io) {       // gated module: the buffer holds the gate pre-activation, SiLU of it replaces it
+        float gt[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          gt[q] = zg[i][q] / (1.f + expf(-zg[i][q]));
+          a[q] = gt[q] * z[i][q];
+        }
+        if (vec) {
+          *reinterpret_cast<float4*>(gate_io + e) = make_float4(gt[0], gt[1], gt[2], gt[3]);
+        } else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (q < cnt) gate_io[e + q] = gt[q];
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) a[q] = fmaxf(z[i][q], 0.f);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) ps[q] += (q < cnt) ? fabsf(a[q]) : 0.f;
+      store_out(A_out, e, a);
+      if (Zb_out) store_out(Zb_out, e, z[i]);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) cs[q] += (double)ps[q];
   }
   if (absA_part)
     for (int q = 0; q < cnt; ++q) absA_part[(int64_t)blockIdx.y * n + c0 + q] = cs[q];
