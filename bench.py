@@ -317,6 +317,10 @@ def main():
         hH, hWo = synth.make_attention_inputs(cfg, layer)
         hH = hH.pin_memory(); hWo = hWo.pin_memory()
         k_heads = max(1, cfg.heads - int(cfg.heads * cfg.sparsity + 0.5))
+        # results come back into pinned host buffers
+        oW1 = torch.empty(cfg.n, cfg.d, dtype=torch.float32).pin_memory(); oW2 = torch.empty(cfg.d, cfg.n, dtype=torch.float32).pin_memory()
+        omask = torch.empty(cfg.n, dtype=torch.uint8).pin_memory()
+        oWo = torch.empty(cfg.d, cfg.d, dtype=torch.float32).pin_memory(); ohm = torch.empty(cfg.heads, dtype=torch.uint8).pin_memory()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
@@ -327,7 +331,8 @@ def main():
         api.sp_struct_scores(api.SP_SCORE_WANDA_L2, cfg.n, W=m2.W2_0, colsq=m2.G_A, colsq_stride=cfg.n + 1)
         for _ in range(iters):
             m2.sp_admm_step(prm)
-        oW1 = m2.W1.cpu(); oW2 = m2.W2.cpu(); omask = m2.mask.cpu()
+        oW1.copy_(m2.W1, non_blocking=True); oW2.copy_(m2.W2, non_blocking=True); omask.copy_(m2.mask, non_blocking=True)
+        torch.cuda.synchronize()
         t_ffn = time.perf_counter()
         # attention module: pre-trained output of the projection, head scores, head mask, W_O recovery on the kept heads
         dH = hH.to(dev, non_blocking=True); dWo = hWo.to(dev, non_blocking=True)
@@ -335,7 +340,7 @@ def main():
         api.sp_gemm(dH, dWo, Ya, transB=True, use_tensor_cores=(dH.dtype == torch.bfloat16))
         hmask, Wo_new, _ = pipeline.prune_attention_heads(dH, Ya, dWo.float(), cfg.heads, k_heads, rho=cfg.rho,
                                                           token_chunk=args.chunk)
-        oWo = Wo_new.cpu(); ohm = hmask.cpu()
+        oWo.copy_(Wo_new, non_blocking=True); ohm.copy_(hmask, non_blocking=True)
         torch.cuda.synchronize()
         t1 = time.perf_counter()
         m2.check_status()
