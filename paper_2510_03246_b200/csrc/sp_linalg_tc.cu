@@ -374,8 +374,8 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
       At[k][i] = xv[q].x; At[k + 1][i] = xv[q].y; At[k + 2][i] = xv[q].z; At[k + 3][i] = xv[q].w;
     }
   }
-  const bool staged = stage_block_wait(bar, 0);
-  __syncthreads();
+  // (the verdict is made uniform over the block: a thread whose wait ran out must not leave while others go on)
+  const bool staged = __syncthreads_and(stage_block_wait(bar, 0) ? 1 : 0) != 0;
   if (!staged) {   // the copies did not land in time: report and leave X untouched
     if (t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 10);
     return;
@@ -435,8 +435,7 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
 #pragma unroll
       for (int j = 0; j < 4; ++j) At[c0 + j][4 * ty + r] = (c0 + j < nb) ? acc[r][j] : 0.f;
     for (int e = t; e < (TB - nb) * TB; e += PA_THREADS) Bn[nb + e / TB][e % TB] = 0.f;
-    const bool staged2 = stage_block_wait(bar + 1, 0);
-    __syncthreads();
+    const bool staged2 = __syncthreads_and(stage_block_wait(bar + 1, 0) ? 1 : 0) != 0;
     if (!staged2) {
       if (t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 12);
       return;
@@ -523,8 +522,7 @@ __global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
     const int i = e / TB, k = e % TB;
     At[k][i] = (i0 + i < nb2) ? A21[(int64_t)(i0 + i) * lda + k] : 0.f;
   }
-  const bool staged = stage_block_wait(bar, 0);
-  __syncthreads();
+  const bool staged = __syncthreads_and(stage_block_wait(bar, 0) ? 1 : 0) != 0;
   if (!staged && t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 11);
   // (a CTA whose copies did not land still takes part in the cluster barrier below; its rows are then wrong and the
   //  status says so)
