@@ -43,6 +43,7 @@ def parse():
     ap.add_argument("--chunk", type=int, default=32768)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-fixed-mask", action="store_true", help="skip the fixed-mask variants of the step")
     ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
     return ap.parse_args()
 
@@ -302,6 +303,38 @@ def main():
                         if v["bytes"] and v["ms"] else {})}
                  for k, v in prof.items() if v["records"]}
 
+    # ---- the variant with the mask fixed after the first iterations (Algorithm 1: Step 3 fixes the masks before the
+    # SparseLLM iterations): the same module stepped without re-selection, and its continuation on the kept channels
+    fixed = None
+    if not args.no_fixed_mask and rank == 0:
+        from paper_2510_03246_b200 import pipeline
+
+        def time_steps(m, prm_v, n_warm=2, n_timed=4):
+            for _ in range(n_warm):
+                m.sp_admm_step(prm_v)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(n_timed):
+                m.sp_admm_step(prm_v)
+            b.record()
+            torch.cuda.synchronize()
+            m.check_status()
+            return a.elapsed_time(b) / n_timed
+
+        api.sp_profile_begin(0)
+        prm_fix = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk, reselect_mask=False,
+                                 skip_scores=True)
+        ms_full = time_steps(mod, prm_fix)
+        cmod, _ = pipeline.compact_module(mod)
+        ms_comp = time_steps(cmod, prm_fix)
+        del cmod
+        torch.cuda.empty_cache()
+        fixed = {"note": "steps with the mask kept fixed (no unrestricted recovery, no scores): on the full-width "
+                         "module, and continued on the kept channels only (accumulators k x k)",
+                 "full_width_ms_per_step": ms_full, "full_width_iterations_per_s": 1e3 / ms_full,
+                 "kept_channels_ms_per_step": ms_comp, "kept_channels_iterations_per_s": 1e3 / ms_comp}
+
     # ---- end to end: host buffers in, host results out, one whole module job of cfg.iters iterations
     e2e = None
     if not args.no_e2e:
@@ -367,7 +400,7 @@ def main():
             "config": {"workload": workload_name(cfg), "token_chunk": args.chunk,
                        "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
                        "parallelism": f"modules x{world} (independent, no collective)"},
-            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e, "cpu_baseline": cpu,
+            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e, "cpu_baseline": cpu, "fixed_mask": fixed,
             "breakdown": breakdown}
     print(json.dumps(line))
     if world > 1:

@@ -115,7 +115,9 @@ typedef struct {
   int32_t refit;           /* 1: recovery solver on the kept support (Algorithm 2); 0: plain M (.) W               */
   int64_t token_chunk;     /* tokens per streamed chunk (0 = library default)                                      */
   int32_t compute_objective; /* 1: also report alpha|Ypre-W2A|^2 (one more product per token chunk)                 */
-  int32_t reserved;
+  int32_t skip_scores;     /* 1 (needs reselect_mask = 0 and refit = 1): the mask is fixed, so the unrestricted
+                              recovery W2~ and the unit scores, which only serve the mask selection, are not computed;
+                              st->scores and st->importance keep their previous values                              */
 } sp_admm_params;
 
 /* Device-side report of one step (all double). */

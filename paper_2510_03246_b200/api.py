@@ -57,7 +57,7 @@ class SpAdmmParams(C.Structure):
     _fields_ = [("alpha", C.c_double), ("beta", C.c_double), ("rho", C.c_double), ("rho_relative", C.c_int32),
                 ("z_rule", C.c_int32), ("dual_mode", C.c_int32), ("score_kind", C.c_int32), ("k_keep", C.c_int64),
                 ("reselect_mask", C.c_int32), ("refit", C.c_int32), ("token_chunk", C.c_int64),
-                ("compute_objective", C.c_int32), ("reserved", C.c_int32)]
+                ("compute_objective", C.c_int32), ("skip_scores", C.c_int32)]
 
 
 class SpScoreInputs(C.Structure):
@@ -366,11 +366,12 @@ class AdmmParams:
     refit: bool = True
     token_chunk: int = 0
     compute_objective: bool = False
+    skip_scores: bool = False       # fixed mask (reselect_mask False, refit True): skip W2~ and the scores
 
     def to_c(self) -> SpAdmmParams:
         return SpAdmmParams(self.alpha, self.beta, self.rho, int(self.rho_relative), self.z_rule, int(self.dual_mode),
                             self.score_kind, int(self.k_keep), int(self.reselect_mask), int(self.refit),
-                            int(self.token_chunk), int(self.compute_objective), 0)
+                            int(self.token_chunk), int(self.compute_objective), int(self.skip_scores))
 
 
 class FfnModule:

@@ -677,6 +677,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   if (prm->z_rule != SP_Z_PAPER && prm->z_rule != SP_Z_EXACT) return SP_ERR_UNSUPPORTED;
   if (prm->score_kind < SP_SCORE_WANDA_L2 || prm->score_kind > SP_SCORE_LEMMA1) return SP_ERR_UNSUPPORTED;
   if (m->act == SP_ACT_SWIGLU && prm->score_kind == SP_SCORE_LEMMA1) return SP_ERR_UNSUPPORTED;
+  if (prm->skip_scores && (prm->reselect_mask || !prm->refit)) return SP_ERR_INVALID_ARG;
   const int32_t cdt = m->X.dtype;
   if (!ws || ws_bytes < plan_admm(nullptr, d, n, N, prm->token_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
   AdmmPlan p = plan_admm(ws, d, n, N, prm->token_chunk, cdt);
@@ -700,11 +701,16 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   // The long chain (W2, on the caller's stream) is queued first: queuing the W1 chain takes the host more than half a
   // millisecond, during which the caller's stream would otherwise sit empty.  (Without a side stream both run on
   // the caller's stream and the order does not matter.)
+  const bool skip_scores = prm->skip_scores != 0;   // fixed mask: W2~ and the scores serve nothing
   CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
-  if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
-                                    side ? &side->assist_main : nullptr));
-  else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
-                                    side ? &side->assist_main : nullptr));
+  if (skip_scores) {
+  } else if (bf16) {
+    SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
+                            side ? &side->assist_main : nullptr));
+  } else {
+    SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
+                             side ? &side->assist_main : nullptr));
+  }
   CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
   if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
                                     side ? &side->assist_side : nullptr));
@@ -714,7 +720,8 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   bool joined = side == nullptr;
 
   // ---- 2. unit scores and layer importance
-  if (prm->score_kind == SP_SCORE_LEMMA1) {
+  if (skip_scores) {
+  } else if (prm->score_kind == SP_SCORE_LEMMA1) {
     if (!joined) { CU(cudaStreamWaitEvent(s, side->join, 0)); joined = true; }   // this score reads W1~
     // b = W1~ X, c = d = t = z^pre = W1_0 X, written through G_X:  T0 = W1_0 G_X
     MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, gx{st->G_X, SP_F32, d}, t0{p.T0, SP_F32, d};

@@ -93,6 +93,43 @@ def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_unit
     return results, r, k_keep, {"importance_s": t1 - t0, "admm_s": t2 - t1, "layers_per_s": len(mine) / max(t2 - t0, 1e-9)}
 
 
+def compact_module(mod: api.FfnModule):
+    """Continuation of a module whose mask is fixed (the flow of Algorithm 1, where Step 3 fixes the masks before the
+    SparseLLM iterations): a new module that holds only the kept channels.  With a fixed mask the pruned channels
+    never enter a kept channel's updates again (their columns of W2 and rows of W1 are zero), so the iterations can
+    go on at width k instead of n: accumulators k x k instead of n x n, no unrestricted recovery, no scores.
+    Pure data movement (gathers); returns (compact module, kept channel indices).  Run it with
+    AdmmParams(k_keep=k, reselect_mask=False, skip_scores=True); with rho_relative the ridge of the W2 recovery is
+    then relative to the trace over the kept channels only."""
+    idx = torch.nonzero(mod.mask, as_tuple=False).flatten()
+    k = int(idx.numel())
+    new = api.FfnModule(mod.X, mod.W1_0[idx], mod.W2_0[:, idx], dual_mode=mod.U is not None,
+                        token_chunk=mod.token_chunk, overlap_k=k, Wg_0=mod.Wg_0[idx] if mod.Wg_0 is not None else None)
+    new.Ypre = mod.Ypre
+    new.Z.copy_(mod.Z[:, idx])
+    if mod.U is not None:
+        new.U.copy_(mod.U[:, idx])
+    if mod.Gate is not None:
+        new.Gate.copy_(mod.Gate[:, idx])
+    new.G_X = mod.G_X
+    new.G_A.copy_(mod.G_A[idx][:, idx])
+    new.R1.copy_(mod.R1[idx])
+    new.R2.copy_(mod.R2[:, idx])
+    new.absA.copy_(mod.absA[idx])
+    new.mask.fill_(1)
+    new.iteration = mod.iteration
+    return new, idx
+
+
+def expand_weights(cmod: api.FfnModule, idx: torch.Tensor, n: int):
+    """W1 [n, d] and W2 [d, n] of the full module from a compact continuation (pruned rows / columns zero)."""
+    W1 = torch.zeros(n, cmod.d, dtype=torch.float32, device=cmod.dev)
+    W2 = torch.zeros(cmod.d, n, dtype=torch.float32, device=cmod.dev)
+    W1[idx] = cmod.W1
+    W2[:, idx] = cmod.W2
+    return W1, W2
+
+
 def prune_attention_heads(H: torch.Tensor, Ypre: torch.Tensor, W_O: torch.Tensor, n_heads: int, k_heads: int,
                           rho: float = 0.1, token_chunk: int = 32768):
     """Head pruning of one attention module with its head outputs held fixed (Algorithm 2, attention branch, W_O part;

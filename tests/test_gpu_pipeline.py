@@ -87,3 +87,47 @@ def test_attention_head_pruning_matches_oracle(dtype):
     ref = O.restricted_refit(R, G, keep_cols, O.effective_ridge(G, 0.1, True))
     assert relerr(np64(W_new), ref) < tol
     assert np.all(np64(W_new)[:, keep_cols == 0] == 0.0)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_fixed_mask_continuation_on_kept_channels(bf16):
+    """After the mask is fixed, the iterations continue on the kept channels only.  Checked two ways: against the
+    oracle run on the reduced module (teacher-forced from the compact state), and against the full-width module
+    stepped with the same fixed mask (absolute ridge, so that both solve the same systems)."""
+    import copy
+    from tests._util import oracle_state_from_gpu
+    cfg = synth.scaled(synth.CONFIGS["C2" if bf16 else "C1"], d=136, n=520, tokens=900, sparsity=0.5, outlier_frac=0.02)
+    X = synth.make_activations(cfg, 0).to(DEV)
+    W1, W2 = (w.to(DEV) for w in synth.make_weights(cfg, 0))
+    tol = TOL[X.dtype]
+    k = cfg.k_keep
+    full = api.FfnModule(X, W1, W2)
+    full.sp_ffn_init()
+    p_sel = api.AdmmParams(k_keep=k, rho=0.05, rho_relative=False)
+    full.sp_admm_step(p_sel)                                   # this step selects the mask
+    comp, idx = pipeline.compact_module(full)
+    assert int(idx.numel()) == k and torch.equal(full.mask.nonzero().flatten(), idx)
+    p_fix_full = api.AdmmParams(k_keep=k, rho=0.05, rho_relative=False, reselect_mask=False, skip_scores=True)
+    p_fix_comp = api.AdmmParams(k_keep=k, rho=0.05, rho_relative=False, reselect_mask=False, skip_scores=True)
+    for it in range(2):
+        # oracle on the reduced module, restarted from the compact state
+        st = oracle_state_from_gpu(comp)
+        st.mask = np.ones(k, np.uint8)
+        p_or = O.AdmmParams(k_keep=k, rho=0.05, rho_relative=False, reselect_mask=False)
+        Xo, Yo = np64(X).T, np64(comp.Ypre).T
+        comp.sp_admm_step(p_fix_comp)
+        full.sp_admm_step(p_fix_full)
+        torch.cuda.synchronize()
+        comp.check_status(); full.check_status()
+        O.admm_step(st, Xo, Yo, np64(comp.W1_0), p_or)
+        assert relerr(np64(comp.W1), st.W1) < tol and relerr(np64(comp.W2), st.W2) < tol
+        assert relerr(np64(comp.Z).T, st.Z) < tol
+        assert relerr(np64(comp.G_A), st.G_A) < tol and relerr(np64(comp.R1), st.R1) < tol
+        # the full-width module with the same fixed mask walks the same path on the kept channels
+        W1e, W2e = pipeline.expand_weights(comp, idx, cfg.n)
+        assert relerr(np64(W1e), np64(full.W1)) < 2 * tol and relerr(np64(W2e), np64(full.W2)) < 2 * tol
+        assert relerr(np64(comp.Z), np64(full.Z[:, idx])) < 2 * tol
+    # skip_scores needs a fixed mask and the recovery on the kept support
+    with pytest.raises(api.SpError) as e:
+        full.sp_admm_step(api.AdmmParams(k_keep=k, skip_scores=True))
+    assert e.value.code == 1
