@@ -31,7 +31,7 @@ __device__ __forceinline__ float rsqrt_refined(float x) {
 constexpr int DIAG_TPAD = TB + 1;
 constexpr size_t DIAG_SMEM = (size_t)TB * DIAG_TPAD * sizeof(float);
 
-// Factorise the nb x nb diagonal block at A (lower triangle), write L back, and write inv(L) and its transpose to
+// Factorise the nb x nb diagonal block at A (lower triangle, left as it is) and write inv(L) and its transpose to
 // dinv[0 : TB*TB] and dinv[TB*TB : 2*TB*TB] (row-major TB x TB, zero above / below the diagonal respectively,
 // identity on the padding rows nb..TB-1).  A non-positive pivot is reported once through `status` and replaced by 1.
 //
@@ -229,18 +229,8 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
       dinv[i * TB + c] = T[i][c];
       dinv[TB * TB + i * TB + c] = T[c][i];      // row i of the transpose = column i of inv(L)
     }
-  // ---- store L (lower triangle of the nb x nb block)
-  __syncthreads();
-  if (active) {
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int s = 0; s < 4; ++s)
-        if (4 * bj + s <= 4 * bi + r) T[4 * bi + r][4 * bj + s] = lcol[r][s];
-  }
-  __syncthreads();
-  for (int i = warp; i < nb; i += NWARP)
-    for (int c = lane; c <= i; c += 32) A[(int64_t)i * lda + c] = T[i][c];
+  // L itself is not written back: the solves use inv(L) of the diagonal blocks and the blocks of L below them only.
+  (void)lcol;
 }
 
 __device__ __forceinline__ void split3(float v, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
