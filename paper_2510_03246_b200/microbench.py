@@ -46,6 +46,9 @@ def gemm_cases(reps, warm):
         ("G_A += A^T A (lower)", N, N, T, False, False, f32, 1.0, True),
         ("R2 += Ypre^T A", D, N, T, False, False, f32, 1.0, False),
         ("R1 += Z^T X", N, D, T, False, False, f32, 1.0, False),
+        ("R2 with Ypre stored transposed", D, N, T, True, False, f32, 1.0, False),
+        ("R1 with X stored transposed", N, D, T, False, True, f32, 1.0, False),
+        ("G_A with A stored transposed", N, N, T, True, True, f32, 1.0, True),
         ("solve update (K = 6 x 128)", 2048, 4096, 768, True, True, f32, 1.0, False),
     ]
     for name, M, Nn, K, ak, bk, cdt, beta, lower in cases:
