@@ -44,6 +44,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fixed-mask", action="store_true", help="skip the fixed-mask variants of the step")
+    ap.add_argument("--dual", action="store_true", help="run with the scaled dual variable U (dual_mode = 1)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
     return ap.parse_args()
 
@@ -217,14 +218,14 @@ def main():
     X = synth.make_activations(cfg, layer, device=dev)
     W1_0, W2_0 = synth.make_weights(cfg, layer, device=dev)
     Wg_0 = synth.make_gate_weights(cfg, layer, device=dev) if cfg.act == "swiglu" else None
-    mod = api.FfnModule(X, W1_0, W2_0, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
+    mod = api.FfnModule(X, W1_0, W2_0, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
     I_all = synth.make_importances(cfg, device=dev)
     n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
     T_soft = float(I_all.abs().mean())
     mod.sp_ffn_init()
     torch.cuda.synchronize()
     mod.check_status()
-    prm = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk)
+    prm = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk, dual_mode=args.dual)
 
     def step():
         mod.sp_admm_step(prm)
@@ -324,7 +325,7 @@ def main():
 
         api.sp_profile_begin(0)
         prm_fix = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk, reselect_mask=False,
-                                 skip_scores=True)
+                                 skip_scores=True, dual_mode=args.dual)
         ms_full = time_steps(mod, prm_fix)
         cmod, _ = pipeline.compact_module(mod)
         ms_comp = time_steps(cmod, prm_fix)
@@ -358,7 +359,7 @@ def main():
         t0 = time.perf_counter()
         dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
         dWg = hWg.to(dev, non_blocking=True) if hWg is not None else None
-        m2 = api.FfnModule(dX, dW1, dW2, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=dWg)
+        m2 = api.FfnModule(dX, dW1, dW2, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=dWg)
         m2.sp_ffn_init()
         # this layer's share of pass 0: the importance of the pre-trained module
         api.sp_struct_scores(api.SP_SCORE_WANDA_L2, cfg.n, W=m2.W2_0, colsq=m2.G_A, colsq_stride=cfg.n + 1)
@@ -397,7 +398,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_name(cfg), "token_chunk": args.chunk,
+            "config": {"workload": workload_name(cfg), "token_chunk": args.chunk, "dual_mode": bool(args.dual),
                        "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
                        "parallelism": f"modules x{world} (independent, no collective)"},
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e, "cpu_baseline": cpu, "fixed_mask": fixed,
