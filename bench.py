@@ -10,8 +10,11 @@ calibration tokens in bf16, 50 % channel sparsity), synthetic seeded inputs gene
 With N > 1 GPUs every rank owns its own module (modules are independent once the kept counts are fixed), so the
 scaling is weak and the data path has no collective.
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (a deliberately plain fp64
-restatement of the paper; context only).
+Prints ONE JSON line (rank 0).  Besides the timed step (mask re-selected in every iteration) the line carries
+`fixed_mask` (the same module stepped without re-selection, and its continuation on the kept channels only), `e2e`
+(one whole pruned layer from and to pinned host buffers: the FFN module's iterations and the attention half with fixed
+head outputs) and `cpu_baseline` (the oracle on a token sample).  `--dual` runs with the scaled dual variable.
+`--impl reference` times the CPU oracle instead (a deliberately plain fp64 restatement of the paper; context only).
 """
 from __future__ import annotations
 
