@@ -145,7 +145,7 @@ template <typename T>
 sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_full,
                      const int32_t* idx, int64_t k, const double* rho_dev, float* W, int64_t ldw, SolveBufs& b,
                      int32_t* status, cudaStream_t stream, const SolveAssist* assist = nullptr,
-                     bool factor_lookahead = true) {
+                     bool split_lookahead = false) {
   const int64_t nn = idx ? k : n_full;
   ProfScope prof(PK_SOLVE, (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
   T* Gs = reinterpret_cast<T*>(b.Gs);
@@ -157,7 +157,7 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
     // the right-hand sides ride through the factorisation as m more rows (their forward substitution); the solve
     // proper is then only the backward sweep
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
-    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, factor_lookahead ? assist : nullptr, m));
+    SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, assist, m, split_lookahead));
     SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist, true, Gs, nn));
   } else {
     CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
@@ -760,10 +760,10 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     CU(cudaEventRecord(side->z1_done, side->stream));
   }
   if (prm->refit) {
-    // beside the z1 products the factorisation keeps to one stream: its lookahead kernel is a cluster of 8 CTAs,
-    // which finds no free group of SMs while the persistent GEMM CTAs hold most of them
+    // beside the z1 products the lookahead kernel of the factorisation runs as two launches of independent CTAs: a
+    // cluster of 8 would wait for a free group of SMs while the persistent GEMM CTAs hold most of them
     if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
-                                      side ? &side->assist_main : nullptr, !z1_ahead));
+                                      side ? &side->assist_main : nullptr, z1_ahead));
     else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
                                       side ? &side->assist_main : nullptr));
   } else {
@@ -799,7 +799,7 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
       CU(convert_matrix(p.W2b, SP_BF16, kp, p.W2cf, SP_F32, kp, d, k, s));
       CU(transpose_convert<float>(p.W2cf, kp, d, k, Rs, d, s));
       SPCHK(potrf_lower_tc(Gs, d, d, reinterpret_cast<float*>(p.sb.dinv), p.sb.P, status_dev, s,
-                           (side && !z1_ahead) ? &side->assist_main : nullptr, k));
+                           side ? &side->assist_main : nullptr, k, z1_ahead));
       SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s,
                            side ? &side->assist_main : nullptr, true, Gs, d));
       CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));

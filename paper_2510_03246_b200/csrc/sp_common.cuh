@@ -117,7 +117,8 @@ struct SolveAssist {
 // m_extra > 0: A has m_extra more rows below row n (same lda), the right-hand sides B of a system X L^T = B; they
 // are carried through the panels and trailing updates and hold X on return (P then needs n + m_extra rows).
 sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P, int32_t* status_dev,
-                         cudaStream_t stream, const SolveAssist* assist = nullptr, int64_t m_extra = 0);
+                         cudaStream_t stream, const SolveAssist* assist = nullptr, int64_t m_extra = 0,
+                         bool split_lookahead = false);   // lookahead kernel as two launches without a cluster
 // Xs holds TWO buffers of [m, 3 * kCholTcNB] bf16.
 // forward_done: X already holds the solution of the forward system (it rode along with the factorisation).
 // Lf / ldl (optional): the fp32 factor potrf_lower_tc left in A; with it the backward sweep updates the next block

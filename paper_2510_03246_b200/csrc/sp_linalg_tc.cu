@@ -494,9 +494,13 @@ __device__ __forceinline__ void cluster_meet() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-__global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
-    chol_next_diag_kernel(const float* __restrict__ A21, const float* __restrict__ A22, int64_t lda, int nb2,
-                          const float* __restrict__ dinv, float* LmT, float* S, int32_t* status) {
+// MODE 0: both stages in one launch, the CTAs being one cluster (they meet between the stages);
+// MODE 1 / MODE 2: the stages as two launches of 8 independent CTAs (for use beside persistent GEMM CTAs that hold
+// most SMs, where a cluster of 8 waits for a free group of SMs).
+template <int MODE>
+__device__ __forceinline__ void next_diag_body(const float* __restrict__ A21, const float* __restrict__ A22,
+                                               int64_t lda, int nb2, const float* __restrict__ dinv, float* LmT,
+                                               float* S, int32_t* status) {
   extern __shared__ __align__(128) float nm_smem[];
   float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(nm_smem);                       // Lt[k][c]
   float (*At)[NM_APAD] = reinterpret_cast<float (*)[NM_APAD]>(nm_smem + TB * TB);   // At[k][row]
@@ -504,49 +508,57 @@ __global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
   const int t = threadIdx.x;
   const int i0 = (int)blockIdx.x * NM_ROWS;
   const int tx = t & 31, ty = t >> 5;   // columns 4 tx .. 4 tx + 3; rows 2 ty, 2 ty + 1
-  // ---- stage 1: rows i0 .. i0 + 15 of Lm; Lt[k][c] = inv(L)[c][k] comes in by bulk copies
-  if (t == 0) stage_bar_init(bar);
-  __syncthreads();
-  if (t == 0) stage_block_issue(nm_smem, dinv + TB * TB, bar);
-  for (int e = t; e < NM_ROWS * TB; e += NM_THREADS) {
-    const int i = e / TB, k = e % TB;
-    At[k][i] = (i0 + i < nb2) ? A21[(int64_t)(i0 + i) * lda + k] : 0.f;
-  }
-  const bool staged = __syncthreads_and(stage_block_wait(bar, 0) ? 1 : 0) != 0;
-  if (!staged && t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 11);
-  // (a CTA whose copies did not land still takes part in the cluster barrier below; its rows are then wrong and the
-  //  status says so)
   float acc[2][4];
-#pragma unroll
-  for (int r = 0; r < 2; ++r)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[r][j] = 0.f;
-#pragma unroll 8
-  for (int k = 0; k < TB; ++k) {
-    const float2 a = *reinterpret_cast<const float2*>(&At[k][2 * ty]);
-    const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][4 * tx]);
-    const float av[2] = {a.x, a.y};
-    const float lv[4] = {l0.x, l0.y, l0.z, l0.w};
+  if (MODE != 2) {
+    // ---- stage 1: rows i0 .. i0 + 15 of Lm; Lt[k][c] = inv(L)[c][k] comes in by bulk copies
+    if (t == 0) stage_bar_init(bar);
+    __syncthreads();
+    if (t == 0) stage_block_issue(nm_smem, dinv + TB * TB, bar);
+    for (int e = t; e < NM_ROWS * TB; e += NM_THREADS) {
+      const int i = e / TB, k = e % TB;
+      At[k][i] = (i0 + i < nb2) ? A21[(int64_t)(i0 + i) * lda + k] : 0.f;
+    }
+    const bool staged = __syncthreads_and(stage_block_wait(bar, 0) ? 1 : 0) != 0;
+    if (!staged && t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 11);
+    // (a CTA whose copies did not land still goes on to the barrier below; its rows are then wrong and the status
+    //  says so)
 #pragma unroll
     for (int r = 0; r < 2; ++r)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
-  }
-  __syncthreads();   // everyone is done with At and Lt
+      for (int j = 0; j < 4; ++j) acc[r][j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < TB; ++k) {
+      const float2 a = *reinterpret_cast<const float2*>(&At[k][2 * ty]);
+      const float4 l0 = *reinterpret_cast<const float4*>(&Lt[k][4 * tx]);
+      const float av[2] = {a.x, a.y};
+      const float lv[4] = {l0.x, l0.y, l0.z, l0.w};
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int c = 4 * tx + j;
-    const float2 v = make_float2(acc[0][j], acc[1][j]);
-    *reinterpret_cast<float2*>(&At[c][2 * ty]) = v;                              // own rows, left operand of stage 2
-    *reinterpret_cast<float2*>(&LmT[(int64_t)c * TB + i0 + 2 * ty]) = v;         // for the other CTAs
+      for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[r][j] = fmaf(av[r], lv[j], acc[r][j]);
+    }
+    __syncthreads();   // everyone is done with At and Lt
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = 4 * tx + j;
+      const float2 v = make_float2(acc[0][j], acc[1][j]);
+      *reinterpret_cast<float2*>(&At[c][2 * ty]) = v;                              // own rows, left operand of stage 2
+      *reinterpret_cast<float2*>(&LmT[(int64_t)c * TB + i0 + 2 * ty]) = v;         // for the other CTAs
+    }
+    if (MODE == 1) return;
+    cluster_meet();
   }
-  cluster_meet();
   // ---- stage 2: rows i0 .. i0 + 15 of S; Lt[c][j] = Lm[j][c]
   {
     const float4* src = reinterpret_cast<const float4*>(LmT);
     float4* dst = reinterpret_cast<float4*>(nm_smem);
 #pragma unroll
     for (int q = 0; q < TB * TB / 4 / NM_THREADS; ++q) dst[t + q * NM_THREADS] = __ldcg(src + t + q * NM_THREADS);
+    if (MODE == 2)     // own rows of Lm come from the first launch
+      for (int e = t; e < NM_ROWS * TB; e += NM_THREADS) {
+        const int c = e / NM_ROWS, i = e % NM_ROWS;
+        At[c][i] = __ldcg(&LmT[(int64_t)c * TB + i0 + i]);
+      }
   }
   __syncthreads();
 #pragma unroll
@@ -577,6 +589,21 @@ __global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
   }
 }
 
+__global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
+    chol_next_diag_kernel(const float* __restrict__ A21, const float* __restrict__ A22, int64_t lda, int nb2,
+                          const float* __restrict__ dinv, float* LmT, float* S, int32_t* status) {
+  next_diag_body<0>(A21, A22, lda, nb2, dinv, LmT, S, status);
+}
+__global__ void __launch_bounds__(NM_THREADS)
+    chol_next_diag_stage1_kernel(const float* __restrict__ A21, int64_t lda, int nb2, const float* __restrict__ dinv,
+                                 float* LmT, int32_t* status) {
+  next_diag_body<1>(A21, nullptr, lda, nb2, dinv, LmT, nullptr, status);
+}
+__global__ void __launch_bounds__(NM_THREADS)
+    chol_next_diag_stage2_kernel(const float* __restrict__ A22, int64_t lda, int nb2, float* LmT, float* S) {
+  next_diag_body<2>(nullptr, A22, lda, nb2, nullptr, LmT, S, nullptr);
+}
+
 constexpr int kPartA[6] = {0, 0, 1, 0, 2, 1};
 constexpr int kPartB[6] = {0, 1, 0, 2, 0, 1};
 
@@ -585,7 +612,7 @@ constexpr int kPartB[6] = {0, 1, 0, 2, 0, 1};
 int64_t chol_tc_pad(int64_t n) { return (n + TB - 1) / TB * TB; }
 
 sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv, int32_t* status_dev,
-                         cudaStream_t stream, const SolveAssist* assist, int64_t m_extra) {
+                         cudaStream_t stream, const SolveAssist* assist, int64_t m_extra, bool split_lookahead) {
   __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
   const int64_t nblk = ceil_div(n, (int64_t)TB);
@@ -594,7 +621,11 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     if (cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM) !=
             cudaSuccess ||
         cudaFuncSetAttribute(chol_next_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NM_SMEM) !=
-            cudaSuccess)
+            cudaSuccess ||
+        cudaFuncSetAttribute(chol_next_diag_stage1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)NM_SMEM) != cudaSuccess ||
+        cudaFuncSetAttribute(chol_next_diag_stage2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)NM_SMEM) != cudaSuccess)
       return SP_ERR_CUDA;
     attr_set = true;
   }
@@ -635,9 +666,17 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       {
         count_launch();
         ProfScope prof(PK_PANEL_APPLY, 4.0 * TB * TB * TB, 0.0, stream);
-        chol_next_diag_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + k0,
-                                                                        A + (k0 + nb) * lda + (k0 + nb), lda, nb2, dk,
-                                                                        LmT, S, status_dev);
+        if (!split_lookahead) {
+          chol_next_diag_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + k0,
+                                                                          A + (k0 + nb) * lda + (k0 + nb), lda, nb2,
+                                                                          dk, LmT, S, status_dev);
+        } else {
+          chol_next_diag_stage1_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + k0, lda, nb2, dk,
+                                                                                 LmT, status_dev);
+          count_launch();
+          chol_next_diag_stage2_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + (k0 + nb), lda,
+                                                                                 nb2, LmT, S);
+        }
         if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
       }
       // the panel overwrites A21 in place: it starts behind the lookahead kernel
