@@ -545,11 +545,30 @@ __global__ void __launch_bounds__(256) init_act_kernel(const float* __restrict__
     for (int q = 0; q < cnt; ++q) absA_part[(int64_t)blockIdx.y * n + c0 + q] = cs[q];
 }
 
-__global__ void reduce_col_partials_kernel(const double* part, int32_t row_blocks, int64_t n, double* out, int acc) {
-  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x) {
-    double s = acc ? out[j] : 0.0;
-    for (int r = 0; r < row_blocks; ++r) s += part[(int64_t)r * n + j];
-    out[j] = s;
+// out[j] (+)= sum_r part[r, j]: a block takes 32 columns, its 8 warps take every 8th row block (four loads in flight
+// each), then the 8 partial sums of a column are added in a fixed order.
+__global__ void __launch_bounds__(256) reduce_col_partials_kernel(const double* __restrict__ part, int32_t row_blocks,
+                                                                  int64_t n, double* out, int acc) {
+  __shared__ double sm[8][33];
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int64_t j = (int64_t)blockIdx.x * 32 + cx;
+  double s = 0.0;
+  if (j < n) {
+    int r = ry;
+    for (; r + 24 < row_blocks; r += 32) {
+      const double v0 = part[(int64_t)r * n + j], v1 = part[(int64_t)(r + 8) * n + j];
+      const double v2 = part[(int64_t)(r + 16) * n + j], v3 = part[(int64_t)(r + 24) * n + j];
+      s += v0; s += v1; s += v2; s += v3;
+    }
+    for (; r < row_blocks; r += 8) s += part[(int64_t)r * n + j];
+  }
+  sm[ry][cx] = s;
+  __syncthreads();
+  if (ry == 0 && j < n) {
+    double tot = acc ? out[j] : 0.0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) tot += sm[q][cx];
+    out[j] = tot;
   }
 }
 
@@ -827,7 +846,8 @@ cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t 
   if (n == 0) return cudaSuccess;
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  reduce_col_partials_kernel<<<grid_for(n, 256), 256, 0, stream>>>(part, row_blocks, n, out, accumulate ? 1 : 0);
+  reduce_col_partials_kernel<<<(unsigned)ceil_div(n, (int64_t)32), 256, 0, stream>>>(part, row_blocks, n, out,
+                                                                                    accumulate ? 1 : 0);
   return cudaGetLastError();
 }
 
