@@ -844,6 +844,12 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     ua.grp_mask = p.grp_mask; ua.A_out = p.Ac; ua.Zb_out = bf16 ? p.Zb : nullptr;
     ua.out_dtype = cdt; ua.T = Tc; ua.n = n; ua.alpha = (float)prm->alpha; ua.beta = (float)prm->beta;
     ua.z_rule = prm->z_rule; ua.partial = p.partial; ua.absA_part = p.absA_part;
+    // bf16 storage: the update writes A transposed (channels x tokens), which makes the token dimension the
+    // contiguous one of both operands of A A^T and of the A operand of Ypre A^T; the row-major A is only needed
+    // when the objective is reported.  The row pitch is a multiple of 16 bytes.
+    const int64_t Tld = (Tc + 7) / 8 * 8;
+    const bool a_transposed = bf16 && n % 4 == 0 && !(rep_dev && prm->compute_objective) && Tld <= p.chunk;
+    if (a_transposed) { ua.At_out = p.Ac; ua.ldt = Tld; }
     const int nblk = fused_update_grid(Tc, n, &ua.row_blocks);
     CU(launch_fused_update(ua, s));
     if (rep_dev) CU(reduce_report(p.partial, nblk, rep_dev, ci > 0, prm->alpha, s));
@@ -856,8 +862,14 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     }
     CU(reduce_col_partials(p.absA_part, ua.row_blocks, n, st->absA, ci > 0, s));
     // accumulators of the new auxiliary variables
-    SPCHK(contract(n, n, Tc, 1.0, ac, false, ac, false, acc, ga, ga, true, acc64, bf16, status_dev, s));
-    SPCHK(contract(d, n, Tc, 1.0, yc, false, ac, false, acc, r2, r2, false, acc64, bf16, status_dev, s));
+    if (a_transposed) {
+      MatRef act{p.Ac, cdt, Tld};
+      SPCHK(contract(n, n, Tc, 1.0, act, true, act, true, acc, ga, ga, true, acc64, bf16, status_dev, s));
+      SPCHK(contract(d, n, Tc, 1.0, yc, false, act, true, acc, r2, r2, false, acc64, bf16, status_dev, s));
+    } else {
+      SPCHK(contract(n, n, Tc, 1.0, ac, false, ac, false, acc, ga, ga, true, acc64, bf16, status_dev, s));
+      SPCHK(contract(d, n, Tc, 1.0, yc, false, ac, false, acc, r2, r2, false, acc64, bf16, status_dev, s));
+    }
     SPCHK(contract(n, d, Tc, 1.0, zb, false, xc, false, acc, r1, r1, false, acc64, bf16, status_dev, s));
   }
   CU(symmetrize_lower(st->G_A, n, n, s));

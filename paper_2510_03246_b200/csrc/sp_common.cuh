@@ -182,6 +182,8 @@ struct UpdateArgs {
   const int32_t* grp_base;   // per group of 8 channels: kept channels before the group
   const uint8_t* grp_mask;   // per group of 8 channels: bit q = channel 8 g + q is kept
   void* A_out;       // [T, n] storage dtype
+  void* At_out = nullptr;  // bf16 [n, ldt]: A transposed (then A_out is not written)
+  int64_t ldt = 0;
   void* Zb_out;      // [T, n] storage dtype copy of Z_new
   int32_t out_dtype;
   int64_t T, n;

@@ -305,6 +305,13 @@ __device__ __forceinline__ void store4(void* base, int32_t dt, int64_t e, const 
 // cover the DRAM latency (the kernel moves 12 n + 8 k bytes per token and does almost no arithmetic).
 // Sums: fp32 within one row and per column over the thread's rows (at most a few hundred terms), fp64 across rows
 // and blocks.
+// Transposed-A tile of one block: kAtRows rows (64-byte pieces per channel) of its 1024 channels, channel-major with a
+// pitch of 72 bytes.  (A layout free of bank conflicts, written out in 8-byte pieces, measured 2 % slower: the kernel
+// is bound by its global stores, not by shared memory.)
+constexpr int kAtRows = 32;
+constexpr int kAtPitch = kAtRows + 4;                 // bf16 elements
+constexpr size_t kAtTileBytes = (size_t)1024 * kAtPitch * sizeof(__nv_bfloat16);
+
 template <bool HAS_U>
 struct UpdRow {
   float zo[4], u[4], z1[4], dc[4], gt[4];
@@ -315,7 +322,8 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
   __shared__ double sm[32];
   const int64_t grp4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t c0 = grp4 * 4;
-  const int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
+  int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
+  if (g.At_out) rows_per = (rows_per + kAtRows - 1) / kAtRows * kAtRows;   // whole tiles: 16-byte aligned pieces
   const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
   const int64_t r_end = (r_begin + rows_per < g.T) ? r_begin + rows_per : g.T;
   const float inv_ab = 1.f / (g.alpha + g.beta);
@@ -325,14 +333,19 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
   const float* __restrict__ Dp = g.D;
   double s_res = 0.0, s_z = 0.0, s_a = 0.0, s_in = 0.0;
   float cs[4] = {0.f, 0.f, 0.f, 0.f};
-  if (c0 < g.n) {
-    const int cnt = (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
+  // With a transposed A every warp stages kAtRows rows of its 128 channels in shared memory (channel-major) and
+  // writes them out as 64-byte pieces; lanes beyond the last channel walk the loop too (without touching memory),
+  // so that the warp-level barriers see all lanes.
+  extern __shared__ __align__(16) __nv_bfloat16 at_tile[];     // [1024][kAtPitch], only with At_out
+  const bool active = c0 < g.n;
+  {
+    const int cnt = !active ? 0 : (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
     const bool vec = (g.n % 4 == 0);
     // kept channels of this half group and their compact offsets
-    const unsigned bits8 = g.grp_mask[grp4 >> 1];
+    const unsigned bits8 = active ? g.grp_mask[grp4 >> 1] : 0u;
     const bool upper = (grp4 & 1) != 0;
     const unsigned bits = upper ? (bits8 >> 4) : (bits8 & 0xFu);
-    const int base = g.grp_base[grp4 >> 1] + (upper ? __popc(bits8 & 0xFu) : 0);
+    const int base = active ? g.grp_base[grp4 >> 1] + (upper ? __popc(bits8 & 0xFu) : 0) : 0;
     int off[4];
     {
       int pos = 0;
@@ -383,7 +396,7 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
         w.dc[q] = kept ? dp[off[q]] : 0.f;
       }
     };
-    auto finish_row = [&](int64_t r, UpdRow<HAS_U>& w) {
+    auto finish_row = [&](int64_t r, UpdRow<HAS_U>& w, __nv_bfloat16* arow) {
       const int64_t e = r * g.n + c0;
       float a[4], zn[4];
       float p_res = 0.f, p_z = 0.f, p_a = 0.f, p_in = 0.f;
@@ -406,7 +419,12 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
       if (vec) {
         *reinterpret_cast<float4*>(Zp + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
         if (HAS_U) *reinterpret_cast<float4*>(Up + e) = make_float4(w.u[0], w.u[1], w.u[2], w.u[3]);
-        store4(g.A_out, g.out_dtype, e, a);
+        if (g.At_out) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) arow[q] = __float2bfloat16_rn(a[q]);
+        } else {
+          store4(g.A_out, g.out_dtype, e, a);
+        }
         if (g.Zb_out) store4(g.Zb_out, g.out_dtype, e, zn);
       } else {
 #pragma unroll
@@ -425,24 +443,68 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
         }
       }
     };
-    int64_t r = r_begin;
-    for (; r + 3 < r_end; r += 4) {
-      UpdRow<HAS_U> w0, w1, w2, w3;
-      load_row(r, w0);
-      load_row(r + 1, w1);
-      load_row(r + 2, w2);
-      load_row(r + 3, w3);
-      finish_row(r, w0);
-      finish_row(r + 1, w1);
-      finish_row(r + 2, w2);
-      finish_row(r + 3, w3);
+    const int ct = 4 * (int)threadIdx.x;                    // first of this thread's channels inside the block
+    const int64_t tile_step = g.At_out ? kAtRows : (r_end > r_begin ? r_end - r_begin : 1);
+    for (int64_t rt = r_begin; rt < r_end; rt += tile_step) {
+      const int64_t rt_end = (rt + tile_step < r_end) ? rt + tile_step : r_end;
+      if (active) {
+        int64_t r = rt;
+        for (; r + 3 < rt_end; r += 4) {
+          UpdRow<HAS_U> w0, w1, w2, w3;
+          load_row(r, w0);
+          load_row(r + 1, w1);
+          load_row(r + 2, w2);
+          load_row(r + 3, w3);
+          __align__(8) __nv_bfloat16 ab[4][4];
+          finish_row(r, w0, ab[0]);
+          finish_row(r + 1, w1, ab[1]);
+          finish_row(r + 2, w2, ab[2]);
+          finish_row(r + 3, w3, ab[3]);
+          if (g.At_out) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              __align__(8) __nv_bfloat16 col[4] = {ab[0][q], ab[1][q], ab[2][q], ab[3][q]};
+              *reinterpret_cast<uint2*>(&at_tile[(ct + q) * kAtPitch + (int)(r - rt)]) =
+                  *reinterpret_cast<const uint2*>(col);
+            }
+          }
+        }
+        for (; r < rt_end; ++r) {
+          UpdRow<HAS_U> w0;
+          __nv_bfloat16 ab1[4];
+          load_row(r, w0);
+          finish_row(r, w0, ab1);
+          if (g.At_out) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) at_tile[(ct + q) * kAtPitch + (int)(r - rt)] = ab1[q];
+          }
+        }
+      }
+      if (g.At_out) {
+        // write the tile out, each warp its own 128 channels (only the warp itself wrote them, so a warp-level
+        // barrier is enough): rows rt .. rt_end - 1 of a channel in pieces of 8 rows (16 bytes), 4 lanes per channel
+        __syncwarp();
+        const int rows_here = (int)(rt_end - rt);
+        const int lane = (int)threadIdx.x & 31, wch0 = ((int)threadIdx.x >> 5) * 128;
+        const int64_t cb = (int64_t)blockIdx.x * 1024 + wch0;
+        const int nch = (g.n - cb < 128) ? (int)((g.n - cb > 0) ? g.n - cb : 0) : 128;
+        __nv_bfloat16* At = reinterpret_cast<__nv_bfloat16*>(g.At_out);
+        for (int e = lane; e < nch * (kAtRows / 8); e += 32) {
+          const int ch = e / (kAtRows / 8), piece = e % (kAtRows / 8);
+          const __nv_bfloat16* src = &at_tile[(wch0 + ch) * kAtPitch + piece * 8];
+          __nv_bfloat16* dst = At + (cb + ch) * g.ldt + rt + piece * 8;
+          if (piece * 8 + 8 <= rows_here) {
+            const uint2 lo = *reinterpret_cast<const uint2*>(src), hi = *reinterpret_cast<const uint2*>(src + 4);
+            *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+          } else {
+            for (int q = 0; q < 8; ++q)
+              if (piece * 8 + q < rows_here) dst[q] = src[q];
+          }
+        }
+        __syncwarp();
+      }
     }
-    for (; r < r_end; ++r) {
-      UpdRow<HAS_U> w0;
-      load_row(r, w0);
-      finish_row(r, w0);
-    }
-    if (g.absA_part) {
+    if (g.absA_part && active) {
 #pragma unroll
       for (int q = 0; q < 4; ++q)
         if (q < cnt) g.absA_part[(int64_t)blockIdx.y * g.n + c0 + q] = (double)cs[q];
@@ -818,16 +880,18 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * ((double)a.n * per_n + (double)a.k * 8.0), stream);
   count_launch();
   const bool pz = a.z_rule == SP_Z_PAPER;
-  if (a.gate) {
-    if (a.U) fused_update_kernel<true, kZGated><<<grid, 256, 0, stream>>>(a);
-    else fused_update_kernel<false, kZGated><<<grid, 256, 0, stream>>>(a);
-  } else if (a.U) {
-    if (pz) fused_update_kernel<true, SP_Z_PAPER><<<grid, 256, 0, stream>>>(a);
-    else fused_update_kernel<true, SP_Z_EXACT><<<grid, 256, 0, stream>>>(a);
-  } else {
-    if (pz) fused_update_kernel<false, SP_Z_PAPER><<<grid, 256, 0, stream>>>(a);
-    else fused_update_kernel<false, SP_Z_EXACT><<<grid, 256, 0, stream>>>(a);
+  // the transposed-A tile of one block is above the default 48 KB limit
+  const size_t smem = a.At_out ? kAtTileBytes : 0;
+  void (*fn)(UpdateArgs) = nullptr;
+  if (a.gate) fn = a.U ? &fused_update_kernel<true, kZGated> : &fused_update_kernel<false, kZGated>;
+  else if (a.U) fn = pz ? &fused_update_kernel<true, SP_Z_PAPER> : &fused_update_kernel<true, SP_Z_EXACT>;
+  else fn = pz ? &fused_update_kernel<false, SP_Z_PAPER> : &fused_update_kernel<false, SP_Z_EXACT>;
+  if (smem) {
+    cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn),
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
   }
+  fn<<<grid, 256, smem, stream>>>(a);
   return cudaGetLastError();
 }
 

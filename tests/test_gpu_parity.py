@@ -433,6 +433,22 @@ def test_admm_step_teacher_forced(cfg, chunk, kind, rule, dual, refit):
         _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
 
 
+@pytest.mark.parametrize("chunk,rule,dual", [(0, "paper", False), (512, "exact", True), (96, "paper", True)])
+def test_admm_step_bf16_without_objective(chunk, rule, dual):
+    """bf16 storage without the output-side objective term: the update then writes the new A channel-major (tokens
+    contiguous) for the accumulator products.  Chunks of 1300, 512 + 512 + 276 and 96 ... + 52 tokens: whole tiles
+    of 32 tokens, tails that are not a multiple of 8, and row blocks that get no token at all."""
+    cfg = SMALL_BF16
+    mod, X, W1, W2 = _make_module(cfg, dual=dual, chunk=chunk)
+    mod.sp_ffn_init()
+    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, z_rule=_RULE[rule], dual_mode=dual,
+                           token_chunk=chunk, compute_objective=False)
+    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, z_rule=rule, dual_mode=dual)
+    audit = []
+    for it in range(2):
+        _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
+
+
 def test_admm_step_with_z1_computed_ahead():
     """Same step with the optional workspace tail: z1 of all tokens is computed on the side stream beside the
     kept-support recovery (the configuration bench.py runs)."""
