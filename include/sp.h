@@ -182,6 +182,18 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
                        int32_t* status_dev, void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
+ * sp_admm_scores — parts 1 and 2 of sp_admm_step alone: the unrestricted recovery the scores read (W2~; W1~ as well
+ * for SP_SCORE_LEMMA1) and the unit scores and layer importance of the module's current state.  Writes st->scores
+ * and st->importance; st->W1, st->W2, st->mask, Z, U and the accumulators are left as they are.
+ * Paper: Appendix B, Algorithm 3 (GSPO) collects the scores of ALL layers before one global threshold decides every
+ * mask; a lock-step run calls this for every module, selects over the concatenated scores (sp_apply_mask), and then
+ * finishes the iteration of each module with sp_admm_step(reselect_mask = 0, skip_scores = 1).
+ * p->k_keep is ignored; p->skip_scores must be 0.  Workspace and errors as sp_admm_step.
+ */
+sp_status sp_admm_scores(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* p, int32_t* status_dev,
+                         void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
  * sp_struct_scores — per-unit importance scores and the layer importance I = mean over units.
  *   SP_SCORE_WANDA_L2 (Section 3.4, Eq. "wanda"): s_u = sqrt( sum_{j in unit u} |W[:,j]|_2^2 * colsq_j )
  *   SP_SCORE_WANDA_L1 (Algorithm 1, Step 3):       s_u = sum_{j in unit u} |W[:,j]|_1 * colabs_j * inv_tokens

@@ -291,6 +291,23 @@ def topk_mask(scores, k_keep):
     return mask, tau
 
 
+def global_threshold_masks(scores_per_layer, keep_fraction, min_keep=0):
+    """Appendix B, Algorithm 3 (GSPO), threshold step: the scores of all L layers are collected, K = floor(r n L)
+    with r the kept fraction of the global budget, and the units holding the K largest scores are kept — one
+    threshold for the whole model, so layers end with different kept counts.  Exactly K units are kept (ties: the
+    earlier layer, then the lower index).  min_keep > 0: a layer left with fewer units keeps its own min_keep
+    largest instead (the algorithm as printed can empty a layer).  Returns (masks u8 [L, n], kept counts, tau)."""
+    S = np.asarray(scores_per_layer, F64)
+    L, n = S.shape
+    K = int(np.floor(keep_fraction * n * L + 1e-9))
+    flat, tau = topk_mask(S.reshape(-1), K)
+    masks = flat.reshape(L, n).copy()
+    for l in range(L):
+        if masks[l].sum() < min_keep:
+            masks[l], _ = topk_mask(S[l], min_keep)
+    return masks, masks.sum(axis=1).astype(np.int64), tau
+
+
 def apply_mask(mask, group=1, W_rows=None, W_cols=None):
     """M (.) W: zero the row groups of W_rows and the column groups of W_cols of pruned units."""
     m = np.repeat(np.asarray(mask).astype(bool), group)

@@ -24,7 +24,8 @@ SP_ALLOC_SOFTMAX, SP_ALLOC_INVERSE, SP_ALLOC_UNIFORM = 0, 1, 2
 (SP_WS_GRAM, SP_WS_ADMM_STEP, SP_WS_SCORES, SP_WS_APPLY_MASK, SP_WS_FFN_INIT, SP_WS_LINEAR_REFIT, SP_WS_GEMM,
  SP_WS_RIDGE_SOLVE) = range(8)
 
-EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_struct_scores", "sp_allocate_sparsity",
+EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_admm_scores", "sp_struct_scores",
+           "sp_allocate_sparsity",
            "sp_apply_mask", "sp_apply_mask_batched", "sp_weight_stats", "sp_distribute_importance",
            "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
@@ -88,6 +89,8 @@ def lib() -> C.CDLL:
         pm = C.POINTER(SpMat)
         L.sp_gram_accumulate.argtypes = [pm, pm, vp, i64, vp, i64, vp, vp, vp, sz, vp]
         L.sp_ffn_init.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), i64, vp, vp, sz, vp]
+        L.sp_admm_scores.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), C.POINTER(SpAdmmParams), vp, vp,
+                                     C.c_size_t, vp]
         L.sp_admm_step.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), C.POINTER(SpAdmmParams), vp, vp, vp,
                                    sz, vp]
         L.sp_struct_scores.argtypes = [i32, i32, C.POINTER(SpScoreInputs), i64, vp, vp, vp, dbl, vp, sz, vp]
@@ -286,11 +289,16 @@ def sp_allocate_sparsity(I, n_units, rbar, T, mode=SP_ALLOC_SOFTMAX, clip_hi=0.9
     return r, k
 
 
-def sp_apply_mask(scores, k_keep, group=1, W_rows=None, W_cols=None, want_index=False):
-    """Returns (mask u8 [n_units], tau fp32 [1], kept_idx int32 [k_keep] or None); W_rows / W_cols are zeroed in place."""
-    _require_cuda(scores, W_rows, W_cols)
+def sp_apply_mask(scores, k_keep, group=1, W_rows=None, W_cols=None, want_index=False, mask_out=None):
+    """Returns (mask u8 [n_units], tau fp32 [1], kept_idx int32 [k_keep] or None); W_rows / W_cols are zeroed in place.
+    mask_out: caller-owned contiguous uint8 [n_units] buffer to write the mask into."""
+    _require_cuda(scores, W_rows, W_cols, mask_out)
     n = scores.numel()
-    mask = torch.empty(n, dtype=torch.uint8, device=scores.device)
+    if mask_out is not None and (mask_out.dtype != torch.uint8 or mask_out.numel() != n or not mask_out.is_contiguous()):
+        raise ValueError("mask_out must be contiguous uint8 [n_units]")
+    if not scores.is_contiguous() or scores.dtype != torch.float32:
+        raise ValueError("scores must be contiguous fp32")
+    mask = mask_out if mask_out is not None else torch.empty(n, dtype=torch.uint8, device=scores.device)
     tau = torch.empty(1, dtype=torch.float32, device=scores.device)
     idx = torch.empty(max(int(k_keep), 1), dtype=torch.int32, device=scores.device) if want_index else None
     wr = mat(W_rows) if W_rows is not None else None
@@ -378,10 +386,14 @@ class FfnModule:
     """Owns the device buffers of one FFN module and forwards to sp_ffn_init / sp_admm_step."""
 
     def __init__(self, X: torch.Tensor, W1_0: torch.Tensor, W2_0: torch.Tensor, dual_mode: bool = False,
-                 token_chunk: int = 0, overlap_k: int = 0, Wg_0: torch.Tensor | None = None):
+                 token_chunk: int = 0, overlap_k: int = 0, Wg_0: torch.Tensor | None = None,
+                 scores: torch.Tensor | None = None, mask: torch.Tensor | None = None, ws_pool: dict | None = None):
         """overlap_k > 0: also reserve the optional workspace tail that lets sp_admm_step compute z1 of all tokens
         beside the kept-support recovery, sized for overlap_k kept units (see sp_admm_overlap_bytes).
-        Wg_0 (gate projection [n, d]) makes the module a SwiGLU one: W1_0 is then its up projection."""
+        Wg_0 (gate projection [n, d]) makes the module a SwiGLU one: W1_0 is then its up projection.
+        scores (fp32 [n]) / mask (uint8 [n]): caller-owned contiguous buffers, e.g. rows of one [L, n] array over
+        which a lock-step run selects a single global threshold.  ws_pool: a dict shared by modules that are never
+        in flight at the same time; they then use one workspace."""
         _require_cuda(X, W1_0, W2_0, Wg_0)
         assert X.dtype in (torch.float32, torch.bfloat16)
         self.X = X.contiguous()
@@ -406,15 +418,27 @@ class FfnModule:
         self.absA = torch.empty(n, dtype=torch.float64, device=dev)
         self.W1 = torch.zeros(n, d, **f32)
         self.W2 = torch.zeros(d, n, **f32)
-        self.scores = torch.zeros(n, **f32)
-        self.mask = torch.ones(n, dtype=torch.uint8, device=dev)
+        if scores is not None:
+            assert scores.dtype == torch.float32 and scores.shape == (n,) and scores.is_contiguous() and scores.is_cuda
+        if mask is not None:
+            assert mask.dtype == torch.uint8 and mask.shape == (n,) and mask.is_contiguous() and mask.is_cuda
+        self.scores = scores if scores is not None else torch.zeros(n, **f32)
+        self.mask = mask if mask is not None else torch.ones(n, dtype=torch.uint8, device=dev)
         self.importance = torch.zeros(1, dtype=torch.float64, device=dev)
         self.report = torch.zeros(len(REPORT_FIELDS), dtype=torch.float64, device=dev)
         self.status = new_status(dev)
         self.token_chunk = token_chunk
         self.overlap_k = int(overlap_k)
-        self._ws = None
+        self._pool = ws_pool if ws_pool is not None else {}
         self.iteration = 0
+
+    @property
+    def _ws(self):
+        return self._pool.get("ws")
+
+    @_ws.setter
+    def _ws(self, t):
+        self._pool["ws"] = t
 
     def _module(self) -> SpFfnModule:
         return SpFfnModule(mat(self.X), mat(self.Ypre), mat(self.W1_0), mat(self.W2_0), self.d, self.n, self.N,
@@ -451,6 +475,16 @@ class FfnModule:
         _check(lib().sp_admm_step(C.byref(m), C.byref(st), C.byref(cp), self.report.data_ptr(),
                                   self.status.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "sp_admm_step")
         self.iteration += 1
+
+    def sp_admm_scores(self, p: AdmmParams):
+        """Unrestricted recovery + unit scores + layer importance of the current state (no mask, no token pass)."""
+        chunk = p.token_chunk or self.token_chunk
+        ws = self._workspace(chunk)
+        m, st = self._module(), self._state()
+        cp = p.to_c()
+        cp.token_chunk = chunk
+        _check(lib().sp_admm_scores(C.byref(m), C.byref(st), C.byref(cp), self.status.data_ptr(), ws.data_ptr(),
+                                    ws.numel(), _stream()), "sp_admm_scores")
 
     def read_report(self) -> dict:
         return dict(zip(REPORT_FIELDS, self.report.cpu().tolist()))

@@ -664,14 +664,16 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   return SP_OK;
 }
 
-sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* prm, sp_step_report* rep_dev,
-                       int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+// One step, or (scores_only) its first two parts: the unrestricted recovery the scores read, and the scores.
+static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* prm, sp_step_report* rep_dev,
+                         int32_t* status_dev, void* ws, size_t ws_bytes, void* stream, bool scores_only) {
   if (!prm) return SP_ERR_INVALID_ARG;
   SPCHK(check_module(m, st, prm->score_kind == SP_SCORE_LEMMA1));
   if (!st->W1 || !st->W2 || !st->scores || !st->mask || !st->importance) return SP_ERR_INVALID_ARG;
   if (prm->dual_mode && !st->U) return SP_ERR_INVALID_ARG;
   const int64_t d = m->d, n = m->n, N = m->N;
-  if (prm->k_keep < 1 || prm->k_keep > n) return SP_ERR_SHAPE;
+  if (scores_only && prm->skip_scores) return SP_ERR_INVALID_ARG;
+  if (!scores_only && (prm->k_keep < 1 || prm->k_keep > n)) return SP_ERR_SHAPE;
   if (prm->score_kind == SP_SCORE_LEMMA1 && m->W1_0.ld != d) return SP_ERR_SHAPE;
   if (!(prm->alpha > 0.0) || !(prm->beta > 0.0) || !(prm->rho >= 0.0) || prm->token_chunk < 0) return SP_ERR_INVALID_ARG;
   if (prm->z_rule != SP_Z_PAPER && prm->z_rule != SP_Z_EXACT) return SP_ERR_UNSUPPORTED;
@@ -711,11 +713,14 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
     SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
                              side ? &side->assist_main : nullptr));
   }
-  CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
-  if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
-                                    side ? &side->assist_side : nullptr));
-  else SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
-                                    side ? &side->assist_side : nullptr));
+  const bool need_w1 = !scores_only || prm->score_kind == SP_SCORE_LEMMA1;   // only the Lemma-1 score reads W1~
+  if (need_w1) {
+    CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
+    if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
+                                      side ? &side->assist_side : nullptr));
+    else SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
+                                      side ? &side->assist_side : nullptr));
+  }
   if (side) CU(cudaEventRecord(side->join, sa));
   bool joined = side == nullptr;
 
@@ -731,6 +736,11 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   } else {
     CU(wanda_scores(prm->score_kind, 1, p.W2t, d, n, st->G_A, n + 1, st->absA, 1.0 / (double)N, n, st->scores,
                     st->importance, p.score_scratch, s));
+  }
+
+  if (scores_only) {
+    if (!joined) CU(cudaStreamWaitEvent(s, side->join, 0));
+    return SP_OK;
   }
 
   // ---- 3. top-k mask
@@ -874,6 +884,16 @@ sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_p
   }
   CU(symmetrize_lower(st->G_A, n, n, s));
   return SP_OK;
+}
+
+sp_status sp_admm_step(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* prm, sp_step_report* rep_dev,
+                       int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+  return admm_step_impl(m, st, prm, rep_dev, status_dev, ws, ws_bytes, stream, false);
+}
+
+sp_status sp_admm_scores(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* prm, int32_t* status_dev,
+                         void* ws, size_t ws_bytes, void* stream) {
+  return admm_step_impl(m, st, prm, nullptr, status_dev, ws, ws_bytes, stream, true);
 }
 
 }  // extern "C"

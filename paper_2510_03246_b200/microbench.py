@@ -4,6 +4,8 @@
     python -m paper_2510_03246_b200.microbench solve [--reps 3 --warm 1]   regularised solves of a C2 step
     python -m paper_2510_03246_b200.microbench mask  [--reps 5 --warm 2]   scores, allocation and top-k as standalone
                                                                            kernels (L2 flushed before every call)
+    python -m paper_2510_03246_b200.microbench lockstep [--reps 3 --warm 1] lock-step iterations of several C2-wide
+                                                                           layers under one global threshold
 
 Inputs are random (torch.randn on the device): these runs time kernels, they check nothing.
 """
@@ -156,6 +158,53 @@ def mask_cases(reps, warm, hbm_gbs):
         line(f"top-k batched  L = {L}, n = {n}", ms, 5.0 * L * n)
 
 
+def lockstep_cases(reps, warm, layers=4, tokens=32768):
+    """Iterations of the lock-step run (all layers' scores, one global threshold, all layers' fixed-mask steps) on
+    `layers` modules of C2's width with `tokens` tokens each, against the same modules stepped one by one with
+    per-layer top-k (the ordinary step)."""
+    from . import pipeline, synth
+    cfg = synth.scaled(synth.CONFIGS["C2"], tokens=tokens, layers=layers)
+    data = []
+    for l in range(layers):
+        X = synth.make_activations(cfg, l).to(DEV)
+        W1, W2 = (w.to(DEV) * (1.0 + 0.03 * l) for w in synth.make_weights(cfg, l))
+        data.append((X, W1, W2))
+    keep = 1.0 - cfg.sparsity
+    results, scores, masks = pipeline.prune_ffn_layers_global(lambda l: data[l], layers, cfg.n, keep, 2,
+                                                              params=api.AdmmParams(rho=cfg.rho), token_chunk=32768)
+    torch.cuda.synchronize()
+    counts = masks.sum(dim=1).cpu().tolist()
+    K = int(keep * cfg.n * layers + 1e-9)
+    del results
+    print(f"lock-step: {layers} layers x {tokens} tokens, d={cfg.d}, n={cfg.n}, kept fraction {keep}: kept per layer "
+          f"after 2 iterations {counts}")
+    sel = _timeit(lambda: api.sp_apply_mask(scores.view(-1), K, mask_out=masks.view(-1)), max(reps, 10), warm)
+    print(f"global select over {layers * cfg.n} scores (K = {K}): {sel * 1e3:.0f} us")
+    # the ordinary step on the same modules, per-layer top-k with the lock-step run's final counts
+    mods = []
+    for l in range(layers):
+        m = api.FfnModule(*data[l], token_chunk=32768, overlap_k=int(counts[l]))
+        m.sp_ffn_init()
+        mods.append(m)
+
+    def ordinary():
+        for l, m in enumerate(mods):
+            m.sp_admm_step(api.AdmmParams(rho=cfg.rho, k_keep=int(counts[l]), token_chunk=32768))
+    ms = _timeit(ordinary, reps, warm)
+    print(f"ordinary steps (per-layer top-k, same kept counts): {ms:.2f} ms per iteration of all layers")
+
+    def lock():
+        pl = api.AdmmParams(rho=cfg.rho, k_keep=1, token_chunk=32768)
+        for m in mods:
+            m.sp_admm_scores(pl)
+        for l, m in enumerate(mods):
+            m.sp_admm_step(api.AdmmParams(rho=cfg.rho, k_keep=int(counts[l]), token_chunk=32768, reselect_mask=False,
+                                          skip_scores=True))
+    ms2 = _timeit(lock, reps, warm)
+    print(f"lock-step calls on the same modules (scores of all layers, then fixed-mask steps; select not included): "
+          f"{ms2:.2f} ms per iteration of all layers")
+
+
 def _hbm_peak():
     import json
     import os
@@ -169,7 +218,7 @@ def _hbm_peak():
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "solve", "mask"])
+    ap.add_argument("what", choices=["gemm", "solve", "mask", "lockstep"])
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warm", type=int, default=2)
     a = ap.parse_args()
@@ -180,6 +229,8 @@ def main():
         peak, src = _hbm_peak()
         print(f"HBM peak {peak:.0f} GB/s ({src})")
         mask_cases(a.reps, a.warm, peak)
+    elif a.what == "lockstep":
+        lockstep_cases(a.reps, a.warm)
     else:
         (gemm_cases if a.what == "gemm" else solve_cases)(a.reps, a.warm)
 

@@ -93,6 +93,55 @@ def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_unit
     return results, r, k_keep, {"importance_s": t1 - t0, "admm_s": t2 - t1, "layers_per_s": len(mine) / max(t2 - t0, 1e-9)}
 
 
+def prune_ffn_layers_global(layer_inputs: Callable[[int], tuple], n_layers: int, n_units: int, keep_fraction: float,
+                            iters: int, params: api.AdmmParams | None = None, token_chunk: int = 0, min_keep: int = 1,
+                            device="cuda"):
+    """Lock-step run of Appendix B, Algorithm 3 (GSPO): in every iteration the scores of ALL layers are computed from
+    their current states, ONE threshold over the concatenated scores keeps K = floor(keep_fraction * n_units *
+    n_layers) units of the whole model, and every layer finishes the iteration (recovery on its kept support, a- and
+    z-updates) with the mask it was given.  The states of all layers stay resident (Z alone is N x n fp32 per layer);
+    the modules share one workspace.  min_keep: a layer the threshold leaves with fewer units keeps its own min_keep
+    best ones (sp_admm_step needs at least one).  Returns (results per layer, scores [L, n], masks [L, n])."""
+    p = params or api.AdmmParams()
+    L, n = n_layers, n_units
+    scores = torch.zeros(L, n, dtype=torch.float32, device=device)
+    masks = torch.ones(L, n, dtype=torch.uint8, device=device)
+    pool, mods = {}, []
+    overlap_k = min(n, int(1.5 * keep_fraction * n) + 1)
+    for l in range(L):
+        X, W1_0, W2_0 = layer_inputs(l)
+        mod = api.FfnModule(X, W1_0, W2_0, dual_mode=p.dual_mode, token_chunk=token_chunk, overlap_k=overlap_k,
+                            scores=scores[l], mask=masks[l], ws_pool=pool)
+        mod.sp_ffn_init()
+        mods.append(mod)
+    K = int(keep_fraction * n * L + 1e-9)
+    results = [LayerResult(l, float("nan"), 0, None, None, None) for l in range(L)]
+    p_scores = api.AdmmParams(**{**p.__dict__, "k_keep": 1, "token_chunk": token_chunk, "skip_scores": False})
+    for _ in range(iters):
+        for mod in mods:
+            mod.sp_admm_scores(p_scores)
+        api.sp_apply_mask(scores.view(-1), K, mask_out=masks.view(-1))
+        counts = masks.sum(dim=1).cpu().tolist()          # kept units per layer: host arguments of the calls below
+        for l in range(L):
+            if counts[l] < min_keep:
+                api.sp_apply_mask(scores[l], min_keep, mask_out=masks[l])
+                counts[l] = min_keep
+        for l, mod in enumerate(mods):
+            # with the recovery on the kept support nothing of the unrestricted recovery is needed again
+            pl = api.AdmmParams(**{**p.__dict__, "k_keep": int(counts[l]), "token_chunk": token_chunk,
+                                   "reselect_mask": False, "skip_scores": bool(p.refit)})
+            mod.sp_admm_step(pl)
+            results[l].reports.append(mod.report.clone())
+            results[l].k_keep = int(counts[l])
+    for l, mod in enumerate(mods):
+        mod.check_status()
+        res = results[l]
+        res.importance = float(mod.importance.item())
+        res.mask, res.W1, res.W2 = mod.mask.clone(), mod.W1.clone(), mod.W2.clone()
+        res.reports = [dict(zip(api.REPORT_FIELDS, t.cpu().tolist())) for t in res.reports]
+    return results, scores, masks
+
+
 def compact_module(mod: api.FfnModule):
     """Continuation of a module whose mask is fixed (the flow of Algorithm 1, where Step 3 fixes the masks before the
     SparseLLM iterations): a new module that holds only the kept channels.  With a fixed mask the pruned channels

@@ -433,6 +433,43 @@ def test_admm_step_teacher_forced(cfg, chunk, kind, rule, dual, refit):
         _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
 
 
+@pytest.mark.parametrize("cfg,kind", [(SMALL_F32, "wanda_l2"), (SMALL_F32, "wanda_l1"), (SMALL_F32, "lemma1"),
+                                      (SMALL_BF16, "wanda_l2"), (SMALL_BF16, "lemma1")])
+def test_admm_scores_alone(cfg, kind):
+    """The score part of a step on its own (what a lock-step run over all layers calls before its global threshold,
+    Appendix B, Algorithm 3): scores and importance of the current state match the oracle's, everything else in the
+    state is left untouched, and the following fixed-mask step gives what a full step with that mask gives."""
+    mod, X, W1, W2 = _make_module(cfg, chunk=256)
+    mod.sp_ffn_init()
+    k = cfg.k_keep
+    p0 = api.AdmmParams(rho=cfg.rho, k_keep=k, score_kind=_KIND[kind], token_chunk=256)
+    mod.sp_admm_step(p0)                                          # a state after one full iteration
+    torch.cuda.synchronize()
+    before = {name: getattr(mod, name).clone() for name in ("W1", "W2", "mask", "Z", "G_A", "R1", "R2", "absA")}
+    mod.scores.fill_(-1.0)
+    mod.sp_admm_scores(api.AdmmParams(rho=cfg.rho, k_keep=0, score_kind=_KIND[kind], token_chunk=256))
+    torch.cuda.synchronize()
+    mod.check_status()
+    for name, t in before.items():
+        assert torch.equal(getattr(mod, name), t), name
+    st = oracle_state_from_gpu(mod)
+    p_or = O.AdmmParams(rho=cfg.rho, k_keep=k, score_kind=kind)
+    s_or, I_or = O.admm_weight_phase(copy.deepcopy(st), np64(W1.float()), p_or, cfg.tokens)
+    tol = TOL[X.dtype]
+    assert relerr(np64(mod.scores), s_or) < tol
+    assert abs(mod.importance.item() - I_or) < tol * abs(I_or)
+    # finish the iteration with a mask chosen outside: the oracle's step with the same mask
+    m_new, _ = O.topk_mask(mod.scores.cpu().numpy(), k - 7)
+    mod.mask.copy_(torch.from_numpy(m_new).to(DEV))
+    p_fix = api.AdmmParams(rho=cfg.rho, k_keep=k - 7, score_kind=_KIND[kind], token_chunk=256, reselect_mask=False,
+                           skip_scores=True)
+    p_or_fix = O.AdmmParams(rho=cfg.rho, k_keep=k - 7, score_kind=kind, reselect_mask=False)
+    _step_and_compare(mod, X, W1.float(), p_fix, p_or_fix, tol, [])
+    with pytest.raises(api.SpError) as e:
+        mod.sp_admm_scores(api.AdmmParams(rho=cfg.rho, k_keep=k, reselect_mask=False, skip_scores=True))
+    assert e.value.code == 1
+
+
 @pytest.mark.parametrize("chunk,rule,dual", [(0, "paper", False), (512, "exact", True), (96, "paper", True)])
 def test_admm_step_bf16_without_objective(chunk, rule, dual):
     """bf16 storage without the output-side objective term: the update then writes the new A channel-major (tokens

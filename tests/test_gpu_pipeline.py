@@ -131,3 +131,68 @@ def test_fixed_mask_continuation_on_kept_channels(bf16):
     with pytest.raises(api.SpError) as e:
         full.sp_admm_step(api.AdmmParams(k_keep=k, skip_scores=True))
     assert e.value.code == 1
+
+
+@pytest.mark.parametrize("kind,bf16", [("wanda_l2", False), ("lemma1", False), ("wanda_l2", True)])
+def test_lockstep_global_threshold(kind, bf16):
+    """Appendix B, Algorithm 3 (GSPO) in lock step over three layers: per iteration the scores of all layers, one
+    global threshold, then every layer's recovery and a-/z-updates with the mask it was given.  The oracle walks the
+    same loop on its own from the same inputs (fp32 case: masks must agree bit for bit and the final weights within
+    tolerance); the last selection is also checked against the oracle's threshold on the GPU's own scores."""
+    import copy
+    cfg = synth.scaled(synth.CONFIGS["C2" if bf16 else "C1"], layers=3, d=96, n=328, tokens=600, outlier_frac=0.02)
+    kinds = {"wanda_l2": api.SP_SCORE_WANDA_L2, "lemma1": api.SP_SCORE_LEMMA1}
+
+    def inputs(layer):
+        X = synth.make_activations(cfg, layer)
+        W1, W2 = synth.make_weights(cfg, layer)
+        return X.to(DEV), (W1 * (1.0 + 0.5 * layer)).to(DEV), (W2 * (1.0 + 0.25 * layer)).to(DEV)
+
+    L, n, keep, iters = cfg.layers, cfg.n, 0.4, 2
+    p = api.AdmmParams(rho=cfg.rho, score_kind=kinds[kind])
+    results, scores, masks = pipeline.prune_ffn_layers_global(inputs, L, n, keep, iters, params=p, token_chunk=256)
+    torch.cuda.synchronize()
+    K = int(keep * n * L + 1e-9)
+    m_gpu = masks.cpu().numpy()
+    assert m_gpu.sum() == K and [r.k_keep for r in results] == m_gpu.sum(axis=1).tolist()
+    # the integer decision in the GPU's precision: the oracle's threshold on the GPU's scores of the last iteration
+    m_ref, counts_ref, _ = O.global_threshold_masks(scores.cpu().numpy(), keep, min_keep=1)
+    assert np.array_equal(m_gpu, m_ref)
+    assert len(set(counts_ref.tolist())) > 1                    # the layers end with different kept counts
+    for l, res in enumerate(results):
+        mk = m_gpu[l]
+        assert np.array_equal(res.mask.cpu().numpy(), mk)
+        assert np.all(np64(res.W1)[mk == 0] == 0) and np.all(np64(res.W2)[:, mk == 0] == 0)
+        assert [rep["kept"] for rep in res.reports] and res.reports[-1]["kept"] == mk.sum()
+    # the oracle's own lock-step run
+    tol = TOL[torch.bfloat16 if bf16 else torch.float32]
+    p_or = O.AdmmParams(rho=cfg.rho, score_kind=kind)
+    states, data = [], []
+    for l in range(L):
+        X, W1, W2 = inputs(l)
+        st, Y = O.ffn_init(np64(X).T, np64(W1), np64(W2))
+        states.append(st)
+        data.append((np64(X).T, Y, np64(W1)))
+    agree = True
+    for it in range(iters):
+        S = np.stack([O.admm_weight_phase(copy.deepcopy(st), data[l][2], p_or, cfg.tokens)[0]
+                      for l, st in enumerate(states)])
+        m_or, counts, _ = O.global_threshold_masks(S, keep, min_keep=1)
+        for l, st in enumerate(states):
+            st.mask = m_or[l].copy()
+            pl = copy.deepcopy(p_or)
+            pl.reselect_mask, pl.k_keep = False, int(counts[l])
+            O.admm_step(st, data[l][0], data[l][1], data[l][2], pl)
+    S_gpu = scores.cpu().numpy().astype(np.float64)
+    assert relerr(S_gpu, S) < tol * 10                           # scores after one full iteration of every layer
+    diff = np.flatnonzero(m_gpu.reshape(-1) != m_or.reshape(-1))
+    if diff.size:                                                # only units within rounding of the threshold may differ
+        tau = np.sort(S.reshape(-1))[::-1][K - 1]
+        assert np.all(np.abs(S.reshape(-1)[diff] - tau) <= 10 * tol * np.abs(S).max())
+        agree = False
+    if not bf16:
+        assert agree
+    if agree:
+        for l, res in enumerate(results):
+            assert relerr(np64(res.W1), states[l].W1) < tol * 10, l
+            assert relerr(np64(res.W2), states[l].W2) < tol * 10, l

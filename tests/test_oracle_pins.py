@@ -557,3 +557,52 @@ def test_distribute_importance_structure():
     # the mean stays rbar
     r, _ = O.allocate_sparsity(Im, np.full(3, n), 0.5, T=float(np.abs(Im).mean()), mode="inverse")
     assert np.all(np.diff(Im) < 0) and np.all(np.diff(r) < 0) and abs(r.mean() - 0.5) < 1e-12
+
+
+# ------------------------------------------------------------------------------------------------ global threshold
+def test_global_threshold_worked_example():
+    """Appendix B, Algorithm 3: one threshold over the scores of all layers, K = floor(r n L) kept.  Two layers of three
+    units, half kept: the three largest of {5, 1, 3, 4, 2, 6} are 6, 5, 4 — one unit of layer 0, two of layer 1."""
+    S = np.array([[5.0, 1.0, 3.0], [4.0, 2.0, 6.0]])
+    masks, counts, tau = O.global_threshold_masks(S, 0.5)
+    assert masks.tolist() == [[1, 0, 0], [1, 0, 1]] and counts.tolist() == [1, 2] and tau == 4.0
+    # K = floor(r n L): 0.6 * 6 = 3.6 -> 3 as well; 2/3 -> 4 kept
+    assert O.global_threshold_masks(S, 0.6)[1].sum() == 3
+    assert O.global_threshold_masks(S, 2.0 / 3.0)[0].tolist() == [[1, 0, 1], [1, 0, 1]]
+
+
+def test_global_threshold_properties_and_special_cases():
+    rng = np.random.default_rng(5)
+    for L, n, r in ((1, 40, 0.3), (4, 33, 0.5), (7, 20, 0.85)):
+        S = np.round(rng.normal(size=(L, n)) * 4) / 4            # many exact ties, also across layers
+        masks, counts, tau = O.global_threshold_masks(S, r)
+        K = int(np.floor(r * n * L + 1e-9))
+        assert masks.sum() == K == counts.sum()
+        kept, pruned = S[masks == 1], S[masks == 0]
+        assert kept.min() >= pruned.max() and kept.min() == tau    # a single threshold separates the two sets
+        # ties at the threshold: the kept ones come first in (layer, index) order
+        at = np.flatnonzero(S.reshape(-1) == tau)
+        m_at = masks.reshape(-1)[at]
+        assert np.all(np.diff(m_at.astype(int)) <= 0)
+        # brute force: repeatedly take the largest remaining score, earliest position first
+        flat = S.reshape(-1).copy()
+        ref = np.zeros(L * n, np.uint8)
+        for _ in range(K):
+            j = int(np.argmax(flat))                                # argmax returns the first maximum
+            ref[j] = 1
+            flat[j] = -np.inf
+        assert np.array_equal(ref.reshape(L, n), masks)
+        if L == 1:                                                  # one layer: the per-layer top-k of Algorithm 1
+            assert np.array_equal(masks[0], O.topk_mask(S[0], K)[0])
+    # equal score distributions in every layer -> the global threshold is the uniform allocation
+    base = rng.permutation(50).astype(float)
+    S = np.stack([rng.permutation(base) for _ in range(5)])
+    assert O.global_threshold_masks(S, 0.4)[1].tolist() == [20] * 5
+
+
+def test_global_threshold_can_empty_a_layer_unless_min_keep():
+    S = np.array([[9.0, 8.0, 7.0], [1.0, 2.0, 3.0]])
+    masks, counts, _ = O.global_threshold_masks(S, 0.5)
+    assert counts.tolist() == [3, 0]
+    masks, counts, _ = O.global_threshold_masks(S, 0.5, min_keep=1)
+    assert masks.tolist() == [[1, 1, 1], [0, 0, 1]] and counts.tolist() == [3, 1]
