@@ -45,13 +45,17 @@ def gemm_cases(reps, warm):
         ("E = Ypre - H W2^T (bf16 out)", T, D, N // 2, True, True, bf, 1.0, False),
         ("D = E Q^T (f32 out)", T, N // 2, D, True, True, f32, 0.0, False),
         ("z1 = X [W1hi W1lo]^T (f32 out)", T, N // 2, 2 * D, True, True, f32, 0.0, False),
-        ("G_A += A^T A (lower)", N, N, T, False, False, f32, 1.0, True),
-        ("R2 += Ypre^T A", D, N, T, False, False, f32, 1.0, False),
+        # the accumulator products as a step issues them: the fused update leaves A channel-major (K-major here)
+        ("G_A += A^T A (lower, A K-major)", N, N, T, True, True, f32, 1.0, True),
+        ("R2 += Ypre^T A (A K-major)", D, N, T, False, True, f32, 1.0, False),
         ("R1 += Z^T X", N, D, T, False, False, f32, 1.0, False),
-        ("R2 with Ypre stored transposed", D, N, T, True, False, f32, 1.0, False),
-        ("R1 with X stored transposed", N, D, T, False, True, f32, 1.0, False),
-        ("G_A with A stored transposed", N, N, T, True, True, f32, 1.0, True),
         ("solve update (K = 6 x 128)", 2048, 4096, 768, True, True, f32, 1.0, False),
+        # other operand layouts: row-major A (fp32-storage path, or when the objective is reported), and transposed
+        # copies of Ypre / X that the module does not keep
+        ("G_A with A row-major", N, N, T, False, False, f32, 1.0, True),
+        ("R2 with A row-major", D, N, T, False, False, f32, 1.0, False),
+        ("R2 with Ypre stored transposed too", D, N, T, True, True, f32, 1.0, False),
+        ("R1 with X stored transposed", N, D, T, False, True, f32, 1.0, False),
     ]
     for name, M, Nn, K, ak, bk, cdt, beta, lower in cases:
         A = _rnd((M, K) if ak else (K, M), bf)
