@@ -48,6 +48,9 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-fixed-mask", action="store_true", help="skip the fixed-mask variants of the step")
     ap.add_argument("--dual", action="store_true", help="run with the scaled dual variable U (dual_mode = 1)")
+    ap.add_argument("--shard", default="modules", choices=["modules", "tokens"],
+                    help="N > 1: every rank its own module (default, no collective), or ONE module with its tokens "
+                         "split over the ranks (accumulators all-reduced once per iteration)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
     return ap.parse_args()
 
@@ -216,22 +219,33 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     api.lib()
 
-    # ---- inputs resident in HBM: this rank's module (layer index = rank)
+    # ---- inputs resident in HBM: this rank's module (layer index = rank), or its token shard of module 0
+    by_tokens = args.shard == "tokens"
+    if by_tokens and cfg.act == "swiglu":
+        raise SystemExit("--shard tokens: ReLU modules only")
     layer = rank
-    X = synth.make_activations(cfg, layer, device=dev)
-    W1_0, W2_0 = synth.make_weights(cfg, layer, device=dev)
+    wl = 0 if by_tokens else layer
+    cfg_local = synth.scaled(cfg, tokens=cfg.tokens // world) if by_tokens else cfg
+    X = synth.make_activations(cfg_local, layer, device=dev)        # another seed per rank: disjoint tokens
+    W1_0, W2_0 = synth.make_weights(cfg, wl, device=dev)
     Wg_0 = synth.make_gate_weights(cfg, layer, device=dev) if cfg.act == "swiglu" else None
     mod = api.FfnModule(X, W1_0, W2_0, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
     I_all = synth.make_importances(cfg, device=dev)
     n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
     T_soft = float(I_all.abs().mean())
-    mod.sp_ffn_init()
+    if by_tokens:
+        parallel.token_sharded_init([mod])
+    else:
+        mod.sp_ffn_init()
     torch.cuda.synchronize()
     mod.check_status()
     prm = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk, dual_mode=args.dual)
 
     def step():
-        mod.sp_admm_step(prm)
+        if by_tokens:
+            parallel.token_sharded_iterations([mod], prm, 1, read_reports=False)
+        else:
+            mod.sp_admm_step(prm)
         # layer importances -> per-layer kept counts (this module's own importance replaces its slot)
         I_all[layer:layer + 1].copy_(mod.importance)
         api.sp_allocate_sparsity(I_all, n_units, cfg.sparsity, T_soft)
@@ -263,7 +277,7 @@ def main():
     api.sp_profile_begin(False)
     mod.check_status()
     ms = parallel.max_over_ranks(ms_local, dev)
-    value = world * args.steps / (ms * 1e-3)
+    value = (1 if by_tokens else world) * args.steps / (ms * 1e-3)      # one module in all when its tokens are split
 
     if rank != 0:
         if world > 1:
@@ -399,11 +413,13 @@ def main():
         cpu = cpu_baseline(cfg, args.cpu_sample_tokens)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong" if by_tokens else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(cfg), "token_chunk": args.chunk, "dual_mode": bool(args.dual),
                        "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
-                       "parallelism": f"modules x{world} (independent, no collective)"},
+                       "parallelism": (f"tokens x{world} of one module (accumulators all-reduced once per iteration)"
+                                       if by_tokens else f"modules x{world} (independent, no collective)")},
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e, "cpu_baseline": cpu, "fixed_mask": fixed,
             "breakdown": breakdown}
     print(json.dumps(line))

@@ -384,6 +384,7 @@ class AdmmParams:
 
 class FfnModule:
     """Owns the device buffers of one FFN module and forwards to sp_ffn_init / sp_admm_step."""
+    report_fields = REPORT_FIELDS
 
     def __init__(self, X: torch.Tensor, W1_0: torch.Tensor, W2_0: torch.Tensor, dual_mode: bool = False,
                  token_chunk: int = 0, overlap_k: int = 0, Wg_0: torch.Tensor | None = None,
@@ -485,6 +486,10 @@ class FfnModule:
         cp.token_chunk = chunk
         _check(lib().sp_admm_scores(C.byref(m), C.byref(st), C.byref(cp), self.status.data_ptr(), ws.data_ptr(),
                                     ws.numel(), _stream()), "sp_admm_scores")
+
+    def select_mask(self, k_keep: int):
+        """Top-k of the current scores into the module's mask (what a step does when it reselects)."""
+        sp_apply_mask(self.scores, k_keep, mask_out=self.mask)
 
     def read_report(self) -> dict:
         return dict(zip(REPORT_FIELDS, self.report.cpu().tolist()))
