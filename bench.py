@@ -8,7 +8,8 @@ calibration tokens) followed by sp_allocate_sparsity over the model's layer impo
 Workload at N = 1 GPU: workload C2 (OPT-1.3B-shaped FFN module: d = 2048, n = 8192, 128 x 2048 = 262144
 calibration tokens in bf16, 50 % channel sparsity), synthetic seeded inputs generated on the device.
 With N > 1 GPUs every rank owns its own module (modules are independent once the kept counts are fixed), so the
-scaling is weak and the data path has no collective.
+scaling is weak and the data path has no collective.  `--shard tokens` instead splits the tokens of ONE module over
+the ranks (strong scaling; the accumulators are all-reduced once per iteration).
 
 Prints ONE JSON line (rank 0).  Besides the timed step (mask re-selected in every iteration) the line carries
 `fixed_mask` (the same module stepped without re-selection, and its continuation on the kept channels only), `e2e`
