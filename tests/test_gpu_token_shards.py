@@ -53,8 +53,12 @@ def test_two_token_shards_equal_the_unsharded_module(storage, kind):
         Z = np.concatenate([np64(m.Z).T for m in shards], axis=1)
         assert relerr(Z, st.Z) < loose
         assert abs(reports[-1]["res_act"] - rep_or["res_act"]) <= 10 * loose * reports[-1]["a_sq"]
-    else:
-        assert same_mask
+    elif not same_mask:
+        # the two runs round differently: they may only disagree on units whose scores sit at the threshold
+        sc = np64(full.scores)
+        tau = np.sort(sc)[::-1][k - 1]
+        diff = np.flatnonzero(full.mask.cpu().numpy() != shards[0].mask.cpu().numpy())
+        assert np.all(np.abs(sc[diff] - tau) <= 10 * tol * np.abs(sc).max())
     if same_mask:
         assert relerr(np64(shards[0].W1), np64(full.W1)) < 10 * tol
         assert relerr(np64(shards[0].W2), np64(full.W2)) < 10 * tol
