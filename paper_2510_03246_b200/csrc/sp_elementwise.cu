@@ -264,7 +264,10 @@ __device__ __forceinline__ float update_one(float zold, float z1, float dcorr, f
     const float h = gate * zold - (has_u ? u : 0.f);
     const float a = h + dcorr;
     const float au = a + (has_u ? u : 0.f);
-    znew = (beta * gate * au + alpha * z1) / fmaf(beta * gate, gate, alpha);
+    // The divisor lies in [alpha, alpha + beta g^2], far from the ends of the exponent range, so its correctly
+    // rounded reciprocal never leaves the fast path.  A plain division also inspects the numerator, which is tiny
+    // wherever the gate factor is: with wide-ranged gate inputs its out-of-range path made the kernel 45 % slower.
+    znew = (beta * gate * au + alpha * z1) * __frcp_rn(fmaf(beta * gate, gate, alpha));
     if (has_u) u = u + a - gate * znew;
     return a;
   }
