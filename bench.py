@@ -312,9 +312,16 @@ def main():
                 "achieved_owning_gpu": tc_own["flops"] / (tc_own["ms"] * 1e-3) / 1e12 if tc_own["ms"] > 0 else 0.0}
     hbm = peaks.get("hbm_gbs", 6650.0)
     fu = prof["fused_update"]
+    # DRAM traffic of one fused-update launch from the ncu capture in profiles/fused_update_prep_h_C2_one_chunk.md:
+    # 2.148 GB read + 2.124 GB written for one 32768-token chunk of C2 without the dual variable (algorithmic 4.29 GB)
+    fu_traffic = None
+    if (cfg.name == "C2" and cfg.n == 8192 and cfg.k_keep == 4096 and args.chunk == 32768 and not args.dual
+            and cfg.tokens % args.chunk == 0):
+        fu_traffic = 4.272e9
     roofline_hbm = {"bound": "hbm", "kernel": "fused_update_kernel",
                     "achieved": fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 if fu["ms"] else 0.0, "peak": hbm, "unit": "GB/s",
-                    "frac": (fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 / hbm) if fu["ms"] else 0.0, "traffic": None,
+                    "frac": (fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 / hbm) if fu["ms"] else 0.0, "traffic": fu_traffic,
+                    "algorithmic_bytes_per_launch": fu["bytes"] / max(fu["records"], 1),
                     "launches": fu["records"]}
     breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / args.steps,
                      **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),
