@@ -548,6 +548,31 @@ def test_swiglu_step_teacher_forced(cfg, chunk, kind, dual):
         _step_and_compare(mod, X, Wu.float(), p_gpu, p_or, TOL[X.dtype], audit, gate=gate)
 
 
+@pytest.mark.parametrize("cfg", [SWIGLU_F32, SWIGLU_BF16])
+def test_swiglu_scores_then_fixed_mask_step(cfg):
+    """The split form of a step (scores alone, then the rest with a mask chosen outside) on a gated module, without
+    the output-side objective term (bf16: the channel-major A of the gated update)."""
+    mod, X, Wg, Wu, W2 = _make_swiglu(cfg, chunk=256)
+    mod.sp_ffn_init()
+    gate = O.silu(np64(Wg) @ np64(X).T)
+    k = cfg.k_keep
+    tol = TOL[X.dtype]
+    for it in range(2):
+        mod.sp_admm_scores(api.AdmmParams(beta=1.5, rho=cfg.rho, token_chunk=256))
+        torch.cuda.synchronize()
+        st = oracle_state_from_gpu(mod)
+        st.gate = gate
+        p_or = O.AdmmParams(beta=1.5, rho=cfg.rho, k_keep=k, act="swiglu")
+        s_or, I_or = O.admm_weight_phase(copy.deepcopy(st), np64(Wu.float()), p_or, cfg.tokens)
+        assert relerr(np64(mod.scores), s_or) < tol
+        m_new, _ = O.topk_mask(mod.scores.cpu().numpy(), k - it)
+        mod.mask.copy_(torch.from_numpy(m_new).to(DEV))
+        p_fix = api.AdmmParams(beta=1.5, rho=cfg.rho, k_keep=k - it, token_chunk=256, reselect_mask=False,
+                               skip_scores=True)
+        p_or_fix = O.AdmmParams(beta=1.5, rho=cfg.rho, k_keep=k - it, act="swiglu", reselect_mask=False)
+        _step_and_compare(mod, X, Wu.float(), p_fix, p_or_fix, tol, [], gate=gate)
+
+
 def test_swiglu_argument_errors():
     mod, X, Wg, Wu, W2 = _make_swiglu(SWIGLU_F32)
     mod.sp_ffn_init()
