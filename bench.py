@@ -299,10 +299,10 @@ def main():
     peak_src = "measured (sustained, MEASURED_PEAKS.json)" if peaks else "fallback (1.4 PFLOP/s sustained)"
     achieved = tc["flops"] / (tc["ms"] * 1e-3) / 1e12 if tc["ms"] > 0 else 0.0
     # DRAM traffic of the token-pass GEMMs from the ncu capture in profiles/gemm_tc_kernel_C2_one_chunk.md: the six
-    # products of one 16384-token chunk of C2 moved 4.66 GB; traffic grows in proportion to the tokens a launch covers.
+    # products of one 16384-token chunk of C2 moved 4.22 GB; traffic grows in proportion to the tokens a launch covers.
     traffic = None
     if cfg.name == "C2" and cfg.d == 2048 and cfg.n == 8192 and cfg.k_keep == 4096 and tc["records"]:
-        traffic = 4.66e9 * (cfg.tokens / 16384.0) * args.steps / tc["records"]
+        traffic = 4.22e9 * (cfg.tokens / 16384.0) * args.steps / tc["records"]
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak_tf,
                 "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": traffic,
                 "traffic_unit": "DRAM bytes per launch (ncu, one chunk, scaled by tokens)", "peak_source": peak_src,

@@ -67,11 +67,25 @@ struct TcParams {
   TcSegments seg;    // K segments: segment s reads A at (k + a_k[s], m + a_mn[s]) and B at (k + b_k[s], n + b_mn[s])
   int32_t seg_kb;    // k-blocks per segment
   int32_t tiles_m, tiles_n, num_tiles;
-  // Work units: unit u is tile u % num_tiles restricted to k-blocks [ks * kb_per_split, (ks + 1) * kb_per_split) with
-  // ks = u / num_tiles.  ksplit > 1 only with the add-reduction epilogue (partial products add up in C).
-  int32_t ksplit, kb_per_split, num_units;
+  // Work units: the first n_plain tiles are one unit each (all of K).  The other n_cut = num_tiles - n_plain tiles are
+  // cut along K: unit n_plain + v is tile n_plain + v % n_cut restricted to k-blocks [ks * kb_per_split,
+  // (ks + 1) * kb_per_split) with ks = v / n_cut.  ksplit > 1 only with the add-reduction epilogue (partial products
+  // add up in C).  n_plain = 0 cuts every tile; n_plain = whole waves of CTA pairs cuts only the tiles of the last,
+  // partly filled wave, so that it keeps every pair busy for 1 / ksplit of a tile time.
+  int32_t ksplit, kb_per_split, num_units, n_plain;
   int32_t* status;
 };
+
+__device__ __forceinline__ void unit_map(const TcParams& p, int u, int num_kb, int& tile, int& kb0, int& kb1) {
+  if (u < p.n_plain) {
+    tile = u; kb0 = 0; kb1 = num_kb;
+    return;
+  }
+  const int v = u - p.n_plain, n_cut = p.num_tiles - p.n_plain;
+  tile = p.n_plain + v % n_cut;
+  kb0 = (v / n_cut) * p.kb_per_split;
+  kb1 = (kb0 + p.kb_per_split < num_kb) ? kb0 + p.kb_per_split : num_kb;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -314,10 +328,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t ph = 0;
       bool ok = true;
       for (int u = cid; u < p.num_units && ok; u += ncl) {
-        int tm, tn;
-        tile_coords(p, u % p.num_tiles, tm, tn);
-        const int kb0 = (u / p.num_tiles) * p.kb_per_split;
-        const int kb1 = (kb0 + p.kb_per_split < num_kb) ? kb0 + p.kb_per_split : num_kb;
+        int tm, tn, tile, kb0, kb1;
+        unit_map(p, u, num_kb, tile, kb0, kb1);
+        tile_coords(p, tile, tm, tn);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           // the leader's barrier collects the bytes of both CTAs' loads of this stage
@@ -366,8 +379,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
-        const int kb0 = (u / p.num_tiles) * p.kb_per_split;
-        const int kb1 = (kb0 + p.kb_per_split < num_kb) ? kb0 + p.kb_per_split : num_kb;
+        int tile, kb0, kb1;
+        unit_map(p, u, num_kb, tile, kb0, kb1);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(s), ph, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           tc_fence_after();
@@ -415,8 +428,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool has_cin = p.beta != 0.f;
     const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
     for (int u = cid; u < p.num_units && ok; u += ncl) {
-      int tm, tn;
-      tile_coords(p, u % p.num_tiles, tm, tn);
+      int tm, tn, tile, kb0_unused, kb1_unused;
+      unit_map(p, u, num_kb, tile, kb0_unused, kb1_unused);
+      tile_coords(p, tile, tm, tn);
       // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
       const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
@@ -733,9 +747,24 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
       p.ksplit = best;
     }
   }
+  p.n_plain = 0;
+  if (p.epi_mode == EPI_TMA_ADD && p.num_tiles > pairs_max && p.num_tiles % pairs_max != 0) {
+    // Alternative: whole waves of uncut tiles, and only the tiles of the last wave cut, as many ways as pairs are
+    // left per tile.  Times in units of one tile on one pair.
+    const int full = p.num_tiles / pairs_max, rem = p.num_tiles % pairs_max;
+    int ways = pairs_max / rem;
+    if (ways > 8) ways = 8;
+    while (ways > 1 && num_kb / ways < 32) --ways;
+    const double t_uniform = ceil((double)p.num_tiles * p.ksplit / pairs_max) / p.ksplit;
+    const double t_tail = full + 1.0 / ways;
+    if (ways > 1 && t_tail < 0.99 * t_uniform) {
+      p.n_plain = full * pairs_max;
+      p.ksplit = ways;
+    }
+  }
   p.kb_per_split = (int32_t)ceil_div(num_kb, p.ksplit);
   p.ksplit = (int32_t)ceil_div(num_kb, p.kb_per_split);
-  p.num_units = p.num_tiles * p.ksplit;
+  p.num_units = p.n_plain + (p.num_tiles - p.n_plain) * p.ksplit;
 
   static bool attr_set = false;
   if (!attr_set) {
