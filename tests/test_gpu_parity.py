@@ -89,6 +89,43 @@ def test_gemm_tensor_core_lower_only_and_persistence():
     assert relerr(np64(G), ref) < 2e-6
 
 
+@pytest.mark.parametrize("lower", [False, True])
+def test_gemm_tensor_core_last_wave_cut_along_k(lower):
+    """Accumulating products with a few more tiles than one wave of CTA pairs (84, or 91 lower-triangle tiles of a
+    Gram product, on the 74 pairs of a 148-SM part) and a long K: the whole waves run uncut and only the tiles of the
+    last wave are cut along K, their parts adding up in C.  Checked on sampled rows against an fp64 product."""
+    K = 16384
+    if lower:
+        M = N = 3328                                           # 13 x 13 tiles, 91 in the lower triangle
+        A = _gauss((M, K), 12, torch.bfloat16).to(DEV)
+        B = A
+    else:
+        M, N = 1792, 3072                                      # 7 x 12 tiles
+        A = _gauss((M, K), 12, torch.bfloat16).to(DEV)
+        B = _gauss((N, K), 13, torch.bfloat16).to(DEV)
+    Cm = _gauss((M, N), 14, torch.float32).to(DEV)
+    C0 = Cm.clone()
+    status = api.new_status()
+    api.sp_gemm(A, B, Cm, transA=False, transB=True, alpha=1.0, beta=1.0, lower_only=lower, use_tensor_cores=True,
+                status=status)
+    torch.cuda.synchronize()
+    _assert_status_clean(status)
+    rows = np.unique(np.concatenate([np.arange(0, M, 97), np.arange(M - 260, M)]))     # includes the last tiles
+    ref = np64(A[rows]) @ np64(B).T + np64(C0[rows])
+    got = np64(Cm[rows])
+    scale = np.abs(ref).max()
+    # fp32 accumulation in the tensor cores: K / 16 sequential additions, each off by up to one unit in the last place
+    # of the running sum (a K range left out or taken twice would be off by a seventh of the sum)
+    tol = (K / 16) * 2.0 ** -23
+    if lower:
+        keep = np.arange(N)[None, :] <= rows[:, None]
+        assert np.abs(np.where(keep, got - ref, 0.0)).max() < tol * scale
+        # tiles strictly above the diagonal keep C as it was
+        assert torch.equal(Cm[:256, 512:], C0[:256, 512:])
+    else:
+        assert np.abs(got - ref).max() < tol * scale
+
+
 def test_gemm_tensor_core_rejects_unaligned():
     A = _gauss((64, 36), 8, torch.bfloat16).to(DEV)   # ld = 36 is not a multiple of 8
     B = _gauss((72, 36), 9, torch.bfloat16).to(DEV)
