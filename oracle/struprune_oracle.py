@@ -393,11 +393,9 @@ def admm_weight_phase(st, W1_0, p, N):
     return s, I
 
 
-def admm_step(st, X, Ypre, W1_0, p, z_hook=None):
+def admm_step(st, X, Ypre, W1_0, p):
     """One outer step: weights from the accumulators, then a-, z- (and dual) updates, then the accumulators
-    of the new auxiliary variables.  Returns (scores, layer importance, report dict, A).
-    z_hook(Znew, z1, z2, A, U) may replace Znew before it is used further; parity tests use it to adopt the other
-    side's choice where the two candidates of the exact rule tie within rounding."""
+    of the new auxiliary variables.  Returns (scores, layer importance, report dict, A)."""
     X = np.asarray(X, F64)
     Ypre = np.asarray(Ypre, F64)
     N = X.shape[1]
@@ -409,8 +407,6 @@ def admm_step(st, X, Ypre, W1_0, p, z_hook=None):
         Znew = swiglu_zu_update(A, st.gate, z1, p.alpha, p.beta, U)    # one closed form, no select
     else:
         Znew = z_select(st.Z, z1, z2, A, p.alpha, p.beta, p.z_rule, U)
-    if z_hook is not None:
-        Znew = z_hook(Znew, z1, z2, A, U)
     if p.dual_mode:
         st.U = dual_update(st.U, A, Znew, p.act, st.gate)
     st.Z = Znew
@@ -433,6 +429,44 @@ def ffn_objective(st_W1, st_W2, X, Ypre, Z, A, alpha, beta, act="relu", gate=Non
     return (alpha * ((np.asarray(Ypre, F64) - st_W2 @ A) ** 2).sum()
             + beta * ((A - phi(Z, act, gate)) ** 2).sum()
             + alpha * ((Z - st_W1 @ X) ** 2).sum())
+
+
+# --------------------------------------------------------------------------------------------------
+# Algorithm 1 for one temperature: Steps 1-5 over the FFN modules of a model, L(T) = sum_l L_l
+# --------------------------------------------------------------------------------------------------
+def pretrained_importance(X, W1_0, W2_0, kind="wanda_l2"):
+    """Step 1 of Algorithm 1 for one FFN module: I_l = mean unit score of the pre-trained down-projection against the
+    pre-trained activation a^pre = phi(W1_0 X) (the Wanda score of Section 3.4 / Step 3 on the unpruned module)."""
+    A = phi(np.asarray(W1_0, F64) @ np.asarray(X, F64))
+    if kind == "wanda_l2":
+        return wanda_scores(W2_0, colsq=(A * A).sum(axis=1), kind="l2")[1]
+    if kind == "wanda_l1":
+        return wanda_scores(W2_0, colabs_mean=np.abs(A).mean(axis=1), kind="l1")[1]
+    raise ValueError(kind)
+
+
+def temperature_loss(layers, rbar, T_rel, iters, p, mode="softmax"):
+    """Algorithm 1 for ONE temperature of its grid.  layers[l] = (X, W1_0, W2_0) of FFN module l (tokens are columns).
+      Step 1  I_l of every pre-trained module
+      Step 2  r_l from the softmax allocation at temperature T = T_rel * mean_l |I_l| (the temperature is given
+              relative to the magnitude of the importances), kept count per layer
+      Step 3/4  the module iterations of Algorithm 2 with that kept count (at least one unit)
+      Step 5  L(T) = sum_l L_l with L_l the FFN objective of Appendix A.1 after the last iteration
+    Returns (L(T), per-layer losses, r, kept counts)."""
+    L = len(layers)
+    I = np.array([pretrained_importance(X, W1, W2, p.score_kind) for (X, W1, W2) in layers], F64)
+    T = T_rel * float(np.abs(I).mean())
+    n_units = [np.shape(W1)[0] for (_, W1, _) in layers]
+    r, k_keep = allocate_sparsity(I, n_units, rbar, T, mode)
+    losses = np.zeros(L, F64)
+    for l, (X, W1_0, W2_0) in enumerate(layers):
+        st, Ypre = ffn_init(X, W1_0, W2_0, dual_mode=p.dual_mode)
+        pl = dataclasses.replace(p, k_keep=max(1, int(k_keep[l])))
+        A = None
+        for _ in range(iters):
+            _, _, _, A = admm_step(st, X, Ypre, W1_0, pl)
+        losses[l] = ffn_objective(st.W1, st.W2, X, Ypre, st.Z, A, p.alpha, p.beta)
+    return float(losses.sum()), losses, r, k_keep
 
 
 # --------------------------------------------------------------------------------------------------

@@ -364,6 +364,59 @@ def test_ffn_init(cfg, chunk):
     assert relerr(np64(mod.absA), st.absA) < tol
 
 
+# Fraction of the entries of Z at which the exact select rule was found undecidable within the rounding of its
+# inputs, per call of the helper below (printed by pytest -s; the bound asserted is a few times what was measured).
+NEAR_TIE_FRACTIONS = []
+NEAR_TIE_LIMIT = 0.03
+
+
+def _oracle_exact_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol):
+    """The oracle's step for z_rule = "exact", composed here from the oracle's own parts so that the one decision that
+    is not unique can be audited.  The exact rule compares the objective values fn, fp of the best point of each half
+    line.  Both sides evaluate them from their own a + u and z1, which differ by rounding, so where |fn - fp| is below
+    what that rounding can move it, either candidate is a valid minimiser: there the candidate nearer to the GPU's Z
+    is adopted, and everything else is checked strictly.
+    Rounding of the inputs: a = h + D with h = phi(z) - u formed in fp32 from stored fp32 values (2^-23 relative) and
+    only the correction D = a - h going through the contractions (error up to tol max|D|); z1 = W1 x comes from the
+    recovered W1 (1e-5 in either mode: fp32 factorisation, weights carried as bf16 hi + lo parts) -- so
+        dA = tol max|D| + 2^-22 max|a + u|,  dz = 2e-5 max|z1|,  dzp = max(dA, dz) for zp = max(z2, 0),
+        |d fn| <= 2 beta |Au| dA + 2 alpha |zn - z1| dz
+        |d fp| <= 2 beta |Au - zp| (dA + dzp) + 2 alpha |zp - z1| (dzp + dz)        (first order).
+    Returns (report dict, A) like O.admm_step and leaves the new state in st."""
+    N = Xo.shape[1]
+    O.admm_weight_phase(st, W1_0, p_t, N)
+    U = st.U if p_t.dual_mode else None
+    A = O.a_update(st.W2, Yo, st.Z, p_t.alpha, p_t.beta, U, p_t.act, st.gate)
+    z1, z2 = O.z_candidates(st.W1, Xo, A, p_t.alpha, p_t.beta, U)
+    zn, zp, fn, fp = O.z_exact_candidates(z1, z2, A, p_t.alpha, p_t.beta, U)
+    Znew = O.z_select(st.Z, z1, z2, A, p_t.alpha, p_t.beta, "exact", U)
+    Au = A + (0.0 if U is None else U)
+    H = O.phi(st.Z, p_t.act, st.gate) - (0.0 if U is None else U)
+    dA = tol * np.abs(A - H).max() + 2.0 ** -22 * np.abs(Au).max()
+    dz = 2e-5 * np.abs(z1).max()
+    dzp = max(dA, dz)
+    margin = (2 * p_t.beta * np.abs(Au) * dA + 2 * p_t.alpha * np.abs(zn - z1) * dz
+              + 2 * p_t.beta * np.abs(Au - zp) * (dA + dzp) + 2 * p_t.alpha * np.abs(zp - z1) * (dzp + dz))
+    amb = (np.abs(fn - fp) <= margin) & (zn != zp)       # identical candidates are no ambiguity
+    frac = float(amb.mean())
+    NEAR_TIE_FRACTIONS.append(frac)
+    print(f"exact select: {int(amb.sum())} of {amb.size} entries ({100 * frac:.3f} %) undecidable within rounding")
+    assert frac <= NEAR_TIE_LIMIT
+    pick_n = np.abs(Zg - zn) <= np.abs(Zg - zp)
+    Znew = np.where(amb, np.where(pick_n, zn, zp), Znew)
+    if p_t.dual_mode:
+        st.U = O.dual_update(st.U, A, Znew, p_t.act, st.gate)
+    st.Z = Znew
+    st.G_A = A @ A.T
+    st.R1 = Znew @ Xo.T
+    st.R2 = Yo @ A.T
+    st.absA = np.abs(A).sum(axis=1)
+    rep = {"res_act": float(((A - O.phi(Znew, p_t.act, st.gate)) ** 2).sum()),
+           "res_out": float(p_t.alpha * ((Yo - st.W2 @ A) ** 2).sum()),
+           "res_in": float(p_t.alpha * ((Znew - st.W1 @ Xo) ** 2).sum())}
+    return rep, A
+
+
 def _step_and_compare(mod, X, W1_0, p_gpu, p_or, tol, audit, gate=None):
     """One teacher-forced step: the oracle restarts from the GPU's state before the call.  `gate` (gated modules): the
     oracle's own gate factor, computed from the inputs."""
@@ -398,25 +451,10 @@ def _step_and_compare(mod, X, W1_0, p_gpu, p_or, tol, audit, gate=None):
     p_t = copy.deepcopy(p_or)
     p_t.reselect_mask = False
     Zg = np64(mod.Z).T
-    n_amb = [0]
-
-    def adopt_near_ties(Znew, z1, z2, A, U):
-        # exact rule: where the two half-line optima have objective values equal within the rounding of the inputs,
-        # either is a valid minimiser; take the one the GPU took and check the rest strictly.
-        if p_t.z_rule != "exact":
-            return Znew
-        zn, zp, fn, fp = O.z_exact_candidates(z1, z2, A, p_t.alpha, p_t.beta, U)
-        Au = A + (0.0 if U is None else U)
-        vmax = max(np.abs(Au).max(), np.abs(z1).max())
-        margin = 4 * tol * vmax * (p_t.beta * (np.abs(Au) + np.abs(zp)) + p_t.alpha * (np.abs(zn - z1) + np.abs(zp - z1))
-                                   + tol * vmax)
-        amb = (np.abs(fn - fp) <= margin) & (zn != zp)       # identical candidates are no ambiguity
-        n_amb[0] = int(amb.sum())
-        pick_n = np.abs(Zg - zn) <= np.abs(Zg - zp)
-        return np.where(amb, np.where(pick_n, zn, zp), Znew)
-
-    _, _, rep, A = O.admm_step(st, Xo, Yo, np64(W1_0), p_t, z_hook=adopt_near_ties)
-    assert n_amb[0] <= 0.2 * Zg.size      # the near-tie set stays a minority (most entries are checked strictly)
+    if p_t.z_rule == "exact" and p_t.act == "relu":
+        rep, A = _oracle_exact_step_adopting_ties(st, Xo, Yo, np64(W1_0), p_t, Zg, tol)
+    else:
+        _, _, rep, A = O.admm_step(st, Xo, Yo, np64(W1_0), p_t)
     assert relerr(np64(mod.W1), st.W1) < tol, "W1"
     assert relerr(np64(mod.W2), st.W2) < tol, "W2"
     assert np.all(np64(mod.W1)[mask_gpu == 0] == 0) and np.all(np64(mod.W2)[:, mask_gpu == 0] == 0)
@@ -648,22 +686,60 @@ def test_admm_step_argument_errors():
     assert e.value.code == 1
 
 
-def test_free_running_iterations_fp32():
-    """K iterations without teacher forcing on a reduced copy of the smallest config: the two trajectories stay
-    together (same masks up to near-ties, values within a loose bound that allows for chaotic amplification)."""
-    cfg = synth.scaled(synth.CONFIGS["C1"], d=128, n=512, tokens=1024)
-    mod, X, W1, W2 = _make_module(cfg)
+def _free_run(cfg, iters, tol, growth, chunk=0):
+    """K iterations WITHOUT teacher forcing: the GPU module and the oracle each start from their own initialisation of
+    the same inputs and never see each other's values again, except for (1) the stored target Ypre, which in bf16 mode
+    is an INPUT of the loop rounded to the storage type, and (2) the integer decision: when the two masks of an
+    iteration differ, every disagreeing unit must be a near tie (its oracle score within twice the largest score
+    difference of the threshold: a perturbation of the scores by at most e moves the k-th largest by at most e, so no
+    other unit can change sides), and the oracle then continues with the GPU's mask, which is an equally valid
+    top-k of scores known to that accuracy.  Values are compared after every iteration; the bound grows with the
+    iteration count because each side's rounding feeds the next iteration.  Returns the per-iteration records."""
+    mod, X, W1, W2 = _make_module(cfg, chunk=chunk)
     mod.sp_ffn_init()
     torch.cuda.synchronize()
-    st, Y = O.ffn_init(np64(X).T, np64(W1), np64(W2))
-    p_gpu = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho)
-    p_or = O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho)
-    for it in range(cfg.iters):
+    Xo = np64(X).T
+    st, Y = O.ffn_init(Xo, np64(W1), np64(W2))
+    if X.dtype == torch.bfloat16:
+        Y = np64(mod.Ypre).T
+    p_gpu = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=chunk)
+    rec = []
+    for it in range(iters):
         mod.sp_admm_step(p_gpu)
-        O.admm_step(st, np64(X).T, Y, np64(W1), p_or)
-    torch.cuda.synchronize()
-    mod.check_status()
-    agree = (mod.mask.cpu().numpy() == st.mask).mean()
-    assert agree > 0.99
-    if agree == 1.0:
-        assert relerr(np64(mod.W2), st.W2) < 1e-3 and relerr(np64(mod.Z).T, st.Z) < 1e-3
+        torch.cuda.synchronize()
+        mod.check_status()
+        probe = copy.deepcopy(st)
+        s_or, _ = O.admm_weight_phase(probe, np64(W1), O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho), cfg.tokens)
+        s_gpu = np64(mod.scores)
+        e = np.abs(s_gpu - s_or).max()
+        bound = tol * growth(it)
+        assert e <= bound * np.abs(s_or).max(), ("scores", it, e / np.abs(s_or).max())
+        mask_gpu = mod.mask.cpu().numpy()
+        assert np.array_equal(mask_gpu, O.topk_mask(mod.scores.cpu().numpy(), cfg.k_keep)[0])
+        diff = np.flatnonzero(mask_gpu != probe.mask)
+        tau = np.sort(s_or)[::-1][cfg.k_keep - 1]
+        assert np.all(np.abs(s_or[diff] - tau) <= 2 * e), ("near-tie audit", it)
+        st.mask = mask_gpu.copy()
+        O.admm_step(st, Xo, Y, np64(W1), O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, reselect_mask=False))
+        errs = dict(it=it, flipped=int(diff.size), scores=e / np.abs(s_or).max(), W1=relerr(np64(mod.W1), st.W1),
+                    W2=relerr(np64(mod.W2), st.W2), Z=relerr(np64(mod.Z).T, st.Z), G_A=relerr(np64(mod.G_A), st.G_A))
+        print(errs)
+        rec.append(errs)
+        for name in ("W1", "W2", "Z", "G_A"):
+            assert errs[name] <= bound, (name, it, errs[name])
+    return rec
+
+
+def test_free_running_iterations_fp32():
+    """All K = 10 iterations of a reduced copy of the smallest workload in fp32 mode, both sides running free."""
+    cfg = synth.scaled(synth.CONFIGS["C1"], d=128, n=512, tokens=1024)
+    _free_run(cfg, cfg.iters, TOL[torch.float32], lambda it: 2.0 * (it + 1))
+
+
+@pytest.mark.parametrize("name,shape,iters", [("C2", dict(d=1024, n=4096, tokens=4096), 6),
+                                              ("C5", dict(d=1792, n=7168, tokens=6144), 5)])
+def test_free_running_iterations_bf16(name, shape, iters):
+    """Free-running iterations in bf16 mode on width- and token-reduced copies of the benchmark workload (half width)
+    and of the widest one (quarter width, 80 % pruned, more channels than tokens)."""
+    cfg = synth.scaled(synth.CONFIGS[name], **shape)
+    _free_run(cfg, iters, TOL[torch.bfloat16], lambda it: 1.0 + 0.5 * it, chunk=2048)

@@ -559,6 +559,43 @@ def test_distribute_importance_structure():
     assert np.all(np.diff(Im) < 0) and np.all(np.diff(r) < 0) and abs(r.mean() - 0.5) < 1e-12
 
 
+def _frac(tok):
+    num, _, den = tok.partition("/")
+    return float(num) / float(den) if den else float(num)
+
+
+def test_distribute_importance_golden():
+    """Algorithm "-distribute", Step 1 on hand-evaluated 2 x 2 weights (tests/golden/distribute_cases.txt): pins the
+    coefficients 0.1 (variance) and 0.01 (l2 norm) of the head term, 0.05 of the MLP term, the head slicing, the
+    attention/MLP ratio and the depth weight gamma^l with layers counted from 1."""
+    rows = {}
+    for ln in _rows("distribute_cases.txt"):
+        name, vals = ln.split("|")
+        rows[name.strip()] = [float(v) for v in vals.split()]
+    layer = {k: np.array(rows[k]).reshape(2, 2) for k in ("Wq", "Wk", "Wv", "Wo", "fc1", "fc2")}
+    rho, gamma = rows["rho_gamma"]
+    for h, want in enumerate(rows["head_terms"]):
+        l1, var, l2 = O.weight_stats(O.head_slices(layer["Wq"], layer["Wk"], layer["Wv"], layer["Wo"], h, 1))
+        assert l1 + 0.1 * var + 0.01 * l2 == pytest.approx(want, rel=1e-13)
+    Ia, Im = O.distribute_importance([layer, layer], 2, 1, rho=rho, gamma=gamma)
+    assert np.allclose(Ia, rows["I_attn"], rtol=1e-13, atol=0)
+    assert np.allclose(Im, rows["I_mlp"], rtol=1e-13, atol=0)
+
+
+def test_inverse_allocation_golden():
+    """Algorithm "-distribute", Step 2 with rational softmax weights, one case without and one with the clip."""
+    T = 0.83
+    for ln in _rows("inverse_allocation_cases.txt"):
+        rbar_s, n_s, q_s, r_s, k_s = ln.split("|")
+        q = np.array([_frac(t) for t in q_s.split()])
+        want_r = np.array([_frac(t) for t in r_s.split()])
+        want_k = [int(t) for t in k_s.split()]
+        I = -T * np.log(q)
+        r, k = O.allocate_sparsity(I, [int(n_s)] * len(q), float(rbar_s), T, mode="inverse")
+        assert np.allclose(r, want_r, rtol=1e-12, atol=0)
+        assert list(k) == want_k
+
+
 # ------------------------------------------------------------------------------------------------ global threshold
 def test_global_threshold_worked_example():
     """Appendix B, Algorithm 3: one threshold over the scores of all layers, K = floor(r n L) kept.  Two layers of three
@@ -606,3 +643,31 @@ def test_global_threshold_can_empty_a_layer_unless_min_keep():
     assert counts.tolist() == [3, 0]
     masks, counts, _ = O.global_threshold_masks(S, 0.5, min_keep=1)
     assert masks.tolist() == [[1, 1, 1], [0, 0, 1]] and counts.tolist() == [3, 1]
+
+
+# ------------------------------------------------------------------------------------------------ Algorithm 1, one temperature
+def test_temperature_loss_special_cases():
+    """L(T) of Algorithm 1 Step 5 against what the paper's construction fixes: with nothing pruned (rbar = 0) and a
+    vanishing ridge the recovered weights are the pre-trained ones and every term of the objective is zero, at any
+    temperature; identical layers get the uniform allocation, so L(T) is L times one layer's loss for every T; and the
+    kept counts follow Step 2 (softmax of -I/T at T = T_rel mean|I|: the least important layer is pruned most)."""
+    rng = _rng(31)
+    d, n, N = 6, 14, 60
+    mk = lambda s: (rng.standard_normal((d, N)), s * rng.standard_normal((n, d)), rng.standard_normal((d, n)))
+    layers = [mk(1.0), mk(2.0), mk(3.0)]
+    p = O.AdmmParams(rho=1e-10, rho_relative=False)
+    for T_rel in (0.3, 3.0):
+        L0, per, r, k = O.temperature_loss(layers, 0.0, T_rel, 2, p)
+        scale = sum(np.linalg.norm(W2 @ np.maximum(W1 @ X, 0)) ** 2 for X, W1, W2 in layers)
+        assert np.all(r == 0) and list(k) == [n] * 3 and L0 < 1e-12 * scale
+    same = [layers[1]] * 3
+    La, per_a, r_a, k_a = O.temperature_loss(same, 0.5, 0.3, 2, O.AdmmParams(rho=0.1))
+    Lb, per_b, r_b, k_b = O.temperature_loss(same, 0.5, 3.0, 2, O.AdmmParams(rho=0.1))
+    assert np.allclose(r_a, 0.5) and np.allclose(r_b, 0.5) and list(k_a) == [7] * 3
+    assert La == pytest.approx(3 * per_a[0], rel=1e-12) and La == pytest.approx(Lb, rel=1e-12) and La > 0
+    # different layers: importances grow with the weight scale, so the first layer is pruned most, and the lower the
+    # temperature the more uneven the kept counts
+    _, _, r_lo, k_lo = O.temperature_loss(layers, 0.5, 0.3, 1, O.AdmmParams(rho=0.1))
+    _, _, r_hi, k_hi = O.temperature_loss(layers, 0.5, 3.0, 1, O.AdmmParams(rho=0.1))
+    assert np.all(np.diff(r_lo) < 0) and np.all(np.diff(r_hi) < 0)
+    assert (k_lo.max() - k_lo.min()) > (k_hi.max() - k_hi.min())
