@@ -34,6 +34,8 @@ if ROOT not in sys.path:
 
 METRIC = "ADMM iterations/sec per module"
 UNIT = "iterations/s"
+DTYPE_NAME = {"bf16": "bf16", "f32": "f32"}
+WORKLOAD_GB = {"C1": 1, "C2": 40, "C3": 60, "C4": 110, "C5": 160}    # free device memory a workload needs
 
 
 def parse():
@@ -53,6 +55,11 @@ def parse():
                     help="N > 1: every rank its own module (default, no collective), or ONE module with its tokens "
                          "split over the ranks (accumulators all-reduced once per iteration)")
     ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
+    ap.add_argument("--workloads", default="C3,C4,C5",
+                    help="1 GPU: further workloads measured after the main one and reported under `workloads` "
+                         "(empty string: none)")
+    ap.add_argument("--workload-steps", type=int, default=5)
+    ap.add_argument("--workload-warmup", type=int, default=2)
     return ap.parse_args()
 
 
@@ -157,6 +164,7 @@ def cpu_baseline(cfg, sample_tokens: int) -> dict:
     tw, tt = oracle_iteration_seconds(cfg, sample_tokens)
     full = tw + tt * (cfg.tokens / sample_tokens)
     return {"value": 1.0 / full, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+            "implementation": "numpy fp64 (LAPACK / BLAS on all threads counted in cores)",
             "sample": (f"one oracle iteration at d={cfg.d}, n={cfg.n} on {sample_tokens} of {cfg.tokens} tokens "
                        f"({tw + tt:.1f} s measured: weight phase {tw:.1f} s + token phase {tt:.1f} s); the token "
                        f"phase is scaled x{cfg.tokens // sample_tokens} to the full token count (extrapolated)")}
@@ -183,7 +191,9 @@ def run_reference(args, cfg):
             "steps": steps, "warmup": args.warmup, "ms_per_step": 1e3 * full, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": workload_name(cfg)},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                             "implementation": "numpy fp64 (LAPACK / BLAS on all threads counted in cores)",
+                             "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "wall_s": time.perf_counter() - t0}
     print(json.dumps(line))
@@ -197,6 +207,149 @@ def workload_name(cfg) -> str:
 
 
 # ------------------------------------------------------------------------------------------------ our arm
+def load_peaks():
+    try:
+        return json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        return {}
+
+
+def captured_traffic(kernel: str, key: str):
+    """DRAM bytes of one launch group from the ncu captures summarised under profiles/ (profiles/ncu_dram_traffic.txt:
+    JSON, one record per captured kernel with the sha256 of the source file it was built from).  Returns None when no
+    record matches or when the kernel's source has changed since the capture (the counters are then stale)."""
+    import hashlib
+    try:
+        recs = json.load(open(os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")))["records"]
+    except Exception:
+        return None
+    for r in recs:
+        if r.get("kernel") == kernel and r.get("key") == key:
+            try:
+                src = open(os.path.join(ROOT, r["source"]), "rb").read()
+            except Exception:
+                return None
+            return r["dram_bytes"] if hashlib.sha256(src).hexdigest() == r.get("source_sha256") else None
+    return None
+
+
+def build_module(cfg, args, dev, layer, by_tokens, world):
+    import torch
+    from paper_2510_03246_b200 import api, parallel, synth
+    wl = 0 if by_tokens else layer
+    cfg_local = synth.scaled(cfg, tokens=cfg.tokens // world) if by_tokens else cfg
+    X = synth.make_activations(cfg_local, layer, device=dev)        # another seed per rank: disjoint tokens
+    W1_0, W2_0 = synth.make_weights(cfg, wl, device=dev)
+    Wg_0 = synth.make_gate_weights(cfg, layer, device=dev) if cfg.act == "swiglu" else None
+    mod = api.FfnModule(X, W1_0, W2_0, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
+    if by_tokens:
+        parallel.token_sharded_init([mod])
+    else:
+        mod.sp_ffn_init()
+    torch.cuda.synchronize()
+    mod.check_status()
+    return mod, X, W1_0, W2_0, Wg_0
+
+
+def measure(cfg, args, dev, mod, layer, by_tokens, world, steps, warmup, local_rank):
+    """Times `steps` steps of the module (profiling off: nothing but the library's own launches in the timed region),
+    then the same number of steps again with a CUDA event pair around every launch / phase for the per-kernel figures.
+    Returns (ms of the timed loop on this rank, launches in it, clocks, per-kind event records, ms of the profiled loop)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2510_03246_b200 import api, parallel, synth
+    I_all = synth.make_importances(cfg, device=dev)
+    n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
+    T_soft = float(I_all.abs().mean())
+    prm = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk, dual_mode=args.dual)
+    slot = layer % cfg.layers
+
+    def step():
+        if by_tokens:
+            parallel.token_sharded_iterations([mod], prm, 1, read_reports=False)
+        else:
+            mod.sp_admm_step(prm)
+        # layer importances -> per-layer kept counts (this module's own importance replaces its slot)
+        I_all[slot:slot + 1].copy_(mod.importance)
+        api.sp_allocate_sparsity(I_all, n_units, cfg.sparsity, T_soft)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    mod.check_status()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    api.sp_profile_begin(0)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    ms_local = ev0.elapsed_time(ev1)
+    launches = api.sp_launch_count()
+    mod.check_status()
+    # second loop: the same steps with events around every launch
+    api.sp_profile_begin(True)
+    ev0.record()
+    for _ in range(steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    prof = api.sp_profile_read()
+    api.sp_profile_begin(False)
+    mod.check_status()
+    return ms_local, launches, clocks, prof, ev0.elapsed_time(ev1), prm
+
+
+def rooflines(cfg, args, prof, steps, peaks):
+    """Roofline records of the dominant kernel (tcgen05 GEMM, tensor bound) and of the fused update (HBM bound) from the
+    per-launch CUDA events, plus the per-kind breakdown."""
+    # launches that own the whole GPU, and the z1 products that run on a subset of the SM pairs beside the recovery
+    # on the kept support (their durations are stretched by design); the roofline figure covers both
+    tc_own, tc_sh = prof["gemm_tc"], prof.get("gemm_tc_shared", {"records": 0, "ms": 0.0, "flops": 0.0, "bytes": 0.0})
+    tc = {k: tc_own[k] + tc_sh[k] for k in ("records", "ms", "flops")}
+    peak_tf = peaks.get("bf16_tflops_sustained", 1400.0)
+    peak_src = "measured (sustained, MEASURED_PEAKS.json)" if peaks else "fallback (1.4 PFLOP/s sustained)"
+    achieved = tc["flops"] / (tc["ms"] * 1e-3) / 1e12 if tc["ms"] > 0 else 0.0
+    # DRAM traffic of the token-pass GEMMs: captured with ncu on one 16384-token chunk; the traffic of each of these
+    # products grows in proportion to the tokens it covers
+    traffic = None
+    t16 = captured_traffic("gemm_tc_kernel", f"{cfg.name}:d={cfg.d},n={cfg.n},k={cfg.k_keep},tokens=16384")
+    if t16 is not None and tc["records"]:
+        traffic = t16 * (cfg.tokens / 16384.0) * steps / tc["records"]
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": traffic,
+                "traffic_unit": "DRAM bytes per launch (ncu, one chunk, scaled by tokens)", "peak_source": peak_src,
+                "launches": tc["records"], "avg_launch_ms": tc["ms"] / max(tc["records"], 1),
+                "algorithmic_flops_per_launch": tc["flops"] / max(tc["records"], 1),
+                "launches_owning_gpu": tc_own["records"],
+                "achieved_owning_gpu": tc_own["flops"] / (tc_own["ms"] * 1e-3) / 1e12 if tc_own["ms"] > 0 else 0.0}
+    hbm = peaks.get("hbm_gbs", 6650.0)
+    fu = prof["fused_update"]
+    fu_traffic = None
+    if args.chunk == 32768 and not args.dual and cfg.tokens % args.chunk == 0:
+        fu_traffic = captured_traffic("fused_update_kernel", f"{cfg.name}:n={cfg.n},k={cfg.k_keep},tokens=32768")
+    fu_gbs = fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 if fu["ms"] else 0.0
+    roofline_hbm = {"bound": "hbm", "kernel": "fused_update_kernel", "achieved": fu_gbs, "peak": hbm, "unit": "GB/s",
+                    "frac": fu_gbs / hbm, "traffic": fu_traffic,
+                    "algorithmic_bytes_per_launch": fu["bytes"] / max(fu["records"], 1), "launches": fu["records"],
+                    "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback (6.65 TB/s)"}
+    breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / steps,
+                     **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),
+                     **({"gbs": v["bytes"] / (v["ms"] * 1e-3) / 1e9, "hbm_frac": v["bytes"] / (v["ms"] * 1e-3) / 1e9 / hbm}
+                        if v["bytes"] and v["ms"] else {})}
+                 for k, v in prof.items() if v["records"]}
+    return roofline, roofline_hbm, breakdown
+
+
 def main():
     args = parse()
     from paper_2510_03246_b200 import synth
@@ -225,58 +378,9 @@ def main():
     if by_tokens and cfg.act == "swiglu":
         raise SystemExit("--shard tokens: ReLU modules only")
     layer = rank
-    wl = 0 if by_tokens else layer
-    cfg_local = synth.scaled(cfg, tokens=cfg.tokens // world) if by_tokens else cfg
-    X = synth.make_activations(cfg_local, layer, device=dev)        # another seed per rank: disjoint tokens
-    W1_0, W2_0 = synth.make_weights(cfg, wl, device=dev)
-    Wg_0 = synth.make_gate_weights(cfg, layer, device=dev) if cfg.act == "swiglu" else None
-    mod = api.FfnModule(X, W1_0, W2_0, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
-    I_all = synth.make_importances(cfg, device=dev)
-    n_units = torch.full((cfg.layers,), cfg.n, dtype=torch.int64, device=dev)
-    T_soft = float(I_all.abs().mean())
-    if by_tokens:
-        parallel.token_sharded_init([mod])
-    else:
-        mod.sp_ffn_init()
-    torch.cuda.synchronize()
-    mod.check_status()
-    prm = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=args.chunk, dual_mode=args.dual)
-
-    def step():
-        if by_tokens:
-            parallel.token_sharded_iterations([mod], prm, 1, read_reports=False)
-        else:
-            mod.sp_admm_step(prm)
-        # layer importances -> per-layer kept counts (this module's own importance replaces its slot)
-        I_all[layer:layer + 1].copy_(mod.importance)
-        api.sp_allocate_sparsity(I_all, n_units, cfg.sparsity, T_soft)
-
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    mod.check_status()
-
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    time.sleep(0.3)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    api.sp_profile_begin(True)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    clocks = sampler.stop()
-    ms_local = ev0.elapsed_time(ev1)
-    launches = api.sp_launch_count()
-    prof = api.sp_profile_read()
-    api.sp_profile_begin(False)
-    mod.check_status()
+    mod, X, W1_0, W2_0, Wg_0 = build_module(cfg, args, dev, layer, by_tokens, world)
+    ms_local, launches, clocks, prof, ms_prof, prm = measure(cfg, args, dev, mod, layer, by_tokens, world, args.steps,
+                                                             args.warmup, local_rank)
     ms = parallel.max_over_ranks(ms_local, dev)
     value = (1 if by_tokens else world) * args.steps / (ms * 1e-3)      # one module in all when its tokens are split
 
@@ -285,49 +389,8 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (the tcgen05 GEMM), from CUDA events recorded around each launch
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except Exception:
-        pass
-    # launches that own the whole GPU, and the z1 products that run on a subset of the SM pairs beside the recovery
-    # on the kept support (their durations are stretched by design); the roofline figure covers both
-    tc_own, tc_sh = prof["gemm_tc"], prof.get("gemm_tc_shared", {"records": 0, "ms": 0.0, "flops": 0.0, "bytes": 0.0})
-    tc = {k: tc_own[k] + tc_sh[k] for k in ("records", "ms", "flops")}
-    peak_tf = peaks.get("bf16_tflops_sustained", 1400.0)
-    peak_src = "measured (sustained, MEASURED_PEAKS.json)" if peaks else "fallback (1.4 PFLOP/s sustained)"
-    achieved = tc["flops"] / (tc["ms"] * 1e-3) / 1e12 if tc["ms"] > 0 else 0.0
-    # DRAM traffic of the token-pass GEMMs from the ncu capture in profiles/gemm_tc_kernel_C2_one_chunk.md: the six
-    # products of one 16384-token chunk of C2 moved 4.22 GB; traffic grows in proportion to the tokens a launch covers.
-    traffic = None
-    if cfg.name == "C2" and cfg.d == 2048 and cfg.n == 8192 and cfg.k_keep == 4096 and tc["records"]:
-        traffic = 4.22e9 * (cfg.tokens / 16384.0) * args.steps / tc["records"]
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved, "peak": peak_tf,
-                "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": traffic,
-                "traffic_unit": "DRAM bytes per launch (ncu, one chunk, scaled by tokens)", "peak_source": peak_src,
-                "launches": tc["records"], "avg_launch_ms": tc["ms"] / max(tc["records"], 1),
-                "algorithmic_flops_per_launch": tc["flops"] / max(tc["records"], 1),
-                "launches_owning_gpu": tc_own["records"],
-                "achieved_owning_gpu": tc_own["flops"] / (tc_own["ms"] * 1e-3) / 1e12 if tc_own["ms"] > 0 else 0.0}
-    hbm = peaks.get("hbm_gbs", 6650.0)
-    fu = prof["fused_update"]
-    # DRAM traffic of one fused-update launch from the ncu capture in profiles/fused_update_prep_h_C2_one_chunk.md:
-    # 2.148 GB read + 2.124 GB written for one 32768-token chunk of C2 without the dual variable (algorithmic 4.29 GB)
-    fu_traffic = None
-    if (cfg.name == "C2" and cfg.n == 8192 and cfg.k_keep == 4096 and args.chunk == 32768 and not args.dual
-            and cfg.tokens % args.chunk == 0):
-        fu_traffic = 4.272e9
-    roofline_hbm = {"bound": "hbm", "kernel": "fused_update_kernel",
-                    "achieved": fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 if fu["ms"] else 0.0, "peak": hbm, "unit": "GB/s",
-                    "frac": (fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 / hbm) if fu["ms"] else 0.0, "traffic": fu_traffic,
-                    "algorithmic_bytes_per_launch": fu["bytes"] / max(fu["records"], 1),
-                    "launches": fu["records"]}
-    breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / args.steps,
-                     **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),
-                     **({"gbs": v["bytes"] / (v["ms"] * 1e-3) / 1e9, "hbm_frac": v["bytes"] / (v["ms"] * 1e-3) / 1e9 / hbm}
-                        if v["bytes"] and v["ms"] else {})}
-                 for k, v in prof.items() if v["records"]}
+    peaks = load_peaks()
+    roofline, roofline_hbm, breakdown = rooflines(cfg, args, prof, args.steps, peaks)
 
     # ---- the variant with the mask fixed after the first iterations (Algorithm 1: Step 3 fixes the masks before the
     # SparseLLM iterations): the same module stepped without re-selection, and its continuation on the kept channels
@@ -375,7 +438,11 @@ def main():
         from paper_2510_03246_b200 import pipeline
         hH, hWo = synth.make_attention_inputs(cfg, layer)
         hH = hH.pin_memory(); hWo = hWo.pin_memory()
-        k_heads = max(1, cfg.heads - int(cfg.heads * cfg.sparsity + 0.5))
+        # kept heads: the uniform allocation of the config's sparsity over the heads, rounded by the library
+        _, kh = api.sp_allocate_sparsity(torch.ones(1, dtype=torch.float64, device=dev),
+                                         torch.tensor([cfg.heads], dtype=torch.int64, device=dev), cfg.sparsity, 1.0,
+                                         api.SP_ALLOC_UNIFORM)
+        k_heads = max(1, int(kh.item()))
         # results come back into pinned host buffers
         oW1 = torch.empty(cfg.n, cfg.d, dtype=torch.float32).pin_memory(); oW2 = torch.empty(cfg.d, cfg.n, dtype=torch.float32).pin_memory()
         omask = torch.empty(cfg.n, dtype=torch.uint8).pin_memory()
@@ -415,6 +482,35 @@ def main():
                        "iterations; W1, W2, mask back to host; then the attention half with fixed head outputs (H, "
                        "W_O in; head scores, head mask, W_O recovery on the kept heads; W_O, mask out); "
                        "layers_per_s is that whole job per second, value = iterations / that time"}
+        del m2, dX, dW1, dW2, dWg, dH, dWo, Ya, Wo_new
+    else:
+        del mod, X, W1_0, W2_0, Wg_0
+    torch.cuda.empty_cache()
+
+    # ---- the other single-GPU workloads, largest last (one module resident at a time)
+    workloads = None
+    if args.workloads and world == 1 and not by_tokens:
+        workloads = {}
+        for name in [w for w in args.workloads.split(",") if w and w != cfg.name]:
+            wcfg = synth.CONFIGS[name]
+            free, _ = torch.cuda.mem_get_info()
+            if free < WORKLOAD_GB.get(name, 0) << 30:
+                workloads[name] = {"skipped": f"needs about {WORKLOAD_GB[name]} GB of free device memory"}
+                continue
+            wmod, wX, wW1, wW2, wWg = build_module(wcfg, args, dev, 0, False, 1)
+            w_ms, w_launches, w_clocks, w_prof, w_ms_prof, _ = measure(wcfg, args, dev, wmod, 0, False, 1,
+                                                                       args.workload_steps, args.workload_warmup,
+                                                                       local_rank)
+            r_tc, r_hbm, w_break = rooflines(wcfg, args, w_prof, args.workload_steps, peaks)
+            workloads[name] = {"workload": workload_name(wcfg), "dtype": DTYPE_NAME[wcfg.storage],
+                               "steps": args.workload_steps, "warmup": args.workload_warmup,
+                               "ms_per_step": w_ms / args.workload_steps, "value": args.workload_steps / (w_ms * 1e-3),
+                               "unit": UNIT, "gpu_launches": w_launches, "clocks": w_clocks, "roofline": r_tc,
+                               "roofline_hbm": r_hbm,
+                               "solve_phase_ms_per_step": w_break.get("solve_phase", {}).get("ms_per_step"),
+                               "profiled_ms_per_step": w_ms_prof / args.workload_steps}
+            del wmod, wX, wW1, wW2, wWg
+            torch.cuda.empty_cache()
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -423,12 +519,17 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "strong" if by_tokens else "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": DTYPE_NAME[cfg.storage], "data": "synthetic",
             "config": {"workload": workload_name(cfg), "token_chunk": args.chunk, "dual_mode": bool(args.dual),
                        "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
                        "parallelism": (f"tokens x{world} of one module (accumulators all-reduced once per iteration)"
                                        if by_tokens else f"modules x{world} (independent, no collective)")},
-            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e, "cpu_baseline": cpu, "fixed_mask": fixed,
+            "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e,
+            "cpu_baseline": cpu, "fixed_mask": fixed, "workloads": workloads,
+            "profiled_ms_per_step": ms_prof / args.steps,
+            "profile_note": "value / ms_per_step: timed loop with nothing but the library's launches; roofline, "
+                            "roofline_hbm and breakdown: the same steps repeated right after it with a CUDA event pair "
+                            "around every launch or phase (profiled_ms_per_step)",
             "breakdown": breakdown}
     print(json.dumps(line))
     if world > 1:

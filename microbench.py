@@ -1,10 +1,10 @@
 """Per-kernel micro-benchmarks of libsp on one GPU (CUDA-event timings; also the small cases profiled with ncu).
 
-    python -m paper_2510_03246_b200.microbench gemm  [--reps 5 --warm 2]   GEMM shapes of one C2 token chunk
-    python -m paper_2510_03246_b200.microbench solve [--reps 3 --warm 1]   regularised solves of a C2 step
-    python -m paper_2510_03246_b200.microbench mask  [--reps 5 --warm 2]   scores, allocation and top-k as standalone
+    python microbench.py gemm  [--reps 5 --warm 2]   GEMM shapes of one C2 token chunk
+    python microbench.py solve [--reps 3 --warm 1]   regularised solves of a C2 step
+    python microbench.py mask  [--reps 5 --warm 2]   scores, allocation and top-k as standalone
                                                                            kernels (L2 flushed before every call)
-    python -m paper_2510_03246_b200.microbench lockstep [--reps 3 --warm 1] lock-step iterations of several C2-wide
+    python microbench.py lockstep [--reps 3 --warm 1] lock-step iterations of several C2-wide
                                                                            layers under one global threshold
 
 Inputs are random (torch.randn on the device): these runs time kernels, they check nothing.
@@ -15,7 +15,7 @@ import argparse
 
 import torch
 
-from . import api
+from paper_2510_03246_b200 import api
 
 DEV = "cuda"
 T, D, N = 16384, 2048, 8192      # tokens of one chunk, d_model, FFN channels of workload C2

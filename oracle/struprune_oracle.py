@@ -500,3 +500,170 @@ def swiglu_zu_update(A, g, z1u, alpha, beta, U=None):
     """argmin_zu beta (a + u - g zu)^2 + alpha (zu - z1u)^2 for a gated unit a = g * zu, g = SiLU(gate)."""
     Au = np.asarray(A, F64) + (0.0 if U is None else np.asarray(U, F64))
     return (beta * g * Au + alpha * z1u) / (beta * g * g + alpha)
+
+
+# --------------------------------------------------------------------------------------------------
+# Multi-head attention, Method 2 (Appendix A, "Computation on Multi-Head Attention layers"; Algorithm 2, SparseLLM2)
+#
+# One attention module on one sequence of T tokens (columns of X in R^{d x T}); h heads of width d_h = d / h; head i
+# owns rows [i d_h, (i+1) d_h) of W_Q X, W_K X, W_V X.  Forward definition (paper, per head):
+#     S_i = Q_i^T K_i / sqrt(d_h)  (T x T, rows = queries),  P_i = softmax over the keys of each row of S_i,
+#     head_i = V_i P_i^T  (d_h x T),  a^attn = Concat_i head_i  (d x T),  z_{l+1}^pre = W_O a^attn.
+# Readings (the section is printed with inconsistent shapes; none of these choices is fixed by the paper):
+#   * Method 2's last two terms are printed as |z_l - (M^Q.W^Q) a_{l-1}|^2 + |z_l - (M^K.W^K) a_{l-1}|^2 with one z_l,
+#     which cannot equal two different d x T products, while z_l is also the T x T argument of the softmax.  Read as
+#     "separate constraints for the Q and K projections": the auxiliary output z_l is the PAIR (Zq, Zk) with
+#     Zq ~ W_Q X, Zk ~ W_K X, and the softmax term sees the logits S(Zq, Zk).  Each projection then has the linear
+#     recovery W = z a^+ that Algorithm 2 runs "for W_Q, W_K, W_V, W_O separately".
+#   * a_l is the attention-probability tensor P (one T x T matrix per head), a^attn_l the concatenated head outputs.
+#   * Eq. (85) [a_l] is quadratic in P; the paper prescribes gradient steps: `a_steps` steps of plain gradient descent
+#     with the step 1 / L, L = 2 (alpha |V_i|_F^2 + beta) >= the largest curvature of that quadratic (so every step
+#     descends), per head.
+#   * Eq. (86) [a^attn_l] is an unconstrained quadratic with the closed-form minimiser
+#     (W_O^T W_O + I)^-1 (W_O^T z_{l+1}^pre + Concat_i V_i P_i^T); the paper names no solver for it, the minimiser is used.
+#   * Eq. (87) [z_l] goes through the softmax: `z_steps` steps of gradient descent on (Zq, Zk) jointly with the step
+#     eta_z / (2 alpha + beta (|Zq_i|_F^2 + |Zk_i|_F^2) / d_h) per head (a bound on the Gauss-Newton curvature of the
+#     softmax term plus the curvature 2 alpha of the quadratic terms), eta_z <= 1.
+#   * The elementwise "if z < 0" select that Algorithm 2 repeats inside SparseLLM2 belongs to the ReLU module and has
+#     no counterpart for a softmax; it is not applied.
+#   * causal = True masks keys after the query (the decoder models the paper prunes are causal; the printed formulas
+#     omit the mask "for clarity").
+# Parity unpinned against the paper (it prints no numbers for this path); what pins the code below is mathematics:
+# finite-difference gradients, stationarity of the closed form, descent of every sub-step, and special cases.
+# --------------------------------------------------------------------------------------------------
+@dataclasses.dataclass
+class MhaParams:
+    n_heads: int = 1
+    alpha: float = 1.0
+    beta: float = 1.0
+    a_steps: int = 4
+    z_steps: int = 4
+    eta_z: float = 1.0
+    causal: bool = True
+
+
+def softmax_rows(S, causal=False):
+    """Row-wise softmax of a T x T logit matrix; with `causal`, key u > query t gets probability 0."""
+    S = np.asarray(S, F64)
+    if causal:
+        T = S.shape[-1]
+        S = np.where(np.tril(np.ones((T, T), bool)), S, -np.inf)
+    E = np.exp(S - S.max(axis=-1, keepdims=True))
+    return E / E.sum(axis=-1, keepdims=True)
+
+
+def mha_logits(Zq_i, Zk_i):
+    """S_i = Q_i^T K_i / sqrt(d_h) for one head (inputs d_h x T, tokens are columns)."""
+    return np.asarray(Zq_i, F64).T @ np.asarray(Zk_i, F64) / math.sqrt(np.shape(Zq_i)[0])
+
+
+def mha_forward(X, Wq, Wk, Wv, Wo, n_heads, causal=True):
+    """The attention module as the paper defines it, on one sequence.  Returns (Zq, Zk, V, P [h, T, T], Aattn, Y)."""
+    X = np.asarray(X, F64)
+    d, T = X.shape
+    dh = d // n_heads
+    Zq, Zk, V = np.asarray(Wq, F64) @ X, np.asarray(Wk, F64) @ X, np.asarray(Wv, F64) @ X
+    P = np.zeros((n_heads, T, T), F64)
+    A = np.zeros((d, T), F64)
+    for i in range(n_heads):
+        r = slice(i * dh, (i + 1) * dh)
+        P[i] = softmax_rows(mha_logits(Zq[r], Zk[r]), causal)
+        A[r] = V[r] @ P[i].T
+    return Zq, Zk, V, P, A, np.asarray(Wo, F64) @ A
+
+
+def mha_heads(V, P, n_heads):
+    """Concat_i V_i P_i^T (d x T)."""
+    d = V.shape[0]
+    dh = d // n_heads
+    return np.concatenate([V[i * dh:(i + 1) * dh] @ P[i].T for i in range(n_heads)], axis=0)
+
+
+def mha_objective(X, Ypre, Wq, Wk, Wv, Wo, Zq, Zk, P, Aattn, p):
+    """Method 2 objective on one sequence; returns its five terms in the printed order."""
+    X = np.asarray(X, F64)
+    V = np.asarray(Wv, F64) @ X
+    dh = X.shape[0] // p.n_heads
+    t1 = p.alpha * ((np.asarray(Ypre, F64) - np.asarray(Wo, F64) @ Aattn) ** 2).sum()
+    t2 = p.alpha * ((Aattn - mha_heads(V, P, p.n_heads)) ** 2).sum()
+    t3 = 0.0
+    for i in range(p.n_heads):
+        r = slice(i * dh, (i + 1) * dh)
+        t3 += p.beta * ((P[i] - softmax_rows(mha_logits(Zq[r], Zk[r]), p.causal)) ** 2).sum()
+    t4 = p.alpha * ((Zq - np.asarray(Wq, F64) @ X) ** 2).sum()
+    t5 = p.alpha * ((Zk - np.asarray(Wk, F64) @ X) ** 2).sum()
+    return np.array([t1, t2, t3, t4, t5], F64)
+
+
+def mha_a_objective_grad(P_i, A_i, V_i, Phi_i, alpha, beta):
+    """Eq. (85) for one head: f(P) = alpha |A_i - V_i P^T|^2 + beta |P - Phi_i|^2 and its gradient in P."""
+    R = A_i - V_i @ P_i.T
+    f = alpha * (R ** 2).sum() + beta * ((P_i - Phi_i) ** 2).sum()
+    g = -2.0 * alpha * (R.T @ V_i) + 2.0 * beta * (P_i - Phi_i)
+    return f, g
+
+
+def mha_a_update(P, Aattn, V, Zq, Zk, p):
+    """`a_steps` gradient steps of Eq. (85) on every head's P_i with the step 1 / (2 (alpha |V_i|_F^2 + beta))."""
+    dh = V.shape[0] // p.n_heads
+    P = P.copy()
+    for i in range(p.n_heads):
+        r = slice(i * dh, (i + 1) * dh)
+        Phi = softmax_rows(mha_logits(Zq[r], Zk[r]), p.causal)
+        step = 1.0 / (2.0 * (p.alpha * (V[r] ** 2).sum() + p.beta))
+        for _ in range(p.a_steps):
+            _, g = mha_a_objective_grad(P[i], Aattn[r], V[r], Phi, p.alpha, p.beta)
+            P[i] = P[i] - step * g
+    return P
+
+
+def mha_attn_update(Ypre, Wo, Hd):
+    """Minimiser of Eq. (86): a^attn = (W_O^T W_O + I)^-1 (W_O^T z_{l+1}^pre + Hd), Hd = Concat_i V_i P_i^T
+    (alpha multiplies both terms and drops out)."""
+    Wo = np.asarray(Wo, F64)
+    d = Wo.shape[1]
+    return np.linalg.solve(Wo.T @ Wo + np.eye(d), Wo.T @ np.asarray(Ypre, F64) + Hd)
+
+
+def mha_z_objective_grad(Zq_i, Zk_i, P_i, Tq_i, Tk_i, alpha, beta, causal):
+    """Eq. (87) for one head: f = beta |P_i - softmax(S(Zq, Zk))|^2 + alpha |Zq - Tq|^2 + alpha |Zk - Tk|^2 with the
+    targets Tq = (W_Q X)_i, Tk = (W_K X)_i; returns (f, df/dZq, df/dZk).  Softmax backward written out:
+    dS = 2 beta Phi * (E - rowsum(E * Phi)), E = Phi - P."""
+    dh = Zq_i.shape[0]
+    Phi = softmax_rows(mha_logits(Zq_i, Zk_i), causal)
+    E = Phi - P_i
+    f = beta * (E ** 2).sum() + alpha * ((Zq_i - Tq_i) ** 2).sum() + alpha * ((Zk_i - Tk_i) ** 2).sum()
+    dS = 2.0 * beta * Phi * (E - (E * Phi).sum(axis=1, keepdims=True))
+    gq = Zk_i @ dS.T / math.sqrt(dh) + 2.0 * alpha * (Zq_i - Tq_i)
+    gk = Zq_i @ dS / math.sqrt(dh) + 2.0 * alpha * (Zk_i - Tk_i)
+    return f, gq, gk
+
+
+def mha_z_step_size(Zq_i, Zk_i, alpha, beta, eta_z):
+    dh = Zq_i.shape[0]
+    return eta_z / (2.0 * alpha + beta * ((Zq_i ** 2).sum() + (Zk_i ** 2).sum()) / dh)
+
+
+def mha_z_update(Zq, Zk, P, Tq, Tk, p):
+    """`z_steps` joint gradient steps of Eq. (87) on (Zq_i, Zk_i) of every head; the step is recomputed from the
+    current iterate before each step."""
+    dh = Zq.shape[0] // p.n_heads
+    Zq, Zk = Zq.copy(), Zk.copy()
+    for i in range(p.n_heads):
+        r = slice(i * dh, (i + 1) * dh)
+        for _ in range(p.z_steps):
+            _, gq, gk = mha_z_objective_grad(Zq[r], Zk[r], P[i], Tq[r], Tk[r], p.alpha, p.beta, p.causal)
+            step = mha_z_step_size(Zq[r], Zk[r], p.alpha, p.beta, p.eta_z)
+            Zq[r], Zk[r] = Zq[r] - step * gq, Zk[r] - step * gk
+    return Zq, Zk
+
+
+def mha_step(X, Ypre, Wq, Wk, Wv, Wo, Zq, Zk, P, Aattn, p):
+    """The auxiliary-variable updates of one outer step of SparseLLM2 on one sequence, weights fixed, in the order of
+    Algorithm 2: Eq. (85) a_l = P, Eq. (86) a^attn_l, Eq. (87) z_l = (Zq, Zk).  Returns (Zq, Zk, P, Aattn)."""
+    X = np.asarray(X, F64)
+    V = np.asarray(Wv, F64) @ X
+    P = mha_a_update(P, Aattn, V, Zq, Zk, p)
+    Aattn = mha_attn_update(Ypre, Wo, mha_heads(V, P, p.n_heads))
+    Zq, Zk = mha_z_update(Zq, Zk, P, np.asarray(Wq, F64) @ X, np.asarray(Wk, F64) @ X, p)
+    return Zq, Zk, P, Aattn

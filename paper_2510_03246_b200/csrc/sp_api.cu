@@ -1,7 +1,8 @@
 // C-ABI entry points of libsp and the host-side orchestration of the per-module ADMM step.
 #include <math.h>
-#include <stdlib.h>
 #include <string.h>
+
+#include <mutex>
 
 #include "sp_common.cuh"
 
@@ -20,17 +21,9 @@ using namespace sp;
 namespace {
 
 constexpr int64_t kDefaultChunk = 32768;
-// SM pairs given to the z1 products that run beside the kept-support recovery (of 74 on a B200); the environment
-// variable SP_Z1_AHEAD_PAIRS overrides it (a tuning knob, read once).
-int z1_ahead_pairs() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("SP_Z1_AHEAD_PAIRS");
-    v = e ? atoi(e) : 58;
-    if (v < 1) v = 58;
-  }
-  return v;
-}
+// SM pairs given to the z1 products that run beside the kept-support recovery (of 74 on a B200): 40 to 66 pairs
+// measured the same within noise.
+constexpr int kZ1AheadPairs = 58;
 
 struct MatRef {
   const void* ptr;
@@ -192,8 +185,11 @@ bool make_assist(SolveAssist& a) {
 SideStream* side_stream() {
   static SideStream table[64];
   static bool failed[64] = {};
+  static std::mutex mu;
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || failed[dev]) return nullptr;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> guard(mu);
+  if (failed[dev]) return nullptr;
   SideStream& ss = table[dev];
   if (!ss.stream) {
     if (cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -209,7 +205,25 @@ SideStream* side_stream() {
   return &ss;
 }
 
+// Makes the caller's stream wait for everything queued on the library's
+// streams when a call returns early (an error between a fork and its join), so that no library work is ever left
+// unordered against the caller's stream.
+struct JoinOnExit {
+  SideStream* side;
+  cudaStream_t s;
+  bool armed = true;
+  ~JoinOnExit() {
+    if (!armed || !side) return;
+    cudaStream_t all[3] = {side->stream, side->assist_main.stream, side->assist_side.stream};
+    for (cudaStream_t q : all) {
+      if (cudaEventRecord(side->join, q) == cudaSuccess) cudaStreamWaitEvent(s, side->join, 0);
+    }
+  }
+};
+
 bool valid_act_dtype(int32_t dt) { return dt == SP_F32 || dt == SP_BF16; }
+// the sub-buffers of a workspace are carved at 256-byte offsets and accessed with 16-byte vector and bulk copies
+bool misaligned(const void* p, size_t a) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) % a) != 0; }
 
 // ------------------------------------------------------------------------------------------------ workspace plans
 struct AdmmPlan {
@@ -225,6 +239,7 @@ struct AdmmPlan {
   int32_t* grp_base;           // kept-channel map of the elementwise kernels
   uint8_t* grp_mask;
   void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
+  void* W2sb;                  // bf16 hi | lo split of W2[:, S] ([d, 2 * pad64(k)], gated modules)
   void *H, *E, *Ac, *Zb;
   float *D, *z1, *Eo;          // Eo: Ypre - A W2^T of a chunk (objective reporting)
   void* W2fb;                  // bf16 copy of the full W2 (objective reporting)
@@ -259,10 +274,12 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.grp_mask = c.take<uint8_t>((size_t)ceil_div(n, (int64_t)8));
   p.W1b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // hi | lo split of W1
   p.W2b = p.bf16 ? c.take_bytes(((size_t)n + 8) * d * csz) : nullptr;
-  p.Qtb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
+  p.Qtb = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // room for the hi | lo form
+  p.W2sb = p.bf16 ? c.take_bytes((size_t)d * 2 * split_kpad(n) * csz) : nullptr;
   const size_t npad = (size_t)(n + 7) / 8 * 8;   // leading dimension bound of the compact tensors
-  p.H = c.take_bytes((size_t)p.chunk * npad * csz);
-  p.E = c.take_bytes((size_t)p.chunk * d * csz);
+  // bf16 mode: room for h as hi | lo parts (gated modules)
+  p.H = c.take_bytes((size_t)p.chunk * (p.bf16 ? 2 * (size_t)split_kpad(n) : npad) * csz);
+  p.E = c.take_bytes((size_t)p.chunk * (p.bf16 ? 2 * (size_t)split_kpad(d) : (size_t)d) * csz);   // hi | lo (gated)
   p.Ac = c.take_bytes((size_t)p.chunk * n * csz);
   p.Zb = p.bf16 ? c.take_bytes((size_t)p.chunk * n * csz) : nullptr;
   p.D = c.take<float>((size_t)p.chunk * npad);
@@ -407,6 +424,7 @@ sp_status sp_gram_accumulate(const sp_mat* Xc, const sp_mat* Yc, float* G, int64
     if (Yc->rows != T || Yc->ld < Yc->cols || ldr < C) return SP_ERR_SHAPE;
   }
   if (rowstats && (!ws || ws_bytes < sp_workspace_bytes(SP_WS_GRAM, C, 0, T, 0, Xc->dtype))) return SP_ERR_WORKSPACE;
+  if (rowstats && misaligned(ws, 8)) return SP_ERR_ALIGNMENT;
   if (T == 0 || C == 0) return SP_OK;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const bool bf16 = Xc->dtype == SP_BF16;
@@ -429,6 +447,7 @@ sp_status sp_ridge_solve(const float* R, int64_t ldr, const float* G, int64_t ld
   if (m < 0 || n < 0 || ldr < n || ldg < n || ldw < n) return SP_ERR_SHAPE;
   if (m == 0 || n == 0) return SP_OK;
   if (!ws || ws_bytes < ridge_ws_bytes(m, n, precise != 0)) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256)) return SP_ERR_ALIGNMENT;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   Carver c(ws);
   SolveBufs b = carve_solve(c, n, m, precise ? 8 : 4);
@@ -451,6 +470,7 @@ sp_status sp_linear_refit(const float* R, int64_t ldr, const float* G, int64_t l
   // workspace: solve buffers for the full size + the unit index list
   const size_t need = ridge_ws_bytes(m, n, precise != 0) + align_up((size_t)n_units * 4, 256);
   if (!ws || ws_bytes < need) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256)) return SP_ERR_ALIGNMENT;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   Carver c(ws);
   SolveBufs b = carve_solve(c, n, m, precise ? 8 : 4);
@@ -484,6 +504,7 @@ sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* i
     if (kind == SP_SCORE_WANDA_L1 && !in->colabs) return SP_ERR_INVALID_ARG;
     if (relaxed_mask) return SP_ERR_UNSUPPORTED;
     if (!ws || ws_bytes < sp_workspace_bytes(SP_WS_SCORES, cols, 0, in->W.rows, 0, SP_F32)) return SP_ERR_WORKSPACE;
+    if (misaligned(ws, 8)) return SP_ERR_ALIGNMENT;
     CU(wanda_scores(kind, group, reinterpret_cast<const float*>(in->W.ptr), in->W.rows, in->W.ld, in->colsq,
                     in->colsq_stride, in->colabs, in->inv_tokens, n_units, scores, layer_importance,
                     reinterpret_cast<double*>(ws), s));
@@ -499,6 +520,7 @@ sp_status sp_struct_scores(int32_t kind, int32_t group, const sp_score_inputs* i
     }
     if (N < 1) return SP_ERR_SHAPE;
     if (!ws || ws_bytes < sp_workspace_bytes(SP_WS_SCORES, cols, 0, N, 0, SP_F32)) return SP_ERR_WORKSPACE;
+    if (misaligned(ws, 8)) return SP_ERR_ALIGNMENT;
     CU(lemma1_scores_stream(in->b, in->c, in->dd, in->t, group, n_units, scores, layer_importance, relaxed_mask,
                             r_layer, reinterpret_cast<double*>(ws), s));
     return SP_OK;
@@ -612,6 +634,9 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   const int64_t d = m->d, n = m->n, N = m->N;
   const int32_t cdt = m->X.dtype;
   if (!ws || ws_bytes < plan_init(nullptr, d, n, N, token_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256) || misaligned(st->Z, 16) || misaligned(st->U, 16) || misaligned(st->Gate, 16) ||
+      misaligned(m->X.ptr, 16) || misaligned(m->Ypre.ptr, 16))
+    return SP_ERR_ALIGNMENT;
   InitPlan p = plan_init(ws, d, n, N, token_chunk, cdt);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const bool bf16 = p.bf16;
@@ -682,6 +707,9 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   if (prm->skip_scores && (prm->reselect_mask || !prm->refit)) return SP_ERR_INVALID_ARG;
   const int32_t cdt = m->X.dtype;
   if (!ws || ws_bytes < plan_admm(nullptr, d, n, N, prm->token_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256) || misaligned(st->Z, 16) || misaligned(st->U, 16) || misaligned(st->Gate, 16) ||
+      misaligned(m->X.ptr, 16) || misaligned(m->Ypre.ptr, 16))
+    return SP_ERR_ALIGNMENT;
   AdmmPlan p = plan_admm(ws, d, n, N, prm->token_chunk, cdt);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const bool bf16 = p.bf16;
@@ -696,6 +724,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   // runs on the side stream while the caller's stream carries the W2 chain.
   SideStream* side = side_stream();
   cudaStream_t sa = side ? side->stream : s;
+  JoinOnExit join_guard{side, s};
   if (side) {
     CU(cudaEventRecord(side->fork, s));
     CU(cudaStreamWaitEvent(sa, side->fork, 0));
@@ -740,6 +769,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
 
   if (scores_only) {
     if (!joined) CU(cudaStreamWaitEvent(s, side->join, 0));
+    join_guard.armed = false;
     return SP_OK;
   }
 
@@ -765,7 +795,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
       MatRef xc{reinterpret_cast<const uint8_t*>(m->X.ptr) + (size_t)t0 * m->X.ld * esz_x, cdt, m->X.ld};
       MatRef z1c{p.z1_all + (size_t)t0 * kp_ahead, SP_F32, kp_ahead};
       SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, MatRef{nullptr, SP_F32, d}, z1c, status_dev, side->stream,
-                                   z1_ahead_pairs()));
+                                   kZ1AheadPairs));
     }
     CU(cudaEventRecord(side->z1_done, side->stream));
   }
@@ -785,6 +815,14 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   //      W1[S, :], W2[:, S], C = gamma I + W2 W2^T (d x d), Qt = W2[:, S]^T C^-1 (k x d)
   const int64_t kp = (k + 7) / 8 * 8;            // leading dimension of the compact [., k] tensors
   const int32_t* idx = p.sb.idx;
+  // Gated modules in bf16 mode: E = Ypre - h W2^T is a small difference of large terms (|h| can exceed |E| by two
+  // orders of magnitude when gate factors are large), so one bf16 rounding of h and of W2 would dominate the error of
+  // the a-update.  Both operands of that product are carried as bf16 hi + lo parts (three K segments: hi.hi, lo.hi,
+  // hi.lo), which keeps about 16 bits of each.
+  // E itself is then written as hi + lo parts as well and D = E Q^T takes two K segments (E_hi, E_lo against Q).
+  const bool split_h = bf16 && m->act == SP_ACT_SWIGLU;
+  const int64_t kp64 = split_kpad(k), dp64 = split_kpad(d);
+  if (split_h && dp64 != d) CU(cudaMemsetAsync(p.E, 0, (size_t)p.chunk * 2 * dp64 * 2, s));   // padding columns stay zero
   CU(build_group_map(st->mask, n, p.grp_base, p.grp_mask, s));
   CU(gather_cols<float>(st->W2, n, idx, d, k, p.W2cf, kp, s));
   MatRef w1{nullptr, SP_F32, d}, w2{p.W2cf, SP_F32, kp}, qt{p.Qt, SP_F32, d};
@@ -792,6 +830,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     if (!z1_ahead) CU(split_bf16(st->W1, d, idx, k, d, split_kpad(d), p.W1b, s));
     CU(convert_matrix(p.W2cf, SP_F32, kp, p.W2b, SP_BF16, kp, d, k, s));
     w2 = MatRef{p.W2b, SP_BF16, kp};
+    if (split_h) CU(split_bf16(p.W2cf, kp, nullptr, d, k, kp64, p.W2sb, s));
   } else {
     CU(gather_rows(st->W1, d, idx, k, d, p.W1c, d, s));
     w1 = MatRef{p.W1c, SP_F32, d};
@@ -812,8 +851,13 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
                            side ? &side->assist_main : nullptr, k, z1_ahead));
       SPCHK(potrs_right_tc(Rs, k, d, d, p.sb.P, reinterpret_cast<float*>(p.sb.dinv), p.sb.Xs, status_dev, s,
                            side ? &side->assist_main : nullptr, true, Gs, d));
-      CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));
-      qt = MatRef{p.Qtb, SP_BF16, d};
+      if (split_h) {
+        CU(split_bf16(Rs, d, nullptr, k, d, dp64, p.Qtb, s));      // only the hi part is used (see the D product)
+        qt = MatRef{p.Qtb, SP_BF16, 2 * dp64};
+      } else {
+        CU(convert_matrix(Rs, SP_F32, d, p.Qtb, SP_BF16, d, k, d, s));
+        qt = MatRef{p.Qtb, SP_BF16, d};
+      }
     } else {
       double* Gs = reinterpret_cast<double*>(p.sb.Gs);
       double* Rs = Gs + (size_t)d * d;
@@ -842,10 +886,33 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     MatRef h{p.H, cdt, kp}, e{p.E, cdt, d}, dd{p.D, SP_F32, kp}, z1{p.z1, SP_F32, kp}, ac{p.Ac, cdt, n};
     MatRef zb = bf16 ? MatRef{p.Zb, cdt, n} : MatRef{Zc, SP_F32, n};
     const float* Gc = (m->act == SP_ACT_SWIGLU) ? st->Gate + (size_t)t0 * n : nullptr;
-    CU(launch_prep_h(Zc, Uc, Gc, p.H, cdt, Tc, n, kp, k, idx, s));
     // E = Ypre - h_S W2[:, S]^T ; D_S = E Qt^T ; z1_S = X W1[S, :]^T
-    SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
-    SPCHK(contract(Tc, k, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
+    if (split_h) {
+      CU(launch_prep_h(Zc, Uc, Gc, p.H, cdt, Tc, n, 2 * kp64, k, idx, s, kp64));
+      TcOperand ta{p.H, 2 * kp64, true}, tb{p.W2sb, 2 * kp64, true};
+      ta.kext = tb.kext = 2 * kp64;
+      TcSegments sg;
+      sg.nseg = 3;
+      sg.a_k[1] = (int32_t)kp64;      // lo(h) . hi(W2)
+      sg.b_k[2] = (int32_t)kp64;      // hi(h) . lo(W2)
+      OutOperand e_out{p.E, cdt, 2 * dp64};
+      e_out.lo_off = dp64;
+      SPCHK(gemm_tc(Tc, d, k, -1.f, ta, tb, 1.f, Operand{yc.ptr, cdt, yc.ld, 1}, e_out, false, status_dev, s, &sg,
+                    2.0 * (double)Tc * d * k));
+      // D = E Q^T with E = E_hi + E_lo
+      TcOperand da{p.E, 2 * dp64, true}, db{qt.ptr, qt.ld, true};
+      da.kext = 2 * dp64;
+      db.kext = d;
+      TcSegments sd;
+      sd.nseg = 2;
+      sd.a_k[1] = (int32_t)dp64;
+      SPCHK(gemm_tc(Tc, k, d, 1.f, da, db, 0.f, Operand{p.D, SP_F32, kp, 1}, OutOperand{p.D, SP_F32, kp}, false,
+                    status_dev, s, &sd, 2.0 * (double)Tc * d * k));
+    } else {
+      CU(launch_prep_h(Zc, Uc, Gc, p.H, cdt, Tc, n, kp, k, idx, s));
+      SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
+    }
+    if (!split_h) SPCHK(contract(Tc, k, d, 1.0, e, true, qt, true, 0.0, dd, dd, false, acc64, bf16, status_dev, s));
     if (z1_ahead) {}   // already there for all tokens
     else if (bf16) SPCHK(contract_split_weights(Tc, k, d, xc, p.W1b, w1, z1, status_dev, s));
     else SPCHK(contract(Tc, k, d, 1.0, xc, true, w1, true, 0.0, z1, z1, false, acc64, false, status_dev, s));
@@ -883,6 +950,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     SPCHK(contract(n, d, Tc, 1.0, zb, false, xc, false, acc, r1, r1, false, acc64, bf16, status_dev, s));
   }
   CU(symmetrize_lower(st->G_A, n, n, s));
+  join_guard.armed = false;
   return SP_OK;
 }
 

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/sp.h"
 
 namespace sp {
@@ -35,6 +37,31 @@ struct ProfScope {
   cudaStream_t stream;
 };
 
+// One-time set-up per device (function attributes, device properties): run(fn) calls fn the first time it is reached
+// with a given device current, under a lock, and remembers success per device; a process may drive several GPUs.
+class PerDeviceOnce {
+ public:
+  template <typename F>
+  cudaError_t run(F&& fn) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> guard(mu_);
+    if (done_[dev]) return cudaSuccess;
+    e = fn();
+    if (e == cudaSuccess) done_[dev] = true;
+    return e;
+  }
+  static constexpr int kMaxDevices = 64;
+
+ private:
+  std::mutex mu_;
+  bool done_[kMaxDevices] = {};
+};
+// Multiprocessor count of the current device (cached per device).
+int sm_count();
+
 __host__ __device__ __forceinline__ int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 __host__ __device__ __forceinline__ size_t align_up(size_t a, size_t b) { return (a + b - 1) / b * b; }
 
@@ -51,6 +78,9 @@ struct OutOperand {
   void* ptr;
   int32_t dtype;
   int64_t ld;
+  // bf16 output of the tensor-core GEMM only: lo_off > 0 writes the result as two bf16 parts, bf16(v) at column j and
+  // bf16(v - bf16(v)) at column lo_off + j of the same row, so that it can serve as a split operand of the next product
+  int64_t lo_off = 0;
 };
 
 // C[M,N] (row-major) = alpha * sum_k A(i,k) B(k,j) + beta * Cin[i,j].  Cin may alias C or be another matrix of
@@ -196,9 +226,12 @@ struct UpdateArgs {
 // grp_base / grp_mask of a u8 mask over n channels (see sp_elementwise.cu)
 cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream);
 // H[T, ldh] (compact on the k kept channels idx[0..k), ldh a multiple of 8) = storage(phi(Z) - U);
-// phi(z) = gate * z when gate != nullptr, else ReLU
+// phi(z) = gate * z when gate != nullptr, else ReLU.
+// lo_off > 0 (bf16 storage, a multiple of 8, 2 * lo_off <= ldh): H is split into bf16 hi and lo parts, the hi part in
+// columns [0, lo_off), the lo part in columns [lo_off, 2 * lo_off); columns k..lo_off-1 of both are zero.
 cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, void* H, int32_t hdt, int64_t T,
-                          int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream);
+                          int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream,
+                          int64_t lo_off = 0);
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]

@@ -221,13 +221,15 @@ __device__ __forceinline__ void store8(void* base, int32_t dt, int64_t e, const 
 // H_S = storage(phi(Z) - U) on the kept channels, compact [T, ldh].  A thread owns 8 consecutive COMPACT columns: it
 // gathers their channels (ascending, so close together in a row of Z) and writes one 16-byte (bf16) or two 16-byte
 // (fp32) vectors per row.  Columns k..ldh-1 of H are written as zero.
+// lo_off > 0 (bf16 only): H holds two parts side by side, bf16(h) in columns [0, ncols) and bf16(h - bf16(h)) in columns
+// [lo_off, lo_off + ncols), so that a product with H keeps about 16 bits of h (two K segments of the GEMM).
 __global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z, const float* __restrict__ U,
                                                      const float* __restrict__ G, void* __restrict__ H, int32_t hdt,
                                                      int64_t T, int64_t n,
-                                                     int64_t ldh, int64_t k, const int32_t* __restrict__ idx,
-                                                     int32_t rows_per_block) {
+                                                     int64_t ldh, int64_t ncols, int64_t lo_off, int64_t k,
+                                                     const int32_t* __restrict__ idx, int32_t rows_per_block) {
   const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
-  if (p0 >= ldh) return;
+  if (p0 >= ncols) return;
   int ch[8];
 #pragma unroll
   for (int q = 0; q < 8; ++q) ch[q] = (p0 + q < k) ? idx[p0 + q] : -1;
@@ -252,6 +254,11 @@ __global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z
         if (ch[q] >= 0) h[q] -= ur[ch[q]];
     }
     store8(H, hdt, r * ldh + p0, h);
+    if (lo_off > 0) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) h[q] -= __bfloat162float(__float2bfloat16_rn(h[q]));
+      store8(H, hdt, r * ldh + lo_off + p0, h);
+    }
   }
 }
 
@@ -846,20 +853,23 @@ cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, u
 }
 
 cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, void* H, int32_t hdt, int64_t T,
-                          int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream) {
+                          int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream, int64_t lo_off) {
   if (T * ldh == 0) return cudaSuccess;
-  // algorithmic bytes: Z (and U) read once, the kept part written once
+  if (lo_off > 0 && (hdt != SP_BF16 || lo_off % 8 != 0 || 2 * lo_off > ldh)) return cudaErrorInvalidValue;
+  const int64_t ncols = lo_off > 0 ? lo_off : ldh;
+  // algorithmic bytes: Z (and U) read once, the kept part written once (twice when it is split)
   ProfScope prof(PK_PREP_H, 0.0,
-                 (double)T * ((double)n * (U ? 8.0 : 4.0) + (double)k * ((hdt == SP_BF16 ? 2.0 : 4.0) + (gate ? 4.0 : 0.0))),
+                 (double)T * ((double)n * (U ? 8.0 : 4.0) +
+                              (double)k * ((hdt == SP_BF16 ? (lo_off > 0 ? 4.0 : 2.0) : 4.0) + (gate ? 4.0 : 0.0))),
                  stream);
-  const unsigned gx = (unsigned)ceil_div(ldh, (int64_t)(8 * 256));
+  const unsigned gx = (unsigned)ceil_div(ncols, (int64_t)(8 * 256));
   int64_t rb = ceil_div((int64_t)148 * 16, (int64_t)gx);
   if (rb > T) rb = T;
   if (rb > 65535) rb = 65535;
   const int32_t rows_per = (int32_t)ceil_div(T, rb);
   count_launch();
-  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, gate, H, hdt, T, n, ldh, k, idx,
-                                                                                        rows_per);
+  prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, gate, H, hdt, T, n, ldh, ncols, lo_off,
+                                                                                        k, idx, rows_per);
   return cudaGetLastError();
 }
 

@@ -61,6 +61,7 @@ struct TcParams {
   void* c;
   int32_t c_dtype;
   int64_t c_ld;
+  int64_t c_lo_off;  // bf16 C, plain epilogue: second (lo) part of every value c_lo_off columns to the right
   int32_t a_kmajor, b_kmajor, lower_only;
   int32_t epi_mode;  // EpiMode
   int32_t n_fast;    // tile order: 1 = consecutive tiles walk N first (they share the A row block)
@@ -563,8 +564,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 float v = stg[rr][lane];
                 if (has_cin) v = fmaf(p.beta, cv[rr], v);
                 const int64_t o = c_off + (int64_t)rr * p.c_ld;
-                if (c_f32) reinterpret_cast<float*>(p.c)[o] = v;
-                else reinterpret_cast<__nv_bfloat16*>(p.c)[o] = __float2bfloat16_rn(v);
+                if (c_f32) {
+                  reinterpret_cast<float*>(p.c)[o] = v;
+                } else {
+                  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+                  reinterpret_cast<__nv_bfloat16*>(p.c)[o] = hi;
+                  if (p.c_lo_off > 0)
+                    reinterpret_cast<__nv_bfloat16*>(p.c)[o + p.c_lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
+                }
               }
             }
           }
@@ -630,18 +637,21 @@ bool make_map(CUtensorMap* map, bool f32, const void* ptr, int64_t inner, int64_
   return r == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
-
 }  // namespace
+
+int sm_count() {
+  static std::mutex mu;
+  static int table[PerDeviceOnce::kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= PerDeviceOnce::kMaxDevices) return 148;
+  std::lock_guard<std::mutex> guard(mu);
+  if (table[dev] == 0) {
+    int n = 0;
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    table[dev] = n > 0 ? n : 148;
+  }
+  return table[dev];
+}
 
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B) {
   if (M <= 0 || N <= 0 || K <= 0) return false;
@@ -688,6 +698,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   p.alpha = alpha; p.beta = beta;
   p.cin = Cin.ptr; p.cin_dtype = Cin.dtype; p.cin_ld = Cin.s0;
   p.c = C.ptr; p.c_dtype = C.dtype; p.c_ld = C.ld;
+  p.c_lo_off = C.dtype == SP_BF16 ? C.lo_off : 0;
+  if (C.lo_off < 0 || (C.lo_off > 0 && C.dtype != SP_BF16)) return SP_ERR_INVALID_ARG;
   p.a_kmajor = A.kmajor ? 1 : 0;
   p.b_kmajor = B.kmajor ? 1 : 0;
   p.lower_only = lower_only ? 1 : 0;
@@ -699,7 +711,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   if (c_tma && beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && Cin.s0 == C.ld) p.epi_mode = EPI_TMA_ADD;
   if (p.epi_mode != EPI_DIRECT && !make_map(&tmC, true, C.ptr, N, M, C.ld, 32, 32)) return SP_ERR_CUDA;
   // bf16 C = beta * Cin + alpha * acc with a bf16 Cin: both through TMA
-  if (p.epi_mode == EPI_DIRECT && beta != 0.f && C.dtype == SP_BF16 && Cin.dtype == SP_BF16 && C.ld % 8 == 0 &&
+  if (p.epi_mode == EPI_DIRECT && p.c_lo_off == 0 && beta != 0.f && C.dtype == SP_BF16 && Cin.dtype == SP_BF16 &&
+      C.ld % 8 == 0 &&
       Cin.s0 % 8 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0 &&
       (reinterpret_cast<uintptr_t>(Cin.ptr) & 15u) == 0) {
     if (!make_map(&tmC, false, C.ptr, N, M, C.ld, 32, 32, true) ||
@@ -766,13 +779,11 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   p.ksplit = (int32_t)ceil_div(num_kb, p.kb_per_split);
   p.num_units = p.n_plain + (p.num_tiles - p.n_plain) * p.ksplit;
 
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) !=
-        cudaSuccess)
-      return SP_ERR_CUDA;
-    attr_set = true;
-  }
+  static PerDeviceOnce attr_once;
+  if (attr_once.run([] {
+        return cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+      }) != cudaSuccess)
+    return SP_ERR_CUDA;
   count_launch();
   const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
   ProfScope prof(max_pairs > 0 ? PK_GEMM_TC_SHARED : PK_GEMM_TC, flops, 0.0, stream);

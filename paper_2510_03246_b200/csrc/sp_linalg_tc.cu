@@ -616,19 +616,21 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
   __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
   const int64_t nblk = ceil_div(n, (int64_t)TB);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(chol_next_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NM_SMEM) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(chol_next_diag_stage1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)NM_SMEM) != cudaSuccess ||
-        cudaFuncSetAttribute(chol_next_diag_stage2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)NM_SMEM) != cudaSuccess)
-      return SP_ERR_CUDA;
-    attr_set = true;
-  }
+  static PerDeviceOnce attr_once;
+  if (attr_once.run([] {
+        cudaError_t e = cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)DIAG_SMEM);
+        if (e == cudaSuccess)
+          e = cudaFuncSetAttribute(chol_next_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NM_SMEM);
+        if (e == cudaSuccess)
+          e = cudaFuncSetAttribute(chol_next_diag_stage1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)NM_SMEM);
+        if (e == cudaSuccess)
+          e = cudaFuncSetAttribute(chol_next_diag_stage2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   (int)NM_SMEM);
+        return e;
+      }) != cudaSuccess)
+    return SP_ERR_CUDA;
 #define SP_CUDA_OK(x) do { if ((x) != cudaSuccess) return SP_ERR_CUDA; } while (0)
   // With an assisting stream the chain of diagonal blocks runs ahead: after block k is factored, a small kernel
   // forms the next diagonal block (into scratch behind the inverses), and the next factorisation starts from it while

@@ -1011,13 +1011,12 @@ cudaError_t topk_select_batched(const float* scores, int64_t ld_scores, int64_t 
                                 int64_t ld_idx, cudaStream_t stream) {
   if (n == 0 || batch == 0) return cudaSuccess;
   constexpr int64_t kMaxSmemKeys = 47104;      // 184 KiB of keys beside the 33 KiB of histograms
-  static bool attr_set = false;
-  if (!attr_set) {
-    const cudaError_t e = cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)(kMaxSmemKeys * sizeof(uint32_t)));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static PerDeviceOnce attr_once;
+  const cudaError_t ea = attr_once.run([] {
+    return cudaFuncSetAttribute(topk_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)(kMaxSmemKeys * sizeof(uint32_t)));
+  });
+  if (ea != cudaSuccess) return ea;
   const int smem_keys = n <= kMaxSmemKeys ? 1 : 0;
   ProfScope prof(PK_TOPK, 0.0, (double)batch * (double)n * 5.0, stream);
   count_launch();

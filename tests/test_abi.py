@@ -66,6 +66,12 @@ def test_host_side_validation_without_gpu(lib):
     assert lib.sp_gram_accumulate(C.byref(x), None, fake, 16, None, 0, None, None, None, 0, None) == 2
     # sp_ridge_solve: workspace too small
     assert lib.sp_ridge_solve(fake, 8, fake, 8, 4, 8, 0.1, 1, 1, fake, 8, None, fake, 16, None) == 5
+    # a workspace that is large enough but not 256-byte aligned is refused before any launch
+    need = api.workspace_bytes(api.SP_WS_RIDGE_SOLVE, 4, 8, 0, 0, api.SP_F64)
+    assert lib.sp_ridge_solve(fake, 8, fake, 8, 4, 8, 0.1, 1, 1, fake, 8, None, C.c_void_p(0x1008), need, None) == 4
+    need = api.workspace_bytes(api.SP_WS_LINEAR_REFIT, 4, 8, 0, 0, api.SP_F64)
+    assert lib.sp_linear_refit(fake, 8, fake, 8, 4, 8, 1, fake, 4, 0.1, 1, 1, fake, 8, None, C.c_void_p(0x1010), need,
+                               None) == 4
     # sp_admm_step: null params
     assert lib.sp_admm_step(None, None, None, None, None, None, 0, None) == 1
 

@@ -143,15 +143,7 @@ def test_mask_and_token_update(run):
     got = run["Z1_rows"].T
     if run["gated"]:
         Znew = O.swiglu_zu_update(A, g, z1, p.alpha, p.beta)
-        # Only the correction term D = a - g z of the a-update goes through bf16 operands; its error (tolerance x
-        # max|D|) reaches z through dz/da = beta g / (beta g^2 + alpha) <= 1/2.  With gate factors far above one |z| is
-        # much smaller than |a| and |D|, so the bound is stated on that scale, plus the usual one on the scale of z.
-        D = A - phi0
-        dzda = p.beta * np.abs(g) / (p.beta * g * g + p.alpha)
-        bound = TOLB * (np.abs(D).max() * dzda + np.abs(Znew).max())
-        err = np.abs(got - Znew)
-        assert np.all(err <= bound), float((err / bound).max())
-        assert relerr(got, Znew) < 2 * TOLB                  # and it stays within twice the plain tolerance
+        assert relerr(got, Znew) < TOLB
     else:
         Znew = O.z_select(z0, z1, z2, A, p.alpha, p.beta, p.z_rule)
         assert relerr(got, Znew) < TOLB
