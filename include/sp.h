@@ -292,6 +292,68 @@ sp_status sp_distribute_importance(const double* head_stats, int32_t n_heads, co
                                    int32_t L, double rho, double gamma, double* I_attn, double* I_mlp, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
+ * sp_mha_init, sp_mha_step — auxiliary-variable updates of one attention module under the paper's second objective
+ * (Appendix A, "Computation on Multi-Head Attention layers", Method 2; Algorithm 2, SparseLLM2), weights held fixed.
+ *
+ * Module (paper, per sequence of T tokens and per head i of width d_h = d / n_heads, tokens as columns):
+ *   Q = W_Q X, K = W_K X, V = W_V X;  S_i = Q_i^T K_i / sqrt(d_h);  P_i = softmax over the keys of each row of S_i;
+ *   head_i = V_i P_i^T;  a_attn = Concat_i head_i;  z_{l+1}^pre = W_O a_attn.
+ * Storage is token-major: X, Ypre, Zq, Zk, Aattn are [n_seq * T, d]; head i owns columns [i d_h, (i+1) d_h);
+ * P is [n_seq, n_heads, T, T] (row = query, column = key), fp32.
+ * Reading of Method 2 (the section prints inconsistent shapes): the auxiliary output z_l is the pair (Zq, Zk) with
+ * Zq ~ W_Q X and Zk ~ W_K X ("separate constraints for each projection"), a_l is P, a_attn_l the concatenated heads:
+ *   alpha |Ypre - W_O Aattn|^2 + alpha |Aattn - Concat_i V_i P_i^T|^2 + beta |P - softmax(S(Zq, Zk))|^2
+ *   + alpha |Zq - W_Q X|^2 + alpha |Zk - W_K X|^2.
+ * sp_mha_init writes the forward definition: Zq, Zk, P, Aattn and Ypre = Aattn W_O^T (the pre-trained state).
+ * sp_mha_step, in the order of Algorithm 2:
+ *   Eq. (85)  a_steps gradient steps on every P_i of alpha |Aattn_i - V_i P_i^T|^2 + beta |P_i - softmax(S_i)|^2 with
+ *             the step 1 / (2 (alpha |V_i|_F^2 + beta));
+ *   Eq. (86)  Aattn = (W_O^T W_O + I)^-1 (W_O^T Ypre + Concat_i V_i P_i^T)   (closed-form minimiser);
+ *   Eq. (87)  z_steps joint gradient steps on (Zq_i, Zk_i) of beta |P_i - softmax(S_i)|^2 + alpha |Zq_i - (W_Q X)_i|^2
+ *             + alpha |Zk_i - (W_K X)_i|^2 through the softmax, with the step
+ *             eta_z / (2 alpha + beta (|Zq_i|_F^2 + |Zk_i|_F^2) / d_h) recomputed before every step.
+ * The elementwise "if z < 0" select that Algorithm 2 repeats for this module belongs to the ReLU module; it is not
+ * applied.  causal != 0 masks keys after the query.  The weights (already masked by the caller: pruned heads have zero
+ * rows in W_Q, W_K, W_V and zero columns in W_O) are read only; their recovery from the updated variables uses
+ * sp_gram_accumulate / sp_ridge_solve / sp_linear_refit.
+ * bf16 mode (X bf16): all contractions are batched tensor-core products (one launch for all heads and sequences of a
+ * chunk), operands whose rounding matters carried as bf16 hi + lo parts; needs d_h % 8 == 0 and T % 8 == 0
+ * (SP_ERR_ALIGNMENT otherwise).  fp32 mode: fp32 operands, fp64 accumulation.
+ * seq_chunk sequences are processed at a time (0 = 1); workspace: sp_mha_workspace_bytes(d, n_heads, T, n_seq,
+ * seq_chunk, dtype of X).  Errors: SP_ERR_INVALID_ARG (null pointers, alpha / beta <= 0, eta_z outside (0, 1],
+ * negative counts), SP_ERR_SHAPE (sizes that do not match d, n_heads, T, n_seq; leading dimensions other than d),
+ * SP_ERR_DTYPE, SP_ERR_ALIGNMENT, SP_ERR_WORKSPACE.
+ */
+typedef struct {
+  sp_mat X;     /* [n_seq * T, d] module input, SP_BF16 or SP_F32 (selects the mode), ld = d                      */
+  sp_mat Ypre;  /* [n_seq * T, d] pre-trained module output, same dtype (sp_mha_init writes it), ld = d             */
+  sp_mat Wq, Wk, Wv, Wo;   /* [d, d] fp32, [out, in], ld = d                                                       */
+  int64_t d, n_heads, T, n_seq;
+} sp_mha_module;
+
+typedef struct {
+  float* Zq;     /* [n_seq * T, d]             auxiliary output of the query projection                            */
+  float* Zk;     /* [n_seq * T, d]             auxiliary output of the key projection                              */
+  float* P;      /* [n_seq, n_heads, T, T]     auxiliary attention probabilities a_l                               */
+  float* Aattn;  /* [n_seq * T, d]             auxiliary concatenated head outputs a_attn_l                        */
+} sp_mha_state;
+
+typedef struct {
+  double alpha, beta;
+  int32_t a_steps, z_steps;  /* gradient steps of Eq. (85) and Eq. (87)                                            */
+  double eta_z;              /* relative step of Eq. (87), in (0, 1]                                               */
+  int32_t causal;
+  int32_t reserved;
+  int64_t seq_chunk;
+} sp_mha_params;
+
+sp_status sp_mha_init(const sp_mha_module* m, sp_mha_state* st, int32_t causal, int64_t seq_chunk, int32_t* status_dev,
+                      void* ws, size_t ws_bytes, void* stream);
+sp_status sp_mha_step(const sp_mha_module* m, sp_mha_state* st, const sp_mha_params* p, int32_t* status_dev, void* ws,
+                      size_t ws_bytes, void* stream);
+size_t sp_mha_workspace_bytes(int64_t d, int64_t n_heads, int64_t T, int64_t n_seq, int64_t seq_chunk, int32_t dtype);
+
+/* ---------------------------------------------------------------------------------------------------------------
  * Helpers.
  * sp_ridge_solve   — W[m,n] = R[m,n] (G[n,n] + rho_eff I)^-1 by Cholesky and two triangular solves (weight
  *                    recovery of Appendix A.1).  G, R, W fp32; factorisation in fp64 when precise != 0, else fp32.

@@ -29,7 +29,7 @@ EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_admm_scores"
            "sp_apply_mask", "sp_apply_mask_batched", "sp_weight_stats", "sp_distribute_importance",
            "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
-           "sp_profile_kind_name", "sp_launch_count"]
+           "sp_profile_kind_name", "sp_launch_count", "sp_mha_init", "sp_mha_step", "sp_mha_workspace_bytes"]
 
 
 class SpError(RuntimeError):
@@ -64,6 +64,20 @@ class SpAdmmParams(C.Structure):
 class SpScoreInputs(C.Structure):
     _fields_ = [("W", SpMat), ("colsq", C.c_void_p), ("colsq_stride", C.c_int64), ("colabs", C.c_void_p),
                 ("inv_tokens", C.c_double), ("b", SpMat), ("c", SpMat), ("dd", SpMat), ("t", SpMat)]
+
+
+class SpMhaModule(C.Structure):
+    _fields_ = [("X", SpMat), ("Ypre", SpMat), ("Wq", SpMat), ("Wk", SpMat), ("Wv", SpMat), ("Wo", SpMat),
+                ("d", C.c_int64), ("n_heads", C.c_int64), ("T", C.c_int64), ("n_seq", C.c_int64)]
+
+
+class SpMhaState(C.Structure):
+    _fields_ = [("Zq", C.c_void_p), ("Zk", C.c_void_p), ("P", C.c_void_p), ("Aattn", C.c_void_p)]
+
+
+class SpMhaParams(C.Structure):
+    _fields_ = [("alpha", C.c_double), ("beta", C.c_double), ("a_steps", C.c_int32), ("z_steps", C.c_int32),
+                ("eta_z", C.c_double), ("causal", C.c_int32), ("reserved", C.c_int32), ("seq_chunk", C.c_int64)]
 
 
 REPORT_FIELDS = ["res_act", "res_out", "res_in", "z_sq", "a_sq", "rho1_eff", "rho2_eff", "kept"]
@@ -104,6 +118,10 @@ def lib() -> C.CDLL:
         L.sp_linear_refit.argtypes = [vp, i64, vp, i64, i64, i64, i32, vp, i64, dbl, i32, i32, vp, i64, vp, vp, sz, vp]
         L.sp_gemm.argtypes = [i32, i32, i64, i64, i64, dbl, pm, pm, dbl, pm, i32, i32, vp, vp]
         L.sp_symmetrize.argtypes = [vp, i64, i64, vp]
+        L.sp_mha_workspace_bytes.restype = C.c_size_t
+        L.sp_mha_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, i32]
+        L.sp_mha_init.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), i32, i64, vp, vp, sz, vp]
+        L.sp_mha_step.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), C.POINTER(SpMhaParams), vp, vp, sz, vp]
         L.sp_profile_begin.argtypes = [i32]
         L.sp_profile_read.argtypes = [vp]
         L.sp_profile_kinds.restype = i32
@@ -111,7 +129,7 @@ def lib() -> C.CDLL:
         L.sp_profile_kind_name.argtypes = [i32]
         L.sp_launch_count.restype = i64
         for name in EXPORTS:
-            if name not in ("sp_workspace_bytes", "sp_admm_overlap_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
+            if name not in ("sp_workspace_bytes", "sp_admm_overlap_bytes", "sp_mha_workspace_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
                             "sp_profile_kind_name", "sp_launch_count"):
                 getattr(L, name).restype = C.c_int32
         _lib = L
@@ -498,3 +516,61 @@ class FfnModule:
         s = self.status.cpu().tolist()
         if s[0] != 0:
             raise SpError(s[0], f"device status (index {s[1]}, aux {s[2]})")
+
+
+@dataclass
+class MhaParams:
+    alpha: float = 1.0
+    beta: float = 1.0
+    a_steps: int = 4
+    z_steps: int = 4
+    eta_z: float = 1.0
+    causal: bool = True
+    seq_chunk: int = 0
+
+
+class MhaModule:
+    """Owns the device buffers of one attention module (Method 2 auxiliary variables) and forwards to sp_mha_init /
+    sp_mha_step.  X: [n_seq * T, d] token-major; Wq, Wk, Wv, Wo: [d, d] ([out, in]), kept in fp32 for the library."""
+
+    def __init__(self, X: torch.Tensor, Wq, Wk, Wv, Wo, n_heads: int, T: int, seq_chunk: int = 0):
+        _require_cuda(X, Wq, Wk, Wv, Wo)
+        self.X = X.contiguous()
+        self.dev = X.device
+        N, d = X.shape
+        assert N % T == 0 and d % n_heads == 0
+        self.d, self.n_heads, self.T, self.n_seq, self.seq_chunk = d, n_heads, T, N // T, seq_chunk
+        self.Wq, self.Wk, self.Wv, self.Wo = (w.float().contiguous() for w in (Wq, Wk, Wv, Wo))
+        self.Ypre = torch.empty_like(self.X)
+        f32 = dict(dtype=torch.float32, device=self.dev)
+        self.Zq, self.Zk, self.Aattn = (torch.empty(N, d, **f32) for _ in range(3))
+        self.P = torch.empty(self.n_seq, n_heads, T, T, **f32)
+        self.status = new_status(self.dev)
+        self._wsbuf = _ws(lib().sp_mha_workspace_bytes(d, n_heads, T, self.n_seq, seq_chunk, _dt(self.X)), self.dev)
+
+    def set_weights(self, Wq, Wk, Wv, Wo):
+        for dst, src in ((self.Wq, Wq), (self.Wk, Wk), (self.Wv, Wv), (self.Wo, Wo)):
+            dst.copy_(src)
+
+    def _module(self) -> SpMhaModule:
+        return SpMhaModule(mat(self.X), mat(self.Ypre), mat(self.Wq), mat(self.Wk), mat(self.Wv), mat(self.Wo), self.d,
+                           self.n_heads, self.T, self.n_seq)
+
+    def _state(self) -> SpMhaState:
+        return SpMhaState(self.Zq.data_ptr(), self.Zk.data_ptr(), self.P.data_ptr(), self.Aattn.data_ptr())
+
+    def sp_mha_init(self, causal: bool = True):
+        m, st = self._module(), self._state()
+        _check(lib().sp_mha_init(C.byref(m), C.byref(st), int(causal), self.seq_chunk, self.status.data_ptr(),
+                                 self._wsbuf.data_ptr(), self._wsbuf.numel(), _stream()), "sp_mha_init")
+
+    def sp_mha_step(self, p: MhaParams):
+        m, st = self._module(), self._state()
+        prm = SpMhaParams(p.alpha, p.beta, p.a_steps, p.z_steps, p.eta_z, int(p.causal), 0, self.seq_chunk)
+        _check(lib().sp_mha_step(C.byref(m), C.byref(st), C.byref(prm), self.status.data_ptr(), self._wsbuf.data_ptr(),
+                                 self._wsbuf.numel(), _stream()), "sp_mha_step")
+
+    def check_status(self):
+        code = int(self.status[0].item())
+        if code != SP_OK:
+            raise SpError(code, "device status")

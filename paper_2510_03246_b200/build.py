@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libsp.so")
 SOURCES = ["sp_api.cu", "sp_gemm_simt.cu", "sp_gemm_tc.cu", "sp_linalg.cu", "sp_linalg_tc.cu", "sp_elementwise.cu", "sp_mask.cu",
-           "sp_profile.cu"]
+           "sp_profile.cu", "sp_mha.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -965,3 +965,343 @@ sp_status sp_admm_scores(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------ attention module
+namespace {
+
+// A token-major tensor seen as one [T, d_h] slice per (head, sequence) pair, or a [pairs, T, T] tensor; `planes`
+// whole copies `plane` elements apart (bf16 hi / lo parts).
+struct BMat {
+  const void* ptr;
+  int32_t dt;
+  int64_t ld, s0, s1;   // leading dimension; element stride of the head (b0) and sequence (b1) index
+  int planes = 1;
+  int64_t plane = 0;
+};
+
+// C_b = alpha * sum over segments A_b[plane pa] B_b[plane pb] + beta * Cin_b for all nb0 x nb1 pairs.
+// bf16 operands: one batched tensor-core launch.  fp32 operands (fp32 mode): plane 0 holds the full value, the
+// segments collapse to one product per pair on the CUDA cores with fp64 accumulation.
+sp_status bcontract(int64_t M, int64_t N, int64_t K, double alpha, BMat A, bool a_kmajor, BMat B, bool b_kmajor,
+                    int nseg, const int* pa, const int* pb, double beta, BMat Cin, BMat C, int64_t c_lo_off, int nb0,
+                    int nb1, int32_t* status, cudaStream_t s) {
+  if (M <= 0 || N <= 0 || nb0 <= 0 || nb1 <= 0) return SP_OK;
+  if (A.dt == SP_BF16 && B.dt == SP_BF16) {
+    TcOperand ta{A.ptr, A.ld, a_kmajor}, tb{B.ptr, B.ld, b_kmajor};
+    TcSegments sg;
+    sg.nseg = nseg;
+    for (int i = 0; i < nseg; ++i) { sg.a_p[i] = pa[i]; sg.b_p[i] = pb[i]; }
+    TcBatch bt;
+    bt.nb0 = nb0; bt.nb1 = nb1;
+    bt.a_s0 = A.s0; bt.a_s1 = A.s1; bt.b_s0 = B.s0; bt.b_s1 = B.s1;
+    bt.c_s0 = C.s0; bt.c_s1 = C.s1; bt.cin_s0 = Cin.s0; bt.cin_s1 = Cin.s1;
+    bt.a_planes = A.planes; bt.a_plane = A.plane; bt.b_planes = B.planes; bt.b_plane = B.plane;
+    OutOperand out{const_cast<void*>(C.ptr), C.dt, C.ld};
+    out.lo_off = c_lo_off;
+    return gemm_tc(M, N, K, (float)alpha, ta, tb, (float)beta, Operand{Cin.ptr, Cin.dt, Cin.ld, 1}, out, false, status,
+                   s, &sg, 2.0 * (double)M * N * K * nb0 * nb1, 0, &bt);
+  }
+  for (int b1 = 0; b1 < nb1; ++b1)
+    for (int b0 = 0; b0 < nb0; ++b0) {
+      auto at = [&](const BMat& m) {
+        return reinterpret_cast<const uint8_t*>(m.ptr) + ((size_t)b0 * m.s0 + (size_t)b1 * m.s1) * dtype_size(m.dt);
+      };
+      Operand a{at(A), A.dt, a_kmajor ? A.ld : 1, a_kmajor ? 1 : A.ld};
+      Operand b{at(B), B.dt, b_kmajor ? 1 : B.ld, b_kmajor ? B.ld : 1};
+      Operand cin{Cin.ptr ? at(Cin) : nullptr, Cin.dt, Cin.ld, 1};
+      OutOperand out{const_cast<uint8_t*>(at(C)), C.dt, C.ld};
+      CU(gemm_simt(M, N, K, alpha, a, b, beta, cin, out, false, true, s));
+    }
+  return SP_OK;
+}
+
+struct MhaPlan {
+  int64_t d, H, T, dh, sc, cap;   // cap = tokens of a full chunk
+  bool bf16;
+  SolveBufs sb;
+  float *Cf, *RW, *MC;            // W_O^T W_O; [W_O; I] right-hand sides; [M1; Cinv] = [W_O; I] (W_O^T W_O + I)^-1
+  void *Wqs, *Wks, *Wvs, *Wos, *M1s, *Cis;   // bf16 hi | lo forms of the weights ([d, 2 pad64(d)])
+  float *Tq, *Tk, *Vf, *Gq, *Gk;  // [cap, d] fp32
+  void *Vs, *Zqs, *Zks;           // bf16 hi / lo planes [2][cap, d]
+  void *Rb, *Hd;                  // R = A_attn - P V ([cap, d]); head outputs as hi | lo ([cap, 2 pad64(d)])
+  float *S, *G;                   // [sc H, T, T] fp32
+  void* Pb;                       // [2][sc H, T, T] bf16: hi / lo planes of P; plane 0 later holds dS
+  double* sums;
+  float *eta_a, *eta_z;
+  size_t bytes;
+};
+
+MhaPlan plan_mha(void* ws, int64_t d, int64_t H, int64_t T, int64_t n_seq, int64_t seq_chunk, int32_t cdt) {
+  MhaPlan p;
+  p.d = d; p.H = H; p.T = T; p.dh = H > 0 ? d / H : d;
+  p.sc = seq_chunk > 0 ? seq_chunk : 1;
+  if (p.sc > n_seq) p.sc = n_seq;
+  if (p.sc < 1) p.sc = 1;
+  p.cap = p.sc * T;
+  p.bf16 = cdt == SP_BF16;
+  const size_t tsize = p.bf16 ? 4 : 8;
+  const size_t dp = (size_t)split_kpad(d);
+  Carver c(ws);
+  p.sb = carve_solve(c, d, 2 * d, tsize);
+  p.Cf = c.take<float>((size_t)d * d);
+  p.RW = c.take<float>((size_t)2 * d * d);
+  p.MC = c.take<float>((size_t)2 * d * d);
+  p.Wqs = p.Wks = p.Wvs = p.Wos = p.M1s = p.Cis = nullptr;
+  if (p.bf16) {
+    p.Wqs = c.take_bytes((size_t)d * 2 * dp * 2); p.Wks = c.take_bytes((size_t)d * 2 * dp * 2);
+    p.Wvs = c.take_bytes((size_t)d * 2 * dp * 2); p.Wos = c.take_bytes((size_t)d * 2 * dp * 2);
+    p.M1s = c.take_bytes((size_t)d * 2 * dp * 2); p.Cis = c.take_bytes((size_t)d * 2 * dp * 2);
+  }
+  const size_t tok = (size_t)p.cap * d, tt = (size_t)p.sc * H * T * T;
+  p.Tq = c.take<float>(tok); p.Tk = c.take<float>(tok); p.Vf = c.take<float>(tok);
+  p.Gq = c.take<float>(tok); p.Gk = c.take<float>(tok);
+  p.Vs = p.Zqs = p.Zks = p.Pb = nullptr;
+  if (p.bf16) {
+    p.Vs = c.take_bytes(2 * tok * 2); p.Zqs = c.take_bytes(2 * tok * 2); p.Zks = c.take_bytes(2 * tok * 2);
+    p.Pb = c.take_bytes(2 * tt * 2);      // hi / lo planes
+  }
+  p.Rb = c.take_bytes(tok * (p.bf16 ? 2 : 4));
+  p.Hd = c.take_bytes((size_t)p.cap * (p.bf16 ? 2 * dp * 2 : (size_t)d * 4));
+  p.S = c.take<float>(tt);
+  p.G = c.take<float>(tt);
+  p.sums = c.take<double>((size_t)p.sc * H);
+  p.eta_a = c.take<float>((size_t)p.sc * H);
+  p.eta_z = c.take<float>((size_t)p.sc * H);
+  p.bytes = align_up(c.off, 256);
+  return p;
+}
+
+sp_status check_mha(const sp_mha_module* m, const sp_mha_state* st) {
+  if (!m || !st) return SP_ERR_INVALID_ARG;
+  if (m->d < 1 || m->n_heads < 1 || m->T < 1 || m->n_seq < 1 || m->d % m->n_heads != 0) return SP_ERR_SHAPE;
+  const int64_t N = m->n_seq * m->T;
+  if (!m->X.ptr || !m->Ypre.ptr) return SP_ERR_INVALID_ARG;
+  if (!valid_act_dtype(m->X.dtype) || m->Ypre.dtype != m->X.dtype) return SP_ERR_DTYPE;
+  if (m->X.rows != N || m->X.cols != m->d || m->X.ld != m->d) return SP_ERR_SHAPE;
+  if (m->Ypre.rows != N || m->Ypre.cols != m->d || m->Ypre.ld != m->d) return SP_ERR_SHAPE;
+  const sp_mat* w[4] = {&m->Wq, &m->Wk, &m->Wv, &m->Wo};
+  for (const sp_mat* x : w) {
+    if (!x->ptr) return SP_ERR_INVALID_ARG;
+    if (x->dtype != SP_F32) return SP_ERR_DTYPE;
+    if (x->rows != m->d || x->cols != m->d || x->ld != m->d) return SP_ERR_SHAPE;
+  }
+  if (!st->Zq || !st->Zk || !st->P || !st->Aattn) return SP_ERR_INVALID_ARG;
+  // the tensor-core path slices heads out of token-major tensors with 16-byte aligned strides
+  if (m->X.dtype == SP_BF16 && ((m->d / m->n_heads) % 8 != 0 || m->T % 8 != 0)) return SP_ERR_ALIGNMENT;
+  if (misaligned(st->Zq, 16) || misaligned(st->Zk, 16) || misaligned(st->P, 16) || misaligned(st->Aattn, 16) ||
+      misaligned(m->X.ptr, 16) || misaligned(m->Ypre.ptr, 16))
+    return SP_ERR_ALIGNMENT;
+  return SP_OK;
+}
+
+// X W^T for all tokens of a chunk with fp32 weights W [d, d] (bf16 mode: hi | lo split Ws), fp32 result [Tc, d].
+sp_status project(const MhaPlan& p, MatRef xc, const void* Ws, const sp_mat& W, float* out, int64_t Tc, int32_t* status,
+                  cudaStream_t s) {
+  MatRef o{out, SP_F32, p.d};
+  if (p.bf16) return contract_split_weights(Tc, p.d, p.d, xc, Ws, MatRef{W.ptr, SP_F32, W.ld}, o, status, s);
+  return contract(Tc, p.d, p.d, 1.0, xc, true, MatRef{W.ptr, SP_F32, W.ld}, true, 0.0, o, o, false, true, false, status, s);
+}
+
+constexpr int kSegHH[1] = {0};
+constexpr int kSeg3A[3] = {0, 1, 0}, kSeg3B[3] = {0, 0, 1};   // hi.hi, lo.hi, hi.lo
+
+}  // namespace
+
+extern "C" {
+
+size_t sp_mha_workspace_bytes(int64_t d, int64_t n_heads, int64_t T, int64_t n_seq, int64_t seq_chunk, int32_t dtype) {
+  if (d < 1 || n_heads < 1 || T < 1 || n_seq < 1) return 0;
+  return plan_mha(nullptr, d, n_heads, T, n_seq, seq_chunk, dtype).bytes + 256;
+}
+
+// Shared body of sp_mha_init (init = true: the forward definition) and sp_mha_step.
+static sp_status mha_impl(const sp_mha_module* m, sp_mha_state* st, const sp_mha_params* prm, bool init,
+                          int64_t seq_chunk, int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+  SPCHK(check_mha(m, st));
+  const int64_t d = m->d, H = m->n_heads, T = m->T, n_seq = m->n_seq, dh = d / H;
+  const int32_t cdt = m->X.dtype;
+  if (!prm) return SP_ERR_INVALID_ARG;
+  if (!init) {
+    if (!(prm->alpha > 0.0) || !(prm->beta > 0.0) || prm->a_steps < 0 || prm->z_steps < 0 || !(prm->eta_z > 0.0) ||
+        prm->eta_z > 1.0 || prm->seq_chunk < 0)
+      return SP_ERR_INVALID_ARG;
+    seq_chunk = prm->seq_chunk;
+  }
+  if (seq_chunk < 0) return SP_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < plan_mha(nullptr, d, H, T, n_seq, seq_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256)) return SP_ERR_ALIGNMENT;
+  MhaPlan p = plan_mha(ws, d, H, T, n_seq, seq_chunk, cdt);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const bool bf16 = p.bf16, causal = prm->causal != 0;
+  const int64_t dp = split_kpad(d);
+  const size_t esz = bf16 ? 2 : 4;
+  const double inv_sqrt = 1.0 / sqrt((double)dh);
+  const int64_t TT = T * T;
+  const int32_t odt = bf16 ? SP_BF16 : SP_F32;      // type of the operand copies
+  const int64_t plane = p.cap * d;                   // distance of the lo plane of [cap, d] operand copies
+
+  // ---- operands that do not depend on the tokens
+  if (bf16) {
+    CU(split_bf16(reinterpret_cast<const float*>(m->Wq.ptr), d, nullptr, d, d, dp, p.Wqs, s));
+    CU(split_bf16(reinterpret_cast<const float*>(m->Wk.ptr), d, nullptr, d, d, dp, p.Wks, s));
+    CU(split_bf16(reinterpret_cast<const float*>(m->Wv.ptr), d, nullptr, d, d, dp, p.Wvs, s));
+    if (init) CU(split_bf16(reinterpret_cast<const float*>(m->Wo.ptr), d, nullptr, d, d, dp, p.Wos, s));
+  }
+  if (!init) {
+    // Eq. (86): a_attn = (W_O^T W_O + I)^-1 (W_O^T ypre + heads); token-major: A_attn = Ypre M1 + Hd Cinv with
+    // [M1; Cinv] = [W_O; I] (W_O^T W_O + I)^-1, one regularised solve with 2 d right-hand sides
+    MatRef wo{m->Wo.ptr, SP_F32, d}, cf{p.Cf, SP_F32, d};
+    SPCHK(contract(d, d, d, 1.0, wo, false, wo, false, 0.0, cf, cf, true, true, false, status_dev, s));
+    CU(symmetrize_lower(p.Cf, d, d, s));
+    CU(cudaMemcpyAsync(p.RW, m->Wo.ptr, (size_t)d * d * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    CU(set_identity(p.RW + (size_t)d * d, d, d, s));
+    CU(effective_ridge(nullptr, 0, 1, 1.0, 0, p.sb.rho, s));
+    if (bf16) SPCHK(ridge_core<float>(p.RW, d, p.Cf, d, 2 * d, d, nullptr, d, p.sb.rho, p.MC, d, p.sb, status_dev, s));
+    else SPCHK(ridge_core<double>(p.RW, d, p.Cf, d, 2 * d, d, nullptr, d, p.sb.rho, p.MC, d, p.sb, status_dev, s));
+    if (bf16) {
+      CU(split_bf16(p.MC, d, nullptr, d, d, dp, p.M1s, s));
+      CU(split_bf16(p.MC + (size_t)d * d, d, nullptr, d, d, dp, p.Cis, s));
+    }
+  }
+
+  for (int64_t q0 = 0; q0 < n_seq; q0 += p.sc) {
+    const int64_t nq = (n_seq - q0 < p.sc) ? n_seq - q0 : p.sc;
+    const int64_t t0 = q0 * T, Tc = nq * T;
+    const int nb0 = (int)H, nb1 = (int)nq;
+    const int64_t pairs = nq * H;
+    MatRef xc{reinterpret_cast<const uint8_t*>(m->X.ptr) + (size_t)t0 * d * esz, cdt, d};
+    MatRef yc{reinterpret_cast<uint8_t*>(m->Ypre.ptr) + (size_t)t0 * d * esz, cdt, d};
+    float* Zq = st->Zq + (size_t)t0 * d;
+    float* Zk = st->Zk + (size_t)t0 * d;
+    float* Aat = st->Aattn + (size_t)t0 * d;
+    float* P = st->P + (size_t)q0 * H * TT;
+    // views: [T, d_h] slices of token-major tensors, and [pairs, T, T] tensors
+    auto tokv = [&](const void* ptr, int32_t dt, int64_t ld, int planes, int64_t pl) {
+      return BMat{ptr, dt, ld, dh, T * ld, planes, pl};
+    };
+    auto ttv = [&](const void* ptr, int32_t dt) { return BMat{ptr, dt, T, TT, H * TT, 1, 0}; };
+    const int64_t pplane = p.sc * H * TT;            // distance of the lo plane of the bf16 copy of P
+    const BMat Pop = bf16 ? BMat{p.Pb, SP_BF16, T, TT, H * TT, 2, pplane} : ttv(P, SP_F32);
+    const BMat none{nullptr, SP_F32, 0, 0, 0, 1, 0};
+
+    // targets of the projections (and, at initialisation, the projections themselves)
+    SPCHK(project(p, xc, p.Wqs, m->Wq, init ? Zq : p.Tq, Tc, status_dev, s));
+    SPCHK(project(p, xc, p.Wks, m->Wk, init ? Zk : p.Tk, Tc, status_dev, s));
+    SPCHK(project(p, xc, p.Wvs, m->Wv, p.Vf, Tc, status_dev, s));
+    const void* Vop = p.Vf;
+    const void* Zqop = Zq;
+    const void* Zkop = Zk;
+    if (bf16) {
+      CU(split_planes(p.Vf, Tc * d, p.Vs, plane, s));
+      CU(split_planes(Zq, Tc * d, p.Zqs, plane, s));
+      CU(split_planes(Zk, Tc * d, p.Zks, plane, s));
+      Vop = p.Vs; Zqop = p.Zqs; Zkop = p.Zks;
+    }
+    const int np2 = bf16 ? 2 : 1;
+    const BMat Vv = tokv(Vop, odt, d, np2, plane), Zqv = tokv(Zqop, odt, d, np2, plane), Zkv = tokv(Zkop, odt, d, np2, plane);
+
+    // logits S = Zq_i Zk_i^T / sqrt(d_h) and Phi = softmax(S)
+    SPCHK(bcontract(T, T, dh, inv_sqrt, Zqv, true, Zkv, true, bf16 ? 3 : 1, kSeg3A, kSeg3B, 0.0, none, ttv(p.S, SP_F32), 0,
+                    nb0, nb1, status_dev, s));
+    if (init) {
+      // forward definition: P = softmax(S), heads = P V, Ypre = heads W_O^T
+      CU(mha_softmax_rows(p.S, pairs, (int)T, causal, p.Pb, pplane, s));
+      CU(cudaMemcpyAsync(P, p.S, (size_t)pairs * TT * sizeof(float), cudaMemcpyDeviceToDevice, s));
+      SPCHK(bcontract(T, dh, T, 1.0, Pop, true, Vv, false, bf16 ? 3 : 1, kSeg3A, kSeg3B, 0.0, none,
+                      tokv(Aat, SP_F32, d, 1, 0), 0, nb0, nb1, status_dev, s));
+      if (bf16) {
+        CU(split_bf16(Aat, d, nullptr, Tc, d, dp, p.Hd, s));
+        TcOperand ta{p.Hd, 2 * dp, true}, tb{p.Wos, 2 * dp, true};
+        ta.kext = tb.kext = 2 * dp;
+        TcSegments sg;
+        sg.nseg = 3;
+        sg.a_k[1] = (int32_t)dp;
+        sg.b_k[2] = (int32_t)dp;
+        SPCHK(gemm_tc(Tc, d, d, 1.f, ta, tb, 0.f, Operand{yc.ptr, cdt, d, 1}, OutOperand{const_cast<void*>(yc.ptr), cdt, d},
+                      false, status_dev, s, &sg, 2.0 * (double)Tc * d * d));
+      } else {
+        MatRef a{Aat, SP_F32, d};
+        SPCHK(contract(Tc, d, d, 1.0, a, true, MatRef{m->Wo.ptr, SP_F32, d}, true, 0.0, yc, yc, false, true, false,
+                       status_dev, s));
+      }
+      continue;
+    }
+
+    // ---- Eq. (85): gradient steps on P with Phi fixed
+    CU(mha_softmax_rows(p.S, pairs, (int)T, causal, nullptr, 0, s));
+    CU(mha_step_sizes(p.Vf, nullptr, d, nq, (int)T, (int)dh, (int)H, 0, prm->alpha, prm->beta, 0.0, p.sums, p.eta_a, s));
+    if (bf16) CU(split_planes(P, pairs * TT, p.Pb, pplane, s));
+    const BMat Rv = tokv(p.Rb, odt, d, 1, 0);
+    for (int it = 0; it < prm->a_steps; ++it) {
+      // R = A_attn_i - P V_i ; G1 = R V_i^T
+      SPCHK(bcontract(T, dh, T, -1.0, Pop, true, Vv, false, bf16 ? 3 : 1, kSeg3A, kSeg3B, 1.0, tokv(Aat, SP_F32, d, 1, 0),
+                      Rv, 0, nb0, nb1, status_dev, s));
+      SPCHK(bcontract(T, T, dh, 1.0, Rv, true, Vv, true, 1, kSegHH, kSegHH, 0.0, none, ttv(p.G, SP_F32), 0, nb0, nb1,
+                      status_dev, s));
+      CU(mha_p_update(P, p.S, p.G, p.eta_a, pairs, (int)T, prm->alpha, prm->beta, p.Pb, pplane, s));
+    }
+    // ---- Eq. (86): head outputs Hd = P V, then A_attn = Ypre M1 + Hd Cinv
+    {
+      BMat hv = bf16 ? tokv(p.Hd, SP_BF16, 2 * dp, 1, 0) : tokv(p.Hd, SP_F32, d, 1, 0);
+      SPCHK(bcontract(T, dh, T, 1.0, Pop, true, Vv, false, bf16 ? 3 : 1, kSeg3A, kSeg3B, 0.0, none, hv, bf16 ? dp : 0,
+                      nb0, nb1, status_dev, s));
+      if (bf16) {
+        TcOperand ya{yc.ptr, d, true}, mb{p.M1s, 2 * dp, false};
+        mb.kext = d;
+        mb.mnext = 2 * dp;
+        TcSegments s1;
+        s1.nseg = 2;
+        s1.b_mn[1] = (int32_t)dp;
+        SPCHK(gemm_tc(Tc, d, d, 1.f, ya, mb, 0.f, Operand{Aat, SP_F32, d, 1}, OutOperand{Aat, SP_F32, d}, false,
+                      status_dev, s, &s1, 2.0 * (double)Tc * d * d));
+        TcOperand ha{p.Hd, 2 * dp, true}, cb{p.Cis, 2 * dp, false};
+        ha.kext = 2 * dp;
+        cb.kext = d;
+        cb.mnext = 2 * dp;
+        TcSegments s2;
+        s2.nseg = 3;
+        s2.a_k[1] = (int32_t)dp;
+        s2.b_mn[2] = (int32_t)dp;
+        SPCHK(gemm_tc(Tc, d, d, 1.f, ha, cb, 1.f, Operand{Aat, SP_F32, d, 1}, OutOperand{Aat, SP_F32, d}, false,
+                      status_dev, s, &s2, 2.0 * (double)Tc * d * d));
+      } else {
+        MatRef a{Aat, SP_F32, d}, m1{p.MC, SP_F32, d}, ci{p.MC + (size_t)d * d, SP_F32, d}, hd{p.Hd, SP_F32, d};
+        SPCHK(contract(Tc, d, d, 1.0, yc, true, m1, false, 0.0, a, a, false, true, false, status_dev, s));
+        SPCHK(contract(Tc, d, d, 1.0, hd, true, ci, false, 1.0, a, a, false, true, false, status_dev, s));
+      }
+    }
+    // ---- Eq. (87): joint gradient steps on (Zq, Zk) through the softmax
+    for (int it = 0; it < prm->z_steps; ++it) {
+      SPCHK(bcontract(T, T, dh, inv_sqrt, Zqv, true, Zkv, true, bf16 ? 3 : 1, kSeg3A, kSeg3B, 0.0, none,
+                      ttv(p.G, SP_F32), 0, nb0, nb1, status_dev, s));
+      CU(mha_softmax_backward_rows(p.G, P, pairs, (int)T, causal, prm->beta, p.Pb, s));
+      const BMat dS = bf16 ? ttv(p.Pb, SP_BF16) : ttv(p.G, SP_F32);
+      // gq = dS Zk_i / sqrt(d_h), gk = dS^T Zq_i / sqrt(d_h) (hi parts of the operands)
+      BMat Zk1 = Zkv, Zq1 = Zqv;
+      Zk1.planes = Zq1.planes = 1;
+      SPCHK(bcontract(T, dh, T, inv_sqrt, dS, true, Zk1, false, 1, kSegHH, kSegHH, 0.0, none, tokv(p.Gq, SP_F32, d, 1, 0),
+                      0, nb0, nb1, status_dev, s));
+      SPCHK(bcontract(T, dh, T, inv_sqrt, dS, false, Zq1, false, 1, kSegHH, kSegHH, 0.0, none, tokv(p.Gk, SP_F32, d, 1, 0),
+                      0, nb0, nb1, status_dev, s));
+      CU(mha_step_sizes(Zq, Zk, d, nq, (int)T, (int)dh, (int)H, 1, prm->alpha, prm->beta, prm->eta_z, p.sums, p.eta_z, s));
+      CU(mha_z_update(Zq, Zk, p.Gq, p.Gk, p.Tq, p.Tk, p.eta_z, Tc, (int)d, (int)T, (int)dh, prm->alpha,
+                      bf16 ? p.Zqs : nullptr, bf16 ? p.Zks : nullptr, plane, s));
+    }
+  }
+  return SP_OK;
+}
+
+sp_status sp_mha_init(const sp_mha_module* m, sp_mha_state* st, int32_t causal, int64_t seq_chunk, int32_t* status_dev,
+                      void* ws, size_t ws_bytes, void* stream) {
+  sp_mha_params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.causal = causal;
+  return mha_impl(m, st, &prm, true, seq_chunk, status_dev, ws, ws_bytes, stream);
+}
+
+sp_status sp_mha_step(const sp_mha_module* m, sp_mha_state* st, const sp_mha_params* p, int32_t* status_dev, void* ws,
+                      size_t ws_bytes, void* stream) {
+  return mha_impl(m, st, p, false, 0, status_dev, ws, ws_bytes, stream);
+}
+
+}  // extern "C"

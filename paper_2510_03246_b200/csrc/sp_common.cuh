@@ -108,12 +108,27 @@ struct TcSegments {
   int32_t nseg = 1;
   int32_t a_k[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, a_mn[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
   int32_t b_k[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, b_mn[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
+  // batched launches only: the plane of A / B the segment reads (see TcBatch)
+  int32_t a_p[kTcMaxSegments] = {0, 0, 0, 0, 0, 0}, b_p[kTcMaxSegments] = {0, 0, 0, 0, 0, 0};
+};
+// Batched form: nb0 * nb1 independent products C_b = alpha A_b B_b (+ beta Cin_b) of the same shape in ONE launch.
+// Operand X of product (b0, b1) starts at ptr + b0 * x_s0 + b1 * x_s1 (elements); this is how the per-head,
+// per-sequence products of an attention module (head = a column slice of a token-major tensor, sequence = a row range)
+// are issued together.  A and B may also consist of several planes (e.g. the hi and lo parts of a split operand, each
+// a whole tensor, x_plane elements apart); a K segment then names the plane it reads.  Every stride times the element
+// size must be a multiple of 16 bytes.  Not available together with lower_only or a cut along K.
+struct TcBatch {
+  int32_t nb0 = 1, nb1 = 1;
+  int64_t a_s0 = 0, a_s1 = 0, b_s0 = 0, b_s1 = 0, c_s0 = 0, c_s1 = 0, cin_s0 = 0, cin_s1 = 0;
+  int32_t a_planes = 1, b_planes = 1;
+  int64_t a_plane = 0, b_plane = 0;
 };
 // K is the extent of ONE segment.  alg_flops >= 0 overrides the flop count recorded for profiling.  max_pairs > 0
 // limits the launch to that many CTA pairs (SM pairs), leaving the other SMs to kernels of another stream.
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
                   OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream,
-                  const TcSegments* segs = nullptr, double alg_flops = -1.0, int max_pairs = 0);
+                  const TcSegments* segs = nullptr, double alg_flops = -1.0, int max_pairs = 0,
+                  const TcBatch* batch = nullptr);
 bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B);
 
 // Dense symmetric positive definite solve in precision T (float or double), all on `stream`.
@@ -252,6 +267,29 @@ cudaError_t launch_init_act(const float* Z, float* gate_io, void* A_out, void* Z
                             int64_t n, double* absA_part, int32_t row_blocks, cudaStream_t stream);
 cudaError_t column_stats(const void* X, int32_t dt, int64_t ld, int64_t T, int64_t C, double* rowstats,
                          double* scratch, cudaStream_t stream);
+
+// ---- multi-head-attention auxiliary updates (sp_mha.cu); [pairs, T, T] tensors, pair = sequence * heads + head --------
+// S <- softmax over each row (in place); causal: key u > query t gets 0; Sb: optional bf16 copy (plane > 0: hi and,
+// `plane` elements further, lo parts)
+cudaError_t mha_softmax_rows(float* S, int64_t pairs, int T, bool causal, void* Sb, int64_t plane, cudaStream_t stream);
+// P <- P - eta_pair (-2 alpha G1 + 2 beta (P - Phi)); Pb: optional bf16 copy of the new P (hi / lo planes as above)
+cudaError_t mha_p_update(float* P, const float* Phi, const float* G1, const float* eta, int64_t pairs, int T,
+                         double alpha, double beta, void* Pb, int64_t plane, cudaStream_t stream);
+// S (logits) <- dS = 2 beta Phi (E - rowsum(E Phi)), Phi = softmax(S), E = Phi - P; dSb: optional bf16 copy
+cudaError_t mha_softmax_backward_rows(float* S, const float* P, int64_t pairs, int T, bool causal, double beta,
+                                      void* dSb, cudaStream_t stream);
+// per-pair step sizes from the squared norms of the [T, d_h] slices of x (and y): mode 0: 1 / (2 (alpha s + beta)),
+// mode 1: eta_z / (2 alpha + beta s / d_h); sums: n_seq * H doubles of scratch
+cudaError_t mha_step_sizes(const float* x, const float* y, int64_t ld, int64_t n_seq, int T, int d_h, int H, int mode,
+                           double alpha, double beta, double eta_z, double* sums, float* eta, cudaStream_t stream);
+// Z <- Z - eta_pair (G + 2 alpha (Z - T)) for Zq and Zk ([tokens, d] dense); Zqs / Zks: optional bf16 hi / lo planes
+cudaError_t mha_z_update(float* Zq, float* Zk, const float* Gq, const float* Gk, const float* Tq, const float* Tk,
+                         const float* eta, int64_t tokens, int d, int T, int d_h, double alpha, void* Zqs, void* Zks,
+                         int64_t plane, cudaStream_t stream);
+// A[n, n] (ld) = identity
+cudaError_t set_identity(float* A, int64_t n, int64_t ld, cudaStream_t stream);
+// dst[e] = bf16(x[e]), dst[plane + e] = bf16(x[e] - hi) (plane == 0: hi only)
+cudaError_t split_planes(const float* x, int64_t total, void* dst, int64_t plane, cudaStream_t stream);
 
 // ---- scores / allocation / selection (sp_mask.cu) -----------------------------------------------------------------
 cudaError_t wanda_scores(int kind, int group, const float* W, int64_t rows, int64_t ldw, const float* colsq,

@@ -74,8 +74,28 @@ struct TcParams {
   // add up in C).  n_plain = 0 cuts every tile; n_plain = whole waves of CTA pairs cuts only the tiles of the last,
   // partly filled wave, so that it keeps every pair busy for 1 / ksplit of a tile time.
   int32_t ksplit, kb_per_split, num_units, n_plain;
+  // batched launches: product (b0, b1) of nb0 x nb1; tile index = product * tiles_per_batch + local tile.  The tensor
+  // maps then have five dimensions; x_ord[r] is the coordinate slot (1..4) of role r = outer dimension, b0, b1, plane
+  // in the map of operand x (the maps order their dimensions by stride).
+  int32_t batched, nb0, nb1, tiles_per_batch;
+  int8_t a_ord[4], b_ord[4], c_ord[4];
+  int64_t c_s0, c_s1, cin_s0, cin_s1;
   int32_t* status;
 };
+
+struct Coord5 {
+  int32_t x[5];
+};
+__device__ __forceinline__ Coord5 make_coord(const int8_t* ord, int32_t inner, int32_t outer, int32_t b0, int32_t b1,
+                                             int32_t plane) {
+  Coord5 c;
+  c.x[0] = inner;
+  c.x[ord[0]] = outer;
+  c.x[ord[1]] = b0;
+  c.x[ord[2]] = b1;
+  c.x[ord[3]] = plane;
+  return c;
+}
 
 __device__ __forceinline__ void unit_map(const TcParams& p, int u, int num_kb, int& tile, int& kb0, int& kb1) {
   if (u < p.n_plain) {
@@ -170,6 +190,24 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, int32_
                ::"l"(map), "r"(c0), "r"(c1), "r"(src)
                : "memory");
 }
+// five-dimensional forms for batched launches
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, const Coord5& c,
+                                            uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(map), "r"(c.x[0]), "r"(c.x[1]), "r"(c.x[2]), "r"(c.x[3]), "r"(c.x[4]), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, const Coord5& c, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4, %5}], [%6];"
+               ::"l"(map), "r"(c.x[0]), "r"(c.x[1]), "r"(c.x[2]), "r"(c.x[3]), "r"(c.x[4]), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_5d(const CUtensorMap* map, const Coord5& c, uint32_t src) {
+  asm volatile("cp.reduce.async.bulk.tensor.5d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3, %4, %5}], [%6];"
+               ::"l"(map), "r"(c.x[0]), "r"(c.x[1]), "r"(c.x[2]), "r"(c.x[3]), "r"(c.x[4]), "r"(src)
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -236,7 +274,15 @@ __device__ __forceinline__ uint32_t make_instr_desc(bool a_kmajor, bool b_kmajor
   return d;
 }
 
-__device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, int& tn) {
+__device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, int& tn, int& b0, int& b1) {
+  b0 = 0;
+  b1 = 0;
+  if (p.batched) {
+    const int bi = t / p.tiles_per_batch;
+    t -= bi * p.tiles_per_batch;
+    b0 = bi % p.nb0;
+    b1 = bi / p.nb0;
+  }
   if (!p.lower_only) {
     if (p.n_fast) {
       tn = t % p.tiles_n;
@@ -329,9 +375,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t ph = 0;
       bool ok = true;
       for (int u = cid; u < p.num_units && ok; u += ncl) {
-        int tm, tn, tile, kb0, kb1;
+        int tm, tn, tile, kb0, kb1, b0, b1;
         unit_map(p, u, num_kb, tile, kb0, kb1);
-        tile_coords(p, tile, tm, tn);
+        tile_coords(p, tile, tm, tn, b0, b1);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           // the leader's barrier collects the bytes of both CTAs' loads of this stage
@@ -344,13 +390,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const int ka = kk + p.seg.a_k[sg], kbb = kk + p.seg.b_k[sg];
           const int am = tm * TILE_M + (int)rank * BM + p.seg.a_mn[sg];
           const int bn = tn * TILE_N + (int)rank * BNH + p.seg.b_mn[sg];
-          if (p.a_kmajor) {
+          if (p.batched) {
+            const int pa = p.seg.a_p[sg], pb = p.seg.b_p[sg];
+            if (p.a_kmajor) {
+              tma_load_5d(a_dst, &tmA, make_coord(p.a_ord, ka, am, b0, b1, pa), fbar);
+            } else {
+#pragma unroll
+              for (int mb = 0; mb < BM / 64; ++mb)
+                tma_load_5d(a_dst + mb * (64 * BK * 2), &tmA, make_coord(p.a_ord, am + mb * 64, ka, b0, b1, pa), fbar);
+            }
+            if (p.b_kmajor) {
+              tma_load_5d(b_dst, &tmB, make_coord(p.b_ord, kbb, bn, b0, b1, pb), fbar);
+            } else {
+#pragma unroll
+              for (int nb = 0; nb < BNH / 64; ++nb)
+                tma_load_5d(b_dst + nb * (64 * BK * 2), &tmB, make_coord(p.b_ord, bn + nb * 64, kbb, b0, b1, pb), fbar);
+            }
+          } else if (p.a_kmajor) {
             tma_load_2d(a_dst, &tmA, ka, am, fbar);
           } else {
 #pragma unroll
             for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, am + mb * 64, ka, fbar);
           }
-          if (p.b_kmajor) {
+          if (p.batched) {
+          } else if (p.b_kmajor) {
             tma_load_2d(b_dst, &tmB, kbb, bn, fbar);
           } else {
 #pragma unroll
@@ -429,9 +492,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool has_cin = p.beta != 0.f;
     const bool cin_f32 = p.cin_dtype == SP_F32, c_f32 = p.c_dtype == SP_F32;
     for (int u = cid; u < p.num_units && ok; u += ncl) {
-      int tm, tn, tile, kb0_unused, kb1_unused;
+      int tm, tn, tile, kb0_unused, kb1_unused, b0, b1;
       unit_map(p, u, num_kb, tile, kb0_unused, kb1_unused);
-      tile_coords(p, tile, tm, tn);
+      tile_coords(p, tile, tm, tn, b0, b1);
+      const int64_t c_boff = (int64_t)b0 * p.c_s0 + (int64_t)b1 * p.c_s1;
+      const int64_t cin_boff = (int64_t)b0 * p.cin_s0 + (int64_t)b1 * p.cin_s1;
       // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
       const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
@@ -520,8 +585,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           __syncwarp();
           if (lane == 0) {
             if (rows_here > 0) {
-              if (p.epi_mode == EPI_TMA_STORE) tma_store_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
-              else tma_reduce_add_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+              if (p.batched) {
+                const Coord5 cc = make_coord(p.c_ord, (int32_t)gj0, (int32_t)row0, b0, b1, 0);
+                if (p.epi_mode == EPI_TMA_STORE) tma_store_5d(&tmC, cc, wstg + buf * 4096);
+                else tma_reduce_add_5d(&tmC, cc, wstg + buf * 4096);
+              } else if (p.epi_mode == EPI_TMA_STORE) {
+                tma_store_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+              } else {
+                tma_reduce_add_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+              }
             }
             bulk_commit();
           }
@@ -539,7 +611,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // block is read from tensor memory and turned)
           float cv[32];
           if (has_cin) {
-            const int64_t cin_off = row0 * p.cin_ld + gj;
+            const int64_t cin_off = cin_boff + row0 * p.cin_ld + gj;
 #pragma unroll
             for (int rr = 0; rr < 32; ++rr) {
               cv[rr] = 0.f;
@@ -557,7 +629,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int i = 0; i < 32; ++i) stg[lane][i] = p.alpha * __uint_as_float(r[i]);
           __syncwarp();
           if (gj < p.N) {
-            const int64_t c_off = row0 * p.c_ld + gj;
+            const int64_t c_off = c_boff + row0 * p.c_ld + gj;
 #pragma unroll
             for (int rr = 0; rr < 32; ++rr) {
               if (rr < rows_here) {
@@ -639,6 +711,49 @@ bool make_map(CUtensorMap* map, bool f32, const void* ptr, int64_t inner, int64_
 
 }  // namespace
 
+namespace {
+// Five-dimensional tensor map of a batched operand.  Roles: inner (contiguous) dimension, outer dimension (stride ld),
+// batch dimensions b0 and b1, plane.  The non-inner dimensions are laid out in the map by ascending stride (extent-1
+// dimensions last); ord[r] receives the slot (1..4) of role r = outer, b0, b1, plane.  Boxes are 1 deep in b0, b1, plane.
+bool make_map5(CUtensorMap* map, bool f32, const void* ptr, int64_t inner, int box_inner, int64_t outer, int64_t ld,
+               int box_outer, int64_t nb0, int64_t s0, int64_t nb1, int64_t s1, int64_t planes, int64_t plane_stride,
+               bool swizzle_none_ok, int8_t ord[4]) {
+  (void)swizzle_none_ok;
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const int64_t es = f32 ? 4 : 2;
+  struct Dim { int64_t ext, stride; int box, role; };
+  Dim dm[4] = {{outer, ld, box_outer, 0}, {nb0, s0, 1, 1}, {nb1, s1, 1, 2}, {planes, plane_stride, 1, 3}};
+  // insertion sort by (extent == 1, stride)
+  for (int i = 1; i < 4; ++i)
+    for (int j = i; j > 0; --j) {
+      const bool a1 = dm[j - 1].ext <= 1, b1 = dm[j].ext <= 1;
+      const bool swap = (a1 && !b1) || (a1 == b1 && !a1 && dm[j].stride < dm[j - 1].stride);
+      if (!swap) break;
+      const Dim t = dm[j - 1]; dm[j - 1] = dm[j]; dm[j] = t;
+    }
+  cuuint64_t dims[5] = {(cuuint64_t)inner, 1, 1, 1, 1};
+  cuuint64_t strides[4];
+  cuuint32_t box[5] = {(cuuint32_t)box_inner, 1, 1, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  int64_t last = 16;
+  for (int i = 0; i < 4; ++i) {
+    dims[i + 1] = (cuuint64_t)(dm[i].ext > 0 ? dm[i].ext : 1);
+    box[i + 1] = (cuuint32_t)dm[i].box;
+    int64_t st = dm[i].stride * es;
+    if (dm[i].ext <= 1 && dm[i].role != 0) st = last;     // unused dimension: any legal stride
+    if (st <= 0 || st % 16 != 0) return false;
+    strides[i] = (cuuint64_t)st;
+    last = st > last ? st : last;
+    ord[dm[i].role] = (int8_t)(i + 1);
+  }
+  CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5,
+                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+}  // namespace
+
 int sm_count() {
   static std::mutex mu;
   static int table[PerDeviceOnce::kMaxDevices] = {};
@@ -663,7 +778,10 @@ bool gemm_tc_supported(int64_t M, int64_t N, int64_t K, TcOperand A, TcOperand B
 
 sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcOperand B, float beta, Operand Cin,
                   OutOperand C, bool lower_only, int32_t* status_dev, cudaStream_t stream, const TcSegments* segs,
-                  double alg_flops, int max_pairs) {
+                  double alg_flops, int max_pairs, const TcBatch* batch) {
+  const bool batched = batch != nullptr;
+  if (batched && (lower_only || batch->nb0 < 1 || batch->nb1 < 1 || batch->a_planes < 1 || batch->b_planes < 1))
+    return SP_ERR_INVALID_ARG;
   TcSegments sg;
   if (segs) sg = *segs;
   else { sg = TcSegments{}; sg.nseg = 1; }
@@ -687,13 +805,36 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   CUtensorMap tmA, tmB, tmC, tmCin;
   memset(&tmC, 0, sizeof(tmC));
   memset(&tmCin, 0, sizeof(tmCin));
-  bool ok = A.kmajor ? make_map(&tmA, false, A.ptr, a_kext, a_mext, A.ld, BK, BM)
-                     : make_map(&tmA, false, A.ptr, a_mext, a_kext, A.ld, 64, BK);
-  ok = ok && (B.kmajor ? make_map(&tmB, false, B.ptr, b_kext, b_next, B.ld, BK, BNH)
-                       : make_map(&tmB, false, B.ptr, b_next, b_kext, B.ld, 64, BK));
-  if (!ok) return SP_ERR_CUDA;
-
   TcParams p;
+  memset(&p, 0, sizeof(p));
+  bool ok;
+  if (batched) {
+    const TcBatch& bt = *batch;
+    for (int i = 0; i < sg.nseg; ++i)
+      if (sg.a_p[i] < 0 || sg.a_p[i] >= bt.a_planes || sg.b_p[i] < 0 || sg.b_p[i] >= bt.b_planes)
+        return SP_ERR_INVALID_ARG;
+    ok = A.kmajor ? make_map5(&tmA, false, A.ptr, a_kext, BK, a_mext, A.ld, BM, bt.nb0, bt.a_s0, bt.nb1, bt.a_s1,
+                              bt.a_planes, bt.a_plane, true, p.a_ord)
+                  : make_map5(&tmA, false, A.ptr, a_mext, 64, a_kext, A.ld, BK, bt.nb0, bt.a_s0, bt.nb1, bt.a_s1,
+                              bt.a_planes, bt.a_plane, true, p.a_ord);
+    ok = ok && (B.kmajor ? make_map5(&tmB, false, B.ptr, b_kext, BK, b_next, B.ld, BNH, bt.nb0, bt.b_s0, bt.nb1,
+                                     bt.b_s1, bt.b_planes, bt.b_plane, true, p.b_ord)
+                         : make_map5(&tmB, false, B.ptr, b_next, 64, b_kext, B.ld, BK, bt.nb0, bt.b_s0, bt.nb1,
+                                     bt.b_s1, bt.b_planes, bt.b_plane, true, p.b_ord));
+    if (!ok) return SP_ERR_ALIGNMENT;
+  } else {
+    ok = A.kmajor ? make_map(&tmA, false, A.ptr, a_kext, a_mext, A.ld, BK, BM)
+                  : make_map(&tmA, false, A.ptr, a_mext, a_kext, A.ld, 64, BK);
+    ok = ok && (B.kmajor ? make_map(&tmB, false, B.ptr, b_kext, b_next, B.ld, BK, BNH)
+                         : make_map(&tmB, false, B.ptr, b_next, b_kext, B.ld, 64, BK));
+    if (!ok) return SP_ERR_CUDA;
+  }
+  p.batched = batched ? 1 : 0;
+  p.nb0 = batched ? batch->nb0 : 1;
+  p.nb1 = batched ? batch->nb1 : 1;
+  p.c_s0 = batched ? batch->c_s0 : 0; p.c_s1 = batched ? batch->c_s1 : 0;
+  p.cin_s0 = batched ? batch->cin_s0 : 0; p.cin_s1 = batched ? batch->cin_s1 : 0;
+
   p.M = M; p.N = N; p.K = K;
   p.alpha = alpha; p.beta = beta;
   p.cin = Cin.ptr; p.cin_dtype = Cin.dtype; p.cin_ld = Cin.s0;
@@ -706,12 +847,23 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   // fp32 C that a tensor map can describe leaves through TMA: a store when nothing is added, an add-reduction when
   // the call accumulates into C itself (each element of C is touched once per launch, so the result is the same sum)
   p.epi_mode = EPI_DIRECT;
-  const bool c_tma = C.dtype == SP_F32 && C.ld % 4 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0;
+  bool c_tma = C.dtype == SP_F32 && C.ld % 4 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0;
+  if (batched && ((batch->nb0 > 1 && batch->c_s0 % 4 != 0) || (batch->nb1 > 1 && batch->c_s1 % 4 != 0))) c_tma = false;
   if (c_tma && beta == 0.f) p.epi_mode = EPI_TMA_STORE;
-  if (c_tma && beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && Cin.s0 == C.ld) p.epi_mode = EPI_TMA_ADD;
-  if (p.epi_mode != EPI_DIRECT && !make_map(&tmC, true, C.ptr, N, M, C.ld, 32, 32)) return SP_ERR_CUDA;
+  if (c_tma && beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && Cin.s0 == C.ld &&
+      (!batched || (batch->cin_s0 == batch->c_s0 && batch->cin_s1 == batch->c_s1)))
+    p.epi_mode = EPI_TMA_ADD;
+  if (p.epi_mode != EPI_DIRECT) {
+    if (batched) {
+      if (!make_map5(&tmC, true, C.ptr, N, 32, M, C.ld, 32, batch->nb0, batch->c_s0, batch->nb1, batch->c_s1, 1, 0,
+                     true, p.c_ord))
+        return SP_ERR_CUDA;
+    } else if (!make_map(&tmC, true, C.ptr, N, M, C.ld, 32, 32)) {
+      return SP_ERR_CUDA;
+    }
+  }
   // bf16 C = beta * Cin + alpha * acc with a bf16 Cin: both through TMA
-  if (p.epi_mode == EPI_DIRECT && p.c_lo_off == 0 && beta != 0.f && C.dtype == SP_BF16 && Cin.dtype == SP_BF16 &&
+  if (p.epi_mode == EPI_DIRECT && !batched && p.c_lo_off == 0 && beta != 0.f && C.dtype == SP_BF16 && Cin.dtype == SP_BF16 &&
       C.ld % 8 == 0 &&
       Cin.s0 % 8 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0 &&
       (reinterpret_cast<uintptr_t>(Cin.ptr) & 15u) == 0) {
@@ -733,6 +885,12 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   } else {
     p.num_tiles = p.tiles_m * p.tiles_n;
   }
+  p.tiles_per_batch = p.num_tiles;
+  if (batched) {
+    const int64_t all = (int64_t)p.num_tiles * batch->nb0 * batch->nb1;
+    if (all > 0x7fffffff) return SP_ERR_SHAPE;
+    p.num_tiles = (int32_t)all;
+  }
   p.status = status_dev;
 
   // Tile counts that do not fill the last wave of CTA pairs leave SMs idle.  A call that accumulates into C through
@@ -743,7 +901,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   if (max_pairs > 0 && max_pairs < pairs_max) pairs_max = max_pairs;
   const int num_kb = p.seg_kb * sg.nseg;
   p.ksplit = 1;
-  if ((p.epi_mode == EPI_TMA_STORE || p.epi_mode == EPI_TMA_ADD) && p.num_tiles > 0) {
+  if (!batched && (p.epi_mode == EPI_TMA_STORE || p.epi_mode == EPI_TMA_ADD) && p.num_tiles > 0) {
     auto eff = [&](int ks) {
       const double u = (double)p.num_tiles * ks;
       return u / (ceil(u / pairs_max) * pairs_max);
@@ -761,7 +919,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
     }
   }
   p.n_plain = 0;
-  if (p.epi_mode == EPI_TMA_ADD && p.num_tiles > pairs_max && p.num_tiles % pairs_max != 0) {
+  if (!batched && p.epi_mode == EPI_TMA_ADD && p.num_tiles > pairs_max && p.num_tiles % pairs_max != 0) {
     // Alternative: whole waves of uncut tiles, and only the tiles of the last wave cut, as many ways as pairs are
     // left per tile.  Times in units of one tile on one pair.
     const int full = p.num_tiles / pairs_max, rem = p.num_tiles % pairs_max;
@@ -785,7 +943,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
       }) != cudaSuccess)
     return SP_ERR_CUDA;
   count_launch();
-  const double flops = alg_flops >= 0.0 ? alg_flops : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K;
+  const double flops = alg_flops >= 0.0 ? alg_flops
+                                        : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K * p.nb0 * p.nb1;
   ProfScope prof(max_pairs > 0 ? PK_GEMM_TC_SHARED : PK_GEMM_TC, flops, 0.0, stream);
   const int pairs = p.num_units < pairs_max ? p.num_units : pairs_max;
   gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);

@@ -1,0 +1,118 @@
+"""Parity of the attention-module path (sp_mha_init, sp_mha_step) with the oracle's Method-2 functions (Appendix A,
+"Computation on Multi-Head Attention layers"; Algorithm 2, SparseLLM2) at reduced size, in fp32 and bf16 mode, through
+the C ABI.  The oracle works on one sequence with tokens as columns; the library stores everything token-major."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import struprune_oracle as O
+from paper_2510_03246_b200 import api, synth
+from tests._util import TOL, bf16_half_ulp, np64, relerr
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _case(dtype, d, H, T, n_seq, seed_layer=0):
+    cfg = synth.scaled(synth.CONFIGS["C2"], d=d, tokens=n_seq * T, outlier_frac=0.0,
+                       storage="f32" if dtype == torch.float32 else "bf16")
+    X = synth.make_activations(cfg, seed_layer)
+    ws = []
+    for tid in (11, 12, 13, 14):
+        w = synth.standard_variates(synth.module_seed(cfg, seed_layer), tid, d * d, "gauss").view(d, d)
+        ws.append((w * (1.2 / np.sqrt(d))).to(X.dtype))       # projections of unit-scale inputs stay O(1)
+    return X, ws
+
+
+def _oracle_forward(X, W, H, T, n_seq, causal):
+    Xo = np64(X)
+    out = []
+    for q in range(n_seq):
+        out.append(O.mha_forward(Xo[q * T:(q + 1) * T].T, *[np64(w) for w in W], H, causal))
+    return out
+
+
+CASES = [(torch.float32, 48, 4, 20, 3, 2, True), (torch.float32, 32, 1, 33, 2, 0, False),
+         (torch.bfloat16, 96, 4, 40, 3, 2, True), (torch.bfloat16, 256, 2, 136, 2, 1, False),
+         (torch.bfloat16, 128, 2, 264, 1, 0, True)]
+
+
+@pytest.mark.parametrize("dtype,d,H,T,n_seq,chunk,causal", CASES)
+def test_mha_init_matches_forward_definition(dtype, d, H, T, n_seq, chunk, causal):
+    X, W = _case(dtype, d, H, T, n_seq)
+    mod = api.MhaModule(X.to(DEV), *[w.to(DEV) for w in W], n_heads=H, T=T, seq_chunk=chunk)
+    mod.sp_mha_init(causal)
+    torch.cuda.synchronize()
+    mod.check_status()
+    tol = TOL[dtype]
+    ref = _oracle_forward(X, W, H, T, n_seq, causal)
+    for q, (Zq, Zk, V, P, A, Y) in enumerate(ref):
+        r = slice(q * T, (q + 1) * T)
+        assert relerr(np64(mod.Zq[r]).T, Zq) < tol and relerr(np64(mod.Zk[r]).T, Zk) < tol
+        assert relerr(np64(mod.P[q]), P) < tol, "P"
+        assert relerr(np64(mod.Aattn[r]).T, A) < tol, "Aattn"
+        got = np64(mod.Ypre[r]).T
+        if dtype == torch.bfloat16:
+            assert np.all(np.abs(got - Y) <= tol * np.abs(Y).max() + bf16_half_ulp(Y) * 1.001)
+        else:
+            assert relerr(got, Y) < tol
+
+
+@pytest.mark.parametrize("dtype,d,H,T,n_seq,chunk,causal", CASES)
+def test_mha_step_teacher_forced(dtype, d, H, T, n_seq, chunk, causal):
+    """Three outer steps with pruned weights (one head removed, the others perturbed); before every step the oracle
+    restarts from the GPU's state, then both take the step: Eq. (85) gradient steps on P, Eq. (86) closed form,
+    Eq. (87) gradient steps on (Zq, Zk)."""
+    X, W = _case(dtype, d, H, T, n_seq, seed_layer=1)
+    mod = api.MhaModule(X.to(DEV), *[w.to(DEV) for w in W], n_heads=H, T=T, seq_chunk=chunk)
+    mod.sp_mha_init(causal)
+    dh = d // H
+    Wp = [w.float().clone() for w in W]
+    if H > 1:
+        for w in Wp[:3]:
+            w[:dh] = 0
+        Wp[3][:, :dh] = 0
+    g = torch.Generator().manual_seed(7)
+    for w in Wp:
+        w.mul_(1.0 + 0.05 * torch.randn(w.shape, generator=g))
+    mod.set_weights(*[w.to(DEV) for w in Wp])
+    p_gpu = api.MhaParams(alpha=0.8, beta=1.3, a_steps=3, z_steps=2, eta_z=0.9, causal=causal)
+    p_or = O.MhaParams(n_heads=H, alpha=0.8, beta=1.3, a_steps=3, z_steps=2, eta_z=0.9, causal=causal)
+    tol = TOL[dtype]
+    Xo, Yo = np64(X), None
+    Wo64 = [np64(w) for w in Wp]
+    for it in range(3):
+        torch.cuda.synchronize()
+        before = [np64(t) for t in (mod.Zq, mod.Zk, mod.P, mod.Aattn)]
+        Yo = np64(mod.Ypre)
+        mod.sp_mha_step(p_gpu)
+        torch.cuda.synchronize()
+        mod.check_status()
+        obj0 = obj1 = 0.0
+        for q in range(n_seq):
+            r = slice(q * T, (q + 1) * T)
+            st = (before[0][r].T, before[1][r].T, before[2][q], before[3][r].T)
+            Zq, Zk, P, A = O.mha_step(Xo[r].T, Yo[r].T, *Wo64, *st, p_or)
+            assert relerr(np64(mod.P[q]), P) < tol, ("P", it, q)
+            assert relerr(np64(mod.Aattn[r]).T, A) < tol, ("Aattn", it, q)
+            assert relerr(np64(mod.Zq[r]).T, Zq) < tol and relerr(np64(mod.Zk[r]).T, Zk) < tol, ("Z", it, q)
+            obj0 += O.mha_objective(Xo[r].T, Yo[r].T, *Wo64, *st, p_or).sum()
+            got = (np64(mod.Zq[r]).T, np64(mod.Zk[r]).T, np64(mod.P[q]), np64(mod.Aattn[r]).T)
+            obj1 += O.mha_objective(Xo[r].T, Yo[r].T, *Wo64, *got, p_or).sum()
+        assert obj1 < obj0            # the GPU's new state lowers the Method-2 objective
+
+
+def test_mha_argument_errors():
+    X, W = _case(torch.bfloat16, 96, 4, 40, 2)
+    mod = api.MhaModule(X.to(DEV), *[w.to(DEV) for w in W], n_heads=4, T=40)
+    mod.sp_mha_init()
+    with pytest.raises(api.SpError) as e:
+        mod.sp_mha_step(api.MhaParams(alpha=-1.0))
+    assert e.value.code == 1
+    with pytest.raises(api.SpError) as e:
+        mod.sp_mha_step(api.MhaParams(eta_z=2.0))
+    assert e.value.code == 1
+    with pytest.raises(api.SpError) as e:          # head width 20 is not a multiple of 8: no 16-byte aligned slices
+        api.MhaModule(X[:, :80].contiguous().to(DEV), *[w[:80, :80].contiguous().to(DEV) for w in W], n_heads=4,
+                      T=40).sp_mha_init()
+    assert e.value.code == 4

@@ -367,12 +367,13 @@ def test_ffn_init(cfg, chunk):
 # Fraction of the entries of Z at which the exact select rule was found undecidable within the rounding of its
 # inputs, per call of the helper below (printed by pytest -s; the bound asserted is a few times what was measured).
 NEAR_TIE_FRACTIONS = []
-NEAR_TIE_LIMIT = 0.03
+NEAR_TIE_LIMIT = 0.005
 
 
-def _oracle_exact_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol):
-    """The oracle's step for z_rule = "exact", composed here from the oracle's own parts so that the one decision that
-    is not unique can be audited.  The exact rule compares the objective values fn, fp of the best point of each half
+def _oracle_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol, sign_delta=0.0):
+    """The oracle's step composed here from the oracle's own parts so that the one elementwise decision that is not
+    unique can be audited (z_rule = "exact" in every comparison; the literal rule only when the two sides run free and
+    their old z differ, see sign_delta below).  The exact rule compares the objective values fn, fp of the best point of each half
     line.  Both sides evaluate them from their own a + u and z1, which differ by rounding, so where |fn - fp| is below
     what that rounding can move it, either candidate is a valid minimiser: there the candidate nearer to the GPU's Z
     is adopted, and everything else is checked strictly.
@@ -388,22 +389,29 @@ def _oracle_exact_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol):
     U = st.U if p_t.dual_mode else None
     A = O.a_update(st.W2, Yo, st.Z, p_t.alpha, p_t.beta, U, p_t.act, st.gate)
     z1, z2 = O.z_candidates(st.W1, Xo, A, p_t.alpha, p_t.beta, U)
-    zn, zp, fn, fp = O.z_exact_candidates(z1, z2, A, p_t.alpha, p_t.beta, U)
-    Znew = O.z_select(st.Z, z1, z2, A, p_t.alpha, p_t.beta, "exact", U)
-    Au = A + (0.0 if U is None else U)
-    H = O.phi(st.Z, p_t.act, st.gate) - (0.0 if U is None else U)
-    dA = tol * np.abs(A - H).max() + 2.0 ** -22 * np.abs(Au).max()
-    dz = 2e-5 * np.abs(z1).max()
-    dzp = max(dA, dz)
-    margin = (2 * p_t.beta * np.abs(Au) * dA + 2 * p_t.alpha * np.abs(zn - z1) * dz
-              + 2 * p_t.beta * np.abs(Au - zp) * (dA + dzp) + 2 * p_t.alpha * np.abs(zp - z1) * (dzp + dz))
-    amb = (np.abs(fn - fp) <= margin) & (zn != zp)       # identical candidates are no ambiguity
+    Znew = O.z_select(st.Z, z1, z2, A, p_t.alpha, p_t.beta, p_t.z_rule, U)
+    if p_t.z_rule == "exact":
+        zn, zp, fn, fp = O.z_exact_candidates(z1, z2, A, p_t.alpha, p_t.beta, U)
+        Au = A + (0.0 if U is None else U)
+        H = O.phi(st.Z, p_t.act, st.gate) - (0.0 if U is None else U)
+        dA = tol * np.abs(A - H).max() + 2.0 ** -22 * np.abs(Au).max()
+        dz = 2e-5 * np.abs(z1).max()
+        dzp = max(dA, dz)
+        margin = (2 * p_t.beta * np.abs(Au) * dA + 2 * p_t.alpha * np.abs(zn - z1) * dz
+                  + 2 * p_t.beta * np.abs(Au - zp) * (dA + dzp) + 2 * p_t.alpha * np.abs(zp - z1) * (dzp + dz))
+        amb = (np.abs(fn - fp) <= margin) & (zn != zp)       # identical candidates are no ambiguity
+        ca, cb = zn, zp
+    else:
+        # literal rule of Algorithms 2 / 3: the sign of the OLD z decides.  When the two sides' old z differ by up to
+        # sign_delta (free-running comparison), an entry with |z_old| <= sign_delta can fall on either side of zero.
+        amb = (np.abs(st.Z) <= sign_delta) & (z1 != z2)
+        ca, cb = z1, z2
     frac = float(amb.mean())
     NEAR_TIE_FRACTIONS.append(frac)
-    print(f"exact select: {int(amb.sum())} of {amb.size} entries ({100 * frac:.3f} %) undecidable within rounding")
+    print(f"{p_t.z_rule} select: {int(amb.sum())} of {amb.size} entries ({100 * frac:.3f} %) undecidable within rounding")
     assert frac <= NEAR_TIE_LIMIT
-    pick_n = np.abs(Zg - zn) <= np.abs(Zg - zp)
-    Znew = np.where(amb, np.where(pick_n, zn, zp), Znew)
+    pick_a = np.abs(Zg - ca) <= np.abs(Zg - cb)
+    Znew = np.where(amb, np.where(pick_a, ca, cb), Znew)
     if p_t.dual_mode:
         st.U = O.dual_update(st.U, A, Znew, p_t.act, st.gate)
     st.Z = Znew
@@ -452,7 +460,7 @@ def _step_and_compare(mod, X, W1_0, p_gpu, p_or, tol, audit, gate=None):
     p_t.reselect_mask = False
     Zg = np64(mod.Z).T
     if p_t.z_rule == "exact" and p_t.act == "relu":
-        rep, A = _oracle_exact_step_adopting_ties(st, Xo, Yo, np64(W1_0), p_t, Zg, tol)
+        rep, A = _oracle_step_adopting_ties(st, Xo, Yo, np64(W1_0), p_t, Zg, tol)
     else:
         _, _, rep, A = O.admm_step(st, Xo, Yo, np64(W1_0), p_t)
     assert relerr(np64(mod.W1), st.W1) < tol, "W1"
@@ -720,13 +728,19 @@ def _free_run(cfg, iters, tol, growth, chunk=0):
         tau = np.sort(s_or)[::-1][cfg.k_keep - 1]
         assert np.all(np.abs(s_or[diff] - tau) <= 2 * e), ("near-tie audit", it)
         st.mask = mask_gpu.copy()
-        O.admm_step(st, Xo, Y, np64(W1), O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, reselect_mask=False))
+        # the literal select tests the sign of the old z, on which the two sides agree only up to their difference so far
+        z_gap = 2.0 * (rec[-1]["Z_abs"] if rec else tol * np.abs(st.Z).max())
+        _oracle_step_adopting_ties(st, Xo, Y, np64(W1), O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, reselect_mask=False),
+                                   np64(mod.Z).T, tol, sign_delta=z_gap)
         errs = dict(it=it, flipped=int(diff.size), scores=e / np.abs(s_or).max(), W1=relerr(np64(mod.W1), st.W1),
-                    W2=relerr(np64(mod.W2), st.W2), Z=relerr(np64(mod.Z).T, st.Z), G_A=relerr(np64(mod.G_A), st.G_A))
+                    W2=relerr(np64(mod.W2), st.W2), Z=relerr(np64(mod.Z).T, st.Z), G_A=relerr(np64(mod.G_A), st.G_A),
+                    Z_abs=float(np.abs(np64(mod.Z).T - st.Z).max()))
         print(errs)
         rec.append(errs)
+        errs["bound"] = bound
+    for errs in rec:
         for name in ("W1", "W2", "Z", "G_A"):
-            assert errs[name] <= bound, (name, it, errs[name])
+            assert errs[name] <= errs["bound"], (name, errs)
     return rec
 
 
@@ -742,4 +756,4 @@ def test_free_running_iterations_bf16(name, shape, iters):
     """Free-running iterations in bf16 mode on width- and token-reduced copies of the benchmark workload (half width)
     and of the widest one (quarter width, 80 % pruned, more channels than tokens)."""
     cfg = synth.scaled(synth.CONFIGS[name], **shape)
-    _free_run(cfg, iters, TOL[torch.bfloat16], lambda it: 1.0 + 0.5 * it, chunk=2048)
+    _free_run(cfg, iters, TOL[torch.bfloat16], lambda it: 5.0, chunk=2048)
