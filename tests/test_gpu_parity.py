@@ -370,7 +370,7 @@ NEAR_TIE_FRACTIONS = []
 NEAR_TIE_LIMIT = 0.005
 
 
-def _oracle_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol, sign_delta=0.0):
+def _oracle_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol, sign_delta=0.0, Zg_old=None):
     """The oracle's step composed here from the oracle's own parts so that the one elementwise decision that is not
     unique can be audited (z_rule = "exact" in every comparison; the literal rule only when the two sides run free and
     their old z differ, see sign_delta below).  The exact rule compares the objective values fn, fp of the best point of each half
@@ -404,7 +404,10 @@ def _oracle_step_adopting_ties(st, Xo, Yo, W1_0, p_t, Zg, tol, sign_delta=0.0):
     else:
         # literal rule of Algorithms 2 / 3: the sign of the OLD z decides.  When the two sides' old z differ by up to
         # sign_delta (free-running comparison), an entry with |z_old| <= sign_delta can fall on either side of zero.
-        amb = (np.abs(st.Z) <= sign_delta) & (z1 != z2)
+        # Only entries whose two old values actually lie on different sides of zero are adopted, and each of them must
+        # be within the two sides' distance of zero.
+        amb = ((Zg_old < 0.0) != (st.Z < 0.0)) & (z1 != z2) if Zg_old is not None else np.zeros(st.Z.shape, bool)
+        assert np.all(np.abs(st.Z[amb]) <= sign_delta)
         ca, cb = z1, z2
     frac = float(amb.mean())
     NEAR_TIE_FRACTIONS.append(frac)
@@ -694,7 +697,7 @@ def test_admm_step_argument_errors():
     assert e.value.code == 1
 
 
-def _free_run(cfg, iters, tol, growth, chunk=0):
+def _free_run(cfg, iters, tol, growth, chunk=0, weight_factor=1.0):
     """K iterations WITHOUT teacher forcing: the GPU module and the oracle each start from their own initialisation of
     the same inputs and never see each other's values again, except for (1) the stored target Ypre, which in bf16 mode
     is an INPUT of the loop rounded to the storage type, and (2) the integer decision: when the two masks of an
@@ -713,6 +716,8 @@ def _free_run(cfg, iters, tol, growth, chunk=0):
     p_gpu = api.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, token_chunk=chunk)
     rec = []
     for it in range(iters):
+        Zg_old = np64(mod.Z).T
+        z_gap = float(np.abs(Zg_old - st.Z).max())                   # how far apart the two old z are at most
         mod.sp_admm_step(p_gpu)
         torch.cuda.synchronize()
         mod.check_status()
@@ -729,9 +734,8 @@ def _free_run(cfg, iters, tol, growth, chunk=0):
         assert np.all(np.abs(s_or[diff] - tau) <= 2 * e), ("near-tie audit", it)
         st.mask = mask_gpu.copy()
         # the literal select tests the sign of the old z, on which the two sides agree only up to their difference so far
-        z_gap = 2.0 * (rec[-1]["Z_abs"] if rec else tol * np.abs(st.Z).max())
         _oracle_step_adopting_ties(st, Xo, Y, np64(W1), O.AdmmParams(k_keep=cfg.k_keep, rho=cfg.rho, reselect_mask=False),
-                                   np64(mod.Z).T, tol, sign_delta=z_gap)
+                                   np64(mod.Z).T, tol, sign_delta=z_gap, Zg_old=Zg_old)
         errs = dict(it=it, flipped=int(diff.size), scores=e / np.abs(s_or).max(), W1=relerr(np64(mod.W1), st.W1),
                     W2=relerr(np64(mod.W2), st.W2), Z=relerr(np64(mod.Z).T, st.Z), G_A=relerr(np64(mod.G_A), st.G_A),
                     Z_abs=float(np.abs(np64(mod.Z).T - st.Z).max()))
@@ -740,7 +744,8 @@ def _free_run(cfg, iters, tol, growth, chunk=0):
         errs["bound"] = bound
     for errs in rec:
         for name in ("W1", "W2", "Z", "G_A"):
-            assert errs[name] <= errs["bound"], (name, errs)
+            factor = weight_factor if name in ("W1", "W2") else 1.0
+            assert errs[name] <= factor * errs["bound"], (name, errs)
     return rec
 
 
@@ -756,4 +761,8 @@ def test_free_running_iterations_bf16(name, shape, iters):
     """Free-running iterations in bf16 mode on width- and token-reduced copies of the benchmark workload (half width)
     and of the widest one (quarter width, 80 % pruned, more channels than tokens)."""
     cfg = synth.scaled(synth.CONFIGS[name], **shape)
-    _free_run(cfg, iters, TOL[torch.bfloat16], lambda it: 5.0, chunk=2048)
+    # The auxiliary variables, accumulators and scores stay within the per-call tolerance over all iterations.  The
+    # recovered weights do not: each side solves with ITS OWN accumulators, which differ by up to the tolerance
+    # (bf16 operands of the token-axis products), and the regularised solve amplifies such a difference by the
+    # conditioning of G + rho I (outlier channels); measured 1.2 to 3.6 times the tolerance, bound 5 times.
+    _free_run(cfg, iters, TOL[torch.bfloat16], lambda it: 1.0, chunk=2048, weight_factor=5.0)
