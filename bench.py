@@ -54,6 +54,8 @@ def parse():
     ap.add_argument("--shard", default="modules", choices=["modules", "tokens"],
                     help="N > 1: every rank its own module (default, no collective), or ONE module with its tokens "
                          "split over the ranks (accumulators all-reduced once per iteration)")
+    ap.add_argument("--reproducible", action="store_true",
+                    help="run with sp_set_reproducible(1): fixed summation order, bit-identical results")
     ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
     ap.add_argument("--workloads", default="C3,C4,C5",
                     help="1 GPU: further workloads measured after the main one and reported under `workloads` "
@@ -372,6 +374,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     api.lib()
+    if args.reproducible:
+        api.sp_set_reproducible(True)
 
     # ---- inputs resident in HBM: this rank's module (layer index = rank), or its token shard of module 0
     by_tokens = args.shard == "tokens"
@@ -521,6 +525,7 @@ def main():
             "scaling": "strong" if by_tokens else "weak",
             "vs_baseline": None, "dtype": DTYPE_NAME[cfg.storage], "data": "synthetic",
             "config": {"workload": workload_name(cfg), "token_chunk": args.chunk, "dual_mode": bool(args.dual),
+                       "reproducible": bool(args.reproducible),
                        "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
                        "parallelism": (f"tokens x{world} of one module (accumulators all-reduced once per iteration)"
                                        if by_tokens else f"modules x{world} (independent, no collective)")},

@@ -24,6 +24,20 @@
  *   - Return value: SP_OK or an error detected on the host before any launch (argument / shape / alignment /
  *     workspace errors).  Numerical failures found on the device (non-positive Cholesky pivot, a bounded wait that
  *     ran out) are written to the caller's `status_dev[4]` = {code, index, aux, 0}; nothing traps or spins forever.
+ *   - Streams: a call is ordered on the caller's stream, but sp_admm_step, sp_admm_scores, sp_ridge_solve and
+ *     sp_linear_refit also fork independent parts (the two weight recoveries, the panels and trailing updates of a
+ *     factorisation, the z^(1) products) onto a few streams and events that the library creates once per device and
+ *     joins back to the caller's stream with events before the call's results are used (also when a call returns an
+ *     error after the fork).  That set is shared by all calls on a device: issue the calls of one device from one
+ *     host thread at a time.  Nothing else persists inside the library.
+ *   - Reproducibility: by default a product whose tile count leaves SMs idle is cut along K and its partial
+ *     products add up in C in an order that is not fixed, and the backward triangular solve adds updates from two
+ *     streams; fp32 results (accumulators, recovered weights, scores) can then differ in their last bits between two
+ *     runs on equal inputs, and a mask can differ at scores that tie within that rounding.  sp_set_reproducible(1)
+ *     switches both off (process-wide): every sum is then taken in an order fixed by the call's arguments and equal
+ *     inputs give bit-identical outputs, at a few per cent of the step time.  The fp32 mode (fp64 accumulation on the
+ *     CUDA cores, fp64 factorisation) and the score, statistics, report and selection kernels are reproducible either
+ *     way.
  *   - Symmetric accumulators (Gram matrices) are stored as full squares; calls that update them keep the LOWER
  *     triangle (including the diagonal) authoritative.  sp_symmetrize() mirrors it to the upper triangle.
  */
@@ -242,6 +256,15 @@ sp_status sp_struct_scores_static(int32_t kind, int32_t group, const sp_score_in
 sp_status sp_allocate_sparsity(const double* I, const int64_t* n_units, int32_t L, double rbar, double T, int32_t mode,
                                double clip_hi, double* r_out, int64_t* k_keep_out, void* stream);
 
+/* sp_allocate_sparsity_grid — the allocation above for a whole grid of temperatures in one launch (the outer loop of
+ * Algorithm 1 runs Step 2 once per temperature of its search grid).  T_list: fp64 [n_T] on the device; T_relative != 0:
+ * entry T_list[g] is given relative to the magnitude of the importances, T = T_list[g] * mean_l |I_l| (computed on the
+ * device; Section 4 scales the temperature to the importance scores).  r_out, k_keep_out: [n_T, L], row g for T_list[g].
+ * Errors as sp_allocate_sparsity, plus SP_ERR_SHAPE for n_T outside [1, 65535]. */
+sp_status sp_allocate_sparsity_grid(const double* I, const int64_t* n_units, int32_t L, double rbar, const double* T_list,
+                                    int32_t n_T, int32_t T_relative, int32_t mode, double clip_hi, double* r_out,
+                                    int64_t* k_keep_out, void* stream);
+
 /* ---------------------------------------------------------------------------------------------------------------
  * sp_apply_mask — top-k selection and M (.) W (Algorithm 1 Step 3; Algorithm 3 threshold and mask lines).
  * Keeps exactly k_keep units: the k largest scores, equal scores resolved toward the lower index, NaN lowest.
@@ -267,6 +290,27 @@ sp_status sp_apply_mask(const float* scores, int64_t n_units, int64_t k_keep, in
 sp_status sp_apply_mask_batched(const float* scores, int64_t ld_scores, int64_t n_units, int32_t L,
                                 const int64_t* k_keep, uint8_t* mask_out, int64_t ld_mask, float* tau_out,
                                 int32_t* kept_idx_out, int64_t ld_idx, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_apply_mask_global — the threshold step of Appendix B, Algorithm 3 (GSPO) over all L layers at once: the scores of
+ * all layers (row l at scores + l * ld_scores, n_units each) are collected, K = floor(keep_fraction * n_units * L),
+ * and the units holding the K largest scores are kept: one threshold for the whole model.  Exactly K units are kept
+ * (ties: the earlier layer, then the lower index; NaN lowest), unless min_keep > 0: a layer the threshold leaves with
+ * fewer than min_keep units keeps its own min_keep best instead (as printed the algorithm can empty a layer).
+ * mask_out: u8, row l at mask_out + l * ld_mask; tau_out (optional): the K-th largest score; kept_out: int64 [L] kept
+ * units per layer after the repair (device).  The select runs on many CTAs (four histogram passes over the keys), so
+ * L * n_units is not limited by one CTA's shared memory.  Workspace: sp_apply_mask_global_bytes(n_units, L).
+ * Errors: SP_ERR_INVALID_ARG (null pointers, keep_fraction outside [0, 1]), SP_ERR_SHAPE, SP_ERR_WORKSPACE,
+ * SP_ERR_ALIGNMENT (workspace not 256-byte aligned). */
+sp_status sp_apply_mask_global(const float* scores, int64_t ld_scores, int64_t n_units, int32_t L, double keep_fraction,
+                               int64_t min_keep, uint8_t* mask_out, int64_t ld_mask, float* tau_out,
+                               int64_t* kept_out, void* ws, size_t ws_bytes, void* stream);
+size_t sp_apply_mask_global_bytes(int64_t n_units, int32_t L);
+
+/* sp_objective_accumulate — Step 5 of Algorithm 1: loss_dev[0] (+)= L_l = res_out + beta * res_act + res_in of a step
+ * report (the FFN objective of Appendix A.1 after that step; needs compute_objective).  All pointers on the device. */
+sp_status sp_objective_accumulate(const sp_step_report* rep_dev, double beta, double* loss_dev, int32_t accumulate,
+                                  void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
  * sp_weight_stats, sp_distribute_importance — the weight-statistic importances of the "-distribute" variant of
@@ -379,6 +423,10 @@ sp_status sp_gemm(int32_t transA, int32_t transB, int64_t M, int64_t N, int64_t 
                   const sp_mat* B, double beta, const sp_mat* C, int32_t lower_only, int32_t use_tensor_cores,
                   int32_t* status_dev, void* stream);
 sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream);
+
+/* sp_set_reproducible(on): see "Reproducibility" at the top of this file; sp_get_reproducible() returns the setting. */
+sp_status sp_set_reproducible(int32_t on);
+int32_t sp_get_reproducible(void);
 
 /* ---------------------------------------------------------------------------------------------------------------
  * Launch accounting and profiling (the paper has no counterpart; used by the benchmark).

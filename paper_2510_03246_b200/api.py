@@ -29,7 +29,9 @@ EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_admm_scores"
            "sp_apply_mask", "sp_apply_mask_batched", "sp_weight_stats", "sp_distribute_importance",
            "sp_struct_scores_static", "sp_ridge_solve", "sp_linear_refit", "sp_gemm", "sp_symmetrize", "sp_workspace_bytes", "sp_admm_overlap_bytes",
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
-           "sp_profile_kind_name", "sp_launch_count", "sp_mha_init", "sp_mha_step", "sp_mha_workspace_bytes"]
+           "sp_profile_kind_name", "sp_launch_count", "sp_mha_init", "sp_mha_step", "sp_mha_workspace_bytes",
+           "sp_set_reproducible", "sp_get_reproducible", "sp_allocate_sparsity_grid", "sp_apply_mask_global",
+           "sp_apply_mask_global_bytes", "sp_objective_accumulate"]
 
 
 class SpError(RuntimeError):
@@ -122,6 +124,13 @@ def lib() -> C.CDLL:
         L.sp_mha_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, i32]
         L.sp_mha_init.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), i32, i64, vp, vp, sz, vp]
         L.sp_mha_step.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), C.POINTER(SpMhaParams), vp, vp, sz, vp]
+        L.sp_allocate_sparsity_grid.argtypes = [vp, vp, i32, dbl, vp, i32, i32, i32, dbl, vp, vp, vp]
+        L.sp_apply_mask_global.argtypes = [vp, i64, i64, i32, dbl, i64, vp, i64, vp, vp, vp, sz, vp]
+        L.sp_apply_mask_global_bytes.restype = C.c_size_t
+        L.sp_apply_mask_global_bytes.argtypes = [i64, i32]
+        L.sp_objective_accumulate.argtypes = [vp, dbl, vp, i32, vp]
+        L.sp_set_reproducible.argtypes = [i32]
+        L.sp_get_reproducible.restype = i32
         L.sp_profile_begin.argtypes = [i32]
         L.sp_profile_read.argtypes = [vp]
         L.sp_profile_kinds.restype = i32
@@ -129,7 +138,8 @@ def lib() -> C.CDLL:
         L.sp_profile_kind_name.argtypes = [i32]
         L.sp_launch_count.restype = i64
         for name in EXPORTS:
-            if name not in ("sp_workspace_bytes", "sp_admm_overlap_bytes", "sp_mha_workspace_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
+            if name not in ("sp_workspace_bytes", "sp_admm_overlap_bytes", "sp_mha_workspace_bytes",
+                            "sp_apply_mask_global_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
                             "sp_profile_kind_name", "sp_launch_count"):
                 getattr(L, name).restype = C.c_int32
         _lib = L
@@ -181,6 +191,11 @@ def _ws(nbytes: int, device) -> torch.Tensor:
 
 def new_status(device="cuda") -> torch.Tensor:
     return torch.zeros(4, dtype=torch.int32, device=device)
+
+
+def sp_set_reproducible(on: bool):
+    """Process-wide switch: fixed summation order everywhere (bit-identical results for equal inputs)."""
+    _check(lib().sp_set_reproducible(int(bool(on))), "sp_set_reproducible")
 
 
 def sp_profile_begin(enable=True):
@@ -305,6 +320,39 @@ def sp_allocate_sparsity(I, n_units, rbar, T, mode=SP_ALLOC_SOFTMAX, clip_hi=0.9
     _check(lib().sp_allocate_sparsity(I.data_ptr(), n_units.data_ptr(), L, float(rbar), float(T), mode,
                                       float(clip_hi), r.data_ptr(), k.data_ptr(), _stream()), "sp_allocate_sparsity")
     return r, k
+
+
+def sp_allocate_sparsity_grid(I, n_units, rbar, T_list, T_relative=True, mode=SP_ALLOC_SOFTMAX, clip_hi=0.95):
+    """Allocation for every temperature of T_list (fp64 [n_T] device) in one launch.  Returns (r [n_T, L], k_keep)."""
+    _require_cuda(I, n_units, T_list)
+    L, nT = I.numel(), T_list.numel()
+    r = torch.empty(nT, L, dtype=torch.float64, device=I.device)
+    k = torch.empty(nT, L, dtype=torch.int64, device=I.device)
+    _check(lib().sp_allocate_sparsity_grid(I.data_ptr(), n_units.data_ptr(), L, float(rbar), T_list.data_ptr(), nT,
+                                           int(bool(T_relative)), mode, float(clip_hi), r.data_ptr(), k.data_ptr(),
+                                           _stream()), "sp_allocate_sparsity_grid")
+    return r, k
+
+
+def sp_apply_mask_global(scores, keep_fraction, min_keep=0, mask_out=None):
+    """scores: fp32 [L, n] (rows contiguous).  Returns (mask u8 [L, n], tau fp32 [1], kept int64 [L])."""
+    _require_cuda(scores, mask_out)
+    L, n = scores.shape
+    mask = mask_out if mask_out is not None else torch.empty(L, n, dtype=torch.uint8, device=scores.device)
+    tau = torch.empty(1, dtype=torch.float32, device=scores.device)
+    kept = torch.empty(L, dtype=torch.int64, device=scores.device)
+    ws = _ws(lib().sp_apply_mask_global_bytes(n, L), scores.device)
+    _check(lib().sp_apply_mask_global(scores.data_ptr(), scores.stride(0), n, L, float(keep_fraction), int(min_keep),
+                                      mask.data_ptr(), mask.stride(0), tau.data_ptr(), kept.data_ptr(), ws.data_ptr(),
+                                      ws.numel(), _stream()), "sp_apply_mask_global")
+    return mask, tau, kept
+
+
+def sp_objective_accumulate(report, beta, loss, accumulate=True):
+    """loss[0] (+)= objective of the step report (device tensors)."""
+    _require_cuda(report, loss)
+    _check(lib().sp_objective_accumulate(report.data_ptr(), float(beta), loss.data_ptr(), int(bool(accumulate)),
+                                         _stream()), "sp_objective_accumulate")
 
 
 def sp_apply_mask(scores, k_keep, group=1, W_rows=None, W_cols=None, want_index=False, mask_out=None):

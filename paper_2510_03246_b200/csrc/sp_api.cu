@@ -539,6 +539,53 @@ sp_status sp_allocate_sparsity(const double* I, const int64_t* n_units, int32_t 
   return SP_OK;
 }
 
+sp_status sp_allocate_sparsity_grid(const double* I, const int64_t* n_units, int32_t L, double rbar, const double* T_list,
+                                    int32_t n_T, int32_t T_relative, int32_t mode, double clip_hi, double* r_out,
+                                    int64_t* k_keep_out, void* stream) {
+  if (!I || !n_units || !T_list || !r_out || !k_keep_out) return SP_ERR_INVALID_ARG;
+  if (L < 1 || L > 65536 || n_T < 1 || n_T > 65535) return SP_ERR_SHAPE;
+  if (!(rbar >= 0.0 && rbar <= 1.0) || !(clip_hi > 0.0 && clip_hi <= 1.0)) return SP_ERR_INVALID_ARG;
+  if (mode != SP_ALLOC_SOFTMAX && mode != SP_ALLOC_INVERSE && mode != SP_ALLOC_UNIFORM) return SP_ERR_UNSUPPORTED;
+  CU(allocate_sparsity_grid(I, n_units, L, rbar, T_list, n_T, T_relative != 0, mode, clip_hi, r_out, k_keep_out,
+                            reinterpret_cast<cudaStream_t>(stream)));
+  return SP_OK;
+}
+
+size_t sp_apply_mask_global_bytes(int64_t n_units, int32_t L) {
+  if (n_units < 0 || L < 0) return 0;
+  return global_select_scratch_bytes(n_units * (int64_t)L, L) + 256;
+}
+
+sp_status sp_apply_mask_global(const float* scores, int64_t ld_scores, int64_t n_units, int32_t L, double keep_fraction,
+                               int64_t min_keep, uint8_t* mask_out, int64_t ld_mask, float* tau_out,
+                               int64_t* kept_out, void* ws, size_t ws_bytes, void* stream) {
+  if (!scores || !mask_out || !kept_out) return SP_ERR_INVALID_ARG;
+  if (n_units < 0 || L < 0 || ld_scores < n_units || ld_mask < n_units || min_keep < 0) return SP_ERR_SHAPE;
+  if (!(keep_fraction >= 0.0 && keep_fraction <= 1.0)) return SP_ERR_INVALID_ARG;
+  if (n_units == 0 || L == 0) return SP_OK;
+  if (!ws || ws_bytes < sp_apply_mask_global_bytes(n_units, L)) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256)) return SP_ERR_ALIGNMENT;
+  // K = floor(r n L) of Algorithm 3; the small offset keeps products like 0.6 * 5 from falling below their integer
+  const int64_t K = (int64_t)floor(keep_fraction * (double)n_units * (double)L + 1e-9);
+  CU(global_select(scores, ld_scores, n_units, L, K, min_keep, mask_out, ld_mask, tau_out, kept_out, ws,
+                   reinterpret_cast<cudaStream_t>(stream)));
+  return SP_OK;
+}
+
+__global__ void objective_accumulate_kernel(const sp_step_report* rep, double beta, double* loss, int accumulate) {
+  const double v = rep->res_out + beta * rep->res_act + rep->res_in;
+  loss[0] = accumulate ? loss[0] + v : v;
+}
+
+sp_status sp_objective_accumulate(const sp_step_report* rep_dev, double beta, double* loss_dev, int32_t accumulate,
+                                  void* stream) {
+  if (!rep_dev || !loss_dev) return SP_ERR_INVALID_ARG;
+  count_launch();
+  objective_accumulate_kernel<<<1, 1, 0, reinterpret_cast<cudaStream_t>(stream)>>>(rep_dev, beta, loss_dev, accumulate);
+  CU(cudaGetLastError());
+  return SP_OK;
+}
+
 sp_status sp_apply_mask(const float* scores, int64_t n_units, int64_t k_keep, int32_t group, uint8_t* mask_out,
                         float* tau_out, int32_t* kept_idx_out, const sp_mat* W_rows, const sp_mat* W_cols, void* ws,
                         size_t ws_bytes, void* stream) {

@@ -28,6 +28,9 @@ enum ProfKind : int {
   PK_COUNT = 12
 };
 void count_launch(int n = 1);
+// sp_set_reproducible: when on, every floating-point sum of the library is taken in an order fixed by the call's
+// arguments (no product is cut along K, the triangular solves run on one stream), so equal inputs give equal bits.
+bool reproducible_mode();
 // Brackets the kernels launched during its lifetime with a CUDA event pair on `stream` when profiling is enabled.
 // Scopes nest: only the outermost one records, so a phase scope absorbs the kernels launched inside it.
 struct ProfScope {
@@ -309,7 +312,18 @@ cudaError_t topk_select(const float* scores, int64_t n, int64_t k, uint8_t* mask
 // `batch` independent problems in one launch (one block each); k_list (device, may be nullptr) overrides k_all.
 cudaError_t topk_select_batched(const float* scores, int64_t ld_scores, int64_t n, int64_t batch, int64_t k_all,
                                 const int64_t* k_list, uint8_t* mask, int64_t ld_mask, float* tau, int32_t* kept_idx,
-                                int64_t ld_idx, cudaStream_t stream);
+                                int64_t ld_idx, cudaStream_t stream, bool skip_negative = false);
+// allocation for a grid of n_T temperatures in one launch: T_list (device), relative to mean |I| when T_relative;
+// r_out / k_out are [n_T, L]
+cudaError_t allocate_sparsity_grid(const double* I, const int64_t* n_units, int L, double rbar, const double* T_list,
+                                   int n_T, bool T_relative, int mode, double clip_hi, double* r_out, int64_t* k_out,
+                                   cudaStream_t stream);
+// one threshold over the L x n scores (rows ld_scores apart): the K largest kept (ties: earlier layer, lower index),
+// a layer left with fewer than min_keep units keeps its own min_keep best; counts_out[l] = kept units of layer l
+size_t global_select_scratch_bytes(int64_t total, int L);
+cudaError_t global_select(const float* scores, int64_t ld_scores, int64_t n, int L, int64_t K, int64_t min_keep,
+                          uint8_t* mask, int64_t ld_mask, float* tau, int64_t* counts_out, void* scratch,
+                          cudaStream_t stream);
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream);
 cudaError_t zero_pruned(const uint8_t* mask, int group, float* W_rows, int64_t r_rows, int64_t r_cols, int64_t r_ld,
                         float* W_cols, int64_t c_rows, int64_t c_cols, int64_t c_ld, cudaStream_t stream);

@@ -274,10 +274,11 @@ __device__ __forceinline__ uint32_t make_instr_desc(bool a_kmajor, bool b_kmajor
   return d;
 }
 
+template <bool BATCHED>
 __device__ __forceinline__ void tile_coords(const TcParams& p, int t, int& tm, int& tn, int& b0, int& b1) {
   b0 = 0;
   b1 = 0;
-  if (p.batched) {
+  if constexpr (BATCHED) {
     const int bi = t / p.tiles_per_batch;
     t -= bi * p.tiles_per_batch;
     b0 = bi % p.nb0;
@@ -318,6 +319,10 @@ __device__ __forceinline__ void tc_commit_local(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// BATCHED = false is the plain two-dimensional form (the products of the FFN path); BATCHED = true adds the batch
+// and plane coordinates (five-dimensional tensor maps).  Two instantiations, so that the plain form carries none of
+// the batched form's instructions.
+template <bool BATCHED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmCin, const TcParams p) {
@@ -377,7 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int u = cid; u < p.num_units && ok; u += ncl) {
         int tm, tn, tile, kb0, kb1, b0, b1;
         unit_map(p, u, num_kb, tile, kb0, kb1);
-        tile_coords(p, tile, tm, tn, b0, b1);
+        tile_coords<BATCHED>(p, tile, tm, tn, b0, b1);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
           // the leader's barrier collects the bytes of both CTAs' loads of this stage
@@ -390,7 +395,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const int ka = kk + p.seg.a_k[sg], kbb = kk + p.seg.b_k[sg];
           const int am = tm * TILE_M + (int)rank * BM + p.seg.a_mn[sg];
           const int bn = tn * TILE_N + (int)rank * BNH + p.seg.b_mn[sg];
-          if (p.batched) {
+          if constexpr (BATCHED) {
             const int pa = p.seg.a_p[sg], pb = p.seg.b_p[sg];
             if (p.a_kmajor) {
               tma_load_5d(a_dst, &tmA, make_coord(p.a_ord, ka, am, b0, b1, pa), fbar);
@@ -406,18 +411,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               for (int nb = 0; nb < BNH / 64; ++nb)
                 tma_load_5d(b_dst + nb * (64 * BK * 2), &tmB, make_coord(p.b_ord, bn + nb * 64, kbb, b0, b1, pb), fbar);
             }
-          } else if (p.a_kmajor) {
-            tma_load_2d(a_dst, &tmA, ka, am, fbar);
           } else {
+            if (p.a_kmajor) {
+              tma_load_2d(a_dst, &tmA, ka, am, fbar);
+            } else {
 #pragma unroll
-            for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, am + mb * 64, ka, fbar);
-          }
-          if (p.batched) {
-          } else if (p.b_kmajor) {
-            tma_load_2d(b_dst, &tmB, kbb, bn, fbar);
-          } else {
+              for (int mb = 0; mb < BM / 64; ++mb) tma_load_2d(a_dst + mb * (64 * BK * 2), &tmA, am + mb * 64, ka, fbar);
+            }
+            if (p.b_kmajor) {
+              tma_load_2d(b_dst, &tmB, kbb, bn, fbar);
+            } else {
 #pragma unroll
-            for (int nb = 0; nb < BNH / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, bn + nb * 64, kbb, fbar);
+              for (int nb = 0; nb < BNH / 64; ++nb) tma_load_2d(b_dst + nb * (64 * BK * 2), &tmB, bn + nb * 64, kbb, fbar);
+            }
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -494,9 +500,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     for (int u = cid; u < p.num_units && ok; u += ncl) {
       int tm, tn, tile, kb0_unused, kb1_unused, b0, b1;
       unit_map(p, u, num_kb, tile, kb0_unused, kb1_unused);
-      tile_coords(p, tile, tm, tn, b0, b1);
-      const int64_t c_boff = (int64_t)b0 * p.c_s0 + (int64_t)b1 * p.c_s1;
-      const int64_t cin_boff = (int64_t)b0 * p.cin_s0 + (int64_t)b1 * p.cin_s1;
+      tile_coords<BATCHED>(p, tile, tm, tn, b0, b1);
+      const int64_t c_boff = BATCHED ? (int64_t)b0 * p.c_s0 + (int64_t)b1 * p.c_s1 : 0;
+      const int64_t cin_boff = BATCHED ? (int64_t)b0 * p.cin_s0 + (int64_t)b1 * p.cin_s1 : 0;
       // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
       const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
@@ -585,14 +591,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           __syncwarp();
           if (lane == 0) {
             if (rows_here > 0) {
-              if (p.batched) {
+              if constexpr (BATCHED) {
                 const Coord5 cc = make_coord(p.c_ord, (int32_t)gj0, (int32_t)row0, b0, b1, 0);
                 if (p.epi_mode == EPI_TMA_STORE) tma_store_5d(&tmC, cc, wstg + buf * 4096);
                 else tma_reduce_add_5d(&tmC, cc, wstg + buf * 4096);
-              } else if (p.epi_mode == EPI_TMA_STORE) {
-                tma_store_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
               } else {
-                tma_reduce_add_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+                if (p.epi_mode == EPI_TMA_STORE) tma_store_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
+                else tma_reduce_add_2d(&tmC, (int32_t)gj0, (int32_t)row0, wstg + buf * 4096);
               }
             }
             bulk_commit();
@@ -901,7 +906,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   if (max_pairs > 0 && max_pairs < pairs_max) pairs_max = max_pairs;
   const int num_kb = p.seg_kb * sg.nseg;
   p.ksplit = 1;
-  if (!batched && (p.epi_mode == EPI_TMA_STORE || p.epi_mode == EPI_TMA_ADD) && p.num_tiles > 0) {
+  const bool may_cut = !batched && !reproducible_mode();   // partial products of a cut tile add in no fixed order
+  if (may_cut && (p.epi_mode == EPI_TMA_STORE || p.epi_mode == EPI_TMA_ADD) && p.num_tiles > 0) {
     auto eff = [&](int ks) {
       const double u = (double)p.num_tiles * ks;
       return u / (ceil(u / pairs_max) * pairs_max);
@@ -919,7 +925,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
     }
   }
   p.n_plain = 0;
-  if (!batched && p.epi_mode == EPI_TMA_ADD && p.num_tiles > pairs_max && p.num_tiles % pairs_max != 0) {
+  if (may_cut && p.epi_mode == EPI_TMA_ADD && p.num_tiles > pairs_max && p.num_tiles % pairs_max != 0) {
     // Alternative: whole waves of uncut tiles, and only the tiles of the last wave cut, as many ways as pairs are
     // left per tile.  Times in units of one tile on one pair.
     const int full = p.num_tiles / pairs_max, rem = p.num_tiles % pairs_max;
@@ -939,7 +945,11 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
 
   static PerDeviceOnce attr_once;
   if (attr_once.run([] {
-        return cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)SMEM_BYTES);
+        if (e == cudaSuccess)
+          e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        return e;
       }) != cudaSuccess)
     return SP_ERR_CUDA;
   count_launch();
@@ -947,7 +957,8 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
                                         : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K * p.nb0 * p.nb1;
   ProfScope prof(max_pairs > 0 ? PK_GEMM_TC_SHARED : PK_GEMM_TC, flops, 0.0, stream);
   const int pairs = p.num_units < pairs_max ? p.num_units : pairs_max;
-  gemm_tc_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);
+  if (batched) gemm_tc_kernel<true><<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);
+  else gemm_tc_kernel<false><<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);
   return cudaGetLastError() == cudaSuccess ? SP_OK : SP_ERR_CUDA;
 }
 

@@ -758,6 +758,9 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
   // without it everything stays on one stream.
   const bool x_al16 = (ldx % 4 == 0) && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0);
   if (!x_al16) assist = nullptr;
+  // Reproducible mode: the far update of a step (assisting stream) and the next step's near update would add into the
+  // same columns in an order that depends on timing; on one stream every column receives its updates in step order.
+  if (reproducible_mode()) assist = nullptr;
   // Backward sweep: the update of the next block column can ride in the panel kernel (fp32, from the fp32 factor)
   // when the factor's rows are 16-byte aligned too.
   // (its 144 KB of shared memory allow one CTA per SM: only while all row blocks fit in one wave)

@@ -536,11 +536,21 @@ __global__ void __launch_bounds__(1024) mean_scores_kernel(const float* scores, 
 }
 
 // ------------------------------------------------------------------------------------------------ allocation
+// One block per temperature of a grid (blockIdx.x): T = T_list[b] (T_list != nullptr) or the scalar T, multiplied by
+// mean_l |I_l| when T_relative; outputs row b of r_out / k_out ([grid, L]).
 __global__ void __launch_bounds__(1024) allocate_kernel(const double* I, const int64_t* n_units, int L, double rbar,
-                                                        double T, int mode, double clip_hi, double* r_out,
-                                                        int64_t* k_out) {
+                                                        double T, const double* T_list, int T_relative, int mode,
+                                                        double clip_hi, double* r_out, int64_t* k_out) {
   __shared__ double sm[33];
   const int t = threadIdx.x;
+  r_out += (int64_t)blockIdx.x * L;
+  k_out += (int64_t)blockIdx.x * L;
+  if (T_list) T = T_list[blockIdx.x];
+  if (T_relative) {
+    double a = 0.0;
+    for (int l = t; l < L; l += blockDim.x) a += fabs(I[l]);
+    T *= block_sum_bcast(a, sm) / (double)L;
+  }
   if (mode == SP_ALLOC_UNIFORM) {
     for (int l = t; l < L; l += blockDim.x) r_out[l] = rbar;
   } else {
@@ -658,7 +668,8 @@ __device__ int2 block_excl_scan2(int a, int b, int2* warp_tot, int2* total) {
 __global__ void __launch_bounds__(1024) topk_select_kernel(const float* __restrict__ scores_all, int64_t ld_scores,
                                                            int64_t n, int64_t k_all, const int64_t* k_list,
                                                            uint8_t* mask_all, int64_t ld_mask, float* tau_all,
-                                                           int32_t* kept_all, int64_t ld_idx, int smem_keys) {
+                                                           int32_t* kept_all, int64_t ld_idx, int smem_keys,
+                                                           int skip_negative) {
   extern __shared__ uint32_t s_keys[];
   __shared__ int hist_w[32][256];     // one histogram per warp: adds collide only inside a warp
   __shared__ int hist[256];
@@ -672,6 +683,7 @@ __global__ void __launch_bounds__(1024) topk_select_kernel(const float* __restri
   float* tau = tau_all ? tau_all + prob : nullptr;
   int32_t* kept_idx = kept_all ? kept_all + prob * ld_idx : nullptr;
   int64_t k = k_list ? k_list[prob] : k_all;
+  if (k < 0 && skip_negative) return;      // this problem keeps the mask it has
   if (k < 0) k = 0;
   if (k <= 0 || k >= n) {
     for (int64_t i = t; i < n; i += blockDim.x) {
@@ -996,7 +1008,17 @@ cudaError_t allocate_sparsity(const double* I, const int64_t* n_units, int L, do
                               double clip_hi, double* r_out, int64_t* k_out, cudaStream_t stream) {
   ProfScope prof(PK_ALLOCATE, 0.0, (double)L * 32.0, stream);
   count_launch();
-  allocate_kernel<<<1, 1024, 0, stream>>>(I, n_units, L, rbar, T, mode, clip_hi, r_out, k_out);
+  allocate_kernel<<<1, 1024, 0, stream>>>(I, n_units, L, rbar, T, nullptr, 0, mode, clip_hi, r_out, k_out);
+  return cudaGetLastError();
+}
+
+cudaError_t allocate_sparsity_grid(const double* I, const int64_t* n_units, int L, double rbar, const double* T_list,
+                                   int n_T, bool T_relative, int mode, double clip_hi, double* r_out, int64_t* k_out,
+                                   cudaStream_t stream) {
+  ProfScope prof(PK_ALLOCATE, 0.0, (double)L * 32.0 * n_T, stream);
+  count_launch();
+  allocate_kernel<<<n_T, 1024, 0, stream>>>(I, n_units, L, rbar, 1.0, T_list, T_relative ? 1 : 0, mode, clip_hi, r_out,
+                                            k_out);
   return cudaGetLastError();
 }
 
@@ -1008,7 +1030,7 @@ cudaError_t topk_select(const float* scores, int64_t n, int64_t k, uint8_t* mask
 
 cudaError_t topk_select_batched(const float* scores, int64_t ld_scores, int64_t n, int64_t batch, int64_t k_all,
                                 const int64_t* k_list, uint8_t* mask, int64_t ld_mask, float* tau, int32_t* kept_idx,
-                                int64_t ld_idx, cudaStream_t stream) {
+                                int64_t ld_idx, cudaStream_t stream, bool skip_negative) {
   if (n == 0 || batch == 0) return cudaSuccess;
   constexpr int64_t kMaxSmemKeys = 47104;      // 184 KiB of keys beside the 33 KiB of histograms
   static PerDeviceOnce attr_once;
@@ -1021,8 +1043,222 @@ cudaError_t topk_select_batched(const float* scores, int64_t ld_scores, int64_t 
   ProfScope prof(PK_TOPK, 0.0, (double)batch * (double)n * 5.0, stream);
   count_launch();
   topk_select_kernel<<<(unsigned)batch, 1024, smem_keys ? (size_t)n * sizeof(uint32_t) : 0, stream>>>(
-      scores, ld_scores, n, k_all, k_list, mask, ld_mask, tau, kept_idx, ld_idx, smem_keys);
+      scores, ld_scores, n, k_all, k_list, mask, ld_mask, tau, kept_idx, ld_idx, smem_keys, skip_negative ? 1 : 0);
   return cudaGetLastError();
+}
+
+__global__ void fill_i32_kernel(int32_t* x, int n, int32_t v) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) x[i] = v;
+}
+
+// ---- one threshold over L * n scores with many CTAs (Appendix B, Algorithm 3): radix select in four launches, each a
+// grid-wide histogram of one key byte whose last block picks the bin; then the eq / gt counts per block, and the mask.
+// state (device, ints): [0..255] histogram, [256] prefix, [257..258] remaining count (lo, hi), [259] ticket,
+// [260 + b] per-block count of keys equal to the threshold key (then their exclusive prefix).
+constexpr int kGselThreads = 256;
+constexpr int kGselPerBlock = 8192;          // keys per block
+constexpr int kGselState = 260;
+
+__global__ void gsel_init_kernel(int32_t* st, int64_t K, int nblocks) {
+  for (int i = threadIdx.x; i < kGselState + nblocks; i += blockDim.x) st[i] = 0;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    st[257] = (int32_t)(K & 0xffffffffll);
+    st[258] = (int32_t)(K >> 32);
+  }
+}
+
+__global__ void __launch_bounds__(kGselThreads) gsel_hist_kernel(const float* __restrict__ scores, int64_t n_row,
+                                                                 int64_t ld, int64_t total, int pass, int32_t* st) {
+  __shared__ int hist[256];
+  __shared__ bool last;
+  const int t = threadIdx.x;
+  hist[t] = 0;
+  __syncthreads();
+  const int shift = 24 - 8 * pass;
+  const uint32_t hi_mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+  const uint32_t prefix = (uint32_t)st[256];
+  const int64_t e0 = (int64_t)blockIdx.x * kGselPerBlock;
+  const int64_t e1 = e0 + kGselPerBlock < total ? e0 + kGselPerBlock : total;
+  for (int64_t e = e0 + t; e < e1; e += kGselThreads) {
+    const uint32_t key = score_key(scores[(e / n_row) * ld + e % n_row]);
+    if ((key & hi_mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xffu], 1);
+  }
+  __syncthreads();
+  if (hist[t]) atomicAdd(&st[t], hist[t]);
+  __threadfence();
+  __syncthreads();
+  if (t == 0) last = atomicAdd(&st[259], 1) == (int)gridDim.x - 1;
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  // the last block: pick the bin that holds the K-th largest key among those matching the prefix
+  hist[t] = __ldcg(&st[t]);
+  __syncthreads();
+  if (t == 0) {
+    int64_t rem = ((int64_t)(uint32_t)st[257]) | ((int64_t)st[258] << 32);
+    int bin = 0;
+    for (int b = 255; b >= 0; --b) {
+      if ((int64_t)hist[b] >= rem) { bin = b; break; }
+      rem -= hist[b];
+    }
+    st[256] = (int32_t)(prefix | ((uint32_t)bin << shift));
+    st[257] = (int32_t)(rem & 0xffffffffll);
+    st[258] = (int32_t)(rem >> 32);
+    st[259] = 0;
+  }
+  __syncthreads();
+  st[t] = 0;     // histogram of the next pass
+}
+
+// per-block counts of keys equal to the threshold key; the last block turns them into exclusive prefixes
+__global__ void __launch_bounds__(kGselThreads) gsel_count_kernel(const float* __restrict__ scores, int64_t n_row,
+                                                                  int64_t ld, int64_t total, int32_t* st) {
+  __shared__ int cnt;
+  __shared__ bool last;
+  const int t = threadIdx.x;
+  if (t == 0) cnt = 0;
+  __syncthreads();
+  const uint32_t tkey = (uint32_t)st[256];
+  const int64_t e0 = (int64_t)blockIdx.x * kGselPerBlock;
+  const int64_t e1 = e0 + kGselPerBlock < total ? e0 + kGselPerBlock : total;
+  int c = 0;
+  for (int64_t e = e0 + t; e < e1; e += kGselThreads) c += score_key(scores[(e / n_row) * ld + e % n_row]) == tkey;
+  if (c) atomicAdd(&cnt, c);
+  __syncthreads();
+  if (t == 0) {
+    st[kGselState + blockIdx.x] = cnt;
+    __threadfence();
+    last = atomicAdd(&st[259], 1) == (int)gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
+  if (t == 0) {
+    int run = 0;
+    for (unsigned b = 0; b < gridDim.x; ++b) {
+      const int v = __ldcg(&st[kGselState + b]);
+      st[kGselState + b] = run;
+      run += v;
+    }
+    st[259] = 0;
+  }
+}
+
+// mask: keys above the threshold key are kept, equal keys in (layer, index) order until the remaining count is used up
+// (a block walks its keys in order: thread t owns a contiguous run).  counts[l] += kept units of layer l.
+__global__ void __launch_bounds__(kGselThreads) gsel_mask_kernel(const float* __restrict__ scores, int64_t n_row,
+                                                                 int64_t ld, int64_t ld_mask, int64_t total,
+                                                                 const int32_t* st, uint8_t* mask, float* tau,
+                                                                 int32_t* counts) {
+  __shared__ int warp_tot[32];
+  const int t = threadIdx.x;
+  const uint32_t tkey = (uint32_t)st[256];
+  const int64_t take_eq = ((int64_t)(uint32_t)st[257]) | ((int64_t)st[258] << 32);
+  const int64_t eq_before_block = st[kGselState + blockIdx.x];
+  const int64_t e0 = (int64_t)blockIdx.x * kGselPerBlock;
+  const int64_t e1 = e0 + kGselPerBlock < total ? e0 + kGselPerBlock : total;
+  constexpr int per = kGselPerBlock / kGselThreads;
+  const int64_t i0 = e0 + (int64_t)t * per, i1 = (i0 + per < e1) ? i0 + per : e1;
+  int n_eq = 0;
+  for (int64_t e = i0; e < i1; ++e) n_eq += score_key(scores[(e / n_row) * ld + e % n_row]) == tkey;
+  // exclusive scan of n_eq over the block
+  const int lane = t & 31, w = t >> 5;
+  int incl = n_eq;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) warp_tot[w] = incl;
+  __syncthreads();
+  int base = 0;
+  for (int i = 0; i < w; ++i) base += warp_tot[i];
+  int64_t eq_seen = eq_before_block + base + incl - n_eq;
+  int kept_here = 0;
+  int64_t cur_layer = i0 < i1 ? i0 / n_row : 0;
+  for (int64_t e = i0; e < i1; ++e) {
+    const int64_t l = e / n_row, j = e % n_row;
+    if (l != cur_layer) {
+      if (kept_here) atomicAdd(&counts[cur_layer], kept_here);
+      kept_here = 0;
+      cur_layer = l;
+    }
+    const float v = scores[l * ld + j];
+    const uint32_t key = score_key(v);
+    const bool is_eq = key == tkey;
+    const bool keep = key > tkey || (is_eq && eq_seen < take_eq);
+    mask[l * ld_mask + j] = (uint8_t)keep;
+    kept_here += keep;
+    if (is_eq) {
+      if (eq_seen == 0 && tau) tau[0] = v != v ? -INFINITY : v;
+      ++eq_seen;
+    }
+  }
+  if (kept_here) atomicAdd(&counts[cur_layer], kept_here);
+}
+
+// layers left with fewer than min_keep units keep their own min_keep best: k_fix[l] = min_keep there, -1 elsewhere
+__global__ void gsel_repair_list_kernel(int32_t* counts, int L, int64_t min_keep, int64_t n_row, int64_t* k_fix,
+                                        int64_t* counts_out) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= L) return;
+  const int64_t mk = min_keep < n_row ? min_keep : n_row;
+  const bool fix = counts[l] < mk;
+  k_fix[l] = fix ? mk : -1;
+  counts_out[l] = fix ? mk : counts[l];
+}
+
+size_t global_select_scratch_bytes(int64_t total, int L) {
+  const int64_t nblocks = ceil_div(total > 0 ? total : 1, (int64_t)kGselPerBlock);
+  return align_up((size_t)(kGselState + nblocks) * 4, 256) + align_up((size_t)L * 4, 256) + align_up((size_t)L * 8, 256);
+}
+
+cudaError_t global_select(const float* scores, int64_t ld_scores, int64_t n, int L, int64_t K, int64_t min_keep,
+                          uint8_t* mask, int64_t ld_mask, float* tau, int64_t* counts_out, void* scratch,
+                          cudaStream_t stream) {
+  const int64_t total = (int64_t)L * n;
+  if (total == 0) return cudaSuccess;
+  const int nblocks = (int)ceil_div(total, (int64_t)kGselPerBlock);
+  uint8_t* sp8 = reinterpret_cast<uint8_t*>(scratch);
+  int32_t* st = reinterpret_cast<int32_t*>(sp8);
+  int32_t* counts = reinterpret_cast<int32_t*>(sp8 + align_up((size_t)(kGselState + nblocks) * 4, 256));
+  int64_t* k_fix = reinterpret_cast<int64_t*>(reinterpret_cast<uint8_t*>(counts) + align_up((size_t)L * 4, 256));
+  ProfScope prof(PK_TOPK, 0.0, (double)total * 25.0, stream);
+  cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)L * 4, stream);
+  if (e != cudaSuccess) return e;
+  if (K <= 0 || K >= total) {      // nothing or everything kept: no threshold to find
+    e = cudaMemset2DAsync(mask, (size_t)ld_mask, K > 0 ? 1 : 0, (size_t)n, (size_t)L, stream);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    gsel_init_kernel<<<1, 256, 0, stream>>>(st, 0, nblocks);
+    // counts = n or 0 per layer through the repair list below
+    e = cudaMemsetAsync(counts, 0, (size_t)L * 4, stream);
+    if (e != cudaSuccess) return e;
+    if (K > 0) {
+      count_launch();
+      fill_i32_kernel<<<(L + 255) / 256, 256, 0, stream>>>(counts, L, (int32_t)n);
+    }
+    if (tau) {
+      e = cudaMemsetAsync(tau, 0xff, sizeof(float), stream);       // NaN: no threshold
+      if (e != cudaSuccess) return e;
+    }
+  } else {
+    count_launch(7);
+    gsel_init_kernel<<<1, 256, 0, stream>>>(st, K, nblocks);
+    for (int pass = 0; pass < 4; ++pass)
+      gsel_hist_kernel<<<nblocks, kGselThreads, 0, stream>>>(scores, n, ld_scores, total, pass, st);
+    gsel_count_kernel<<<nblocks, kGselThreads, 0, stream>>>(scores, n, ld_scores, total, st);
+    gsel_mask_kernel<<<nblocks, kGselThreads, 0, stream>>>(scores, n, ld_scores, ld_mask, total, st, mask, tau, counts);
+  }
+  count_launch();
+  gsel_repair_list_kernel<<<(L + 255) / 256, 256, 0, stream>>>(counts, L, min_keep, n, k_fix, counts_out);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (min_keep > 0)   // per-layer top-k where the threshold left too few units (layers with k_fix < 0 are skipped)
+    e = topk_select_batched(scores, ld_scores, n, L, 0, k_fix, mask, ld_mask, nullptr, nullptr, 0, stream, true);
+  return e;
 }
 
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream) {

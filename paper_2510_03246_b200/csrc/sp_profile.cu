@@ -14,12 +14,15 @@ struct Slot {
   double flops, bytes;
 };
 std::atomic<long long> g_launches{0};
+std::atomic<int> g_reproducible{0};
 int g_enabled = 0;   // 0 off, 1 outermost scopes only, 2 every scope (nested ones are then counted twice)
 std::vector<Slot> g_slots;
 int g_used = 0;
 thread_local int g_depth = 0;
 
 }  // namespace
+
+bool reproducible_mode() { return g_reproducible.load(std::memory_order_relaxed) != 0; }
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -46,6 +49,12 @@ ProfScope::~ProfScope() {
 }  // namespace sp
 
 extern "C" {
+
+sp_status sp_set_reproducible(int32_t on) {
+  sp::g_reproducible.store(on ? 1 : 0);
+  return SP_OK;
+}
+int32_t sp_get_reproducible(void) { return sp::g_reproducible.load(); }
 
 int64_t sp_launch_count(void) { return (int64_t)sp::g_launches.load(); }
 

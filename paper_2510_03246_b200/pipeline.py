@@ -33,6 +33,7 @@ class LayerResult:
     W1: torch.Tensor              # fp32 [n, d]
     W2: torch.Tensor              # fp32 [d, n]
     reports: list = field(default_factory=list)
+    last_report: torch.Tensor | None = None    # device copy of the last step's report
 
 
 def layer_importance(X, W1_0, W2_0, score_kind=api.SP_SCORE_WANDA_L2, token_chunk=0) -> float:
@@ -50,25 +51,36 @@ def layer_importance(X, W1_0, W2_0, score_kind=api.SP_SCORE_WANDA_L2, token_chun
     return float(imp.item())
 
 
+def layer_importances(layer_inputs, n_layers, score_kind=api.SP_SCORE_WANDA_L2, token_chunk=0, device="cuda"):
+    """Step 1 of Algorithm 1 for all layers (each rank its own, then gathered): fp64 [n_layers] on the device."""
+    rank, _, world = parallel.env_world()
+    local = {}
+    for l in parallel.layers_of_rank(n_layers, rank, world):
+        X, W1_0, W2_0 = layer_inputs(l)
+        local[l] = layer_importance(X, W1_0, W2_0, score_kind, token_chunk)
+    return parallel.gather_importances(local, n_layers, device=device).to(device)
+
+
 def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_units: int, rbar: float, iters: int,
                      params: api.AdmmParams | None = None, T_rel: float = 1.0, alloc_mode=api.SP_ALLOC_SOFTMAX,
-                     token_chunk: int = 0, device="cuda"):
+                     token_chunk: int = 0, device="cuda", planned=None):
     """Runs Algorithm 1 over `n_layers` FFN modules.  layer_inputs(l) returns (X [N, d], W1_0 [n, d], W2_0 [d, n]) on the
-    device for layer l.  Returns (results of the layers this rank owns, r per layer, kept counts per layer, timings)."""
+    device for layer l.  planned = (I_all, r, k_keep) skips Steps 1 and 2 (the outer temperature loop computes the
+    importances once and the allocations of its whole grid in one launch).
+    Returns (results of the layers this rank owns, r per layer, kept counts per layer, timings)."""
     rank, _, world = parallel.env_world()
     mine = parallel.layers_of_rank(n_layers, rank, world)
     p = params or api.AdmmParams()
     t0 = time.perf_counter()
-    # Step 1
-    local = {}
-    for l in mine:
-        X, W1_0, W2_0 = layer_inputs(l)
-        local[l] = layer_importance(X, W1_0, W2_0, p.score_kind, token_chunk)
-    I_all = parallel.gather_importances(local, n_layers, device=device)
-    # Step 2 (the temperature is given relative to the magnitude of the importances)
-    T = T_rel * float(I_all.abs().mean())
-    nu = torch.full((n_layers,), n_units, dtype=torch.int64, device=device)
-    r, k_keep = api.sp_allocate_sparsity(I_all.to(device), nu, rbar, T, alloc_mode)
+    if planned is None:
+        I_all = layer_importances(layer_inputs, n_layers, p.score_kind, token_chunk, device)       # Step 1
+        # Step 2 (the temperature is given relative to the magnitude of the importances; the library scales it)
+        nu = torch.full((n_layers,), n_units, dtype=torch.int64, device=device)
+        T_list = torch.tensor([float(T_rel)], dtype=torch.float64, device=device)
+        r, k_keep = api.sp_allocate_sparsity_grid(I_all, nu, rbar, T_list, True, alloc_mode)
+        r, k_keep = r[0], k_keep[0]
+    else:
+        I_all, r, k_keep = planned
     k_host = k_keep.cpu().tolist()
     t1 = time.perf_counter()
     # Steps 3 and 4
@@ -85,6 +97,7 @@ def prune_ffn_layers(layer_inputs: Callable[[int], tuple], n_layers: int, n_unit
             res.reports.append(mod.report.clone())
         mod.check_status()
         res.mask, res.W1, res.W2 = mod.mask.clone(), mod.W1.clone(), mod.W2.clone()
+        res.last_report = res.reports[-1] if res.reports else None
         res.reports = [dict(zip(api.REPORT_FIELDS, t.cpu().tolist())) for t in res.reports]
         results.append(res)
         del mod
@@ -114,18 +127,14 @@ def prune_ffn_layers_global(layer_inputs: Callable[[int], tuple], n_layers: int,
                             scores=scores[l], mask=masks[l], ws_pool=pool)
         mod.sp_ffn_init()
         mods.append(mod)
-    K = int(keep_fraction * n * L + 1e-9)
     results = [LayerResult(l, float("nan"), 0, None, None, None) for l in range(L)]
     p_scores = api.AdmmParams(**{**p.__dict__, "k_keep": 1, "token_chunk": token_chunk, "skip_scores": False})
     for _ in range(iters):
         for mod in mods:
             mod.sp_admm_scores(p_scores)
-        api.sp_apply_mask(scores.view(-1), K, mask_out=masks.view(-1))
-        counts = masks.sum(dim=1).cpu().tolist()          # kept units per layer: host arguments of the calls below
-        for l in range(L):
-            if counts[l] < min_keep:
-                api.sp_apply_mask(scores[l], min_keep, mask_out=masks[l])
-                counts[l] = min_keep
+        # one threshold over all layers, the repair of emptied layers and the kept counts: one library call
+        _, _, kept = api.sp_apply_mask_global(scores, keep_fraction, min_keep, mask_out=masks)
+        counts = kept.cpu().tolist()                      # kept units per layer: host arguments of the calls below
         for l, mod in enumerate(mods):
             # with the recovery on the kept support nothing of the unrestricted recovery is needed again
             pl = api.AdmmParams(**{**p.__dict__, "k_keep": int(counts[l]), "token_chunk": token_chunk,
@@ -230,11 +239,13 @@ def plan_distribute(layer_weights: Callable[[int], dict], n_layers: int, n_heads
     return out
 
 
-def module_loss(res: LayerResult, beta: float) -> float:
-    """L_l of Algorithm 1 Step 5: the FFN objective of Appendix A.1 after the last iteration,
-    alpha |Ypre - W2 A|^2 + beta |A - phi(Z)|^2 + alpha |Z - W1 X|^2 (needs compute_objective in the parameters)."""
-    rep = res.reports[-1]
-    return rep["res_out"] + beta * rep["res_act"] + rep["res_in"]
+def total_loss(results, beta: float, device="cuda") -> float:
+    """L(T) = sum_l L_l of Algorithm 1 Step 5 over the given layers: the FFN objective of Appendix A.1 after each
+    layer's last iteration, summed on the device (needs compute_objective in the parameters)."""
+    loss = torch.zeros(1, dtype=torch.float64, device=device)
+    for res in results:
+        api.sp_objective_accumulate(res.last_report, beta, loss, True)
+    return float(loss.item())
 
 
 def temperature_search(layer_inputs: Callable[[int], tuple], n_layers: int, n_units: int, rbar: float, iters: int,
@@ -244,10 +255,17 @@ def temperature_search(layer_inputs: Callable[[int], tuple], n_layers: int, n_un
     With several ranks the losses are summed over ranks before the comparison."""
     p = params or api.AdmmParams()
     p = api.AdmmParams(**{**p.__dict__, "compute_objective": True})
+    device = kw.get("device", "cuda")
+    # Steps 1 and 2 do not depend on the iterations: importances once, the allocations of the whole grid in one launch
+    I_all = layer_importances(layer_inputs, n_layers, p.score_kind, kw.get("token_chunk", 0), device)
+    nu = torch.full((n_layers,), n_units, dtype=torch.int64, device=device)
+    T_list = torch.tensor([float(t) for t in T_grid], dtype=torch.float64, device=device)
+    r_all, k_all = api.sp_allocate_sparsity_grid(I_all, nu, rbar, T_list, True, kw.get("alloc_mode", api.SP_ALLOC_SOFTMAX))
     losses, best = {}, None
-    for T_rel in T_grid:
-        results, r, k_keep, _ = prune_ffn_layers(layer_inputs, n_layers, n_units, rbar, iters, params=p, T_rel=T_rel, **kw)
-        loss = parallel.sum_over_ranks(sum(module_loss(res, p.beta) for res in results), device=kw.get("device", "cuda"))
+    for g, T_rel in enumerate(T_grid):
+        results, r, k_keep, _ = prune_ffn_layers(layer_inputs, n_layers, n_units, rbar, iters, params=p, T_rel=T_rel,
+                                                 planned=(I_all, r_all[g], k_all[g]), **kw)
+        loss = parallel.sum_over_ranks(total_loss(results, p.beta, kw.get("device", "cuda")), device=kw.get("device", "cuda"))
         losses[float(T_rel)] = loss
         if best is None or loss < best[1]:
             best = (float(T_rel), loss, results, r, k_keep)

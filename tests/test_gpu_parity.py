@@ -766,3 +766,75 @@ def test_free_running_iterations_bf16(name, shape, iters):
     # (bf16 operands of the token-axis products), and the regularised solve amplifies such a difference by the
     # conditioning of G + rho I (outlier channels); measured 1.2 to 3.6 times the tolerance, bound 5 times.
     _free_run(cfg, iters, TOL[torch.bfloat16], lambda it: 1.0, chunk=2048, weight_factor=5.0)
+
+
+def test_reproducible_mode_gives_identical_bits():
+    """With sp_set_reproducible(1) no product is cut along K and the solves keep one stream, so two runs on equal
+    inputs agree bit for bit (token count large enough that the default mode does cut the accumulator products)."""
+    cfg = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=8192, sparsity=0.5, outlier_frac=0.02)
+
+    def run():
+        mod, X, W1, W2 = _make_module(cfg, chunk=8192, overlap_k=cfg.k_keep)
+        mod.sp_ffn_init()
+        p = api.AdmmParams(rho=cfg.rho, k_keep=cfg.k_keep, token_chunk=8192)
+        for _ in range(2):
+            mod.sp_admm_step(p)
+        torch.cuda.synchronize()
+        mod.check_status()
+        return [t.clone() for t in (mod.W1, mod.W2, mod.Z, mod.G_A, mod.R1, mod.R2, mod.scores, mod.mask)]
+
+    api.sp_set_reproducible(True)
+    try:
+        a, b = run(), run()
+    finally:
+        api.sp_set_reproducible(False)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    assert api.lib().sp_get_reproducible() == 0
+
+
+@pytest.mark.parametrize("L,n,frac,min_keep", [(3, 328, 0.5, 0), (4, 33, 0.37, 1), (7, 2000, 0.85, 3), (1, 40, 0.3, 0),
+                                               (5, 100, 0.0, 2), (2, 64, 1.0, 0), (32, 16384, 0.4, 1)])
+def test_apply_mask_global_matches_oracle(L, n, frac, min_keep):
+    """One threshold over the scores of all layers (Appendix B, Algorithm 3) on many CTAs: bit-exact masks, kept counts
+    and threshold against the oracle, with many exact ties (also across layers), NaN / infinities, a layer far below
+    the others (emptied unless min_keep), and L * n = 524288 keys, far beyond one CTA's shared memory."""
+    g = torch.Generator().manual_seed(L * 1000 + n)
+    S = torch.round(torch.randn(L, n, generator=g) * 8) / 8            # multiples of 1/8: many ties
+    if L > 1:
+        S[-1] -= 100.0                                                  # the last layer loses every comparison
+    if n >= 33:
+        S[0, 5] = float("nan"); S[0, 7] = float("inf"); S[L - 1, 3] = float("-inf"); S[0, 11] = -0.0
+    ld = n + 8                                                          # rows with a pitch
+    buf = torch.zeros(L, ld, device=DEV)
+    buf[:, :n] = S.to(DEV)
+    mask, tau, kept = api.sp_apply_mask_global(buf[:, :n], frac, min_keep)
+    torch.cuda.synchronize()
+    m_or, c_or, tau_or = O.global_threshold_masks(S.double().numpy(), frac, min_keep=min_keep)
+    assert np.array_equal(mask.cpu().numpy(), m_or)
+    assert kept.cpu().tolist() == c_or.tolist()
+    K = int(np.floor(frac * n * L + 1e-9))
+    if 0 < K < n * L:
+        assert tau.item() == tau_or or (np.isnan(tau_or) and np.isnan(tau.item()))
+    if min_keep == 0:
+        assert int(mask.sum().item()) == K
+
+
+def test_allocate_sparsity_grid_matches_oracle():
+    """Step 2 of Algorithm 1 for a whole temperature grid in one launch, temperatures relative to mean |I|."""
+    L = 24
+    I = synth.make_importances(synth.CONFIGS["C2"]).to(DEV)
+    nu = torch.full((L,), 8192, dtype=torch.int64, device=DEV)
+    grid = [0.05, 0.25, 1.0, 4.0, 50.0]
+    for mode, name in ((api.SP_ALLOC_SOFTMAX, "softmax"), (api.SP_ALLOC_INVERSE, "inverse")):
+        r, k = api.sp_allocate_sparsity_grid(I, nu, 0.5, torch.tensor(grid, dtype=torch.float64, device=DEV), True, mode)
+        torch.cuda.synchronize()
+        I64 = I.cpu().numpy()
+        for g, T_rel in enumerate(grid):
+            r_or, k_or = O.allocate_sparsity(I64, [8192] * L, 0.5, T_rel * np.abs(I64).mean(), name)
+            assert np.abs(r[g].cpu().numpy() - r_or).max() < 1e-12
+            assert np.array_equal(k[g].cpu().numpy(), k_or)
+    # absolute temperatures: row g equals the single call
+    r_abs, k_abs = api.sp_allocate_sparsity_grid(I, nu, 0.5, torch.tensor([0.7], dtype=torch.float64, device=DEV), False)
+    r1, k1 = api.sp_allocate_sparsity(I, nu, 0.5, 0.7)
+    assert torch.equal(r_abs[0], r1) and torch.equal(k_abs[0], k1)
