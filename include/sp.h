@@ -71,7 +71,8 @@ typedef enum { SP_Z_PAPER = 0, SP_Z_EXACT = 1 } sp_z_rule;
 typedef enum { SP_SCORE_WANDA_L2 = 0, SP_SCORE_WANDA_L1 = 1, SP_SCORE_LEMMA1 = 2 } sp_score_kind;
 typedef enum { SP_ALLOC_SOFTMAX = 0, SP_ALLOC_INVERSE = 1, SP_ALLOC_UNIFORM = 2 } sp_alloc_mode;
 typedef enum { SP_WS_GRAM = 0, SP_WS_ADMM_STEP = 1, SP_WS_SCORES = 2, SP_WS_APPLY_MASK = 3, SP_WS_FFN_INIT = 4,
-               SP_WS_LINEAR_REFIT = 5, SP_WS_GEMM = 6, SP_WS_RIDGE_SOLVE = 7, SP_WS_WEIGHT_STATS = 8 } sp_ws_op;
+               SP_WS_LINEAR_REFIT = 5, SP_WS_GEMM = 6, SP_WS_RIDGE_SOLVE = 7, SP_WS_WEIGHT_STATS = 8,
+               SP_WS_INPUT_INVERSE = 9 } sp_ws_op;
 
 /* A row-major device matrix view. */
 typedef struct {
@@ -115,6 +116,8 @@ typedef struct {
   uint8_t* mask;   /* [n]             in/out: 1 = kept                                                           */
   double* importance; /* [1]          out: layer importance I_l = mean_j s_j                                      */
   float* Gate;     /* [N, n] ld = n   SP_ACT_SWIGLU only: g = SiLU(Wg_0 X), written by sp_ffn_init, then read-only   */
+  float* G_X_inv;  /* [d, d]          optional cache (may be NULL): (G_X + rho1 I)^-1 written by
+                                      sp_ffn_cache_input_inverse; read by sp_admm_step in bf16 mode                  */
 } sp_ffn_state;
 
 typedef struct {
@@ -176,6 +179,19 @@ sp_status sp_gram_accumulate(const sp_mat* Xc, const sp_mat* Yc, float* G, int64
  */
 sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_chunk, int32_t* status_dev,
                       void* ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------------
+ * sp_ffn_cache_input_inverse — the cached pseudo-inverse of the module input of Algorithm 2 (SparseLLM1, "pre-compute
+ * and cache a_{l-1}^+"): the input never changes over the iterations, so neither does G_X + rho1 I.  Writes
+ * st->G_X_inv = (G_X + rho1 I)^-1 (fp32 [d, d], factorised and inverted in fp64) after sp_ffn_init.  With it,
+ * sp_admm_step (bf16 mode) recovers W1~ = R1 (G_X + rho1 I)^-1 as ONE tensor-core product with both operands carried
+ * as three bf16 parts instead of a factorisation and two triangular sweeps per step.  rho / rho_relative must be the
+ * values later passed in sp_admm_params (the caller's responsibility; a step with st->G_X_inv == NULL, and every step
+ * in fp32 mode, solves the system itself).  Workspace: sp_workspace_bytes(SP_WS_INPUT_INVERSE, d, 0, 0, 0, 0).
+ * Errors: SP_ERR_INVALID_ARG (null G_X / G_X_inv, rho < 0), SP_ERR_SHAPE, SP_ERR_WORKSPACE, SP_ERR_ALIGNMENT.
+ */
+sp_status sp_ffn_cache_input_inverse(const sp_ffn_module* m, sp_ffn_state* st, double rho, int32_t rho_relative,
+                                     int32_t* status_dev, void* ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------------
  * sp_admm_step — one outer step of Algorithm 2 (SparseLLM1) in the per-step order of Algorithm 3 (GSPO):
@@ -424,6 +440,13 @@ sp_status sp_gemm(int32_t transA, int32_t transB, int64_t M, int64_t N, int64_t 
                   int32_t* status_dev, void* stream);
 sp_status sp_symmetrize(float* G, int64_t n, int64_t ldg, void* stream);
 
+/* sp_set_wait_budget(cycles): every barrier wait inside the tensor-core GEMM kernel is bounded by a clock budget
+ * (about two seconds by default); a wait that outlasts it makes the kernel record SP_ERR_TIMEOUT in status_dev, drain
+ * its copies and tensor-core work in flight, free its tensor memory and return, leaving C incomplete.  This call
+ * changes the budget process-wide (0 restores the default).  It exists for diagnosis and for testing the time-out
+ * path: with a budget of a few cycles an ordinary wait for a long K loop already runs out. */
+sp_status sp_set_wait_budget(int64_t cycles);
+
 /* sp_set_reproducible(on): see "Reproducibility" at the top of this file; sp_get_reproducible() returns the setting. */
 sp_status sp_set_reproducible(int32_t on);
 int32_t sp_get_reproducible(void);
@@ -447,7 +470,7 @@ int64_t sp_launch_count(void);
  *   SP_WS_GRAM: d = channels C, N = tokens T.   SP_WS_ADMM_STEP / SP_WS_FFN_INIT: module sizes, dtype of X.
  *   SP_WS_SCORES: d = n_units*group, N = tokens (LEMMA1) or rows of W (WANDA).
  *   SP_WS_RIDGE_SOLVE / SP_WS_LINEAR_REFIT: d = m (rows of R), n = system size, dtype SP_F64 when precise != 0.
- *   SP_WS_WEIGHT_STATS: d = number of blocks. */
+ *   SP_WS_WEIGHT_STATS: d = number of blocks.   SP_WS_INPUT_INVERSE: d = d_model. */
 size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t token_chunk, int32_t dtype);
 /* Optional extra workspace of sp_admm_step (bf16 mode): when ws_bytes >= sp_workspace_bytes(SP_WS_ADMM_STEP, ...) +
  * sp_admm_overlap_bytes(N, k_keep), the step keeps z^(1) = W1 X of all N tokens on the kept channels (fp32) in the

@@ -68,11 +68,15 @@ def gemm_cases(reps, warm):
     print("status", st.cpu().tolist())
 
 
+SOLVE_SIZES = [(2048, 8192), (2048, 4096), (8192, 2048), (4096, 2048)]
+
+
 def solve_cases(reps, warm):
     st = api.new_status()
-    for m, n in ((2048, 8192), (2048, 4096), (8192, 2048), (4096, 2048)):
-        A = torch.relu(torch.randn(n, 2 * n, device=DEV))
+    for m, n in SOLVE_SIZES:
+        A = torch.relu(torch.randn(n, n + 1024, device=DEV))
         G = (A @ A.T).contiguous()
+        del A
         R = torch.randn(m, n, device=DEV)
         W = torch.empty_like(R)
         ws = torch.empty(api.workspace_bytes(api.SP_WS_RIDGE_SOLVE, m, n, 0, 0, api.SP_F32), dtype=torch.uint8,
@@ -225,6 +229,7 @@ def main():
     ap.add_argument("what", choices=["gemm", "solve", "mask", "lockstep"])
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warm", type=int, default=2)
+    ap.add_argument("--sizes", default="", help="solve: m:n pairs, e.g. 7168:28672,4096:16384 (default: those of a C2 step)")
     a = ap.parse_args()
     if not torch.cuda.is_available():
         raise RuntimeError("microbench needs a CUDA device")
@@ -236,6 +241,8 @@ def main():
     elif a.what == "lockstep":
         lockstep_cases(a.reps, a.warm)
     else:
+        if a.sizes:
+            SOLVE_SIZES[:] = [tuple(int(v) for v in pair.split(":")) for pair in a.sizes.split(",")]
         (gemm_cases if a.what == "gemm" else solve_cases)(a.reps, a.warm)
 
 

@@ -31,7 +31,8 @@ EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_admm_scores"
            "sp_status_string", "sp_version", "sp_profile_begin", "sp_profile_read", "sp_profile_kinds",
            "sp_profile_kind_name", "sp_launch_count", "sp_mha_init", "sp_mha_step", "sp_mha_workspace_bytes",
            "sp_set_reproducible", "sp_get_reproducible", "sp_allocate_sparsity_grid", "sp_apply_mask_global",
-           "sp_apply_mask_global_bytes", "sp_objective_accumulate"]
+           "sp_apply_mask_global_bytes", "sp_objective_accumulate", "sp_ffn_cache_input_inverse",
+           "sp_set_wait_budget"]
 
 
 class SpError(RuntimeError):
@@ -53,7 +54,8 @@ class SpFfnModule(C.Structure):
 class SpFfnState(C.Structure):
     _fields_ = [("Z", C.c_void_p), ("U", C.c_void_p), ("G_X", C.c_void_p), ("G_A", C.c_void_p), ("R1", C.c_void_p),
                 ("R2", C.c_void_p), ("absA", C.c_void_p), ("W1", C.c_void_p), ("W2", C.c_void_p),
-                ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p), ("Gate", C.c_void_p)]
+                ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p), ("Gate", C.c_void_p),
+                ("G_X_inv", C.c_void_p)]
 
 
 class SpAdmmParams(C.Structure):
@@ -105,6 +107,7 @@ def lib() -> C.CDLL:
         pm = C.POINTER(SpMat)
         L.sp_gram_accumulate.argtypes = [pm, pm, vp, i64, vp, i64, vp, vp, vp, sz, vp]
         L.sp_ffn_init.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), i64, vp, vp, sz, vp]
+        L.sp_ffn_cache_input_inverse.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), dbl, i32, vp, vp, sz, vp]
         L.sp_admm_scores.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), C.POINTER(SpAdmmParams), vp, vp,
                                      C.c_size_t, vp]
         L.sp_admm_step.argtypes = [C.POINTER(SpFfnModule), C.POINTER(SpFfnState), C.POINTER(SpAdmmParams), vp, vp, vp,
@@ -130,6 +133,7 @@ def lib() -> C.CDLL:
         L.sp_apply_mask_global_bytes.argtypes = [i64, i32]
         L.sp_objective_accumulate.argtypes = [vp, dbl, vp, i32, vp]
         L.sp_set_reproducible.argtypes = [i32]
+        L.sp_set_wait_budget.argtypes = [i64]
         L.sp_get_reproducible.restype = i32
         L.sp_profile_begin.argtypes = [i32]
         L.sp_profile_read.argtypes = [vp]
@@ -393,6 +397,7 @@ def sp_apply_mask_batched(scores, k_keep, want_index=False):
 
 
 SP_WS_WEIGHT_STATS = 8
+SP_WS_INPUT_INVERSE = 9
 
 
 def sp_weight_stats(W, axis=0, group=0, stats=None, accumulate=False):
@@ -479,6 +484,9 @@ class FfnModule:
         self.Z = torch.empty(N, n, **f32)
         self.U = torch.zeros(N, n, **f32) if dual_mode else None
         self.G_X = torch.empty(d, d, **f32)
+        self.G_X_inv = None           # cache of (G_X + rho1 I)^-1, see sp_ffn_cache_input_inverse
+        self._inv_key = None
+        self.cache_input_inverse = X.dtype == torch.bfloat16
         self.G_A = torch.empty(n, n, **f32)
         self.R1 = torch.empty(n, d, **f32)
         self.R2 = torch.empty(d, n, **f32)
@@ -515,7 +523,7 @@ class FfnModule:
         return SpFfnState(self.Z.data_ptr(), _ptr(self.U), self.G_X.data_ptr(), self.G_A.data_ptr(),
                           self.R1.data_ptr(), self.R2.data_ptr(), self.absA.data_ptr(), self.W1.data_ptr(),
                           self.W2.data_ptr(), self.scores.data_ptr(), self.mask.data_ptr(),
-                          self.importance.data_ptr(), _ptr(self.Gate))
+                          self.importance.data_ptr(), _ptr(self.Gate), _ptr(self.G_X_inv))
 
     def _workspace(self, chunk: int) -> torch.Tensor:
         need = max(workspace_bytes(SP_WS_ADMM_STEP, self.d, self.n, self.N, chunk, _dt(self.X)),
@@ -527,13 +535,30 @@ class FfnModule:
         return self._ws
 
     def sp_ffn_init(self):
+        self._inv_key = None            # G_X is about to change
         ws = self._workspace(self.token_chunk)
         m, st = self._module(), self._state()
         _check(lib().sp_ffn_init(C.byref(m), C.byref(st), self.token_chunk, self.status.data_ptr(), ws.data_ptr(),
                                  ws.numel(), _stream()), "sp_ffn_init")
         self.iteration = 0
 
+    def sp_ffn_cache_input_inverse(self, rho: float, rho_relative: bool = True):
+        """(G_X + rho1 I)^-1 of the constant module input into self.G_X_inv (once per module and ridge)."""
+        if self.G_X_inv is None:
+            self.G_X_inv = torch.empty(self.d, self.d, dtype=torch.float32, device=self.dev)
+        ws = _ws(workspace_bytes(SP_WS_INPUT_INVERSE, self.d, 0, 0, 0, 0), self.dev)
+        m, st = self._module(), self._state()
+        _check(lib().sp_ffn_cache_input_inverse(C.byref(m), C.byref(st), float(rho), int(bool(rho_relative)),
+                                                self.status.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+               "sp_ffn_cache_input_inverse")
+        self._inv_key = (float(rho), bool(rho_relative))
+
+    def _ensure_inverse(self, p):
+        if self.cache_input_inverse and self._inv_key != (float(p.rho), bool(p.rho_relative)):
+            self.sp_ffn_cache_input_inverse(p.rho, p.rho_relative)
+
     def sp_admm_step(self, p: AdmmParams):
+        self._ensure_inverse(p)
         chunk = p.token_chunk or self.token_chunk
         ws = self._workspace(chunk)
         m, st = self._module(), self._state()
@@ -545,6 +570,7 @@ class FfnModule:
 
     def sp_admm_scores(self, p: AdmmParams):
         """Unrestricted recovery + unit scores + layer importance of the current state (no mask, no token pass)."""
+        self._ensure_inverse(p)
         chunk = p.token_chunk or self.token_chunk
         ws = self._workspace(chunk)
         m, st = self._module(), self._state()

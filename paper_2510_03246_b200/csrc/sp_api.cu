@@ -240,6 +240,7 @@ struct AdmmPlan {
   uint8_t* grp_mask;
   void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
   void* W2sb;                  // bf16 hi | lo split of W2[:, S] ([d, 2 * pad64(k)], gated modules)
+  void *R1p, *Gip;             // three-part bf16 forms of R1 [n, 3 pad64(d)] and of the cached (G_X + rho1 I)^-1
   void *H, *E, *Ac, *Zb;
   float *D, *z1, *Eo;          // Eo: Ypre - A W2^T of a chunk (objective reporting)
   void* W2fb;                  // bf16 copy of the full W2 (objective reporting)
@@ -276,6 +277,8 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.W2b = p.bf16 ? c.take_bytes(((size_t)n + 8) * d * csz) : nullptr;
   p.Qtb = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // room for the hi | lo form
   p.W2sb = p.bf16 ? c.take_bytes((size_t)d * 2 * split_kpad(n) * csz) : nullptr;
+  p.R1p = p.bf16 ? c.take_bytes((size_t)n * 3 * split_kpad(d) * csz) : nullptr;
+  p.Gip = p.bf16 ? c.take_bytes((size_t)d * 3 * split_kpad(d) * csz) : nullptr;
   const size_t npad = (size_t)(n + 7) / 8 * 8;   // leading dimension bound of the compact tensors
   // bf16 mode: room for h as hi | lo parts (gated modules)
   p.H = c.take_bytes((size_t)p.chunk * (p.bf16 ? 2 * (size_t)split_kpad(n) : npad) * csz);
@@ -376,6 +379,8 @@ size_t sp_workspace_bytes(int32_t op, int64_t d, int64_t n, int64_t N, int64_t t
     case SP_WS_LINEAR_REFIT: return ridge_ws_bytes(d, n, dtype == SP_F64) + align_up((size_t)(n > 0 ? n : 1) * 4, 256) + 512;
     case SP_WS_RIDGE_SOLVE: return ridge_ws_bytes(d, n, dtype == SP_F64) + 256;
     case SP_WS_GEMM: return 256;
+    case SP_WS_INPUT_INVERSE:
+      return ridge_ws_bytes(d, d, true) + align_up((size_t)(d > 0 ? d : 1) * (size_t)(d > 0 ? d : 1) * 4, 256) + 512;
     case SP_WS_WEIGHT_STATS: return align_up((size_t)(148 * 8 + (d > 0 ? d : 1)) * 3 * sizeof(double), 256) + 256;
     default: return 0;
   }
@@ -736,6 +741,22 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   return SP_OK;
 }
 
+sp_status sp_ffn_cache_input_inverse(const sp_ffn_module* m, sp_ffn_state* st, double rho, int32_t rho_relative,
+                                     int32_t* status_dev, void* ws, size_t ws_bytes, void* stream) {
+  if (!m || !st || !st->G_X || !st->G_X_inv || !(rho >= 0.0)) return SP_ERR_INVALID_ARG;
+  const int64_t d = m->d;
+  if (d < 1) return SP_ERR_SHAPE;
+  if (!ws || ws_bytes < sp_workspace_bytes(SP_WS_INPUT_INVERSE, d, 0, 0, 0, 0)) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256)) return SP_ERR_ALIGNMENT;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  Carver c(ws);
+  SolveBufs b = carve_solve(c, d, d, 8);
+  float* eye = c.take<float>((size_t)d * d);
+  CU(set_identity(eye, d, d, s));
+  CU(effective_ridge(st->G_X, d, d, rho, rho_relative, b.rho, s));
+  return ridge_core<double>(eye, d, st->G_X, d, d, d, nullptr, d, b.rho, st->G_X_inv, d, b, status_dev, s);
+}
+
 // One step, or (scores_only) its first two parts: the unrestricted recovery the scores read, and the scores.
 static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const sp_admm_params* prm, sp_step_report* rep_dev,
                          int32_t* status_dev, void* ws, size_t ws_bytes, void* stream, bool scores_only) {
@@ -792,7 +813,25 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   const bool need_w1 = !scores_only || prm->score_kind == SP_SCORE_LEMMA1;   // only the Lemma-1 score reads W1~
   if (need_w1) {
     CU(effective_ridge(st->G_X, d, d, prm->rho, prm->rho_relative, rho1, sa));
-    if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
+    if (bf16 && st->G_X_inv) {
+      // cached inverse of the constant system: W1~ = R1 Ginv, both operands as three bf16 parts, the six part products
+      // of weight >= 2^-16 as K segments (Ginv is symmetric, so its rows serve as the K-major B operand)
+      const int64_t dp3 = split_kpad(d);
+      CU(split3_bf16(st->R1, d, n, d, dp3, p.R1p, sa));
+      CU(split3_bf16(st->G_X_inv, d, d, d, dp3, p.Gip, sa));
+      TcOperand ta{p.R1p, 3 * dp3, true}, tb{p.Gip, 3 * dp3, true};
+      ta.kext = tb.kext = 3 * dp3;
+      TcSegments sg;
+      sg.nseg = 6;
+      static const int pa[6] = {0, 0, 1, 0, 2, 1}, pb[6] = {0, 1, 0, 2, 0, 1};
+      for (int q = 0; q < 6; ++q) {
+        sg.a_k[q] = (int32_t)(pa[q] * dp3);
+        sg.b_k[q] = (int32_t)(pb[q] * dp3);
+      }
+      ProfScope prof(PK_SOLVE, 2.0 * (double)n * d * d, 0.0, sa);
+      SPCHK(gemm_tc(n, d, d, 1.f, ta, tb, 0.f, Operand{p.W1t, SP_F32, d, 1}, OutOperand{p.W1t, SP_F32, d}, false,
+                    status_dev, sa, &sg, 2.0 * (double)n * d * d));
+    } else if (bf16) SPCHK(ridge_core<float>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
                                       side ? &side->assist_side : nullptr));
     else SPCHK(ridge_core<double>(st->R1, d, st->G_X, d, n, d, nullptr, d, rho1, p.W1t, d, p.sbA, status_dev, sa,
                                       side ? &side->assist_side : nullptr));

@@ -31,6 +31,8 @@ void count_launch(int n = 1);
 // sp_set_reproducible: when on, every floating-point sum of the library is taken in an order fixed by the call's
 // arguments (no product is cut along K, the triangular solves run on one stream), so equal inputs give equal bits.
 bool reproducible_mode();
+// sp_set_wait_budget: clock cycles a barrier wait of the tensor-core GEMM may take (0: the built-in default)
+long long wait_budget_cycles();
 // Brackets the kernels launched during its lifetime with a CUDA event pair on `stream` when profiling is enabled.
 // Scopes nest: only the outermost one records, so a phase scope absorbs the kernels launched inside it.
 struct ProfScope {
@@ -184,6 +186,9 @@ cudaError_t symmetrize_lower(float* G, int64_t n, int64_t ld, cudaStream_t strea
 // row_idx != nullptr: row i of dst comes from row row_idx[i] of src.
 cudaError_t split_bf16(const float* src, int64_t lds, const int32_t* row_idx, int64_t rows, int64_t cols, int64_t kpad,
                        void* dst, cudaStream_t stream);
+// dst [rows, 3 * kpad] bf16: the hi, mid and lo parts of src side by side (an fp32 value as an exact sum of three bf16)
+cudaError_t split3_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad, void* dst,
+                        cudaStream_t stream);
 // dst[j, i] = (TD) src[i, j]
 template <typename TD>
 cudaError_t transpose_convert(const float* src, int64_t lds, int64_t rows, int64_t cols, TD* dst, int64_t ldd,

@@ -85,6 +85,28 @@ __global__ void split_bf16_kernel(const float* __restrict__ src, int64_t lds, co
   }
 }
 
+// dst[i, part * kpad + j] = part `part` of the three-part bf16 split of src[i, j] (hi + mid + lo = src exactly up to
+// 2^-24); padding columns are zero.
+__global__ void split3_bf16_kernel(const float* __restrict__ src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad,
+                                   __nv_bfloat16* __restrict__ dst) {
+  const int64_t total = rows * kpad;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / kpad, j = e % kpad;
+    const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+    __nv_bfloat16 hi = zero, mid = zero, lo = zero;
+    if (j < cols) {
+      const float v = src[i * lds + j];
+      hi = __float2bfloat16_rn(v);
+      const float r1 = v - __bfloat162float(hi);
+      mid = __float2bfloat16_rn(r1);
+      lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    }
+    dst[i * 3 * kpad + j] = hi;
+    dst[i * 3 * kpad + kpad + j] = mid;
+    dst[i * 3 * kpad + 2 * kpad + j] = lo;
+  }
+}
+
 __global__ void symmetrize_kernel(float* G, int64_t n, int64_t ld) {
   __shared__ float tile[32][33];
   // block (bx, by) with bx > by mirrors lower tile (row block bx, col block by) to (by, bx); diagonal blocks in place
@@ -754,6 +776,16 @@ template cudaError_t transpose_convert<double>(const float*, int64_t, int64_t, i
                                                cudaStream_t);
 template cudaError_t transpose_convert<__nv_bfloat16>(const float*, int64_t, int64_t, int64_t, __nv_bfloat16*,
                                                       int64_t, cudaStream_t);
+
+cudaError_t split3_bf16(const float* src, int64_t lds, int64_t rows, int64_t cols, int64_t kpad, void* dst,
+                        cudaStream_t stream) {
+  if (rows * kpad == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, (double)rows * cols * 10.0, stream);
+  count_launch();
+  split3_bf16_kernel<<<grid_for(rows * kpad, 256), 256, 0, stream>>>(src, lds, rows, cols, kpad,
+                                                                     reinterpret_cast<__nv_bfloat16*>(dst));
+  return cudaGetLastError();
+}
 
 cudaError_t split_bf16(const float* src, int64_t lds, const int32_t* row_idx, int64_t rows, int64_t cols, int64_t kpad,
                        void* dst, cudaStream_t stream) {

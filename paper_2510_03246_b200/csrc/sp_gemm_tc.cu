@@ -80,6 +80,7 @@ struct TcParams {
   int32_t batched, nb0, nb1, tiles_per_batch;
   int8_t a_ord[4], b_ord[4], c_ord[4];
   int64_t c_s0, c_s1, cin_s0, cin_s1;
+  long long wait_budget;   // clock cycles a role may wait on one barrier before it gives up (SP_ERR_TIMEOUT)
   int32_t* status;
 };
 
@@ -384,7 +385,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         unit_map(p, u, num_kb, tile, kb0, kb1);
         tile_coords<BATCHED>(p, tile, tm, tn, b0, b1);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.wait_budget)) { ok = false; break; }
           // the leader's barrier collects the bytes of both CTAs' loads of this stage
           if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
           const uint32_t fbar = map_to_cta(full_bar(s), 0);
@@ -446,13 +447,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       bool issued = false;
       for (int u = cid; u < p.num_units && ok; u += ncl) {
-        if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
+        if (!mbar_wait(tempty_bar(acc), aph ^ 1u, abort_flag, p.wait_budget)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * TILE_N);
         int tile, kb0, kb1;
         unit_map(p, u, num_kb, tile, kb0, kb1);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(full_bar(s), ph, abort_flag, WAIT_BUDGET_CYCLES)) { ok = false; break; }
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.wait_budget)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles + s * STAGE_BYTES;
           const uint32_t b_src = a_src + A_BYTES;
@@ -473,13 +474,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_commit_pair(tfull_bar(acc));   // accumulator complete: wakes the epilogue warps of both CTAs
         if (++acc == 2) { acc = 0; aph ^= 1u; }
       }
-      if (!ok) {
-        report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 2);
-        if (issued) {   // wait for MMAs in flight before shared and tensor memory are released
-          tc_commit_local(drain_bar);
-          const long long t0 = clock64();
-          while (!mbar_try(drain_bar, 0u) && clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
-        }
+      if (!ok) report_status(p.status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 2);
+      // Wait for the MMAs in flight before shared and tensor memory are released.  In a complete run the epilogue
+      // has already seen the last accumulator, so this returns at once; it matters when a role gave up (here, or an
+      // epilogue warp that left without waiting for its accumulator).
+      if (issued && (!ok || *abort_flag)) {
+        tc_commit_local(drain_bar);
+        const long long t0 = clock64();
+        while (!mbar_try(drain_bar, 0u) && clock64() - t0 < DRAIN_BUDGET_CYCLES) {}
       }
     }
   } else {
@@ -504,7 +506,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int64_t c_boff = BATCHED ? (int64_t)b0 * p.c_s0 + (int64_t)b1 * p.c_s1 : 0;
       const int64_t cin_boff = BATCHED ? (int64_t)b0 * p.cin_s0 + (int64_t)b1 * p.cin_s1 : 0;
       // every lane observes the barrier itself; the vote keeps the warp converged for the aligned TMEM loads
-      const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, WAIT_BUDGET_CYCLES);
+      const bool got = mbar_wait(tfull_bar(acc), aph, abort_flag, p.wait_budget);
       if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
       tc_fence_after();
       const int64_t row0 = (int64_t)tm * TILE_M + (int64_t)rank * BM + q * 32;   // first global row of this warp
@@ -534,7 +536,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               tma_load_2d_local(wstg + (cbuf ^ 1) * 2048, &tmCin, (int32_t)(gj0 + 32), (int32_t)row0,
                                 cin_bar(q, cbuf ^ 1));
             }
-            const bool got_c = mbar_wait(cin_bar(q, cbuf), (cph >> cbuf) & 1u, abort_flag, WAIT_BUDGET_CYCLES);
+            const bool got_c = mbar_wait(cin_bar(q, cbuf), (cph >> cbuf) & 1u, abort_flag, p.wait_budget);
             if (!__all_sync(0xffffffffu, got_c)) { ok = false; break; }
             if (lane == 0) bulk_wait_read_1();
             __syncwarp();
@@ -897,6 +899,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
     p.num_tiles = (int32_t)all;
   }
   p.status = status_dev;
+  p.wait_budget = wait_budget_cycles() > 0 ? wait_budget_cycles() : WAIT_BUDGET_CYCLES;
 
   // Tile counts that do not fill the last wave of CTA pairs leave SMs idle.  A call that accumulates into C through
   // the add-reduction epilogue may cut K into a few ranges per tile instead: the partial products add up in C (in an

@@ -604,6 +604,11 @@ __global__ void __launch_bounds__(NM_THREADS)
   next_diag_body<2>(nullptr, A22, lda, nb2, nullptr, LmT, S, nullptr);
 }
 
+// two-level blocking of the factorisation (see potrf_lower_tc): systems of at least kOuterMinN rows, outer blocks of
+// kOuterBlocks diagonal blocks
+constexpr int64_t kOuterMinN = 12288;
+constexpr int64_t kOuterBlocks = 4;
+
 constexpr int kPartA[6] = {0, 0, 1, 0, 2, 1};
 constexpr int kPartB[6] = {0, 1, 0, 2, 0, 1};
 
@@ -638,12 +643,26 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
   float* S = dinv + nblk * 2 * TB * TB;      // [128, 128] next diagonal block
   float* LmT = S + TB * TB;                  // [128, 128] scratch of the lookahead kernel
   bool rec[2] = {false, false};
+  // Two-level blocking for large systems: the trailing update of a step is bound by the read-modify-write of the fp32
+  // matrix when K is only 128 (n = 28672: 430 GB per factorisation).  With OB > 1 the steps of an outer block of OB
+  // diagonal blocks update only the rest of that outer block's columns at once; everything to the right of it gets
+  // ONE update per outer block with K = OB * 128, which divides that traffic by OB.
+  const int64_t OB = (assist && n >= kOuterMinN) ? kOuterBlocks : 1;
   for (int64_t kb = 0; kb < nblk; ++kb) {
     const int64_t k0 = kb * TB;
     const int nb = (int)((n - k0 < TB) ? (n - k0) : TB);
     float* dk = dinv + kb * 2 * TB * TB;
+    const int64_t ob_start = kb / OB * OB;
+    const int64_t ob_end_blk = (ob_start + OB < nblk) ? ob_start + OB : nblk;
+    const int64_t ob_end_col = (ob_end_blk * TB < n) ? ob_end_blk * TB : n;
+    const bool outer = OB > 1;
+    const bool inner_last = outer && kb == ob_end_blk - 1;
+    const bool inner_first = outer && kb == ob_start;
     {
-      const bool from_scratch = assist && kb > 0;
+      // the first block of an outer block is read from the matrix itself, once the first columns of the previous
+      // outer block's update have landed; every other block comes from the lookahead kernel's scratch
+      const bool from_scratch = assist && kb > 0 && !inner_first;
+      if (assist && inner_first && kb > 0) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->near_done, 0));
       count_launch();
       ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
       chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
@@ -661,11 +680,11 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     // last block with appended rows: their panel runs on `stream`, behind the assisting stream's last update
     if (assist && rem <= 0 && kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
     if (assist && rem > 0) {
-      // next diagonal block: it reads blocks (kb+1, kb) and (kb+1, kb+1), i.e. the first two block columns of the
-      // trailing update of step kb - 1, which that step issues first and signals on their own
-      if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->near_done, 0));
-      const int nb2 = (int)(rem < TB ? rem : TB);
-      {
+      if (!inner_last) {
+        // next diagonal block: it reads blocks (kb+1, kb) and (kb+1, kb+1), i.e. the first two block columns of the
+        // trailing update of step kb - 1, which that step issues first and signals on their own
+        if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->near_done, 0));
+        const int nb2 = (int)(rem < TB ? rem : TB);
         count_launch();
         ProfScope prof(PK_PANEL_APPLY, 4.0 * TB * TB * TB, 0.0, stream);
         if (!split_lookahead) {
@@ -704,7 +723,52 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     }
     float* A22 = A + (k0 + nb) * lda + (k0 + nb);
     constexpr int64_t kNear = 2 * TB;     // block columns of the update that the next step's chain kernels read
-    if (assist && rem > kNear) {
+    if (outer) {
+      // (a) the rest of this outer block's columns, all rows below: K = 128
+      const int64_t cols_in = ob_end_col - (k0 + nb);
+      if (cols_in > 0) {
+        tb.mnext = cols_in;
+        sp_status st = gemm_tc(prow, cols_in, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1},
+                               OutOperand{A22, SP_F32, lda}, true, status_dev, sb, &sg,
+                               (2.0 * (double)prow * (double)cols_in - (double)cols_in * (double)cols_in) * (double)nb);
+        if (st != SP_OK) return st;
+        SP_CUDA_OK(cudaEventRecord(assist->near_done, sb));
+      }
+      // (b) after the outer block's last step: everything to its right, K = the outer block's width
+      const int64_t cols_out = n - ob_end_col;
+      if (inner_last && cols_out > 0) {
+        const int64_t o0 = ob_start * TB, kw = ob_end_col - o0, prow_out = cols_out + m_extra;
+        TcSegments so;
+        so.nseg = 6;
+        for (int q = 0; q < 6; ++q) {
+          so.a_k[q] = (int32_t)(kPartA[q] * np + o0);
+          so.b_k[q] = (int32_t)(kPartB[q] * np + o0);
+        }
+        float* Aout = A + ob_end_col * lda + ob_end_col;
+        const int64_t wn = cols_out < kNear ? cols_out : kNear;
+        TcOperand na{P + ob_end_col * ldp, ldp, true}, nbo{P + ob_end_col * ldp, ldp, true};
+        na.kext = nbo.kext = ldp;
+        na.mnext = prow_out;
+        nbo.mnext = wn;
+        sp_status st = gemm_tc(prow_out, wn, kw, -1.f, na, nbo, 1.f, Operand{Aout, SP_F32, lda, 1},
+                               OutOperand{Aout, SP_F32, lda}, true, status_dev, sb, &so,
+                               (2.0 * (double)prow_out * (double)wn - (double)wn * (double)wn) * (double)kw);
+        if (st != SP_OK) return st;
+        SP_CUDA_OK(cudaEventRecord(assist->near_done, sb));
+        if (cols_out > wn) {
+          TcOperand fa{P + (ob_end_col + wn) * ldp, ldp, true}, fb{P + (ob_end_col + wn) * ldp, ldp, true};
+          fa.kext = fb.kext = ldp;
+          fa.mnext = prow_out - wn;
+          fb.mnext = cols_out - wn;
+          float* Afar = Aout + wn * lda + wn;
+          const double fr = (double)(cols_out - wn);
+          st = gemm_tc(prow_out - wn, cols_out - wn, kw, -1.f, fa, fb, 1.f, Operand{Afar, SP_F32, lda, 1},
+                       OutOperand{Afar, SP_F32, lda}, true, status_dev, sb, &so,
+                       (fr * fr + 2.0 * (double)m_extra * fr) * (double)kw);
+          if (st != SP_OK) return st;
+        }
+      }
+    } else if (assist && rem > kNear) {
       // two launches: the first two block columns (all rows below), signalled at once, then the rest
       tb.mnext = kNear;
       sp_status st = gemm_tc(prow, kNear, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1},

@@ -15,12 +15,15 @@ struct Slot {
 };
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_reproducible{0};
+std::atomic<long long> g_wait_budget{0};
 int g_enabled = 0;   // 0 off, 1 outermost scopes only, 2 every scope (nested ones are then counted twice)
 std::vector<Slot> g_slots;
 int g_used = 0;
 thread_local int g_depth = 0;
 
 }  // namespace
+
+long long wait_budget_cycles() { return g_wait_budget.load(std::memory_order_relaxed); }
 
 bool reproducible_mode() { return g_reproducible.load(std::memory_order_relaxed) != 0; }
 
@@ -54,6 +57,12 @@ sp_status sp_set_reproducible(int32_t on) {
   sp::g_reproducible.store(on ? 1 : 0);
   return SP_OK;
 }
+sp_status sp_set_wait_budget(int64_t cycles) {
+  if (cycles < 0) return SP_ERR_INVALID_ARG;
+  sp::g_wait_budget.store((long long)cycles);
+  return SP_OK;
+}
+
 int32_t sp_get_reproducible(void) { return sp::g_reproducible.load(); }
 
 int64_t sp_launch_count(void) { return (int64_t)sp::g_launches.load(); }

@@ -838,3 +838,51 @@ def test_allocate_sparsity_grid_matches_oracle():
     r_abs, k_abs = api.sp_allocate_sparsity_grid(I, nu, 0.5, torch.tensor([0.7], dtype=torch.float64, device=DEV), False)
     r1, k1 = api.sp_allocate_sparsity(I, nu, 0.5, 0.7)
     assert torch.equal(r_abs[0], r1) and torch.equal(k_abs[0], k1)
+
+
+def test_cached_input_inverse_and_step_without_it():
+    """Algorithm 2 caches the pseudo-inverse of the constant module input: sp_ffn_cache_input_inverse against the fp64
+    inverse of G_X + rho1 I, and the step that solves the input system itself (no cache) against the oracle as well
+    (the teacher-forced bf16 cases above run with the cache, which the binding fills by default)."""
+    cfg = SMALL_BF16
+    mod, X, W1, W2 = _make_module(cfg, chunk=512)
+    mod.sp_ffn_init()
+    mod.sp_ffn_cache_input_inverse(cfg.rho, True)
+    torch.cuda.synchronize()
+    mod.check_status()
+    G = np64(mod.G_X)
+    want = np.linalg.inv(G + O.effective_ridge(G, cfg.rho, True) * np.eye(G.shape[0]))
+    assert relerr(np64(mod.G_X_inv), want) < 1e-5
+    mod2, X, W1, W2 = _make_module(cfg, chunk=512)
+    mod2.cache_input_inverse = False
+    mod2.sp_ffn_init()
+    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, token_chunk=512, compute_objective=True)
+    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep)
+    for it in range(2):
+        _step_and_compare(mod2, X, W1.float(), p_gpu, p_or, TOL[X.dtype], [])
+    assert mod2.G_X_inv is None
+
+
+def test_wait_budget_runs_out_and_context_stays_usable():
+    """Time-out path of the tensor-core GEMM: with a wait budget of one clock cycle the epilogue's ordinary wait for a
+    long K loop runs out (nothing is withheld, no kernel is altered); the kernel reports SP_ERR_TIMEOUT through the
+    status word, drains and returns; afterwards the same product with the default budget is correct."""
+    g = torch.Generator().manual_seed(3)
+    M, N, K = 512, 512, 32768
+    A = (torch.randn(M, K, generator=g) * 0.1).to(torch.bfloat16).to(DEV)
+    B = (torch.randn(N, K, generator=g) * 0.1).to(torch.bfloat16).to(DEV)
+    Cm = torch.zeros(M, N, device=DEV)
+    st = api.new_status()
+    assert api.lib().sp_set_wait_budget(1) == 0
+    try:
+        api.sp_gemm(A, B, Cm, transB=True, use_tensor_cores=True, status=st)
+        torch.cuda.synchronize()
+    finally:
+        api.lib().sp_set_wait_budget(0)
+    assert st.cpu().tolist()[0] == 7                     # SP_ERR_TIMEOUT
+    st.zero_()
+    api.sp_gemm(A, B, Cm, transB=True, use_tensor_cores=True, status=st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == 0
+    ref = A.double() @ B.double().T
+    assert relerr(np64(Cm), ref.cpu().numpy()) < 1e-5
