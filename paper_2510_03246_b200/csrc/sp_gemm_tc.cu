@@ -150,15 +150,13 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false when the budget ran out or another role of this CTA already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget) {
   if (mbar_try(bar, parity)) return true;
+  // (a try_wait may itself suspend the thread for a while, so the clock is read after every unsuccessful try)
   const long long t0 = clock64();
-  uint32_t it = 0;
   while (!mbar_try(bar, parity)) {
-    if ((++it & 0x3ffu) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > budget) {
-        *abort_flag = 1;
-        return false;
-      }
+    if (*abort_flag) return false;
+    if (clock64() - t0 > budget) {
+      *abort_flag = 1;
+      return false;
     }
   }
   return true;
