@@ -54,6 +54,7 @@ def parse():
     ap.add_argument("--shard", default="modules", choices=["modules", "tokens"],
                     help="N > 1: every rank its own module (default, no collective), or ONE module with its tokens "
                          "split over the ranks (accumulators all-reduced once per iteration)")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing of the step")
     ap.add_argument("--reproducible", action="store_true",
                     help="run with sp_set_reproducible(1): fixed summation order, bit-identical results")
     ap.add_argument("--cpu-sample-tokens", type=int, default=1024)
@@ -253,7 +254,7 @@ def build_module(cfg, args, dev, layer, by_tokens, world):
     return mod, X, W1_0, W2_0, Wg_0
 
 
-def measure(cfg, args, dev, mod, layer, by_tokens, world, steps, warmup, local_rank):
+def measure(cfg, args, dev, mod, layer, by_tokens, world, steps, warmup, local_rank, graph=False):
     """Times `steps` steps of the module (profiling off: nothing but the library's own launches in the timed region),
     then the same number of steps again with a CUDA event pair around every launch / phase for the per-kernel figures.
     Returns (ms of the timed loop on this rank, launches in it, clocks, per-kind event records, ms of the profiled loop)."""
@@ -298,6 +299,29 @@ def measure(cfg, args, dev, mod, layer, by_tokens, world, steps, warmup, local_r
     ms_local = ev0.elapsed_time(ev1)
     launches = api.sp_launch_count()
     mod.check_status()
+    # the same steps replayed from a CUDA graph (one captured step; the library's forks onto its own streams are
+    # event-ordered and capture with it): what a caller gains who captures the loop body
+    graph_ms = None
+    if graph and not by_tokens:
+        try:
+            cap = torch.cuda.Stream()
+            cap.wait_stream(torch.cuda.current_stream())
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
+                step()
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            ev0.record()
+            for _ in range(steps):
+                g.replay()
+            ev1.record()
+            torch.cuda.synchronize()
+            graph_ms = ev0.elapsed_time(ev1) / steps
+            mod.check_status()
+            del g
+        except Exception as exc:   # capture is optional: report why it was not taken
+            graph_ms = f"not captured: {type(exc).__name__}"
     # second loop: the same steps with events around every launch
     api.sp_profile_begin(True)
     ev0.record()
@@ -308,7 +332,7 @@ def measure(cfg, args, dev, mod, layer, by_tokens, world, steps, warmup, local_r
     prof = api.sp_profile_read()
     api.sp_profile_begin(False)
     mod.check_status()
-    return ms_local, launches, clocks, prof, ev0.elapsed_time(ev1), prm
+    return ms_local, launches, clocks, prof, ev0.elapsed_time(ev1), prm, graph_ms
 
 
 def rooflines(cfg, args, prof, steps, peaks):
@@ -383,8 +407,9 @@ def main():
         raise SystemExit("--shard tokens: ReLU modules only")
     layer = rank
     mod, X, W1_0, W2_0, Wg_0 = build_module(cfg, args, dev, layer, by_tokens, world)
-    ms_local, launches, clocks, prof, ms_prof, prm = measure(cfg, args, dev, mod, layer, by_tokens, world, args.steps,
-                                                             args.warmup, local_rank)
+    ms_local, launches, clocks, prof, ms_prof, prm, graph_ms = measure(cfg, args, dev, mod, layer, by_tokens, world,
+                                                                       args.steps, args.warmup, local_rank,
+                                                                       graph=(world == 1 and not args.no_graph))
     ms = parallel.max_over_ranks(ms_local, dev)
     value = (1 if by_tokens else world) * args.steps / (ms * 1e-3)      # one module in all when its tokens are split
 
@@ -502,7 +527,7 @@ def main():
                 workloads[name] = {"skipped": f"needs about {WORKLOAD_GB[name]} GB of free device memory"}
                 continue
             wmod, wX, wW1, wW2, wWg = build_module(wcfg, args, dev, 0, False, 1)
-            w_ms, w_launches, w_clocks, w_prof, w_ms_prof, _ = measure(wcfg, args, dev, wmod, 0, False, 1,
+            w_ms, w_launches, w_clocks, w_prof, w_ms_prof, _, _ = measure(wcfg, args, dev, wmod, 0, False, 1,
                                                                        args.workload_steps, args.workload_warmup,
                                                                        local_rank)
             r_tc, r_hbm, w_break = rooflines(wcfg, args, w_prof, args.workload_steps, peaks)
@@ -531,7 +556,7 @@ def main():
                                        if by_tokens else f"modules x{world} (independent, no collective)")},
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e,
             "cpu_baseline": cpu, "fixed_mask": fixed, "workloads": workloads,
-            "profiled_ms_per_step": ms_prof / args.steps,
+            "profiled_ms_per_step": ms_prof / args.steps, "graph_replay_ms_per_step": graph_ms,
             "profile_note": "value / ms_per_step: timed loop with nothing but the library's launches; roofline, "
                             "roofline_hbm and breakdown: the same steps repeated right after it with a CUDA event pair "
                             "around every launch or phase (profiled_ms_per_step)",

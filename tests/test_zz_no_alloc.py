@@ -52,6 +52,37 @@ def test_static_scores_match_workspace_scores_on_two_calls_in_a_row():
         assert np.array_equal(got_s.cpu().numpy(), ref_s.cpu().numpy())
 
 
+def test_static_scores_units_that_straddle_column_groups_and_unaligned_weights():
+    """Units whose width does not divide the kernel's 128-column groups (3 and 96 columns per unit) take the path that
+    gathers a unit's column values across groups; a weight view with a pitch larger than its width and a start that is
+    not 16-byte aligned takes the scalar loads.  Each runs right after a call that left other values in the scratch,
+    and is also checked against the definition evaluated in fp64 on the host."""
+    first = _inputs(300, 2500, 1, 40, 21)
+    _static_call(api.SP_SCORE_WANDA_L2, 2500, 1, *first, 40)            # dirties the scratch
+    for kind, d, n_units, group, N, seed in ((api.SP_SCORE_WANDA_L2, 210, 333, 3, 50, 22),
+                                             (api.SP_SCORE_WANDA_L1, 130, 21, 96, 32, 23)):
+        n = n_units * group
+        W, colsq, colabs = _inputs(d, n_units, group, N, seed)
+        wide = torch.zeros(d, n + 5, device=DEV)
+        wide[:, 1:n + 1] = W
+        Wv = wide[:, 1:n + 1]                                            # pitch n + 5, first element 4 bytes in
+        for Wm in (W, Wv):
+            got_s, got_i = _static_call(kind, n_units, group, Wm, colsq, colabs, N)
+            ref_s, ref_i, _ = api.sp_struct_scores(kind, n_units, group, W=Wm, colsq=colsq, colabs=colabs,
+                                                   inv_tokens=1.0 / N)
+            torch.cuda.synchronize()
+            assert np.array_equal(got_s.cpu().numpy(), ref_s.cpu().numpy())
+            assert abs(got_i.item() - ref_i.item()) <= 1e-12 * abs(ref_i.item())
+            W64 = np64(W)
+            if kind == api.SP_SCORE_WANDA_L2:
+                per = (W64 * W64).sum(0) * np64(colsq)
+                want = np.sqrt(per.reshape(n_units, group).sum(1))
+            else:
+                per = np.abs(W64).sum(0) * np64(colabs) / N
+                want = per.reshape(n_units, group).sum(1)
+            assert relerr(np64(got_s), want) < 1e-6
+
+
 def test_static_scores_reject_sizes_beyond_the_builtin_scratch():
     n_units = api.STATIC_SCORES_MAX_COLS + 8
     W = torch.zeros(2, n_units, device=DEV)
