@@ -233,179 +233,6 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, in
   (void)lcol;
 }
 
-// ---- second form of the diagonal-block kernel: 32-wide sub-blocks.
-// The 128 x 128 block lives in shared memory.  For each of its four 32-column sub-blocks:
-//   1. ONE warp factorises the 32 x 32 diagonal sub-block with the rows in registers (lane = row; the column being
-//      eliminated is exchanged by shuffles) and inverts the factor the same way (lane = column of the inverse);
-//   2. all threads: panel  L21 = A21 M^T  (M = inverse of the sub-block's factor), and the same row operation on the
-//      identity block that becomes inv(L):  B[kb, :] <- M B[kb, :];
-//   3. all threads, 4 x 4 register tiles: trailing update  A22 -= L21 L21^T  and  B[rows below, :] -= L21 B[kb, :].
-// Four sequential sub-block factorisations of about 2 microseconds instead of 32 four-column steps of the first form.
-constexpr int D2_THREADS = 512;
-constexpr int D2_SB = 32;                    // sub-block width
-constexpr int D2_TP = TB + 1;                // pitch of T and B (floats)
-constexpr int D2_MP = D2_SB + 1;             // pitch of the 32-wide scratch blocks
-constexpr size_t D2_SMEM = ((size_t)2 * TB * D2_TP + (size_t)D2_SB * D2_MP + (size_t)(TB - D2_SB) * D2_MP +
-                            (size_t)D2_SB * D2_TP) * sizeof(float);
-
-__global__ void __launch_bounds__(D2_THREADS, 1) chol_diag128_sb_kernel(const float* __restrict__ A, int64_t lda, int nb,
-                                                                        float* __restrict__ dinv, int64_t row0,
-                                                                        int32_t* status) {
-  extern __shared__ __align__(16) float d2_smem[];
-  float (*T)[D2_TP] = reinterpret_cast<float (*)[D2_TP]>(d2_smem);                         // matrix -> factor
-  float (*B)[D2_TP] = reinterpret_cast<float (*)[D2_TP]>(d2_smem + TB * D2_TP);            // identity -> inv(L)
-  float (*Mi)[D2_MP] = reinterpret_cast<float (*)[D2_MP]>(d2_smem + 2 * TB * D2_TP);       // inverse of the sub-block
-  float (*Lp)[D2_MP] = reinterpret_cast<float (*)[D2_MP]>(d2_smem + 2 * TB * D2_TP + D2_SB * D2_MP);   // new panel
-  float (*Bp)[D2_TP] = reinterpret_cast<float (*)[D2_TP]>(d2_smem + 2 * TB * D2_TP + D2_SB * D2_MP +
-                                                          (TB - D2_SB) * D2_MP);           // new block row of B
-  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-  constexpr int NW = D2_THREADS / 32;
-
-  // ---- load (lower triangle; identity on the padding), four rows per warp in flight
-  for (int i0 = warp * 4; i0 < TB; i0 += NW * 4) {
-    float v[4][4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int i = i0 + q, c = lane + 32 * cc;
-        v[q][cc] = (i < nb && c <= i) ? A[(int64_t)i * lda + c] : ((i >= nb && i == c) ? 1.f : 0.f);
-      }
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int i = i0 + q, c = lane + 32 * cc;
-        T[i][c] = v[q][cc];
-        B[i][c] = (i == c) ? 1.f : 0.f;
-      }
-  }
-  __syncthreads();
-
-  for (int kb = 0; kb < TB / D2_SB; ++kb) {
-    const int c0 = kb * D2_SB;
-    // ---- 1. the diagonal sub-block, one warp
-    if (warp == 0) {
-      float r[D2_SB], m[D2_SB], rinv[D2_SB];
-#pragma unroll
-      for (int j = 0; j < D2_SB; ++j) r[j] = T[c0 + lane][c0 + j];
-      int bad = -1;
-#pragma unroll
-      for (int j = 0; j < D2_SB; ++j) {
-        float dj = __shfl_sync(0xffffffffu, r[j], j);
-        if (!(dj > 0.f)) {
-          if (bad < 0) bad = j;
-          dj = 1.f;
-        }
-        const float rs = rsqrt_refined(dj);
-        rinv[j] = rs;
-        const float l = (lane == j ? dj : r[j]) * rs;
-        r[j] = l;
-#pragma unroll
-        for (int k = j + 1; k < D2_SB; ++k) {
-          const float lk = __shfl_sync(0xffffffffu, l, k);
-          r[k] = fmaf(-l, lk, r[k]);
-        }
-      }
-      if (bad >= 0 && lane == 0) report_status(status, SP_ERR_NOT_SPD, (int32_t)(row0 + c0 + bad), 0);
-#pragma unroll
-      for (int j = 0; j < D2_SB; ++j) T[c0 + lane][c0 + j] = (j <= lane) ? r[j] : 0.f;
-      // inverse of the factor: lane c owns column c of M, forward substitution down the rows
-#pragma unroll
-      for (int i = 0; i < D2_SB; ++i) {
-        float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-        for (int k = 0; k < i; ++k) {
-          const float lik = __shfl_sync(0xffffffffu, r[k], i);
-          if (k & 1) acc1 = fmaf(lik, m[k], acc1);
-          else acc0 = fmaf(lik, m[k], acc0);
-        }
-        m[i] = ((i == lane ? 1.f : 0.f) - (acc0 + acc1)) * rinv[i];
-        if (i < lane) m[i] = 0.f;
-      }
-#pragma unroll
-      for (int i = 0; i < D2_SB; ++i) Mi[i][lane] = m[i];
-    }
-    __syncthreads();
-    // ---- 2. panel below the sub-block and block row kb of B, into scratch
-    const int pr = TB - c0 - D2_SB;            // rows below
-    const int bw = c0 + D2_SB;                 // columns of B touched so far
-    for (int e = t; e < pr * D2_SB; e += D2_THREADS) {
-      const int rr = e / D2_SB, j = e % D2_SB;
-      const float* arow = &T[c0 + D2_SB + rr][c0];
-      float acc = 0.f;
-      for (int c = 0; c <= j; ++c) acc = fmaf(arow[c], Mi[j][c], acc);
-      Lp[rr][j] = acc;
-    }
-    for (int e = t; e < D2_SB * bw; e += D2_THREADS) {
-      const int i = e / bw, q = e % bw;
-      float acc = 0.f;
-      for (int c = 0; c <= i; ++c) acc = fmaf(Mi[i][c], B[c0 + c][q], acc);
-      Bp[i][q] = acc;
-    }
-    __syncthreads();
-    // ---- 3. copy the scratch back and update what lies below (4 x 4 tiles)
-    for (int e = t; e < pr * D2_SB; e += D2_THREADS) T[c0 + D2_SB + e / D2_SB][c0 + e % D2_SB] = Lp[e / D2_SB][e % D2_SB];
-    for (int e = t; e < D2_SB * bw; e += D2_THREADS) B[c0 + e / bw][e % bw] = Bp[e / bw][e % bw];
-    const int pt = pr / 4, bt = bw / 4;
-    const int tiles_a = pt * (pt + 1) / 2, tiles = tiles_a + pt * bt;
-    for (int tl = t; tl < tiles; tl += D2_THREADS) {
-      int ti, tj;
-      bool is_a = tl < tiles_a;
-      if (is_a) {
-        ti = (int)((sqrtf(8.f * (float)tl + 1.f) - 1.f) * 0.5f);
-        while ((ti + 1) * (ti + 2) / 2 <= tl) ++ti;
-        while (ti * (ti + 1) / 2 > tl) --ti;
-        tj = tl - ti * (ti + 1) / 2;
-      } else {
-        ti = (tl - tiles_a) / bt;
-        tj = (tl - tiles_a) % bt;
-      }
-      float acc[4][4];
-#pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-#pragma unroll 4
-      for (int j = 0; j < D2_SB; ++j) {
-        float av[4], bv[4];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) av[a] = Lp[4 * ti + a][j];
-#pragma unroll
-        for (int b = 0; b < 4; ++b) bv[b] = is_a ? Lp[4 * tj + b][j] : Bp[j][4 * tj + b];
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
-      }
-      const int rbase = c0 + D2_SB + 4 * ti;
-      if (is_a) {
-        const int cbase = c0 + D2_SB + 4 * tj;
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int b = 0; b < 4; ++b)
-            if (cbase + b <= rbase + a) T[rbase + a][cbase + b] -= acc[a][b];
-      } else {
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int b = 0; b < 4; ++b) B[rbase + a][4 * tj + b] -= acc[a][b];
-      }
-    }
-    __syncthreads();
-  }
-
-  // ---- store inv(L) (zero above the diagonal) and its transpose
-  for (int i = warp; i < TB; i += NW)
-#pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-      const int c = lane + 32 * cc;
-      dinv[i * TB + c] = (c <= i) ? B[i][c] : 0.f;
-      dinv[TB * TB + i * TB + c] = (i <= c) ? B[c][i] : 0.f;
-    }
-}
-
 __device__ __forceinline__ void split3(float v, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
   hi = __float2bfloat16_rn(v);
   const float r1 = v - __bfloat162float(hi);
@@ -779,7 +606,6 @@ __global__ void __launch_bounds__(NM_THREADS)
 
 // two-level blocking of the factorisation (see potrf_lower_tc): systems of at least kOuterMinN rows, outer blocks of
 // kOuterBlocks diagonal blocks
-constexpr bool kDiagSubBlocks = true;     // diagonal blocks by the 32-wide sub-block kernel
 constexpr int64_t kOuterMinN = 12288;
 constexpr int64_t kOuterBlocks = 4;
 
@@ -799,8 +625,6 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
   if (attr_once.run([] {
         cudaError_t e = cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)DIAG_SMEM);
-        if (e == cudaSuccess)
-          e = cudaFuncSetAttribute(chol_diag128_sb_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)D2_SMEM);
         if (e == cudaSuccess)
           e = cudaFuncSetAttribute(chol_next_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NM_SMEM);
         if (e == cudaSuccess)
@@ -841,14 +665,9 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       if (assist && inner_first && kb > 0) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->near_done, 0));
       count_launch();
       ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
-      if (kDiagSubBlocks)
-        chol_diag128_sb_kernel<<<1, D2_THREADS, D2_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
-                                                                   from_scratch ? (int64_t)TB : lda, nb, dk, k0,
-                                                                   status_dev);
-      else
-        chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
-                                                                    from_scratch ? (int64_t)TB : lda, nb, dk, k0,
-                                                                    status_dev);
+      chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
+                                                                  from_scratch ? (int64_t)TB : lda, nb, dk, k0,
+                                                                  status_dev);
       if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     }
     const int64_t rem = n - k0 - nb;
