@@ -4,6 +4,8 @@
     python microbench.py solve [--reps 3 --warm 1]   regularised solves of a C2 step
     python microbench.py mask  [--reps 5 --warm 2]   scores, allocation and top-k as standalone
                                                                            kernels (L2 flushed before every call)
+    python microbench.py mha   [--reps 3 --warm 1]   one outer step of the attention-module updates (Method 2):
+                                                                           d = 2048, 32 heads, sequences of 1024 tokens
     python microbench.py lockstep [--reps 3 --warm 1] lock-step iterations of several C2-wide
                                                                            layers under one global threshold
 
@@ -92,6 +94,33 @@ def solve_cases(reps, warm):
         print("   " + "; ".join(f"{k}: {v['records']} x {1e3 * v['ms'] / max(v['records'], 1):.1f} us"
                                 for k, v in pr.items() if v["records"]), flush=True)
     print("status", st.cpu().tolist())
+
+
+def mha_case(reps, warm):
+    """One sp_mha_step (2 gradient steps of Eq. 85, the closed form of Eq. 86, 2 gradient steps of Eq. 87) on an
+    attention module of workload C2's width: d = 2048, 32 heads of 64, 16 sequences of 1024 tokens, 8 per chunk."""
+    d, H, T, n_seq, chunk = 2048, 32, 1024, 16, 8
+    X = _rnd((n_seq * T, d), torch.bfloat16)
+    W = [(torch.randn(d, d, device=DEV) * (1.0 / d ** 0.5)) for _ in range(4)]
+    mod = api.MhaModule(X, *W, n_heads=H, T=T, seq_chunk=chunk)
+    mod.sp_mha_init(True)
+    p = api.MhaParams(a_steps=2, z_steps=2, seq_chunk=chunk)
+    ms = _timeit(lambda: mod.sp_mha_step(p), reps, warm)
+    api.sp_profile_begin(2)
+    mod.sp_mha_step(p)
+    torch.cuda.synchronize()
+    pr = api.sp_profile_read()
+    api.sp_profile_begin(0)
+    mod.check_status()
+    pairs = n_seq * H
+    # batched products per step: logits (1 + z_steps), P V / R V^T (2 a_steps + 1), gradients (2 z_steps), 3 segments
+    # where an operand is split; counted once each: 2 T^2 d_h flop per pair
+    n_b = (1 + p.z_steps) + (2 * p.a_steps + 1) + 2 * p.z_steps
+    fl = n_b * 2.0 * T * T * (d // H) * pairs + 5 * 2.0 * n_seq * T * d * d
+    print(f"mha step d={d} H={H} T={T} n_seq={n_seq}: {ms:8.3f} ms  {fl / ms / 1e9:7.1f} TFLOP/s (algorithmic)")
+    print("   " + "; ".join(f"{k}: {v['records']} x {1e3 * v['ms'] / max(v['records'], 1):.1f} us"
+                            for k, v in pr.items() if v["records"]), flush=True)
+    print("status", mod.status.cpu().tolist())
 
 
 def _timeit_cold(fn, reps, warm, flush):
@@ -226,7 +255,7 @@ def _hbm_peak():
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "solve", "mask", "lockstep"])
+    ap.add_argument("what", choices=["gemm", "solve", "mask", "lockstep", "mha"])
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warm", type=int, default=2)
     ap.add_argument("--sizes", default="", help="solve: m:n pairs, e.g. 7168:28672,4096:16384 (default: those of a C2 step)")
@@ -241,6 +270,9 @@ def main():
     elif a.what == "lockstep":
         lockstep_cases(a.reps, a.warm)
     else:
+        if a.what == "mha":
+            mha_case(a.reps, a.warm)
+            return
         if a.sizes:
             SOLVE_SIZES[:] = [tuple(int(v) for v in pair.split(":")) for pair in a.sizes.split(",")]
         (gemm_cases if a.what == "gemm" else solve_cases)(a.reps, a.warm)
