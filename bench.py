@@ -364,9 +364,20 @@ def rooflines(cfg, args, prof, steps, peaks):
     if args.chunk == 32768 and not args.dual and cfg.tokens % args.chunk == 0:
         fu_traffic = captured_traffic("fused_update_kernel", f"{cfg.name}:n={cfg.n},k={cfg.k_keep},tokens=32768")
     fu_gbs = fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 if fu["ms"] else 0.0
+    # bytes the two elementwise kernels of the token pass move per token (their own algorithmic counts), against the
+    # minimum of a pass that reads X, Ypre, Z once and writes Z once in the storage type: s (2 d + 2 n)
+    ph = prof.get("prep_h", {"bytes": 0.0})
+    esz = 2.0 if cfg.storage == "bf16" else 4.0
+    per_token = (fu["bytes"] + ph["bytes"]) / max(steps, 1) / cfg.tokens
+    minimum = esz * (2.0 * cfg.d + 2.0 * cfg.n)
     roofline_hbm = {"bound": "hbm", "kernel": "fused_update_kernel", "achieved": fu_gbs, "peak": hbm, "unit": "GB/s",
                     "frac": fu_gbs / hbm, "traffic": fu_traffic,
                     "algorithmic_bytes_per_launch": fu["bytes"] / max(fu["records"], 1), "launches": fu["records"],
+                    "elementwise_bytes_per_token": per_token, "minimum_bytes_per_token": minimum,
+                    "bytes_over_minimum": per_token / minimum,
+                    "bytes_note": "elementwise_bytes_per_token: h gather + fused update (Z kept in fp32, A and a "
+                                  "storage copy of Z written for the accumulator products, D and z1 read); minimum: "
+                                  "X, Ypre, Z read once and Z written once in the storage type",
                     "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback (6.65 TB/s)"}
     breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / steps,
                      **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),

@@ -32,7 +32,9 @@ implemented identically by the CUDA path):
     sparsity r_l"); kept count = n_l - round_half_up(r_l n_l).
 
 Parity unpinned (no statement in the paper fixes them; only self-consistency tests exist): the
-SwiGLU extension `swiglu_zu_update`, and the default values of alpha, beta, rho, T.
+SwiGLU extension `swiglu_zu_update`, the default values of alpha, beta, rho, T, and the multi-head
+attention functions `mha_*` (Method 2 is printed with inconsistent shapes and without step sizes; the
+reading taken is stated above those functions and pinned by mathematics only).
 """
 from __future__ import annotations
 
