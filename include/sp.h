@@ -396,6 +396,16 @@ typedef struct {
   float* Zk;     /* [n_seq * T, d]             auxiliary output of the key projection                              */
   float* P;      /* [n_seq, n_heads, T, T]     auxiliary attention probabilities a_l                               */
   float* Aattn;  /* [n_seq * T, d]             auxiliary concatenated head outputs a_attn_l                        */
+  /* Optional accumulators over all tokens (all five or none; NULL = not computed), rebuilt by sp_mha_init and by
+   * every sp_mha_step from the variables it leaves, for the weight recoveries W = z a^+ of the next outer iteration
+   * ("do for W_Q, W_K, W_V, W_O separately"):  W_Q = R_Q (G_X + rho I)^-1, W_K = R_K (G_X + rho I)^-1 by
+   * sp_ridge_solve;  W_O[:, S] = R_O[:, S] (G_attn[S,S] + rho I)^-1 on the columns of the kept heads by
+   * sp_linear_refit.  fp32 [d, d] each, Gram matrices as full squares. */
+  float* G_X;    /* X^T X                                                                                          */
+  float* R_Q;    /* Zq^T X                                                                                         */
+  float* R_K;    /* Zk^T X                                                                                         */
+  float* G_attn; /* Aattn^T Aattn                                                                                  */
+  float* R_O;    /* Ypre^T Aattn                                                                                   */
 } sp_mha_state;
 
 typedef struct {

@@ -669,3 +669,25 @@ def mha_step(X, Ypre, Wq, Wk, Wv, Wo, Zq, Zk, P, Aattn, p):
     Aattn = mha_attn_update(Ypre, Wo, mha_heads(V, P, p.n_heads))
     Zq, Zk = mha_z_update(Zq, Zk, P, np.asarray(Wq, F64) @ X, np.asarray(Wk, F64) @ X, p)
     return Zq, Zk, P, Aattn
+
+
+def mha_recover_weights(Xs, Ys, Zqs, Zks, As, head_mask, d_head, rho, rho_relative=True):
+    """Weight recovery of one outer step of SparseLLM2 ("prune by importance + recovery solver, do for W_Q, W_K, W_V,
+    W_O separately") from the auxiliary variables of all sequences (lists, tokens as columns), for the projections
+    whose recovery is linear in them:
+      W_Q = Zq X^+ and W_K = Zk X^+ as ridge solves on G_X = sum X X^T, rows of pruned heads set to zero (for a row
+      mask the restricted solution is the row-masked one);  W_O = Ypre Aattn^+ on the columns of the kept heads
+      (restricted ridge solve, ridge of the full system), other columns zero.
+    Returns (W_Q, W_K, W_O)."""
+    d = Xs[0].shape[0]
+    G_X = sum(X @ X.T for X in Xs)
+    R_Q = sum(Zq @ X.T for Zq, X in zip(Zqs, Xs))
+    R_K = sum(Zk @ X.T for Zk, X in zip(Zks, Xs))
+    G_A = sum(A @ A.T for A in As)
+    R_O = sum(Y @ A.T for Y, A in zip(Ys, As))
+    keep = np.repeat(np.asarray(head_mask).astype(bool), d_head)
+    rho1 = effective_ridge(G_X, rho, rho_relative)
+    Wq = np.where(keep[:, None], ridge_solve(R_Q, G_X, rho1), 0.0)
+    Wk = np.where(keep[:, None], ridge_solve(R_K, G_X, rho1), 0.0)
+    Wo = restricted_refit(R_O, G_A, keep, effective_ridge(G_A, rho, rho_relative))
+    return Wq, Wk, Wo

@@ -76,7 +76,9 @@ class SpMhaModule(C.Structure):
 
 
 class SpMhaState(C.Structure):
-    _fields_ = [("Zq", C.c_void_p), ("Zk", C.c_void_p), ("P", C.c_void_p), ("Aattn", C.c_void_p)]
+    _fields_ = [("Zq", C.c_void_p), ("Zk", C.c_void_p), ("P", C.c_void_p), ("Aattn", C.c_void_p),
+                ("G_X", C.c_void_p), ("R_Q", C.c_void_p), ("R_K", C.c_void_p), ("G_attn", C.c_void_p),
+                ("R_O", C.c_void_p)]
 
 
 class SpMhaParams(C.Structure):
@@ -607,7 +609,8 @@ class MhaModule:
     """Owns the device buffers of one attention module (Method 2 auxiliary variables) and forwards to sp_mha_init /
     sp_mha_step.  X: [n_seq * T, d] token-major; Wq, Wk, Wv, Wo: [d, d] ([out, in]), kept in fp32 for the library."""
 
-    def __init__(self, X: torch.Tensor, Wq, Wk, Wv, Wo, n_heads: int, T: int, seq_chunk: int = 0):
+    def __init__(self, X: torch.Tensor, Wq, Wk, Wv, Wo, n_heads: int, T: int, seq_chunk: int = 0,
+                 accumulators: bool = True):
         _require_cuda(X, Wq, Wk, Wv, Wo)
         self.X = X.contiguous()
         self.dev = X.device
@@ -619,6 +622,9 @@ class MhaModule:
         f32 = dict(dtype=torch.float32, device=self.dev)
         self.Zq, self.Zk, self.Aattn = (torch.empty(N, d, **f32) for _ in range(3))
         self.P = torch.empty(self.n_seq, n_heads, T, T, **f32)
+        # accumulators of the weight recoveries (rebuilt by every init / step)
+        self.G_X, self.R_Q, self.R_K, self.G_attn, self.R_O = ((torch.empty(d, d, **f32) for _ in range(5))
+                                                               if accumulators else (None,) * 5)
         self.status = new_status(self.dev)
         self._wsbuf = _ws(lib().sp_mha_workspace_bytes(d, n_heads, T, self.n_seq, seq_chunk, _dt(self.X)), self.dev)
 
@@ -631,7 +637,8 @@ class MhaModule:
                            self.n_heads, self.T, self.n_seq)
 
     def _state(self) -> SpMhaState:
-        return SpMhaState(self.Zq.data_ptr(), self.Zk.data_ptr(), self.P.data_ptr(), self.Aattn.data_ptr())
+        return SpMhaState(self.Zq.data_ptr(), self.Zk.data_ptr(), self.P.data_ptr(), self.Aattn.data_ptr(),
+                          _ptr(self.G_X), _ptr(self.R_Q), _ptr(self.R_K), _ptr(self.G_attn), _ptr(self.R_O))
 
     def sp_mha_init(self, causal: bool = True):
         m, st = self._module(), self._state()

@@ -1172,6 +1172,11 @@ sp_status check_mha(const sp_mha_module* m, const sp_mha_state* st) {
     if (x->rows != m->d || x->cols != m->d || x->ld != m->d) return SP_ERR_SHAPE;
   }
   if (!st->Zq || !st->Zk || !st->P || !st->Aattn) return SP_ERR_INVALID_ARG;
+  {
+    const int have = (st->G_X != nullptr) + (st->R_Q != nullptr) + (st->R_K != nullptr) + (st->G_attn != nullptr) +
+                     (st->R_O != nullptr);
+    if (have != 0 && have != 5) return SP_ERR_INVALID_ARG;
+  }
   // the tensor-core path slices heads out of token-major tensors with 16-byte aligned strides
   if (m->X.dtype == SP_BF16 && ((m->d / m->n_heads) % 8 != 0 || m->T % 8 != 0)) return SP_ERR_ALIGNMENT;
   if (misaligned(st->Zq, 16) || misaligned(st->Zk, 16) || misaligned(st->P, 16) || misaligned(st->Aattn, 16) ||
@@ -1186,6 +1191,34 @@ sp_status project(const MhaPlan& p, MatRef xc, const void* Ws, const sp_mat& W, 
   MatRef o{out, SP_F32, p.d};
   if (p.bf16) return contract_split_weights(Tc, p.d, p.d, xc, Ws, MatRef{W.ptr, SP_F32, W.ld}, o, status, s);
   return contract(Tc, p.d, p.d, 1.0, xc, true, MatRef{W.ptr, SP_F32, W.ld}, true, 0.0, o, o, false, true, false, status, s);
+}
+
+// The accumulators of the weight recoveries over one chunk of tokens (first chunk: overwrite).  bf16 mode: Zq, Zk and
+// Aattn enter as their bf16 roundings (the precision model of the FFN path's accumulators): the hi planes of Zq / Zk
+// kept for the logits, a bf16 copy of Aattn in the buffer of R.
+sp_status mha_accumulate(const MhaPlan& p, const sp_mha_module* m, sp_mha_state* st, MatRef xc, MatRef yc, const float* Zq,
+                         const float* Zk, const float* Aat, int64_t Tc, bool first, int32_t* status, cudaStream_t s) {
+  if (!st->G_X) return SP_OK;
+  (void)m;
+  const int64_t d = p.d;
+  const double acc = first ? 0.0 : 1.0;
+  const bool bf16 = p.bf16, acc64 = !bf16;
+  MatRef zq{Zq, SP_F32, d}, zk{Zk, SP_F32, d}, aa{Aat, SP_F32, d};
+  if (bf16) {
+    // the hi planes of Zq / Zk are current (written by the last update, or by the split at the start of the chunk)
+    CU(split_planes(Aat, Tc * d, p.Rb, 0, s));
+    zq = MatRef{p.Zqs, SP_BF16, d};
+    zk = MatRef{p.Zks, SP_BF16, d};
+    aa = MatRef{p.Rb, SP_BF16, d};
+  }
+  MatRef gx{st->G_X, SP_F32, d}, rq{st->R_Q, SP_F32, d}, rk{st->R_K, SP_F32, d}, ga{st->G_attn, SP_F32, d},
+      ro{st->R_O, SP_F32, d};
+  SPCHK(contract(d, d, Tc, 1.0, xc, false, xc, false, acc, gx, gx, true, acc64, bf16, status, s));
+  SPCHK(contract(d, d, Tc, 1.0, zq, false, xc, false, acc, rq, rq, false, acc64, bf16, status, s));
+  SPCHK(contract(d, d, Tc, 1.0, zk, false, xc, false, acc, rk, rk, false, acc64, bf16, status, s));
+  SPCHK(contract(d, d, Tc, 1.0, aa, false, aa, false, acc, ga, ga, true, acc64, bf16, status, s));
+  SPCHK(contract(d, d, Tc, 1.0, yc, false, aa, false, acc, ro, ro, false, acc64, bf16, status, s));
+  return SP_OK;
 }
 
 constexpr int kSegHH[1] = {0};
@@ -1310,6 +1343,7 @@ static sp_status mha_impl(const sp_mha_module* m, sp_mha_state* st, const sp_mha
         SPCHK(contract(Tc, d, d, 1.0, a, true, MatRef{m->Wo.ptr, SP_F32, d}, true, 0.0, yc, yc, false, true, false,
                        status_dev, s));
       }
+      SPCHK(mha_accumulate(p, m, st, xc, yc, Zq, Zk, Aat, Tc, q0 == 0, status_dev, s));
       continue;
     }
 
@@ -1373,6 +1407,11 @@ static sp_status mha_impl(const sp_mha_module* m, sp_mha_state* st, const sp_mha
       CU(mha_z_update(Zq, Zk, p.Gq, p.Gk, p.Tq, p.Tk, p.eta_z, Tc, (int)d, (int)T, (int)dh, prm->alpha,
                       bf16 ? p.Zqs : nullptr, bf16 ? p.Zks : nullptr, plane, s));
     }
+    SPCHK(mha_accumulate(p, m, st, xc, yc, Zq, Zk, Aat, Tc, q0 == 0, status_dev, s));
+  }
+  if (st->G_X) {
+    CU(symmetrize_lower(st->G_X, d, d, s));
+    CU(symmetrize_lower(st->G_attn, d, d, s));
   }
   return SP_OK;
 }

@@ -116,3 +116,57 @@ def test_mha_argument_errors():
         api.MhaModule(X[:, :80].contiguous().to(DEV), *[w[:80, :80].contiguous().to(DEV) for w in W], n_heads=4,
                       T=40).sp_mha_init()
     assert e.value.code == 4
+
+
+@pytest.mark.parametrize("dtype,d,H,T,n_seq", [(torch.float32, 48, 4, 20, 3), (torch.bfloat16, 128, 4, 72, 3)])
+def test_mha_outer_iterations_match_oracle(dtype, d, H, T, n_seq):
+    """Two outer iterations of SparseLLM2 with one head pruned, teacher-forced per iteration: the accumulators the
+    module holds, the projections recovered from them (W_Q, W_K by ridge solves with masked rows, W_O on the kept heads)
+    and the auxiliary updates that follow, each against the oracle restarted from the GPU's state."""
+    from paper_2510_03246_b200 import pipeline
+    X, W = _case(dtype, d, H, T, n_seq, seed_layer=2)
+    mod = api.MhaModule(X.to(DEV), *[w.to(DEV) for w in W], n_heads=H, T=T, seq_chunk=2)
+    mod.sp_mha_init(True)
+    dh = d // H
+    head_mask = torch.ones(H, dtype=torch.uint8)
+    head_mask[1] = 0
+    hm = head_mask.to(DEV)
+    p_gpu = api.MhaParams(alpha=1.0, beta=1.2, a_steps=2, z_steps=2, causal=True)
+    p_or = O.MhaParams(n_heads=H, alpha=1.0, beta=1.2, a_steps=2, z_steps=2, causal=True)
+    tol = TOL[dtype]
+    Xo = np64(X)
+    Xs = [Xo[q * T:(q + 1) * T].T for q in range(n_seq)]
+    Wv_masked = np64(W[2].float()).copy()
+    Wv_masked[dh:2 * dh] = 0
+    for it in range(2):
+        torch.cuda.synchronize()
+        Yo = np64(mod.Ypre)
+        seqs = lambda t: [np64(t)[q * T:(q + 1) * T].T for q in range(n_seq)]
+        Zqs, Zks, As, Ys = seqs(mod.Zq), seqs(mod.Zk), seqs(mod.Aattn), [Yo[q * T:(q + 1) * T].T for q in range(n_seq)]
+        Ps = [np64(mod.P[q]) for q in range(n_seq)]
+        # accumulators left by the previous call
+        assert relerr(np64(mod.G_X), sum(x @ x.T for x in Xs)) < tol
+        assert relerr(np64(mod.R_Q), sum(z @ x.T for z, x in zip(Zqs, Xs))) < tol
+        assert relerr(np64(mod.R_K), sum(z @ x.T for z, x in zip(Zks, Xs))) < tol
+        assert relerr(np64(mod.G_attn), sum(a @ a.T for a in As)) < tol
+        assert relerr(np64(mod.R_O), sum(y @ a.T for y, a in zip(Ys, As))) < tol
+        acc = {k: np64(getattr(mod, k)) for k in ("G_X", "R_Q", "R_K", "G_attn", "R_O")}
+        pipeline.mha_outer_iterations(mod, hm, 1, p_gpu, rho=0.1)
+        torch.cuda.synchronize()
+        # weights: the oracle's recovery from the GPU's accumulators (teacher-forced)
+        keep = np.repeat(head_mask.numpy().astype(bool), dh)
+        rho1 = O.effective_ridge(acc["G_X"], 0.1, True)
+        Wq_or = np.where(keep[:, None], O.ridge_solve(acc["R_Q"], acc["G_X"], rho1), 0.0)
+        Wk_or = np.where(keep[:, None], O.ridge_solve(acc["R_K"], acc["G_X"], rho1), 0.0)
+        Wo_or = O.restricted_refit(acc["R_O"], acc["G_attn"], keep, O.effective_ridge(acc["G_attn"], 0.1, True))
+        assert relerr(np64(mod.Wq), Wq_or) < tol and relerr(np64(mod.Wk), Wk_or) < tol, "W_Q / W_K"
+        assert relerr(np64(mod.Wo), Wo_or) < tol, "W_O"
+        assert np.all(np64(mod.Wq)[~keep] == 0) and np.all(np64(mod.Wo)[:, ~keep] == 0) and np.all(np64(mod.Wv)[~keep] == 0)
+        assert relerr(np64(mod.Wv), Wv_masked) < 1e-7
+        # auxiliary updates with the GPU's weights
+        Wg = [np64(w) for w in (mod.Wq, mod.Wk, mod.Wv, mod.Wo)]
+        for q in range(n_seq):
+            r = slice(q * T, (q + 1) * T)
+            Zq, Zk, P, A = O.mha_step(Xs[q], Ys[q], *Wg, Zqs[q], Zks[q], Ps[q], As[q], p_or)
+            assert relerr(np64(mod.P[q]), P) < tol and relerr(np64(mod.Aattn[r]).T, A) < tol
+            assert relerr(np64(mod.Zq[r]).T, Zq) < tol and relerr(np64(mod.Zk[r]).T, Zk) < tol

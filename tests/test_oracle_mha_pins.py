@@ -159,3 +159,24 @@ def test_special_cases():
     assert np.abs(P[0] - np.eye(T)).max() < 1e-9 and np.allclose(A, V, atol=1e-7)
     # the step of Eq. (87) shrinks with the size of the iterate and never exceeds the step of its quadratic part
     assert O.mha_z_step_size(Xs, Xs, 1.0, 1.0, 1.0) < O.mha_z_step_size(0.1 * Xs, 0.1 * Xs, 1.0, 1.0, 1.0) < 0.5
+
+
+def test_recovered_projections_reproduce_the_pretrained_ones_and_respect_the_head_mask():
+    """W = z a^+ for the projections that are linear in the auxiliary variables: from the pre-trained state, all heads
+    kept and a vanishing ridge, the recoveries return W_Q, W_K, W_O (X and the head outputs have full row rank over the
+    sequences); with a head removed its rows of W_Q, W_K and its columns of W_O are zero, the other rows of W_Q, W_K
+    are unchanged, and the kept columns of W_O are the least-squares fit on those columns alone."""
+    rng = np.random.default_rng(8)
+    d, T, h, dh, n_seq = 8, 9, 2, 4, 3
+    W = [0.7 * rng.standard_normal((d, d)) for _ in range(4)]
+    Xs = [rng.standard_normal((d, T)) for _ in range(n_seq)]
+    fw = [O.mha_forward(X, *W, h, True) for X in Xs]
+    Zqs, Zks, As, Ys = [f[0] for f in fw], [f[1] for f in fw], [f[4] for f in fw], [f[5] for f in fw]
+    Wq, Wk, Wo = O.mha_recover_weights(Xs, Ys, Zqs, Zks, As, [1, 1], dh, 1e-12, False)
+    assert np.allclose(Wq, W[0], atol=1e-8) and np.allclose(Wk, W[1], atol=1e-8) and np.allclose(Wo, W[3], atol=1e-7)
+    Wq1, Wk1, Wo1 = O.mha_recover_weights(Xs, Ys, Zqs, Zks, As, [0, 1], dh, 1e-12, False)
+    assert np.all(Wq1[:dh] == 0) and np.all(Wk1[:dh] == 0) and np.all(Wo1[:, :dh] == 0)
+    assert np.allclose(Wq1[dh:], W[0][dh:], atol=1e-8) and np.allclose(Wk1[dh:], W[1][dh:], atol=1e-8)
+    A_all, Y_all = np.concatenate(As, axis=1), np.concatenate(Ys, axis=1)
+    fit = np.linalg.lstsq(A_all[dh:].T, Y_all.T, rcond=None)[0].T          # Ypre ~ W_O[:, kept] Aattn[kept]
+    assert np.allclose(Wo1[:, dh:], fit, atol=1e-7)
