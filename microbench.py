@@ -193,6 +193,15 @@ def mask_cases(reps, warm, hbm_gbs):
         kk = torch.full((L,), n // 2, dtype=torch.int64, device=DEV)
         ms = _timeit_cold(lambda: api.sp_apply_mask_batched(sc, kk), reps, warm, flush)
         line(f"top-k batched  L = {L}, n = {n}", ms, 5.0 * L * n)
+    # one threshold over all layers (Algorithm 3): the many-CTA select, and the one-CTA select over the same keys
+    for L, n in ((4, 8192), (24, 8192), (32, 16384), (32, 28672)):
+        sc = torch.randn(L, n, device=DEV)
+        msk = torch.empty(L, n, dtype=torch.uint8, device=DEV)
+        ms = _timeit_cold(lambda: api.sp_apply_mask_global(sc, 0.4, 1, mask_out=msk), reps, warm, flush)
+        line(f"global threshold, many CTAs  L = {L}, n = {n}", ms, 25.0 * L * n)
+        K = int(0.4 * n * L)
+        ms = _timeit_cold(lambda: api.sp_apply_mask(sc.view(-1), K, mask_out=msk.view(-1)), reps, warm, flush)
+        line(f"global threshold, one CTA    L = {L}, n = {n}", ms, 25.0 * L * n)
 
 
 def lockstep_cases(reps, warm, layers=4, tokens=32768):

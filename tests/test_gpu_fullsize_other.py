@@ -143,8 +143,8 @@ def test_mask_and_token_update(run):
     got = run["Z1_rows"].T
     if run["gated"]:
         Znew = O.swiglu_zu_update(A, g, z1, p.alpha, p.beta)
-        assert relerr(got, Znew) < TOLB
     else:
         Znew = O.z_select(z0, z1, z2, A, p.alpha, p.beta, p.z_rule)
-        assert relerr(got, Znew) < TOLB
+    print(f"{cfg.name}: max relative error of Z on the sampled tokens {relerr(got, Znew):.2e} (tolerance {TOLB:.0e})")
+    assert relerr(got, Znew) < TOLB
     assert run["report"]["kept"] == cfg.k_keep and run["report"]["res_act"] >= 0.0
