@@ -364,7 +364,7 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
       At[k][i] = xv[q].x; At[k + 1][i] = xv[q].y; At[k + 2][i] = xv[q].z; At[k + 3][i] = xv[q].w;
     }
   }
-  // (the verdict is made uniform over the block: a thread whose wait ran out must not leave while others go on)
+  // (the outcome is made uniform over the block: a thread whose wait ran out must not leave while others go on)
   const bool staged = __syncthreads_and(stage_block_wait(bar, 0) ? 1 : 0) != 0;
   if (!staged) {   // the copies did not land in time: report and leave X untouched
     if (t == 0) report_status(status, SP_ERR_TIMEOUT, (int32_t)blockIdx.x, 10);

@@ -572,14 +572,15 @@ def test_admm_step_bf16_without_objective(chunk, rule, dual):
         _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
 
 
-def test_admm_step_with_z1_computed_ahead():
+@pytest.mark.parametrize("dual", [False, True])
+def test_admm_step_with_z1_computed_ahead(dual):
     """Same step with the optional workspace tail: z1 of all tokens is computed on the side stream beside the
-    kept-support recovery (the configuration bench.py runs)."""
+    kept-support recovery (the configuration bench.py runs), without and with the dual variable."""
     cfg = SMALL_BF16
-    mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=cfg.k_keep)
+    mod, X, W1, W2 = _make_module(cfg, dual=dual, chunk=512, overlap_k=cfg.k_keep)
     mod.sp_ffn_init()
-    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, token_chunk=512)
-    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep)
+    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, token_chunk=512, dual_mode=dual)
+    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=cfg.k_keep, dual_mode=dual)
     audit = []
     for it in range(3):
         _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
