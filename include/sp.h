@@ -315,7 +315,8 @@ sp_status sp_apply_mask_batched(const float* scores, int64_t ld_scores, int64_t 
  * fewer than min_keep units keeps its own min_keep best instead (as printed the algorithm can empty a layer).
  * mask_out: u8, row l at mask_out + l * ld_mask; tau_out (optional): the K-th largest score; kept_out: int64 [L] kept
  * units per layer after the repair (device).  The select runs on many CTAs (four histogram passes over the keys), so
- * L * n_units is not limited by one CTA's shared memory.  Workspace: sp_apply_mask_global_bytes(n_units, L).
+ * L * n_units is not limited by one CTA's shared memory; up to 47104 keys in contiguous rows are selected by one CTA
+ * instead, which is faster there (same result).  Workspace: sp_apply_mask_global_bytes(n_units, L).
  * Errors: SP_ERR_INVALID_ARG (null pointers, keep_fraction outside [0, 1]), SP_ERR_SHAPE, SP_ERR_WORKSPACE,
  * SP_ERR_ALIGNMENT (workspace not 256-byte aligned). */
 sp_status sp_apply_mask_global(const float* scores, int64_t ld_scores, int64_t n_units, int32_t L, double keep_fraction,

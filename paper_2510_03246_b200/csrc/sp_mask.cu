@@ -1210,6 +1210,21 @@ __global__ void gsel_repair_list_kernel(int32_t* counts, int L, int64_t min_keep
   counts_out[l] = fix ? mk : counts[l];
 }
 
+// counts[l] = kept units of layer l of an L x n mask (rows ld apart); one block per layer
+__global__ void __launch_bounds__(256) mask_row_counts_kernel(const uint8_t* __restrict__ mask, int64_t n, int64_t ld,
+                                                              int32_t* __restrict__ counts) {
+  __shared__ int sm[256];
+  int c = 0;
+  for (int64_t j = threadIdx.x; j < n; j += 256) c += mask[(int64_t)blockIdx.x * ld + j] != 0;
+  sm[threadIdx.x] = c;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) counts[blockIdx.x] = sm[0];
+}
+
 size_t global_select_scratch_bytes(int64_t total, int L) {
   const int64_t nblocks = ceil_div(total > 0 ? total : 1, (int64_t)kGselPerBlock);
   return align_up((size_t)(kGselState + nblocks) * 4, 256) + align_up((size_t)L * 4, 256) + align_up((size_t)L * 8, 256);
@@ -1228,7 +1243,14 @@ cudaError_t global_select(const float* scores, int64_t ld_scores, int64_t n, int
   ProfScope prof(PK_TOPK, 0.0, (double)total * 25.0, stream);
   cudaError_t e = cudaMemsetAsync(counts, 0, (size_t)L * 4, stream);
   if (e != cudaSuccess) return e;
-  if (K <= 0 || K >= total) {      // nothing or everything kept: no threshold to find
+  constexpr int64_t kOneCtaKeys = 47104;      // what the one-CTA select keeps in shared memory
+  if (K > 0 && K < total && total <= kOneCtaKeys && ld_scores == n && ld_mask == n) {
+    // few keys in one contiguous array: the one-CTA select over the concatenation is faster than the launch chain
+    e = topk_select(scores, total, K, mask, tau, nullptr, stream);
+    if (e != cudaSuccess) return e;
+    count_launch();
+    mask_row_counts_kernel<<<L, 256, 0, stream>>>(mask, n, ld_mask, counts);
+  } else if (K <= 0 || K >= total) {      // nothing or everything kept: no threshold to find
     e = cudaMemset2DAsync(mask, (size_t)ld_mask, K > 0 ? 1 : 0, (size_t)n, (size_t)L, stream);
     if (e != cudaSuccess) return e;
     count_launch();

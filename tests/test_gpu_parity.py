@@ -809,16 +809,18 @@ def test_apply_mask_global_matches_oracle(L, n, frac, min_keep):
     ld = n + 8                                                          # rows with a pitch
     buf = torch.zeros(L, ld, device=DEV)
     buf[:, :n] = S.to(DEV)
-    mask, tau, kept = api.sp_apply_mask_global(buf[:, :n], frac, min_keep)
-    torch.cuda.synchronize()
     m_or, c_or, tau_or = O.global_threshold_masks(S.double().numpy(), frac, min_keep=min_keep)
-    assert np.array_equal(mask.cpu().numpy(), m_or)
-    assert kept.cpu().tolist() == c_or.tolist()
     K = int(np.floor(frac * n * L + 1e-9))
-    if 0 < K < n * L:
-        assert tau.item() == tau_or or (np.isnan(tau_or) and np.isnan(tau.item()))
-    if min_keep == 0:
-        assert int(mask.sum().item()) == K
+    # pitched rows always take the many-CTA select; contiguous rows with few keys take the one-CTA select
+    for scores in (buf[:, :n], S.to(DEV).contiguous()):
+        mask, tau, kept = api.sp_apply_mask_global(scores, frac, min_keep)
+        torch.cuda.synchronize()
+        assert np.array_equal(mask.cpu().numpy(), m_or)
+        assert kept.cpu().tolist() == c_or.tolist()
+        if 0 < K < n * L:
+            assert tau.item() == tau_or or (np.isnan(tau_or) and np.isnan(tau.item()))
+        if min_keep == 0:
+            assert int(mask.sum().item()) == K
 
 
 def test_allocate_sparsity_grid_matches_oracle():
