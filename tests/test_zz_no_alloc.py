@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import struprune_oracle as O
 from paper_2510_03246_b200 import api, synth
 from tests._util import np64, relerr
 
@@ -56,7 +57,7 @@ def test_static_scores_units_that_straddle_column_groups_and_unaligned_weights()
     """Units whose width does not divide the kernel's 128-column groups (3 and 96 columns per unit) take the path that
     gathers a unit's column values across groups; a weight view with a pitch larger than its width and a start that is
     not 16-byte aligned takes the scalar loads.  Each runs right after a call that left other values in the scratch,
-    and is also checked against the definition evaluated in fp64 on the host."""
+    and is also checked against the oracle's scores of the same inputs."""
     first = _inputs(300, 2500, 1, 40, 21)
     _static_call(api.SP_SCORE_WANDA_L2, 2500, 1, *first, 40)            # dirties the scratch
     for kind, d, n_units, group, N, seed in ((api.SP_SCORE_WANDA_L2, 210, 333, 3, 50, 22),
@@ -73,14 +74,11 @@ def test_static_scores_units_that_straddle_column_groups_and_unaligned_weights()
             torch.cuda.synchronize()
             assert np.array_equal(got_s.cpu().numpy(), ref_s.cpu().numpy())
             assert abs(got_i.item() - ref_i.item()) <= 1e-12 * abs(ref_i.item())
-            W64 = np64(W)
             if kind == api.SP_SCORE_WANDA_L2:
-                per = (W64 * W64).sum(0) * np64(colsq)
-                want = np.sqrt(per.reshape(n_units, group).sum(1))
+                want, want_i = O.wanda_scores(np64(W), colsq=np64(colsq), kind="l2", group=group)
             else:
-                per = np.abs(W64).sum(0) * np64(colabs) / N
-                want = per.reshape(n_units, group).sum(1)
-            assert relerr(np64(got_s), want) < 1e-6
+                want, want_i = O.wanda_scores(np64(W), colabs_mean=np64(colabs) / N, kind="l1", group=group)
+            assert relerr(np64(got_s), want) < 1e-6 and abs(got_i.item() - want_i) < 1e-6 * abs(want_i)
 
 
 def test_static_scores_reject_sizes_beyond_the_builtin_scratch():
