@@ -193,13 +193,22 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": steps, "warmup": args.warmup, "ms_per_step": 1e3 * full, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": workload_name(cfg)},
+            "config": config_dict(cfg, args, int(os.environ.get("WORLD_SIZE", 1)), args.shard == "tokens"),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                              "implementation": "numpy fp64 (LAPACK / BLAS on all threads counted in cores)",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "wall_s": time.perf_counter() - t0}
     print(json.dumps(line))
+
+
+def config_dict(cfg, args, world: int, by_tokens: bool) -> dict:
+    """The `config` object of the JSON line; both arms describe the workload with the same one."""
+    return {"workload": workload_name(cfg), "token_chunk": args.chunk, "dual_mode": bool(args.dual),
+            "reproducible": bool(args.reproducible),
+            "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
+            "parallelism": (f"tokens x{world} of one module (accumulators all-reduced once per iteration)"
+                            if by_tokens else f"modules x{world} (independent, no collective)")}
 
 
 def workload_name(cfg) -> str:
@@ -560,11 +569,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "strong" if by_tokens else "weak",
             "vs_baseline": None, "dtype": DTYPE_NAME[cfg.storage], "data": "synthetic",
-            "config": {"workload": workload_name(cfg), "token_chunk": args.chunk, "dual_mode": bool(args.dual),
-                       "reproducible": bool(args.reproducible),
-                       "l2": "inputs larger than L2 (Z alone is %.1f GB)" % (cfg.tokens * cfg.n * 4 / 1e9),
-                       "parallelism": (f"tokens x{world} of one module (accumulators all-reduced once per iteration)"
-                                       if by_tokens else f"modules x{world} (independent, no collective)")},
+            "config": config_dict(cfg, args, world, by_tokens),
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e,
             "cpu_baseline": cpu, "fixed_mask": fixed, "workloads": workloads,
             "profiled_ms_per_step": ms_prof / args.steps, "graph_replay_ms_per_step": graph_ms,
