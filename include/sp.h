@@ -146,6 +146,8 @@ typedef struct {
   double a_sq;      /* |A|^2                                                                                      */
   double rho1_eff, rho2_eff; /* ridge terms actually used                                                         */
   double kept;      /* number of kept units                                                                       */
+  double factor_reused; /* 1: the recovery on the kept support was one backward sweep with the leading block of the
+                           unrestricted factor (the new mask kept the channels of the previous one); else 0         */
 } sp_step_report;
 
 /* Inputs of sp_struct_scores; only the fields of the chosen kind are read. */
@@ -203,6 +205,11 @@ sp_status sp_ffn_cache_input_inverse(const sp_ffn_module* m, sp_ffn_state* st, d
  *      which equals a_l = (alpha W2^T W2 + beta I)^-1 (alpha W2^T Ypre + beta h) of Appendix A.1;
  *      z^(1) = X W1^T, z^(2) = (beta (A+U) + alpha z^(1))/(alpha+beta); select; U += A - phi(Z_new);
  *      G_A, R1, R2, absA are rebuilt from the new A and Z.
+ * Steps 1 and 4 share a factorisation when they can (bf16 storage, refit): the system of step 1 is factorised with
+ * the channels that st->mask kept BEFORE the call in front, so the leading block of its factor is the factor of
+ * G_A[S',S'] + rho2 I for that support S'.  When the mask of step 3 keeps exactly those channels, step 4 is a backward
+ * sweep with that block (rep->factor_reused = 1); otherwise the restricted system is factorised.  The decision is
+ * taken on the device; both ways give the same restricted ridge solution up to rounding.
  * In/out: st (Z, U, accumulators, mask); out: st->W1, st->W2, st->scores, st->importance, *rep_dev.
  * rep_dev and status_dev are device pointers (status_dev: int32[4], must be zeroed by the caller beforehand).
  * Workspace: sp_workspace_bytes(SP_WS_ADMM_STEP, d, n, N, token_chunk, dtype).

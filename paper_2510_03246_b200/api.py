@@ -86,7 +86,7 @@ class SpMhaParams(C.Structure):
                 ("eta_z", C.c_double), ("causal", C.c_int32), ("reserved", C.c_int32), ("seq_chunk", C.c_int64)]
 
 
-REPORT_FIELDS = ["res_act", "res_out", "res_in", "z_sq", "a_sq", "rho1_eff", "rho2_eff", "kept"]
+REPORT_FIELDS = ["res_act", "res_out", "res_in", "z_sq", "a_sq", "rho1_eff", "rho2_eff", "kept", "factor_reused"]
 
 _lib = None
 

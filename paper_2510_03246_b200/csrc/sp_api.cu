@@ -133,14 +133,22 @@ SolveBufs carve_solve(Carver& c, int64_t nmax, int64_t mmax, size_t tsize) {
   return b;
 }
 
+// Copy of the forward-substituted right-hand sides on the leading k columns of a system (tensor-core path): with it
+// and the factor's leading block the system restricted to its first k unknowns is solved by a backward sweep alone.
+struct LeadSave {
+  float* Y;       // [m, kpad] dense, columns k..kpad zero
+  int64_t k, kpad;
+};
+
 // W[m, n_full] = R[:, idx] (G[idx, idx] + rho I)^-1 scattered back to the idx columns (idx == nullptr: identity).
+// conditional: the call runs under a SkipScope (its work is not counted in the profile's flops).
 template <typename T>
 sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, int64_t m, int64_t n_full,
                      const int32_t* idx, int64_t k, const double* rho_dev, float* W, int64_t ldw, SolveBufs& b,
                      int32_t* status, cudaStream_t stream, const SolveAssist* assist = nullptr,
-                     bool split_lookahead = false) {
+                     bool split_lookahead = false, const LeadSave* save = nullptr, bool conditional = false) {
   const int64_t nn = idx ? k : n_full;
-  ProfScope prof(PK_SOLVE, (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
+  ProfScope prof(PK_SOLVE, conditional ? 0.0 : (double)nn * nn * nn / 3.0 + 2.0 * (double)m * nn * nn, 0.0, stream);
   T* Gs = reinterpret_cast<T*>(b.Gs);
   T* dinv = reinterpret_cast<T*>(b.dinv);
   T* Rs = Gs + (size_t)nn * nn;     // the right-hand sides sit right below the system matrix, same leading dimension
@@ -151,6 +159,7 @@ sp_status ridge_core(const float* R, int64_t ldr, const float* G, int64_t ldg, i
     // proper is then only the backward sweep
     CU(gather_cols<T>(R, ldr, idx, m, nn, Rs, nn, stream));
     SPCHK(potrf_lower_tc(Gs, nn, nn, dinv, b.P, status, stream, assist, m, split_lookahead));
+    if (save) CU(copy_cols_padded(Rs, nn, m, save->k, save->kpad, save->Y, stream));
     SPCHK(potrs_right_tc(Rs, m, nn, nn, b.P, dinv, b.Xs, status, stream, assist, true, Gs, nn));
   } else {
     CU(potrf_lower<T>(Gs, nn, nn, dinv, status, stream));
@@ -236,6 +245,8 @@ struct AdmmPlan {
   SolveBufs sbA;               // buffers of the W1 recovery (system d, n right-hand sides), which runs concurrently
   float *W1t, *W2t, *Qt, *T0, *Cf;
   float *W2cf, *W1c;           // compact fp32 copies on the kept support: W2[:, S] ([d, kp]) and W1[S, :] ([k, d])
+  int32_t* perm;               // channels ordered "kept by the previous mask first" (reuse of the G_A factor)
+  int32_t* reuse_flags;        // [0] support changed, [1] support unchanged, [2] kept count of the previous mask
   int32_t* grp_base;           // kept-channel map of the elementwise kernels
   uint8_t* grp_mask;
   void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
@@ -271,6 +282,8 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.Cf = c.take<float>((size_t)d * d);
   p.W2cf = c.take<float>((size_t)n * d + 8 * (size_t)d);
   p.W1c = p.bf16 ? nullptr : c.take<float>((size_t)n * d);
+  p.perm = c.take<int32_t>((size_t)n);
+  p.reuse_flags = c.take<int32_t>(4);
   p.grp_base = c.take<int32_t>((size_t)ceil_div(n, (int64_t)8));
   p.grp_mask = c.take<uint8_t>((size_t)ceil_div(n, (int64_t)8));
   p.W1b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // hi | lo split of W1
@@ -793,6 +806,17 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   SideStream* side = side_stream();
   cudaStream_t sa = side ? side->stream : s;
   JoinOnExit join_guard{side, s};
+  // Reuse of the factorisation for the recovery on the kept support (tensor-core path): the unrestricted system is
+  // solved with the channels that the mask kept so far in front.  The leading block of that factor is the factor of
+  // the restricted system of those channels, and the leading columns of the forward-substituted right-hand sides are
+  // its forward substitution.  When the new top-k selects the same channels (a device flag, no host round trip), the
+  // restricted recovery is one backward sweep; otherwise the restricted system is factorised as usual.  The kernels
+  // of both branches are always queued and return at once when their branch is not taken.
+  const bool skip_scores = prm->skip_scores != 0;   // fixed mask: W2~ and the scores serve nothing
+  const int64_t k_lead = chol_tc_pad(k);
+  const bool reuse = bf16 && !skip_scores && !scores_only && prm->refit && k < n && k_lead <= n;
+  const LeadSave lead{p.W2cf, k, k_lead};     // W2cf is free until the operands of the token pass are built
+  if (reuse) CU(mask_to_perm(st->mask, n, p.perm, p.reuse_flags + 2, s));
   if (side) {
     CU(cudaEventRecord(side->fork, s));
     CU(cudaStreamWaitEvent(sa, side->fork, 0));
@@ -800,12 +824,11 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   // The long chain (W2, on the caller's stream) is queued first: queuing the W1 chain takes the host more than half a
   // millisecond, during which the caller's stream would otherwise sit empty.  (Without a side stream both run on
   // the caller's stream and the order does not matter.)
-  const bool skip_scores = prm->skip_scores != 0;   // fixed mask: W2~ and the scores serve nothing
   CU(effective_ridge(st->G_A, n, n, prm->rho, prm->rho_relative, rho2, s));
   if (skip_scores) {
   } else if (bf16) {
-    SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
-                            side ? &side->assist_main : nullptr));
+    SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, reuse ? p.perm : nullptr, n, rho2, p.W2t, n, p.sb, status_dev,
+                            s, side ? &side->assist_main : nullptr, false, reuse ? &lead : nullptr));
   } else {
     SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, nullptr, n, rho2, p.W2t, n, p.sb, status_dev, s,
                              side ? &side->assist_main : nullptr));
@@ -862,6 +885,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   // ---- 3. top-k mask
   if (prm->reselect_mask) CU(topk_select(st->scores, n, k, st->mask, nullptr, p.sb.idx, s));
   else CU(mask_to_index(st->mask, n, p.sb.idx, s));
+  if (reuse) CU(mask_changed(st->mask, p.perm, p.reuse_flags + 2, k, p.reuse_flags, s));
 
   // ---- 4. masked weights: W1 = diag(M) W1~ ; W2 = recovery on the kept support (or M (.) W2~)
   if (!joined) { CU(cudaStreamWaitEvent(s, side->join, 0)); joined = true; }
@@ -888,10 +912,27 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   if (prm->refit) {
     // beside the z1 products the lookahead kernel of the factorisation runs as two launches of independent CTAs: a
     // cluster of 8 would wait for a free group of SMs while the persistent GEMM CTAs hold most of them
-    if (bf16) SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
-                                      side ? &side->assist_main : nullptr, z1_ahead));
-    else SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
-                                      side ? &side->assist_main : nullptr));
+    if (reuse) {
+      {
+        SkipScope skip_if_changed(p.reuse_flags + 0);
+        ProfScope prof(PK_SOLVE, 2.0 * (double)d * k_lead * k_lead, 0.0, s);
+        SPCHK(potrs_right_tc(lead.Y, d, k_lead, k_lead, p.sb.P, reinterpret_cast<const float*>(p.sb.dinv), p.sb.Xs,
+                             status_dev, s, side ? &side->assist_main : nullptr, true,
+                             reinterpret_cast<const float*>(p.sb.Gs), n, n));
+        CU(scatter_cols<float>(lead.Y, k_lead, p.sb.idx, d, k, n, st->W2, n, s));
+      }
+      {
+        SkipScope skip_if_unchanged(p.reuse_flags + 1);
+        SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
+                                side ? &side->assist_main : nullptr, z1_ahead, nullptr, true));
+      }
+    } else if (bf16) {
+      SPCHK(ridge_core<float>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
+                              side ? &side->assist_main : nullptr, z1_ahead));
+    } else {
+      SPCHK(ridge_core<double>(st->R2, n, st->G_A, n, d, n, p.sb.idx, k, rho2, st->W2, n, p.sb, status_dev, s,
+                               side ? &side->assist_main : nullptr));
+    }
   } else {
     CU(cudaMemcpyAsync(st->W2, p.W2t, (size_t)d * n * sizeof(float), cudaMemcpyDeviceToDevice, s));
     CU(zero_pruned(st->mask, 1, nullptr, 0, 0, 0, st->W2, d, n, n, s));
@@ -959,7 +1000,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
 
   // ---- 5b. token pass
   if (z1_ahead) CU(cudaStreamWaitEvent(s, side->z1_done, 0));
-  if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, s));
+  if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, reuse ? p.reuse_flags + 1 : nullptr, s));
   const size_t esz = bf16 ? 2 : 4;
   MatRef ga{st->G_A, SP_F32, n}, r1{st->R1, SP_F32, d}, r2{st->R2, SP_F32, n};
   for (int64_t t0 = 0, ci = 0; t0 < N; t0 += p.chunk, ++ci) {

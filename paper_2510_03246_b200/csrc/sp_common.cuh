@@ -33,6 +33,15 @@ void count_launch(int n = 1);
 bool reproducible_mode();
 // sp_set_wait_budget: clock cycles a barrier wait of the tensor-core GEMM may take (0: the built-in default)
 long long wait_budget_cycles();
+// Device-side conditional work without a host round trip: while a SkipScope is alive on the calling host thread, the
+// launchers that honour it (the kernels of the regularised solves, the tensor-core GEMM, the column gathers and
+// scatters) pass its flag to their kernels, and every such kernel returns at once when the flag is non-zero at the
+// time it starts.  The flag is written by an earlier kernel of the same stream order.  Scopes do not nest.
+const int32_t* skip_flag();
+struct SkipScope {
+  explicit SkipScope(const int32_t* flag);
+  ~SkipScope();
+};
 // Brackets the kernels launched during its lifetime with a CUDA event pair on `stream` when profiling is enabled.
 // Scopes nest: only the outermost one records, so a phase scope absorbs the kernels launched inside it.
 struct ProfScope {
@@ -175,7 +184,10 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* P,
 // column inside the panel kernel instead of by a GEMM of its own.
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* P, const float* dinv, void* Xs,
                          int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist = nullptr,
-                         bool forward_done = false, const float* Lf = nullptr, int64_t ldl = 0);
+                         bool forward_done = false, const float* Lf = nullptr, int64_t ldl = 0,
+                         int64_t n_factor = 0);
+// n_factor > n: the factor in P / dinv / Lf is that of a larger system of n_factor rows and the solve uses its leading
+// n x n block, which is the factor of the system's leading block (n a multiple of kCholTcNB).
 
 // ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
@@ -210,6 +222,9 @@ cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_d
 template <typename T>
 cudaError_t load_spd_gather(const float* G, int64_t ldg, const int32_t* idx, int64_t k, const double* rho_dev, T* dst,
                             int64_t ldd, cudaStream_t stream);
+// dst [rows, kpad] (dense) = the first k columns of src followed by zero columns
+cudaError_t copy_cols_padded(const float* src, int64_t lds, int64_t rows, int64_t k, int64_t kpad, float* dst,
+                             cudaStream_t stream);
 // dst[i, a] = (T) src[i, idx[a]]  (idx == nullptr: identity)
 template <typename T>
 cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
@@ -267,8 +282,9 @@ cudaError_t reduce_report(const double* partial, int nblocks, sp_step_report* re
 constexpr int kSumsqBlocks = 592;
 cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t cols, double scale, double* out,
                              bool accumulate, double* scratch, cudaStream_t stream);
+// reused (device, may be null): non-zero when the recovery on the kept support reused the unrestricted factor
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
-                        cudaStream_t stream);
+                        const int32_t* reused, cudaStream_t stream);
 // relu + storage conversion for the init pass: A = phi(Z) -> storage dtype, and |A| column partials
 // gate_io (gated modules): holds the gate pre-activation on entry and SiLU of it on return; A = gate * Z then
 cudaError_t launch_init_act(const float* Z, float* gate_io, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T,
@@ -330,6 +346,11 @@ cudaError_t global_select(const float* scores, int64_t ld_scores, int64_t n, int
                           uint8_t* mask, int64_t ld_mask, float* tau, int64_t* counts_out, void* scratch,
                           cudaStream_t stream);
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream);
+// perm[0..n) = the kept channels of `mask` in ascending order followed by the pruned ones; count[0] = kept channels
+cudaError_t mask_to_perm(const uint8_t* mask, int64_t n, int32_t* perm, int32_t* count, cudaStream_t stream);
+// flags[0] = 1 when the kept channels of `mask` are not exactly perm[0..k) with count_old[0] == k; flags[1] = 1 - flags[0]
+cudaError_t mask_changed(const uint8_t* mask, const int32_t* perm, const int32_t* count_old, int64_t k, int32_t* flags,
+                         cudaStream_t stream);
 cudaError_t zero_pruned(const uint8_t* mask, int group, float* W_rows, int64_t r_rows, int64_t r_cols, int64_t r_ld,
                         float* W_cols, int64_t c_rows, int64_t c_cols, int64_t c_ld, cudaStream_t stream);
 // dst[i,:] = mask[i] ? src[i,:] : 0

@@ -126,7 +126,8 @@ __global__ void symmetrize_kernel(float* G, int64_t n, int64_t ld) {
 
 template <typename T>
 __global__ void load_spd_kernel(const float* G, int64_t ldg, const int32_t* idx, int64_t n, const double* rho, T* dst,
-                                int64_t ldd) {
+                                int64_t ldd, const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;   // conditional launch (see SkipScope)
   const double r = rho ? rho[0] : 0.0;
   const int64_t total = n * n;
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -143,7 +144,8 @@ __global__ void load_spd_kernel(const float* G, int64_t ldg, const int32_t* idx,
 
 template <typename T>
 __global__ void gather_cols_kernel(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k, T* dst,
-                                   int64_t ldd) {
+                                   int64_t ldd, const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   const int64_t total = rows * k;
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t i = e / k, a = e % k;
@@ -162,7 +164,8 @@ __global__ void gather_rows_kernel(const float* __restrict__ src, int64_t lds, c
 
 template <typename T>
 __global__ void scatter_cols_kernel(const T* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t k,
-                                    float* dst, int64_t ldd) {
+                                    float* dst, int64_t ldd, const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   const int64_t total = rows * k;
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
     const int64_t i = e / k, a = e % k;
@@ -170,10 +173,21 @@ __global__ void scatter_cols_kernel(const T* src, int64_t lds, const int32_t* id
   }
 }
 
-__global__ void fill_zero_kernel(float* dst, int64_t ld, int64_t rows, int64_t cols) {
+__global__ void fill_zero_kernel(float* dst, int64_t ld, int64_t rows, int64_t cols, const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   const int64_t total = rows * cols;
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x)
     dst[(e / cols) * ld + (e % cols)] = 0.f;
+}
+
+// dst[i, 0:kpad] = src[i, 0:k] followed by zeros
+__global__ void copy_cols_padded_kernel(const float* __restrict__ src, int64_t lds, int64_t rows, int64_t k,
+                                        int64_t kpad, float* __restrict__ dst) {
+  const int64_t total = rows * kpad;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / kpad, a = e % kpad;
+    dst[e] = a < k ? src[i * lds + a] : 0.f;
+  }
 }
 
 __global__ void effective_ridge_kernel(const float* G, int64_t ldg, int64_t n, double rho, int rel, double* out) {
@@ -701,7 +715,8 @@ __global__ void sumsq_finish_kernel(const double* part, int nblocks, double scal
   if (threadIdx.x == 0) out[0] = (acc ? out[0] : 0.0) + scale * r;
 }
 
-__global__ void init_report_kernel(sp_step_report* rep, const double* rho1, const double* rho2, double kept) {
+__global__ void init_report_kernel(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
+                                   const int32_t* reused) {
   rep->res_act = 0.0;
   rep->res_out = nan("");
   rep->res_in = 0.0;
@@ -710,6 +725,7 @@ __global__ void init_report_kernel(sp_step_report* rep, const double* rho1, cons
   rep->rho1_eff = rho1 ? rho1[0] : 0.0;
   rep->rho2_eff = rho2 ? rho2[0] : 0.0;
   rep->kept = kept;
+  rep->factor_reused = (reused != nullptr && reused[0] != 0) ? 1.0 : 0.0;
 }
 
 // per-column sum |x| and sum x^2 of a [T, C] chunk: grid (col blocks of 256, row blocks) -> scratch, then reduced
@@ -812,7 +828,7 @@ cudaError_t load_spd(const float* G, int64_t ldg, int64_t n, const double* rho_d
   if (n == 0) return cudaSuccess;
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  load_spd_kernel<T><<<grid_for(n * n, 256), 256, 0, stream>>>(G, ldg, nullptr, n, rho_dev, dst, ldd);
+  load_spd_kernel<T><<<grid_for(n * n, 256), 256, 0, stream>>>(G, ldg, nullptr, n, rho_dev, dst, ldd, skip_flag());
   return cudaGetLastError();
 }
 template <typename T>
@@ -821,7 +837,7 @@ cudaError_t load_spd_gather(const float* G, int64_t ldg, const int32_t* idx, int
   if (k == 0) return cudaSuccess;
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  load_spd_kernel<T><<<grid_for(k * k, 256), 256, 0, stream>>>(G, ldg, idx, k, rho_dev, dst, ldd);
+  load_spd_kernel<T><<<grid_for(k * k, 256), 256, 0, stream>>>(G, ldg, idx, k, rho_dev, dst, ldd, skip_flag());
   return cudaGetLastError();
 }
 template <typename T>
@@ -830,7 +846,15 @@ cudaError_t gather_cols(const float* src, int64_t lds, const int32_t* idx, int64
   if (rows * k == 0) return cudaSuccess;
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  gather_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
+  gather_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd, skip_flag());
+  return cudaGetLastError();
+}
+cudaError_t copy_cols_padded(const float* src, int64_t lds, int64_t rows, int64_t k, int64_t kpad, float* dst,
+                             cudaStream_t stream) {
+  if (rows * kpad == 0) return cudaSuccess;
+  ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
+  count_launch();
+  copy_cols_padded_kernel<<<grid_for(rows * kpad, 256), 256, 0, stream>>>(src, lds, rows, k, kpad, dst);
   return cudaGetLastError();
 }
 cudaError_t gather_rows(const float* src, int64_t lds, const int32_t* idx, int64_t rows, int64_t cols, float* dst,
@@ -849,11 +873,12 @@ cudaError_t scatter_cols(const T* src, int64_t lds, const int32_t* idx, int64_t 
   if (idx) {
     ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
     count_launch();
-    fill_zero_kernel<<<grid_for(rows * n, 256), 256, 0, stream>>>(dst, ldd, rows, n);
+    fill_zero_kernel<<<grid_for(rows * n, 256), 256, 0, stream>>>(dst, ldd, rows, n, skip_flag());
   }
   if (rows * k == 0) return cudaGetLastError();
   count_launch();
-  scatter_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd);
+  scatter_cols_kernel<T><<<grid_for(rows * k, 256), 256, 0, stream>>>(src, lds, idx, rows, k, dst, ldd,
+                                                                      skip_flag());
   return cudaGetLastError();
 }
 #define SP_INST(T)                                                                                                  \
@@ -979,10 +1004,10 @@ cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t c
 }
 
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
-                        cudaStream_t stream) {
+                        const int32_t* reused, cudaStream_t stream) {
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  init_report_kernel<<<1, 1, 0, stream>>>(rep, rho1, rho2, kept);
+  init_report_kernel<<<1, 1, 0, stream>>>(rep, rho1, rho2, kept, reused);
   return cudaGetLastError();
 }
 

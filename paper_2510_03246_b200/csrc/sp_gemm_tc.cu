@@ -82,6 +82,7 @@ struct TcParams {
   int64_t c_s0, c_s1, cin_s0, cin_s1;
   long long wait_budget;   // clock cycles a role may wait on one barrier before it gives up (SP_ERR_TIMEOUT)
   int32_t* status;
+  const int32_t* skip;     // conditional launch: every CTA returns at once when *skip != 0 (see SkipScope)
 };
 
 struct Coord5 {
@@ -325,6 +326,7 @@ template <bool BATCHED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmCin, const TcParams p) {
+  if (p.skip != nullptr && *p.skip != 0) return;   // the same answer in every CTA: nothing is allocated yet
   extern __shared__ uint8_t smem_raw[];
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
@@ -898,6 +900,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   }
   p.status = status_dev;
   p.wait_budget = wait_budget_cycles() > 0 ? wait_budget_cycles() : WAIT_BUDGET_CYCLES;
+  p.skip = skip_flag();
 
   // Tile counts that do not fill the last wave of CTA pairs leave SMs idle.  A call that accumulates into C through
   // the add-reduction epilogue may cut K into a few ranges per tile instead: the partial products add up in C (in an
@@ -916,6 +919,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
     int best = 1;
     for (int ks = 2; ks <= 4; ++ks)
       if (num_kb / ks >= 32 && eff(ks) > eff(best) + 0.03) best = ks;
+    if (best > 1 && p.epi_mode == EPI_TMA_STORE && p.skip != nullptr) best = 1;   // no unconditional clear of C
     if (best > 1) {
       if (p.epi_mode == EPI_TMA_STORE) {
         if (cudaMemset2DAsync(C.ptr, (size_t)C.ld * 4, 0, (size_t)N * 4, (size_t)M, stream) != cudaSuccess)

@@ -48,7 +48,9 @@ constexpr size_t DIAG_SMEM = (size_t)TB * DIAG_TPAD * sizeof(float);
 //      holds the matrix, the update of B where it holds B (a block of block column jb starts its life as B from 0).
 // Global input and output go through a padded shared tile so that every global access is a full coalesced row.
 __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, int64_t lda, int nb, float* dinv,
-                                                                    int64_t row0, int32_t* status) {
+                                                                    int64_t row0, int32_t* status,
+                                                                    const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;                  // conditional launch (see SkipScope)
   extern __shared__ __align__(16) float diag_tile[];          // T[TB][TB + 1]
   float (*T)[DIAG_TPAD] = reinterpret_cast<float (*)[DIAG_TPAD]>(diag_tile);
   __shared__ __align__(16) float W[2][4][TB];   // W[k][index]: conflict-free 16-byte accesses along the index
@@ -306,7 +308,9 @@ template <bool TRANS>
 __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64_t ldx, int64_t rows, int nb,
                                                                  const float* __restrict__ dinv, __nv_bfloat16* S,
                                                                  int64_t lds, int64_t s_seg, int write_f32,
-                                                                 int32_t* status, PanelNear near) {
+                                                                 int32_t* status, PanelNear near,
+                                                                 const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   extern __shared__ __align__(128) float pa_smem[];
   float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(pa_smem);                       // Lt[k][c]
   float (*At)[PA_APAD] = reinterpret_cast<float (*)[PA_APAD]>(pa_smem + TB * TB);   // At[k][row]
@@ -473,7 +477,7 @@ cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, cons
   const bool with_near = TRANS && near.L != nullptr;
   ProfScope prof(PK_PANEL_APPLY, (with_near ? 4.0 : 2.0) * (double)rows * TB * TB, 0.0, stream);
   panel_apply_kernel<TRANS><<<(unsigned)ceil_div(rows, PA_ROWS), PA_THREADS, with_near ? PA_SMEM_NEAR : PA_SMEM, stream>>>(
-      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status, near);
+      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status, near, skip_flag());
   return cudaGetLastError();
 }
 
@@ -591,16 +595,21 @@ __device__ __forceinline__ void next_diag_body(const float* __restrict__ A21, co
 
 __global__ void __cluster_dims__(NM_CTAS, 1, 1) __launch_bounds__(NM_THREADS)
     chol_next_diag_kernel(const float* __restrict__ A21, const float* __restrict__ A22, int64_t lda, int nb2,
-                          const float* __restrict__ dinv, float* LmT, float* S, int32_t* status) {
+                          const float* __restrict__ dinv, float* LmT, float* S, int32_t* status,
+                          const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   next_diag_body<0>(A21, A22, lda, nb2, dinv, LmT, S, status);
 }
 __global__ void __launch_bounds__(NM_THREADS)
     chol_next_diag_stage1_kernel(const float* __restrict__ A21, int64_t lda, int nb2, const float* __restrict__ dinv,
-                                 float* LmT, int32_t* status) {
+                                 float* LmT, int32_t* status, const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   next_diag_body<1>(A21, nullptr, lda, nb2, dinv, LmT, nullptr, status);
 }
 __global__ void __launch_bounds__(NM_THREADS)
-    chol_next_diag_stage2_kernel(const float* __restrict__ A22, int64_t lda, int nb2, float* LmT, float* S) {
+    chol_next_diag_stage2_kernel(const float* __restrict__ A22, int64_t lda, int nb2, float* LmT, float* S,
+                                 const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;
   next_diag_body<2>(nullptr, A22, lda, nb2, nullptr, LmT, S, nullptr);
 }
 
@@ -621,6 +630,7 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
   __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
   const int64_t np = chol_tc_pad(n), ldp = 3 * np;
   const int64_t nblk = ceil_div(n, (int64_t)TB);
+  const int32_t* skip = skip_flag();
   static PerDeviceOnce attr_once;
   if (attr_once.run([] {
         cudaError_t e = cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -667,7 +677,7 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
       chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
                                                                   from_scratch ? (int64_t)TB : lda, nb, dk, k0,
-                                                                  status_dev);
+                                                                  status_dev, skip);
       if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     }
     const int64_t rem = n - k0 - nb;
@@ -690,13 +700,13 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
         if (!split_lookahead) {
           chol_next_diag_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + k0,
                                                                           A + (k0 + nb) * lda + (k0 + nb), lda, nb2,
-                                                                          dk, LmT, S, status_dev);
+                                                                          dk, LmT, S, status_dev, skip);
         } else {
           chol_next_diag_stage1_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + k0, lda, nb2, dk,
-                                                                                 LmT, status_dev);
+                                                                                 LmT, status_dev, skip);
           count_launch();
           chol_next_diag_stage2_kernel<<<NM_CTAS, NM_THREADS, NM_SMEM, stream>>>(A + (k0 + nb) * lda + (k0 + nb), lda,
-                                                                                 nb2, LmT, S);
+                                                                                 nb2, LmT, S, skip);
         }
         if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
       }
@@ -807,10 +817,11 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
 
 sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void* Pv, const float* dinv, void* Xsv,
                          int32_t* status_dev, cudaStream_t stream, const SolveAssist* assist, bool forward_done,
-                         const float* Lf, int64_t ldl) {
+                         const float* Lf, int64_t ldl, int64_t n_factor) {
   const __nv_bfloat16* P = reinterpret_cast<const __nv_bfloat16*>(Pv);
   __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(Xsv);
-  const int64_t np = chol_tc_pad(n), ldp = 3 * np;
+  if (n_factor > n && n % TB != 0) return SP_ERR_SHAPE;
+  const int64_t np = chol_tc_pad(n_factor > n ? n_factor : n), ldp = 3 * np;
   const int64_t lds = 3 * TB;
   const int64_t nblk = ceil_div(n, (int64_t)TB);
   // Every step applies the inverse diagonal block to one block column (panel) and then updates the columns still to

@@ -809,6 +809,49 @@ __global__ void __launch_bounds__(1024) mask_to_index_kernel(const uint8_t* mask
   }
 }
 
+// perm = the kept channels in ascending order, then the pruned ones in ascending order; count[0] = kept channels
+__global__ void __launch_bounds__(1024) mask_to_perm_kernel(const uint8_t* mask, int64_t n, int32_t* perm,
+                                                            int32_t* count) {
+  __shared__ int warp_tot[32];
+  __shared__ int s_kept;
+  int kept = 0;
+  for (int64_t base = 0; base < n; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    int tot;
+    block_excl_scan((i < n) && mask[i] != 0, warp_tot, &tot);
+    kept += tot;
+  }
+  if (threadIdx.x == 0) { s_kept = kept; count[0] = kept; }
+  __syncthreads();
+  kept = s_kept;
+  int64_t before = 0;
+  for (int64_t base = 0; base < n; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    const int keep = (i < n) && mask[i] != 0;
+    int tot;
+    const int rank = block_excl_scan(keep, warp_tot, &tot);
+    if (i < n) perm[keep ? before + rank : kept + (i - before - rank)] = (int32_t)i;
+    before += tot;
+  }
+}
+
+// flags[0] = 1 when the k kept channels of `mask` are not exactly perm[0..k) (the support the permutation was built
+// from, count_old of them); flags[1] = 1 - flags[0]
+__global__ void __launch_bounds__(1024) mask_changed_kernel(const uint8_t* mask, const int32_t* perm,
+                                                            const int32_t* count_old, int64_t k, int32_t* flags) {
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = (int64_t)count_old[0] != k;
+  __syncthreads();
+  int bad = 0;
+  for (int64_t a = threadIdx.x; a < k; a += blockDim.x) bad |= mask[perm[a]] == 0;
+  if (bad) s_bad = 1;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    flags[0] = s_bad ? 1 : 0;
+    flags[1] = s_bad ? 0 : 1;
+  }
+}
+
 __global__ void zero_rows_kernel(const uint8_t* mask, int group, float* W, int64_t rows, int64_t cols, int64_t ld) {
   const int64_t total = rows * cols;
   for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
@@ -1287,6 +1330,20 @@ cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cud
   if (n == 0) return cudaSuccess;
   count_launch();
   mask_to_index_kernel<<<1, 1024, 0, stream>>>(mask, n, kept_idx);
+  return cudaGetLastError();
+}
+
+cudaError_t mask_to_perm(const uint8_t* mask, int64_t n, int32_t* perm, int32_t* count, cudaStream_t stream) {
+  if (n == 0) return cudaSuccess;
+  count_launch();
+  mask_to_perm_kernel<<<1, 1024, 0, stream>>>(mask, n, perm, count);
+  return cudaGetLastError();
+}
+
+cudaError_t mask_changed(const uint8_t* mask, const int32_t* perm, const int32_t* count_old, int64_t k, int32_t* flags,
+                         cudaStream_t stream) {
+  count_launch();
+  mask_changed_kernel<<<1, 1024, 0, stream>>>(mask, perm, count_old, k, flags);
   return cudaGetLastError();
 }
 

@@ -20,12 +20,17 @@ int g_enabled = 0;   // 0 off, 1 outermost scopes only, 2 every scope (nested on
 std::vector<Slot> g_slots;
 int g_used = 0;
 thread_local int g_depth = 0;
+thread_local const int32_t* g_skip = nullptr;
 
 }  // namespace
 
 long long wait_budget_cycles() { return g_wait_budget.load(std::memory_order_relaxed); }
 
 bool reproducible_mode() { return g_reproducible.load(std::memory_order_relaxed) != 0; }
+
+const int32_t* skip_flag() { return g_skip; }
+SkipScope::SkipScope(const int32_t* flag) { g_skip = flag; }
+SkipScope::~SkipScope() { g_skip = nullptr; }
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 

@@ -586,8 +586,62 @@ def test_admm_step_with_z1_computed_ahead(dual):
         _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
 
 
+@pytest.mark.parametrize("cfg,overlap", [(SMALL_BF16, False), (SMALL_BF16, True),
+                                         (synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=1300, sparsity=0.33,
+                                                       outlier_frac=0.02), True)])
+def test_kept_support_recovery_reuses_the_factor(cfg, overlap):
+    """bf16 storage: the unrestricted system is factorised with the previously kept channels in front, and when the new
+    top-k keeps the same channels the recovery on the kept support is a backward sweep with the factor's leading block
+    (report field factor_reused); when it keeps others the restricted system is factorised.  Both branches are forced
+    here by what st->mask holds before the step, and both must give the oracle's exact restricted ridge solution.
+    Kept counts 388 (leading block 512 wide, 124 padding columns) and 520 (640 wide) of 776 channels."""
+    k = cfg.k_keep
+    assert k % 128 != 0
+    mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=k if overlap else 0)
+    mod.sp_ffn_init()
+    p_gpu = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, token_chunk=512)
+    p_or = O.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k)
+    tol = TOL[X.dtype]
+    audit = []
+    # first step: the mask holds all channels, so the support changes
+    _step_and_compare(mod, X, W1.float(), p_gpu, p_or, tol, audit)
+    assert mod.read_report()["factor_reused"] == 0.0
+    seen = set()
+    for it, plant in enumerate(["selected", "rolled", "selected", "fewer"]):
+        # what the coming step will select: the top-k of the scores of the current state
+        mod.sp_admm_scores(api.AdmmParams(rho=cfg.rho, k_keep=0, token_chunk=512))
+        torch.cuda.synchronize()
+        m_next, _ = O.topk_mask(mod.scores.cpu().numpy(), k)
+        if plant == "selected":
+            m_prev = m_next
+        elif plant == "rolled":               # same count, other channels
+            m_prev = np.roll(m_next, 1)
+            assert not np.array_equal(m_prev, m_next)
+        else:                                 # a subset: every previously kept channel is kept again, but not only those
+            m_prev = m_next.copy()
+            m_prev[np.flatnonzero(m_next)[::7]] = 0
+        mod.mask.copy_(torch.from_numpy(m_prev.astype(np.uint8)).to(DEV))
+        _step_and_compare(mod, X, W1.float(), p_gpu, p_or, tol, audit)
+        reused = mod.read_report()["factor_reused"]
+        # (the scores of the step can differ from those of the call before it in their last bits: what counts is the
+        # mask the step selected)
+        assert reused == float(np.array_equal(mod.mask.cpu().numpy(), m_prev)), plant
+        if plant != "selected":
+            assert reused == 0.0
+        seen.add(reused)
+    assert seen == {0.0, 1.0}
+    # a given mask (no selection) is its own previous mask: reuse in every step; fp32 storage and M (.) W2~ never reuse
+    mod.sp_admm_step(api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, token_chunk=512, reselect_mask=False))
+    torch.cuda.synchronize()
+    assert mod.read_report()["factor_reused"] == 1.0
+    mod.sp_admm_step(api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, token_chunk=512, refit=False))
+    torch.cuda.synchronize()
+    assert mod.read_report()["factor_reused"] == 0.0
+    mod.check_status()
+
+
 # ------------------------------------------------------------------------------------------------ SwiGLU modules
-SWIGLU_F32 = synth.scaled(synth.CONFIGS["C4"], d=88, n=300, tokens=520, sparsity=0.5, storage="f32")
+SWIGLU_F32 =synth.scaled(synth.CONFIGS["C4"], d=88, n=300, tokens=520, sparsity=0.5, storage="f32")
 SWIGLU_BF16 = synth.scaled(synth.CONFIGS["C4"], d=264, n=776, tokens=1300, sparsity=0.7, outlier_frac=0.02)
 
 
