@@ -31,10 +31,14 @@ implemented identically by the CUDA path):
   * allocation: r_l is the fraction PRUNED in layer l, as Algorithm 1 uses it (clip at 0.95, "mask with
     sparsity r_l"); kept count = n_l - round_half_up(r_l n_l).
 
-Parity unpinned (no statement in the paper fixes them; only self-consistency tests exist): the
-SwiGLU extension `swiglu_zu_update`, the default values of alpha, beta, rho, T, and the multi-head
-attention functions `mha_*` (Method 2 is printed with inconsistent shapes and without step sizes; the
-reading taken is stated above those functions and pinned by mathematics only).
+Pins.  Every function is pinned by tests/test_oracle_pins.py and tests/test_oracle_mha_pins.py to
+something other than itself: values the paper's formulas give by hand (golden files), closed forms,
+stationarity and finite-difference checks, brute force on tiny inputs, special cases that reduce to a
+library routine.  Two groups have no printed number or worked example in the paper to compare with, so
+their pins are mathematical only and the READING they implement is a choice stated above them: the
+SwiGLU extension (`swiglu_init`, `swiglu_zu_update`, the gated branches) and the multi-head attention
+functions `mha_*` (Method 2 is printed with inconsistent shapes and without step sizes).
+Parity unpinned: the default values of alpha, beta, rho, T (the paper fixes none of them).
 """
 from __future__ import annotations
 
@@ -472,8 +476,8 @@ def temperature_loss(layers, rbar, T_rel, iters, p, mode="softmax"):
 
 
 # --------------------------------------------------------------------------------------------------
-# SwiGLU extension (not in the paper: its modules are ReLU FFNs).  Parity unpinned against the paper; what pins
-# it is the mathematics of the subproblems it solves (stationarity, monotone descent, the g = 1 special case).
+# SwiGLU extension (not in the paper: its modules are ReLU FFNs, so there is no printed value to compare with).
+# What pins it is the mathematics of the subproblems it solves (stationarity, monotone descent, the g = 1 special case).
 #   module: y = W2 (SiLU(Wg x) * (Wu x)).  Only the "up" branch is split: Z = z_u with Z ~ Wu X, A ~ g * Z, where
 #   g = SiLU(Wg_0 X) is computed once from the pre-trained gate and kept fixed; the gate weights are only row-masked.
 #   With g fixed, phi(z) = g z is linear, so every subproblem of the FFN objective of Appendix A.1 keeps its closed
@@ -530,8 +534,9 @@ def swiglu_zu_update(A, g, z1u, alpha, beta, U=None):
 #     no counterpart for a softmax; it is not applied.
 #   * causal = True masks keys after the query (the decoder models the paper prunes are causal; the printed formulas
 #     omit the mask "for clarity").
-# Parity unpinned against the paper (it prints no numbers for this path); what pins the code below is mathematics:
-# finite-difference gradients, stationarity of the closed form, descent of every sub-step, and special cases.
+# The paper prints no numbers for this path; what pins the code below is mathematics (tests/test_oracle_mha_pins.py):
+# the forward definition as plain loops, central differences of both gradients, stationarity of the closed form,
+# convergence of the Eq. (85) steps to the linear-solve minimiser, descent of every sub-step, and special cases.
 # --------------------------------------------------------------------------------------------------
 @dataclasses.dataclass
 class MhaParams:
