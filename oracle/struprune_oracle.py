@@ -696,3 +696,28 @@ def mha_recover_weights(Xs, Ys, Zqs, Zks, As, head_mask, d_head, rho, rho_relati
     Wk = np.where(keep[:, None], ridge_solve(R_K, G_X, rho1), 0.0)
     Wo = restricted_refit(R_O, G_A, keep, effective_ridge(G_A, rho, rho_relative))
     return Wq, Wk, Wo
+
+
+def mha_recover_value_weights(Xs, Ps, As, head_mask, d_head, rho, rho_relative=True):
+    """Recovery of W_V ("W = z a^+", done "for W_Q, W_K, W_V, W_O separately") from the auxiliary variables of all
+    sequences.  The second term of the Method 2 objective ties head i's rows of a^attn to W_V through
+        a^attn_i = W_V,i X P_i^T        (d_h x T per sequence, tokens as columns),
+    so the regressors of head i are R_i = X P_i^T (d x T) and its least-squares recovery over all sequences s is
+        W_V,i = (sum_s A_i,s R_i,s^T) (sum_s R_i,s R_i,s^T + rho_i I)^-1,
+    one ridge system per head (rho_i relative to the mean diagonal of that head's Gram matrix when rho_relative).
+    Rows of pruned heads are zero.  Xs: list of [d, T]; Ps: list of [h, T, T]; As: list of [d, T]."""
+    d = Xs[0].shape[0]
+    h = len(head_mask)
+    Wv = np.zeros((d, d), F64)
+    for i in range(h):
+        if not head_mask[i]:
+            continue
+        r = slice(i * d_head, (i + 1) * d_head)
+        G = np.zeros((d, d), F64)
+        C = np.zeros((d_head, d), F64)
+        for X, P, A in zip(Xs, Ps, As):
+            R = np.asarray(X, F64) @ np.asarray(P[i], F64).T
+            G += R @ R.T
+            C += np.asarray(A, F64)[r] @ R.T
+        Wv[r] = ridge_solve(C, G, effective_ridge(G, rho, rho_relative))
+    return Wv

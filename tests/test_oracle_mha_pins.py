@@ -180,3 +180,54 @@ def test_recovered_projections_reproduce_the_pretrained_ones_and_respect_the_hea
     A_all, Y_all = np.concatenate(As, axis=1), np.concatenate(Ys, axis=1)
     fit = np.linalg.lstsq(A_all[dh:].T, Y_all.T, rcond=None)[0].T          # Ypre ~ W_O[:, kept] Aattn[kept]
     assert np.allclose(Wo1[:, dh:], fit, atol=1e-7)
+
+
+def test_recovered_value_projection():
+    """W_V = a^attn (X P^T)^+ per head.  Pins: (1) from the pre-trained state with a vanishing ridge it returns W_V (the
+    regressors X P_i^T of three sequences have full row rank); (2) the result is the minimiser of the second term of the
+    Method 2 objective plus the ridge: central differences of that term, evaluated by O.mha_objective, vanish there
+    and every perturbation raises it; (3) one token per sequence (P = 1): the regressors are X itself and the recovery is
+    the plain ridge solve on G_X, as lstsq on the stacked system gives it; (4) rows of a pruned head are zero and the
+    other heads do not change (the heads' systems are separate)."""
+    rng = np.random.default_rng(11)
+    d, T, h, dh, n_seq = 8, 9, 2, 4, 3
+    W = [0.7 * rng.standard_normal((d, d)) for _ in range(4)]
+    Xs = [rng.standard_normal((d, T)) for _ in range(n_seq)]
+    fw = [O.mha_forward(X, *W, h, True) for X in Xs]
+    Ps, As = [f[3] for f in fw], [f[4] for f in fw]
+    Wv = O.mha_recover_value_weights(Xs, Ps, As, [1, 1], dh, 1e-13, False)
+    assert np.allclose(Wv, W[2], atol=1e-6)
+    # (2) perturbed auxiliary variables, a real ridge: stationarity of  sum_s |A_s - heads(Wv X_s, P_s)|^2 + rho |Wv|^2
+    As2 = [A + 0.3 * rng.standard_normal(A.shape) for A in As]
+    Ps2 = [np.abs(P + 0.05 * rng.standard_normal(P.shape)) for P in Ps]
+    rho = 0.37
+    Wv2 = O.mha_recover_value_weights(Xs, Ps2, As2, [1, 1], dh, rho, False)
+    prm = O.MhaParams(n_heads=h, alpha=1.0, beta=1.0)
+
+    def f(Wtry):
+        t2 = sum(O.mha_objective(X, np.zeros((d, T)), W[0], W[1], Wtry, W[3], np.zeros((d, T)), np.zeros((d, T)), P, A,
+                                 prm)[1] for X, P, A in zip(Xs, Ps2, As2))
+        return t2 + rho * (Wtry ** 2).sum()
+
+    f0 = f(Wv2)
+    eps = 1e-5
+    for (i, j) in [(0, 0), (3, 5), (4, 1), (7, 7)]:
+        E = np.zeros((d, d)); E[i, j] = eps
+        assert abs(f(Wv2 + E) - f(Wv2 - E)) / (2 * eps) < 1e-6 * max(f0, 1.0)
+    for _ in range(5):
+        assert f(Wv2 + 1e-3 * rng.standard_normal((d, d))) > f0
+    # (3) T = 1: softmax of one logit is 1
+    X1 = [rng.standard_normal((d, 1)) for _ in range(20)]
+    A1 = [rng.standard_normal((d, 1)) for _ in range(20)]
+    P1 = [np.ones((h, 1, 1)) for _ in range(20)]
+    Wv3 = O.mha_recover_value_weights(X1, P1, A1, [1, 1], dh, 1e-13, False)
+    Xa, Aa = np.concatenate(X1, axis=1), np.concatenate(A1, axis=1)
+    assert np.allclose(Wv3, np.linalg.lstsq(Xa.T, Aa.T, rcond=None)[0].T, atol=1e-7)
+    # relative ridge: rho times the mean diagonal of the head's own Gram matrix
+    G0 = sum((X @ P[0].T) @ (X @ P[0].T).T for X, P in zip(Xs, Ps2))
+    C0 = sum(A[:dh] @ (X @ P[0].T).T for X, P, A in zip(Xs, Ps2, As2))
+    Wrel = O.mha_recover_value_weights(Xs, Ps2, As2, [1, 1], dh, 0.1, True)
+    assert np.allclose(Wrel[:dh], C0 @ np.linalg.inv(G0 + 0.1 * np.trace(G0) / d * np.eye(d)), atol=1e-9)
+    # (4) head mask
+    Wv4 = O.mha_recover_value_weights(Xs, Ps2, As2, [0, 1], dh, rho, False)
+    assert np.all(Wv4[:dh] == 0) and np.array_equal(Wv4[dh:], Wv2[dh:])
