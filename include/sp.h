@@ -432,6 +432,30 @@ sp_status sp_mha_step(const sp_mha_module* m, sp_mha_state* st, const sp_mha_par
 size_t sp_mha_workspace_bytes(int64_t d, int64_t n_heads, int64_t T, int64_t n_seq, int64_t seq_chunk, int32_t dtype);
 
 /* ---------------------------------------------------------------------------------------------------------------
+ * sp_mha_value_refit — recovery of W_V from the auxiliary variables of an attention module.
+ * Paper: Appendix A, Method 2, "Recovering weight matrices" (W = z a^+) applied to the second term of the objective,
+ * alpha |a_attn - Concat_i(W_V,i a_i)|^2; Algorithm 2 runs the recovery "for W_Q, W_K, W_V, W_O separately".
+ * With a_l the attention probabilities P the term ties head i's columns of Aattn to W_V through
+ *   Aattn_i = (P_i X) W_V,i^T      per sequence (token-major: [T, d_h] = [T, T] [T, d] [d, d_h]),
+ * so the regressors of head i are R_i = P_i X and its ridge least-squares solution over all sequences s is
+ *   W_V,i = (sum_s Aattn_i,s^T R_i,s) (sum_s R_i,s^T R_i,s + rho_i I)^-1        ([d_h, d], rows i d_h .. of W_V),
+ * one system of size d per kept head; rho_i = rho * trace / d of that head's Gram matrix when rho_relative.
+ * Reads m->X, st->P, st->Aattn (the weights in m are not read).  head_mask_host: HOST array of n_heads bytes
+ * (0 = pruned; NULL = all heads kept) — the host decides which systems to build.  Wv_out: device, fp32 [d, ldw >= d],
+ * rows of pruned heads are written as zero; it may be m->Wv.ptr.
+ * bf16 mode: P, Aattn and the regressors are carried as bf16 hi + lo parts (the systems of the heads are worse
+ * conditioned than G_X: their regressors are running averages of the inputs); fp32 mode: fp64 accumulation and
+ * factorisation.
+ * Workspace: sp_mha_value_refit_workspace_bytes (it holds n_heads Gram matrices of d x d floats).
+ * Errors: as sp_mha_step; SP_ERR_INVALID_ARG also for rho < 0 or Wv_out == NULL; SP_ERR_NOT_SPD through status_dev.
+ */
+sp_status sp_mha_value_refit(const sp_mha_module* m, const sp_mha_state* st, const uint8_t* head_mask_host, double rho,
+                             int32_t rho_relative, int64_t seq_chunk, float* Wv_out, int64_t ldw, int32_t* status_dev,
+                             void* ws, size_t ws_bytes, void* stream);
+size_t sp_mha_value_refit_workspace_bytes(int64_t d, int64_t n_heads, int64_t T, int64_t n_seq, int64_t seq_chunk,
+                                          int32_t dtype);
+
+/* ---------------------------------------------------------------------------------------------------------------
  * Helpers.
  * sp_ridge_solve   — W[m,n] = R[m,n] (G[n,n] + rho_eff I)^-1 by Cholesky and two triangular solves (weight
  *                    recovery of Appendix A.1).  G, R, W fp32; factorisation in fp64 when precise != 0, else fp32.

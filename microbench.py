@@ -120,6 +120,19 @@ def mha_case(reps, warm):
     print(f"mha step d={d} H={H} T={T} n_seq={n_seq}: {ms:8.3f} ms  {fl / ms / 1e9:7.1f} TFLOP/s (algorithmic)")
     print("   " + "; ".join(f"{k}: {v['records']} x {1e3 * v['ms'] / max(v['records'], 1):.1f} us"
                             for k, v in pr.items() if v["records"]), flush=True)
+    # recovery of W_V: per head the regressors P_i X (2 parts of P), their Gram matrix (3 part products, lower
+    # triangle) and the cross product with Aattn_i (3 part products), then one system of size d per head
+    ms_v = _timeit(lambda: mod.sp_mha_value_refit(None, 0.05, True), reps, warm)
+    api.sp_profile_begin(2)
+    mod.sp_mha_value_refit(None, 0.05, True)
+    torch.cuda.synchronize()
+    pr = api.sp_profile_read()
+    api.sp_profile_begin(0)
+    mod.check_status()
+    fl_v = pairs * (2.0 * T * T * d + 1.0 * d * d * T + 2.0 * (d // H) * d * T) + H * (d ** 3 / 3 + 2.0 * (d // H) * d * d)
+    print(f"W_V recovery d={d} H={H} T={T} n_seq={n_seq}: {ms_v:8.3f} ms  {fl_v / ms_v / 1e9:7.1f} TFLOP/s (algorithmic)")
+    print("   " + "; ".join(f"{k}: {v['records']} x {1e3 * v['ms'] / max(v['records'], 1):.1f} us"
+                            for k, v in pr.items() if v["records"]), flush=True)
     print("status", mod.status.cpu().tolist())
 
 

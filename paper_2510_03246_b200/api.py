@@ -32,7 +32,7 @@ EXPORTS = ["sp_gram_accumulate", "sp_ffn_init", "sp_admm_step", "sp_admm_scores"
            "sp_profile_kind_name", "sp_launch_count", "sp_mha_init", "sp_mha_step", "sp_mha_workspace_bytes",
            "sp_set_reproducible", "sp_get_reproducible", "sp_allocate_sparsity_grid", "sp_apply_mask_global",
            "sp_apply_mask_global_bytes", "sp_objective_accumulate", "sp_ffn_cache_input_inverse",
-           "sp_set_wait_budget"]
+           "sp_set_wait_budget", "sp_mha_value_refit", "sp_mha_value_refit_workspace_bytes"]
 
 
 class SpError(RuntimeError):
@@ -129,6 +129,10 @@ def lib() -> C.CDLL:
         L.sp_mha_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, i32]
         L.sp_mha_init.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), i32, i64, vp, vp, sz, vp]
         L.sp_mha_step.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), C.POINTER(SpMhaParams), vp, vp, sz, vp]
+        L.sp_mha_value_refit_workspace_bytes.restype = C.c_size_t
+        L.sp_mha_value_refit_workspace_bytes.argtypes = [i64, i64, i64, i64, i64, i32]
+        L.sp_mha_value_refit.argtypes = [C.POINTER(SpMhaModule), C.POINTER(SpMhaState), vp, dbl, i32, i64, vp, i64, vp, vp,
+                                         sz, vp]
         L.sp_allocate_sparsity_grid.argtypes = [vp, vp, i32, dbl, vp, i32, i32, i32, dbl, vp, vp, vp]
         L.sp_apply_mask_global.argtypes = [vp, i64, i64, i32, dbl, i64, vp, i64, vp, vp, vp, sz, vp]
         L.sp_apply_mask_global_bytes.restype = C.c_size_t
@@ -145,6 +149,7 @@ def lib() -> C.CDLL:
         L.sp_launch_count.restype = i64
         for name in EXPORTS:
             if name not in ("sp_workspace_bytes", "sp_admm_overlap_bytes", "sp_mha_workspace_bytes",
+                            "sp_mha_value_refit_workspace_bytes",
                             "sp_apply_mask_global_bytes", "sp_status_string", "sp_version", "sp_profile_kinds",
                             "sp_profile_kind_name", "sp_launch_count"):
                 getattr(L, name).restype = C.c_int32
@@ -627,6 +632,7 @@ class MhaModule:
                                                                if accumulators else (None,) * 5)
         self.status = new_status(self.dev)
         self._wsbuf = _ws(lib().sp_mha_workspace_bytes(d, n_heads, T, self.n_seq, seq_chunk, _dt(self.X)), self.dev)
+        self._ws_refit = None       # workspace of sp_mha_value_refit, allocated on first use
 
     def set_weights(self, Wq, Wk, Wv, Wo):
         for dst, src in ((self.Wq, Wq), (self.Wk, Wk), (self.Wv, Wv), (self.Wo, Wo)):
@@ -650,6 +656,26 @@ class MhaModule:
         prm = SpMhaParams(p.alpha, p.beta, p.a_steps, p.z_steps, p.eta_z, int(p.causal), 0, self.seq_chunk)
         _check(lib().sp_mha_step(C.byref(m), C.byref(st), C.byref(prm), self.status.data_ptr(), self._wsbuf.data_ptr(),
                                  self._wsbuf.numel(), _stream()), "sp_mha_step")
+
+    def sp_mha_value_refit(self, head_mask=None, rho: float = 0.0, rho_relative: bool = True,
+                           out: torch.Tensor | None = None) -> torch.Tensor:
+        """W_V recovered from the module's P and Aattn (see sp.h); head_mask: n_heads values on the HOST (None = all
+        kept).  Writes into `out` (default: the module's own Wv) and returns it."""
+        m, st = self._module(), self._state()
+        out = self.Wv if out is None else out
+        assert out.is_cuda and out.dtype == torch.float32 and out.shape == (self.d, self.d) and out.stride(1) == 1
+        hm = None
+        if head_mask is not None:
+            hm = (C.c_uint8 * self.n_heads)(*[1 if int(v) else 0 for v in head_mask])
+        need = lib().sp_mha_value_refit_workspace_bytes(self.d, self.n_heads, self.T, self.n_seq, self.seq_chunk,
+                                                        _dt(self.X))
+        if self._ws_refit is None or self._ws_refit.numel() < need:
+            self._ws_refit = _ws(need, self.dev)
+        _check(lib().sp_mha_value_refit(C.byref(m), C.byref(st), hm, float(rho), int(rho_relative), self.seq_chunk,
+                                        out.data_ptr(), out.stride(0), self.status.data_ptr(),
+                                        self._ws_refit.data_ptr(), self._ws_refit.numel(), _stream()),
+               "sp_mha_value_refit")
+        return out
 
     def check_status(self):
         code = int(self.status[0].item())

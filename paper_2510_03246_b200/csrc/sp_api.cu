@@ -1470,4 +1470,152 @@ sp_status sp_mha_step(const sp_mha_module* m, sp_mha_state* st, const sp_mha_par
   return mha_impl(m, st, p, false, 0, status_dev, ws, ws_bytes, stream);
 }
 
+// ---- recovery of W_V from the auxiliary head outputs
+namespace {
+struct ValueRefitPlan {
+  int64_t dh, sc, cap;
+  bool bf16;
+  SolveBufs sb, sb2;   // two sets: the systems of the heads are independent and are solved two at a time
+  void* Pb;     // bf16 mode: hi / lo planes of P of one chunk, [2][sc H, T, T]
+  void* Ab;     // bf16 mode: Aattn of one chunk as bf16 hi | lo parts, [cap, 2 pad64(d)]
+  void* R;      // regressors of one head and chunk: bf16 hi | lo [cap, 2 pad64(d)], or fp32 [cap, d]
+  float* G;     // [H][d, d]   sum over sequences of R^T R per head (lower triangle)
+  float* Cv;    // [H][d_h, d] sum over sequences of Aattn_i^T R per head
+  size_t bytes;
+};
+
+ValueRefitPlan plan_value_refit(void* ws, int64_t d, int64_t H, int64_t T, int64_t n_seq, int64_t seq_chunk,
+                                int32_t cdt) {
+  ValueRefitPlan p;
+  p.dh = H > 0 ? d / H : d;
+  p.sc = seq_chunk > 0 ? seq_chunk : 1;
+  if (p.sc > n_seq) p.sc = n_seq;
+  if (p.sc < 1) p.sc = 1;
+  p.cap = p.sc * T;
+  p.bf16 = cdt == SP_BF16;
+  Carver c(ws);
+  p.sb = carve_solve(c, d, p.dh, p.bf16 ? 4 : 8);
+  p.sb2 = carve_solve(c, d, p.dh, p.bf16 ? 4 : 8);
+  p.Pb = p.bf16 ? c.take_bytes((size_t)2 * p.sc * H * T * T * 2) : nullptr;
+  p.Ab = p.bf16 ? c.take_bytes((size_t)p.cap * 2 * split_kpad(d) * 2) : nullptr;
+  p.R = c.take_bytes(p.bf16 ? (size_t)p.cap * 2 * split_kpad(d) * 2 : (size_t)p.cap * d * 4);
+  p.G = c.take<float>((size_t)H * d * d);
+  p.Cv = c.take<float>((size_t)d * d);
+  p.bytes = align_up(c.off, 256);
+  return p;
+}
+}  // namespace
+
+size_t sp_mha_value_refit_workspace_bytes(int64_t d, int64_t n_heads, int64_t T, int64_t n_seq, int64_t seq_chunk,
+                                          int32_t dtype) {
+  if (d < 1 || n_heads < 1 || T < 1 || n_seq < 1) return 0;
+  return plan_value_refit(nullptr, d, n_heads, T, n_seq, seq_chunk, dtype).bytes + 256;
+}
+
+sp_status sp_mha_value_refit(const sp_mha_module* m, const sp_mha_state* st, const uint8_t* head_mask_host, double rho,
+                             int32_t rho_relative, int64_t seq_chunk, float* Wv_out, int64_t ldw, int32_t* status_dev,
+                             void* ws, size_t ws_bytes, void* stream) {
+  SPCHK(check_mha(m, st));
+  if (!Wv_out || !(rho >= 0.0) || seq_chunk < 0) return SP_ERR_INVALID_ARG;
+  const int64_t d = m->d, H = m->n_heads, T = m->T, n_seq = m->n_seq, dh = d / H;
+  if (ldw < d) return SP_ERR_SHAPE;
+  const int32_t cdt = m->X.dtype;
+  if (!ws || ws_bytes < plan_value_refit(nullptr, d, H, T, n_seq, seq_chunk, cdt).bytes) return SP_ERR_WORKSPACE;
+  if (misaligned(ws, 256)) return SP_ERR_ALIGNMENT;
+  ValueRefitPlan p = plan_value_refit(ws, d, H, T, n_seq, seq_chunk, cdt);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const bool bf16 = p.bf16;
+  const size_t esz = bf16 ? 2 : 4;
+  const int64_t TT = T * T, dp = split_kpad(d);
+  auto kept = [&](int64_t i) { return head_mask_host == nullptr || head_mask_host[i] != 0; };
+  CU(cudaMemset2DAsync(Wv_out, (size_t)ldw * sizeof(float), 0, (size_t)d * sizeof(float), (size_t)d, s));
+
+  // ---- per head: G_i = sum_s R^T R and C_i = sum_s Aattn_i^T R with the regressors R = P_i X of every sequence
+  // (token-major: row q of R is sum_k P_i[q, k] x_k)
+  for (int64_t q0 = 0; q0 < n_seq; q0 += p.sc) {
+    const int64_t nq = (n_seq - q0 < p.sc) ? n_seq - q0 : p.sc;
+    const int64_t t0 = q0 * T, Tc = nq * T, pairs = nq * H;
+    const double acc = q0 > 0 ? 1.0 : 0.0;
+    const uint8_t* xptr = reinterpret_cast<const uint8_t*>(m->X.ptr) + (size_t)t0 * d * esz;
+    const float* Aat = st->Aattn + (size_t)t0 * d;
+    const float* P = st->P + (size_t)q0 * H * TT;
+    const int64_t pplane = p.sc * H * TT;
+    if (bf16) {
+      CU(split_planes(P, pairs * TT, p.Pb, pplane, s));
+      CU(split_bf16(Aat, d, nullptr, Tc, d, dp, p.Ab, s));
+    }
+    const BMat none{nullptr, SP_F32, 0, 0, 0, 1, 0};
+    for (int64_t i = 0; i < H; ++i) {
+      if (!kept(i)) continue;
+      float* Gi = p.G + (size_t)i * d * d;
+      float* Ci = p.Cv + (size_t)i * dh * d;
+      // one launch for the nq sequences of the chunk (the batch index b0 is not used: one head at a time)
+      const BMat Xb{xptr, cdt, d, d, T * d, 1, 0};
+      if (bf16) {
+        const BMat Pi{reinterpret_cast<const __nv_bfloat16*>(p.Pb) + (size_t)i * TT, SP_BF16, T, TT, H * TT, 2, pplane};
+        const BMat Rb{p.R, SP_BF16, 2 * dp, 2 * dp, T * 2 * dp, 1, 0};
+        static const int pa[2] = {0, 1}, pb[2] = {0, 0};     // (P hi + P lo) X
+        SPCHK(bcontract(T, d, T, 1.0, Pi, true, Xb, false, 2, pa, pb, 0.0, none, Rb, dp, 1, (int)nq, status_dev, s));
+        // G_i (+)= R^T R with R = R_hi + R_lo: hi.hi, lo.hi, hi.lo; the token axis is K, both operands MN-major
+        TcOperand ra{p.R, 2 * dp, false}, rb{p.R, 2 * dp, false};
+        ra.kext = rb.kext = Tc;
+        ra.mnext = rb.mnext = 2 * dp;
+        TcSegments sg;
+        sg.nseg = 3;
+        sg.a_mn[1] = (int32_t)dp;
+        sg.b_mn[2] = (int32_t)dp;
+        SPCHK(gemm_tc(d, d, Tc, 1.f, ra, rb, (float)acc, Operand{Gi, SP_F32, d, 1}, OutOperand{Gi, SP_F32, d}, true,
+                      status_dev, s, &sg, (double)d * d * Tc));
+        // C_i (+)= Aattn_i^T R: the head's d_h columns of Aattn (hi | lo) against R (hi | lo): hi.hi, lo.hi, hi.lo
+        TcOperand aa{reinterpret_cast<const __nv_bfloat16*>(p.Ab) + i * dh, 2 * dp, false};
+        aa.kext = Tc;
+        aa.mnext = dp + dh;      // the lo part of the head's columns sits dp columns to the right
+        TcSegments sc2;
+        sc2.nseg = 3;
+        sc2.a_mn[1] = (int32_t)dp;
+        sc2.b_mn[2] = (int32_t)dp;
+        SPCHK(gemm_tc(dh, d, Tc, 1.f, aa, rb, (float)acc, Operand{Ci, SP_F32, d, 1}, OutOperand{Ci, SP_F32, d}, false,
+                      status_dev, s, &sc2, 2.0 * (double)dh * d * Tc));
+      } else {
+        const BMat Pi{P + (size_t)i * TT, SP_F32, T, TT, H * TT, 1, 0};
+        const BMat Rb{p.R, SP_F32, d, d, T * d, 1, 0};
+        SPCHK(bcontract(T, d, T, 1.0, Pi, true, Xb, false, 1, kSegHH, kSegHH, 0.0, none, Rb, 0, 1, (int)nq, status_dev,
+                        s));
+        MatRef r{p.R, SP_F32, d}, g{Gi, SP_F32, d}, c{Ci, SP_F32, d}, a{Aat + i * dh, SP_F32, d};
+        SPCHK(contract(d, d, Tc, 1.0, r, false, r, false, acc, g, g, true, true, false, status_dev, s));
+        SPCHK(contract(dh, d, Tc, 1.0, a, false, r, false, acc, c, c, false, true, false, status_dev, s));
+      }
+    }
+  }
+  // ---- W_V,i = C_i (G_i + rho_i I)^-1, one regularised solve per kept head.  A solve is a chain of short kernels that
+  // leaves most SMs idle, and the heads' systems are independent: they alternate between the caller's stream and the
+  // library's side stream, each with its own buffers and assisting stream.
+  SideStream* side = side_stream();
+  JoinOnExit join_guard{side, s};
+  if (side) {
+    CU(cudaEventRecord(side->fork, s));
+    CU(cudaStreamWaitEvent(side->stream, side->fork, 0));
+  }
+  int64_t turn = 0;
+  for (int64_t i = 0; i < H; ++i) {
+    if (!kept(i)) continue;
+    const float* Gi = p.G + (size_t)i * d * d;
+    const float* Ci = p.Cv + (size_t)i * dh * d;
+    float* Wi = Wv_out + (size_t)i * dh * ldw;
+    const bool on_side = side != nullptr && (turn++ & 1) != 0;
+    cudaStream_t sq = on_side ? side->stream : s;
+    SolveBufs& sb = on_side ? p.sb2 : p.sb;
+    const SolveAssist* assist = !side ? nullptr : on_side ? &side->assist_side : &side->assist_main;
+    CU(effective_ridge(Gi, d, d, rho, rho_relative, sb.rho, sq));
+    if (bf16) SPCHK(ridge_core<float>(Ci, d, Gi, d, dh, d, nullptr, d, sb.rho, Wi, ldw, sb, status_dev, sq, assist));
+    else SPCHK(ridge_core<double>(Ci, d, Gi, d, dh, d, nullptr, d, sb.rho, Wi, ldw, sb, status_dev, sq));
+  }
+  if (side) {
+    CU(cudaEventRecord(side->join, side->stream));
+    CU(cudaStreamWaitEvent(s, side->join, 0));
+  }
+  join_guard.armed = false;
+  return SP_OK;
+}
+
 }  // extern "C"

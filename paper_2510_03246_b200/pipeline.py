@@ -213,16 +213,18 @@ def prune_attention_heads(H: torch.Tensor, Ypre: torch.Tensor, W_O: torch.Tensor
 
 
 def mha_outer_iterations(mod: api.MhaModule, head_mask: torch.Tensor, iters: int, params: api.MhaParams | None = None,
-                         rho: float = 0.1, rho_relative: bool = True):
+                         rho: float = 0.1, rho_relative: bool = True, recover_wv: bool = True):
     """Outer loop of Algorithm 2's SparseLLM2 for one attention module with a fixed head mask (u8 [n_heads], from the
-    head scores): per iteration (1) the weight recoveries W = z a^+ that are linear in the auxiliary variables, from
-    the accumulators the previous step left -- W_Q, W_K by sp_ridge_solve with the rows of pruned heads zeroed, W_O by
-    sp_linear_refit on the columns of the kept heads -- with W_V kept as the row-masked pre-trained matrix, then (2)
-    sp_mha_step: Eq. (85), (86), (87).  `mod` must have been initialised (sp_mha_init) with its accumulators.
+    head scores): per iteration (1) the weight recoveries W = z a^+ "for W_Q, W_K, W_V, W_O separately" -- W_Q, W_K by
+    sp_ridge_solve from the accumulators the previous step left, with the rows of pruned heads zeroed, W_O by
+    sp_linear_refit on the columns of the kept heads, W_V by sp_mha_value_refit from P and Aattn (one system per kept
+    head; recover_wv = False keeps the row-masked pre-trained W_V instead) -- then (2) sp_mha_step: Eq. (85), (86),
+    (87).  `mod` must have been initialised (sp_mha_init) with its accumulators.
     All arithmetic runs in the library; this function only orders the calls.  Returns the module."""
     p = params or api.MhaParams()
     d_head = mod.d // mod.n_heads
     k_heads = int(head_mask.sum().item())
+    mask_host = head_mask.cpu().tolist()
     # row masks of the projections: sp_apply_mask zeroes the rows of pruned units given their scores; with the mask
     # already known its 0 / 1 values serve as the scores and k_heads as the kept count
     unit_scores = head_mask.to(torch.float32)
@@ -235,6 +237,8 @@ def mha_outer_iterations(mod: api.MhaModule, head_mask: torch.Tensor, iters: int
         api.sp_apply_mask(unit_scores, k_heads, group=d_head, W_rows=Wk)
         Wo = api.sp_linear_refit(mod.R_O, mod.G_attn, head_mask, k_heads, rho, group=d_head, precise=precise,
                                  rho_relative=rho_relative)
+        if recover_wv:
+            mod.sp_mha_value_refit(mask_host, rho, rho_relative)      # writes mod.Wv, rows of pruned heads zero
         mod.set_weights(Wq, Wk, mod.Wv, Wo)
         mod.sp_mha_step(p)
     mod.check_status()

@@ -151,7 +151,8 @@ def test_mha_outer_iterations_match_oracle(dtype, d, H, T, n_seq):
         assert relerr(np64(mod.G_attn), sum(a @ a.T for a in As)) < tol
         assert relerr(np64(mod.R_O), sum(y @ a.T for y, a in zip(Ys, As))) < tol
         acc = {k: np64(getattr(mod, k)) for k in ("G_X", "R_Q", "R_K", "G_attn", "R_O")}
-        pipeline.mha_outer_iterations(mod, hm, 1, p_gpu, rho=0.1)
+        # first iteration with the row-masked pre-trained W_V, second with W_V recovered from P and Aattn
+        pipeline.mha_outer_iterations(mod, hm, 1, p_gpu, rho=0.1, recover_wv=(it == 1))
         torch.cuda.synchronize()
         # weights: the oracle's recovery from the GPU's accumulators (teacher-forced)
         keep = np.repeat(head_mask.numpy().astype(bool), dh)
@@ -162,7 +163,11 @@ def test_mha_outer_iterations_match_oracle(dtype, d, H, T, n_seq):
         assert relerr(np64(mod.Wq), Wq_or) < tol and relerr(np64(mod.Wk), Wk_or) < tol, "W_Q / W_K"
         assert relerr(np64(mod.Wo), Wo_or) < tol, "W_O"
         assert np.all(np64(mod.Wq)[~keep] == 0) and np.all(np64(mod.Wo)[:, ~keep] == 0) and np.all(np64(mod.Wv)[~keep] == 0)
-        assert relerr(np64(mod.Wv), Wv_masked) < 1e-7
+        if it == 0:
+            assert relerr(np64(mod.Wv), Wv_masked) < 1e-7
+        else:
+            Wv_or = O.mha_recover_value_weights(Xs, Ps, As, head_mask.numpy(), dh, 0.1, True)
+            assert relerr(np64(mod.Wv), Wv_or) < tol, "W_V"
         # auxiliary updates with the GPU's weights
         Wg = [np64(w) for w in (mod.Wq, mod.Wk, mod.Wv, mod.Wo)]
         for q in range(n_seq):
@@ -170,3 +175,61 @@ def test_mha_outer_iterations_match_oracle(dtype, d, H, T, n_seq):
             Zq, Zk, P, A = O.mha_step(Xs[q], Ys[q], *Wg, Zqs[q], Zks[q], Ps[q], As[q], p_or)
             assert relerr(np64(mod.P[q]), P) < tol and relerr(np64(mod.Aattn[r]).T, A) < tol
             assert relerr(np64(mod.Zq[r]).T, Zq) < tol and relerr(np64(mod.Zk[r]).T, Zk) < tol
+
+
+@pytest.mark.parametrize("dtype,d,H,T,n_seq,chunk,causal", CASES)
+def test_mha_value_refit_matches_oracle(dtype, d, H, T, n_seq, chunk, causal):
+    """W_V = a_attn (P X)^+ per kept head (sp_mha_value_refit) against the oracle's recovery from the same P, Aattn, X,
+    after one step with perturbed weights (so that P and Aattn are no longer the forward values): with a relative
+    ridge and one head pruned, then with all heads and an absolute ridge written into a pitched output."""
+    X, W = _case(dtype, d, H, T, n_seq, seed_layer=3)
+    mod = api.MhaModule(X.to(DEV), *[w.to(DEV) for w in W], n_heads=H, T=T, seq_chunk=chunk)
+    mod.sp_mha_init(causal)
+    g = torch.Generator().manual_seed(9)
+    Wp = [w.float() * (1.0 + 0.05 * torch.randn(w.shape, generator=g)) for w in W]
+    mod.set_weights(*[w.to(DEV) for w in Wp])
+    mod.sp_mha_step(api.MhaParams(alpha=1.0, beta=1.0, a_steps=2, z_steps=1, causal=causal))
+    torch.cuda.synchronize()
+    mod.check_status()
+    dh = d // H
+    tol = TOL[dtype]
+    Xo = np64(X)
+    Xs = [Xo[q * T:(q + 1) * T].T for q in range(n_seq)]
+    As = [np64(mod.Aattn)[q * T:(q + 1) * T].T for q in range(n_seq)]
+    Ps = [np64(mod.P[q]) for q in range(n_seq)]
+    head_mask = [1] * H
+    if H > 1:
+        head_mask[H // 2] = 0
+    Wv = mod.sp_mha_value_refit(head_mask, 0.05, True)
+    torch.cuda.synchronize()
+    mod.check_status()
+    ref = O.mha_recover_value_weights(Xs, Ps, As, head_mask, dh, 0.05, True)
+    assert relerr(np64(Wv), ref) < tol
+    keep = np.repeat(np.asarray(head_mask, bool), dh)
+    assert np.all(np64(Wv)[~keep] == 0)
+    # all heads, absolute ridge, output rows 8 floats apart from a dense layout; the padding is not touched
+    out = torch.full((d, d + 8), -3.0, device=DEV)
+    rho_abs = 0.02 * float(np.trace(sum(x @ x.T for x in Xs))) / d
+    mod.sp_mha_value_refit(None, rho_abs, False, out=out[:, :d])
+    torch.cuda.synchronize()
+    mod.check_status()
+    ref2 = O.mha_recover_value_weights(Xs, Ps, As, [1] * H, dh, rho_abs, False)
+    assert relerr(np64(out[:, :d]), ref2) < tol
+    assert torch.all(out[:, d:] == -3.0)
+
+
+def test_mha_value_refit_argument_errors():
+    X, W = _case(torch.bfloat16, 96, 4, 40, 2)
+    mod = api.MhaModule(X.to(DEV), *[w.to(DEV) for w in W], n_heads=4, T=40)
+    mod.sp_mha_init()
+    with pytest.raises(api.SpError) as e:
+        mod.sp_mha_value_refit(None, -1.0, True)
+    assert e.value.code == 1
+    m, st = mod._module(), mod._state()
+    import ctypes as C
+    rc = api.lib().sp_mha_value_refit(C.byref(m), C.byref(st), None, 0.1, 1, 0, mod.Wv.data_ptr(), mod.d,
+                                      mod.status.data_ptr(), mod._wsbuf.data_ptr(), 256, None)
+    assert rc == 5                                   # SP_ERR_WORKSPACE
+    rc = api.lib().sp_mha_value_refit(C.byref(m), C.byref(st), None, 0.1, 1, 0, mod.Wv.data_ptr(), mod.d - 8,
+                                      mod.status.data_ptr(), mod._wsbuf.data_ptr(), mod._wsbuf.numel(), None)
+    assert rc == 2                                   # SP_ERR_SHAPE: leading dimension below d
