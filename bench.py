@@ -14,7 +14,9 @@ the ranks (strong scaling; the accumulators are all-reduced once per iteration).
 Prints ONE JSON line (rank 0).  Besides the timed step (mask re-selected in every iteration) the line carries
 `fixed_mask` (the same module stepped without re-selection, and its continuation on the kept channels only), `e2e`
 (one whole pruned layer from and to pinned host buffers: the FFN module's iterations and the attention half with fixed
-head outputs) and `cpu_baseline` (the oracle on a token sample).  `--dual` runs with the scaled dual variable.
+head outputs), `attention_module` (the attention module's step under the second MHA objective and the recovery of
+W_V, timed on 16 sequences of 1024 tokens at the workload's width) and `cpu_baseline` (the oracle on a token sample).
+`--dual` runs with the scaled dual variable.
 `--impl reference` times the CPU oracle instead (a deliberately plain fp64 restatement of the paper; context only).
 """
 from __future__ import annotations
@@ -61,6 +63,8 @@ def parse():
     ap.add_argument("--workloads", default="C3,C4,C5",
                     help="1 GPU: further workloads measured after the main one and reported under `workloads` "
                          "(empty string: none)")
+    ap.add_argument("--no-attention", action="store_true",
+                    help="skip the timing of the attention module's step and W_V recovery (`attention_module`)")
     ap.add_argument("--workload-steps", type=int, default=5)
     ap.add_argument("--workload-warmup", type=int, default=2)
     return ap.parse_args()
@@ -396,6 +400,49 @@ def rooflines(cfg, args, prof, steps, peaks):
     return roofline, roofline_hbm, breakdown
 
 
+def attention_module_timing(cfg, dev, n_seq=16, T=1024, seq_chunk=8, steps=3):
+    """The attention half of a layer of the workload's width under the paper's second MHA objective: sp_mha_step (two
+    gradient steps of Eq. 85, the closed form of Eq. 86, two gradient steps of Eq. 87) and the recovery of W_V
+    (sp_mha_value_refit), on n_seq synthetic sequences of T tokens, timed with CUDA events after one warm-up call.
+    Not part of `value`: the headline metric counts iterations of the FFN module."""
+    import torch
+    from paper_2510_03246_b200 import api, synth
+    d, H = cfg.d, cfg.heads
+    acfg = synth.scaled(cfg, tokens=n_seq * T, outlier_frac=0.0)
+    X = synth.make_activations(acfg, 0).to(dev)
+    W = []
+    for tid in (11, 12, 13, 14):
+        w = synth.standard_variates(synth.module_seed(acfg, 0), tid, d * d, "gauss").view(d, d)
+        W.append((w * (1.2 / d ** 0.5)).to(dev))
+    mod = api.MhaModule(X, *W, n_heads=H, T=T, seq_chunk=seq_chunk)
+    mod.sp_mha_init(True)
+    prm = api.MhaParams(a_steps=2, z_steps=2, seq_chunk=seq_chunk)
+
+    def timed(fn):
+        fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        mod.check_status()
+        return a.elapsed_time(b) / steps
+
+    ms_step = timed(lambda: mod.sp_mha_step(prm))
+    ms_refit = timed(lambda: mod.sp_mha_value_refit(None, cfg.rho, True))
+    out = {"workload": f"attention module d={d}, {H} heads of {d // H}, {n_seq} sequences of {T} tokens "
+                       f"({seq_chunk} per chunk), bf16, causal",
+           "mha_step_ms": ms_step, "mha_step_note": "2 gradient steps of Eq. (85), Eq. (86) in closed form, 2 gradient "
+                                                    "steps of Eq. (87); accumulators of the recoveries rebuilt",
+           "value_refit_ms": ms_refit, "value_refit_note": "W_V from P and Aattn: one ridge system of size d per head",
+           "tokens": n_seq * T}
+    del mod, X, W
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     args = parse()
     from paper_2510_03246_b200 import synth
@@ -561,6 +608,10 @@ def main():
             del wmod, wX, wW1, wW2, wWg
             torch.cuda.empty_cache()
 
+    attention = None
+    if world == 1 and not args.no_attention and cfg.storage == "bf16":
+        attention = attention_module_timing(cfg, dev)
+
     cpu = None
     if not args.no_cpu_baseline:
         cpu = cpu_baseline(cfg, args.cpu_sample_tokens)
@@ -571,7 +622,7 @@ def main():
             "vs_baseline": None, "dtype": DTYPE_NAME[cfg.storage], "data": "synthetic",
             "config": config_dict(cfg, args, world, by_tokens),
             "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "roofline_hbm": roofline_hbm, "e2e": e2e,
-            "cpu_baseline": cpu, "fixed_mask": fixed, "workloads": workloads,
+            "cpu_baseline": cpu, "fixed_mask": fixed, "workloads": workloads, "attention_module": attention,
             "profiled_ms_per_step": ms_prof / args.steps, "graph_replay_ms_per_step": graph_ms,
             "profile_note": "value / ms_per_step: timed loop with nothing but the library's launches; roofline, "
                             "roofline_hbm and breakdown: the same steps repeated right after it with a CUDA event pair "
