@@ -72,12 +72,11 @@ constexpr size_t diag_smem_bytes() { return 2 * sizeof(T) * NB * (NB + 1); }
 
 template <typename T>
 cudaError_t prepare_diag_kernel() {
-  static bool done = false;
-  if (done) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(chol_diag_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)diag_smem_bytes<T>());
-  if (e == cudaSuccess) done = true;
-  return e;
+  static PerDeviceOnce once;           // one per instantiation; the attribute belongs to the device's context
+  return once.run([] {
+    return cudaFuncSetAttribute(chol_diag_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)diag_smem_bytes<T>());
+  });
 }
 
 template <typename T>

@@ -465,12 +465,13 @@ template <bool TRANS>
 cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, const float* dinv, __nv_bfloat16* S,
                                int64_t lds, int64_t s_seg, bool write_f32, int32_t* status, cudaStream_t stream,
                                PanelNear near = PanelNear{nullptr, 0, nullptr}) {
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(panel_apply_kernel<TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)PA_SMEM_NEAR);
+  static PerDeviceOnce attr_once;      // one per instantiation; the attribute belongs to the device's context
+  {
+    cudaError_t e = attr_once.run([] {
+      return cudaFuncSetAttribute(panel_apply_kernel<TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)PA_SMEM_NEAR);
+    });
     if (e != cudaSuccess) return e;
-    attr = true;
   }
   if (rows <= 0) return cudaSuccess;
   count_launch();
