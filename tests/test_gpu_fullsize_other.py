@@ -61,6 +61,23 @@ def run(request):
     mod.check_status()
     snap.update(Z1_rows=np64(mod.Z[ti]), W1=np64(mod.W1), W2=np64(mod.W2), mask=mod.mask.cpu().numpy().copy(),
                 scores=mod.scores.cpu().numpy().copy(), report=mod.read_report())
+    assert snap["report"]["factor_reused"] == 0.0        # the first step starts from a mask that keeps every channel
+    # further steps until one recovers W2 on the kept support from the unrestricted factor (the mask of that step
+    # keeps the channels of the one before): its inputs and outputs for test_later_step_reuses_the_factor
+    snap["later"] = None
+    for it in range(3):
+        torch.cuda.synchronize()
+        acc = dict(G_A=mod.G_A.cpu().numpy().copy(), R2=mod.R2.cpu().numpy().copy(), mask_before=mod.mask.cpu().numpy().copy())
+        mod.sp_admm_step(p)
+        torch.cuda.synchronize()
+        mod.check_status()
+        rep = mod.read_report()
+        mask_after = mod.mask.cpu().numpy().copy()
+        assert rep["factor_reused"] == float(np.array_equal(mask_after, acc["mask_before"]))
+        if rep["factor_reused"] == 1.0:
+            acc.update(W2=np64(mod.W2), mask=mask_after, step=it + 2)
+            snap["later"] = acc
+            break
     del mod, X, Wu, W2, Wg
     torch.cuda.empty_cache()
     return snap
@@ -148,3 +165,19 @@ def test_mask_and_token_update(run):
     print(f"{cfg.name}: max relative error of Z on the sampled tokens {relerr(got, Znew):.2e} (tolerance {TOLB:.0e})")
     assert relerr(got, Znew) < TOLB
     assert run["report"]["kept"] == cfg.k_keep and run["report"]["res_act"] >= 0.0
+
+
+def test_later_step_reuses_the_factor(run):
+    """A later step whose mask keeps the channels of the step before recovers W2 on the kept support by a backward
+    sweep with the leading block of the unrestricted factor (kept counts 6554, 3302 and 5734: leading blocks of 6656, 3328 and 5760 columns with padding; the two largest
+    systems are factorised with outer blocks of 512 columns): W2 against the fp64
+    restricted ridge solution from the accumulators the GPU held when that step began."""
+    cfg = run["cfg"]
+    later = run["later"]
+    assert later is not None, "no step reused the factor within three further steps"
+    G_A = later["G_A"].astype(np.float64)
+    rho2 = O.effective_ridge(G_A, cfg.rho, True)
+    W2 = O.restricted_refit(later["R2"].astype(np.float64), G_A, later["mask"], rho2)
+    print(f"{cfg.name}: step {later['step']} reused the factor, W2 error {relerr(later['W2'], W2):.2e}")
+    assert relerr(later["W2"], W2) < TOLB
+    assert np.all(later["W2"][:, later["mask"] == 0] == 0)
