@@ -1481,6 +1481,11 @@ struct ValueRefitPlan {
   void* R;      // regressors of one head and chunk: bf16 hi | lo [cap, 2 pad64(d)], or fp32 [cap, d]
   float* G;     // [H][d, d]   sum over sequences of R^T R per head (lower triangle)
   float* Cv;    // [H][d_h, d] sum over sequences of Aattn_i^T R per head
+  // the heads' systems solved together (bf16 mode, d a multiple of the solver's block): see potrf_potrs_tc_batched
+  bool batched;
+  float *Gs_all, *dinv_all;
+  void *P_all, *Xs_all;
+  double* rho_all;
   size_t bytes;
 };
 
@@ -1501,6 +1506,17 @@ ValueRefitPlan plan_value_refit(void* ws, int64_t d, int64_t H, int64_t T, int64
   p.R = c.take_bytes(p.bf16 ? (size_t)p.cap * 2 * split_kpad(d) * 2 : (size_t)p.cap * d * 4);
   p.G = c.take<float>((size_t)H * d * d);
   p.Cv = c.take<float>((size_t)d * d);
+  p.batched = p.bf16 && d % kCholTcNB == 0;
+  p.Gs_all = p.dinv_all = nullptr;
+  p.P_all = p.Xs_all = nullptr;
+  p.rho_all = nullptr;
+  if (p.batched) {
+    p.rho_all = c.take<double>((size_t)H);
+    p.Gs_all = c.take<float>((size_t)H * (d + p.dh) * d);
+    p.dinv_all = c.take<float>((size_t)H * dinv_elems(d));
+    p.P_all = c.take_bytes((size_t)H * (d + p.dh) * 3 * d * 2);
+    p.Xs_all = c.take_bytes((size_t)H * 2 * p.dh * 3 * kCholTcNB * 2);
+  }
   p.bytes = align_up(c.off, 256);
   return p;
 }
@@ -1587,9 +1603,35 @@ sp_status sp_mha_value_refit(const sp_mha_module* m, const sp_mha_state* st, con
       }
     }
   }
-  // ---- W_V,i = C_i (G_i + rho_i I)^-1, one regularised solve per kept head.  A solve is a chain of short kernels that
-  // leaves most SMs idle, and the heads' systems are independent: they alternate between the caller's stream and the
-  // library's side stream, each with its own buffers and assisting stream.
+  // ---- W_V,i = C_i (G_i + rho_i I)^-1, one regularised solve per kept head.
+  if (p.batched) {
+    // all kept heads' systems together: every step of the factorisation and of the sweep is one launch over them
+    const int64_t a_bs = (d + dh) * d, d_bs = (int64_t)dinv_elems(d);
+    int nk = 0;
+    for (int64_t i = 0; i < H; ++i) {
+      if (!kept(i)) continue;
+      float* Gs = p.Gs_all + (size_t)nk * a_bs;
+      CU(effective_ridge(p.G + (size_t)i * d * d, d, d, rho, rho_relative, p.rho_all + nk, s));
+      CU(load_spd<float>(p.G + (size_t)i * d * d, d, d, p.rho_all + nk, Gs, d, s));
+      CU(gather_cols<float>(p.Cv + (size_t)i * dh * d, d, nullptr, dh, d, Gs + (size_t)d * d, d, s));
+      ++nk;
+    }
+    if (nk > 0) {
+      ProfScope prof(PK_SOLVE, (double)nk * ((double)d * d * d / 3.0 + 2.0 * (double)dh * d * d), 0.0, s);
+      SPCHK(potrf_potrs_tc_batched(p.Gs_all, d, dh, nk, a_bs, p.dinv_all, d_bs, p.P_all, p.Xs_all, status_dev, s));
+    }
+    nk = 0;
+    for (int64_t i = 0; i < H; ++i) {
+      if (!kept(i)) continue;
+      const float* Xi = p.Gs_all + (size_t)nk * a_bs + (size_t)d * d;
+      CU(scatter_cols<float>(Xi, d, nullptr, dh, d, d, Wv_out + (size_t)i * dh * ldw, ldw, s));
+      ++nk;
+    }
+    return SP_OK;
+  }
+  // Otherwise one system at a time.  A solve is a chain of short kernels that leaves most SMs idle, and the heads'
+  // systems are independent: they alternate between the caller's stream and the library's side stream, each with its
+  // own buffers and assisting stream.
   SideStream* side = side_stream();
   JoinOnExit join_guard{side, s};
   if (side) {

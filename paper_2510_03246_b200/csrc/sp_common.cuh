@@ -189,6 +189,13 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
 // n_factor > n: the factor in P / dinv / Lf is that of a larger system of n_factor rows and the solve uses its leading
 // n x n block, which is the factor of the system's leading block (n a multiple of kCholTcNB).
 
+// `batch` independent systems of one size n (a multiple of kCholTcNB) with m right-hand sides each, every step one launch
+// over all of them.  System b: A + b * a_bs = [n + m, n] fp32 (lower triangle of the matrix, then the right-hand sides
+// B of X (L L^T) = B; on return they hold X), dinv + b * d_bs (room as for potrf_lower_tc), P = batch x
+// [n + m, 3 n] bf16, Xs = batch x 2 x [m, 3 * kCholTcNB] bf16.
+sp_status potrf_potrs_tc_batched(float* A, int64_t n, int64_t m, int batch, int64_t a_bs, float* dinv, int64_t d_bs,
+                                 void* P, void* Xs, int32_t* status_dev, cudaStream_t stream);
+
 // ---- elementwise / reduction launchers (sp_elementwise.cu) ------------------------------------------------------
 cudaError_t convert_matrix(const void* src, int32_t sdt, int64_t lds, void* dst, int32_t ddt, int64_t ldd,
                            int64_t rows, int64_t cols, cudaStream_t stream);

@@ -49,8 +49,10 @@ constexpr size_t DIAG_SMEM = (size_t)TB * DIAG_TPAD * sizeof(float);
 // Global input and output go through a padded shared tile so that every global access is a full coalesced row.
 __global__ void __launch_bounds__(DIAG_THREADS) chol_diag128_kernel(float* A, int64_t lda, int nb, float* dinv,
                                                                     int64_t row0, int32_t* status,
-                                                                    const int32_t* skip) {
+                                                                    const int32_t* skip, int64_t a_bs, int64_t d_bs) {
   if (skip != nullptr && *skip != 0) return;                  // conditional launch (see SkipScope)
+  A += (int64_t)blockIdx.x * a_bs;                            // batched launch: one CTA per system
+  dinv += (int64_t)blockIdx.x * d_bs;
   extern __shared__ __align__(16) float diag_tile[];          // T[TB][TB + 1]
   float (*T)[DIAG_TPAD] = reinterpret_cast<float (*)[DIAG_TPAD]>(diag_tile);
   __shared__ __align__(16) float W[2][4][TB];   // W[k][index]: conflict-free 16-byte accesses along the index
@@ -298,6 +300,10 @@ struct PanelNear {
   int64_t ldl;
   float* Xn;
 };
+// Batched launch of the panel kernel (grid.y = systems): element strides between the systems' arrays
+struct PanelBatch {
+  int64_t x = 0, dinv = 0, s = 0, near_l = 0;    // X (and the near columns), dinv, S, near.L
+};
 
 // X[i, 0:nb] <- X[i, 0:nb] inv(L)^T (TRANS == false) or X[i, 0:nb] inv(L) (TRANS == true), for `rows` rows.
 // dinv is the pair of TB x TB blocks written by chol_diag128_kernel.  The result is written back in fp32 (write_f32)
@@ -309,8 +315,12 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
                                                                  const float* __restrict__ dinv, __nv_bfloat16* S,
                                                                  int64_t lds, int64_t s_seg, int write_f32,
                                                                  int32_t* status, PanelNear near,
-                                                                 const int32_t* skip) {
+                                                                 const int32_t* skip, PanelBatch pb) {
   if (skip != nullptr && *skip != 0) return;
+  X += (int64_t)blockIdx.y * pb.x;
+  dinv += (int64_t)blockIdx.y * pb.dinv;
+  if (S) S += (int64_t)blockIdx.y * pb.s;
+  if (near.L) { near.L += (int64_t)blockIdx.y * pb.near_l; near.Xn += (int64_t)blockIdx.y * pb.x; }
   extern __shared__ __align__(128) float pa_smem[];
   float (*Lt)[TB] = reinterpret_cast<float (*)[TB]>(pa_smem);                       // Lt[k][c]
   float (*At)[PA_APAD] = reinterpret_cast<float (*)[PA_APAD]>(pa_smem + TB * TB);   // At[k][row]
@@ -464,7 +474,8 @@ __global__ void __launch_bounds__(PA_THREADS) panel_apply_kernel(float* X, int64
 template <bool TRANS>
 cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, const float* dinv, __nv_bfloat16* S,
                                int64_t lds, int64_t s_seg, bool write_f32, int32_t* status, cudaStream_t stream,
-                               PanelNear near = PanelNear{nullptr, 0, nullptr}) {
+                               PanelNear near = PanelNear{nullptr, 0, nullptr}, int batch = 1,
+                               PanelBatch pb = PanelBatch{}) {
   static PerDeviceOnce attr_once;      // one per instantiation; the attribute belongs to the device's context
   {
     cudaError_t e = attr_once.run([] {
@@ -477,8 +488,9 @@ cudaError_t launch_panel_apply(float* X, int64_t ldx, int64_t rows, int nb, cons
   count_launch();
   const bool with_near = TRANS && near.L != nullptr;
   ProfScope prof(PK_PANEL_APPLY, (with_near ? 4.0 : 2.0) * (double)rows * TB * TB, 0.0, stream);
-  panel_apply_kernel<TRANS><<<(unsigned)ceil_div(rows, PA_ROWS), PA_THREADS, with_near ? PA_SMEM_NEAR : PA_SMEM, stream>>>(
-      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status, near, skip_flag());
+  panel_apply_kernel<TRANS><<<dim3((unsigned)ceil_div(rows, PA_ROWS), (unsigned)batch), PA_THREADS,
+                              with_near ? PA_SMEM_NEAR : PA_SMEM, stream>>>(
+      X, ldx, rows, nb, dinv, S, lds, s_seg, write_f32 ? 1 : 0, status, near, skip_flag(), pb);
   return cudaGetLastError();
 }
 
@@ -678,7 +690,7 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       ProfScope prof(PK_CHOL_DIAG, (double)nb * nb * nb * (2.0 / 3.0), 0.0, stream);
       chol_diag128_kernel<<<1, DIAG_THREADS, DIAG_SMEM, stream>>>(from_scratch ? S : A + k0 * lda + k0,
                                                                   from_scratch ? (int64_t)TB : lda, nb, dk, k0,
-                                                                  status_dev, skip);
+                                                                  status_dev, skip, 0, 0);
       if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
     }
     const int64_t rem = n - k0 - nb;
@@ -921,6 +933,102 @@ sp_status potrs_right_tc(float* X, int64_t m, int64_t n, int64_t ldx, const void
   }
   return run_sweep(false);          // W L = Y, block columns right to left
 #undef SP_CUDA_OK
+}
+
+
+// ---------------------------------------------------------------------------------------------------------------
+// B independent systems of one size, solved together: every step of the factorisation and of the backward sweep is
+// one launch over all systems (diagonal blocks: one CTA per system; panels: grid.y = systems; updates: one batched
+// tensor-core launch), so the parallelism comes from the batch and no lookahead or second stream is used.
+// Layout: system b at A + b * a_bs ([n + m, n] fp32, the m right-hand sides below the matrix, lda = n), its bf16 parts
+// at P + b * (np + m) * 3 np, its inverse diagonal blocks at dinv + b * d_bs, its sweep buffers at Xs + b * 2 m 3 TB.
+// n must be a multiple of 128 here (the callers' systems are d x d with d % 128 == 0; others take the plain path).
+sp_status potrf_potrs_tc_batched(float* A, int64_t n, int64_t m, int batch, int64_t a_bs, float* dinv, int64_t d_bs,
+                                 void* Pv, void* Xsv, int32_t* status_dev, cudaStream_t stream) {
+  if (n % TB != 0 || batch < 1 || m < 1) return SP_ERR_SHAPE;
+  __nv_bfloat16* P = reinterpret_cast<__nv_bfloat16*>(Pv);
+  __nv_bfloat16* Xs = reinterpret_cast<__nv_bfloat16*>(Xsv);
+  const int64_t np = n, ldp = 3 * np, lda = n;
+  const int64_t p_bs = (np + m) * ldp;
+  const int64_t nblk = n / TB;
+  const int32_t* skip = skip_flag();
+  static PerDeviceOnce attr_once;
+  if (attr_once.run([] {
+        return cudaFuncSetAttribute(chol_diag128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM);
+      }) != cudaSuccess)
+    return SP_ERR_CUDA;
+  TcBatch bt;
+  bt.nb0 = batch; bt.nb1 = 1;
+  bt.a_s0 = bt.b_s0 = p_bs; bt.a_s1 = bt.b_s1 = p_bs;
+  bt.c_s0 = bt.cin_s0 = a_bs; bt.c_s1 = bt.cin_s1 = a_bs;
+  bt.a_planes = bt.b_planes = 1; bt.a_plane = bt.b_plane = 0;
+  // ---- factorisation; the appended rows receive their forward substitution on the way
+  for (int64_t kb = 0; kb < nblk; ++kb) {
+    const int64_t k0 = kb * TB;
+    float* dk = dinv + kb * 2 * TB * TB;
+    count_launch();
+    chol_diag128_kernel<<<batch, DIAG_THREADS, DIAG_SMEM, stream>>>(A + k0 * lda + k0, lda, TB, dk, k0, status_dev, skip,
+                                                                  a_bs, d_bs);
+    if (cudaGetLastError() != cudaSuccess) return SP_ERR_CUDA;
+    const int64_t rem = n - k0 - TB, prow = rem + m;
+    PanelBatch pb;
+    pb.x = a_bs; pb.dinv = d_bs; pb.s = p_bs;
+    if (launch_panel_apply<false>(A + (k0 + TB) * lda + k0, lda, prow, TB, dk, P + (k0 + TB) * ldp + k0, ldp, np, true,
+                                  status_dev, stream, PanelNear{nullptr, 0, nullptr}, batch, pb) != cudaSuccess)
+      return SP_ERR_CUDA;
+    if (rem <= 0) break;
+    TcOperand ta{P + (k0 + TB) * ldp, ldp, true}, tb{P + (k0 + TB) * ldp, ldp, true};
+    ta.kext = tb.kext = ldp;
+    ta.mnext = prow;
+    tb.mnext = rem;
+    TcSegments sg;
+    sg.nseg = 6;
+    for (int q = 0; q < 6; ++q) {
+      sg.a_k[q] = (int32_t)(kPartA[q] * np + k0);
+      sg.b_k[q] = (int32_t)(kPartB[q] * np + k0);
+    }
+    float* A22 = A + (k0 + TB) * lda + (k0 + TB);
+    sp_status st = gemm_tc(prow, rem, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1}, OutOperand{A22, SP_F32, lda},
+                           false, status_dev, stream, &sg,
+                           ((double)rem * rem + 2.0 * (double)m * rem) * TB * batch, 0, &bt);
+    if (st != SP_OK) return st;
+  }
+  // ---- backward sweep W L = Y on the appended rows, block columns right to left
+  float* X = A + n * lda;                       // [m, n] per system
+  const int64_t lds = 3 * TB, xs_bs = 2 * m * lds;
+  const bool fuse_near = ceil_div(m, (int64_t)PA_ROWS) * batch <= 148;
+  TcBatch bs = bt;
+  bs.a_s0 = bs.a_s1 = xs_bs;
+  for (int64_t step = 0; step < nblk; ++step) {
+    const int64_t jb = nblk - 1 - step, j0 = jb * TB;
+    const float* dj = dinv + jb * 2 * TB * TB;
+    __nv_bfloat16* Xcur = Xs + (step & 1) * m * lds;
+    const bool near_in_panel = fuse_near && j0 > 0;
+    PanelNear pn{nullptr, 0, nullptr};
+    if (near_in_panel) pn = PanelNear{A + j0 * lda + (j0 - TB), lda, X + (j0 - TB)};
+    PanelBatch pb;
+    pb.x = a_bs; pb.dinv = d_bs; pb.s = xs_bs; pb.near_l = a_bs;
+    if (launch_panel_apply<true>(X + j0, lda, m, TB, dj, Xcur, lds, TB, true, status_dev, stream, pn, batch, pb) !=
+        cudaSuccess)
+      return SP_ERR_CUDA;
+    const int64_t w = near_in_panel ? j0 - TB : j0;     // columns still to be updated by a product: [0, w)
+    if (w <= 0) continue;
+    TcOperand ta{Xcur, lds, true}, tb{P + j0 * ldp, ldp, false};
+    ta.kext = lds;
+    ta.mnext = m;
+    tb.kext = n - j0;
+    tb.mnext = ldp;
+    TcSegments sg;
+    sg.nseg = 6;
+    for (int q = 0; q < 6; ++q) {
+      sg.a_k[q] = kPartA[q] * TB;
+      sg.b_mn[q] = (int32_t)(kPartB[q] * np);
+    }
+    sp_status st = gemm_tc(m, w, TB, -1.f, ta, tb, 1.f, Operand{X, SP_F32, lda, 1}, OutOperand{X, SP_F32, lda}, false,
+                           status_dev, stream, &sg, 2.0 * (double)m * w * TB * batch, 0, &bs);
+    if (st != SP_OK) return st;
+  }
+  return SP_OK;
 }
 
 }  // namespace sp
