@@ -640,6 +640,53 @@ def test_kept_support_recovery_reuses_the_factor(cfg, overlap):
     mod.check_status()
 
 
+def test_captured_step_takes_either_branch_on_replay():
+    """One sp_admm_step captured into a CUDA graph by the caller and replayed: the choice between the backward sweep
+    with the reused factor and the restricted factorisation is a device flag read by kernels that were all captured, so
+    ONE graph serves steps whose mask stays and steps whose mask changes.  Every replay is compared with an eager step
+    of a second module brought to the same state (the two run the same kernels, hence the same arithmetic up to the
+    order of the accumulating adds)."""
+    cfg = SMALL_BF16
+    k = cfg.k_keep
+    p = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, token_chunk=512)
+    mods = []
+    for _ in range(2):
+        mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=k)
+        mod.sp_ffn_init()
+        mod.sp_admm_step(p)                        # warm-up outside the capture (one-time set-up of the library)
+        mods.append(mod)
+    torch.cuda.synchronize()
+    cap_mod, ref_mod = mods
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=cap, capture_error_mode="relaxed"):
+        cap_mod.sp_admm_step(p)
+    torch.cuda.synchronize()                       # (capturing does not run the step)
+    tol = TOL[X.dtype]
+    seen = set()
+    for plant in ["as is", "rolled", "as is", "as is"]:
+        if plant == "rolled":                      # another support with the same count: the coming step must refactorise
+            m = torch.roll(cap_mod.mask, 1)
+            cap_mod.mask.copy_(m)
+            ref_mod.mask.copy_(m)
+        mask_before = cap_mod.mask.cpu().numpy().copy()
+        g.replay()
+        ref_mod.sp_admm_step(p)
+        torch.cuda.synchronize()
+        cap_mod.check_status()
+        ref_mod.check_status()
+        rep_c, rep_r = cap_mod.read_report(), ref_mod.read_report()
+        assert torch.equal(cap_mod.mask, ref_mod.mask)
+        assert rep_c["factor_reused"] == rep_r["factor_reused"] == float(
+            np.array_equal(cap_mod.mask.cpu().numpy(), mask_before))
+        seen.add(rep_c["factor_reused"])
+        for name in ("W1", "W2", "Z", "G_A", "R1", "R2"):
+            # far below the parity tolerance: only the order of the accumulating adds differs between the two runs
+            assert relerr(np64(getattr(cap_mod, name)), np64(getattr(ref_mod, name))) < tol / 20, name
+    assert seen == {0.0, 1.0}
+
+
 # ------------------------------------------------------------------------------------------------ SwiGLU modules
 SWIGLU_F32 =synth.scaled(synth.CONFIGS["C4"], d=88, n=300, tokens=520, sparsity=0.5, storage="f32")
 SWIGLU_BF16 = synth.scaled(synth.CONFIGS["C4"], d=264, n=776, tokens=1300, sparsity=0.7, outlier_frac=0.02)
