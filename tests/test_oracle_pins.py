@@ -411,6 +411,46 @@ def test_block_descent_monotone_with_fixed_mask_and_exact_rule():
     assert vals[-1] < vals[0]
 
 
+def test_pruned_channels_decay_geometrically_while_the_mask_stays():
+    """A consequence of the updates of Appendix A.1 that the CUDA path uses to skip work: a pruned channel has a zero
+    row in W1 and a zero column in W2, so a = phi(z), z1 = 0 and (ReLU, no dual, either select rule)
+    z_new = beta / (alpha + beta) * max(z, 0).  From the second consecutive step with the same mask on, its row of A is
+    therefore c = beta / (alpha + beta) times its row of the step before, and so are its row of Z and its columns /
+    rows of the accumulators: G_A[pruned, pruned] scales by c^2, R2[:, pruned] and R1[pruned, :] by c.  Checked on the
+    oracle's own steps, for both select rules; kept channels do not obey it."""
+    X, W1_0, W2_0 = _small_module(31)
+    for rule in ("paper", "exact"):
+        st, Y = O.ffn_init(X, W1_0, W2_0)
+        alpha, beta = 1.3, 0.7
+        c = beta / (alpha + beta)
+        p = O.AdmmParams(alpha=alpha, beta=beta, rho=0.05, k_keep=5, z_rule=rule)
+        prev = None
+        obeyed = []
+        for it in range(6):
+            mask_before = None if st.mask is None else st.mask.copy()
+            s, I, rep, A = O.admm_step(st, X, Y, W1_0, p)
+            pruned = st.mask == 0
+            if prev is not None and np.array_equal(st.mask, prev["mask"]) and prev["mask_before"] is not None \
+                    and np.array_equal(prev["mask"], prev["mask_before"]):
+                # the same mask in this step, the one before it, and the one before that
+                assert np.allclose(A[pruned], c * prev["A"][pruned], rtol=1e-12, atol=0)
+                assert np.allclose(st.Z[pruned], c * prev["Z"][pruned], rtol=1e-12, atol=0)
+                assert np.allclose(st.G_A[np.ix_(pruned, pruned)], c * c * prev["G_A"][np.ix_(pruned, pruned)], rtol=1e-12)
+                assert np.allclose(st.R2[:, pruned], c * prev["R2"][:, pruned], rtol=1e-12)
+                assert np.allclose(st.R1[pruned], c * prev["R1"][pruned], rtol=1e-12)
+                obeyed.append(it)
+            elif prev is not None and np.array_equal(st.mask, prev["mask"]):
+                # second step with this mask: A follows already (z of the step before was c max(z, 0) >= 0)
+                assert np.allclose(A[pruned], c * prev["A"][pruned], rtol=1e-12, atol=0)
+            prev_kept_A = None if prev is None else prev["A"]
+            prev = dict(mask=st.mask.copy(), mask_before=mask_before, A=A.copy(), Z=st.Z.copy(), G_A=st.G_A.copy(),
+                        R1=st.R1.copy(), R2=st.R2.copy())
+        assert obeyed, "the mask never stayed for three steps in this run"
+    # the kept channels do not follow the rule
+    kept = st.mask == 1
+    assert not np.allclose(A[kept], c * prev_kept_A[kept], rtol=1e-3)
+
+
 def test_admm_step_equals_its_parts_and_keeps_budget():
     X, W1_0, W2_0 = _small_module(23)
     st, Y = O.ffn_init(X, W1_0, W2_0)
