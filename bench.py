@@ -63,6 +63,9 @@ def parse():
     ap.add_argument("--workloads", default="C3,C4,C5",
                     help="1 GPU: further workloads measured after the main one and reported under `workloads` "
                          "(empty string: none)")
+    ap.add_argument("--no-pruned-decay", action="store_true",
+                    help="do not keep the ordered accumulators that let a step scale, instead of recompute, the parts of "
+                         "G_A and R2 that belong to pruned channels while the mask stays")
     ap.add_argument("--no-attention", action="store_true",
                     help="skip the timing of the attention module's step and W_V recovery (`attention_module`)")
     ap.add_argument("--workload-steps", type=int, default=5)
@@ -257,7 +260,8 @@ def build_module(cfg, args, dev, layer, by_tokens, world):
     X = synth.make_activations(cfg_local, layer, device=dev)        # another seed per rank: disjoint tokens
     W1_0, W2_0 = synth.make_weights(cfg, wl, device=dev)
     Wg_0 = synth.make_gate_weights(cfg, layer, device=dev) if cfg.act == "swiglu" else None
-    mod = api.FfnModule(X, W1_0, W2_0, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0)
+    mod = api.FfnModule(X, W1_0, W2_0, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=Wg_0,
+                        pruned_decay=not args.no_pruned_decay)
     if by_tokens:
         parallel.token_sharded_init([mod])
     else:

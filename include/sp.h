@@ -118,6 +118,17 @@ typedef struct {
   float* Gate;     /* [N, n] ld = n   SP_ACT_SWIGLU only: g = SiLU(Wg_0 X), written by sp_ffn_init, then read-only   */
   float* G_X_inv;  /* [d, d]          optional cache (may be NULL): (G_X + rho1 I)^-1 written by
                                       sp_ffn_cache_input_inverse; read by sp_admm_step in bf16 mode                  */
+  /* Optional (all three or none; used with bf16 storage, SP_ACT_RELU, dual_mode == 0, n % 4 == 0): the accumulators
+   * of the new A in "kept channels first" order, kept from one step to the next.  A pruned channel has a zero row in
+   * W1 and a zero column in W2, so its a = phi(z) and z_new = beta / (alpha + beta) * max(z, 0): from the second step
+   * with an unchanged mask on, its row of A is c = beta / (alpha + beta) times the row of the step before.  With these
+   * buffers sp_admm_step then obtains G_A[pruned, pruned] and R2[:, pruned] by scaling last step's values (c^2, c)
+   * instead of contracting over the tokens again; the decision is taken on the device from decay_tag, which records
+   * the channel order, k_keep and c of the last token pass.  G_A and R2 above are still written in channel order by
+   * every step.  Whoever changes Z outside the library must set decay_tag[1] = -1; sp_ffn_init does. */
+  float* G_A_perm;     /* [n, n]                                                                                     */
+  float* R2_perm;      /* [d, n]                                                                                     */
+  int32_t* decay_tag;  /* int32 [n + 8]                                                                              */
 } sp_ffn_state;
 
 typedef struct {
@@ -148,6 +159,8 @@ typedef struct {
   double kept;      /* number of kept units                                                                       */
   double factor_reused; /* 1: the recovery on the kept support was one backward sweep with the leading block of the
                            unrestricted factor (the new mask kept the channels of the previous one); else 0         */
+  double pruned_scaled; /* 1: G_A[pruned, pruned] and R2[:, pruned] were obtained by scaling last step's values
+                           (see sp_ffn_state.G_A_perm); else 0                                                      */
 } sp_step_report;
 
 /* Inputs of sp_struct_scores; only the fields of the chosen kind are read. */

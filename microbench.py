@@ -47,11 +47,18 @@ def gemm_cases(reps, warm):
         ("E = Ypre - H W2^T (bf16 out)", T, D, N // 2, True, True, bf, 1.0, False),
         ("D = E Q^T (f32 out)", T, N // 2, D, True, True, f32, 0.0, False),
         ("z1 = X [W1hi W1lo]^T (f32 out)", T, N // 2, 2 * D, True, True, f32, 0.0, False),
-        # the accumulator products as a step issues them: the fused update leaves A channel-major (K-major here)
-        ("G_A += A^T A (lower, A K-major)", N, N, T, True, True, f32, 1.0, True),
-        ("R2 += Ypre^T A (A K-major)", D, N, T, False, True, f32, 1.0, False),
+        # the accumulator products as a step issues them while the mask stays: the fused update leaves A channel-major
+        # (K-major here) with the kept channels first, and only the kept columns are contracted anew
+        ("G_A[:, kept] += A^T A_kept (lower)", N, N // 2, T, True, True, f32, 1.0, True),
+        ("R2[:, kept] += Ypre^T A_kept", D, N // 2, T, False, True, f32, 1.0, False),
         ("R1 += Z^T X", N, D, T, False, False, f32, 1.0, False),
         ("solve update (K = 6 x 128)", 2048, 4096, 768, True, True, f32, 1.0, False),
+        # the pruned parts, contracted only in a step whose mask changed
+        ("G_A[pruned, pruned] (lower)", N // 2, N // 2, T, True, True, f32, 1.0, True),
+        ("R2[:, pruned]", D, N // 2, T, False, True, f32, 1.0, False),
+        # the full products of a module without the ordered accumulators
+        ("G_A += A^T A (lower, A K-major)", N, N, T, True, True, f32, 1.0, True),
+        ("R2 += Ypre^T A (A K-major)", D, N, T, False, True, f32, 1.0, False),
         # other operand layouts: row-major A (fp32-storage path, or when the objective is reported), and transposed
         # copies of Ypre / X that the module does not keep
         ("G_A with A row-major", N, N, T, False, False, f32, 1.0, True),
@@ -61,11 +68,12 @@ def gemm_cases(reps, warm):
     ]
     for name, M, Nn, K, ak, bk, cdt, beta, lower in cases:
         A = _rnd((M, K) if ak else (K, M), bf)
-        B = _rnd((Nn, K) if bk else (K, Nn), bf)
+        # the Gram products multiply a matrix by (the first rows of) itself
+        B = A[:Nn] if name.startswith("G_A") and ak and bk else _rnd((Nn, K) if bk else (K, Nn), bf)
         C = _rnd((M, Nn), cdt)
         ms = _timeit(lambda: api.sp_gemm(A, B, C, transA=not ak, transB=bk, alpha=1.0, beta=beta, lower_only=lower,
                                          use_tensor_cores=True, status=st), reps, warm)
-        fl = (1.0 if lower else 2.0) * M * Nn * K
+        fl = K * Nn * (2.0 * M - Nn) if lower else 2.0 * M * Nn * K     # lower: triangle of the square + rows below it
         print(f"{name:34s} {M:6d} x {Nn:6d} x {K:6d}  {ms:8.3f} ms  {fl / ms / 1e9:8.1f} TFLOP/s", flush=True)
     print("status", st.cpu().tolist())
 

@@ -55,7 +55,7 @@ class SpFfnState(C.Structure):
     _fields_ = [("Z", C.c_void_p), ("U", C.c_void_p), ("G_X", C.c_void_p), ("G_A", C.c_void_p), ("R1", C.c_void_p),
                 ("R2", C.c_void_p), ("absA", C.c_void_p), ("W1", C.c_void_p), ("W2", C.c_void_p),
                 ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p), ("Gate", C.c_void_p),
-                ("G_X_inv", C.c_void_p)]
+                ("G_X_inv", C.c_void_p), ("G_A_perm", C.c_void_p), ("R2_perm", C.c_void_p), ("decay_tag", C.c_void_p)]
 
 
 class SpAdmmParams(C.Structure):
@@ -86,7 +86,8 @@ class SpMhaParams(C.Structure):
                 ("eta_z", C.c_double), ("causal", C.c_int32), ("reserved", C.c_int32), ("seq_chunk", C.c_int64)]
 
 
-REPORT_FIELDS = ["res_act", "res_out", "res_in", "z_sq", "a_sq", "rho1_eff", "rho2_eff", "kept", "factor_reused"]
+REPORT_FIELDS = ["res_act", "res_out", "res_in", "z_sq", "a_sq", "rho1_eff", "rho2_eff", "kept", "factor_reused",
+                 "pruned_scaled"]
 
 _lib = None
 
@@ -466,7 +467,8 @@ class FfnModule:
 
     def __init__(self, X: torch.Tensor, W1_0: torch.Tensor, W2_0: torch.Tensor, dual_mode: bool = False,
                  token_chunk: int = 0, overlap_k: int = 0, Wg_0: torch.Tensor | None = None,
-                 scores: torch.Tensor | None = None, mask: torch.Tensor | None = None, ws_pool: dict | None = None):
+                 scores: torch.Tensor | None = None, mask: torch.Tensor | None = None, ws_pool: dict | None = None,
+                 pruned_decay: bool = True):
         """overlap_k > 0: also reserve the optional workspace tail that lets sp_admm_step compute z1 of all tokens
         beside the kept-support recovery, sized for overlap_k kept units (see sp_admm_overlap_bytes).
         Wg_0 (gate projection [n, d]) makes the module a SwiGLU one: W1_0 is then its up projection.
@@ -511,6 +513,13 @@ class FfnModule:
         self.status = new_status(dev)
         self.token_chunk = token_chunk
         self.overlap_k = int(overlap_k)
+        # ordered accumulators that let a step scale, instead of recompute, the parts of G_A and R2 that belong to
+        # pruned channels while the mask stays (see sp_ffn_state.G_A_perm); ReLU modules without the dual variable
+        self.G_A_perm = self.R2_perm = self.decay_tag = None
+        if pruned_decay and X.dtype == torch.bfloat16 and Wg_0 is None and not dual_mode and n % 4 == 0:
+            self.G_A_perm = torch.empty(n, n, **f32)
+            self.R2_perm = torch.empty(d, n, **f32)
+            self.decay_tag = torch.full((n + 8,), -1, dtype=torch.int32, device=dev)
         self._pool = ws_pool if ws_pool is not None else {}
         self.iteration = 0
 
@@ -530,7 +539,8 @@ class FfnModule:
         return SpFfnState(self.Z.data_ptr(), _ptr(self.U), self.G_X.data_ptr(), self.G_A.data_ptr(),
                           self.R1.data_ptr(), self.R2.data_ptr(), self.absA.data_ptr(), self.W1.data_ptr(),
                           self.W2.data_ptr(), self.scores.data_ptr(), self.mask.data_ptr(),
-                          self.importance.data_ptr(), _ptr(self.Gate), _ptr(self.G_X_inv))
+                          self.importance.data_ptr(), _ptr(self.Gate), _ptr(self.G_X_inv), _ptr(self.G_A_perm),
+                          _ptr(self.R2_perm), _ptr(self.decay_tag))
 
     def _workspace(self, chunk: int) -> torch.Tensor:
         need = max(workspace_bytes(SP_WS_ADMM_STEP, self.d, self.n, self.N, chunk, _dt(self.X)),

@@ -246,7 +246,8 @@ struct AdmmPlan {
   float *W1t, *W2t, *Qt, *T0, *Cf;
   float *W2cf, *W1c;           // compact fp32 copies on the kept support: W2[:, S] ([d, kp]) and W1[S, :] ([k, d])
   int32_t* perm;               // channels ordered "kept by the previous mask first" (reuse of the G_A factor)
-  int32_t* reuse_flags;        // [0] support changed, [1] support unchanged, [2] kept count of the previous mask
+  int32_t* reuse_flags;        // [0] support changed, [1] support unchanged, [2] kept count of the previous mask;
+                               // [4] / [5] channel order changed / unchanged against the last token pass (decay_tag)
   int32_t* grp_base;           // kept-channel map of the elementwise kernels
   uint8_t* grp_mask;
   void *W1b, *W2b, *Qtb;       // bf16 operands on the kept support (bf16 mode only)
@@ -283,7 +284,7 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.W2cf = c.take<float>((size_t)n * d + 8 * (size_t)d);
   p.W1c = p.bf16 ? nullptr : c.take<float>((size_t)n * d);
   p.perm = c.take<int32_t>((size_t)n);
-  p.reuse_flags = c.take<int32_t>(4);
+  p.reuse_flags = c.take<int32_t>(8);
   p.grp_base = c.take<int32_t>((size_t)ceil_div(n, (int64_t)8));
   p.grp_mask = c.take<uint8_t>((size_t)ceil_div(n, (int64_t)8));
   p.W1b = p.bf16 ? c.take_bytes((size_t)n * 2 * split_kpad(d) * csz) : nullptr;   // hi | lo split of W1
@@ -705,6 +706,7 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   InitPlan p = plan_init(ws, d, n, N, token_chunk, cdt);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const bool bf16 = p.bf16;
+  if (st->decay_tag != nullptr) CU(decay_tag_set(st->decay_tag, 0, 0.f, false, s));   // Z is rewritten
   const bool acc64 = !bf16;
   const bool gated = m->act == SP_ACT_SWIGLU;
   MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, w20{m->W2_0.ptr, SP_F32, m->W2_0.ld};
@@ -999,8 +1001,34 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
   if (rep_dev && prm->compute_objective && bf16) CU(convert_matrix(st->W2, SP_F32, n, p.W2fb, SP_BF16, n, d, n, s));
 
   // ---- 5b. token pass
+  // Pruned channels (ReLU, no dual variable): a = phi(z) and z_new = c max(z, 0) with c = beta / (alpha + beta), so
+  // from the second step with an unchanged mask on their rows of A are c times those of the step before.  The
+  // accumulators are therefore built in "kept channels first" order in buffers that persist in the state: the kept
+  // columns are contracted over the tokens in every step, the pruned x pruned block of G_A and the pruned columns
+  // of R2 only when the channel order differs from the last token pass; otherwise they are last step's values times
+  // c^2 and c (c of the step that wrote them).  The branch is a device flag; both sets of kernels are queued.
+  const bool decay = bf16 && !scores_only && m->act == SP_ACT_RELU && !prm->dual_mode && n % 4 == 0 && k < n &&
+                     p.chunk % 8 == 0 && !(rep_dev && prm->compute_objective) && st->G_A_perm != nullptr &&
+                     st->R2_perm != nullptr && st->decay_tag != nullptr && !misaligned(st->G_A_perm, 16) &&
+                     !misaligned(st->R2_perm, 16) && !misaligned(st->decay_tag, 4);
+  int32_t* order_changed = p.reuse_flags + 4;
+  int32_t* order_same = p.reuse_flags + 5;
+  if (decay) {
+    int32_t* tag = st->decay_tag;     // [1] k of the last pass (-1: none), [2] its c (float bits), [8..] its channel order
+    CU(mask_changed(st->mask, tag + 8, tag + 1, k, order_changed, s));
+    {
+      SkipScope unless_same(order_changed);
+      CU(scale_block(st->G_A_perm + (size_t)k * n + k, n, n - k, n - k, tag + 2, 2, s));
+      CU(scale_block(st->R2_perm + k, n, d, n - k, tag + 2, 1, s));
+    }
+    CU(mask_to_perm(st->mask, n, tag + 8, tag + 3, s));
+    CU(decay_tag_set(tag, k, (float)(prm->beta / (prm->alpha + prm->beta)), true, s));
+  } else if (!scores_only && st->decay_tag != nullptr) {
+    CU(decay_tag_set(st->decay_tag, 0, 0.f, false, s));    // Z changes without the ordered accumulators being rebuilt
+  }
   if (z1_ahead) CU(cudaStreamWaitEvent(s, side->z1_done, 0));
-  if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, reuse ? p.reuse_flags + 1 : nullptr, s));
+  if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, reuse ? p.reuse_flags + 1 : nullptr,
+                              decay ? order_same : nullptr, s));
   const size_t esz = bf16 ? 2 : 4;
   MatRef ga{st->G_A, SP_F32, n}, r1{st->R1, SP_F32, d}, r2{st->R2, SP_F32, n};
   for (int64_t t0 = 0, ci = 0; t0 < N; t0 += p.chunk, ++ci) {
@@ -1054,6 +1082,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     const int64_t Tld = (Tc + 7) / 8 * 8;
     const bool a_transposed = bf16 && n % 4 == 0 && !(rep_dev && prm->compute_objective) && Tld <= p.chunk;
     if (a_transposed) { ua.At_out = p.Ac; ua.ldt = Tld; }
+    if (decay) ua.at_kept_first = 1;     // (the pruned rows are still needed: G_A[pruned, kept] is contracted anew)
     const int nblk = fused_update_grid(Tc, n, &ua.row_blocks);
     CU(launch_fused_update(ua, s));
     if (rep_dev) CU(reduce_report(p.partial, nblk, rep_dev, ci > 0, prm->alpha, s));
@@ -1066,7 +1095,20 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     }
     CU(reduce_col_partials(p.absA_part, ua.row_blocks, n, st->absA, ci > 0, s));
     // accumulators of the new auxiliary variables
-    if (a_transposed) {
+    if (decay) {
+      // rows of A^T in "kept first" order: [0, k) kept, [k, n) pruned
+      MatRef act{p.Ac, cdt, Tld};
+      MatRef actp{reinterpret_cast<const __nv_bfloat16*>(p.Ac) + (size_t)k * Tld, cdt, Tld};
+      MatRef gp{st->G_A_perm, SP_F32, n}, gpp{st->G_A_perm + (size_t)k * n + k, SP_F32, n};
+      MatRef r2k{st->R2_perm, SP_F32, n}, r2p{st->R2_perm + k, SP_F32, n};
+      SPCHK(contract(n, k, Tc, 1.0, act, true, act, true, acc, gp, gp, true, acc64, bf16, status_dev, s));
+      SPCHK(contract(d, k, Tc, 1.0, yc, false, act, true, acc, r2k, r2k, false, acc64, bf16, status_dev, s));
+      {
+        SkipScope unless_changed(order_same);
+        SPCHK(contract(n - k, n - k, Tc, 1.0, actp, true, actp, true, acc, gpp, gpp, true, acc64, bf16, status_dev, s));
+        SPCHK(contract(d, n - k, Tc, 1.0, yc, false, actp, true, acc, r2p, r2p, false, acc64, bf16, status_dev, s));
+      }
+    } else if (a_transposed) {
       MatRef act{p.Ac, cdt, Tld};
       SPCHK(contract(n, n, Tc, 1.0, act, true, act, true, acc, ga, ga, true, acc64, bf16, status_dev, s));
       SPCHK(contract(d, n, Tc, 1.0, yc, false, act, true, acc, r2, r2, false, acc64, bf16, status_dev, s));
@@ -1076,7 +1118,13 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     }
     SPCHK(contract(n, d, Tc, 1.0, zb, false, xc, false, acc, r1, r1, false, acc64, bf16, status_dev, s));
   }
-  CU(symmetrize_lower(st->G_A, n, n, s));
+  if (decay) {
+    // the accumulators in channel order for the next step's weight phase and for the caller
+    CU(unpermute_gram(st->G_A_perm, st->decay_tag + 8, n, st->G_A, s));
+    CU(unpermute_cols(st->R2_perm, st->decay_tag + 8, d, n, st->R2, s));
+  } else {
+    CU(symmetrize_lower(st->G_A, n, n, s));
+  }
   join_guard.armed = false;
   return SP_OK;
 }

@@ -25,7 +25,9 @@ enum ProfKind : int {
   PK_GEMM_TC = 0, PK_GEMM_SIMT = 1, PK_SOLVE = 2, PK_FUSED_UPDATE = 3, PK_PREP_H = 4, PK_SCORES = 5, PK_TOPK = 6,
   PK_ELEMENTWISE = 7, PK_ALLOCATE = 8, PK_CHOL_DIAG = 9, PK_PANEL_APPLY = 10,
   PK_GEMM_TC_SHARED = 11,   // tensor-core GEMMs launched on a subset of the SM pairs, beside other work
-  PK_COUNT = 12
+  PK_CONDITIONAL = 12,      // tensor-core GEMMs queued under a SkipScope: whether they run is decided on the device, so
+                            // neither their flops nor their time is attributed to the GEMM kinds
+  PK_COUNT = 13
 };
 void count_launch(int n = 1);
 // sp_set_reproducible: when on, every floating-point sum of the library is taken in an order fixed by the call's
@@ -267,6 +269,9 @@ struct UpdateArgs {
   double* partial;   // [blocks * 4] block partial sums: res_act, z_sq, a_sq, |z_new - z1|^2
   double* absA_part; // [row_blocks, n] partial column sums of |A|
   int32_t row_blocks;
+  // At_out with its rows in "kept channels first" order: kept channel c goes to row (number of kept channels before
+  // c), pruned channel c to row k + (number of pruned channels before c).
+  int32_t at_kept_first = 0;
 };
 // grp_base / grp_mask of a u8 mask over n channels (see sp_elementwise.cu)
 cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream);
@@ -290,8 +295,9 @@ constexpr int kSumsqBlocks = 592;
 cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t cols, double scale, double* out,
                              bool accumulate, double* scratch, cudaStream_t stream);
 // reused (device, may be null): non-zero when the recovery on the kept support reused the unrestricted factor
+// scaled (device, may be null): non-zero when the pruned parts of G_A and R2 were obtained by scaling
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
-                        const int32_t* reused, cudaStream_t stream);
+                        const int32_t* reused, const int32_t* scaled, cudaStream_t stream);
 // relu + storage conversion for the init pass: A = phi(Z) -> storage dtype, and |A| column partials
 // gate_io (gated modules): holds the gate pre-activation on entry and SiLU of it on return; A = gate * Z then
 cudaError_t launch_init_act(const float* Z, float* gate_io, void* A_out, void* Zb_out, int32_t out_dtype, int64_t T,
@@ -353,6 +359,16 @@ cudaError_t global_select(const float* scores, int64_t ld_scores, int64_t n, int
                           uint8_t* mask, int64_t ld_mask, float* tau, int64_t* counts_out, void* scratch,
                           cudaStream_t stream);
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream);
+// C[i, j] *= f^power for the rows x cols block at C (ld); f is read from the device (a float stored in an int32 slot)
+cudaError_t scale_block(float* C, int64_t ld, int64_t rows, int64_t cols, const int32_t* f_bits, int power,
+                        cudaStream_t stream);
+// G[perm[i], perm[j]] = G[perm[j], perm[i]] = Gp[i, j] for i >= j (Gp: lower triangle in permuted order)
+cudaError_t unpermute_gram(const float* Gp, const int32_t* perm, int64_t n, float* G, cudaStream_t stream);
+// R[r, perm[j]] = Rp[r, j]
+cudaError_t unpermute_cols(const float* Rp, const int32_t* perm, int64_t rows, int64_t n, float* R,
+                           cudaStream_t stream);
+// tag[1] = k when `valid`, else -1; tag[2] = bits of the float c
+cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, cudaStream_t stream);
 // perm[0..n) = the kept channels of `mask` in ascending order followed by the pruned ones; count[0] = kept channels
 cudaError_t mask_to_perm(const uint8_t* mask, int64_t n, int32_t* perm, int32_t* count, cudaStream_t stream);
 // flags[0] = 1 when the kept channels of `mask` are not exactly perm[0..k) with count_old[0] == k; flags[1] = 1 - flags[0]

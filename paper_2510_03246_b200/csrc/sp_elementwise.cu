@@ -538,7 +538,17 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
         for (int e = lane; e < nch * (kAtRows / 8); e += 32) {
           const int ch = e / (kAtRows / 8), piece = e % (kAtRows / 8);
           const __nv_bfloat16* src = &at_tile[(wch0 + ch) * kAtPitch + piece * 8];
-          __nv_bfloat16* dst = At + (cb + ch) * g.ldt + rt + piece * 8;
+          int64_t row = cb + ch;
+          if (g.at_kept_first) {
+            // row of channel c in "kept first" order, from the group map of its 8 channels
+            const int64_t c = cb + ch;
+            const unsigned m8 = g.grp_mask[c >> 3];
+            const int qb = (int)(c & 7);
+            const int64_t kept_before = g.grp_base[c >> 3] + __popc(m8 & ((1u << qb) - 1u));
+            const bool is_kept = (m8 >> qb) & 1u;
+            row = is_kept ? kept_before : g.k + (c - kept_before);
+          }
+          __nv_bfloat16* dst = At + row * g.ldt + rt + piece * 8;
           if (piece * 8 + 8 <= rows_here) {
             const uint2 lo = *reinterpret_cast<const uint2*>(src), hi = *reinterpret_cast<const uint2*>(src + 4);
             *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
@@ -716,7 +726,7 @@ __global__ void sumsq_finish_kernel(const double* part, int nblocks, double scal
 }
 
 __global__ void init_report_kernel(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
-                                   const int32_t* reused) {
+                                   const int32_t* reused, const int32_t* scaled) {
   rep->res_act = 0.0;
   rep->res_out = nan("");
   rep->res_in = 0.0;
@@ -726,6 +736,7 @@ __global__ void init_report_kernel(sp_step_report* rep, const double* rho1, cons
   rep->rho2_eff = rho2 ? rho2[0] : 0.0;
   rep->kept = kept;
   rep->factor_reused = (reused != nullptr && reused[0] != 0) ? 1.0 : 0.0;
+  rep->pruned_scaled = (scaled != nullptr && scaled[0] != 0) ? 1.0 : 0.0;
 }
 
 // per-column sum |x| and sum x^2 of a [T, C] chunk: grid (col blocks of 256, row blocks) -> scratch, then reduced
@@ -1004,10 +1015,10 @@ cudaError_t sumsq_accumulate(const float* x, int64_t ld, int64_t rows, int64_t c
 }
 
 cudaError_t init_report(sp_step_report* rep, const double* rho1, const double* rho2, double kept,
-                        const int32_t* reused, cudaStream_t stream) {
+                        const int32_t* reused, const int32_t* scaled, cudaStream_t stream) {
   ProfScope prof(PK_ELEMENTWISE, 0.0, 0.0, stream);
   count_launch();
-  init_report_kernel<<<1, 1, 0, stream>>>(rep, rho1, rho2, kept, reused);
+  init_report_kernel<<<1, 1, 0, stream>>>(rep, rho1, rho2, kept, reused, scaled);
   return cudaGetLastError();
 }
 

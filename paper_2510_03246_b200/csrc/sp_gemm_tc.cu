@@ -854,7 +854,9 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   // fp32 C that a tensor map can describe leaves through TMA: a store when nothing is added, an add-reduction when
   // the call accumulates into C itself (each element of C is touched once per launch, so the result is the same sum)
   p.epi_mode = EPI_DIRECT;
-  bool c_tma = C.dtype == SP_F32 && C.ld % 4 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0;
+  // (a bulk tensor store moves whole 16-byte pieces: with N % 4 != 0 the last piece of a row would reach past
+  // column N and overwrite up to three floats that belong to the caller)
+  bool c_tma = C.dtype == SP_F32 && C.ld % 4 == 0 && N % 4 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0;
   if (batched && ((batch->nb0 > 1 && batch->c_s0 % 4 != 0) || (batch->nb1 > 1 && batch->c_s1 % 4 != 0))) c_tma = false;
   if (c_tma && beta == 0.f) p.epi_mode = EPI_TMA_STORE;
   if (c_tma && beta == 1.f && Cin.ptr == C.ptr && Cin.dtype == SP_F32 && Cin.s0 == C.ld &&
@@ -871,7 +873,7 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
   }
   // bf16 C = beta * Cin + alpha * acc with a bf16 Cin: both through TMA
   if (p.epi_mode == EPI_DIRECT && !batched && p.c_lo_off == 0 && beta != 0.f && C.dtype == SP_BF16 && Cin.dtype == SP_BF16 &&
-      C.ld % 8 == 0 &&
+      C.ld % 8 == 0 && N % 8 == 0 &&
       Cin.s0 % 8 == 0 && (reinterpret_cast<uintptr_t>(C.ptr) & 15u) == 0 &&
       (reinterpret_cast<uintptr_t>(Cin.ptr) & 15u) == 0) {
     if (!make_map(&tmC, false, C.ptr, N, M, C.ld, 32, 32, true) ||
@@ -958,9 +960,12 @@ sp_status gemm_tc(int64_t M, int64_t N, int64_t K, float alpha, TcOperand A, TcO
       }) != cudaSuccess)
     return SP_ERR_CUDA;
   count_launch();
+  // lower-only: the triangle of the leading N x N square and all of the M - N rows below it
   const double flops = alg_flops >= 0.0 ? alg_flops
-                                        : (lower_only ? 1.0 : 2.0) * (double)M * (double)N * (double)K * p.nb0 * p.nb1;
-  ProfScope prof(max_pairs > 0 ? PK_GEMM_TC_SHARED : PK_GEMM_TC, flops, 0.0, stream);
+                       : lower_only     ? (double)K * (double)N * (2.0 * (double)M - (double)N)
+                                        : 2.0 * (double)M * (double)N * (double)K * p.nb0 * p.nb1;
+  ProfScope prof(p.skip != nullptr ? PK_CONDITIONAL : max_pairs > 0 ? PK_GEMM_TC_SHARED : PK_GEMM_TC,
+                 p.skip != nullptr ? 0.0 : flops, 0.0, stream);
   const int pairs = p.num_units < pairs_max ? p.num_units : pairs_max;
   if (batched) gemm_tc_kernel<true><<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);
   else gemm_tc_kernel<false><<<2 * pairs, NUM_THREADS, SMEM_BYTES, stream>>>(tmA, tmB, tmC, tmCin, p);

@@ -2,6 +2,7 @@
 // Lemma 2 / Algorithm 1 Step 2, the exact top-k selection by radix select, and M (.) W.
 #include <math.h>
 
+#include <algorithm>
 #include <mutex>
 
 #include "sp_common.cuh"
@@ -843,7 +844,9 @@ __global__ void __launch_bounds__(1024) mask_changed_kernel(const uint8_t* mask,
   if (threadIdx.x == 0) s_bad = (int64_t)count_old[0] != k;
   __syncthreads();
   int bad = 0;
-  for (int64_t a = threadIdx.x; a < k; a += blockDim.x) bad |= mask[perm[a]] == 0;
+  if (!s_bad)      // (with another count the list may not be one of this mask's size at all: it is not read)
+    for (int64_t a = threadIdx.x; a < k; a += blockDim.x) bad |= mask[perm[a]] == 0;
+  __syncthreads();
   if (bad) s_bad = 1;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -1330,6 +1333,73 @@ cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cud
   if (n == 0) return cudaSuccess;
   count_launch();
   mask_to_index_kernel<<<1, 1024, 0, stream>>>(mask, n, kept_idx);
+  return cudaGetLastError();
+}
+
+__global__ void scale_block_kernel(float* C, int64_t ld, int64_t rows, int64_t cols, const int32_t* f_bits, int power,
+                                   const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;   // conditional launch (see SkipScope)
+  const float f = __int_as_float(f_bits[0]);
+  const float s = power == 2 ? f * f : f;
+  const int64_t total = rows * cols;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x)
+    C[(e / cols) * ld + (e % cols)] *= s;
+}
+
+__global__ void unpermute_gram_kernel(const float* __restrict__ Gp, const int32_t* __restrict__ perm, int64_t n,
+                                      float* __restrict__ G) {
+  const int64_t total = n * n;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / n, j = e % n;
+    // entry (i, j) of the permuted matrix from its lower triangle
+    const float v = i >= j ? Gp[i * n + j] : Gp[j * n + i];
+    G[(int64_t)perm[i] * n + perm[j]] = v;
+  }
+}
+
+__global__ void unpermute_cols_kernel(const float* __restrict__ Rp, const int32_t* __restrict__ perm, int64_t rows,
+                                      int64_t n, float* __restrict__ R) {
+  const int64_t total = rows * n;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = e / n, j = e % n;
+    R[r * n + perm[j]] = Rp[e];
+  }
+}
+
+__global__ void decay_tag_set_kernel(int32_t* tag, int k, float c, int valid) {
+  tag[1] = valid ? k : -1;
+  tag[2] = __float_as_int(c);
+}
+
+cudaError_t scale_block(float* C, int64_t ld, int64_t rows, int64_t cols, const int32_t* f_bits, int power,
+                        cudaStream_t stream) {
+  if (rows * cols <= 0) return cudaSuccess;
+  count_launch();
+  scale_block_kernel<<<(unsigned)std::min<int64_t>(ceil_div(rows * cols, (int64_t)256), 148 * 16), 256, 0, stream>>>(
+      C, ld, rows, cols, f_bits, power, skip_flag());
+  return cudaGetLastError();
+}
+
+cudaError_t unpermute_gram(const float* Gp, const int32_t* perm, int64_t n, float* G, cudaStream_t stream) {
+  if (n <= 0) return cudaSuccess;
+  count_launch();
+  unpermute_gram_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n * n, (int64_t)256), 148 * 32), 256, 0, stream>>>(Gp, perm,
+                                                                                                               n, G);
+  return cudaGetLastError();
+}
+
+cudaError_t unpermute_cols(const float* Rp, const int32_t* perm, int64_t rows, int64_t n, float* R,
+                           cudaStream_t stream) {
+  if (rows * n <= 0) return cudaSuccess;
+  count_launch();
+  unpermute_cols_kernel<<<(unsigned)std::min<int64_t>(ceil_div(rows * n, (int64_t)256), 148 * 32), 256, 0, stream>>>(
+      Rp, perm, rows, n, R);
+  return cudaGetLastError();
+}
+
+cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, cudaStream_t stream) {
+  count_launch();
+  decay_tag_set_kernel<<<1, 1, 0, stream>>>(tag, (int)k, c, valid ? 1 : 0);
   return cudaGetLastError();
 }
 

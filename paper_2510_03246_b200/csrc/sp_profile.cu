@@ -84,7 +84,7 @@ int32_t sp_profile_kinds(void) { return sp::PK_COUNT; }
 const char* sp_profile_kind_name(int32_t kind) {
   static const char* names[sp::PK_COUNT] = {"gemm_tc", "gemm_simt", "solve_phase", "fused_update", "prep_h",
                                             "scores", "topk_select", "elementwise", "allocate", "chol_diag",
-                                            "panel_apply", "gemm_tc_shared"};
+                                            "panel_apply", "gemm_tc_shared", "conditional"};
   return (kind >= 0 && kind < sp::PK_COUNT) ? names[kind] : "unknown";
 }
 

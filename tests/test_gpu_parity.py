@@ -68,6 +68,30 @@ def test_gemm_tensor_core(a_kmajor, b_kmajor, M, N, K):
             assert np.all(np.abs(got - ref) <= 2e-6 * np.abs(ref).max() + bf16_half_ulp(ref) * 1.001)
 
 
+@pytest.mark.parametrize("N,out_dtype", [(262, torch.float32), (1434, torch.float32), (260, torch.bfloat16)])
+def test_gemm_tensor_core_pitched_output_keeps_what_lies_right_of_it(N, out_dtype):
+    """C is a block of columns inside a wider array whose width N is not a multiple of 16 bytes: the columns to the
+    right of the block belong to the caller and must come back untouched (bulk tensor stores move whole 16-byte
+    pieces, so such a C takes the plain epilogue), for a plain store and for an accumulating call."""
+    M, K, ld = 300, 200, 1440
+    A = _gauss((M, K), 31, torch.bfloat16).to(DEV)
+    B = _gauss((N, K), 32, torch.bfloat16).to(DEV)
+    status = api.new_status()
+    for beta in (0.0, 1.0):
+        wide = _gauss((M, ld), 33, out_dtype).to(DEV)
+        before = wide.clone()
+        Cm = wide[:, :N]
+        api.sp_gemm(A, B, Cm, transA=False, transB=True, alpha=1.0, beta=beta, use_tensor_cores=True, status=status)
+        torch.cuda.synchronize()
+        _assert_status_clean(status)
+        assert torch.equal(wide[:, N:], before[:, N:])
+        ref = np64(A) @ np64(B).T + beta * np64(before[:, :N])
+        if out_dtype == torch.float32:
+            assert relerr(np64(Cm), ref) < 2e-6
+        else:
+            assert np.all(np.abs(np64(Cm) - ref) <= 2e-6 * np.abs(ref).max() + bf16_half_ulp(ref) * 1.001)
+
+
 def test_gemm_tensor_core_lower_only_and_persistence():
     # square Gram-type product with more tiles than SMs, lower triangle only
     n, K = 2304, 520
@@ -638,6 +662,60 @@ def test_kept_support_recovery_reuses_the_factor(cfg, overlap):
     torch.cuda.synchronize()
     assert mod.read_report()["factor_reused"] == 0.0
     mod.check_status()
+
+
+@pytest.mark.parametrize("rule", ["paper", "exact"])
+def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule):
+    """bf16 storage, ReLU, no dual variable: from the second step with an unchanged mask on, a pruned channel's row of A
+    is c = beta / (alpha + beta) times its row of the step before (tests/test_oracle_pins.py pins that on the oracle),
+    and the library then obtains G_A[pruned, pruned] and R2[:, pruned] by scaling (report field pruned_scaled) instead
+    of contracting over the tokens.  Every step is compared with the oracle's full recomputation: steps that scale,
+    a step after a planted other mask (which must recompute), a step after alpha and beta changed (the factor is
+    the c of the step that wrote the values, not of the current one), and a module without the ordered accumulators."""
+    cfg = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=1300, sparsity=0.63, outlier_frac=0.02)   # k = 287
+    k = cfg.k_keep
+    assert k % 4 != 0            # the pruned block starts at a column that is not 16-byte aligned
+    mod, X, W1, W2 = _make_module(cfg, chunk=512)
+    mod.sp_ffn_init()
+    tol = TOL[X.dtype]
+    audit = []
+
+    def params(alpha, beta):
+        return (api.AdmmParams(alpha=alpha, beta=beta, rho=cfg.rho, k_keep=k, z_rule=_RULE[rule], token_chunk=512,
+                               compute_objective=False),
+                O.AdmmParams(alpha=alpha, beta=beta, rho=cfg.rho, k_keep=k, z_rule=rule))
+
+    seen = []
+    plan = [(1.0, 1.5, None), (1.0, 1.5, None), (1.0, 1.5, None), (0.7, 2.0, None), (0.7, 2.0, None)]
+    if rule == "paper":     # (an arbitrary other mask leaves the exact rule's audit more near ties than it accepts)
+        plan += [(0.7, 2.0, "rolled"), (0.7, 2.0, None)]
+    for alpha, beta, plant in plan:
+        p_gpu, p_or = params(alpha, beta)
+        if plant == "rolled":       # a given mask with other channels (no selection in this step)
+            mod.mask.copy_(torch.roll(mod.mask, 1))
+            p_gpu.reselect_mask = False
+            p_or.reselect_mask = False
+        order_before = mod.decay_tag[8:].cpu().numpy().copy()
+        k_before = int(mod.decay_tag[1].item())
+        _step_and_compare(mod, X, W1.float(), p_gpu, p_or, tol, audit)          # G_A, R2 (and the rest) against the oracle
+        mask = mod.mask.cpu().numpy()
+        same_order = k_before == k and np.array_equal(np.sort(order_before[:k]), np.flatnonzero(mask))
+        assert mod.read_report()["pruned_scaled"] == float(same_order)
+        # the ordered copies agree with the channel-order accumulators the step returns
+        perm = mod.decay_tag[8:].long()
+        assert torch.equal(torch.sort(perm[:k]).values, torch.nonzero(mod.mask).flatten())
+        Gp = torch.tril(mod.G_A_perm)
+        assert torch.equal(torch.tril(mod.G_A[perm][:, perm]), Gp)
+        assert torch.equal(mod.R2[:, perm], mod.R2_perm)
+        seen.append(same_order)
+    assert seen[0] is False and any(seen[1:5]) and (rule != "paper" or seen[5] is False)
+    # without the ordered accumulators nothing is scaled and the same checks hold
+    mod2 = api.FfnModule(X.to(DEV), W1.to(DEV), W2.to(DEV), token_chunk=512, pruned_decay=False)
+    mod2.sp_ffn_init()
+    p_gpu, p_or = params(1.0, 1.5)
+    for _ in range(3):
+        _step_and_compare(mod2, X, W1.float(), p_gpu, p_or, tol, audit)
+        assert mod2.read_report()["pruned_scaled"] == 0.0
 
 
 def test_captured_step_takes_either_branch_on_replay():
