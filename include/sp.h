@@ -129,6 +129,14 @@ typedef struct {
   float* G_A_perm;     /* [n, n]                                                                                     */
   float* R2_perm;      /* [d, n]                                                                                     */
   int32_t* decay_tag;  /* int32 [n + 8]                                                                              */
+  /* Optional on top of the three above (both or none): R1 in the same way — Z of a pruned channel is c times its old
+   * value too, so R1[pruned, :] is scaled, and only the kept rows are contracted.  For that a pass over the new Z of
+   * every chunk writes its bf16 copy transposed with the kept channels first (instead of the row-major copy the fused
+   * update would write), and in the same pass h = max(Z_new, 0) of the kept channels into H_next: the a-update of the
+   * NEXT step starts from it and skips its own gather pass over Z while the mask stays. */
+  float* R1_perm;      /* [n, d]                                                                                     */
+  void* H_next;        /* [N, H_next_ld] bf16                                                                        */
+  int64_t H_next_ld;   /* a multiple of 8, at least ceil8(k_keep); smaller: R1_perm / H_next are not used             */
 } sp_ffn_state;
 
 typedef struct {

@@ -51,14 +51,16 @@ def gemm_cases(reps, warm):
         # (K-major here) with the kept channels first, and only the kept columns are contracted anew
         ("G_A[:, kept] += A^T A_kept (lower)", N, N // 2, T, True, True, f32, 1.0, True),
         ("R2[:, kept] += Ypre^T A_kept", D, N // 2, T, False, True, f32, 1.0, False),
-        ("R1 += Z^T X", N, D, T, False, False, f32, 1.0, False),
+        ("R1[kept, :] += Z_kept^T X (Z^T K-major)", N // 2, D, T, True, False, f32, 1.0, False),
         ("solve update (K = 6 x 128)", 2048, 4096, 768, True, True, f32, 1.0, False),
         # the pruned parts, contracted only in a step whose mask changed
         ("G_A[pruned, pruned] (lower)", N // 2, N // 2, T, True, True, f32, 1.0, True),
         ("R2[:, pruned]", D, N // 2, T, False, True, f32, 1.0, False),
+        ("R1[pruned, :]", N // 2, D, T, True, False, f32, 1.0, False),
         # the full products of a module without the ordered accumulators
         ("G_A += A^T A (lower, A K-major)", N, N, T, True, True, f32, 1.0, True),
         ("R2 += Ypre^T A (A K-major)", D, N, T, False, True, f32, 1.0, False),
+        ("R1 += Z^T X (row-major copy of Z)", N, D, T, False, False, f32, 1.0, False),
         # other operand layouts: row-major A (fp32-storage path, or when the objective is reported), and transposed
         # copies of Ypre / X that the module does not keep
         ("G_A with A row-major", N, N, T, False, False, f32, 1.0, True),

@@ -55,7 +55,8 @@ class SpFfnState(C.Structure):
     _fields_ = [("Z", C.c_void_p), ("U", C.c_void_p), ("G_X", C.c_void_p), ("G_A", C.c_void_p), ("R1", C.c_void_p),
                 ("R2", C.c_void_p), ("absA", C.c_void_p), ("W1", C.c_void_p), ("W2", C.c_void_p),
                 ("scores", C.c_void_p), ("mask", C.c_void_p), ("importance", C.c_void_p), ("Gate", C.c_void_p),
-                ("G_X_inv", C.c_void_p), ("G_A_perm", C.c_void_p), ("R2_perm", C.c_void_p), ("decay_tag", C.c_void_p)]
+                ("G_X_inv", C.c_void_p), ("G_A_perm", C.c_void_p), ("R2_perm", C.c_void_p), ("decay_tag", C.c_void_p),
+                ("R1_perm", C.c_void_p), ("H_next", C.c_void_p), ("H_next_ld", C.c_int64)]
 
 
 class SpAdmmParams(C.Structure):
@@ -515,11 +516,14 @@ class FfnModule:
         self.overlap_k = int(overlap_k)
         # ordered accumulators that let a step scale, instead of recompute, the parts of G_A and R2 that belong to
         # pruned channels while the mask stays (see sp_ffn_state.G_A_perm); ReLU modules without the dual variable
-        self.G_A_perm = self.R2_perm = self.decay_tag = None
+        self.G_A_perm = self.R2_perm = self.decay_tag = self.R1_perm = self.H_next = None
         if pruned_decay and X.dtype == torch.bfloat16 and Wg_0 is None and not dual_mode and n % 4 == 0:
             self.G_A_perm = torch.empty(n, n, **f32)
             self.R2_perm = torch.empty(d, n, **f32)
             self.decay_tag = torch.full((n + 8,), -1, dtype=torch.int32, device=dev)
+            if overlap_k > 0:        # sized for that many kept units, like the other optional buffers
+                self.R1_perm = torch.empty(n, d, **f32)
+                self.H_next = torch.empty(N, (int(overlap_k) + 7) // 8 * 8, dtype=torch.bfloat16, device=dev)
         self._pool = ws_pool if ws_pool is not None else {}
         self.iteration = 0
 
@@ -540,7 +544,8 @@ class FfnModule:
                           self.R1.data_ptr(), self.R2.data_ptr(), self.absA.data_ptr(), self.W1.data_ptr(),
                           self.W2.data_ptr(), self.scores.data_ptr(), self.mask.data_ptr(),
                           self.importance.data_ptr(), _ptr(self.Gate), _ptr(self.G_X_inv), _ptr(self.G_A_perm),
-                          _ptr(self.R2_perm), _ptr(self.decay_tag))
+                          _ptr(self.R2_perm), _ptr(self.decay_tag), _ptr(self.R1_perm), _ptr(self.H_next),
+                          self.H_next.shape[1] if self.H_next is not None else 0)
 
     def _workspace(self, chunk: int) -> torch.Tensor:
         need = max(workspace_bytes(SP_WS_ADMM_STEP, self.d, self.n, self.N, chunk, _dt(self.X)),

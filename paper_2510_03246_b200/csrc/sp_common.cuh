@@ -283,6 +283,11 @@ cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, voi
                           int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream,
                           int64_t lo_off = 0);
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
+// From the new Z of a chunk (n % 4 == 0): Zt [n, ldt] bf16 = Z^T with the kept channels' rows first (the order of the
+// transposed A), and Hn [T, ldh] bf16 = max(Z, 0) on the kept channels, compact (h of the next step; ReLU, no dual).
+cudaError_t launch_gather_next(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
+                               const uint8_t* grp_mask, void* Zt, int64_t ldt, void* Hn, int64_t ldh,
+                               cudaStream_t stream);
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]
 cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
@@ -367,8 +372,14 @@ cudaError_t unpermute_gram(const float* Gp, const int32_t* perm, int64_t n, floa
 // R[r, perm[j]] = Rp[r, j]
 cudaError_t unpermute_cols(const float* Rp, const int32_t* perm, int64_t rows, int64_t n, float* R,
                            cudaStream_t stream);
-// tag[1] = k when `valid`, else -1; tag[2] = bits of the float c
-cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, cudaStream_t stream);
+// tag[1] = k when `valid`, else -1; tag[2] = bits of the float c; tag[4] = row pitch of the h written for the next
+// step (0: none was written)
+cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, int64_t h_ld, cudaStream_t stream);
+// ready[0] = 1 when same[0] != 0 and the tag says that h was written with row pitch h_ld, else 0; ready[1] = 1 - ready[0]
+cudaError_t h_next_ready(const int32_t* same, const int32_t* tag, int64_t h_ld, int32_t* ready, cudaStream_t stream);
+// R[perm[i], :] = Rp[i, :]
+cudaError_t unpermute_rows(const float* Rp, const int32_t* perm, int64_t n, int64_t cols, float* R,
+                           cudaStream_t stream);
 // perm[0..n) = the kept channels of `mask` in ascending order followed by the pruned ones; count[0] = kept channels
 cudaError_t mask_to_perm(const uint8_t* mask, int64_t n, int32_t* perm, int32_t* count, cudaStream_t stream);
 // flags[0] = 1 when the kept channels of `mask` are not exactly perm[0..k) with count_old[0] == k; flags[1] = 1 - flags[0]

@@ -383,6 +383,7 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
   // writes them out as 64-byte pieces; lanes beyond the last channel walk the loop too (without touching memory),
   // so that the warp-level barriers see all lanes.
   extern __shared__ __align__(16) __nv_bfloat16 at_tile[];     // [1024][kAtPitch], only with At_out
+  __shared__ int32_t at_row[1024];                             // row of each channel of the block in "kept first" order
   const bool active = c0 < g.n;
   {
     const int cnt = !active ? 0 : (g.n - c0 >= 4) ? 4 : (int)(g.n - c0);
@@ -400,6 +401,16 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
         off[q] = pos;
         pos += (bits >> q) & 1u;
       }
+    }
+    if (g.at_kept_first) {
+      // looked up once: kept channel -> its compact position, pruned channel -> k + its rank among the pruned ones
+      // (only the warp that owns the channels reads them back: a warp-level barrier below is enough)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int kb = base + off[q];
+        at_row[4 * (int)threadIdx.x + q] = ((bits >> q) & 1u) ? kb : (int32_t)(g.k + (c0 + q - kb));
+      }
+      __syncwarp();
     }
     auto load_row = [&](int64_t r, UpdRow<HAS_U>& w) {
       const int64_t e = r * g.n + c0;
@@ -538,16 +549,7 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
         for (int e = lane; e < nch * (kAtRows / 8); e += 32) {
           const int ch = e / (kAtRows / 8), piece = e % (kAtRows / 8);
           const __nv_bfloat16* src = &at_tile[(wch0 + ch) * kAtPitch + piece * 8];
-          int64_t row = cb + ch;
-          if (g.at_kept_first) {
-            // row of channel c in "kept first" order, from the group map of its 8 channels
-            const int64_t c = cb + ch;
-            const unsigned m8 = g.grp_mask[c >> 3];
-            const int qb = (int)(c & 7);
-            const int64_t kept_before = g.grp_base[c >> 3] + __popc(m8 & ((1u << qb) - 1u));
-            const bool is_kept = (m8 >> qb) & 1u;
-            row = is_kept ? kept_before : g.k + (c - kept_before);
-          }
+          const int64_t row = g.at_kept_first ? (int64_t)at_row[(wch0 + ch)] : cb + ch;
           __nv_bfloat16* dst = At + row * g.ldt + rt + piece * 8;
           if (piece * 8 + 8 <= rows_here) {
             const uint2 lo = *reinterpret_cast<const uint2*>(src), hi = *reinterpret_cast<const uint2*>(src + 4);
@@ -576,6 +578,115 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
     g.partial[bid * 4 + 1] = r1;
     g.partial[bid * 4 + 2] = r2;
     g.partial[bid * 4 + 3] = r3;
+  }
+}
+
+// After the fused update of a chunk (bf16 storage, ReLU, no dual variable), from the NEW Z of the chunk:
+//   Zt[row(c), t] = bf16(Z[t, c]) for every channel c, rows in "kept channels first" order as in the transposed A
+//                   (the K-major operand of R1 = Z^T X, whose pruned rows are only contracted when the mask changed);
+//   Hn[t, p(c)]   = bf16(max(Z[t, c], 0)) for the kept channels at their compact positions: h of the NEXT step's
+//                   a-update, which then needs no gather pass over Z of its own.
+// Same decomposition as the fused update: a thread owns 4 consecutive channels, a warp stages kAtRows rows of its 128
+// channels in shared memory and writes them out as 64-byte pieces.
+__global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __restrict__ Z, int64_t T, int64_t n, int64_t k,
+                                                             const int32_t* __restrict__ grp_base,
+                                                             const uint8_t* __restrict__ grp_mask,
+                                                             __nv_bfloat16* __restrict__ Zt, int64_t ldt,
+                                                             __nv_bfloat16* __restrict__ Hn, int64_t ldh,
+                                                             int32_t row_blocks) {
+  extern __shared__ __align__(16) __nv_bfloat16 zt_tile[];     // [1024][kAtPitch]
+  __shared__ uint8_t kept_ch[8][128];                          // per warp: its kept channels (0..127), ascending
+  __shared__ int32_t row_of[8][128];                           // per warp: row of each of its channels in Zt
+  const int64_t grp4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int64_t c0 = grp4 * 4;
+  int64_t rows_per = ceil_div(T, (int64_t)row_blocks);
+  rows_per = (rows_per + kAtRows - 1) / kAtRows * kAtRows;
+  const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
+  const int64_t r_end = (r_begin + rows_per < T) ? r_begin + rows_per : T;
+  const bool active = c0 < n;                                   // n % 4 == 0: a thread's channels exist together
+  const int lane = (int)threadIdx.x & 31, warp = (int)threadIdx.x >> 5;
+  const unsigned bits8 = active ? grp_mask[grp4 >> 1] : 0u;
+  const bool upper = (grp4 & 1) != 0;
+  const unsigned bits = upper ? (bits8 >> 4) : (bits8 & 0xFu);
+  const int base = active ? grp_base[grp4 >> 1] + (upper ? __popc(bits8 & 0xFu) : 0) : 0;
+  // the warp's kept channels: a contiguous run of compact positions [base_w, base_w + cnt_w)
+  int before = __popc(bits);
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int u = __shfl_up_sync(0xffffffffu, before, o);
+    if (lane >= o) before += u;
+  }
+  const int cnt_w = __shfl_sync(0xffffffffu, before, 31);
+  before -= __popc(bits);
+  const int base_w = __shfl_sync(0xffffffffu, base, 0);
+  {
+    int pos = before, kb = base;       // kb: kept channels before channel c0 + q
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const bool is_kept = (bits >> q) & 1u;
+      if (is_kept) kept_ch[warp][pos++] = (uint8_t)(4 * lane + q);
+      // row of the channel in "kept first" order (looked up once, not per piece of the write-out loop)
+      row_of[warp][4 * lane + q] = is_kept ? kb : (int32_t)(k + (c0 + q - kb));
+      kb += is_kept ? 1 : 0;
+    }
+  }
+  __syncwarp();
+  const int ct = 4 * (int)threadIdx.x;
+  const int wch0 = warp * 128;
+  const int64_t cb = (int64_t)blockIdx.x * 1024 + wch0;
+  const int nch = (n - cb < 128) ? (int)((n - cb > 0) ? n - cb : 0) : 128;
+  for (int64_t rt = r_begin; rt < r_end; rt += kAtRows) {
+    const int64_t rt_end = (rt + kAtRows < r_end) ? rt + kAtRows : r_end;
+    if (active) {
+      for (int64_t r = rt; r < rt_end; r += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          v[i] = (r + i < rt_end) ? *reinterpret_cast<const float4*>(Z + (r + i) * n + c0) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          __align__(16) __nv_bfloat16 col[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float z = q == 0 ? v[i].x : q == 1 ? v[i].y : q == 2 ? v[i].z : v[i].w;
+            col[i] = __float2bfloat16_rn(z);
+          }
+          // (kAtPitch = 36 elements: a row of the tile starts 8-byte aligned, so two 8-byte stores)
+          uint2* dst = reinterpret_cast<uint2*>(&zt_tile[(ct + q) * kAtPitch + (int)(r - rt)]);
+          dst[0] = *reinterpret_cast<const uint2*>(col);
+          dst[1] = *reinterpret_cast<const uint2*>(col + 4);
+        }
+      }
+    }
+    __syncwarp();
+    const int rows_here = (int)(rt_end - rt);
+    // Z^T: rows rt .. rt_end - 1 of every channel of the warp as pieces of 8 rows, in "kept first" row order
+    for (int e = lane; e < nch * (kAtRows / 8); e += 32) {
+      const int ch = e / (kAtRows / 8), piece = e % (kAtRows / 8);
+      const __nv_bfloat16* src = &zt_tile[(wch0 + ch) * kAtPitch + piece * 8];
+      __nv_bfloat16* dst = Zt + (int64_t)row_of[warp][ch] * ldt + rt + piece * 8;
+      if (piece * 8 + 8 <= rows_here) {
+        const uint2 lo = *reinterpret_cast<const uint2*>(src), hi = *reinterpret_cast<const uint2*>(src + 4);
+        *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
+      } else {
+        for (int q = 0; q < 8; ++q)
+          if (piece * 8 + q < rows_here) dst[q] = src[q];
+      }
+    }
+    // h of the next step: per row the warp's kept channels are one contiguous run of H; consecutive lanes write
+    // consecutive elements (max(bf16(z), 0) = bf16(max(z, 0)): rounding keeps the sign)
+    for (int e = lane; e < cnt_w; e += 32) {
+      // the 32 rows of this kept channel: 64 contiguous bytes of the tile (8-byte aligned rows)
+      __align__(8) __nv_bfloat16 zr[kAtRows];
+      const uint2* src = reinterpret_cast<const uint2*>(&zt_tile[(wch0 + kept_ch[warp][e]) * kAtPitch]);
+#pragma unroll
+      for (int i = 0; i < kAtRows / 4; ++i) reinterpret_cast<uint2*>(zr)[i] = src[i];
+      __nv_bfloat16* hcol = Hn + rt * ldh + base_w + e;
+#pragma unroll
+      for (int rr = 0; rr < kAtRows; ++rr)
+        if (rr < rows_here) hcol[(int64_t)rr * ldh] = __hgt(zr[rr], __float2bfloat16_rn(0.f)) ? zr[rr] : __float2bfloat16_rn(0.f);
+    }
+    __syncwarp();
   }
 }
 
@@ -973,6 +1084,26 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
   }
   fn<<<grid, 256, smem, stream>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_next(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
+                               const uint8_t* grp_mask, void* Zt, int64_t ldt, void* Hn, int64_t ldh,
+                               cudaStream_t stream) {
+  if (T * n == 0) return cudaSuccess;
+  if (n % 4 != 0 || ldt % 8 != 0) return cudaErrorInvalidValue;
+  int row_blocks = 1;
+  fused_update_grid(T, n, &row_blocks);
+  dim3 grid((unsigned)ceil_div(n, (int64_t)1024), (unsigned)row_blocks);
+  // Z read once; its bf16 copy written transposed, the kept part once more as next step's h
+  ProfScope prof(PK_PREP_H, 0.0, (double)T * ((double)n * 6.0 + (double)k * 2.0), stream);
+  count_launch();
+  cudaError_t e = cudaFuncSetAttribute(gather_next_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kAtTileBytes);
+  if (e != cudaSuccess) return e;
+  gather_next_kernel<<<grid, 256, kAtTileBytes, stream>>>(Z, T, n, k, grp_base, grp_mask,
+                                                         reinterpret_cast<__nv_bfloat16*>(Zt), ldt,
+                                                         reinterpret_cast<__nv_bfloat16*>(Hn), ldh, row_blocks);
   return cudaGetLastError();
 }
 

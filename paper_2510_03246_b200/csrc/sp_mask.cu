@@ -1366,9 +1366,24 @@ __global__ void unpermute_cols_kernel(const float* __restrict__ Rp, const int32_
   }
 }
 
-__global__ void decay_tag_set_kernel(int32_t* tag, int k, float c, int valid) {
+__global__ void decay_tag_set_kernel(int32_t* tag, int k, float c, int valid, int h_ld) {
   tag[1] = valid ? k : -1;
   tag[2] = __float_as_int(c);
+  tag[4] = valid ? h_ld : 0;
+}
+
+__global__ void h_next_ready_kernel(const int32_t* same, const int32_t* tag, int h_ld, int32_t* ready) {
+  ready[0] = (same[0] != 0 && tag[4] == h_ld && h_ld > 0) ? 1 : 0;
+  ready[1] = 1 - ready[0];
+}
+
+__global__ void unpermute_rows_kernel(const float* __restrict__ Rp, const int32_t* __restrict__ perm, int64_t n,
+                                      int64_t cols, float* __restrict__ R) {
+  const int64_t total = n * cols;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = e / cols, j = e % cols;
+    R[(int64_t)perm[i] * cols + j] = Rp[e];
+  }
 }
 
 cudaError_t scale_block(float* C, int64_t ld, int64_t rows, int64_t cols, const int32_t* f_bits, int power,
@@ -1397,9 +1412,24 @@ cudaError_t unpermute_cols(const float* Rp, const int32_t* perm, int64_t rows, i
   return cudaGetLastError();
 }
 
-cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, cudaStream_t stream) {
+cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, int64_t h_ld, cudaStream_t stream) {
   count_launch();
-  decay_tag_set_kernel<<<1, 1, 0, stream>>>(tag, (int)k, c, valid ? 1 : 0);
+  decay_tag_set_kernel<<<1, 1, 0, stream>>>(tag, (int)k, c, valid ? 1 : 0, (int)h_ld);
+  return cudaGetLastError();
+}
+
+cudaError_t h_next_ready(const int32_t* same, const int32_t* tag, int64_t h_ld, int32_t* ready, cudaStream_t stream) {
+  count_launch();
+  h_next_ready_kernel<<<1, 1, 0, stream>>>(same, tag, (int)h_ld, ready);
+  return cudaGetLastError();
+}
+
+cudaError_t unpermute_rows(const float* Rp, const int32_t* perm, int64_t n, int64_t cols, float* R,
+                           cudaStream_t stream) {
+  if (n * cols <= 0) return cudaSuccess;
+  count_launch();
+  unpermute_rows_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n * cols, (int64_t)256), 148 * 32), 256, 0, stream>>>(
+      Rp, perm, n, cols, R);
   return cudaGetLastError();
 }
 

@@ -664,18 +664,21 @@ def test_kept_support_recovery_reuses_the_factor(cfg, overlap):
     mod.check_status()
 
 
-@pytest.mark.parametrize("rule", ["paper", "exact"])
-def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule):
+@pytest.mark.parametrize("rule,with_r1", [("paper", False), ("exact", False), ("paper", True), ("exact", True)])
+def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, with_r1):
     """bf16 storage, ReLU, no dual variable: from the second step with an unchanged mask on, a pruned channel's row of A
     is c = beta / (alpha + beta) times its row of the step before (tests/test_oracle_pins.py pins that on the oracle),
     and the library then obtains G_A[pruned, pruned] and R2[:, pruned] by scaling (report field pruned_scaled) instead
     of contracting over the tokens.  Every step is compared with the oracle's full recomputation: steps that scale,
     a step after a planted other mask (which must recompute), a step after alpha and beta changed (the factor is
-    the c of the step that wrote the values, not of the current one), and a module without the ordered accumulators."""
+    the c of the step that wrote the values, not of the current one), and a module without the ordered accumulators.
+    with_r1: the module also holds R1_perm / H_next, so R1[pruned, :] is scaled too, the bf16 copy of the new Z is
+    written transposed by a pass of its own, and the next step takes its h from H_next instead of gathering it."""
     cfg = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=1300, sparsity=0.63, outlier_frac=0.02)   # k = 287
     k = cfg.k_keep
     assert k % 4 != 0            # the pruned block starts at a column that is not 16-byte aligned
-    mod, X, W1, W2 = _make_module(cfg, chunk=512)
+    mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=k if with_r1 else 0)
+    assert (mod.R1_perm is not None) == with_r1
     mod.sp_ffn_init()
     tol = TOL[X.dtype]
     audit = []
@@ -707,6 +710,11 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule):
         Gp = torch.tril(mod.G_A_perm)
         assert torch.equal(torch.tril(mod.G_A[perm][:, perm]), Gp)
         assert torch.equal(mod.R2[:, perm], mod.R2_perm)
+        if with_r1:
+            assert torch.equal(mod.R1[perm], mod.R1_perm)
+            # what the pass over the new Z left for the next step: max(Z, 0) on the kept channels, compact
+            kept = torch.nonzero(mod.mask).flatten()
+            assert torch.equal(mod.H_next[:, :k], torch.clamp(mod.Z[:, kept], min=0).to(torch.bfloat16))
         seen.append(same_order)
     assert seen[0] is False and any(seen[1:5]) and (rule != "paper" or seen[5] is False)
     # without the ordered accumulators nothing is scaled and the same checks hold
