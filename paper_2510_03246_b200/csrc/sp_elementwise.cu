@@ -263,7 +263,9 @@ __global__ void __launch_bounds__(256) prep_h_kernel(const float* __restrict__ Z
                                                      const float* __restrict__ G, void* __restrict__ H, int32_t hdt,
                                                      int64_t T, int64_t n,
                                                      int64_t ldh, int64_t ncols, int64_t lo_off, int64_t k,
-                                                     const int32_t* __restrict__ idx, int32_t rows_per_block) {
+                                                     const int32_t* __restrict__ idx, int32_t rows_per_block,
+                                                     const int32_t* skip) {
+  if (skip != nullptr && *skip != 0) return;   // conditional launch (see SkipScope)
   const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (p0 >= ncols) return;
   int ch[8];
@@ -1036,8 +1038,10 @@ cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, voi
   if (T * ldh == 0) return cudaSuccess;
   if (lo_off > 0 && (hdt != SP_BF16 || lo_off % 8 != 0 || 2 * lo_off > ldh)) return cudaErrorInvalidValue;
   const int64_t ncols = lo_off > 0 ? lo_off : ldh;
-  // algorithmic bytes: Z (and U) read once, the kept part written once (twice when it is split)
+  // algorithmic bytes: Z (and U) read once, the kept part written once (twice when it is split); a conditional
+  // launch (SkipScope) is not counted: whether it moves anything is decided on the device
   ProfScope prof(PK_PREP_H, 0.0,
+                 skip_flag() != nullptr ? 0.0 :
                  (double)T * ((double)n * (U ? 8.0 : 4.0) +
                               (double)k * ((hdt == SP_BF16 ? (lo_off > 0 ? 4.0 : 2.0) : 4.0) + (gate ? 4.0 : 0.0))),
                  stream);
@@ -1048,7 +1052,7 @@ cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, voi
   const int32_t rows_per = (int32_t)ceil_div(T, rb);
   count_launch();
   prep_h_kernel<<<dim3(gx, (unsigned)ceil_div(T, (int64_t)rows_per)), 256, 0, stream>>>(Z, U, gate, H, hdt, T, n, ldh, ncols, lo_off,
-                                                                                        k, idx, rows_per);
+                                                                                        k, idx, rows_per, skip_flag());
   return cudaGetLastError();
 }
 

@@ -717,6 +717,46 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
             assert torch.equal(mod.H_next[:, :k], torch.clamp(mod.Z[:, kept], min=0).to(torch.bfloat16))
         seen.append(same_order)
     assert seen[0] is False and any(seen[1:5]) and (rule != "paper" or seen[5] is False)
+    if with_r1:
+        # the a-update of a step whose mask stays really starts from the h in the state (its gather kernels are queued
+        # but return at once): a planted change of that h must show in the step's result; after a mask change the
+        # gather runs and overwrites the planted value
+        twins = []
+        for _ in range(2):
+            t, _, _, _ = _make_module(cfg, chunk=512, overlap_k=k)
+            t.sp_ffn_init()
+            p_gpu, _ = params(1.0, 1.5)
+            for _ in range(2):
+                t.sp_admm_step(p_gpu)
+            twins.append(t)
+        torch.cuda.synchronize()
+        ta, tb = twins
+        assert ta.read_report()["pruned_scaled"] == 1.0 and torch.equal(ta.mask, tb.mask)
+        kept0 = int(torch.nonzero(ta.mask).flatten()[0])
+        tb.H_next[0, 0] += 4.0
+        for t in twins:
+            t.sp_admm_step(p_gpu)
+        torch.cuda.synchronize()
+        assert ta.read_report()["pruned_scaled"] == 1.0
+        assert float((ta.Z[0] - tb.Z[0]).abs().max()) > 1e-2 * float(ta.Z[0].abs().max())     # token 0 saw the planted h
+        assert float((ta.Z[1:] - tb.Z[1:]).abs().max()) < 1e-3 * float(ta.Z.abs().max())      # the others did not
+        # other mask -> the gather runs: the planted value is gone and both modules agree again
+        for t in twins:
+            t.mask.copy_(torch.roll(t.mask, 1))
+        tb.H_next[0, 0] += 4.0
+        p_fix = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=_RULE[rule], token_chunk=512,
+                               compute_objective=False, reselect_mask=False)
+        Za, Zb = ta.Z.clone(), tb.Z.clone()
+        for t in twins:
+            t.sp_admm_step(p_fix)
+        torch.cuda.synchronize()
+        assert ta.read_report()["pruned_scaled"] == 0.0
+        # (the two modules entered this step with slightly different Z in token 0 only; what matters is that the
+        # planted h did not enter: the change of token 0 is of the size of its earlier difference, not of the plant)
+        d_before = float((Za[0] - Zb[0]).abs().max())
+        d_after = float((ta.Z[0] - tb.Z[0]).abs().max())
+        assert d_after < 4.0 * max(d_before, 1e-3 * float(ta.Z.abs().max()))
+        del twins, ta, tb
     # without the ordered accumulators nothing is scaled and the same checks hold
     mod2 = api.FfnModule(X.to(DEV), W1.to(DEV), W2.to(DEV), token_chunk=512, pruned_decay=False)
     mod2.sp_ffn_init()
