@@ -75,6 +75,12 @@ def run():
     for it in range(3):
         torch.cuda.synchronize()
         acc = dict(G_A=mod.G_A.cpu().numpy().copy(), R2=mod.R2.cpu().numpy().copy(), mask_before=mod.mask.cpu().numpy().copy())
+        # a few channels that the mask prunes, and their columns of Z before the step: with an unchanged mask their
+        # a of this step is max(z, 0) of that Z
+        pruned_ch = np.flatnonzero(acc["mask_before"] == 0)
+        pruned_ch = pruned_ch[np.linspace(0, pruned_ch.size - 1, 6).astype(int)] if pruned_ch.size else pruned_ch
+        pc = torch.tensor(pruned_ch, device=DEV, dtype=torch.long)
+        acc.update(pruned_ch=pruned_ch, Zp_before=np64(mod.Z[:, pc]))
         mod.sp_admm_step(p)
         torch.cuda.synchronize()
         mod.check_status()
@@ -82,7 +88,10 @@ def run():
         mask_after = mod.mask.cpu().numpy().copy()
         assert rep["factor_reused"] == float(np.array_equal(mask_after, acc["mask_before"]))
         if rep["factor_reused"] == 1.0:
-            acc.update(W2=np64(mod.W2), mask=mask_after, step=it + 2)
+            dsel = torch.tensor(snap["ch_d"], device=DEV, dtype=torch.long)
+            acc.update(W2=np64(mod.W2), mask=mask_after, step=it + 2, pruned_scaled=rep["pruned_scaled"],
+                       G_pp=np64(mod.G_A[pc][:, pc]), R2_p=np64(mod.R2[dsel][:, pc]), R1_p=np64(mod.R1[pc][:, dsel]),
+                       Zp_after=np64(mod.Z[:, pc]), Yd=np64(mod.Ypre[:, dsel]), Xd=np64(X[:, dsel]))
             snap["later"] = acc
             break
     del mod
@@ -165,3 +174,24 @@ def test_later_step_reuses_the_factor(run):
     print(f"{cfg.name}: step {later['step']} reused the factor, W2 error {relerr(later['W2'], W2):.2e}")
     assert relerr(later["W2"], W2) < TOLB
     assert np.all(later["W2"][:, later["mask"] == 0] == 0)
+
+
+def test_later_step_scales_the_pruned_parts_of_the_accumulators(run):
+    """The same later step (mask unchanged): the library obtained G_A[pruned, pruned], R2[:, pruned] and R1[pruned, :]
+    by scaling the values of the step before (report field pruned_scaled; ReLU modules).  Sampled entries against their
+    definitions as fp64 sums over ALL tokens: a pruned channel's a of this step is max(z, 0) of its Z before the step,
+    and its new Z is what the step left."""
+    later = run["later"]
+    assert later is not None
+    gated = bool(run.get("gated", False))
+    assert later["pruned_scaled"] == (0.0 if gated else 1.0)
+    if gated:
+        return          # a gated module contracts these parts in every step; test_accumulator_entries covers its products
+    Ap = np.maximum(later["Zp_before"], 0.0)                 # [N, 6]
+    dg = np.sqrt((Ap * Ap).sum(0))
+    assert np.all(np.abs(later["G_pp"] - Ap.T @ Ap) <= TOLB * np.outer(dg, dg))
+    ys = np.sqrt((later["Yd"] ** 2).sum(0))
+    assert np.all(np.abs(later["R2_p"] - later["Yd"].T @ Ap) <= TOLB * np.outer(ys, dg))
+    zs = np.sqrt((later["Zp_after"] ** 2).sum(0))
+    xs = np.sqrt((later["Xd"] ** 2).sum(0))
+    assert np.all(np.abs(later["R1_p"] - later["Zp_after"].T @ later["Xd"]) <= TOLB * np.outer(zs, xs))
