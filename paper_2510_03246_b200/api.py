@@ -475,7 +475,11 @@ class FfnModule:
         Wg_0 (gate projection [n, d]) makes the module a SwiGLU one: W1_0 is then its up projection.
         scores (fp32 [n]) / mask (uint8 [n]): caller-owned contiguous buffers, e.g. rows of one [L, n] array over
         which a lock-step run selects a single global threshold.  ws_pool: a dict shared by modules that are never
-        in flight at the same time; they then use one workspace."""
+        in flight at the same time; they then use one workspace.
+        pruned_decay (bf16 storage, ReLU, no dual variable): hold the ordered accumulators of sp_ffn_state (G_A_perm,
+        R2_perm, decay_tag; with overlap_k > 0 also R1_perm and H_next, sized for overlap_k kept units), with which a
+        step whose mask stays scales the pruned channels' parts of G_A, R1, R2 instead of contracting them again.
+        Code that writes Z of such a module itself must set decay_tag[1] = -1 afterwards."""
         _require_cuda(X, W1_0, W2_0, Wg_0)
         assert X.dtype in (torch.float32, torch.bfloat16)
         self.X = X.contiguous()
