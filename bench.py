@@ -547,42 +547,51 @@ def main():
         oW1 = torch.empty(cfg.n, cfg.d, dtype=torch.float32).pin_memory(); oW2 = torch.empty(cfg.d, cfg.n, dtype=torch.float32).pin_memory()
         omask = torch.empty(cfg.n, dtype=torch.uint8).pin_memory()
         oWo = torch.empty(cfg.d, cfg.d, dtype=torch.float32).pin_memory(); ohm = torch.empty(cfg.heads, dtype=torch.uint8).pin_memory()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
-        dWg = hWg.to(dev, non_blocking=True) if hWg is not None else None
-        m2 = api.FfnModule(dX, dW1, dW2, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=dWg)
-        m2.sp_ffn_init()
-        # this layer's share of pass 0: the importance of the pre-trained module
-        api.sp_struct_scores(api.SP_SCORE_WANDA_L2, cfg.n, W=m2.W2_0, colsq=m2.G_A, colsq_stride=cfg.n + 1)
-        for _ in range(iters):
-            m2.sp_admm_step(prm)
-        oW1.copy_(m2.W1, non_blocking=True); oW2.copy_(m2.W2, non_blocking=True); omask.copy_(m2.mask, non_blocking=True)
-        torch.cuda.synchronize()
-        t_ffn = time.perf_counter()
-        # attention module: pre-trained output of the projection, head scores, head mask, W_O recovery on the kept heads
-        dH = hH.to(dev, non_blocking=True); dWo = hWo.to(dev, non_blocking=True)
-        Ya = torch.empty(dH.shape[0], cfg.d, dtype=dH.dtype, device=dev)
-        api.sp_gemm(dH, dWo, Ya, transB=True, use_tensor_cores=(dH.dtype == torch.bfloat16))
-        hmask, Wo_new, _ = pipeline.prune_attention_heads(dH, Ya, dWo.float(), cfg.heads, k_heads, rho=cfg.rho,
-                                                          token_chunk=args.chunk)
-        oWo.copy_(Wo_new, non_blocking=True); ohm.copy_(hmask, non_blocking=True)
-        torch.cuda.synchronize()
-        t1 = time.perf_counter()
-        m2.check_status()
+        def one_layer():
+            """The whole job of one layer, host buffers in, host buffers out; returns (t_ffn, t_total) in seconds."""
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            dX = hX.to(dev, non_blocking=True); dW1 = hW1.to(dev, non_blocking=True); dW2 = hW2.to(dev, non_blocking=True)
+            dWg = hWg.to(dev, non_blocking=True) if hWg is not None else None
+            m2 = api.FfnModule(dX, dW1, dW2, dual_mode=args.dual, token_chunk=args.chunk, overlap_k=cfg.k_keep, Wg_0=dWg,
+                               pruned_decay=not args.no_pruned_decay)
+            m2.sp_ffn_init()
+            # this layer's share of pass 0: the importance of the pre-trained module
+            api.sp_struct_scores(api.SP_SCORE_WANDA_L2, cfg.n, W=m2.W2_0, colsq=m2.G_A, colsq_stride=cfg.n + 1)
+            for _ in range(iters):
+                m2.sp_admm_step(prm)
+            oW1.copy_(m2.W1, non_blocking=True); oW2.copy_(m2.W2, non_blocking=True); omask.copy_(m2.mask, non_blocking=True)
+            torch.cuda.synchronize()
+            t_ffn = time.perf_counter()
+            # attention module: pre-trained output of the projection, head scores, head mask, W_O recovery on the kept heads
+            dH = hH.to(dev, non_blocking=True); dWo = hWo.to(dev, non_blocking=True)
+            Ya = torch.empty(dH.shape[0], cfg.d, dtype=dH.dtype, device=dev)
+            api.sp_gemm(dH, dWo, Ya, transB=True, use_tensor_cores=(dH.dtype == torch.bfloat16))
+            hmask, Wo_new, _ = pipeline.prune_attention_heads(dH, Ya, dWo.float(), cfg.heads, k_heads, rho=cfg.rho,
+                                                              token_chunk=args.chunk)
+            oWo.copy_(Wo_new, non_blocking=True); ohm.copy_(hmask, non_blocking=True)
+            torch.cuda.synchronize()
+            t1 = time.perf_counter()
+            m2.check_status()
+            return t_ffn - t0, t1 - t0
+
+        # a model is a sequence of such layers: the first one here warms the allocator's cache and the library's
+        # one-time set-ups (as every layer after the first of a real run finds them), the second one is timed
+        first_ffn, first_total = one_layer()
+        t_ffn_s, t_total_s = one_layer()
         h2d = hX.numel() * hX.element_size() + hW1.numel() * hW1.element_size() + hW2.numel() * hW2.element_size()
         if hWg is not None:
             h2d += hWg.numel() * hWg.element_size()
         h2d += hH.numel() * hH.element_size() + hWo.numel() * hWo.element_size()
         d2h = oW1.numel() * 4 + oW2.numel() * 4 + omask.numel() + oWo.numel() * 4 + ohm.numel()
-        e2e = {"value": iters / (t1 - t0), "unit": UNIT, "layers_per_s": 1.0 / (t1 - t0), "h2d_bytes_per_step": h2d / iters,
-               "d2h_bytes_per_step": d2h / iters, "iterations": iters, "ffn_seconds": t_ffn - t0,
-               "attention_seconds": t1 - t_ffn,
+        e2e = {"value": iters / t_total_s, "unit": UNIT, "layers_per_s": 1.0 / t_total_s, "h2d_bytes_per_step": h2d / iters,
+               "d2h_bytes_per_step": d2h / iters, "iterations": iters, "ffn_seconds": t_ffn_s,
+               "attention_seconds": t_total_s - t_ffn_s, "first_layer_seconds": first_total,
                "note": "one pruned layer: pinned-host X, W1_0, W2_0 in; init + importance of the pre-trained module + "
                        "iterations; W1, W2, mask back to host; then the attention half with fixed head outputs (H, "
                        "W_O in; head scores, head mask, W_O recovery on the kept heads; W_O, mask out); "
-                       "layers_per_s is that whole job per second, value = iterations / that time"}
-        del m2, dX, dW1, dW2, dWg, dH, dWo, Ya, Wo_new
+                       "layers_per_s is that whole job per second, value = iterations / that time; the job runs twice "
+                       "(two layers of a model) and the second run is the one reported, first_layer_seconds is the first"}
     else:
         del mod, X, W1_0, W2_0, Wg_0
     torch.cuda.empty_cache()
