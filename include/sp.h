@@ -147,7 +147,8 @@ typedef struct {
   int32_t dual_mode;       /* 0: paper's penalty form; 1: scaled dual U on a = phi(z) (an extension of the paper)  */
   int32_t score_kind;      /* sp_score_kind                                                                       */
   int64_t k_keep;          /* units kept in this module (from sp_allocate_sparsity)                                */
-  int32_t reselect_mask;   /* 1: recompute the top-k mask from this step's scores; 0: keep st->mask                */
+  int32_t reselect_mask;   /* 1: recompute the top-k mask from this step's scores; 0: keep st->mask, which must keep
+                              exactly k_keep units (else SP_ERR_SHAPE through status_dev, index = units it keeps)   */
   int32_t refit;           /* 1: recovery solver on the kept support (Algorithm 2); 0: plain M (.) W               */
   int64_t token_chunk;     /* tokens per streamed chunk (0 = library default)                                      */
   int32_t compute_objective; /* 1: also report alpha|Ypre-W2A|^2 (one more product per token chunk)                 */

@@ -886,7 +886,10 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
 
   // ---- 3. top-k mask
   if (prm->reselect_mask) CU(topk_select(st->scores, n, k, st->mask, nullptr, p.sb.idx, s));
-  else CU(mask_to_index(st->mask, n, p.sb.idx, s));
+  else {
+    CU(mask_to_index(st->mask, n, p.sb.idx, s));
+    CU(mask_count_check(st->mask, n, k, status_dev, s));     // a given mask must keep exactly k_keep units
+  }
   if (reuse) CU(mask_changed(st->mask, p.perm, p.reuse_flags + 2, k, p.reuse_flags, s));
 
   // ---- 4. masked weights: W1 = diag(M) W1~ ; W2 = recovery on the kept support (or M (.) W2~)

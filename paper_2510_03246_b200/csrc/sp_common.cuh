@@ -364,6 +364,9 @@ cudaError_t global_select(const float* scores, int64_t ld_scores, int64_t n, int
                           uint8_t* mask, int64_t ld_mask, float* tau, int64_t* counts_out, void* scratch,
                           cudaStream_t stream);
 cudaError_t mask_to_index(const uint8_t* mask, int64_t n, int32_t* kept_idx, cudaStream_t stream);
+// reports SP_ERR_SHAPE (index = the number of kept units found) through the device status word when `mask` does not
+// keep exactly k units; no-op without a status word
+cudaError_t mask_count_check(const uint8_t* mask, int64_t n, int64_t k, int32_t* status, cudaStream_t stream);
 // C[i, j] *= f^power for the rows x cols block at C (ld); f is read from the device (a float stored in an int32 slot)
 cudaError_t scale_block(float* C, int64_t ld, int64_t rows, int64_t cols, const int32_t* f_bits, int power,
                         cudaStream_t stream);

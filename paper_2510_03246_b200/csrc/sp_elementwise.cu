@@ -677,7 +677,9 @@ __global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __rest
     }
     // h of the next step: per row the warp's kept channels are one contiguous run of H; consecutive lanes write
     // consecutive elements (max(bf16(z), 0) = bf16(max(z, 0)): rounding keeps the sign)
-    for (int e = lane; e < cnt_w; e += 32) {
+    // (compact positions beyond k exist only if the caller's mask keeps more channels than k_keep says: they are not
+    // written, so that a wrong argument cannot reach past a row of Hn)
+    for (int e = lane; e < cnt_w && base_w + e < k; e += 32) {
       // the 32 rows of this kept channel: 64 contiguous bytes of the tile (8-byte aligned rows)
       __align__(8) __nv_bfloat16 zr[kAtRows];
       const uint2* src = reinterpret_cast<const uint2*>(&zt_tile[(wch0 + kept_ch[warp][e]) * kAtPitch]);

@@ -1433,6 +1433,26 @@ cudaError_t unpermute_rows(const float* Rp, const int32_t* perm, int64_t n, int6
   return cudaGetLastError();
 }
 
+__global__ void __launch_bounds__(1024) mask_count_check_kernel(const uint8_t* mask, int64_t n, int64_t k,
+                                                                int32_t* status) {
+  __shared__ int warp_tot[32];
+  int kept = 0;
+  for (int64_t base = 0; base < n; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    int tot;
+    block_excl_scan((i < n) && mask[i] != 0, warp_tot, &tot);
+    kept += tot;
+  }
+  if (threadIdx.x == 0 && kept != k) report_status(status, SP_ERR_SHAPE, kept, 21);
+}
+
+cudaError_t mask_count_check(const uint8_t* mask, int64_t n, int64_t k, int32_t* status, cudaStream_t stream) {
+  if (status == nullptr) return cudaSuccess;
+  count_launch();
+  mask_count_check_kernel<<<1, 1024, 0, stream>>>(mask, n, k, status);
+  return cudaGetLastError();
+}
+
 cudaError_t mask_to_perm(const uint8_t* mask, int64_t n, int32_t* perm, int32_t* count, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
   count_launch();

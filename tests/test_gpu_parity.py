@@ -911,6 +911,28 @@ def test_admm_step_fixed_mask():
     assert torch.equal(mask1, mod.mask)
 
 
+def test_given_mask_with_another_count_is_reported():
+    """reselect_mask = 0 with a mask that does not keep k_keep units: the device status word carries SP_ERR_SHAPE and the
+    number of units the mask keeps (the host cannot see the mask)."""
+    cfg = SMALL_BF16
+    k = cfg.k_keep
+    mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=k)
+    mod.sp_ffn_init()
+    mod.sp_admm_step(api.AdmmParams(rho=cfg.rho, k_keep=k, token_chunk=512))
+    torch.cuda.synchronize()
+    mod.check_status()
+    guard = mod.H_next.clone()
+    mod.mask.fill_(0)
+    mod.mask[: k - 40] = 1                       # keeps 40 units too few (every compact position stays below k_keep)
+    mod.sp_admm_step(api.AdmmParams(rho=cfg.rho, k_keep=k, token_chunk=512, reselect_mask=False, skip_scores=True))
+    torch.cuda.synchronize()
+    st = mod.status.cpu().tolist()
+    assert st[0] == 2 and st[1] == k - 40        # SP_ERR_SHAPE, units kept
+    assert mod.H_next.shape == guard.shape and torch.isfinite(mod.H_next.float()).all()
+    with pytest.raises(api.SpError):
+        mod.check_status()
+
+
 def test_admm_step_argument_errors():
     mod, X, W1, W2 = _make_module(SMALL_F32)
     mod.sp_ffn_init()
