@@ -34,7 +34,9 @@ def _oracle_forward(X, W, H, T, n_seq, causal):
 
 CASES = [(torch.float32, 48, 4, 20, 3, 2, True), (torch.float32, 32, 1, 33, 2, 0, False),
          (torch.bfloat16, 96, 4, 40, 3, 2, True), (torch.bfloat16, 256, 2, 136, 2, 1, False),
-         (torch.bfloat16, 128, 2, 264, 1, 0, True), (torch.bfloat16, 512, 8, 520, 2, 1, True)]
+         (torch.bfloat16, 128, 2, 264, 1, 0, True), (torch.bfloat16, 512, 8, 520, 2, 1, True),
+         # three heads of width 128: three blocks per system in the batched solves of the W_V recovery
+         (torch.bfloat16, 384, 3, 72, 2, 1, True)]
 
 
 @pytest.mark.parametrize("dtype,d,H,T,n_seq,chunk,causal", CASES)
