@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
     auto load_row = [&](int64_t r, UpdRow<HAS_U>& w) {
       const int64_t e = r * g.n + c0;
       if (vec) {
-        const float4 v = *reinterpret_cast<const float4*>(Zp + e);
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(Zp + e));     // read once: streaming
         w.zo[0] = v.x; w.zo[1] = v.y; w.zo[2] = v.z; w.zo[3] = v.w;
         if (HAS_U) {
           const float4 x = *reinterpret_cast<const float4*>(Up + e);
@@ -451,8 +451,8 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const bool kept = (bits >> q) & 1u;
-        w.z1[q] = kept ? zp[off[q]] : 0.f;
-        w.dc[q] = kept ? dp[off[q]] : 0.f;
+        w.z1[q] = kept ? __ldcs(zp + off[q]) : 0.f;
+        w.dc[q] = kept ? __ldcs(dp + off[q]) : 0.f;
       }
     };
     auto finish_row = [&](int64_t r, UpdRow<HAS_U>& w, __nv_bfloat16* arow) {
@@ -476,7 +476,9 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
       s_a += (double)p_a;
       s_in += (double)p_in;
       if (vec) {
-        *reinterpret_cast<float4*>(Zp + e) = make_float4(zn[0], zn[1], zn[2], zn[3]);
+        // Z and its operands are touched once per step: streaming accesses keep them from displacing the transposed A,
+        // which the accumulator products read next (measured: 6.8 against 6.95 ms per C2 step)
+        __stcs(reinterpret_cast<float4*>(Zp + e), make_float4(zn[0], zn[1], zn[2], zn[3]));
         if (HAS_U) *reinterpret_cast<float4*>(Up + e) = make_float4(w.u[0], w.u[1], w.u[2], w.u[3]);
         if (g.At_out) {
 #pragma unroll
