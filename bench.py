@@ -378,8 +378,13 @@ def rooflines(cfg, args, prof, steps, peaks):
     hbm = peaks.get("hbm_gbs", 6650.0)
     fu = prof["fused_update"]
     fu_traffic = None
+    # ReLU modules without the dual variable that hold the ordered accumulators run the form of the update that also
+    # writes the next step's operands (the transposed bf16 copy of Z and h)
+    writes_next = (cfg.storage == "bf16" and cfg.act == "relu" and not args.dual and not args.no_pruned_decay
+                   and cfg.n % 4 == 0 and cfg.tokens % 8 == 0 and args.chunk % 8 == 0)
+    fu_kernel = "fused_update_next_kernel" if writes_next else "fused_update_kernel"
     if args.chunk == 32768 and not args.dual and cfg.tokens % args.chunk == 0:
-        fu_traffic = captured_traffic("fused_update_kernel", f"{cfg.name}:n={cfg.n},k={cfg.k_keep},tokens=32768")
+        fu_traffic = captured_traffic(fu_kernel, f"{cfg.name}:n={cfg.n},k={cfg.k_keep},tokens=32768")
     fu_gbs = fu["bytes"] / (fu["ms"] * 1e-3) / 1e9 if fu["ms"] else 0.0
     # bytes the two elementwise kernels of the token pass move per token (their own algorithmic counts), against the
     # minimum of a pass that reads X, Ypre, Z once and writes Z once in the storage type: s (2 d + 2 n)
@@ -387,14 +392,15 @@ def rooflines(cfg, args, prof, steps, peaks):
     esz = 2.0 if cfg.storage == "bf16" else 4.0
     per_token = (fu["bytes"] + ph["bytes"]) / max(steps, 1) / cfg.tokens
     minimum = esz * (2.0 * cfg.d + 2.0 * cfg.n)
-    roofline_hbm = {"bound": "hbm", "kernel": "fused_update_kernel", "achieved": fu_gbs, "peak": hbm, "unit": "GB/s",
+    roofline_hbm = {"bound": "hbm", "kernel": fu_kernel, "achieved": fu_gbs, "peak": hbm, "unit": "GB/s",
                     "frac": fu_gbs / hbm, "traffic": fu_traffic,
                     "algorithmic_bytes_per_launch": fu["bytes"] / max(fu["records"], 1), "launches": fu["records"],
                     "elementwise_bytes_per_token": per_token, "minimum_bytes_per_token": minimum,
                     "bytes_over_minimum": per_token / minimum,
-                    "bytes_note": "elementwise_bytes_per_token: h gather + fused update (Z kept in fp32, A and a "
-                                  "storage copy of Z written for the accumulator products, D and z1 read); minimum: "
-                                  "X, Ypre, Z read once and Z written once in the storage type",
+                    "bytes_note": "elementwise_bytes_per_token: h gather (none while the mask stays when the update "
+                                  "leaves h for the next step) + fused update (Z kept in fp32, A and a storage copy of "
+                                  "Z written for the accumulator products, D and z1 read); minimum: X, Ypre, Z read "
+                                  "once and Z written once in the storage type",
                     "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback (6.65 TB/s)"}
     breakdown = {k: {"records": v["records"], "ms_per_step": v["ms"] / steps,
                      **({"tflops": v["flops"] / (v["ms"] * 1e-3) / 1e12} if v["flops"] and v["ms"] else {}),

@@ -130,12 +130,15 @@ typedef struct {
   float* R2_perm;      /* [d, n]                                                                                     */
   int32_t* decay_tag;  /* int32 [n + 8]                                                                              */
   /* Optional on top of the three above (both or none): R1 in the same way — Z of a pruned channel is c times its old
-   * value too, so R1[pruned, :] is scaled, and only the kept rows are contracted.  For that a pass over the new Z of
-   * every chunk writes its bf16 copy transposed with the kept channels first (instead of the row-major copy the fused
-   * update would write), and in the same pass h = max(Z_new, 0) of the kept channels into H_next: the a-update of the
-   * NEXT step starts from it and skips its own gather pass over Z while the mask stays. */
+   * value too, so R1[pruned, :] is scaled, and only the kept rows are contracted.  For that the fused update writes the
+   * bf16 copy of the new Z transposed with the kept channels first (instead of a row-major copy), and from the same
+   * registers h = max(Z_new, 0) of the kept channels into H_next: the a-update of the NEXT step starts from it and makes
+   * no gather pass over Z while the mask stays, so that Z is read once and written once per step.  Used when N % 8 == 0.
+   * Layout of H_next (the library's own; it depends on the token chunk): for the chunk of Tc tokens that starts at
+   * token t0, the k_keep x Tc block h^T (kept channels in ascending order, tokens contiguous) at element
+   * t0 * H_next_ld. */
   float* R1_perm;      /* [n, d]                                                                                     */
-  void* H_next;        /* [N, H_next_ld] bf16                                                                        */
+  void* H_next;        /* N * H_next_ld bf16 elements                                                                */
   int64_t H_next_ld;   /* a multiple of 8, at least ceil8(k_keep); smaller: R1_perm / H_next are not used             */
 } sp_ffn_state;
 

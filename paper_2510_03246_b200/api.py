@@ -531,6 +531,17 @@ class FfnModule:
         self._pool = ws_pool if ws_pool is not None else {}
         self.iteration = 0
 
+    def h_next_rows(self, k: int, token_chunk: int) -> torch.Tensor:
+        """[N, k] view-by-copy of the h that the last step left for the next one in H_next (sp_ffn_state.H_next: per
+        token chunk a [k, Tc] block, tokens contiguous, at element t0 * H_next_ld)."""
+        flat, ld = self.H_next.view(-1), self.H_next.shape[1]
+        chunk = int(token_chunk) if token_chunk else self.N
+        out = []
+        for t0 in range(0, self.N, chunk):
+            Tc = min(chunk, self.N - t0)
+            out.append(flat[t0 * ld: t0 * ld + k * Tc].view(k, Tc).t())
+        return torch.cat(out, 0)
+
     @property
     def _ws(self):
         return self._pool.get("ws")

@@ -302,6 +302,12 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.D = c.take<float>((size_t)p.chunk * npad);
   p.z1 = c.take<float>((size_t)p.chunk * npad);
   p.nblocks = fused_update_grid(p.chunk, n, &p.row_blocks);
+  {
+    int rb2 = 1;       // the form of the update that also writes the next step's operands has its own grid
+    const int nb2 = fused_update_next_grid(p.chunk, n, &rb2);
+    if (nb2 > p.nblocks) p.nblocks = nb2;
+    if (rb2 > p.row_blocks) p.row_blocks = rb2;
+  }
   p.partial = c.take<double>((size_t)p.nblocks * 4 + kSumsqBlocks);
   p.Eo = c.take<float>((size_t)p.chunk * d);
   p.W2fb = p.bf16 ? c.take_bytes((size_t)n * d * csz) : nullptr;
@@ -706,7 +712,7 @@ sp_status sp_ffn_init(const sp_ffn_module* m, sp_ffn_state* st, int64_t token_ch
   InitPlan p = plan_init(ws, d, n, N, token_chunk, cdt);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const bool bf16 = p.bf16;
-  if (st->decay_tag != nullptr) CU(decay_tag_set(st->decay_tag, 0, 0.f, false, 0, s));   // Z is rewritten
+  if (st->decay_tag != nullptr) CU(decay_tag_set(st->decay_tag, 0, 0.f, false, 0, 0, s));   // Z is rewritten
   const bool acc64 = !bf16;
   const bool gated = m->act == SP_ACT_SWIGLU;
   MatRef w10{m->W1_0.ptr, SP_F32, m->W1_0.ld}, w20{m->W2_0.ptr, SP_F32, m->W2_0.ld};
@@ -1015,12 +1021,13 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
                      st->R2_perm != nullptr && st->decay_tag != nullptr && !misaligned(st->G_A_perm, 16) &&
                      !misaligned(st->R2_perm, 16) && !misaligned(st->decay_tag, 4);
   // R1 the same way (Z of a pruned channel is c times its old value as well).  Its operand then is a bf16 copy of the
-  // new Z written TRANSPOSED with the kept channels first, by a pass of its own over the new Z of each chunk; that pass
-  // also leaves h = max(Z_new, 0) of the kept channels for the next step, whose own gather pass over Z is then skipped
-  // while the mask stays (so Z is still read twice and written once per step).
+  // new Z written TRANSPOSED with the kept channels first, by the fused update itself, which also leaves
+  // h = max(Z_new, 0) of the kept channels (transposed as well: chunk by chunk a [k, chunk] block of H_next, the block
+  // of the chunk that starts at token t0 at element t0 * H_next_ld) for the next step, whose own gather pass over Z is
+  // then skipped while the mask stays: Z is read once and written once per step.
   const int64_t ldh_next = st->H_next_ld;
   const bool decay_z = decay && st->R1_perm != nullptr && st->H_next != nullptr && ldh_next % 8 == 0 && ldh_next >= kp &&
-                       !misaligned(st->R1_perm, 16) && !misaligned(st->H_next, 16);
+                       N % 8 == 0 && !misaligned(st->R1_perm, 16) && !misaligned(st->H_next, 16);
   int32_t* order_changed = p.reuse_flags + 4;
   int32_t* order_same = p.reuse_flags + 5;
   int32_t* h_ready = p.reuse_flags + 6;
@@ -1028,14 +1035,14 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     // tag: [1] k of the last pass (-1: none), [2] its c (float bits), [4] row pitch of the h it left, [8..] its order
     int32_t* tag = st->decay_tag;
     CU(mask_changed(st->mask, tag + 8, tag + 1, k, order_changed, s));
-    if (decay_z) CU(h_next_ready(order_same, tag, ldh_next, h_ready, s));
+    if (decay_z) CU(h_next_ready(order_same, tag, ldh_next, p.chunk, h_ready, s));
     {
       SkipScope unless_same(order_changed);
       CU(scale_block(st->G_A_perm + (size_t)k * n + k, n, n - k, n - k, tag + 2, 2, s));
       CU(scale_block(st->R2_perm + k, n, d, n - k, tag + 2, 1, s));
     }
     CU(mask_to_perm(st->mask, n, tag + 8, tag + 3, s));
-    CU(decay_tag_set(tag, k, (float)(prm->beta / (prm->alpha + prm->beta)), true, decay_z ? ldh_next : 0, s));
+    CU(decay_tag_set(tag, k, (float)(prm->beta / (prm->alpha + prm->beta)), true, decay_z ? ldh_next : 0, p.chunk, s));
     if (decay_z) {
       // Z_new = c max(Z, 0) with THIS step's c (A above is max(Z, 0) of the old Z: the c of the step that wrote it);
       // R1_perm and H_next hold the last pass's values only if that pass wrote them
@@ -1043,7 +1050,7 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
       CU(scale_block(st->R1_perm + (size_t)k * d, d, n - k, d, tag + 2, 1, s));
     }
   } else if (!scores_only && st->decay_tag != nullptr) {
-    CU(decay_tag_set(st->decay_tag, 0, 0.f, false, 0, s));    // Z changes without the ordered accumulators being rebuilt
+    CU(decay_tag_set(st->decay_tag, 0, 0.f, false, 0, 0, s));    // Z changes without the ordered accumulators being rebuilt
   }
   if (z1_ahead) CU(cudaStreamWaitEvent(s, side->z1_done, 0));
   if (rep_dev) CU(init_report(rep_dev, rho1, rho2, (double)k, reuse ? p.reuse_flags + 1 : nullptr,
@@ -1083,14 +1090,15 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
       SPCHK(gemm_tc(Tc, k, d, 1.f, da, db, 0.f, Operand{p.D, SP_F32, kp, 1}, OutOperand{p.D, SP_F32, kp}, false,
                     status_dev, s, &sd, 2.0 * (double)Tc * d * k));
     } else if (decay_z) {
-      // h of this chunk sits in the state: written by the last step's pass over its new Z, or gathered now
+      // h of this chunk sits in the state, transposed ([k, Tc], tokens contiguous): written by the last step's update,
+      // or gathered now
       __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(st->H_next) + (size_t)t0 * ldh_next;
       {
         SkipScope unless_stale(h_ready);
-        CU(launch_prep_h(Zc, Uc, Gc, Hc, cdt, Tc, n, ldh_next, k, idx, s));
+        CU(launch_gather_ht(Zc, Tc, n, k, p.grp_base, p.grp_mask, Hc, Tc, s));
       }
-      MatRef hn{Hc, cdt, ldh_next};
-      SPCHK(contract(Tc, d, k, -1.0, hn, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
+      MatRef hn{Hc, cdt, Tc};
+      SPCHK(contract(Tc, d, k, -1.0, hn, false, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
     } else {
       CU(launch_prep_h(Zc, Uc, Gc, p.H, cdt, Tc, n, kp, k, idx, s));
       SPCHK(contract(Tc, d, k, -1.0, h, true, w2, true, 1.0, yc, e, false, acc64, bf16, status_dev, s));
@@ -1111,8 +1119,14 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
     const bool a_transposed = bf16 && n % 4 == 0 && !(rep_dev && prm->compute_objective) && Tld <= p.chunk;
     if (a_transposed) { ua.At_out = p.Ac; ua.ldt = Tld; }
     if (decay) ua.at_kept_first = 1;     // (the pruned rows are still needed: G_A[pruned, kept] is contracted anew)
-    if (decay_z) ua.Zb_out = nullptr;    // the copy of Z for R1 is written transposed by the pass below
-    const int nblk = fused_update_grid(Tc, n, &ua.row_blocks);
+    if (decay_z) {
+      // the copy of Z for R1 and the next step's h are written transposed, by the same kernel
+      ua.Zb_out = nullptr;
+      ua.Zt_out = p.Zb;
+      ua.Ht_out = reinterpret_cast<__nv_bfloat16*>(st->H_next) + (size_t)t0 * ldh_next;
+      ua.zt_pruned_flag = h_ready + 1;       // the pruned rows of R1 are contracted only in a step that found h stale
+    }
+    const int nblk = decay_z ? fused_update_next_grid(Tc, n, &ua.row_blocks) : fused_update_grid(Tc, n, &ua.row_blocks);
     CU(launch_fused_update(ua, s));
     if (rep_dev) CU(reduce_report(p.partial, nblk, rep_dev, ci > 0, prm->alpha, s));
     if (rep_dev && prm->compute_objective) {
@@ -1146,8 +1160,6 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
       SPCHK(contract(d, n, Tc, 1.0, yc, false, ac, false, acc, r2, r2, false, acc64, bf16, status_dev, s));
     }
     if (decay_z) {
-      __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(st->H_next) + (size_t)t0 * ldh_next;
-      CU(launch_gather_next(Zc, Tc, n, k, p.grp_base, p.grp_mask, p.Zb, Tld, Hc, ldh_next, s));
       MatRef zt{p.Zb, cdt, Tld}, ztp{reinterpret_cast<const __nv_bfloat16*>(p.Zb) + (size_t)k * Tld, cdt, Tld};
       MatRef r1k{st->R1_perm, SP_F32, d}, r1p{st->R1_perm + (size_t)k * d, SP_F32, d};
       SPCHK(contract(k, d, Tc, 1.0, zt, true, xc, false, acc, r1k, r1k, false, acc64, bf16, status_dev, s));

@@ -272,6 +272,13 @@ struct UpdateArgs {
   // At_out with its rows in "kept channels first" order: kept channel c goes to row (number of kept channels before
   // c), pruned channel c to row k + (number of pruned channels before c).
   int32_t at_kept_first = 0;
+  // Both set (bf16 storage, ReLU, no dual variable, n % 4 == 0, At_out with at_kept_first; grid from
+  // fused_update_next_grid): the update also writes what the next step reads, rows in the order of At_out, pitch ldt:
+  // Zt_out [n, ldt] = bf16(Z_new)^T (the pruned channels' rows only when *zt_pruned_flag != 0 or the flag is null) and
+  // Ht_out [k, ldt] = bf16(max(Z_new, 0))^T on the kept channels.  Zb_out is then not written.
+  void* Zt_out = nullptr;
+  void* Ht_out = nullptr;
+  const int32_t* zt_pruned_flag = nullptr;
 };
 // grp_base / grp_mask of a u8 mask over n channels (see sp_elementwise.cu)
 cudaError_t build_group_map(const uint8_t* mask, int64_t n, int32_t* grp_base, uint8_t* grp_mask, cudaStream_t stream);
@@ -283,11 +290,11 @@ cudaError_t launch_prep_h(const float* Z, const float* U, const float* gate, voi
                           int64_t n, int64_t ldh, int64_t k, const int32_t* idx, cudaStream_t stream,
                           int64_t lo_off = 0);
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
-// From the new Z of a chunk (n % 4 == 0): Zt [n, ldt] bf16 = Z^T with the kept channels' rows first (the order of the
-// transposed A), and Hn [T, ldh] bf16 = max(Z, 0) on the kept channels, compact (h of the next step; ReLU, no dual).
-cudaError_t launch_gather_next(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
-                               const uint8_t* grp_mask, void* Zt, int64_t ldt, void* Hn, int64_t ldh,
-                               cudaStream_t stream);
+// Ht [k, ldt] bf16 = max(Z, 0)^T on the kept channels, rows in compact order (n % 4 == 0; ReLU, no dual variable): h of
+// a step in the transposed layout in which the fused update leaves it for the next one.  Honours SkipScope.
+cudaError_t launch_gather_ht(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
+                             const uint8_t* grp_mask, void* Ht, int64_t ldt, cudaStream_t stream);
+int fused_update_next_grid(int64_t T, int64_t n, int* row_blocks);
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]
 cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
@@ -375,11 +382,13 @@ cudaError_t unpermute_gram(const float* Gp, const int32_t* perm, int64_t n, floa
 // R[r, perm[j]] = Rp[r, j]
 cudaError_t unpermute_cols(const float* Rp, const int32_t* perm, int64_t rows, int64_t n, float* R,
                            cudaStream_t stream);
-// tag[1] = k when `valid`, else -1; tag[2] = bits of the float c; tag[4] = row pitch of the h written for the next
-// step (0: none was written)
-cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, int64_t h_ld, cudaStream_t stream);
-// ready[0] = 1 when same[0] != 0 and the tag says that h was written with row pitch h_ld, else 0; ready[1] = 1 - ready[0]
-cudaError_t h_next_ready(const int32_t* same, const int32_t* tag, int64_t h_ld, int32_t* ready, cudaStream_t stream);
+// tag[1] = k when `valid`, else -1; tag[2] = bits of the float c; tag[4], tag[5] = size of the h buffer per token and
+// token chunk with which h was written for the next step (0: none was written; its layout depends on both)
+cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, int64_t h_ld, int64_t h_chunk,
+                          cudaStream_t stream);
+// ready[0] = 1 when same[0] != 0 and the tag says that h was written for h_ld and h_chunk, else 0; ready[1] = 1 - ready[0]
+cudaError_t h_next_ready(const int32_t* same, const int32_t* tag, int64_t h_ld, int64_t h_chunk, int32_t* ready,
+                         cudaStream_t stream);
 // R[perm[i], :] = Rp[i, :]
 cudaError_t unpermute_rows(const float* Rp, const int32_t* perm, int64_t n, int64_t cols, float* R,
                            cudaStream_t stream);

@@ -451,8 +451,9 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const bool kept = (bits >> q) & 1u;
-        w.z1[q] = kept ? __ldcs(zp + off[q]) : 0.f;
-        w.dc[q] = kept ? __ldcs(dp + off[q]) : 0.f;
+        // (plain loads: a warp's run of kept channels starts and ends inside sectors that the neighbouring warps read too)
+        w.z1[q] = kept ? zp[off[q]] : 0.f;
+        w.dc[q] = kept ? dp[off[q]] : 0.f;
       }
     };
     auto finish_row = [&](int64_t r, UpdRow<HAS_U>& w, __nv_bfloat16* arow) {
@@ -585,22 +586,199 @@ __global__ void __launch_bounds__(256, 2) fused_update_kernel(UpdateArgs g) {
   }
 }
 
-// After the fused update of a chunk (bf16 storage, ReLU, no dual variable), from the NEW Z of the chunk:
-//   Zt[row(c), t] = bf16(Z[t, c]) for every channel c, rows in "kept channels first" order as in the transposed A
-//                   (the K-major operand of R1 = Z^T X, whose pruned rows are only contracted when the mask changed);
-//   Hn[t, p(c)]   = bf16(max(Z[t, c], 0)) for the kept channels at their compact positions: h of the NEXT step's
-//                   a-update, which then needs no gather pass over Z of its own.
-// Same decomposition as the fused update: a thread owns 4 consecutive channels, a warp stages kAtRows rows of its 128
-// channels in shared memory and writes them out as 64-byte pieces.
-__global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __restrict__ Z, int64_t T, int64_t n, int64_t k,
-                                                             const int32_t* __restrict__ grp_base,
-                                                             const uint8_t* __restrict__ grp_mask,
-                                                             __nv_bfloat16* __restrict__ Zt, int64_t ldt,
-                                                             __nv_bfloat16* __restrict__ Hn, int64_t ldh,
-                                                             int32_t row_blocks) {
+// The fused update of a chunk in the form that also leaves what the NEXT step reads (bf16 storage, ReLU, no dual
+// variable, n % 4 == 0, accumulators kept in "kept channels first" order).  Besides the new Z (fp32, in place) and the
+// transposed A it writes, from the same registers,
+//   Zt[row(c), t] = bf16(Z_new[t, c])          the K-major operand of R1 = Z^T X: the kept channels' rows always, the
+//                                              pruned ones only when *zt_pruned_flag != 0 (their part of R1 is a scaled
+//                                              copy of the step before while the mask stays),
+//   Ht[p(c), t]   = bf16(max(Z_new[t, c], 0))  for the kept channels: h of the next step's a-update, transposed,
+// so that Z is read once and written once per step and no separate pass over the new Z is needed.
+// A block owns 512 channels, a warp 64 of them (a thread 2 consecutive ones) and 32 rows at a time: four rounds of
+// eight rows, all loads of a round in flight before its first store.  The warp stages its rows of a and z_new in two
+// shared tiles of its own (channel-major) and writes the 32 rows of every channel out as 64-byte pieces.  (A form in
+// which two warps shared 128 channels and met at a barrier before the write-out, and one in which each of them wrote
+// 32-byte pieces, measured 13 % and 6 % slower.)
+constexpr int kNextChannels = 512;
+constexpr size_t kNextTileBytes = (size_t)2 * kNextChannels * kAtPitch * sizeof(__nv_bfloat16);
+
+__device__ __forceinline__ uint32_t relu_bf16x2(uint32_t v) {
+  __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&v);
+  x = __hmax2(x, __float2bfloat162_rn(0.f));
+  return *reinterpret_cast<uint32_t*>(&x);
+}
+
+struct NextRow {
+  float zo[2], z1[2], dc[2];
+};
+
+template <int Z_RULE>
+__global__ void __launch_bounds__(256, 2) fused_update_next_kernel(UpdateArgs g) {
+  __shared__ double sm[32];
+  extern __shared__ __align__(16) __nv_bfloat16 next_tiles[];  // a_tile[512][kAtPitch], then z_tile[512][kAtPitch]
+  __shared__ int32_t at_row[kNextChannels];                    // row of each channel of the block in "kept first" order
+  __nv_bfloat16* a_tile = next_tiles;
+  __nv_bfloat16* z_tile = next_tiles + kNextChannels * kAtPitch;
+  const int lane = (int)threadIdx.x & 31, warp = (int)threadIdx.x >> 5;
+  const int64_t cb = (int64_t)blockIdx.x * kNextChannels + warp * 64;      // the warp's 64 channels
+  const int64_t c0 = cb + 2 * lane;
+  int64_t rows_per = ceil_div(g.T, (int64_t)g.row_blocks);
+  rows_per = (rows_per + kAtRows - 1) / kAtRows * kAtRows;
+  const int64_t r_begin = (int64_t)blockIdx.y * rows_per;
+  const int64_t r_end = (r_begin + rows_per < g.T) ? r_begin + rows_per : g.T;
+  const float inv_ab = 1.f / (g.alpha + g.beta);
+  float* __restrict__ Zp = g.Z;
+  const float* __restrict__ z1p = g.z1;
+  const float* __restrict__ Dp = g.D;
+  double s_res = 0.0, s_z = 0.0, s_a = 0.0, s_in = 0.0;
+  float cs[2] = {0.f, 0.f};
+  const bool active = c0 < g.n;                                 // n % 4 == 0: a thread's channels exist together
+  const unsigned bits8 = active ? g.grp_mask[c0 >> 3] : 0u;
+  const int sh = (int)(c0 & 7);                                 // 0, 2, 4, 6
+  const unsigned bits = (bits8 >> sh) & 3u;
+  const int base = active ? g.grp_base[c0 >> 3] + __popc(bits8 & ((1u << sh) - 1u)) : 0;
+  const int off1 = (int)(bits & 1u);
+  const int ct = warp * 64 + 2 * lane;                          // first of this thread's channels inside the block
+  {
+    // (only the warp itself reads its entries back: a warp-level barrier is enough)
+    at_row[ct] = (bits & 1u) ? base : (int32_t)(g.k + (c0 - base));
+    at_row[ct + 1] = (bits & 2u) ? base + off1 : (int32_t)(g.k + (c0 + 1 - (base + off1)));
+    __syncwarp();
+  }
+  const bool write_pruned_z = g.zt_pruned_flag == nullptr || *g.zt_pruned_flag != 0;
+  auto load_row = [&](int64_t r, NextRow& w) {
+    const float2 v = __ldcs(reinterpret_cast<const float2*>(Zp + r * g.n + c0));     // read once: streaming
+    w.zo[0] = v.x; w.zo[1] = v.y;
+    const float* zp = z1p + r * g.ldk + base;
+    const float* dp = Dp + r * g.ldk + base;
+    // (plain loads: a warp's run of kept channels starts and ends inside sectors that the neighbouring warps read too)
+    w.z1[0] = (bits & 1u) ? zp[0] : 0.f;
+    w.dc[0] = (bits & 1u) ? dp[0] : 0.f;
+    w.z1[1] = (bits & 2u) ? zp[off1] : 0.f;
+    w.dc[1] = (bits & 2u) ? dp[off1] : 0.f;
+  };
+  auto finish_row = [&](int64_t r, NextRow& w, __nv_bfloat16& a0, __nv_bfloat16& a1, __nv_bfloat16& zb0,
+                        __nv_bfloat16& zb1) {
+    float a[2], zn[2];
+    float p_res = 0.f, p_z = 0.f, p_a = 0.f, p_in = 0.f;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      float u = 0.f;
+      a[q] = update_one(w.zo[q], w.z1[q], w.dc[q], u, false, g.alpha, g.beta, inv_ab, Z_RULE, 0.f, zn[q]);
+      const float din = zn[q] - w.z1[q];
+      p_in = fmaf(din, din, p_in);
+      const float diff = a[q] - fmaxf(zn[q], 0.f);
+      p_res = fmaf(diff, diff, p_res);
+      p_z = fmaf(zn[q], zn[q], p_z);
+      p_a = fmaf(a[q], a[q], p_a);
+      cs[q] += fabsf(a[q]);
+    }
+    a0 = __float2bfloat16_rn(a[0]); a1 = __float2bfloat16_rn(a[1]);
+    zb0 = __float2bfloat16_rn(zn[0]); zb1 = __float2bfloat16_rn(zn[1]);
+    s_res += (double)p_res;
+    s_z += (double)p_z;
+    s_a += (double)p_a;
+    s_in += (double)p_in;
+    __stcs(reinterpret_cast<float2*>(Zp + r * g.n + c0), make_float2(zn[0], zn[1]));
+  };
+  __nv_bfloat16* At = reinterpret_cast<__nv_bfloat16*>(g.At_out);
+  __nv_bfloat16* Zt = reinterpret_cast<__nv_bfloat16*>(g.Zt_out);
+  __nv_bfloat16* Ht = reinterpret_cast<__nv_bfloat16*>(g.Ht_out);
+  const int nch = (g.n - cb < 64) ? (int)((g.n - cb > 0) ? g.n - cb : 0) : 64;
+  for (int64_t rt = r_begin; rt < r_end; rt += kAtRows) {
+    const int64_t rt_end = (rt + kAtRows < r_end) ? rt + kAtRows : r_end;
+    if (active) {
+      int64_t r = rt;
+      for (; r + 7 < rt_end; r += 8) {
+        NextRow w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) load_row(r + i, w[i]);
+        __align__(16) __nv_bfloat16 ca[2][8], cz[2][8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) finish_row(r + i, w[i], ca[0][i], ca[1][i], cz[0][i], cz[1][i]);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          // (kAtPitch = 36 elements: a row of the tile starts 8-byte aligned, so two 8-byte stores)
+          const int at = (ct + q) * kAtPitch + (int)(r - rt);
+          uint2* da = reinterpret_cast<uint2*>(&a_tile[at]);
+          uint2* dz = reinterpret_cast<uint2*>(&z_tile[at]);
+          da[0] = *reinterpret_cast<const uint2*>(&ca[q][0]);
+          da[1] = *reinterpret_cast<const uint2*>(&ca[q][4]);
+          dz[0] = *reinterpret_cast<const uint2*>(&cz[q][0]);
+          dz[1] = *reinterpret_cast<const uint2*>(&cz[q][4]);
+        }
+      }
+      for (; r < rt_end; ++r) {
+        NextRow w0;
+        __nv_bfloat16 a0, a1, zb0, zb1;
+        load_row(r, w0);
+        finish_row(r, w0, a0, a1, zb0, zb1);
+        const int at = ct * kAtPitch + (int)(r - rt);
+        a_tile[at] = a0; a_tile[at + kAtPitch] = a1;
+        z_tile[at] = zb0; z_tile[at + kAtPitch] = zb1;
+      }
+    }
+    __syncwarp();
+    // the warp writes its 64 channels out: rows rt .. rt_end - 1 of a channel in pieces of 8 rows (16 bytes), 4 lanes
+    // per channel
+    const int rows_here = (int)(rt_end - rt);
+    for (int e = lane; e < nch * (kAtRows / 8); e += 32) {
+      const int ch = e / (kAtRows / 8), piece = e % (kAtRows / 8);
+      const int at = (warp * 64 + ch) * kAtPitch + piece * 8;
+      const int64_t row = at_row[warp * 64 + ch];
+      const bool kept = row < g.k;
+      const int64_t dst = row * g.ldt + rt + piece * 8;
+      if (piece * 8 + 8 <= rows_here) {
+        const uint2 alo = *reinterpret_cast<const uint2*>(&a_tile[at]), ahi = *reinterpret_cast<const uint2*>(&a_tile[at + 4]);
+        *reinterpret_cast<uint4*>(At + dst) = make_uint4(alo.x, alo.y, ahi.x, ahi.y);
+        if (kept || write_pruned_z) {
+          const uint2 zlo = *reinterpret_cast<const uint2*>(&z_tile[at]), zhi = *reinterpret_cast<const uint2*>(&z_tile[at + 4]);
+          *reinterpret_cast<uint4*>(Zt + dst) = make_uint4(zlo.x, zlo.y, zhi.x, zhi.y);
+          if (kept)
+            *reinterpret_cast<uint4*>(Ht + dst) =
+                make_uint4(relu_bf16x2(zlo.x), relu_bf16x2(zlo.y), relu_bf16x2(zhi.x), relu_bf16x2(zhi.y));
+        }
+      } else {
+        const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
+        for (int q = 0; q < 8; ++q)
+          if (piece * 8 + q < rows_here) {
+            At[dst + q] = a_tile[at + q];
+            if (kept || write_pruned_z) Zt[dst + q] = z_tile[at + q];
+            if (kept) Ht[dst + q] = __hgt(z_tile[at + q], zero) ? z_tile[at + q] : zero;
+          }
+      }
+    }
+    __syncwarp();
+  }
+  if (active && g.absA_part) {
+    g.absA_part[(int64_t)blockIdx.y * g.n + c0] = (double)cs[0];
+    g.absA_part[(int64_t)blockIdx.y * g.n + c0 + 1] = (double)cs[1];
+  }
+  const int64_t bid = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;
+  const double r0 = block_sum<double>(s_res, sm);
+  const double r1 = block_sum<double>(s_z, sm);
+  const double r2 = block_sum<double>(s_a, sm);
+  const double r3 = block_sum<double>(s_in, sm);
+  if (threadIdx.x == 0) {
+    g.partial[bid * 4 + 0] = r0;
+    g.partial[bid * 4 + 1] = r1;
+    g.partial[bid * 4 + 2] = r2;
+    g.partial[bid * 4 + 3] = r3;
+  }
+}
+
+// h of a step whose mask differs from the one the last token pass left h for (bf16 storage, ReLU, no dual variable,
+// n % 4 == 0): Ht[p(c), t] = bf16(max(Z[t, c], 0)) for the kept channels c, p(c) = its rank among them — the transposed
+// layout in which the fused update above leaves it.  A thread owns 4 consecutive channels, a warp stages kAtRows rows
+// of its 128 channels in shared memory and writes the kept ones out as 64-byte pieces.
+__global__ void __launch_bounds__(256, 3) gather_ht_kernel(const float* __restrict__ Z, int64_t T, int64_t n, int64_t k,
+                                                           const int32_t* __restrict__ grp_base,
+                                                           const uint8_t* __restrict__ grp_mask,
+                                                           __nv_bfloat16* __restrict__ Ht, int64_t ldt,
+                                                           int32_t row_blocks, const int32_t* __restrict__ skip) {
+  if (skip != nullptr && *skip != 0) return;
   extern __shared__ __align__(16) __nv_bfloat16 zt_tile[];     // [1024][kAtPitch]
-  __shared__ uint8_t kept_ch[8][128];                          // per warp: its kept channels (0..127), ascending
-  __shared__ int32_t row_of[8][128];                           // per warp: row of each of its channels in Zt
+  __shared__ int32_t row_of[8][128];                           // per warp: row of each of its channels in Ht, -1: pruned
   const int64_t grp4 = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int64_t c0 = grp4 * 4;
   int64_t rows_per = ceil_div(T, (int64_t)row_blocks);
@@ -613,24 +791,13 @@ __global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __rest
   const bool upper = (grp4 & 1) != 0;
   const unsigned bits = upper ? (bits8 >> 4) : (bits8 & 0xFu);
   const int base = active ? grp_base[grp4 >> 1] + (upper ? __popc(bits8 & 0xFu) : 0) : 0;
-  // the warp's kept channels: a contiguous run of compact positions [base_w, base_w + cnt_w)
-  int before = __popc(bits);
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int u = __shfl_up_sync(0xffffffffu, before, o);
-    if (lane >= o) before += u;
-  }
-  const int cnt_w = __shfl_sync(0xffffffffu, before, 31);
-  before -= __popc(bits);
-  const int base_w = __shfl_sync(0xffffffffu, base, 0);
   {
-    int pos = before, kb = base;       // kb: kept channels before channel c0 + q
+    int kb = base;       // kept channels before channel c0 + q
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const bool is_kept = (bits >> q) & 1u;
-      if (is_kept) kept_ch[warp][pos++] = (uint8_t)(4 * lane + q);
-      // row of the channel in "kept first" order (looked up once, not per piece of the write-out loop)
-      row_of[warp][4 * lane + q] = is_kept ? kb : (int32_t)(k + (c0 + q - kb));
+      // (a mask that keeps more channels than k is reported elsewhere; its surplus channels are not written)
+      row_of[warp][4 * lane + q] = (is_kept && kb < k) ? kb : -1;
       kb += is_kept ? 1 : 0;
     }
   }
@@ -653,7 +820,7 @@ __global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __rest
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float z = q == 0 ? v[i].x : q == 1 ? v[i].y : q == 2 ? v[i].z : v[i].w;
-            col[i] = __float2bfloat16_rn(z);
+            col[i] = __float2bfloat16_rn(fmaxf(z, 0.f));
           }
           // (kAtPitch = 36 elements: a row of the tile starts 8-byte aligned, so two 8-byte stores)
           uint2* dst = reinterpret_cast<uint2*>(&zt_tile[(ct + q) * kAtPitch + (int)(r - rt)]);
@@ -664,11 +831,12 @@ __global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __rest
     }
     __syncwarp();
     const int rows_here = (int)(rt_end - rt);
-    // Z^T: rows rt .. rt_end - 1 of every channel of the warp as pieces of 8 rows, in "kept first" row order
     for (int e = lane; e < nch * (kAtRows / 8); e += 32) {
       const int ch = e / (kAtRows / 8), piece = e % (kAtRows / 8);
+      const int row = row_of[warp][ch];
+      if (row < 0) continue;
       const __nv_bfloat16* src = &zt_tile[(wch0 + ch) * kAtPitch + piece * 8];
-      __nv_bfloat16* dst = Zt + (int64_t)row_of[warp][ch] * ldt + rt + piece * 8;
+      __nv_bfloat16* dst = Ht + (int64_t)row * ldt + rt + piece * 8;
       if (piece * 8 + 8 <= rows_here) {
         const uint2 lo = *reinterpret_cast<const uint2*>(src), hi = *reinterpret_cast<const uint2*>(src + 4);
         *reinterpret_cast<uint4*>(dst) = make_uint4(lo.x, lo.y, hi.x, hi.y);
@@ -676,21 +844,6 @@ __global__ void __launch_bounds__(256, 3) gather_next_kernel(const float* __rest
         for (int q = 0; q < 8; ++q)
           if (piece * 8 + q < rows_here) dst[q] = src[q];
       }
-    }
-    // h of the next step: per row the warp's kept channels are one contiguous run of H; consecutive lanes write
-    // consecutive elements (max(bf16(z), 0) = bf16(max(z, 0)): rounding keeps the sign)
-    // (compact positions beyond k exist only if the caller's mask keeps more channels than k_keep says: they are not
-    // written, so that a wrong argument cannot reach past a row of Hn)
-    for (int e = lane; e < cnt_w && base_w + e < k; e += 32) {
-      // the 32 rows of this kept channel: 64 contiguous bytes of the tile (8-byte aligned rows)
-      __align__(8) __nv_bfloat16 zr[kAtRows];
-      const uint2* src = reinterpret_cast<const uint2*>(&zt_tile[(wch0 + kept_ch[warp][e]) * kAtPitch]);
-#pragma unroll
-      for (int i = 0; i < kAtRows / 4; ++i) reinterpret_cast<uint2*>(zr)[i] = src[i];
-      __nv_bfloat16* hcol = Hn + rt * ldh + base_w + e;
-#pragma unroll
-      for (int rr = 0; rr < kAtRows; ++rr)
-        if (rr < rows_here) hcol[(int64_t)rr * ldh] = __hgt(zr[rr], __float2bfloat16_rn(0.f)) ? zr[rr] : __float2bfloat16_rn(0.f);
     }
     __syncwarp();
   }
@@ -1070,8 +1223,38 @@ int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
   return col_blocks * rb;
 }
 
+// grid of the form that also writes the next step's operands: column blocks of 512 channels
+int fused_update_next_grid(int64_t T, int64_t n, int* row_blocks) {
+  const int col_blocks = (int)ceil_div(n, (int64_t)kNextChannels);
+  int rb = (148 * 16 + col_blocks - 1) / col_blocks;
+  if (rb > T) rb = (int)T;
+  if (rb < 1) rb = 1;
+  if (rb > 65535) rb = 65535;
+  *row_blocks = rb;
+  return col_blocks * rb;
+}
+
+static cudaError_t launch_fused_update_next(const UpdateArgs& a, cudaStream_t stream) {
+  if (a.U || a.gate || a.n % 4 != 0 || a.ldt % 8 != 0 || !a.At_out || !a.Zt_out || !a.Ht_out || !a.at_kept_first ||
+      a.out_dtype != SP_BF16)
+    return cudaErrorInvalidValue;
+  dim3 grid((unsigned)ceil_div(a.n, (int64_t)kNextChannels), (unsigned)a.row_blocks);
+  // per row: Z read and written, A^T written; z1 and D read, Z^T and h^T written on the kept channels (the pruned rows
+  // of Z^T, written only after a mask change, are not counted)
+  ProfScope prof(PK_FUSED_UPDATE, 0.0, (double)a.T * ((double)a.n * 10.0 + (double)a.k * 12.0), stream);
+  count_launch();
+  const bool pz = a.z_rule == SP_Z_PAPER;
+  void (*fn)(UpdateArgs) = pz ? &fused_update_next_kernel<SP_Z_PAPER> : &fused_update_next_kernel<SP_Z_EXACT>;
+  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kNextTileBytes);
+  if (e != cudaSuccess) return e;
+  fn<<<grid, 256, kNextTileBytes, stream>>>(a);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   if (a.T * a.n == 0) return cudaSuccess;
+  if (a.Zt_out || a.Ht_out) return launch_fused_update_next(a, stream);
   dim3 grid((unsigned)ceil_div(a.n, 1024), (unsigned)a.row_blocks);
   // algorithmic bytes per row: Z (and U) read and written, A and the storage copy of Z written, z1 and D read on the
   // kept channels
@@ -1095,23 +1278,22 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather_next(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
-                               const uint8_t* grp_mask, void* Zt, int64_t ldt, void* Hn, int64_t ldh,
-                               cudaStream_t stream) {
+cudaError_t launch_gather_ht(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
+                             const uint8_t* grp_mask, void* Ht, int64_t ldt, cudaStream_t stream) {
   if (T * n == 0) return cudaSuccess;
   if (n % 4 != 0 || ldt % 8 != 0) return cudaErrorInvalidValue;
   int row_blocks = 1;
   fused_update_grid(T, n, &row_blocks);
   dim3 grid((unsigned)ceil_div(n, (int64_t)1024), (unsigned)row_blocks);
-  // Z read once; its bf16 copy written transposed, the kept part once more as next step's h
-  ProfScope prof(PK_PREP_H, 0.0, (double)T * ((double)n * 6.0 + (double)k * 2.0), stream);
+  const int32_t* skip = skip_flag();
+  ProfScope prof(skip ? PK_CONDITIONAL : PK_PREP_H, 0.0, skip ? 0.0 : (double)T * ((double)n * 4.0 + (double)k * 2.0),
+                 stream);
   count_launch();
-  cudaError_t e = cudaFuncSetAttribute(gather_next_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(gather_ht_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)kAtTileBytes);
   if (e != cudaSuccess) return e;
-  gather_next_kernel<<<grid, 256, kAtTileBytes, stream>>>(Z, T, n, k, grp_base, grp_mask,
-                                                         reinterpret_cast<__nv_bfloat16*>(Zt), ldt,
-                                                         reinterpret_cast<__nv_bfloat16*>(Hn), ldh, row_blocks);
+  gather_ht_kernel<<<grid, 256, kAtTileBytes, stream>>>(Z, T, n, k, grp_base, grp_mask,
+                                                       reinterpret_cast<__nv_bfloat16*>(Ht), ldt, row_blocks, skip);
   return cudaGetLastError();
 }
 

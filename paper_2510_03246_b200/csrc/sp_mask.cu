@@ -1366,14 +1366,15 @@ __global__ void unpermute_cols_kernel(const float* __restrict__ Rp, const int32_
   }
 }
 
-__global__ void decay_tag_set_kernel(int32_t* tag, int k, float c, int valid, int h_ld) {
+__global__ void decay_tag_set_kernel(int32_t* tag, int k, float c, int valid, int h_ld, int h_chunk) {
   tag[1] = valid ? k : -1;
   tag[2] = __float_as_int(c);
   tag[4] = valid ? h_ld : 0;
+  tag[5] = valid ? h_chunk : 0;
 }
 
-__global__ void h_next_ready_kernel(const int32_t* same, const int32_t* tag, int h_ld, int32_t* ready) {
-  ready[0] = (same[0] != 0 && tag[4] == h_ld && h_ld > 0) ? 1 : 0;
+__global__ void h_next_ready_kernel(const int32_t* same, const int32_t* tag, int h_ld, int h_chunk, int32_t* ready) {
+  ready[0] = (same[0] != 0 && tag[4] == h_ld && tag[5] == h_chunk && h_ld > 0) ? 1 : 0;
   ready[1] = 1 - ready[0];
 }
 
@@ -1412,15 +1413,17 @@ cudaError_t unpermute_cols(const float* Rp, const int32_t* perm, int64_t rows, i
   return cudaGetLastError();
 }
 
-cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, int64_t h_ld, cudaStream_t stream) {
+cudaError_t decay_tag_set(int32_t* tag, int64_t k, float c, bool valid, int64_t h_ld, int64_t h_chunk,
+                          cudaStream_t stream) {
   count_launch();
-  decay_tag_set_kernel<<<1, 1, 0, stream>>>(tag, (int)k, c, valid ? 1 : 0, (int)h_ld);
+  decay_tag_set_kernel<<<1, 1, 0, stream>>>(tag, (int)k, c, valid ? 1 : 0, (int)h_ld, (int)h_chunk);
   return cudaGetLastError();
 }
 
-cudaError_t h_next_ready(const int32_t* same, const int32_t* tag, int64_t h_ld, int32_t* ready, cudaStream_t stream) {
+cudaError_t h_next_ready(const int32_t* same, const int32_t* tag, int64_t h_ld, int64_t h_chunk, int32_t* ready,
+                         cudaStream_t stream) {
   count_launch();
-  h_next_ready_kernel<<<1, 1, 0, stream>>>(same, tag, (int)h_ld, ready);
+  h_next_ready_kernel<<<1, 1, 0, stream>>>(same, tag, (int)h_ld, (int)h_chunk, ready);
   return cudaGetLastError();
 }
 

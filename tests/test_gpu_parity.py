@@ -664,7 +664,8 @@ def test_kept_support_recovery_reuses_the_factor(cfg, overlap):
     mod.check_status()
 
 
-@pytest.mark.parametrize("rule,with_r1", [("paper", False), ("exact", False), ("paper", True), ("exact", True)])
+@pytest.mark.parametrize("rule,with_r1", [("paper", False), ("exact", False), ("paper", True), ("exact", True),
+                                          ("paper", "unused")])
 def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, with_r1):
     """bf16 storage, ReLU, no dual variable: from the second step with an unchanged mask on, a pruned channel's row of A
     is c = beta / (alpha + beta) times its row of the step before (tests/test_oracle_pins.py pins that on the oracle),
@@ -672,13 +673,19 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
     of contracting over the tokens.  Every step is compared with the oracle's full recomputation: steps that scale,
     a step after a planted other mask (which must recompute), a step after alpha and beta changed (the factor is
     the c of the step that wrote the values, not of the current one), and a module without the ordered accumulators.
-    with_r1: the module also holds R1_perm / H_next, so R1[pruned, :] is scaled too, the bf16 copy of the new Z is
-    written transposed by a pass of its own, and the next step takes its h from H_next instead of gathering it."""
-    cfg = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=1300, sparsity=0.63, outlier_frac=0.02)   # k = 287
+    with_r1: the module also holds R1_perm / H_next, so R1[pruned, :] is scaled too, the fused update writes the bf16
+    copy of the new Z and the next step's h transposed, and the next step takes its h from H_next instead of gathering
+    it (token count a multiple of 8, last chunk of 280 tokens).  "unused": the buffers are there but the token count is
+    not a multiple of 8, so the library must leave them alone and still scale G_A and R2."""
+    tokens = 1304 if with_r1 is True else 1300
+    cfg = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=tokens, sparsity=0.63, outlier_frac=0.02)   # k = 287
     k = cfg.k_keep
     assert k % 4 != 0            # the pruned block starts at a column that is not 16-byte aligned
     mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=k if with_r1 else 0)
-    assert (mod.R1_perm is not None) == with_r1
+    assert (mod.R1_perm is not None) == bool(with_r1)
+    if with_r1 == "unused":
+        mod.R1_perm.fill_(7.0)
+        mod.H_next.fill_(7.0)
     mod.sp_ffn_init()
     tol = TOL[X.dtype]
     audit = []
@@ -710,14 +717,16 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
         Gp = torch.tril(mod.G_A_perm)
         assert torch.equal(torch.tril(mod.G_A[perm][:, perm]), Gp)
         assert torch.equal(mod.R2[:, perm], mod.R2_perm)
-        if with_r1:
+        if with_r1 == "unused":
+            assert bool((mod.R1_perm == 7.0).all()) and bool((mod.H_next == 7.0).all())
+        elif with_r1:
             assert torch.equal(mod.R1[perm], mod.R1_perm)
             # what the pass over the new Z left for the next step: max(Z, 0) on the kept channels, compact
             kept = torch.nonzero(mod.mask).flatten()
-            assert torch.equal(mod.H_next[:, :k], torch.clamp(mod.Z[:, kept], min=0).to(torch.bfloat16))
+            assert torch.equal(mod.h_next_rows(k, 512), torch.clamp(mod.Z[:, kept], min=0).to(torch.bfloat16))
         seen.append(same_order)
     assert seen[0] is False and any(seen[1:5]) and (rule != "paper" or seen[5] is False)
-    if with_r1:
+    if with_r1 is True:
         # the a-update of a step whose mask stays really starts from the h in the state (its gather kernels are queued
         # but return at once): a planted change of that h must show in the step's result; after a mask change the
         # gather runs and overwrites the planted value
@@ -733,7 +742,7 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
         ta, tb = twins
         assert ta.read_report()["pruned_scaled"] == 1.0 and torch.equal(ta.mask, tb.mask)
         kept0 = int(torch.nonzero(ta.mask).flatten()[0])
-        tb.H_next[0, 0] += 4.0
+        tb.H_next.view(-1)[0] += 4.0       # (token 0, first kept channel)
         for t in twins:
             t.sp_admm_step(p_gpu)
         torch.cuda.synchronize()
@@ -743,7 +752,7 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
         # other mask -> the gather runs: the planted value is gone and both modules agree again
         for t in twins:
             t.mask.copy_(torch.roll(t.mask, 1))
-        tb.H_next[0, 0] += 4.0
+        tb.H_next.view(-1)[0] += 4.0       # (token 0, first kept channel)
         p_fix = api.AdmmParams(alpha=1.0, beta=1.5, rho=cfg.rho, k_keep=k, z_rule=_RULE[rule], token_chunk=512,
                                compute_objective=False, reselect_mask=False)
         Za, Zb = ta.Z.clone(), tb.Z.clone()
@@ -914,9 +923,10 @@ def test_admm_step_fixed_mask():
 def test_given_mask_with_another_count_is_reported():
     """reselect_mask = 0 with a mask that does not keep k_keep units: the device status word carries SP_ERR_SHAPE and the
     number of units the mask keeps (the host cannot see the mask)."""
-    cfg = SMALL_BF16
+    cfg = synth.scaled(synth.CONFIGS["C2"], d=264, n=776, tokens=1304, sparsity=0.5, outlier_frac=0.02)
     k = cfg.k_keep
     mod, X, W1, W2 = _make_module(cfg, chunk=512, overlap_k=k)
+    mod.H_next.fill_(1.0)                        # (what no step writes stays 1)
     mod.sp_ffn_init()
     mod.sp_admm_step(api.AdmmParams(rho=cfg.rho, k_keep=k, token_chunk=512))
     torch.cuda.synchronize()
