@@ -721,7 +721,7 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
             assert bool((mod.R1_perm == 7.0).all()) and bool((mod.H_next == 7.0).all())
         elif with_r1:
             assert torch.equal(mod.R1[perm], mod.R1_perm)
-            # what the pass over the new Z left for the next step: max(Z, 0) on the kept channels, compact
+            # what the update left for the next step: max(Z_new, 0) on the kept channels (stored transposed per chunk)
             kept = torch.nonzero(mod.mask).flatten()
             assert torch.equal(mod.h_next_rows(k, 512), torch.clamp(mod.Z[:, kept], min=0).to(torch.bfloat16))
         seen.append(same_order)
