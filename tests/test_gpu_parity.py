@@ -775,6 +775,31 @@ def test_pruned_parts_of_the_accumulators_are_scaled_while_the_mask_stays(rule, 
         assert mod2.read_report()["pruned_scaled"] == 0.0
 
 
+@pytest.mark.parametrize("n,sparsity,tokens,chunk", [(300, 0.98, 520, 256), (776, 0.01, 264, 0), (64, 0.5, 72, 32)])
+def test_update_that_leaves_the_next_operands_at_edge_shapes(n, sparsity, tokens, chunk):
+    """The form of the fused update that also writes the transposed bf16 copy of the new Z and the next step's h, at
+    the ends of its ranges: a handful of kept channels, all but a handful, widths that end inside a warp's 64 channels
+    and inside a block's 512, token chunks that end inside a 32-row tile (8 and 24 rows) and a last chunk of 8 tokens.
+    Three steps each (the first gathers h, the others take it from the state), every one against the oracle."""
+    cfg = synth.scaled(synth.CONFIGS["C2"], d=72, n=n, tokens=tokens, sparsity=sparsity, outlier_frac=0.02)
+    k = cfg.k_keep
+    assert 0 < k < n and tokens % 8 == 0
+    mod, X, W1, W2 = _make_module(cfg, chunk=chunk, overlap_k=k)
+    assert mod.H_next is not None
+    mod.sp_ffn_init()
+    audit = []
+    seen = []
+    for _ in range(3):
+        p_gpu = api.AdmmParams(rho=cfg.rho, k_keep=k, token_chunk=chunk, compute_objective=False)
+        p_or = O.AdmmParams(rho=cfg.rho, k_keep=k)
+        _step_and_compare(mod, X, W1.float(), p_gpu, p_or, TOL[X.dtype], audit)
+        seen.append(mod.read_report()["pruned_scaled"])
+        kept = torch.nonzero(mod.mask).flatten()
+        assert torch.equal(mod.h_next_rows(k, chunk), torch.clamp(mod.Z[:, kept], min=0).to(torch.bfloat16))
+        assert torch.equal(mod.R1[mod.decay_tag[8:].long()], mod.R1_perm)
+    assert seen[0] == 0.0
+
+
 def test_captured_step_takes_either_branch_on_replay():
     """One sp_admm_step captured into a CUDA graph by the caller and replayed: the choice between the backward sweep
     with the reused factor and the restricted factorisation is a device flag read by kernels that were all captured, so
