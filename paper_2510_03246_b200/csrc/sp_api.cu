@@ -189,7 +189,11 @@ bool make_assist(SolveAssist& a) {
          cudaEventCreateWithFlags(&a.panel_done, cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&a.rest_done[0], cudaEventDisableTiming) == cudaSuccess &&
          cudaEventCreateWithFlags(&a.rest_done[1], cudaEventDisableTiming) == cudaSuccess &&
-         cudaEventCreateWithFlags(&a.near_done, cudaEventDisableTiming) == cudaSuccess;
+         cudaEventCreateWithFlags(&a.near_done, cudaEventDisableTiming) == cudaSuccess &&
+         cudaStreamCreateWithFlags(&a.far_stream, cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.far_go, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.far_done[0], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&a.far_done[1], cudaEventDisableTiming) == cudaSuccess;
 }
 SideStream* side_stream() {
   static SideStream table[64];
@@ -223,7 +227,8 @@ struct JoinOnExit {
   bool armed = true;
   ~JoinOnExit() {
     if (!armed || !side) return;
-    cudaStream_t all[3] = {side->stream, side->assist_main.stream, side->assist_side.stream};
+    cudaStream_t all[5] = {side->stream, side->assist_main.stream, side->assist_side.stream,
+                           side->assist_main.far_stream, side->assist_side.far_stream};
     for (cudaStream_t q : all) {
       if (cudaEventRecord(side->join, q) == cudaSuccess) cudaStreamWaitEvent(s, side->join, 0);
     }

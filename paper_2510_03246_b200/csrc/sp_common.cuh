@@ -173,6 +173,10 @@ struct SolveAssist {
   cudaStream_t stream;
   cudaEvent_t panel_done, rest_done[2];
   cudaEvent_t near_done;   // factorisation: the first two block columns of a step's trailing update have landed
+  // Optional third stream of a factorisation: the far part of a step's trailing update (everything right of the first
+  // two block columns), so that the next step's panel and near update do not queue behind it.
+  cudaStream_t far_stream = nullptr;
+  cudaEvent_t far_go = nullptr, far_done[2] = {nullptr, nullptr};
 };
 // dinv must have room for ceil(n / 128) + 1 pairs of 128 x 128 blocks (the last pair is scratch).
 // m_extra > 0: A has m_extra more rows below row n (same lda), the right-hand sides B of a system X L^T = B; they

@@ -666,6 +666,15 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
   float* S = dinv + nblk * 2 * TB * TB;      // [128, 128] next diagonal block
   float* LmT = S + TB * TB;                  // [128, 128] scratch of the lookahead kernel
   bool rec[2] = {false, false};
+  // Far part of a step's trailing update on a stream of its own: it adds into the matrix through the GEMM's atomic TMA
+  // reduction (which needs 16-byte aligned rows and a width that is a multiple of 4), so it commutes with the near
+  // update of the next step, which touches one of its block columns.  What must see it complete waits for its event:
+  // the lookahead kernel of step kb reads block (kb+1, kb+1), last touched by the far update of step kb - 2.
+  // The far GEMM leaves a few SM pairs to the kernels of the chain, which would otherwise wait for its tiles to end.
+  const bool far_apart = assist && assist->far_stream && n % 4 == 0 && lda % 4 == 0 &&
+                         (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && !reproducible_mode();
+  bool far_rec[2] = {false, false};
+  constexpr int kFarPairs = 64;
   // Two-level blocking for large systems: the trailing update of a step is bound by the read-modify-write of the fp32
   // matrix when K is only 128 (n = 28672: 430 GB per factorisation).  With OB > 1 the steps of an outer block of OB
   // diagonal blocks update only the rest of that outer block's columns at once; everything to the right of it gets
@@ -701,12 +710,17 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     if (prow <= 0) break;
     cudaStream_t sb = stream;
     // last block with appended rows: their panel runs on `stream`, behind the assisting stream's last update
-    if (assist && rem <= 0 && kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
+    if (assist && rem <= 0 && kb >= 1) {
+      SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[(kb - 1) & 1], 0));
+      for (int q = 0; q < 2; ++q)
+        if (far_rec[q]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->far_done[q], 0));
+    }
     if (assist && rem > 0) {
       if (!inner_last) {
         // next diagonal block: it reads blocks (kb+1, kb) and (kb+1, kb+1), i.e. the first two block columns of the
         // trailing update of step kb - 1, which that step issues first and signals on their own
         if (kb >= 1) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->near_done, 0));
+        if (far_rec[kb & 1]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->far_done[kb & 1], 0));   // far update of step kb - 2
         const int nb2 = (int)(rem < TB ? rem : TB);
         count_launch();
         ProfScope prof(PK_PANEL_APPLY, 4.0 * TB * TB * TB, 0.0, stream);
@@ -733,6 +747,7 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
                                   status_dev, sb) != cudaSuccess)
       return SP_ERR_CUDA;
     if (rem <= 0) break;     // last block: the appended rows are done, nothing is left to update
+    if (far_apart && !outer && rem > 2 * TB) SP_CUDA_OK(cudaEventRecord(assist->far_go, sb));   // the panel's parts exist
     // A22 -= L21 L21^T on the lower triangle
     TcOperand ta{P + (k0 + nb) * ldp, ldp, true}, tb{P + (k0 + nb) * ldp, ldp, true};
     ta.kext = tb.kext = ldp;
@@ -805,10 +820,19 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
       fb.mnext = rem - kNear;
       float* Afar = A22 + kNear * lda + kNear;
       const double fr = (double)(rem - kNear);
+      cudaStream_t sf = sb;
+      if (far_apart) {
+        sf = assist->far_stream;
+        SP_CUDA_OK(cudaStreamWaitEvent(sf, assist->far_go, 0));
+      }
       st = gemm_tc(prow - kNear, rem - kNear, TB, -1.f, fa, fb, 1.f, Operand{Afar, SP_F32, lda, 1},
-                   OutOperand{Afar, SP_F32, lda}, true, status_dev, sb, &sg,
-                   (fr * fr + 2.0 * (double)m_extra * fr) * (double)nb);
+                   OutOperand{Afar, SP_F32, lda}, true, status_dev, sf, &sg,
+                   (fr * fr + 2.0 * (double)m_extra * fr) * (double)nb, far_apart ? kFarPairs : 0);
       if (st != SP_OK) return st;
+      if (far_apart) {
+        SP_CUDA_OK(cudaEventRecord(assist->far_done[kb & 1], sf));
+        far_rec[kb & 1] = true;
+      }
     } else {
       sp_status st = gemm_tc(prow, rem, TB, -1.f, ta, tb, 1.f, Operand{A22, SP_F32, lda, 1},
                              OutOperand{A22, SP_F32, lda}, true, status_dev, sb, &sg,
@@ -822,8 +846,10 @@ sp_status potrf_lower_tc(float* A, int64_t n, int64_t lda, float* dinv, void* Pv
     }
   }
   // the factor is complete on `stream` once the assisting stream has drained
-  for (int q = 0; q < 2; ++q)
+  for (int q = 0; q < 2; ++q) {
     if (assist && rec[q]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->rest_done[q], 0));
+    if (far_rec[q]) SP_CUDA_OK(cudaStreamWaitEvent(stream, assist->far_done[q], 0));
+  }
 #undef SP_CUDA_OK
   return SP_OK;
 }
