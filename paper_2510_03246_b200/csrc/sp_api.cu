@@ -311,7 +311,8 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
     int rb2 = 1;       // the form of the update that also writes the next step's operands has its own grid
     const int nb2 = fused_update_next_grid(p.chunk, n, &rb2);
     if (nb2 > p.nblocks) p.nblocks = nb2;
-    if (rb2 > p.row_blocks) p.row_blocks = rb2;
+    const int pr2 = fused_update_next_partial_rows(rb2);     // (that form leaves several rows of |A| partials per row block)
+    if (pr2 > p.row_blocks) p.row_blocks = pr2;
   }
   p.partial = c.take<double>((size_t)p.nblocks * 4 + kSumsqBlocks);
   p.Eo = c.take<float>((size_t)p.chunk * d);
@@ -1141,7 +1142,8 @@ static sp_status admm_step_impl(const sp_ffn_module* m, sp_ffn_state* st, const 
       SPCHK(contract(Tc, d, n, -1.0, ac, true, w2f, true, 1.0, yc, eo, false, acc64, bf16, status_dev, s));
       CU(sumsq_accumulate(p.Eo, d, Tc, d, prm->alpha, &rep_dev->res_out, ci > 0, p.partial + (size_t)p.nblocks * 4, s));
     }
-    CU(reduce_col_partials(p.absA_part, ua.row_blocks, n, st->absA, ci > 0, s));
+    CU(reduce_col_partials(p.absA_part, decay_z ? fused_update_next_partial_rows(ua.row_blocks) : ua.row_blocks, n,
+                           st->absA, ci > 0, s));
     // accumulators of the new auxiliary variables
     if (decay) {
       // rows of A^T in "kept first" order: [0, k) kept, [k, n) pruned

@@ -299,6 +299,7 @@ cudaError_t launch_fused_update(const UpdateArgs& a, cudaStream_t stream);
 cudaError_t launch_gather_ht(const float* Z, int64_t T, int64_t n, int64_t k, const int32_t* grp_base,
                              const uint8_t* grp_mask, void* Ht, int64_t ldt, cudaStream_t stream);
 int fused_update_next_grid(int64_t T, int64_t n, int* row_blocks);
+int fused_update_next_partial_rows(int row_blocks);   // rows of absA_part that this form of the update writes
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]
 cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,
