@@ -308,9 +308,11 @@ AdmmPlan plan_admm(void* ws, int64_t d, int64_t n, int64_t N, int64_t chunk, int
   p.z1 = c.take<float>((size_t)p.chunk * npad);
   p.nblocks = fused_update_grid(p.chunk, n, &p.row_blocks);
   {
-    int rb2 = 1;       // the form of the update that also writes the next step's operands has its own grid
-    const int nb2 = fused_update_next_grid(p.chunk, n, &rb2);
-    if (nb2 > p.nblocks) p.nblocks = nb2;
+    // the form of the update that also writes the next step's operands has its own grid, whose row blocks depend on
+    // the chunk's token count: sized for its upper bound
+    const int rb2 = fused_update_next_row_cap(n);
+    const int64_t nb2 = fused_update_next_max_blocks(n);
+    if (nb2 > p.nblocks) p.nblocks = (int)nb2;
     const int pr2 = fused_update_next_partial_rows(rb2);     // (that form leaves several rows of |A| partials per row block)
     if (pr2 > p.row_blocks) p.row_blocks = pr2;
   }

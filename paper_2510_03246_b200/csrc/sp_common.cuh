@@ -300,6 +300,8 @@ cudaError_t launch_gather_ht(const float* Z, int64_t T, int64_t n, int64_t k, co
                              const uint8_t* grp_mask, void* Ht, int64_t ldt, cudaStream_t stream);
 int fused_update_next_grid(int64_t T, int64_t n, int* row_blocks);
 int fused_update_next_partial_rows(int row_blocks);   // rows of absA_part that this form of the update writes
+int fused_update_next_row_cap(int64_t n);              // upper bound of the row blocks fused_update_next_grid returns
+int64_t fused_update_next_max_blocks(int64_t n);       // ... and of its blocks
 int fused_update_grid(int64_t T, int64_t n, int* row_blocks);
 // out[j] (+)= sum_r part[r, j]
 cudaError_t reduce_col_partials(const double* part, int32_t row_blocks, int64_t n, double* out, bool accumulate,

@@ -1,6 +1,8 @@
 // Elementwise and reduction kernels of the ADMM step: the fused auxiliary-variable update (a-update epilogue,
 // z^(2), select, dual update, residual and |A| statistics in one pass over the chunk), operand preparation,
 // conversions, gathers and small reductions.  All reductions use a fixed order (no floating-point atomics).
+#include <algorithm>
+
 #include "sp_common.cuh"
 
 namespace sp {
@@ -1229,16 +1231,31 @@ int fused_update_grid(int64_t T, int64_t n, int* row_blocks) {
   return col_blocks * rb;
 }
 
-// grid of the form that also writes the next step's operands: column blocks of 512 channels
+// Grid of the form that also writes the next step's operands: column blocks of kNextChannels channels, row blocks of
+// a multiple of kNextTiles * kAtRows rows.  The rows per block are chosen so that the blocks fill whole waves of the
+// 2 x 148 resident blocks as nearly as possible (at n = 28672 the plain rule "16 blocks per SM" left the last of 8.3
+// waves 30 % full); the number of row blocks never exceeds fused_update_next_row_cap(n), which sizes the partial sums.
 int fused_update_next_partial_rows(int row_blocks) { return kNextTiles * row_blocks; }
+int fused_update_next_row_cap(int64_t n) {
+  const int64_t col_blocks = ceil_div(n, (int64_t)kNextChannels);
+  return (int)std::min<int64_t>(65535, ceil_div((int64_t)148 * 32, col_blocks) + 1);
+}
+int64_t fused_update_next_max_blocks(int64_t n) {
+  return ceil_div(n, (int64_t)kNextChannels) * fused_update_next_row_cap(n);
+}
 int fused_update_next_grid(int64_t T, int64_t n, int* row_blocks) {
-  const int col_blocks = (int)ceil_div(n, (int64_t)kNextChannels);
-  int rb = (148 * 16 + col_blocks - 1) / col_blocks;
-  if (rb > T) rb = (int)T;
-  if (rb < 1) rb = 1;
-  if (rb > 65535) rb = 65535;
-  *row_blocks = rb;
-  return col_blocks * rb;
+  const int64_t col_blocks = ceil_div(n, (int64_t)kNextChannels);
+  const int64_t unit = (int64_t)kNextTiles * kAtRows, slots = 2 * 148, cap = fused_update_next_row_cap(n);
+  int64_t best_rb = 1, best_span = -1;
+  for (int64_t r = unit * ceil_div(T, unit); r >= unit; r -= unit) {
+    const int64_t rb = ceil_div(T, r);
+    if (rb > cap) break;
+    const int64_t span = ceil_div(col_blocks * rb, slots) * r;     // waves x rows per block
+    if (best_span < 0 || span < best_span) { best_span = span; best_rb = rb; }
+    if (r > 64 * unit) r -= (r / (64 * unit) - 1) * unit;          // (coarser steps among very tall blocks)
+  }
+  *row_blocks = (int)best_rb;
+  return (int)(col_blocks * best_rb);
 }
 
 static cudaError_t launch_fused_update_next(const UpdateArgs& a, cudaStream_t stream) {
